@@ -1,0 +1,190 @@
+"""ctypes loader for the plain-C fp64 oracle (``gsi_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: nothing in the product path may import this module.
+It marshals numpy arrays into the C functions and holds no arithmetic of the
+method itself; each C function cites the passage of the paper it follows
+(Algorithm 1, Eq. (3.1)-(3.3), Section 4.2).
+
+Array conventions: bf16 data travel as ``numpy.uint16`` bit patterns; the basis
+P is ``[d][k]`` (uint16 bf16 bits or float32), weights W are ``[o][d]`` uint16,
+activations x are ``[T][d]`` float32.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "gsi_oracle.c")
+_LIB = os.path.join(_HERE, "libgsi_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+BF16 = 0
+F32 = 1
+
+
+def build(force: bool = False) -> str:
+    """Compile ``gsi_oracle.c`` with gcc (OpenMP over output rows / tokens)."""
+    with _lock:
+        stale = (not os.path.exists(_LIB)) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC)
+        if force or stale:
+            tmp = _LIB + f".tmp{os.getpid()}"
+            subprocess.check_call(
+                ["gcc", "-O2", "-fopenmp", "-shared", "-fPIC", "-Wall", "-o", tmp, _SRC, "-lm"]
+            )
+            os.replace(tmp, _LIB)
+    return _LIB
+
+
+def _load():
+    global _lib
+    if _lib is None:
+        lib = ctypes.CDLL(build())
+        vp, i, f, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_float, ctypes.c_size_t
+        lib.gsi_oracle_num_threads.restype = i
+        lib.gsi_oracle_set_threads.argtypes = [i]
+        lib.gsi_oracle_bf16_to_f64.argtypes = [vp, sz, vp]
+        lib.gsi_oracle_f64_to_bf16_rne_array.argtypes = [vp, sz, vp]
+        lib.gsi_oracle_image.argtypes = [vp, vp, i, i, i, i, vp]
+        lib.gsi_oracle_image.restype = i
+        lib.gsi_oracle_project.argtypes = [vp, i, vp, i, i, i, f, vp, vp, vp, vp, vp, vp]
+        lib.gsi_oracle_project.restype = i
+        lib.gsi_oracle_map.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, vp]
+        lib.gsi_oracle_map.restype = i
+        _lib = lib
+    return _lib
+
+
+def _ptr(a):
+    return None if a is None else a.ctypes.data_as(ctypes.c_void_p)
+
+
+def _c(a, dtype):
+    a = np.ascontiguousarray(a)
+    if a.dtype != dtype:
+        raise TypeError(f"expected {dtype}, got {a.dtype}")
+    return a
+
+
+def _basis(P):
+    P = np.ascontiguousarray(P)
+    if P.dtype == np.uint16:
+        return P, BF16
+    if P.dtype == np.float32:
+        return P, F32
+    raise TypeError("basis must be uint16 (bf16 bits) or float32")
+
+
+def num_threads() -> int:
+    return int(_load().gsi_oracle_num_threads())
+
+
+def set_threads(n: int) -> None:
+    _load().gsi_oracle_set_threads(int(n))
+
+
+def bf16_to_f64(bits) -> np.ndarray:
+    bits = _c(bits, np.uint16)
+    out = np.empty(bits.shape, np.float64)
+    _load().gsi_oracle_bf16_to_f64(_ptr(bits), bits.size, _ptr(out))
+    return out
+
+
+def f64_to_bf16_rne(v) -> np.ndarray:
+    v = _c(v, np.float64)
+    out = np.empty(v.shape, np.uint16)
+    _load().gsi_oracle_f64_to_bf16_rne_array(_ptr(v), v.size, _ptr(out))
+    return out
+
+
+def image(W, P) -> np.ndarray:
+    """M = W V_k in fp64, unrounded (Eq. (3.2), Section 4.2)."""
+    W = _c(W, np.uint16)
+    P, pd = _basis(P)
+    o, d = W.shape
+    d2, k = P.shape
+    assert d == d2
+    M = np.empty((o, k), np.float64)
+    rc = _load().gsi_oracle_image(_ptr(W), _ptr(P), pd, o, d, k, _ptr(M))
+    if rc:
+        raise RuntimeError("gsi_oracle_image failed")
+    return M
+
+
+def project(x, P, eps: float) -> dict:
+    """Algorithm 1 lines 1-4: g, r, rho and the gate byte (1 = slow path)."""
+    x = _c(x, np.float32)
+    P, pd = _basis(P)
+    T, d = x.shape
+    d2, k = P.shape
+    assert d == d2
+    out = dict(
+        g=np.empty((T, k), np.float64),
+        r=np.empty((T, d), np.float64),
+        rho=np.empty(T, np.float64),
+        norm_x=np.empty(T, np.float64),
+        norm_r=np.empty(T, np.float64),
+        gate=np.empty(T, np.uint8),
+    )
+    rc = _load().gsi_oracle_project(
+        _ptr(x), T, _ptr(P), pd, d, k, float(np.float32(eps)),
+        _ptr(out["g"]), _ptr(out["r"]), _ptr(out["rho"]),
+        _ptr(out["norm_x"]), _ptr(out["norm_r"]), _ptr(out["gate"]),
+    )
+    if rc:
+        raise RuntimeError("gsi_oracle_project failed")
+    return out
+
+
+def apply_map(M, W, g, r, gate, x=None, want_alt: bool = False):
+    """y = M g (+ W r on gated tokens); optionally Algorithm 1 read literally."""
+    M = _c(M, np.float64)
+    W = _c(W, np.uint16)
+    g = _c(g, np.float64)
+    r = _c(r, np.float64)
+    gate = _c(gate, np.uint8)
+    o, d = W.shape
+    T, k = g.shape
+    assert M.shape == (o, k) and r.shape == (T, d) and gate.shape == (T,)
+    y = np.empty((T, o), np.float64)
+    y_alt = None
+    if want_alt:
+        x = _c(x, np.float32)
+        assert x.shape == (T, d)
+        y_alt = np.empty((T, o), np.float64)
+    rc = _load().gsi_oracle_map(
+        _ptr(M), _ptr(W), _ptr(g), _ptr(r), _ptr(x) if want_alt else None,
+        _ptr(gate), T, o, d, k, _ptr(y), _ptr(y_alt),
+    )
+    if rc:
+        raise RuntimeError("gsi_oracle_map failed")
+    return (y, y_alt) if want_alt else y
+
+
+def forward(x, P, eps: float, Ws, gate_override=None, rows=None) -> dict:
+    """The whole layer for one input group: the maps in ``Ws`` share x, P, g, r
+    and one gate decision per token.
+
+    ``rows`` (one index array per map, or None) restricts each map to a sample
+    of its output rows; the projection and the gate always use the full basis.
+    ``gate_override`` substitutes given gate bytes when forming y (used for
+    tokens whose rho sits on the threshold); the oracle's own decision is still
+    returned as ``gate``.
+    """
+    pr = project(x, P, eps)
+    gate_used = pr["gate"] if gate_override is None else _c(gate_override, np.uint8)
+    ys = []
+    for j, W in enumerate(Ws):
+        W = _c(W, np.uint16)
+        if rows is not None and rows[j] is not None:
+            W = np.ascontiguousarray(W[np.asarray(rows[j])])
+        M = image(W, P)
+        ys.append(apply_map(M, W, pr["g"], pr["r"], gate_used))
+    pr["y"] = ys
+    pr["gate_used"] = gate_used
+    return pr
