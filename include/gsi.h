@@ -1,0 +1,216 @@
+/*
+ * gsi.h - C ABI of the B200 (sm_100a) gated subspace linear layer.
+ *
+ * The library implements the per-token procedure of Algorithm 1 ("Gated
+ * Subspace Inference") for batch-1 and small-batch decode.  For one input
+ * activation x (fp32, length d), a stored basis P (d x k; the paper's V_k) and
+ * one or more weight matrices W_j (d_out_j x d, bf16) that share this input:
+ *
+ *   c   = P^T x                          Algorithm 1 line 1 (paper: g = V_k^T x)
+ *   r   = x - P c                        line 2, Eq. (3.1); explicit residual
+ *   rho = ||r||_2 / ||x||_2              line 3, Eq. (3.3)
+ *   y_j = W_P,j c                        line 5; W_P,j = W_j P is the cached
+ *                                        image M of Eq. (3.2) / Section 4.2
+ *   if !(||r|| < eps ||x||):  y_j += W_j r      Eq. (3.2): y = M g + W r = W x
+ *
+ * The gate test is the strict comparison of Section 3.2 (fast path iff
+ * rho < eps) taken in the division-free form ||r|| < eps*||x||, so x = 0 and
+ * non-finite inputs take the slow path.  A token whose gate byte is 1 is
+ * "gated" / "fired": the full correction W r was added for it.
+ *
+ * A "group" is the set of maps sharing one input x (hence one P, c, r and one
+ * gate decision per token), e.g. {q, k, v, fc} of a GPT-J block.
+ *
+ * Conventions
+ *   - All pointers are DEVICE pointers unless the name ends in _host.
+ *   - Matrices are dense row-major: W [d_out][d], P [d][k], W_P [sum d_out][k].
+ *   - bf16 = upper half of IEEE fp32, stored as 16-bit words.
+ *   - x is [n_tokens][d] fp32.  y is ONE buffer [n_tokens][sum_j d_out_j] fp32:
+ *     token t, map j occupies columns [off_j, off_j + d_out_j), off_j the
+ *     running sum of d_out.  y is overwritten, never accumulated into.
+ *   - Pointers must be 16-byte aligned; d, k and every d_out multiples of 8;
+ *     8 <= k <= min(d, 1024).  Otherwise GSI_ERR_UNSUPPORTED / INVALID_ARG.
+ *   - Every function returns gsi_status_t; no exception crosses the boundary.
+ *     Argument errors are found on the host before anything is launched.
+ *   - Ownership: the caller owns W, P, x, y, the logs and the workspace.  The
+ *     library borrows W and P (they must outlive the handle) and owns what it
+ *     places in the workspace.  Nothing below allocates device memory; the
+ *     forward calls do not synchronise the host and may be stream-captured
+ *     (the *_host variants copy and synchronise, and may not).
+ *   - One handle / stack may be used by one stream at a time.
+ */
+#ifndef GSI_H_
+#define GSI_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  GSI_OK = 0,
+  GSI_ERR_INVALID_ARG = 1, /* null pointer, non-positive size, misaligned pointer */
+  GSI_ERR_UNSUPPORTED = 2, /* shape outside the supported set                       */
+  GSI_ERR_ALLOC = 3,       /* host allocation failed                                */
+  GSI_ERR_CUDA = 4,        /* a CUDA runtime call failed                            */
+  GSI_ERR_TIMEOUT = 5,     /* a bounded device-side wait gave up (status word)      */
+  GSI_ERR_WORKSPACE = 6    /* workspace smaller than gsi_workspace_bytes()          */
+} gsi_status_t;
+
+typedef enum { GSI_BF16 = 0, GSI_F32 = 1 } gsi_dtype_t;
+
+/* A CUDA stream (cudaStream_t), spelt without the CUDA headers. */
+typedef struct CUstream_st* gsi_stream_t;
+
+typedef struct gsi_layer* gsi_handle_t; /* one group */
+typedef struct gsi_stack* gsi_stack_t;  /* an ordered chain of groups */
+
+enum {
+  GSI_FLAG_NONE = 0u,
+  /* Static projection (Remark after Theorem 3.1, "Mode C"): never add W r.
+     Gate bytes and rho are still reported. */
+  GSI_FLAG_STATIC_PROJECTION = 1u,
+  /* Dense baseline: y = W x by the streaming GEMV, no projection, no image.
+     Gate bytes are written as 1.  Used to measure the speed-up honestly. */
+  GSI_FLAG_DENSE = 2u
+};
+
+typedef struct {
+  int d;               /* input width                                           */
+  int k;               /* basis rank                                            */
+  int n_maps;          /* maps sharing this input, 1..GSI_MAX_MAPS              */
+  const int* d_out;    /* HOST array [n_maps]                                   */
+  float eps;           /* gate threshold: fast path iff ||r|| < eps*||x||       */
+  int max_tokens;      /* largest batch a forward call may carry, 1..GSI_MAX_TOKENS */
+  gsi_dtype_t p_dtype; /* storage type of P                                     */
+  unsigned flags;      /* GSI_FLAG_*                                            */
+} gsi_desc_t;
+
+#define GSI_MAX_MAPS 8
+#define GSI_MAX_TOKENS 64
+
+const char* gsi_status_string(gsi_status_t s);
+
+/*
+ * Cached image of Eq. (3.2) / Section 4.2 ("computed once per weight matrix"):
+ *   W_P[a][j] = bf16_rne( sum_i W[a][i] * P[i][j] ),  fp32 accumulation.
+ * W [o][d] bf16, P [d][k] of p_dtype, W_P_out [o][k] bf16; all device.
+ * Enqueued on `stream`; no host synchronisation.
+ */
+gsi_status_t gsi_build_image(const void* W, const void* P, int o, int d, int k,
+                             gsi_dtype_t p_dtype, void* W_P_out, gsi_stream_t stream);
+
+/* Bytes of device workspace a handle for `desc` needs (0 if desc is invalid).
+ * The workspace holds the images of all maps and the per-call scratch (c, r,
+ * partial sums, fired-token list, status word). */
+size_t gsi_workspace_bytes(const gsi_desc_t* desc);
+
+/*
+ * Create a handle for one group.  W_host_array is a HOST array of n_maps DEVICE
+ * pointers, W_j [d_out_j][d] bf16.  P is [d][k].  `workspace` is device memory
+ * of at least gsi_workspace_bytes(desc), 256-byte aligned, owned by the caller
+ * and used exclusively by this handle until gsi_destroy.  The images W_P,j are
+ * built on `stream` inside this call (Section 4.2); W is not needed for that
+ * again, but is read by every gated token afterwards.
+ */
+gsi_status_t gsi_create(const gsi_desc_t* desc, const void* const* W_host_array,
+                        const void* P, void* workspace, size_t workspace_bytes,
+                        gsi_stream_t stream, gsi_handle_t* out);
+
+/*
+ * Algorithm 1 for desc.max_tokens tokens (gsi_forward) or n_tokens <=
+ * max_tokens tokens (gsi_forward_n).  x [n][d] fp32; y [n][sum d_out] fp32;
+ * gate_mask_out [n] bytes (1 = slow path, W r added); rho_out [n] fp32 or NULL.
+ * Each token's gate byte and output do not depend on the other tokens of the
+ * call.  Enqueues on `stream` and returns; n_tokens = 0 is a no-op.
+ */
+gsi_status_t gsi_forward(gsi_handle_t h, const float* x, float* y,
+                         unsigned char* gate_mask_out, gsi_stream_t stream);
+gsi_status_t gsi_forward_n(gsi_handle_t h, const float* x, int n_tokens, float* y,
+                           unsigned char* gate_mask_out, float* rho_out,
+                           gsi_stream_t stream);
+
+/*
+ * Same as gsi_forward_n with HOST buffers: copies x to the device, runs the
+ * layer, copies y / gate / rho back and synchronises `stream`.  Staging space
+ * for x, y, gate and rho is part of the handle's workspace.
+ */
+gsi_status_t gsi_forward_host(gsi_handle_t h, const float* x_host, int n_tokens,
+                              float* y_host, unsigned char* gate_mask_host,
+                              float* rho_host, gsi_stream_t stream);
+
+/* Device pointer to the image of map j inside the workspace ([d_out_j][k] bf16),
+ * so a caller can inspect or persist it. */
+gsi_status_t gsi_get_image(gsi_handle_t h, int map, const void** W_P_out);
+
+/* Synchronises the handle's last stream and returns the device status word:
+ * 0, or a GSI_ERR_* code recorded by a kernel (e.g. a bounded wait that gave
+ * up).  Kernels never trap. */
+gsi_status_t gsi_get_status(gsi_handle_t h, int* device_status);
+
+gsi_status_t gsi_destroy(gsi_handle_t h);
+
+/* ------------------------------------------------------------------------ *
+ * Stack driver: one decode step = every group of every layer, in order, on
+ * one stream (Section 1: the method is applied to all linear maps of all
+ * layers).  Groups keep their own handles; the stack only chains them.
+ * ------------------------------------------------------------------------ */
+
+typedef struct {
+  const float* x; /* [n_steps][max_tokens][d]: input of this group at every step */
+  float* y;       /* [max_tokens][sum d_out]: overwritten at every step          */
+} gsi_stack_io_t;
+
+/* Bytes of extra device workspace the stack itself needs (step counter,
+ * barrier words, per-group parameter table). */
+size_t gsi_stack_workspace_bytes(int n_groups);
+
+/* groups_host_array: HOST array of n_groups handles in execution order; all
+ * must have the same max_tokens.  The handles must outlive the stack. */
+gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups_host_array,
+                              void* workspace, size_t workspace_bytes,
+                              gsi_stream_t stream, gsi_stack_t* out);
+
+/*
+ * Bind the I/O of every group.  io_host_array: HOST array [n_groups].  The
+ * stack keeps a DEVICE-side step counter s; step number s reads
+ * x + (s mod n_steps)*max_tokens*d of each group and writes
+ *   gate_log[(s mod n_steps)][group][token]   (bytes, may not be NULL)
+ *   rho_log [(s mod n_steps)][group][token]   (fp32, may be NULL)
+ * so that replaying one captured CUDA graph walks through the pre-staged
+ * inputs without host involvement.
+ */
+gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io_host_array,
+                            int n_steps, unsigned char* gate_log, float* rho_log,
+                            gsi_stream_t stream);
+
+/* Set the device-side step counter (enqueued on `stream`). */
+gsi_status_t gsi_stack_seek(gsi_stack_t s, int step, gsi_stream_t stream);
+
+/* Enqueue one decode step and advance the device-side counter.  No host
+ * synchronisation; may be stream-captured into a CUDA graph and replayed. */
+gsi_status_t gsi_stack_step(gsi_stack_t s, gsi_stream_t stream);
+
+/* Number of kernels one gsi_stack_step enqueues (for launch accounting). */
+gsi_status_t gsi_stack_launches_per_step(gsi_stack_t s, int* n_out);
+
+/*
+ * One decode step with HOST buffers: x_host_array[g] -> device slot of the
+ * current step, run the step, copy every group's y and the step's gate bytes
+ * back, synchronise.  x_host_array / y_host_array: HOST arrays [n_groups] of
+ * HOST pointers ([max_tokens][d] and [max_tokens][sum d_out]); pinned memory
+ * makes the copies asynchronous.  gate_host [n_groups][max_tokens].
+ */
+gsi_status_t gsi_stack_step_host(gsi_stack_t s, const float* const* x_host_array,
+                                 float* const* y_host_array, unsigned char* gate_host,
+                                 gsi_stream_t stream);
+
+gsi_status_t gsi_stack_get_status(gsi_stack_t s, int* device_status);
+gsi_status_t gsi_stack_destroy(gsi_stack_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* GSI_H_ */

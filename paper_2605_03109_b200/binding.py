@@ -1,0 +1,288 @@
+"""ctypes binding of ``include/gsi.h`` (same names, argument marshalling only).
+
+``Layer`` and ``Stack`` wrap a handle together with the torch tensors that back
+its workspace; they add no computation.  If the CUDA library cannot be loaded
+the import fails loudly: there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+
+import torch
+
+from . import build as _build
+
+GSI_BF16, GSI_F32 = 0, 1
+GSI_FLAG_NONE, GSI_FLAG_STATIC_PROJECTION, GSI_FLAG_DENSE = 0, 1, 2
+GSI_MAX_MAPS, GSI_MAX_TOKENS = 8, 64
+
+EXPORTED = [
+    "gsi_status_string", "gsi_build_image", "gsi_workspace_bytes", "gsi_create",
+    "gsi_forward", "gsi_forward_n", "gsi_forward_host", "gsi_get_image", "gsi_get_status",
+    "gsi_destroy", "gsi_stack_workspace_bytes", "gsi_stack_create", "gsi_stack_bind",
+    "gsi_stack_seek", "gsi_stack_step", "gsi_stack_launches_per_step",
+    "gsi_stack_step_host", "gsi_stack_get_status", "gsi_stack_destroy",
+]
+
+
+class GsiDesc(C.Structure):
+    _fields_ = [("d", C.c_int), ("k", C.c_int), ("n_maps", C.c_int),
+                ("d_out", C.POINTER(C.c_int)), ("eps", C.c_float), ("max_tokens", C.c_int),
+                ("p_dtype", C.c_int), ("flags", C.c_uint)]
+
+
+class GsiStackIo(C.Structure):
+    _fields_ = [("x", C.c_void_p), ("y", C.c_void_p)]
+
+
+class GsiError(RuntimeError):
+    def __init__(self, code, where):
+        self.code = int(code)
+        super().__init__(f"{where}: {gsi_status_string(code)} ({int(code)})")
+
+
+def lib_path() -> str:
+    return _build.LIB
+
+
+def _load():
+    path = _build.LIB
+    if not os.path.exists(path):
+        path = _build.build()
+    l = C.CDLL(path)
+    vp, i, sz = C.c_void_p, C.c_int, C.c_size_t
+    l.gsi_status_string.restype = C.c_char_p
+    l.gsi_status_string.argtypes = [i]
+    l.gsi_build_image.argtypes = [vp, vp, i, i, i, i, vp, vp]
+    l.gsi_workspace_bytes.restype = sz
+    l.gsi_workspace_bytes.argtypes = [C.POINTER(GsiDesc)]
+    l.gsi_create.argtypes = [C.POINTER(GsiDesc), C.POINTER(vp), vp, vp, sz, vp, C.POINTER(vp)]
+    l.gsi_forward.argtypes = [vp, vp, vp, vp, vp]
+    l.gsi_forward_n.argtypes = [vp, vp, i, vp, vp, vp, vp]
+    l.gsi_forward_host.argtypes = [vp, vp, i, vp, vp, vp, vp]
+    l.gsi_get_image.argtypes = [vp, i, C.POINTER(vp)]
+    l.gsi_get_status.argtypes = [vp, C.POINTER(i)]
+    l.gsi_destroy.argtypes = [vp]
+    l.gsi_stack_workspace_bytes.restype = sz
+    l.gsi_stack_workspace_bytes.argtypes = [i]
+    l.gsi_stack_create.argtypes = [i, C.POINTER(vp), vp, sz, vp, C.POINTER(vp)]
+    l.gsi_stack_bind.argtypes = [vp, C.POINTER(GsiStackIo), i, vp, vp, vp]
+    l.gsi_stack_seek.argtypes = [vp, i, vp]
+    l.gsi_stack_step.argtypes = [vp, vp]
+    l.gsi_stack_launches_per_step.argtypes = [vp, C.POINTER(i)]
+    l.gsi_stack_step_host.argtypes = [vp, C.POINTER(vp), C.POINTER(vp), vp, vp]
+    l.gsi_stack_get_status.argtypes = [vp, C.POINTER(i)]
+    l.gsi_stack_destroy.argtypes = [vp]
+    for name in EXPORTED:
+        if name not in ("gsi_status_string", "gsi_workspace_bytes", "gsi_stack_workspace_bytes"):
+            getattr(l, name).restype = i
+    return l
+
+
+lib = _load()
+
+
+def gsi_status_string(code) -> str:
+    return lib.gsi_status_string(int(code)).decode()
+
+
+def _check(code, where):
+    if code != 0:
+        raise GsiError(code, where)
+
+
+def _stream_ptr(stream) -> int:
+    if stream is None:
+        stream = torch.cuda.current_stream()
+    return int(stream.cuda_stream) if hasattr(stream, "cuda_stream") else int(stream)
+
+
+def _dtype_code(t: torch.Tensor) -> int:
+    if t.dtype == torch.bfloat16:
+        return GSI_BF16
+    if t.dtype == torch.float32:
+        return GSI_F32
+    raise TypeError("basis must be bfloat16 or float32")
+
+
+def make_desc(d, k, d_out, eps, max_tokens, p_dtype=GSI_BF16, flags=0):
+    arr = (C.c_int * len(d_out))(*[int(v) for v in d_out])
+    desc = GsiDesc(int(d), int(k), len(d_out), C.cast(arr, C.POINTER(C.c_int)), float(eps),
+                   int(max_tokens), int(p_dtype), int(flags))
+    desc._keep = arr
+    return desc
+
+
+def gsi_workspace_bytes(d, k, d_out, eps, max_tokens, p_dtype=GSI_BF16, flags=0) -> int:
+    return int(lib.gsi_workspace_bytes(C.byref(make_desc(d, k, d_out, eps, max_tokens, p_dtype, flags))))
+
+
+def gsi_build_image(W: torch.Tensor, P: torch.Tensor, out: torch.Tensor | None = None,
+                    stream=None) -> torch.Tensor:
+    """W_P = bf16(W P) on the device (Section 4.2 of the paper)."""
+    assert W.is_cuda and P.is_cuda and W.dtype == torch.bfloat16
+    assert W.is_contiguous() and P.is_contiguous()
+    o, d = W.shape
+    d2, k = P.shape
+    assert d == d2
+    if out is None:
+        out = torch.empty((o, k), dtype=torch.bfloat16, device=W.device)
+    _check(lib.gsi_build_image(W.data_ptr(), P.data_ptr(), o, d, k, _dtype_code(P),
+                               out.data_ptr(), _stream_ptr(stream)), "gsi_build_image")
+    return out
+
+
+class Layer:
+    """One group: maps ``Ws`` (list of [d_out_j][d] bf16) sharing basis ``P``."""
+
+    def __init__(self, Ws, P, eps: float, max_tokens: int = 1, flags: int = 0, stream=None):
+        Ws = list(Ws)
+        dense = bool(flags & GSI_FLAG_DENSE)
+        dev = Ws[0].device
+        assert dev.type == "cuda", "the gated subspace layer runs on a CUDA device only"
+        for W in Ws:
+            assert W.dtype == torch.bfloat16 and W.is_contiguous() and W.device == dev
+        self.d = int(Ws[0].shape[1])
+        self.d_out = [int(W.shape[0]) for W in Ws]
+        self.O = sum(self.d_out)
+        self.k = 8 if (dense and P is None) else int(P.shape[1])
+        self.max_tokens = int(max_tokens)
+        self.eps = float(eps)
+        self.flags = int(flags)
+        self._Ws, self._P = Ws, P
+        pd = GSI_BF16 if P is None else _dtype_code(P)
+        self._desc = make_desc(self.d, self.k, self.d_out, eps, max_tokens, pd, flags)
+        nbytes = int(lib.gsi_workspace_bytes(C.byref(self._desc)))
+        if nbytes == 0:
+            raise GsiError(2, "gsi_workspace_bytes (descriptor rejected)")
+        self.workspace = torch.empty(nbytes, dtype=torch.uint8, device=dev)
+        warr = (C.c_void_p * len(Ws))(*[W.data_ptr() for W in Ws])
+        h = C.c_void_p()
+        _check(lib.gsi_create(C.byref(self._desc), warr, None if P is None else P.data_ptr(),
+                              self.workspace.data_ptr(), nbytes, _stream_ptr(stream),
+                              C.byref(h)), "gsi_create")
+        self.handle = h
+        self.device = dev
+
+    def forward(self, x: torch.Tensor, y: torch.Tensor | None = None,
+                gate: torch.Tensor | None = None, rho: torch.Tensor | None = None, stream=None):
+        assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+        n = int(x.shape[0])
+        if y is None:
+            y = torch.empty((n, self.O), dtype=torch.float32, device=x.device)
+        if gate is None:
+            gate = torch.empty(n, dtype=torch.uint8, device=x.device)
+        if rho is None:
+            rho = torch.empty(n, dtype=torch.float32, device=x.device)
+        _check(lib.gsi_forward_n(self.handle, x.data_ptr(), n, y.data_ptr(), gate.data_ptr(),
+                                 rho.data_ptr(), _stream_ptr(stream)), "gsi_forward_n")
+        return y, gate, rho
+
+    def forward_host(self, x: torch.Tensor, stream=None):
+        """Host tensors in, host tensors out (copies inside the call)."""
+        assert not x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+        n = int(x.shape[0])
+        y = torch.empty((n, self.O), dtype=torch.float32).pin_memory()
+        gate = torch.empty(n, dtype=torch.uint8).pin_memory()
+        rho = torch.empty(n, dtype=torch.float32).pin_memory()
+        _check(lib.gsi_forward_host(self.handle, x.data_ptr(), n, y.data_ptr(), gate.data_ptr(),
+                                    rho.data_ptr(), _stream_ptr(stream)), "gsi_forward_host")
+        return y, gate, rho
+
+    def image(self, j: int) -> torch.Tensor:
+        """Copy of the cached image of map j ([d_out_j][k] bf16)."""
+        p = C.c_void_p()
+        _check(lib.gsi_get_image(self.handle, j, C.byref(p)), "gsi_get_image")
+        base = self.workspace.data_ptr()
+        off = p.value - base
+        nbytes = self.d_out[j] * self.k * 2
+        return self.workspace[off:off + nbytes].view(torch.bfloat16).view(self.d_out[j], self.k).clone()
+
+    def status(self) -> int:
+        v = C.c_int()
+        _check(lib.gsi_get_status(self.handle, C.byref(v)), "gsi_get_status")
+        return v.value
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib.gsi_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+class Stack:
+    """An ordered chain of groups stepped as one decode step."""
+
+    def __init__(self, layers, stream=None):
+        self.layers = list(layers)
+        n = len(self.layers)
+        dev = self.layers[0].device
+        self.B = self.layers[0].max_tokens
+        nbytes = int(lib.gsi_stack_workspace_bytes(n))
+        self.workspace = torch.zeros(nbytes, dtype=torch.uint8, device=dev)
+        arr = (C.c_void_p * n)(*[l.handle for l in self.layers])
+        h = C.c_void_p()
+        _check(lib.gsi_stack_create(n, arr, self.workspace.data_ptr(), nbytes,
+                                    _stream_ptr(stream), C.byref(h)), "gsi_stack_create")
+        self.handle = h
+        self.device = dev
+
+    def bind(self, xs, ys=None, n_steps: int = 1, want_rho: bool = True, stream=None):
+        """xs[g]: [n_steps][B][d] fp32 device tensors.  Allocates y and the logs."""
+        n = len(self.layers)
+        if ys is None:
+            ys = [torch.empty((self.B, l.O), dtype=torch.float32, device=self.device)
+                  for l in self.layers]
+        self.xs, self.ys, self.n_steps = list(xs), list(ys), int(n_steps)
+        for x, l in zip(self.xs, self.layers):
+            assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous()
+            assert x.numel() == n_steps * self.B * l.d
+        self.gate_log = torch.zeros((n_steps, n, self.B), dtype=torch.uint8, device=self.device)
+        self.rho_log = (torch.zeros((n_steps, n, self.B), dtype=torch.float32, device=self.device)
+                        if want_rho else None)
+        io = (GsiStackIo * n)(*[GsiStackIo(x.data_ptr(), y.data_ptr())
+                                for x, y in zip(self.xs, self.ys)])
+        _check(lib.gsi_stack_bind(self.handle, io, n_steps, self.gate_log.data_ptr(),
+                                  None if self.rho_log is None else self.rho_log.data_ptr(),
+                                  _stream_ptr(stream)), "gsi_stack_bind")
+
+    def seek(self, step: int, stream=None):
+        _check(lib.gsi_stack_seek(self.handle, int(step), _stream_ptr(stream)), "gsi_stack_seek")
+
+    def step(self, stream=None):
+        _check(lib.gsi_stack_step(self.handle, _stream_ptr(stream)), "gsi_stack_step")
+
+    def launches_per_step(self) -> int:
+        v = C.c_int()
+        _check(lib.gsi_stack_launches_per_step(self.handle, C.byref(v)),
+               "gsi_stack_launches_per_step")
+        return v.value
+
+    def step_host(self, xs_host, ys_host, gate_host, stream=None):
+        n = len(self.layers)
+        xa = (C.c_void_p * n)(*[x.data_ptr() for x in xs_host])
+        ya = (C.c_void_p * n)(*[y.data_ptr() for y in ys_host])
+        _check(lib.gsi_stack_step_host(self.handle, xa, ya, gate_host.data_ptr(),
+                                       _stream_ptr(stream)), "gsi_stack_step_host")
+
+    def status(self) -> int:
+        v = C.c_int()
+        _check(lib.gsi_stack_get_status(self.handle, C.byref(v)), "gsi_stack_get_status")
+        return v.value
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib.gsi_stack_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass

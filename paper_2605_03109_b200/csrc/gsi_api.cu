@@ -1,0 +1,424 @@
+// C ABI of the gated subspace layer: argument checking, workspace layout,
+// handle and stack bookkeeping, kernel sequencing.  No arithmetic lives here.
+#include <new>
+#include <vector>
+#include <cstring>
+
+#include "gsi_common.cuh"
+
+using namespace gsi;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kSlabTarget = 148;  // one basis slab per SM of a B200
+
+inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+struct Layout {
+  size_t wp, c, cpart, r, normpart, ctrl, fired, rho, x_stage, y_stage, gate_stage, rho_stage, total;
+  int O, n_slabs, slab_rows;
+};
+
+gsi_status_t check_desc(const gsi_desc_t* d) {
+  if (!d || !d->d_out) return GSI_ERR_INVALID_ARG;
+  if (d->d <= 0 || d->n_maps <= 0 || d->max_tokens <= 0) return GSI_ERR_INVALID_ARG;
+  if (d->n_maps > GSI_MAX_MAPS || d->max_tokens > GSI_MAX_TOKENS) return GSI_ERR_UNSUPPORTED;
+  if (d->p_dtype != GSI_BF16 && d->p_dtype != GSI_F32) return GSI_ERR_INVALID_ARG;
+  if (d->d % 8) return GSI_ERR_UNSUPPORTED;
+  for (int j = 0; j < d->n_maps; ++j) {
+    if (d->d_out[j] <= 0) return GSI_ERR_INVALID_ARG;
+    if (d->d_out[j] % 8) return GSI_ERR_UNSUPPORTED;
+  }
+  if (!(d->flags & GSI_FLAG_DENSE)) {
+    if (d->k <= 0) return GSI_ERR_INVALID_ARG;
+    if (d->k % 8 || d->k > 1024 || d->k > d->d) return GSI_ERR_UNSUPPORTED;
+    if (!(d->eps >= 0.f)) return GSI_ERR_INVALID_ARG;  // also rejects NaN
+  }
+  return GSI_OK;
+}
+
+Layout make_layout_ws(const gsi_desc_t* d) {
+  Layout L{};
+  const bool dense = d->flags & GSI_FLAG_DENSE;
+  const size_t B = d->max_tokens, k = dense ? 0 : d->k;
+  int O = 0;
+  for (int j = 0; j < d->n_maps; ++j) O += d->d_out[j];
+  L.O = O;
+  int slab = (d->d + kSlabTarget - 1) / kSlabTarget;
+  if (slab < 8) slab = 8;
+  L.slab_rows = slab;
+  L.n_slabs = (d->d + slab - 1) / slab;
+  size_t at = 0;
+  auto take = [&](size_t bytes) { size_t o = at; at += align_up(bytes); return o; };
+  L.wp = take((size_t)O * k * 2);
+  L.c = take(B * k * 4);
+  L.cpart = take((size_t)L.n_slabs * B * k * 4);
+  L.r = take(dense ? 0 : B * d->d * 4);
+  L.normpart = take((size_t)L.n_slabs * B * 2 * 4);
+  L.ctrl = take(256);
+  L.fired = take(B * 4);
+  L.rho = take(B * 4);
+  L.x_stage = take(B * d->d * 4);
+  L.y_stage = take(B * (size_t)O * 4);
+  L.gate_stage = take(B);
+  L.rho_stage = take(B * 4);
+  L.total = at;
+  return L;
+}
+
+}  // namespace
+
+struct gsi_layer {
+  gsi_desc_t desc;
+  int d_out[GSI_MAX_MAPS];
+  Layout lay;
+  GroupParams gp;
+  char* ws;
+  cudaStream_t last_stream;
+};
+
+struct gsi_stack {
+  std::vector<gsi_layer*> groups;
+  std::vector<gsi_stack_io_t> io;
+  int B;
+  int n_steps;
+  unsigned char* gate_log;
+  float* rho_log;
+  int* step;  // device
+  bool bound;
+  cudaStream_t last_stream;
+};
+
+extern "C" {
+
+const char* gsi_status_string(gsi_status_t s) {
+  switch (s) {
+    case GSI_OK: return "ok";
+    case GSI_ERR_INVALID_ARG: return "invalid argument";
+    case GSI_ERR_UNSUPPORTED: return "unsupported shape";
+    case GSI_ERR_ALLOC: return "host allocation failed";
+    case GSI_ERR_CUDA: return "CUDA runtime error";
+    case GSI_ERR_TIMEOUT: return "device-side wait timed out";
+    case GSI_ERR_WORKSPACE: return "workspace too small";
+  }
+  return "unknown status";
+}
+
+gsi_status_t gsi_build_image(const void* W, const void* P, int o, int d, int k,
+                             gsi_dtype_t p_dtype, void* W_P_out, gsi_stream_t stream) {
+  if (!W || !P || !W_P_out || o <= 0 || d <= 0 || k <= 0) return GSI_ERR_INVALID_ARG;
+  if (p_dtype != GSI_BF16 && p_dtype != GSI_F32) return GSI_ERR_INVALID_ARG;
+  if (!aligned16(W) || !aligned16(P) || !aligned16(W_P_out)) return GSI_ERR_INVALID_ARG;
+  if (o % 8 || d % 8 || k % 8) return GSI_ERR_UNSUPPORTED;
+  return launch_build_image(W, P, o, d, k, p_dtype == GSI_F32, W_P_out, stream) == cudaSuccess
+             ? GSI_OK
+             : GSI_ERR_CUDA;
+}
+
+size_t gsi_workspace_bytes(const gsi_desc_t* desc) {
+  if (check_desc(desc) != GSI_OK) return 0;
+  return make_layout_ws(desc).total;
+}
+
+gsi_status_t gsi_create(const gsi_desc_t* desc, const void* const* W, const void* P,
+                        void* workspace, size_t workspace_bytes, gsi_stream_t stream,
+                        gsi_handle_t* out) {
+  if (!out) return GSI_ERR_INVALID_ARG;
+  *out = nullptr;
+  gsi_status_t st = check_desc(desc);
+  if (st != GSI_OK) return st;
+  const bool dense = desc->flags & GSI_FLAG_DENSE;
+  if (!W || !workspace || (!dense && !P)) return GSI_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) % kAlign) || (P && !aligned16(P)))
+    return GSI_ERR_INVALID_ARG;
+  for (int j = 0; j < desc->n_maps; ++j)
+    if (!W[j] || !aligned16(W[j])) return GSI_ERR_INVALID_ARG;
+  Layout L = make_layout_ws(desc);
+  if (workspace_bytes < L.total) return GSI_ERR_WORKSPACE;
+
+  gsi_layer* h = new (std::nothrow) gsi_layer();
+  if (!h) return GSI_ERR_ALLOC;
+  h->desc = *desc;
+  std::memcpy(h->d_out, desc->d_out, sizeof(int) * desc->n_maps);
+  h->desc.d_out = h->d_out;
+  h->lay = L;
+  h->ws = static_cast<char*>(workspace);
+  h->last_stream = stream;
+
+  GroupParams& g = h->gp;
+  std::memset(&g, 0, sizeof g);
+  g.d = desc->d;
+  g.k = dense ? 8 : desc->k;
+  g.O = L.O;
+  g.B = desc->max_tokens;
+  g.p_f32 = desc->p_dtype == GSI_F32;
+  g.eps = desc->eps;
+  g.flags = desc->flags;
+  g.P = P;
+  g.WP = reinterpret_cast<const uint16_t*>(h->ws + L.wp);
+  g.n_maps = desc->n_maps;
+  int off = 0;
+  for (int j = 0; j < desc->n_maps; ++j) {
+    g.W[j] = static_cast<const uint16_t*>(W[j]);
+    g.d_out[j] = desc->d_out[j];
+    g.off[j] = off;
+    off += desc->d_out[j];
+  }
+  g.off[desc->n_maps] = off;
+  g.c = reinterpret_cast<float*>(h->ws + L.c);
+  g.cpart = reinterpret_cast<float*>(h->ws + L.cpart);
+  g.r = reinterpret_cast<float*>(h->ws + L.r);
+  g.normpart = reinterpret_cast<float*>(h->ws + L.normpart);
+  int* ctrl = reinterpret_cast<int*>(h->ws + L.ctrl);
+  g.n_fired = ctrl + 0;
+  g.counter = reinterpret_cast<unsigned*>(ctrl + 1);
+  g.status = ctrl + 2;
+  g.fired = reinterpret_cast<int*>(h->ws + L.fired);
+  g.rho_scratch = reinterpret_cast<float*>(h->ws + L.rho);
+  g.n_slabs = L.n_slabs;
+  g.slab_rows = L.slab_rows;
+
+  if (cudaMemsetAsync(ctrl, 0, 256, stream) != cudaSuccess) {
+    delete h;
+    return GSI_ERR_CUDA;
+  }
+  if (!dense) {
+    for (int j = 0; j < desc->n_maps; ++j) {
+      void* dst = h->ws + L.wp + (size_t)g.off[j] * desc->k * 2;
+      if (launch_build_image(W[j], P, desc->d_out[j], desc->d, desc->k, g.p_f32, dst, stream) !=
+          cudaSuccess) {
+        delete h;
+        return GSI_ERR_CUDA;
+      }
+    }
+  }
+  *out = h;
+  return GSI_OK;
+}
+
+gsi_status_t gsi_forward_n(gsi_handle_t h, const float* x, int n_tokens, float* y,
+                           unsigned char* gate_mask_out, float* rho_out, gsi_stream_t stream) {
+  if (!h || n_tokens < 0 || n_tokens > h->desc.max_tokens) return GSI_ERR_INVALID_ARG;
+  if (n_tokens == 0) return GSI_OK;
+  if (!x || !y || !gate_mask_out) return GSI_ERR_INVALID_ARG;
+  if (!aligned16(x) || !aligned16(y)) return GSI_ERR_INVALID_ARG;
+  IoRef io{};
+  io.x = x;
+  io.y = y;
+  io.gate = gate_mask_out;
+  io.rho = rho_out;
+  io.step = nullptr;
+  io.n_steps = 1;
+  h->last_stream = stream;
+  return launch_generic_forward(h->gp, io, n_tokens, stream, nullptr) == cudaSuccess ? GSI_OK
+                                                                                      : GSI_ERR_CUDA;
+}
+
+gsi_status_t gsi_forward(gsi_handle_t h, const float* x, float* y, unsigned char* gate_mask_out,
+                         gsi_stream_t stream) {
+  if (!h) return GSI_ERR_INVALID_ARG;
+  return gsi_forward_n(h, x, h->desc.max_tokens, y, gate_mask_out, nullptr, stream);
+}
+
+gsi_status_t gsi_forward_host(gsi_handle_t h, const float* x_host, int n_tokens, float* y_host,
+                              unsigned char* gate_mask_host, float* rho_host,
+                              gsi_stream_t stream) {
+  if (!h || n_tokens < 0 || n_tokens > h->desc.max_tokens) return GSI_ERR_INVALID_ARG;
+  if (n_tokens == 0) return GSI_OK;
+  if (!x_host || !y_host || !gate_mask_host) return GSI_ERR_INVALID_ARG;
+  const Layout& L = h->lay;
+  float* xs = reinterpret_cast<float*>(h->ws + L.x_stage);
+  float* ys = reinterpret_cast<float*>(h->ws + L.y_stage);
+  unsigned char* gs = reinterpret_cast<unsigned char*>(h->ws + L.gate_stage);
+  float* rs = reinterpret_cast<float*>(h->ws + L.rho_stage);
+  const size_t n = n_tokens;
+  if (cudaMemcpyAsync(xs, x_host, n * h->desc.d * 4, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+    return GSI_ERR_CUDA;
+  gsi_status_t st = gsi_forward_n(h, xs, n_tokens, ys, gs, rs, stream);
+  if (st != GSI_OK) return st;
+  // rows of y are contiguous because the device buffer is [n][O] for any n
+  if (cudaMemcpyAsync(y_host, ys, n * L.O * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess ||
+      cudaMemcpyAsync(gate_mask_host, gs, n, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+    return GSI_ERR_CUDA;
+  if (rho_host &&
+      cudaMemcpyAsync(rho_host, rs, n * 4, cudaMemcpyDeviceToHost, stream) != cudaSuccess)
+    return GSI_ERR_CUDA;
+  return cudaStreamSynchronize(stream) == cudaSuccess ? GSI_OK : GSI_ERR_CUDA;
+}
+
+gsi_status_t gsi_get_image(gsi_handle_t h, int map, const void** out) {
+  if (!h || !out || map < 0 || map >= h->desc.n_maps) return GSI_ERR_INVALID_ARG;
+  if (h->desc.flags & GSI_FLAG_DENSE) return GSI_ERR_UNSUPPORTED;
+  *out = h->ws + h->lay.wp + (size_t)h->gp.off[map] * h->desc.k * 2;
+  return GSI_OK;
+}
+
+gsi_status_t gsi_get_status(gsi_handle_t h, int* device_status) {
+  if (!h || !device_status) return GSI_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(h->last_stream) != cudaSuccess) return GSI_ERR_CUDA;
+  if (cudaMemcpy(device_status, h->gp.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return GSI_ERR_CUDA;
+  return GSI_OK;
+}
+
+gsi_status_t gsi_destroy(gsi_handle_t h) {
+  if (!h) return GSI_ERR_INVALID_ARG;
+  delete h;
+  return GSI_OK;
+}
+
+// ------------------------------------------------------------------ stack
+size_t gsi_stack_workspace_bytes(int n_groups) {
+  if (n_groups <= 0) return 0;
+  return align_up(256) + align_up((size_t)n_groups * 512);
+}
+
+gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* workspace,
+                              size_t workspace_bytes, gsi_stream_t stream, gsi_stack_t* out) {
+  if (!out) return GSI_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (n_groups <= 0 || !groups || !workspace) return GSI_ERR_INVALID_ARG;
+  if (reinterpret_cast<uintptr_t>(workspace) % kAlign) return GSI_ERR_INVALID_ARG;
+  if (workspace_bytes < gsi_stack_workspace_bytes(n_groups)) return GSI_ERR_WORKSPACE;
+  for (int i = 0; i < n_groups; ++i) {
+    if (!groups[i]) return GSI_ERR_INVALID_ARG;
+    if (groups[i]->desc.max_tokens != groups[0]->desc.max_tokens) return GSI_ERR_INVALID_ARG;
+  }
+  gsi_stack* s = new (std::nothrow) gsi_stack();
+  if (!s) return GSI_ERR_ALLOC;
+  s->groups.assign(groups, groups + n_groups);
+  s->io.resize(n_groups);
+  s->B = groups[0]->desc.max_tokens;
+  s->n_steps = 0;
+  s->gate_log = nullptr;
+  s->rho_log = nullptr;
+  s->step = static_cast<int*>(workspace);
+  s->bound = false;
+  s->last_stream = stream;
+  if (cudaMemsetAsync(workspace, 0, 256, stream) != cudaSuccess) {
+    delete s;
+    return GSI_ERR_CUDA;
+  }
+  *out = s;
+  return GSI_OK;
+}
+
+gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps,
+                            unsigned char* gate_log, float* rho_log, gsi_stream_t stream) {
+  if (!s || !io || n_steps <= 0 || !gate_log) return GSI_ERR_INVALID_ARG;
+  for (size_t i = 0; i < s->groups.size(); ++i)
+    if (!io[i].x || !io[i].y || !aligned16(io[i].x) || !aligned16(io[i].y))
+      return GSI_ERR_INVALID_ARG;
+  std::copy(io, io + s->groups.size(), s->io.begin());
+  s->n_steps = n_steps;
+  s->gate_log = gate_log;
+  s->rho_log = rho_log;
+  s->bound = true;
+  s->last_stream = stream;
+  return GSI_OK;
+}
+
+gsi_status_t gsi_stack_seek(gsi_stack_t s, int step, gsi_stream_t stream) {
+  if (!s || step < 0) return GSI_ERR_INVALID_ARG;
+  // 4-byte pattern set is not available through cudaMemsetAsync; stage via a
+  // pageable copy, which the runtime completes before returning.
+  s->last_stream = stream;
+  return cudaMemcpyAsync(s->step, &step, sizeof(int), cudaMemcpyHostToDevice, stream) ==
+                 cudaSuccess
+             ? GSI_OK
+             : GSI_ERR_CUDA;
+}
+
+static gsi_status_t stack_enqueue(gsi_stack_t s, bool use_counter, gsi_stream_t stream,
+                                  int* n_launches) {
+  const int G = (int)s->groups.size();
+  for (int i = 0; i < G; ++i) {
+    gsi_layer* h = s->groups[i];
+    IoRef io{};
+    io.x = s->io[i].x;
+    io.y = s->io[i].y;
+    io.gate = s->gate_log + (size_t)i * s->B;
+    io.rho = s->rho_log ? s->rho_log + (size_t)i * s->B : nullptr;
+    io.step = use_counter ? s->step : nullptr;
+    io.n_steps = s->n_steps;
+    io.x_step_stride = (long long)s->B * h->desc.d;
+    io.log_step_stride = (long long)G * s->B;
+    h->last_stream = stream;
+    if (launch_generic_forward(h->gp, io, s->B, stream, n_launches) != cudaSuccess)
+      return GSI_ERR_CUDA;
+  }
+  if (use_counter) {
+    if (launch_advance_step(s->step, stream) != cudaSuccess) return GSI_ERR_CUDA;
+    if (n_launches) *n_launches += 1;
+  }
+  return GSI_OK;
+}
+
+gsi_status_t gsi_stack_step(gsi_stack_t s, gsi_stream_t stream) {
+  if (!s || !s->bound) return GSI_ERR_INVALID_ARG;
+  s->last_stream = stream;
+  return stack_enqueue(s, true, stream, nullptr);
+}
+
+gsi_status_t gsi_stack_launches_per_step(gsi_stack_t s, int* n_out) {
+  if (!s || !n_out) return GSI_ERR_INVALID_ARG;
+  int n = 0;
+  for (gsi_layer* h : s->groups) {
+    if (h->desc.flags & GSI_FLAG_DENSE) n += 1;
+    else n += (h->desc.flags & GSI_FLAG_STATIC_PROJECTION) ? 4 : 5;
+  }
+  *n_out = n + 1;
+  return GSI_OK;
+}
+
+gsi_status_t gsi_stack_step_host(gsi_stack_t s, const float* const* x_host, float* const* y_host,
+                                 unsigned char* gate_host, gsi_stream_t stream) {
+  if (!s || !s->bound || !x_host || !y_host || !gate_host) return GSI_ERR_INVALID_ARG;
+  const int G = (int)s->groups.size();
+  for (int i = 0; i < G; ++i) {
+    if (!x_host[i] || !y_host[i]) return GSI_ERR_INVALID_ARG;
+    const size_t bytes = (size_t)s->B * s->groups[i]->desc.d * 4;
+    if (cudaMemcpyAsync(const_cast<float*>(s->io[i].x), x_host[i], bytes, cudaMemcpyHostToDevice,
+                        stream) != cudaSuccess)
+      return GSI_ERR_CUDA;
+  }
+  s->last_stream = stream;
+  gsi_status_t st = stack_enqueue(s, false, stream, nullptr);
+  if (st != GSI_OK) return st;
+  for (int i = 0; i < G; ++i) {
+    const size_t bytes = (size_t)s->B * s->groups[i]->lay.O * 4;
+    if (cudaMemcpyAsync(y_host[i], s->io[i].y, bytes, cudaMemcpyDeviceToHost, stream) !=
+        cudaSuccess)
+      return GSI_ERR_CUDA;
+  }
+  if (cudaMemcpyAsync(gate_host, s->gate_log, (size_t)G * s->B, cudaMemcpyDeviceToHost, stream) !=
+      cudaSuccess)
+    return GSI_ERR_CUDA;
+  return cudaStreamSynchronize(stream) == cudaSuccess ? GSI_OK : GSI_ERR_CUDA;
+}
+
+gsi_status_t gsi_stack_get_status(gsi_stack_t s, int* device_status) {
+  if (!s || !device_status) return GSI_ERR_INVALID_ARG;
+  if (cudaStreamSynchronize(s->last_stream) != cudaSuccess) return GSI_ERR_CUDA;
+  *device_status = 0;
+  for (gsi_layer* h : s->groups) {
+    int v = 0;
+    if (cudaMemcpy(&v, h->gp.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+      return GSI_ERR_CUDA;
+    if (v) {
+      *device_status = v;
+      break;
+    }
+  }
+  return GSI_OK;
+}
+
+gsi_status_t gsi_stack_destroy(gsi_stack_t s) {
+  if (!s) return GSI_ERR_INVALID_ARG;
+  delete s;
+  return GSI_OK;
+}
+
+}  // extern "C"

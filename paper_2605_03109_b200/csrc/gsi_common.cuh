@@ -1,0 +1,104 @@
+// Shared device helpers and internal declarations of the gated subspace layer.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+#include "gsi.h"
+
+namespace gsi {
+
+constexpr int kWarp = 32;
+constexpr int kTokChunk = 4;  // tokens held in registers at once by the generic kernels
+
+// Where a group's activations and logs live for the current decode step.  A
+// plain gsi_forward call has step == nullptr (offset 0).
+struct IoRef {
+  const float* x;       // [n_steps][B][d] (or [B][d])
+  float* y;             // [B][O]
+  unsigned char* gate;  // [n_steps][log_groups][B] (or [B])
+  float* rho;           // same shape as gate, or nullptr
+  const int* step;      // device step counter or nullptr
+  int n_steps;
+  long long x_step_stride;    // elements between steps of x
+  long long log_step_stride;  // elements between steps of gate / rho
+};
+
+__device__ __forceinline__ int io_slot(const IoRef& io) {
+  return io.step ? (*io.step % io.n_steps) : 0;
+}
+
+// 8 consecutive basis / image entries as fp32.
+__device__ __forceinline__ void unpack_bf16x8(const uint4& v, float (&f)[8]) {
+  f[0] = __uint_as_float(v.x << 16);
+  f[1] = __uint_as_float(v.x & 0xFFFF0000u);
+  f[2] = __uint_as_float(v.y << 16);
+  f[3] = __uint_as_float(v.y & 0xFFFF0000u);
+  f[4] = __uint_as_float(v.z << 16);
+  f[5] = __uint_as_float(v.z & 0xFFFF0000u);
+  f[6] = __uint_as_float(v.w << 16);
+  f[7] = __uint_as_float(v.w & 0xFFFF0000u);
+}
+
+// Element index `idx8` counts groups of 8 elements from `base`.
+template <bool kF32>
+__device__ __forceinline__ void load8(const void* base, size_t idx8, float (&f)[8]) {
+  if constexpr (kF32) {
+    const float4* p = reinterpret_cast<const float4*>(base) + idx8 * 2;
+    float4 a = __ldg(p), b = __ldg(p + 1);
+    f[0] = a.x; f[1] = a.y; f[2] = a.z; f[3] = a.w;
+    f[4] = b.x; f[5] = b.y; f[6] = b.z; f[7] = b.w;
+  } else {
+    uint4 v = __ldg(reinterpret_cast<const uint4*>(base) + idx8);
+    unpack_bf16x8(v, f);
+  }
+}
+
+// One-shot weight stream: do not keep it in L1.
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+  uint4 v;
+  asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];"
+               : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w)
+               : "l"(p));
+  return v;
+}
+
+__device__ __forceinline__ float warp_sum(float v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+  return v;
+}
+
+// ---- generic path (any supported shape, any batch <= GSI_MAX_TOKENS) --------
+struct GroupParams {
+  int d, k, O, B;            // O = sum of d_out
+  int p_f32;                 // basis stored as fp32
+  float eps;
+  unsigned flags;
+  const void* P;             // [d][k]
+  const uint16_t* WP;        // [O][k] bf16 (concatenated images)
+  int n_maps;
+  const uint16_t* W[GSI_MAX_MAPS];  // [d_out_j][d] bf16
+  int d_out[GSI_MAX_MAPS];
+  int off[GSI_MAX_MAPS + 1];
+  // scratch
+  float* c;         // [B][k]
+  float* cpart;     // [n_slabs][B][k]
+  float* r;         // [B][d]
+  float* normpart;  // [n_slabs][B][2]
+  int* fired;       // [B] token indices, ascending
+  int* n_fired;     // [1]
+  unsigned* counter;  // [1] arrival counter of the residual kernel
+  float* rho_scratch; // [B]
+  int* status;      // [1]
+  int n_slabs, slab_rows;
+};
+
+cudaError_t launch_generic_forward(const GroupParams& g, const IoRef& io, int n_tokens,
+                                   cudaStream_t stream, int* n_launches);
+cudaError_t launch_advance_step(int* step, cudaStream_t stream);
+cudaError_t launch_build_image(const void* W, const void* P, int o, int d, int k, bool p_f32,
+                               void* WP, cudaStream_t stream);
+
+}  // namespace gsi

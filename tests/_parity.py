@@ -1,0 +1,73 @@
+"""Shared comparison logic: CUDA path vs fp64 oracle on the same stored inputs."""
+from __future__ import annotations
+
+import numpy as np
+import torch
+
+import synthetic as S
+from oracle import gsi_oracle as O
+
+Y_TOL = 1e-2        # max-abs error <= Y_TOL * ||y_ref||_inf per token and map (bf16 weights, fp32 accumulation)
+BAND = 1e-3         # gate bytes may differ only where |rho_oracle/eps - 1| < BAND
+RHO_RTOL = 2e-5     # fp32 explicit residual vs fp64
+
+
+def compare_group(x, P, Ws, eps, y_gpu, gate_gpu, rho_gpu=None, rows=None, static=False):
+    """x [T][d] fp32 (cpu tensor), P stored basis (cpu tensor), Ws list of bf16
+    cpu tensors (already row-sampled if ``rows`` given: then y_gpu holds the
+    same sampled columns per map).  Returns a dict of statistics; raises on a
+    violation of the acceptance bar."""
+    xn = x.numpy()
+    Pn = S.bits_of(P)
+    Wn = [S.to_bf16_bits(W) for W in Ws]
+    eps32 = float(np.float32(eps))
+    pr = O.project(xn, Pn, eps32)
+    gate_o = pr["gate"]
+    gate_g = np.asarray(gate_gpu, dtype=np.uint8)
+    with np.errstate(divide="ignore", invalid="ignore"):
+        near = np.abs(pr["rho"] / eps32 - 1.0) < BAND if eps32 > 0 else np.zeros_like(gate_o, bool)
+    mism = gate_o != gate_g
+    bad = mism & ~near
+    assert not bad.any(), (
+        f"gate mismatch outside the +-{BAND} band at tokens {np.nonzero(bad)[0][:8]}, "
+        f"rho={pr['rho'][bad][:8]}, eps={eps32}")
+    # y against the oracle evaluated with the GPU's gate decision
+    used = np.zeros_like(gate_g) if static else gate_g
+    off = 0
+    max_rel = 0.0
+    for j, W in enumerate(Wn):
+        M = O.image(W, Pn)
+        y_ref = O.apply_map(M, W, pr["g"], pr["r"], used)
+        o = W.shape[0]
+        yg = np.asarray(y_gpu[:, off:off + o], dtype=np.float64)
+        off += o
+        scale = np.max(np.abs(y_ref), axis=1)
+        err = np.max(np.abs(yg - y_ref), axis=1)
+        finite = np.isfinite(scale) & (scale > 0)
+        if finite.any():
+            rel = err[finite] / scale[finite]
+            max_rel = max(max_rel, float(rel.max()))
+            assert rel.max() <= Y_TOL, f"map {j}: max-abs error {rel.max():.3e} * ||y||_inf > {Y_TOL}"
+        zero = np.isfinite(scale) & (scale == 0)
+        assert np.all(err[zero] == 0)
+    if rho_gpu is not None:
+        rg = np.asarray(rho_gpu, dtype=np.float64)
+        ok = np.isfinite(pr["rho"]) & (pr["rho"] > 1e-5)
+        if ok.any():
+            assert np.max(np.abs(rg[ok] / pr["rho"][ok] - 1.0)) <= RHO_RTOL
+    return dict(gate_rate=float(gate_g.mean()), near=int(near.sum()), flips=int(mism.sum()),
+                max_rel_err=max_rel, oracle=pr)
+
+
+def image_ulp_check(W, P, wp_gpu):
+    """The stored image equals bf16_rne(W P in fp64) up to one bf16 ulp (ties
+    and fp32 accumulation order may flip the last bit)."""
+    M = O.image(S.to_bf16_bits(W), S.bits_of(P))
+    ref_bits = O.f64_to_bf16_rne(M).astype(np.int32)
+    got_bits = S.to_bf16_bits(wp_gpu).astype(np.int32)
+
+    def ordered(b):  # sign-magnitude -> monotone integer
+        return np.where(b & 0x8000, -(b & 0x7FFF), b & 0x7FFF)
+    diff = np.abs(ordered(ref_bits) - ordered(got_bits))
+    assert diff.max() <= 1, f"image differs from bf16(M_fp64) by {diff.max()} ulp"
+    return float((diff > 0).mean())

@@ -1,0 +1,291 @@
+"""Parity of the CUDA path with the fp64 oracle, through the C ABI.
+
+Acceptance (per token and map): gate bytes bit-exact except where the oracle's
+rho lies within 1e-3 (relative) of eps; max-abs error of y at most
+1e-2 * ||y_ref||_inf, y_ref being the oracle evaluated with the GPU's gate bit.
+"""
+import numpy as np
+import pytest
+import torch
+
+import synthetic as S
+from _parity import compare_group, image_ulp_check
+
+pytestmark = pytest.mark.gpu
+
+
+def G():
+    import paper_2605_03109_b200 as g
+    return g
+
+
+def make_small(d, k, d_out, T, seed, noise=0.03, p_dtype="bf16", rank=None, outlier_every=0):
+    q = S.gen_basis(d, k, seed)
+    P = S.store_basis(q, p_dtype)
+    Ws = [S.gen_weight(o, d, seed + 10 + j) for j, o in enumerate(d_out)]
+    rank = rank or max(1, k // 2)
+    pt = S.gen_true_basis(q, rank, rank, seed + 1)
+    x, _ = S.gen_activations(pt, T, noise, 0.0, dict(z=seed + 2, noise=seed + 3,
+                                                     outlier_mask=0, outlier_values=0))
+    if outlier_every:
+        g = torch.Generator().manual_seed(seed + 4)
+        x[::outlier_every] = torch.randn((len(range(0, T, outlier_every)), d), generator=g)
+    return x.contiguous(), P, Ws
+
+
+def run_layer(x, P, Ws, eps, batch, flags=0):
+    g = G()
+    dev = "cuda"
+    lay = g.Layer([W.to(dev) for W in Ws], None if P is None else P.to(dev), eps,
+                  max_tokens=batch, flags=flags)
+    T = x.shape[0]
+    ys, gates, rhos = [], [], []
+    xd = x.to(dev)
+    for t0 in range(0, T, batch):
+        y, gate, rho = lay.forward(xd[t0:t0 + batch].contiguous())
+        ys.append(y.cpu())
+        gates.append(gate.cpu())
+        rhos.append(rho.cpu())
+    torch.cuda.synchronize()
+    assert lay.status() == 0
+    return lay, torch.cat(ys).numpy(), torch.cat(gates).numpy(), torch.cat(rhos).numpy()
+
+
+@pytest.mark.parametrize("d,k,d_out,T,batch", [
+    (64, 8, (8,), 3, 1),
+    (72, 24, (40, 16), 5, 2),          # k/8 = 3: not a power of two
+    (256, 64, (264,), 7, 3),           # ragged batch tail
+    (1000, 96, (120, 8, 8), 9, 4),     # d not a multiple of the slab size
+    (520, 264, (72,), 4, 4),           # k > 256: two vectors per lane
+    (2048, 512, (136,), 6, 5),
+    (1536, 1024, (64,), 3, 1),         # largest supported k
+])
+def test_small_and_odd_shapes(d, k, d_out, T, batch):
+    x, P, Ws = make_small(d, k, d_out, T, seed=d + k, noise=0.05, outlier_every=3)
+    for eps in (0.05, 0.3):
+        lay, y, gate, rho = run_layer(x, P, Ws, eps, batch)
+        st = compare_group(x, P, Ws, eps, y, gate, rho)
+        assert 0 < st["gate_rate"] <= 1.0
+
+
+def test_config1_literal_batch1_all_tokens():
+    st = S.config1()
+    m = S.materialize_group(st, 0, 0, st.steps)
+    lay, y, gate, rho = run_layer(m["x"], m["P"], m["W"], st.eps, 1)
+    res = compare_group(m["x"], m["P"], m["W"], st.eps, y, gate, rho)
+    assert res["gate_rate"] > 0.95          # this recipe fires (nearly) every token
+    frac = image_ulp_check(m["W"][0], m["P"], lay.image(0).cpu())
+    assert frac < 0.05
+
+
+def test_config1_fast_companion_exercises_the_fast_path():
+    st = S.config1_fast()
+    m = S.materialize_group(st, 0, 0, st.steps)
+    lay, y, gate, rho = run_layer(m["x"], m["P"], m["W"], st.eps, 1)
+    res = compare_group(m["x"], m["P"], m["W"], st.eps, y, gate, rho)
+    assert 0.0 < res["gate_rate"] < 0.2
+    # the fired tokens are exactly the full-rank outliers
+    assert np.array_equal(gate.astype(bool), m["outlier"].numpy())
+
+
+@pytest.mark.parametrize("batch", [1, 2, 3, 64])
+def test_batches_and_batch_invariance(batch):
+    x, P, Ws = make_small(768, 128, (768, 2304), 64, seed=5, noise=0.02, outlier_every=5)
+    lay, y, gate, rho = run_layer(x, P, Ws, 0.05, batch)
+    compare_group(x, P, Ws, 0.05, y, gate, rho)
+    _, y1, gate1, rho1 = run_layer(x, P, Ws, 0.05, 1)
+    assert np.array_equal(gate, gate1)
+    # fixed-order reductions: a token's result does not depend on its batch
+    assert np.array_equal(y, y1) and np.array_equal(rho, rho1)
+
+
+def test_rerun_is_bit_identical():
+    x, P, Ws = make_small(4096, 256, (4096, 512), 8, seed=9, noise=0.0107, rank=200, outlier_every=4)
+    _, y_a, g_a, r_a = run_layer(x, P, Ws, 0.05, 4)
+    _, y_b, g_b, r_b = run_layer(x, P, Ws, 0.05, 4)
+    assert np.array_equal(y_a, y_b) and np.array_equal(g_a, g_b) and np.array_equal(r_a, r_b)
+
+
+def test_eps_zero_is_the_dense_product():
+    """eps = 0 gates every token and y = W x up to rounding."""
+    x, P, Ws = make_small(512, 64, (256,), 6, seed=11)
+    lay, y, gate, rho = run_layer(x, P, Ws, 0.0, 2)
+    assert gate.all()
+    W = Ws[0].to(torch.float64)
+    ref = (x.to(torch.float64) @ W.T).numpy()
+    assert np.max(np.abs(y - ref)) <= 1e-2 * np.max(np.abs(ref))
+    compare_group(x, P, Ws, 0.0, y, gate, rho)
+
+
+def test_fp32_basis_and_x_in_span():
+    d, k = 512, 64
+    q = S.gen_basis(d, k, 21)
+    P = S.store_basis(q, "f32")
+    Ws = [S.gen_weight(128, d, 22)]
+    z = torch.randn((5, k), dtype=torch.float64, generator=torch.Generator().manual_seed(23))
+    x = (z @ q.T).to(torch.float32).contiguous()
+    lay, y, gate, rho = run_layer(x, P, Ws, 0.01, 1)
+    assert not gate.any() and rho.max() < 1e-5
+    compare_group(x, P, Ws, 0.01, y, gate)
+    # the same tokens against the bf16-stored basis: rho ~ 1e-3, still fast
+    Pb = S.store_basis(q, "bf16")
+    lay, y, gate, rho = run_layer(x, Pb, Ws, 0.01, 1)
+    assert not gate.any() and 1e-5 < rho.max() < 5e-3
+    compare_group(x, Pb, Ws, 0.01, y, gate, rho)
+
+
+def test_k_equals_d():
+    d = 64
+    x, P, Ws = make_small(d, d, (32,), 4, seed=31, p_dtype="f32", rank=d)
+    lay, y, gate, rho = run_layer(x, P, Ws, 0.05, 2)
+    assert not gate.any()
+    ref = (x.to(torch.float64) @ Ws[0].to(torch.float64).T).numpy()
+    assert np.max(np.abs(y - ref)) <= 1e-2 * np.max(np.abs(ref))
+
+
+def test_zero_and_nonfinite_tokens_take_the_slow_path():
+    x, P, Ws = make_small(256, 32, (64,), 4, seed=41)
+    x[1] = 0.0
+    x[2, 7] = float("nan")
+    lay, y, gate, rho = run_layer(x, P, Ws, 0.5, 4)
+    assert gate[1] == 1 and gate[2] == 1
+    assert np.all(y[1] == 0.0)
+    assert np.isnan(y[2]).all()
+    keep = [0, 3]
+    compare_group(x[keep], P, Ws, 0.5, y[keep], gate[keep], rho[keep])
+
+
+def test_static_projection_flag_never_adds_the_residual():
+    g = G()
+    x, P, Ws = make_small(512, 64, (128,), 6, seed=51, noise=0.2)
+    lay, y, gate, rho = run_layer(x, P, Ws, 0.05, 3, flags=g.GSI_FLAG_STATIC_PROJECTION)
+    assert gate.all()                      # the gate is still reported
+    compare_group(x, P, Ws, 0.05, y, gate, rho, static=True)
+
+
+def test_dense_baseline_flag():
+    g = G()
+    x, P, Ws = make_small(1024, 64, (256, 64), 5, seed=61)
+    lay, y, gate, rho = run_layer(x, None, Ws, 0.0, 2, flags=g.GSI_FLAG_DENSE)
+    assert gate.all()
+    ref = torch.cat([x.to(torch.float64) @ W.to(torch.float64).T for W in Ws], dim=1).numpy()
+    assert np.max(np.abs(y - ref)) <= 1e-5 * np.max(np.abs(ref))
+
+
+def test_build_image_entry_point_matches_bf16_of_fp64_product():
+    g = G()
+    for p_dtype in ("bf16", "f32"):
+        q = S.gen_basis(520, 72, 71)
+        P = S.store_basis(q, p_dtype)
+        W = S.gen_weight(200, 520, 72)
+        wp = g.gsi_build_image(W.cuda(), P.cuda())
+        torch.cuda.synchronize()
+        image_ulp_check(W, P, wp.cpu())
+
+
+def test_forward_host_variant():
+    x, P, Ws = make_small(768, 64, (3072,), 4, seed=81, outlier_every=2)
+    g = G()
+    lay = g.Layer([W.cuda() for W in Ws], P.cuda(), 0.05, max_tokens=4)
+    y, gate, rho = lay.forward_host(x.pin_memory())
+    compare_group(x, P, Ws, 0.05, y.numpy(), gate.numpy(), rho.numpy())
+    yd, gd, rd = lay.forward(x.cuda())
+    assert torch.equal(yd.cpu(), y) and torch.equal(gd.cpu(), gate)
+
+
+def build_stack(st, n_layers, n_steps, device="cuda", flags=0):
+    g = G()
+    layers, xs, mats = [], [], []
+    for layer in range(n_layers):
+        for gi, spec in enumerate(st.groups):
+            m = S.materialize_group(st, layer, gi, n_steps * st.batch)
+            lay = g.Layer([W.to(device) for W in m["W"]], m["P"].to(device), st.eps,
+                          max_tokens=st.batch, flags=flags)
+            layers.append(lay)
+            xs.append(m["x"].to(device).contiguous())
+            mats.append(m)
+    stack = g.Stack(layers)
+    stack.bind(xs, n_steps=n_steps)
+    return stack, mats
+
+
+def test_stack_config2_two_layers_step_by_step_and_graph_replay():
+    st = S.config2()
+    n_layers, n_steps = 2, 6
+    stack, mats = build_stack(st, n_layers, n_steps)
+    ys = [[] for _ in mats]
+    for s in range(n_steps):
+        stack.step()
+        torch.cuda.synchronize()
+        for i, y in enumerate(stack.ys):
+            ys[i].append(y.cpu().clone())
+    assert stack.status() == 0
+    gate_log = stack.gate_log.cpu().numpy()
+    rho_log = stack.rho_log.cpu().numpy()
+    for i, m in enumerate(mats):
+        y = torch.cat(ys[i]).numpy()
+        compare_group(m["x"], m["P"], m["W"], st.eps, y, gate_log[:, i, 0], rho_log[:, i, 0])
+    # the same steps replayed from one captured graph give the same logs
+    stack.gate_log.zero_()
+    stack.seek(0)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        stack.step(stream)            # warm-up outside capture
+        stack.seek(0, stream)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            stack.step(stream)
+        for _ in range(n_steps):
+            graph.replay()
+    torch.cuda.synchronize()
+    assert np.array_equal(stack.gate_log.cpu().numpy(), gate_log)
+    for i, y in enumerate(stack.ys):
+        assert torch.equal(y.cpu(), ys[i][-1])
+
+
+def test_stack_step_host_matches_device_step():
+    st = S.config2()
+    stack, mats = build_stack(st, 1, 2)
+    stack.step()
+    torch.cuda.synchronize()
+    ref = [y.cpu().clone() for y in stack.ys]
+    gate_ref = stack.gate_log[0].cpu().clone()
+    xs_host = [m["x"][:st.batch].contiguous().pin_memory() for m in mats]
+    ys_host = [torch.empty_like(r).pin_memory() for r in ref]
+    gate_host = torch.empty((len(mats), st.batch), dtype=torch.uint8).pin_memory()
+    stack.step_host(xs_host, ys_host, gate_host)
+    for a, b in zip(ref, ys_host):
+        assert torch.equal(a, b)
+    assert torch.equal(gate_ref, gate_host)
+
+
+def test_gptj_layer_full_size_sampled_rows():
+    """One GPT-J-shaped layer at full size (k=256, eps=0.05), batch 1, in the
+    launch configuration the benchmark uses; the oracle evaluates a sample of
+    the output rows of every map."""
+    st = S.config3("10")
+    n_steps = 24
+    g = G()
+    rng = np.random.default_rng(0)
+    for gi, spec in enumerate(st.groups):
+        m = S.materialize_group(st, 0, gi, n_steps, device="cuda")
+        lay = g.Layer(m["W"], m["P"], st.eps, max_tokens=1)
+        ys, gates, rhos = [], [], []
+        for s in range(n_steps):
+            y, gate, rho = lay.forward(m["x"][s:s + 1].contiguous())
+            ys.append(y)
+            gates.append(gate)
+            rhos.append(rho)
+        torch.cuda.synchronize()
+        y = torch.cat(ys).cpu().numpy()
+        rows, Wsamp, cols, off = [], [], [], 0
+        for W in m["W"]:
+            r = np.sort(rng.choice(W.shape[0], 48, replace=False))
+            rows.append(r)
+            Wsamp.append(W[torch.as_tensor(r, device="cuda")].cpu())
+            cols.append(off + r)
+            off += W.shape[0]
+        ysamp = y[:, np.concatenate(cols)]
+        res = compare_group(m["x"].cpu(), m["P"].cpu(), Wsamp, st.eps, ysamp,
+                            torch.cat(gates).cpu().numpy(), torch.cat(rhos).cpu().numpy())
+        assert res["gate_rate"] < 0.6
