@@ -1,0 +1,391 @@
+#!/usr/bin/env python
+"""Benchmark of the gated subspace decode step on B200.
+
+One "step" is one decode step of the whole stack: every group of every layer
+(projection, gate, image GEMV, gated residual) on one batch of synthetic
+activations.  At N=1 the workload is the GPT-J-6B-shaped stack (28 layers,
+k=256, eps=0.05, batch 1, ~10 % of tokens gated).  With N>1 every rank runs an
+independent replica (the path does not shard; no collective on the data path).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference]
+
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "decode tokens/s at GPT-J shapes, k=256, eps=0.05 (effective weight GB/s and % of HBM roofline alongside)"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+
+def measured_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return json.load(open(p)), "measured"
+        except Exception:
+            pass
+    return {"hbm_gbs": FALLBACK_HBM_GBS}, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while a region runs."""
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.index = index
+        self.rows = []
+        self.proc = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 7:
+                self.rows.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0]))
+                mx.append(float(r[1]))
+            except ValueError:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------
+def build_workload(spec, device, n_steps):
+    """Draw the whole stack on the device.  Returns (gsi layers, dense layers,
+    x tensors per group, host-side copies needed later)."""
+    import torch
+    import synthetic as S
+    import paper_2605_03109_b200 as G
+    layers, dense, xs, keep = [], [], [], []
+    for layer in range(spec.n_layers):
+        for gi, g in enumerate(spec.groups):
+            m = S.materialize_group(spec, layer, gi, n_steps * spec.batch, device=device)
+            lay = G.Layer(m["W"], m["P"], spec.eps, max_tokens=spec.batch)
+            den = G.Layer(m["W"], None, 0.0, max_tokens=spec.batch, flags=G.GSI_FLAG_DENSE)
+            layers.append(lay)
+            dense.append(den)
+            xs.append(m["x"].contiguous())
+            keep.append((m["W"], m["P"]))
+            del m
+    torch.cuda.synchronize()
+    return layers, dense, xs, keep
+
+
+def capture_step(stack, stream):
+    import torch
+    with torch.cuda.stream(stream):
+        stack.step(stream)
+        stream.synchronize()
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            stack.step(stream)
+    return graph
+
+
+def time_graph(graph, stack, stream, steps, warmup, barrier=None):
+    import torch
+    with torch.cuda.stream(stream):
+        stack.seek(0, stream)
+        for _ in range(warmup):
+            graph.replay()
+        stream.synchronize()
+        stack.seek(0, stream)
+        if barrier:
+            barrier()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            graph.replay()
+        e1.record(stream)
+        stream.synchronize()
+        torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps  # ms per step
+
+
+def time_host_steps(stack, xs, steps, warmup, stream):
+    """End-to-end: host buffers in, host buffers out, copies inside the timed region."""
+    import torch
+    n = len(stack.layers)
+    B = stack.B
+    xs_host = [x[:B].reshape(B, -1).cpu().contiguous().pin_memory() for x in xs]
+    ys_host = [torch.empty((B, l.O), dtype=torch.float32).pin_memory() for l in stack.layers]
+    gate_host = torch.empty((n, B), dtype=torch.uint8).pin_memory()
+    h2d = sum(x.numel() * 4 for x in xs_host)
+    d2h = sum(y.numel() * 4 for y in ys_host) + gate_host.numel()
+    with torch.cuda.stream(stream):
+        for _ in range(max(1, warmup)):
+            stack.step_host(xs_host, ys_host, gate_host, stream)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(steps):
+            stack.step_host(xs_host, ys_host, gate_host, stream)
+        e1.record(stream)
+        stream.synchronize()
+        wall = (time.perf_counter() - t0) * 1e3 / steps
+    ms = max(e0.elapsed_time(e1) / steps, wall)
+    return ms, h2d, d2h
+
+
+def algorithmic_bytes(spec, fired_per_group_step):
+    """bytes(P) + bytes(W_P) + fired*bytes(W) + activations, per step, from the
+    REALISED fired indicator (any token of the batch gated -> W streamed once)."""
+    ng = len(spec.groups)
+    wbytes = spec.bytes_w_per_group()
+    fast = spec.bytes_fast_per_step()
+    act = spec.bytes_act_per_token() * spec.batch
+    w = 0.0
+    for gi in range(ng):
+        # fired_per_group_step: [steps][n_groups] bool
+        w += float(fired_per_group_step[:, gi::ng].sum()) * wbytes[gi]
+    steps = fired_per_group_step.shape[0]
+    w_per_step = w / steps
+    return dict(fast=fast, w=w_per_step, act=act, total=fast + w_per_step + act,
+                weight_only=fast + w_per_step,
+                dense=sum(wbytes) * spec.n_layers + act)
+
+
+def oracle_sample_rate(spec, n_tokens=4, row_frac=8, threads=None):
+    """Time the oracle, as it stands, on a bounded sample of the workload: the
+    three groups of ONE layer, n_tokens tokens, 1/row_frac of the output rows of
+    every map (images of the sampled rows precomputed, untimed, as the method
+    caches them).  Scaled to whole-stack tokens/s."""
+    import numpy as np
+    import synthetic as S
+    from oracle import gsi_oracle as O
+    if threads:
+        O.set_threads(threads)
+    t_proj = t_map = 0.0
+    for gi, g in enumerate(spec.groups):
+        m = S.materialize_group(spec, 0, gi, n_tokens, device="cpu")
+        x = m["x"].numpy()
+        P = S.bits_of(m["P"])
+        Ws = [S.to_bf16_bits(W)[:: row_frac].copy() for W in m["W"]]
+        Ms = [O.image(W, P) for W in Ws]
+        t0 = time.perf_counter()
+        pr = O.project(x, P, spec.eps)
+        t1 = time.perf_counter()
+        for W, M in zip(Ws, Ms):
+            O.apply_map(M, W, pr["g"], pr["r"], pr["gate"])
+        t2 = time.perf_counter()
+        t_proj += t1 - t0
+        t_map += t2 - t1
+    per_token_layer = (t_proj + row_frac * t_map) / n_tokens
+    tok_s = 1.0 / (per_token_layer * spec.n_layers)
+    sample = (f"1 of {spec.n_layers} layers, {n_tokens} tokens, every {row_frac}th output row of "
+              f"each map (map time scaled x{row_frac}), images precomputed; "
+              f"measured {t_proj + t_map:.1f} s of oracle work")
+    return tok_s, O.num_threads(), sample
+
+
+def run_reference(args, spec):
+    """The reference arm is the oracle timed on the host cores."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    vals = []
+    sample = ""
+    cores = 1
+    for i in range(args.warmup + args.steps):
+        v, cores, sample = oracle_sample_rate(spec, n_tokens=2, row_frac=16)
+        if i >= args.warmup:
+            vals.append(v)
+    v = statistics.median(vals)
+    out = {
+        "impl": "reference", "metric": METRIC, "value": v, "unit": "tokens/s",
+        "n_gpus": args.gpus, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": 1e3 / v, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": spec.name, "batch": spec.batch, "k": spec.groups[0].k,
+                   "eps": spec.eps},
+        "cpu_baseline": {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": v, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }
+    print(json.dumps(out))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=256)
+    ap.add_argument("--warmup", type=int, default=16)
+    ap.add_argument("--impl", default="gsi", choices=["gsi", "reference"])
+    ap.add_argument("--gate", default="10", choices=["0", "10", "23", "100"],
+                    help="target gate rate of the GPT-J workload (percent)")
+    ap.add_argument("--workload", default="gptj", choices=["gptj", "gpt2"])
+    ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "gsi" else args.warmup
+
+    import synthetic as S
+    from dataclasses import replace
+    spec = S.config3(args.gate) if args.workload == "gptj" else S.config2()
+    if args.layers:
+        spec = replace(spec, n_layers=args.layers, name=f"{spec.name}_L{args.layers}")
+
+    if args.impl == "reference":
+        run_reference(args, spec)
+        return
+
+    import numpy as np
+    import torch
+    import paper_2605_03109_b200 as G
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the gated subspace layer has no CPU path")
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=device)
+
+    n_steps = min(spec.steps, max(args.steps, 1))
+    layers, dense_layers, xs, keep = build_workload(spec, device, n_steps)
+    stack = G.Stack(layers)
+    stack.bind(xs, n_steps=n_steps)
+    dstack = G.Stack(dense_layers)
+    dstack.bind(xs, n_steps=n_steps, want_rho=False)
+    stream = torch.cuda.Stream(device)
+    graph = capture_step(stack, stream)
+    dgraph = capture_step(dstack, stream)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    ms = time_graph(graph, stack, stream, args.steps, args.warmup, barrier)
+    clocks = sampler.stop()
+    ms_dense = time_graph(dgraph, dstack, stream, max(8, args.steps // 8), 3)
+    gate_log = stack.gate_log.cpu().numpy()          # [n_steps][groups][B]
+    used_steps = min(args.steps, n_steps)
+    fired = gate_log[:used_steps].any(axis=2)        # [steps][groups]
+    status = stack.status()
+    if status != 0:
+        raise SystemExit(f"device status word {status}: {G.gsi_status_string(status)}")
+
+    e2e = None
+    if not args.no_e2e:
+        ms_e2e, h2d, d2h = time_host_steps(stack, xs, max(8, args.steps // 8), 3, stream)
+        e2e = {"value": world * spec.batch * 1e3 / ms_e2e, "unit": "tokens/s",
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
+
+    t = torch.tensor([ms], dtype=torch.float64, device=device)
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_max = float(t.item())
+
+    if rank == 0:
+        peaks, peak_kind = measured_peaks()
+        ab = algorithmic_bytes(spec, fired)
+        sec = ms_max * 1e-3
+        achieved = ab["total"] / sec / 1e9
+        peak = float(peaks["hbm_gbs"])
+        launches = stack.launches_per_step()
+        out = {
+            "metric": METRIC,
+            "value": world * spec.batch / sec,
+            "unit": "tokens/s",
+            "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_max, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {
+                "workload": spec.name, "layers": spec.n_layers,
+                "groups_per_layer": [f"{g.name}:{g.d}->{'+'.join(map(str, g.d_out))}" for g in spec.groups],
+                "k": spec.groups[0].k, "eps": spec.eps, "batch": spec.batch,
+                "weights": "bf16", "basis": spec.groups[0].p_dtype, "activations": "f32",
+                "distinct_input_steps": n_steps,
+                "l2": "inputs_larger_than_l2 (0.88 GB of basis+image per step, distinct per layer)",
+                "replicas": world, "timing": "one CUDA graph per step, CUDA events on the launch stream",
+            },
+            "gate_rate": float(gate_log[:used_steps].mean()),
+            "fired_groups_per_step": float(fired.sum(axis=1).mean()),
+            "effective_weight_gbs": ab["weight_only"] / sec / 1e9,
+            "bytes_per_step": {k: float(v) for k, v in ab.items()},
+            "roofline": {
+                "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": None,
+                "kernel": "whole decode step (all launches of one graph replay)",
+                "peak_source": f"{peak_kind} copy bandwidth",
+                "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
+            },
+            "dense_baseline": {
+                "ms_per_step": ms_dense, "tokens_per_s": spec.batch * 1e3 / ms_dense,
+                "achieved_gbs": ab["dense"] / (ms_dense * 1e-3) / 1e9,
+                "frac_of_peak": ab["dense"] / (ms_dense * 1e-3) / 1e9 / peak,
+                "speedup_of_gsi": ms_dense / ms_max,
+            },
+            "paper_context": "paper quotes 3.0-10.5x effective speed-up on weight reads (MI300X, computed from gate statistics, not measured)",
+            "clocks": clocks,
+            "gpu_launches": launches * args.steps,
+            "launches_per_step": launches,
+        }
+        if e2e:
+            out["e2e"] = e2e
+        if not args.no_cpu_baseline and world == 1:
+            v, cores, sample = oracle_sample_rate(spec)
+            out["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": cores,
+                                   "kind": "oracle", "sample": sample}
+        print(json.dumps(out))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

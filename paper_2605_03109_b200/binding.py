@@ -150,6 +150,7 @@ class Layer:
         self.max_tokens = int(max_tokens)
         self.eps = float(eps)
         self.flags = int(flags)
+        assert P is None or (P.is_contiguous() and P.device == dev and tuple(P.shape) == (self.d, self.k))
         self._Ws, self._P = Ws, P
         pd = GSI_BF16 if P is None else _dtype_code(P)
         self._desc = make_desc(self.d, self.k, self.d_out, eps, max_tokens, pd, flags)

@@ -48,7 +48,7 @@ def gen_basis(d: int, k: int, seed: int, device="cpu") -> torch.Tensor:
     q, r = torch.linalg.qr(a, mode="reduced")
     sign = torch.sign(torch.diagonal(r))
     sign[sign == 0] = 1.0
-    return q * sign
+    return (q * sign).contiguous()   # LAPACK hands back column-major strides
 
 
 def gen_true_basis(q: torch.Tensor, rank: int, s: int, seed: int) -> torch.Tensor:
@@ -56,7 +56,7 @@ def gen_true_basis(q: torch.Tensor, rank: int, s: int, seed: int) -> torch.Tenso
     d, k = q.shape
     assert 0 <= s <= min(rank, k) and rank <= d
     if s == rank:
-        return q[:, :s].clone()
+        return q[:, :s].contiguous()
     extra = torch.empty((d, rank - s), dtype=torch.float64, device=q.device)
     extra.normal_(0.0, 1.0, generator=_gen(seed, q.device))
     # two sweeps of projection out of span(q), then orthonormalise among themselves
@@ -66,7 +66,7 @@ def gen_true_basis(q: torch.Tensor, rank: int, s: int, seed: int) -> torch.Tenso
     for _ in range(2):
         e = e - q @ (q.T @ e)
         e, _ = torch.linalg.qr(e, mode="reduced")
-    return torch.cat([q[:, :s], e], dim=1)
+    return torch.cat([q[:, :s], e], dim=1).contiguous()
 
 
 def gen_activations(p_true: torch.Tensor, n_tokens: int, sigma: float, p_outlier: float,
@@ -93,7 +93,8 @@ def gen_activations(p_true: torch.Tensor, n_tokens: int, sigma: float, p_outlier
 
 def store_basis(q: torch.Tensor, dtype: str = "bf16") -> torch.Tensor:
     """Round the fp64 basis to its storage type."""
-    return q.to(torch.bfloat16) if dtype == "bf16" else q.to(torch.float32)
+    q = q.contiguous()
+    return (q.to(torch.bfloat16) if dtype == "bf16" else q.to(torch.float32)).contiguous()
 
 
 def to_bf16_bits(t: torch.Tensor) -> np.ndarray:
