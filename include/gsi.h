@@ -186,6 +186,20 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io_host_array,
                             int n_steps, unsigned char* gate_log, float* rho_log,
                             gsi_stream_t stream);
 
+/*
+ * Execution mode, taken at the next gsi_stack_bind:
+ *   0 (default)  one persistent launch per step when every group qualifies
+ *                (batch 1, bf16 basis with k a power of two <= 512, d a
+ *                multiple of 16, 32-byte aligned W), else the per-stage kernels;
+ *   1            always the per-stage kernels;
+ *   2            the persistent launch or GSI_ERR_UNSUPPORTED from bind.
+ * Both modes compute the same layer; they differ in reduction order only.
+ */
+gsi_status_t gsi_stack_set_mode(gsi_stack_t s, int mode);
+
+/* 1 if the bound stack runs as one persistent launch per step. */
+gsi_status_t gsi_stack_is_persistent(gsi_stack_t s, int* out);
+
 /* Set the device-side step counter (enqueued on `stream`). */
 gsi_status_t gsi_stack_seek(gsi_stack_t s, int step, gsi_stream_t stream);
 

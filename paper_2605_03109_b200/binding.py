@@ -21,7 +21,7 @@ EXPORTED = [
     "gsi_status_string", "gsi_build_image", "gsi_workspace_bytes", "gsi_create",
     "gsi_forward", "gsi_forward_n", "gsi_forward_host", "gsi_get_image", "gsi_get_status",
     "gsi_destroy", "gsi_stack_workspace_bytes", "gsi_stack_create", "gsi_stack_bind",
-    "gsi_stack_seek", "gsi_stack_step", "gsi_stack_launches_per_step",
+    "gsi_stack_set_mode", "gsi_stack_is_persistent", "gsi_stack_seek", "gsi_stack_step", "gsi_stack_launches_per_step",
     "gsi_stack_step_host", "gsi_stack_get_status", "gsi_stack_destroy",
 ]
 
@@ -47,9 +47,7 @@ def lib_path() -> str:
 
 
 def _load():
-    path = _build.LIB
-    if not os.path.exists(path):
-        path = _build.build()
+    path = _build.build()   # no-op when the library matches the sources
     l = C.CDLL(path)
     vp, i, sz = C.c_void_p, C.c_int, C.c_size_t
     l.gsi_status_string.restype = C.c_char_p
@@ -68,6 +66,8 @@ def _load():
     l.gsi_stack_workspace_bytes.argtypes = [i]
     l.gsi_stack_create.argtypes = [i, C.POINTER(vp), vp, sz, vp, C.POINTER(vp)]
     l.gsi_stack_bind.argtypes = [vp, C.POINTER(GsiStackIo), i, vp, vp, vp]
+    l.gsi_stack_set_mode.argtypes = [vp, i]
+    l.gsi_stack_is_persistent.argtypes = [vp, C.POINTER(i)]
     l.gsi_stack_seek.argtypes = [vp, i, vp]
     l.gsi_stack_step.argtypes = [vp, vp]
     l.gsi_stack_launches_per_step.argtypes = [vp, C.POINTER(i)]
@@ -220,8 +220,9 @@ class Layer:
 class Stack:
     """An ordered chain of groups stepped as one decode step."""
 
-    def __init__(self, layers, stream=None):
+    def __init__(self, layers, stream=None, mode: int = 0):
         self.layers = list(layers)
+        self._mode = int(mode)
         n = len(self.layers)
         dev = self.layers[0].device
         self.B = self.layers[0].max_tokens
@@ -233,6 +234,13 @@ class Stack:
                                     _stream_ptr(stream), C.byref(h)), "gsi_stack_create")
         self.handle = h
         self.device = dev
+        if self._mode:
+            _check(lib.gsi_stack_set_mode(self.handle, self._mode), "gsi_stack_set_mode")
+
+    def is_persistent(self) -> bool:
+        v = C.c_int()
+        _check(lib.gsi_stack_is_persistent(self.handle, C.byref(v)), "gsi_stack_is_persistent")
+        return bool(v.value)
 
     def bind(self, xs, ys=None, n_steps: int = 1, want_rho: bool = True, stream=None):
         """xs[g]: [n_steps][B][d] fp32 device tensors.  Allocates y and the logs."""

@@ -5,6 +5,7 @@
 #include <cstring>
 
 #include "gsi_common.cuh"
+#include "gsi_persistent.cuh"
 
 using namespace gsi;
 
@@ -17,7 +18,8 @@ inline size_t align_up(size_t v) { return (v + kAlign - 1) / kAlign * kAlign; }
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 struct Layout {
-  size_t wp, c, cpart, r, normpart, ctrl, fired, rho, x_stage, y_stage, gate_stage, rho_stage, total;
+  size_t wp, c, cpart, r, normpart, ctrl, fired, rho, x_stage, y_stage, gate_stage, rho_stage,
+      pk_acc, pk_slot, total;
   int O, n_slabs, slab_rows;
 };
 
@@ -64,6 +66,8 @@ Layout make_layout_ws(const gsi_desc_t* d) {
   L.y_stage = take(B * (size_t)O * 4);
   L.gate_stage = take(B);
   L.rho_stage = take(B * 4);
+  L.pk_acc = take(2 * k * 8);                       // persistent kernel: c accumulators
+  L.pk_slot = take((size_t)kPersistMaxGrid * 8);    // persistent kernel: ||r||^2 words
   L.total = at;
   return L;
 }
@@ -76,10 +80,19 @@ struct gsi_layer {
   Layout lay;
   GroupParams gp;
   char* ws;
+  float* pmax;     // device: max |P| (bf16 basis only)
+  unsigned* bar;   // device: [2] barrier counters of the persistent kernel
   cudaStream_t last_stream;
 };
 
 struct gsi_stack {
+  int mode;                 // 0 auto, 1 generic kernels, 2 persistent kernel required
+  bool persistent;          // the persistent kernel is in use
+  int grid;                 // CTAs of the persistent kernel (= SMs)
+  PersistGroup* dev_groups; // device table
+  std::vector<PersistGroup> host_groups;
+  int* epoch;               // device
+  int* status;              // device
   std::vector<gsi_layer*> groups;
   std::vector<gsi_stack_io_t> io;
   int B;
@@ -88,6 +101,7 @@ struct gsi_stack {
   float* rho_log;
   int* step;  // device
   bool bound;
+  int seek_value;
   cudaStream_t last_stream;
 };
 
@@ -180,7 +194,15 @@ gsi_status_t gsi_create(const gsi_desc_t* desc, const void* const* W, const void
   g.n_slabs = L.n_slabs;
   g.slab_rows = L.slab_rows;
 
-  if (cudaMemsetAsync(ctrl, 0, 256, stream) != cudaSuccess) {
+  if (cudaMemsetAsync(ctrl, 0, 256, stream) != cudaSuccess ||
+      cudaMemsetAsync(h->ws + L.pk_acc, 0, L.total - L.pk_acc, stream) != cudaSuccess) {
+    delete h;
+    return GSI_ERR_CUDA;
+  }
+  h->pmax = reinterpret_cast<float*>(ctrl + 8);
+  h->bar = reinterpret_cast<unsigned*>(ctrl + 16);
+  if (!dense && !g.p_f32 &&
+      launch_abs_max_bf16(P, (size_t)desc->d * desc->k, h->pmax, stream) != cudaSuccess) {
     delete h;
     return GSI_ERR_CUDA;
   }
@@ -272,6 +294,7 @@ gsi_status_t gsi_destroy(gsi_handle_t h) {
 // ------------------------------------------------------------------ stack
 size_t gsi_stack_workspace_bytes(int n_groups) {
   if (n_groups <= 0) return 0;
+  static_assert(sizeof(PersistGroup) <= 512, "group descriptor outgrew its slot");
   return align_up(256) + align_up((size_t)n_groups * 512);
 }
 
@@ -295,6 +318,12 @@ gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* wo
   s->gate_log = nullptr;
   s->rho_log = nullptr;
   s->step = static_cast<int*>(workspace);
+  s->epoch = s->step + 1;
+  s->status = s->step + 2;
+  s->dev_groups = reinterpret_cast<PersistGroup*>(static_cast<char*>(workspace) + 256);
+  s->mode = 0;
+  s->persistent = false;
+  s->grid = 0;
   s->bound = false;
   s->last_stream = stream;
   if (cudaMemsetAsync(workspace, 0, 256, stream) != cudaSuccess) {
@@ -305,35 +334,119 @@ gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* wo
   return GSI_OK;
 }
 
+// Can this stack run as one persistent launch?  (batch 1, bf16 basis with a
+// power-of-two rank up to 512, rows that fit the per-CTA buffers, 32-byte
+// aligned weight rows for the 256-bit loads.)
+static bool persistent_eligible(const gsi_stack* s, int grid) {
+  if (s->B != 1 || grid <= 0 || grid > kPersistMaxGrid) return false;
+  for (const gsi_layer* h : s->groups) {
+    const gsi_desc_t& d = h->desc;
+    const bool dense = d.flags & GSI_FLAG_DENSE;
+    if (d.d % 16) return false;
+    if ((d.d + grid - 1) / grid > kPersistMaxPRows) return false;
+    if ((h->lay.O + grid - 1) / grid > kPersistMaxORows) return false;
+    for (int j = 0; j < d.n_maps; ++j)
+      if (reinterpret_cast<uintptr_t>(h->gp.W[j]) & 31u) return false;
+    if (!dense) {
+      if (d.p_dtype != GSI_BF16) return false;
+      if (d.k < 8 || d.k > 512 || (d.k & (d.k - 1))) return false;
+    }
+  }
+  return true;
+}
+
+gsi_status_t gsi_stack_set_mode(gsi_stack_t s, int mode) {
+  if (!s || mode < 0 || mode > 2) return GSI_ERR_INVALID_ARG;
+  s->mode = mode;
+  s->bound = false;  // the choice is taken at bind time
+  return GSI_OK;
+}
+
 gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps,
                             unsigned char* gate_log, float* rho_log, gsi_stream_t stream) {
   if (!s || !io || n_steps <= 0 || !gate_log) return GSI_ERR_INVALID_ARG;
-  for (size_t i = 0; i < s->groups.size(); ++i)
+  const int G = (int)s->groups.size();
+  for (int i = 0; i < G; ++i)
     if (!io[i].x || !io[i].y || !aligned16(io[i].x) || !aligned16(io[i].y))
       return GSI_ERR_INVALID_ARG;
-  std::copy(io, io + s->groups.size(), s->io.begin());
+  std::copy(io, io + G, s->io.begin());
   s->n_steps = n_steps;
   s->gate_log = gate_log;
   s->rho_log = rho_log;
-  s->bound = true;
   s->last_stream = stream;
+
+  s->persistent = false;
+  if (s->mode != 1) {
+    int dev = 0, sms = 0, coop = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess ||
+        cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, dev) != cudaSuccess)
+      return GSI_ERR_CUDA;
+    s->grid = sms;
+    s->persistent = coop && persistent_eligible(s, sms);
+    if (s->mode == 2 && !s->persistent) return GSI_ERR_UNSUPPORTED;
+  }
+  if (s->persistent) {
+    s->host_groups.assign(G, PersistGroup{});
+    for (int i = 0; i < G; ++i) {
+      const gsi_layer* h = s->groups[i];
+      PersistGroup& pg = s->host_groups[i];
+      const GroupParams& gp = h->gp;
+      pg.P = static_cast<const uint16_t*>(gp.P);
+      pg.WP = gp.WP;
+      for (int j = 0; j < gp.n_maps; ++j) pg.W[j] = gp.W[j];
+      for (int j = 0; j <= gp.n_maps; ++j) pg.off[j] = gp.off[j];
+      pg.n_maps = gp.n_maps;
+      pg.d = gp.d;
+      pg.k = gp.k;
+      pg.O = gp.O;
+      pg.eps = gp.eps;
+      pg.flags = gp.flags;
+      pg.pmax = h->pmax;
+      pg.x = io[i].x;
+      pg.y = io[i].y;
+      pg.r = gp.r;
+      pg.acc_c = reinterpret_cast<unsigned long long*>(h->ws + h->lay.pk_acc);
+      pg.slot_r = reinterpret_cast<unsigned long long*>(h->ws + h->lay.pk_slot);
+      pg.bar = h->bar;
+      pg.p_rows = (gp.d + s->grid - 1) / s->grid;
+      pg.o_rows = (gp.O + s->grid - 1) / s->grid;
+      pg.x_step_stride = gp.d;
+    }
+    if (cudaMemcpyAsync(s->dev_groups, s->host_groups.data(), sizeof(PersistGroup) * G,
+                        cudaMemcpyHostToDevice, stream) != cudaSuccess)
+      return GSI_ERR_CUDA;
+  }
+  s->bound = true;
   return GSI_OK;
 }
 
 gsi_status_t gsi_stack_seek(gsi_stack_t s, int step, gsi_stream_t stream) {
   if (!s || step < 0) return GSI_ERR_INVALID_ARG;
-  // 4-byte pattern set is not available through cudaMemsetAsync; stage via a
-  // pageable copy, which the runtime completes before returning.
   s->last_stream = stream;
-  return cudaMemcpyAsync(s->step, &step, sizeof(int), cudaMemcpyHostToDevice, stream) ==
+  s->seek_value = step;  // pageable source: staged by the runtime before the call returns
+  return cudaMemcpyAsync(s->step, &s->seek_value, sizeof(int), cudaMemcpyHostToDevice, stream) ==
                  cudaSuccess
              ? GSI_OK
              : GSI_ERR_CUDA;
 }
 
-static gsi_status_t stack_enqueue(gsi_stack_t s, bool use_counter, gsi_stream_t stream,
-                                  int* n_launches) {
+static gsi_status_t stack_enqueue(gsi_stack_t s, bool use_counter, gsi_stream_t stream) {
   const int G = (int)s->groups.size();
+  if (s->persistent) {
+    PersistParams p{};
+    p.groups = s->dev_groups;
+    p.n_groups = G;
+    p.step = s->step;
+    p.epoch = s->epoch;
+    p.n_steps = s->n_steps;
+    p.use_counter = use_counter ? 1 : 0;
+    p.gate_log = s->gate_log;
+    p.rho_log = s->rho_log;
+    p.log_step_stride = G;
+    p.status = s->status;
+    return launch_decode_step(p, s->grid, stream) == cudaSuccess ? GSI_OK : GSI_ERR_CUDA;
+  }
   for (int i = 0; i < G; ++i) {
     gsi_layer* h = s->groups[i];
     IoRef io{};
@@ -346,24 +459,25 @@ static gsi_status_t stack_enqueue(gsi_stack_t s, bool use_counter, gsi_stream_t 
     io.x_step_stride = (long long)s->B * h->desc.d;
     io.log_step_stride = (long long)G * s->B;
     h->last_stream = stream;
-    if (launch_generic_forward(h->gp, io, s->B, stream, n_launches) != cudaSuccess)
+    if (launch_generic_forward(h->gp, io, s->B, stream, nullptr) != cudaSuccess)
       return GSI_ERR_CUDA;
   }
-  if (use_counter) {
-    if (launch_advance_step(s->step, stream) != cudaSuccess) return GSI_ERR_CUDA;
-    if (n_launches) *n_launches += 1;
-  }
+  if (use_counter && launch_advance_step(s->step, stream) != cudaSuccess) return GSI_ERR_CUDA;
   return GSI_OK;
 }
 
 gsi_status_t gsi_stack_step(gsi_stack_t s, gsi_stream_t stream) {
   if (!s || !s->bound) return GSI_ERR_INVALID_ARG;
   s->last_stream = stream;
-  return stack_enqueue(s, true, stream, nullptr);
+  return stack_enqueue(s, true, stream);
 }
 
 gsi_status_t gsi_stack_launches_per_step(gsi_stack_t s, int* n_out) {
-  if (!s || !n_out) return GSI_ERR_INVALID_ARG;
+  if (!s || !n_out || !s->bound) return GSI_ERR_INVALID_ARG;
+  if (s->persistent) {
+    *n_out = 1;
+    return GSI_OK;
+  }
   int n = 0;
   for (gsi_layer* h : s->groups) {
     if (h->desc.flags & GSI_FLAG_DENSE) n += 1;
@@ -385,7 +499,7 @@ gsi_status_t gsi_stack_step_host(gsi_stack_t s, const float* const* x_host, floa
       return GSI_ERR_CUDA;
   }
   s->last_stream = stream;
-  gsi_status_t st = stack_enqueue(s, false, stream, nullptr);
+  gsi_status_t st = stack_enqueue(s, false, stream);
   if (st != GSI_OK) return st;
   for (int i = 0; i < G; ++i) {
     const size_t bytes = (size_t)s->B * s->groups[i]->lay.O * 4;
@@ -399,10 +513,19 @@ gsi_status_t gsi_stack_step_host(gsi_stack_t s, const float* const* x_host, floa
   return cudaStreamSynchronize(stream) == cudaSuccess ? GSI_OK : GSI_ERR_CUDA;
 }
 
+gsi_status_t gsi_stack_is_persistent(gsi_stack_t s, int* out) {
+  if (!s || !out || !s->bound) return GSI_ERR_INVALID_ARG;
+  *out = s->persistent ? 1 : 0;
+  return GSI_OK;
+}
+
 gsi_status_t gsi_stack_get_status(gsi_stack_t s, int* device_status) {
   if (!s || !device_status) return GSI_ERR_INVALID_ARG;
   if (cudaStreamSynchronize(s->last_stream) != cudaSuccess) return GSI_ERR_CUDA;
   *device_status = 0;
+  if (cudaMemcpy(device_status, s->status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)
+    return GSI_ERR_CUDA;
+  if (*device_status) return GSI_OK;
   for (gsi_layer* h : s->groups) {
     int v = 0;
     if (cudaMemcpy(&v, h->gp.status, sizeof(int), cudaMemcpyDeviceToHost) != cudaSuccess)

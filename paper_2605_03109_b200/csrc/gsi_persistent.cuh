@@ -1,0 +1,51 @@
+// Descriptors of the persistent decode-step kernel (device-resident tables).
+#pragma once
+
+#include "gsi_common.cuh"
+
+namespace gsi {
+
+constexpr int kPersistConsumerWarps = 12;
+constexpr int kPersistMaxPRows = 128;   // basis rows one CTA may own
+constexpr int kPersistMaxORows = 512;   // output rows one CTA may own
+constexpr int kPersistMaxGrid = 256;    // CTAs (exchange-2 slots per group)
+
+struct PersistGroup {
+  const uint16_t* P;                 // [d][k] bf16
+  const uint16_t* WP;                // [O][k] bf16, images of all maps concatenated
+  const uint16_t* W[GSI_MAX_MAPS];   // [d_out_j][d] bf16
+  int off[GSI_MAX_MAPS + 1];
+  int n_maps;
+  int d, k, O;
+  float eps;
+  unsigned flags;
+  const float* pmax;                 // device scalar: max |P|
+  const float* x;                    // [n_steps][d]
+  float* y;                          // [O]
+  float* r;                          // [d]
+  unsigned long long* acc_c;         // [2][k] fixed-point accumulators, one set per launch parity
+  unsigned long long* slot_r;        // [kPersistMaxGrid] (launch tag | partial ||r||^2)
+  unsigned* bar;                     // [2] end-of-residual barrier counters
+  int p_rows, o_rows;                // rows per CTA of P and of the outputs
+  long long x_step_stride;
+};
+
+struct PersistParams {
+  const PersistGroup* groups;  // device
+  int n_groups;
+  int* step;                   // device: decode-step counter (selects the I/O slot)
+  int* epoch;                  // device: launches so far (parity of the exchange buffers)
+  int n_steps;
+  int use_counter;             // 0: I/O slot 0, counter not advanced
+  unsigned char* gate_log;     // [n_steps][n_groups]
+  float* rho_log;              // same shape or nullptr
+  int log_step_stride;
+  int* status;
+};
+
+int persist_smem_bytes();
+int persist_threads();
+cudaError_t launch_decode_step(const PersistParams& p, int grid, cudaStream_t st);
+cudaError_t launch_abs_max_bf16(const void* p, size_t n, float* out, cudaStream_t st);
+
+}  // namespace gsi

@@ -193,7 +193,7 @@ def test_forward_host_variant():
     assert torch.equal(yd.cpu(), y) and torch.equal(gd.cpu(), gate)
 
 
-def build_stack(st, n_layers, n_steps, device="cuda", flags=0):
+def build_stack(st, n_layers, n_steps, device="cuda", flags=0, mode=0):
     g = G()
     layers, xs, mats = [], [], []
     for layer in range(n_layers):
@@ -204,15 +204,19 @@ def build_stack(st, n_layers, n_steps, device="cuda", flags=0):
             layers.append(lay)
             xs.append(m["x"].to(device).contiguous())
             mats.append(m)
-    stack = g.Stack(layers)
+    stack = g.Stack(layers, mode=mode)
     stack.bind(xs, n_steps=n_steps)
     return stack, mats
 
 
-def test_stack_config2_two_layers_step_by_step_and_graph_replay():
+@pytest.mark.parametrize("mode", [1, 2])
+def test_stack_config2_two_layers_step_by_step_and_graph_replay(mode):
+    """mode 1: per-stage kernels; mode 2: one persistent launch per step."""
     st = S.config2()
     n_layers, n_steps = 2, 6
-    stack, mats = build_stack(st, n_layers, n_steps)
+    stack, mats = build_stack(st, n_layers, n_steps, mode=mode)
+    assert stack.is_persistent() == (mode == 2)
+    assert stack.launches_per_step() == (1 if mode == 2 else 5 * len(mats) + 1)
     ys = [[] for _ in mats]
     for s in range(n_steps):
         stack.step()
@@ -243,9 +247,10 @@ def test_stack_config2_two_layers_step_by_step_and_graph_replay():
         assert torch.equal(y.cpu(), ys[i][-1])
 
 
-def test_stack_step_host_matches_device_step():
+@pytest.mark.parametrize("mode", [1, 2])
+def test_stack_step_host_matches_device_step(mode):
     st = S.config2()
-    stack, mats = build_stack(st, 1, 2)
+    stack, mats = build_stack(st, 1, 2, mode=mode)
     stack.step()
     torch.cuda.synchronize()
     ref = [y.cpu().clone() for y in stack.ys]
@@ -289,3 +294,133 @@ def test_gptj_layer_full_size_sampled_rows():
         res = compare_group(m["x"].cpu(), m["P"].cpu(), Wsamp, st.eps, ysamp,
                             torch.cat(gates).cpu().numpy(), torch.cat(rhos).cpu().numpy())
         assert res["gate_rate"] < 0.6
+
+
+def _stack_against_oracle(st, n_layers, n_steps, mode, sample_rows=0, device="cuda"):
+    """Run n_steps decode steps and compare every group with the oracle (on a
+    sample of output rows when the maps are large)."""
+    g = G()
+    rng = np.random.default_rng(1)
+    layers, xs, mats = [], [], []
+    for layer in range(n_layers):
+        for gi, spec in enumerate(st.groups):
+            m = S.materialize_group(st, layer, gi, n_steps, device=device)
+            layers.append(g.Layer(m["W"], m["P"], st.eps, max_tokens=1))
+            xs.append(m["x"].contiguous())
+            mats.append(m)
+    stack = g.Stack(layers, mode=mode)
+    stack.bind(xs, n_steps=n_steps)
+    ys = [[] for _ in mats]
+    for s in range(n_steps):
+        stack.step()
+        torch.cuda.synchronize()
+        for i, y in enumerate(stack.ys):
+            ys[i].append(y.cpu().clone())
+    assert stack.status() == 0
+    gate_log = stack.gate_log.cpu().numpy()
+    rho_log = stack.rho_log.cpu().numpy()
+    stats = []
+    for i, m in enumerate(mats):
+        y = torch.cat(ys[i]).numpy()
+        Ws = [W.cpu() for W in m["W"]]
+        if sample_rows:
+            cols, Wsamp, off = [], [], 0
+            for W in Ws:
+                r = np.sort(rng.choice(W.shape[0], min(sample_rows, W.shape[0]), replace=False))
+                Wsamp.append(W[torch.as_tensor(r)].contiguous())
+                cols.append(off + r)
+                off += W.shape[0]
+            y = y[:, np.concatenate(cols)]
+            Ws = Wsamp
+        stats.append(compare_group(m["x"].cpu(), m["P"].cpu(), Ws, st.eps, y,
+                                   gate_log[:, i, 0], rho_log[:, i, 0]))
+    return stack, stats, ys, gate_log
+
+
+def test_persistent_gptj_two_layers_full_size_sampled_rows():
+    """The launch configuration the benchmark times (one persistent launch per
+    step, GPT-J shapes, k=256, eps=0.05), two layers, 12 steps; the oracle
+    evaluates a sample of the output rows of every map."""
+    st = S.config3("10")
+    stack, stats, ys, gate_log = _stack_against_oracle(st, 2, 12, mode=2, sample_rows=40)
+    assert stack.is_persistent()
+    rates = [s["gate_rate"] for s in stats]
+    assert 0.0 < np.mean(rates) < 0.5   # both paths occur
+
+
+def test_persistent_matches_generic_kernels_and_is_reproducible():
+    st = S.config2()
+    a, _, ys_a, gate_a = _stack_against_oracle(st, 1, 8, mode=2)
+    b, _, ys_b, gate_b = _stack_against_oracle(st, 1, 8, mode=2)
+    c, _, ys_c, gate_c = _stack_against_oracle(st, 1, 8, mode=1)
+    assert np.array_equal(gate_a, gate_b) and np.array_equal(gate_a, gate_c)
+    for i in range(len(ys_a)):
+        for s in range(8):
+            assert torch.equal(ys_a[i][s], ys_b[i][s])      # order-free fixed-point exchange
+            ref = ys_c[i][s]
+            assert (ys_a[i][s] - ref).abs().max() <= 1e-4 * ref.abs().max()
+
+
+@pytest.mark.parametrize("k", [64, 128, 512])
+def test_persistent_other_ranks_and_flags(k):
+    g = G()
+    d, d_out, n_steps = 2048, (1024, 512), 6
+    q = S.gen_basis(d, k, 100 + k)
+    P = S.store_basis(q)
+    Ws = [S.gen_weight(o, d, 200 + k + j) for j, o in enumerate(d_out)]
+    pt = S.gen_true_basis(q, k // 2, k // 2, 300 + k)
+    x, _ = S.gen_activations(pt, n_steps, 0.01, 0.0, dict(z=1, noise=2, outlier_mask=0, outlier_values=0))
+    x[::3] = torch.randn((len(range(0, n_steps, 3)), d), generator=torch.Generator().manual_seed(k))
+    x[4] = 0.0
+    for flags in (0, g.GSI_FLAG_STATIC_PROJECTION):
+        lay = g.Layer([W.cuda() for W in Ws], P.cuda(), 0.05, max_tokens=1, flags=flags)
+        dense = g.Layer([W.cuda() for W in Ws], None, 0.0, max_tokens=1, flags=g.GSI_FLAG_DENSE)
+        stack = g.Stack([lay, dense], mode=2)
+        stack.bind([x.cuda().contiguous(), x.cuda().contiguous()], n_steps=n_steps)
+        y0, y1 = [], []
+        for s in range(n_steps):
+            stack.step()
+            torch.cuda.synchronize()
+            y0.append(stack.ys[0].cpu().clone())
+            y1.append(stack.ys[1].cpu().clone())
+        assert stack.status() == 0 and stack.is_persistent()
+        gate = stack.gate_log[:, 0, 0].cpu().numpy()
+        rho = stack.rho_log[:, 0, 0].cpu().numpy()
+        keep = [s for s in range(n_steps) if s != 4]
+        yy = torch.cat(y0).numpy()
+        compare_group(x[keep], P, Ws, 0.05, yy[keep], gate[keep], rho[keep], static=bool(flags))
+        assert gate[4] == 1 and np.all(yy[4] == 0.0)
+        assert stack.gate_log[:, 1, 0].cpu().numpy().all()
+        ref = torch.cat([x.to(torch.float64) @ W.to(torch.float64).T for W in Ws], dim=1).numpy()
+        assert np.max(np.abs(torch.cat(y1).numpy() - ref)) <= 1e-5 * np.max(np.abs(ref))
+
+
+def test_persistent_nonfinite_token():
+    g = G()
+    x, P, Ws = make_small(256, 32, (64,), 3, seed=41)
+    x[1, 7] = float("nan")
+    lay = g.Layer([W.cuda() for W in Ws], P.cuda(), 0.5, max_tokens=1)
+    stack = g.Stack([lay], mode=2)
+    stack.bind([x.cuda().contiguous()], n_steps=3)
+    ys = []
+    for s in range(3):
+        stack.step()
+        torch.cuda.synchronize()
+        ys.append(stack.ys[0].cpu().clone())
+    assert stack.status() == 0
+    gate = stack.gate_log[:, 0, 0].cpu().numpy()
+    assert gate[1] == 1 and torch.isnan(ys[1]).all()
+    keep = [0, 2]
+    compare_group(x[keep], P, Ws, 0.5, torch.cat(ys).numpy()[keep], gate[keep])
+
+
+def test_persistent_falls_back_when_a_group_does_not_qualify():
+    g = G()
+    x, P, Ws = make_small(256, 24, (64,), 2, seed=43)      # k = 24 is not a power of two
+    lay = g.Layer([W.cuda() for W in Ws], P.cuda(), 0.05, max_tokens=1)
+    stack = g.Stack([lay])
+    stack.bind([x.cuda().contiguous()], n_steps=2)
+    assert not stack.is_persistent()
+    forced = g.Stack([lay], mode=2)
+    with pytest.raises(g.GsiError):
+        forced.bind([x.cuda().contiguous()], n_steps=2)
