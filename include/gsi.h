@@ -189,7 +189,7 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io_host_array,
 /*
  * Execution mode, taken at the next gsi_stack_bind:
  *   0 (default)  one persistent launch per step when every group qualifies
- *                (batch 1, bf16 basis with k a power of two <= 512, d a
+ *                (batch 1, bf16 basis with k in {64,128,256,512}, d a
  *                multiple of 16, 32-byte aligned W), else the per-stage kernels;
  *   1            always the per-stage kernels;
  *   2            the persistent launch or GSI_ERR_UNSUPPORTED from bind.
@@ -199,6 +199,21 @@ gsi_status_t gsi_stack_set_mode(gsi_stack_t s, int mode);
 
 /* 1 if the bound stack runs as one persistent launch per step. */
 gsi_status_t gsi_stack_is_persistent(gsi_stack_t s, int* out);
+
+/*
+ * Tracing.  `cycles` is a DEVICE array [n_CTAs][GSI_TRACE_SECTIONS] of 64-bit
+ * counters (n_CTAs = SM count; NULL switches tracing off).  While set, thread 0
+ * of every CTA of the persistent launch adds the SM cycles it spends in each
+ * section of the per-group pipeline:
+ *   0 loads of x           1 statistics of x     2 wait for basis slab
+ *   3 pass 1               4 partial-c atomics   5 wait for c
+ *   6 pass 2               7 wait for image slab 8 image rows
+ *   9 publish ||r||^2      10 wait for all ||r||^2   11 gate decision
+ *   12 gated residual      13 grid barrier after it
+ * The caller clears and reads the counters.  Applies from the next step.
+ */
+#define GSI_TRACE_SECTIONS 16
+gsi_status_t gsi_stack_set_trace(gsi_stack_t s, unsigned long long* cycles);
 
 /* Set the device-side step counter (enqueued on `stream`). */
 gsi_status_t gsi_stack_seek(gsi_stack_t s, int step, gsi_stream_t stream);

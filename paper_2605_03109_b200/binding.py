@@ -21,7 +21,7 @@ EXPORTED = [
     "gsi_status_string", "gsi_build_image", "gsi_workspace_bytes", "gsi_create",
     "gsi_forward", "gsi_forward_n", "gsi_forward_host", "gsi_get_image", "gsi_get_status",
     "gsi_destroy", "gsi_stack_workspace_bytes", "gsi_stack_create", "gsi_stack_bind",
-    "gsi_stack_set_mode", "gsi_stack_is_persistent", "gsi_stack_seek", "gsi_stack_step", "gsi_stack_launches_per_step",
+    "gsi_stack_set_mode", "gsi_stack_is_persistent", "gsi_stack_set_trace", "gsi_stack_seek", "gsi_stack_step", "gsi_stack_launches_per_step",
     "gsi_stack_step_host", "gsi_stack_get_status", "gsi_stack_destroy",
 ]
 
@@ -68,6 +68,7 @@ def _load():
     l.gsi_stack_bind.argtypes = [vp, C.POINTER(GsiStackIo), i, vp, vp, vp]
     l.gsi_stack_set_mode.argtypes = [vp, i]
     l.gsi_stack_is_persistent.argtypes = [vp, C.POINTER(i)]
+    l.gsi_stack_set_trace.argtypes = [vp, vp]
     l.gsi_stack_seek.argtypes = [vp, i, vp]
     l.gsi_stack_step.argtypes = [vp, vp]
     l.gsi_stack_launches_per_step.argtypes = [vp, C.POINTER(i)]
@@ -260,6 +261,13 @@ class Stack:
         _check(lib.gsi_stack_bind(self.handle, io, n_steps, self.gate_log.data_ptr(),
                                   None if self.rho_log is None else self.rho_log.data_ptr(),
                                   _stream_ptr(stream)), "gsi_stack_bind")
+
+    def set_trace(self, on: bool = True):
+        """Per-section SM-cycle counters of CTA 0 (persistent launch only)."""
+        self.trace = torch.zeros((256, 16), dtype=torch.int64, device=self.device) if on else None
+        _check(lib.gsi_stack_set_trace(self.handle, self.trace.data_ptr() if on else None),
+               "gsi_stack_set_trace")
+        return self.trace
 
     def seek(self, step: int, stream=None):
         _check(lib.gsi_stack_seek(self.handle, int(step), _stream_ptr(stream)), "gsi_stack_seek")

@@ -66,7 +66,7 @@ Layout make_layout_ws(const gsi_desc_t* d) {
   L.y_stage = take(B * (size_t)O * 4);
   L.gate_stage = take(B);
   L.rho_stage = take(B * 4);
-  L.pk_acc = take(2 * k * 8);                       // persistent kernel: c accumulators
+  L.pk_acc = take(2 * k * 8 * kAccStride);          // persistent kernel: c accumulators
   L.pk_slot = take((size_t)kPersistMaxGrid * 8);    // persistent kernel: ||r||^2 words
   L.total = at;
   return L;
@@ -91,8 +91,10 @@ struct gsi_stack {
   int grid;                 // CTAs of the persistent kernel (= SMs)
   PersistGroup* dev_groups; // device table
   std::vector<PersistGroup> host_groups;
+  std::vector<const float*> host_pmax_ptrs;
   int* epoch;               // device
   int* status;              // device
+  unsigned long long* trace; // device, optional
   std::vector<gsi_layer*> groups;
   std::vector<gsi_stack_io_t> io;
   int B;
@@ -295,7 +297,7 @@ gsi_status_t gsi_destroy(gsi_handle_t h) {
 size_t gsi_stack_workspace_bytes(int n_groups) {
   if (n_groups <= 0) return 0;
   static_assert(sizeof(PersistGroup) <= 512, "group descriptor outgrew its slot");
-  return align_up(256) + align_up((size_t)n_groups * 512);
+  return align_up(256) + align_up((size_t)n_groups * 512) + align_up((size_t)n_groups * 8);
 }
 
 gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* workspace,
@@ -322,6 +324,7 @@ gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* wo
   s->status = s->step + 2;
   s->dev_groups = reinterpret_cast<PersistGroup*>(static_cast<char*>(workspace) + 256);
   s->mode = 0;
+  s->trace = nullptr;
   s->persistent = false;
   s->grid = 0;
   s->bound = false;
@@ -349,7 +352,7 @@ static bool persistent_eligible(const gsi_stack* s, int grid) {
       if (reinterpret_cast<uintptr_t>(h->gp.W[j]) & 31u) return false;
     if (!dense) {
       if (d.p_dtype != GSI_BF16) return false;
-      if (d.k < 8 || d.k > 512 || (d.k & (d.k - 1))) return false;
+      if (d.k < 64 || d.k > 512 || (d.k & (d.k - 1))) return false;
     }
   }
   return true;
@@ -388,6 +391,7 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
   }
   if (s->persistent) {
     s->host_groups.assign(G, PersistGroup{});
+    s->host_pmax_ptrs.assign(G, nullptr);
     for (int i = 0; i < G; ++i) {
       const gsi_layer* h = s->groups[i];
       PersistGroup& pg = s->host_groups[i];
@@ -402,7 +406,8 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
       pg.O = gp.O;
       pg.eps = gp.eps;
       pg.flags = gp.flags;
-      pg.pmax = h->pmax;
+      pg.pmax = 0.f;
+      s->host_pmax_ptrs[i] = (gp.flags & GSI_FLAG_DENSE) ? nullptr : h->pmax;
       pg.x = io[i].x;
       pg.y = io[i].y;
       pg.r = gp.r;
@@ -413,8 +418,13 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
       pg.o_rows = (gp.O + s->grid - 1) / s->grid;
       pg.x_step_stride = gp.d;
     }
+    const float** dev_ptrs = reinterpret_cast<const float**>(
+        reinterpret_cast<char*>(s->dev_groups) + (size_t)G * 512);
     if (cudaMemcpyAsync(s->dev_groups, s->host_groups.data(), sizeof(PersistGroup) * G,
-                        cudaMemcpyHostToDevice, stream) != cudaSuccess)
+                        cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(dev_ptrs, s->host_pmax_ptrs.data(), sizeof(float*) * G,
+                        cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        launch_patch_pmax(s->dev_groups, dev_ptrs, G, stream) != cudaSuccess)
       return GSI_ERR_CUDA;
   }
   s->bound = true;
@@ -445,6 +455,7 @@ static gsi_status_t stack_enqueue(gsi_stack_t s, bool use_counter, gsi_stream_t 
     p.rho_log = s->rho_log;
     p.log_step_stride = G;
     p.status = s->status;
+    p.trace = s->trace;
     return launch_decode_step(p, s->grid, stream) == cudaSuccess ? GSI_OK : GSI_ERR_CUDA;
   }
   for (int i = 0; i < G; ++i) {
@@ -511,6 +522,12 @@ gsi_status_t gsi_stack_step_host(gsi_stack_t s, const float* const* x_host, floa
       cudaSuccess)
     return GSI_ERR_CUDA;
   return cudaStreamSynchronize(stream) == cudaSuccess ? GSI_OK : GSI_ERR_CUDA;
+}
+
+gsi_status_t gsi_stack_set_trace(gsi_stack_t s, unsigned long long* cycles) {
+  if (!s) return GSI_ERR_INVALID_ARG;
+  s->trace = cycles;
+  return GSI_OK;
 }
 
 gsi_status_t gsi_stack_is_persistent(gsi_stack_t s, int* out) {

@@ -45,12 +45,15 @@ constexpr int kOffMisc = 256;       // abort flag, scalars
 constexpr int kOffX = 512;          // x of this CTA's basis rows      (kPersistMaxPRows floats)
 constexpr int kOffC = 1024;         // c                                (512 floats)
 constexpr int kOffVals = 3072;      // exchange-2 values                (256 floats)
-constexpr int kOffRed = 4096;       // cross-warp scratch               (kNW*512 floats)
+constexpr int kOffDesc = 4096;      // 3 group descriptors, 512 B each (current, next, previous)
+constexpr int kOffRed = kOffDesc + 3 * 512;       // cross-warp scratch (kNW*512 floats)
 constexpr int kOffRq = kOffRed + kNW * 512 * 4;   // staged r, 4 interleaved quarters (16 KB)
 constexpr int kOffYacc = kOffRq + 16384;          // per-row accumulators (kPersistMaxORows floats)
 constexpr int kOffRing = ((kOffYacc + kPersistMaxORows * 4 + 1023) / 1024) * 1024;
 constexpr int kSmemBytes = kOffRing + kSlots * kChunk;
 static_assert(kSmemBytes <= 232448, "shared memory budget of one sm_100 CTA");
+static_assert(sizeof(PersistGroup) <= 512 && sizeof(PersistGroup) % 4 == 0, "descriptor slot");
+constexpr int kDescWords = (int)(sizeof(PersistGroup) / 4);
 
 struct Misc {
   int abort;
@@ -111,16 +114,16 @@ __device__ __forceinline__ unsigned long long ld_relaxed_u64(const unsigned long
 __device__ __forceinline__ void red_add_u64(unsigned long long* p, unsigned long long v) {
   asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
-__device__ __forceinline__ void st_release_u64(unsigned long long* p, unsigned long long v) {
-  asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+__device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
+  asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
-__device__ __forceinline__ unsigned ld_acquire_u32(const unsigned* p) {
+__device__ __forceinline__ unsigned ld_relaxed_u32(const unsigned* p) {
   unsigned v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
-__device__ __forceinline__ void red_release_u32(unsigned* p, unsigned v) {
-  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+__device__ __forceinline__ void red_relaxed_u32(unsigned* p, unsigned v) {
+  asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ void ld256_stream(const void* p, uint32_t (&v)[8]) {
   asm volatile(
@@ -138,8 +141,24 @@ __device__ __forceinline__ void fail(const PersistParams& p, Misc* misc) {
   atomicExch(p.status, (int)GSI_ERR_TIMEOUT);
 }
 
-// Rows [r0, r1) of a slab, in chunks of `rc` rows; returns the chunk count.
-__device__ __forceinline__ int n_chunks(int rows, int rc) { return (rows + rc - 1) / rc; }
+// Optional cycle trace of CTA 0 (sections of the per-group pipeline, summed
+// over groups); p.trace == nullptr disables it.
+struct Trace {
+  unsigned long long* out;
+  long long t;
+  __device__ __forceinline__ void start(const PersistParams& p) {
+    out = (threadIdx.x == 0 && p.trace) ? p.trace + (size_t)blockIdx.x * 16 : nullptr;
+    if (out) t = clock64();
+  }
+  __device__ __forceinline__ void mark(int section) {
+    if (out) {
+      const long long now = clock64();
+      out[section] += (unsigned long long)(now - t);
+      t = now;
+    }
+  }
+};
+
 
 struct Slab {
   int p0, p1;  // basis rows owned by this CTA
@@ -203,10 +222,185 @@ struct Ctx {
   int step, slot_io;
   unsigned parity, tag;
   unsigned n;  // ring sequence number, advances exactly as in producer()
+  Trace tr;
 };
 
+// ---- consumer building blocks.  The per-group code below is executed once per
+// group and is deliberately compact (no templates, shifts instead of divisions,
+// the rarely-taken gated residual out of line): the per-group loop has to stay
+// resident in the SM's instruction cache, a loop that does not is bound by
+// instruction fetch, not by memory.
+
+// Sum eight per-lane row partials across the LPR = 1<<lpr_log2 lanes (8, 16 or
+// 32) that share the rows.  Halving exchange: each level sends half of the
+// values to the partner lane, so eight rows cost 4+2+1 shuffles plus
+// log2(LPR/8) for the tail instead of 8*log2(LPR).  On return the lanes with
+// cl % (LPR/8) == 0 hold the total of row cl / (LPR/8).
+__device__ __forceinline__ float reduce8(float (&v)[8], int cl, int LPR) {
+  int m = LPR >> 1;
+  {
+    const bool up = cl & m;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float send = up ? v[i] : v[i + 4];
+      const float recv = __shfl_xor_sync(0xffffffffu, send, m);
+      v[i] = (up ? v[i + 4] : v[i]) + recv;
+    }
+  }
+  m >>= 1;
+  {
+    const bool up = cl & m;
+#pragma unroll
+    for (int i = 0; i < 2; ++i) {
+      const float send = up ? v[i] : v[i + 2];
+      const float recv = __shfl_xor_sync(0xffffffffu, send, m);
+      v[i] = (up ? v[i + 2] : v[i]) + recv;
+    }
+  }
+  m >>= 1;
+  {
+    const bool up = cl & m;
+    const float send = up ? v[0] : v[1];
+    const float recv = __shfl_xor_sync(0xffffffffu, send, m);
+    v[0] = (up ? v[1] : v[0]) + recv;
+  }
+#pragma unroll 1
+  for (m >>= 1; m > 0; m >>= 1) v[0] += __shfl_xor_sync(0xffffffffu, v[0], m);
+  return v[0];
+}
+
+struct Geo {       // lane geometry of one group (k a power of two, 64..512)
+  int KV;          // 16-byte vectors per row
+  int lpr_log2;    // log2(lanes per row), lanes per row = min(32, KV)
+  int vpl;         // vectors per lane (1, or 2 for k = 512)
+  int rc_log2;     // log2(rows per 16 KB chunk)
+  int sub, cl;     // this lane: row sub-group and column lane
+};
+
+// out[i] = tile[row0 + i][:] . c   for eight rows, this lane's share of the columns
+__device__ __forceinline__ void dot8(const uint4* tile, const float* s_c, const Geo& q, int row0,
+                                     int rows, float (&v)[8]) {
+#pragma unroll
+  for (int i = 0; i < 8; ++i) v[i] = 0.f;
+  const int LPR = 1 << q.lpr_log2;
+#pragma unroll 1
+  for (int u = 0; u < q.vpl; ++u) {
+    const int cv = q.cl + u * LPR;
+    const float4 ca = *reinterpret_cast<const float4*>(s_c + cv * 8);
+    const float4 cb = *reinterpret_cast<const float4*>(s_c + cv * 8 + 4);
+#pragma unroll
+    for (int i = 0; i < 8; ++i) {
+      if (row0 + i < rows) {
+        const uint4 w = tile[(size_t)(row0 + i) * q.KV + cv];
+        float d = v[i];
+        d = fmaf(__uint_as_float(w.x << 16), ca.x, d);
+        d = fmaf(__uint_as_float(w.x & 0xFFFF0000u), ca.y, d);
+        d = fmaf(__uint_as_float(w.y << 16), ca.z, d);
+        d = fmaf(__uint_as_float(w.y & 0xFFFF0000u), ca.w, d);
+        d = fmaf(__uint_as_float(w.z << 16), cb.x, d);
+        d = fmaf(__uint_as_float(w.z & 0xFFFF0000u), cb.y, d);
+        d = fmaf(__uint_as_float(w.w << 16), cb.z, d);
+        d = fmaf(__uint_as_float(w.w & 0xFFFF0000u), cb.w, d);
+        v[i] = d;
+      }
+    }
+  }
+}
+
+// 2^e as a double, e in the normal range
+__device__ __forceinline__ double pow2d(int e) { return __hiloint2double((1023 + e) << 20, 0); }
+
+// Grid-wide arrival counter: add one, wait (bounded) until `target` arrived.
+__device__ __forceinline__ bool grid_arrive_wait(unsigned* ctr, unsigned target,
+                                                 const PersistParams& p, Misc* misc) {
+  volatile int* abort = &misc->abort;
+  red_relaxed_u32(ctr, 1u);
+  unsigned it = 0;
+  while (ld_relaxed_u32(ctr) < target) {
+    if (++it > kSpinLimit || *abort) {
+      if (!*abort) fail(p, misc);
+      return false;
+    }
+  }
+  return true;
+}
+
+// ---- F. gated residual: y_rows (+)= W_rows . src (src = r, or x for the dense
+// baseline).  Out of line: most groups skip it.
+__device__ __noinline__ void gated_pass(const PersistGroup& g, const Slab& s, const float* src,
+                                        bool dense, unsigned char* smem) {
+  float4* s_rq = reinterpret_cast<float4*>(smem + kOffRq);
+  float* s_yacc = reinterpret_cast<float*>(smem + kOffYacc);
+  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  const int rows = s.o1 - s.o0;
+  const int nsl = (g.d + kSlice - 1) / kSlice;
+#pragma unroll 1
+  for (int sl = 0; sl < nsl; ++sl) {
+    const int c0 = sl * kSlice, cols = min(kSlice, g.d - c0), nv = cols >> 4;
+    csync();
+#pragma unroll 1
+    for (int v = tid; v < nv; v += kNC) {
+      const float4* sp = reinterpret_cast<const float4*>(src + c0 + v * 16);
+#pragma unroll
+      for (int q = 0; q < 4; ++q) s_rq[q * 256 + v] = __ldcg(sp + q);
+    }
+    csync();
+#pragma unroll 1
+    for (int rw = warp; rw < rows; rw += kNW) {
+      const int a = s.o0 + rw;
+      int j = 0;
+      while (j + 1 < g.n_maps && a >= g.off[j + 1]) ++j;
+      const uint16_t* wrow = g.W[j] + (size_t)(a - g.off[j]) * g.d + c0;
+      float acc = 0.f;
+#pragma unroll 1
+      for (int v0 = lane; v0 < nv; v0 += 4 * 32) {
+        uint32_t w[4][8];
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int v = v0 + u * 32;
+          if (v < nv) ld256_stream(wrow + (size_t)v * 16, w[u]);
+        }
+#pragma unroll
+        for (int u = 0; u < 4; ++u) {
+          const int v = v0 + u * 32;
+          if (v < nv) {
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+              const float4 rr = s_rq[q * 256 + v];
+              const uint32_t lo = w[u][2 * q], hi = w[u][2 * q + 1];
+              acc = fmaf(__uint_as_float(lo << 16), rr.x, acc);
+              acc = fmaf(__uint_as_float(lo & 0xFFFF0000u), rr.y, acc);
+              acc = fmaf(__uint_as_float(hi << 16), rr.z, acc);
+              acc = fmaf(__uint_as_float(hi & 0xFFFF0000u), rr.w, acc);
+            }
+          }
+        }
+      }
+      acc = warp_sum(acc);
+      if (lane == 0) s_yacc[rw] = (sl == 0 ? 0.f : s_yacc[rw]) + acc;
+    }
+  }
+  __syncwarp();
+#pragma unroll 1
+  for (int rw = warp; rw < rows; rw += kNW) {
+    if (lane == 0) {
+      float* yp = g.y + s.o0 + rw;
+      *yp = dense ? s_yacc[rw] : (*yp + s_yacc[rw]);
+    }
+  }
+}
+
+// Make the next group's activations L2-resident while this group runs (a real
+// pipeline would find them there, written by the preceding operator).
+__device__ __forceinline__ void prefetch_next_x(const PersistGroup& gn, int slot_io) {
+  if (blockIdx.x == 0) {
+    const char* xn = reinterpret_cast<const char*>(gn.x + (long long)slot_io * gn.x_step_stride);
+    const int lines = (gn.d * 4 + 127) >> 7;
+    for (int l = threadIdx.x; l < lines; l += kNC) prefetch_l2(xn + (size_t)l * 128);
+  }
+}
+
 // One group.  Returns false when the CTA must stop (a wait gave up).
-template <int VPL>
 __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* misc, Ctx& ctx,
                             int gi) {
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + kOffBar);
@@ -215,8 +409,6 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
   float* s_c = reinterpret_cast<float*>(smem + kOffC);
   float* s_vals = reinterpret_cast<float*>(smem + kOffVals);
   float* s_red = reinterpret_cast<float*>(smem + kOffRed);
-  float4* s_rq = reinterpret_cast<float4*>(smem + kOffRq);
-  float* s_yacc = reinterpret_cast<float*>(smem + kOffYacc);
   unsigned char* ring = smem + kOffRing;
   volatile int* abort = &misc->abort;
 
@@ -225,342 +417,356 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
   const int slot_io = ctx.slot_io;
   const unsigned parity = ctx.parity, tag = ctx.tag;
   unsigned& n = ctx.n;
-  {
-    const PersistGroup& g = p.groups[gi];
-    const int KV = g.k / 8;
-    const Slab s = slab_of(g, cta);
-    const float* x = g.x + (long long)slot_io * g.x_step_stride;
-    const bool dense = g.flags & GSI_FLAG_DENSE;
-    int gate = 1;
-    const float* rsrc = x;
+  Trace& tr = ctx.tr;
 
-    // make the next group's activations L2-resident while this one runs
-    if (gi + 1 < p.n_groups) {
-      const PersistGroup& gn = p.groups[gi + 1];
-      const char* xn = reinterpret_cast<const char*>(gn.x + (long long)slot_io * gn.x_step_stride);
-      const int lines = (gn.d * 4 + 127) / 128;
-      for (int l = cta * kNC + tid; l < lines; l += G * kNC) prefetch_l2(xn + (size_t)l * 128);
+  // The descriptor of this group was staged in shared memory one group ago;
+  // stage the next one now (three slots: current, next, previous).
+  const PersistGroup& g = *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + (gi % 3) * 512);
+  const PersistGroup& g_next =
+      *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + ((gi + 1) % 3) * 512);
+  const bool has_next = gi + 1 < p.n_groups;
+  uint32_t desc_word = 0;  // one word of the next descriptor, in flight during section A
+  if (has_next && tid < kDescWords)
+    desc_word = __ldg(reinterpret_cast<const uint32_t*>(p.groups + gi + 1) + tid);
+
+  const Slab s = slab_of(g, cta);
+  const float* x = g.x + (long long)slot_io * g.x_step_stride;
+  const bool dense = g.flags & GSI_FLAG_DENSE;
+  const bool zeroer = cta == gi % G;  // this CTA clears the group's counters for the next launch
+  int gate = 1;
+  const float* rsrc = x;
+
+  if (!dense) {
+    const int k = g.k;
+    Geo q;
+    q.KV = k >> 3;
+    q.lpr_log2 = q.KV >= 32 ? 5 : 31 - __clz(q.KV);
+    q.vpl = q.KV > 32 ? q.KV >> 5 : 1;
+    q.rc_log2 = 31 - __clz(kChunk / 2) - (31 - __clz(k));  // rows per chunk = 8192 / k
+    const int LPR = 1 << q.lpr_log2;
+    q.sub = lane >> q.lpr_log2;
+    q.cl = lane & (LPR - 1);
+    const int rpp_log2 = 5 - q.lpr_log2;  // rows per warp pass
+    const int rc = 1 << q.rc_log2;
+    const int n_contrib = (g.d + g.p_rows - 1) / g.p_rows;
+    unsigned long long* acc = g.acc_c + (size_t)parity * k * kAccStride;
+    const int prow = s.p1 - s.p0, orow = s.o1 - s.o0;
+    const int pchunks = (prow + rc - 1) >> q.rc_log2, ochunks = (orow + rc - 1) >> q.rc_log2;
+
+    // ---- A. statistics of x (every CTA, the whole vector): max |x|, sum x^2,
+    //      non-finite flag; x of this CTA's basis rows goes to shared memory.
+    float amax = 0.f, sum2 = 0.f;
+    const int d4 = g.d >> 2;
+#pragma unroll 1
+    for (int i0 = tid; i0 < d4; i0 += 4 * kNC) {
+      float4 v[4];
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        const int i4 = i0 + u * kNC;
+        v[u] = i4 < d4 ? __ldcg(reinterpret_cast<const float4*>(x) + i4) : make_float4(0, 0, 0, 0);
+      }
+#pragma unroll
+      for (int u = 0; u < 4; ++u) {
+        amax = fmaxf(fmaxf(amax, fmaxf(fabsf(v[u].x), fabsf(v[u].y))),
+                     fmaxf(fabsf(v[u].z), fabsf(v[u].w)));
+        sum2 = fmaf(v[u].x, v[u].x, sum2);
+        sum2 = fmaf(v[u].y, v[u].y, sum2);
+        sum2 = fmaf(v[u].z, v[u].z, sum2);
+        sum2 = fmaf(v[u].w, v[u].w, sum2);
+      }
     }
+    if (tid < prow) s_x[tid] = __ldcg(x + s.p0 + tid);
+    if (has_next && tid < kDescWords)
+      reinterpret_cast<uint32_t*>(smem + kOffDesc + ((gi + 1) % 3) * 512)[tid] = desc_word;
+    tr.mark(0);
+    // fmaxf drops NaN, the sum keeps it (and overflows to inf for huge inputs):
+    // sum2 - sum2 is non-zero exactly when some x_i is NaN or inf (or x^2 overflowed)
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+      sum2 += __shfl_xor_sync(0xffffffffu, sum2, o);
+    }
+    if (lane == 0) {
+      s_red[warp * 2 + 0] = amax;
+      s_red[warp * 2 + 1] = sum2;
+    }
+    if (zeroer) {  // clear what the NEXT launch will accumulate into
+#pragma unroll 1
+      for (int j = tid; j < k; j += kNC)
+        g.acc_c[((size_t)(parity ^ 1u) * k + j) * kAccStride] = 0ull;
+      if (tid < 3) g.bar[2 * tid + (parity ^ 1u)] = 0u;
+    }
+    csync();
+    if (has_next) prefetch_next_x(g_next, slot_io);
+    {  // every thread folds the warp partials in the same order
+      float a = 0.f, t = 0.f;
+#pragma unroll
+      for (int w = 0; w < kNW; ++w) {
+        a = fmaxf(a, s_red[w * 2]);
+        t += s_red[w * 2 + 1];
+      }
+      amax = a;
+      sum2 = t;
+    }
+    const bool nonfinite = !(sum2 - sum2 == 0.f);
+    tr.mark(1);
+    // fixed-point scale: |partial c_j| <= amax * rows * max|P| < 2^e
+    double scale = 0.0, inv_scale = 0.0;
+    {
+      const float bound = amax * (float)g.p_rows * g.pmax;
+      if (!nonfinite && bound > 0.f && bound < 3.0e38f) {
+        const int e = max((int)((__float_as_uint(bound) >> 23) & 0xFFu), 1) - 126;
+        scale = pow2d(43 - e);
+        inv_scale = pow2d(e - 43);
+      }
+    }
+    csync();  // s_red is reused by pass 1
 
-    if (!dense) {
-      const int k = g.k;
-      const int LPR = KV < 32 ? KV : 32, RPP = 32 / LPR;
-      const int sub = lane / LPR, cl = lane % LPR;
-      const int rc = kChunk / (k * 2);
-      const int n_contrib = (g.d + g.p_rows - 1) / g.p_rows;
-      unsigned long long* acc = g.acc_c + (size_t)parity * k;
-
-      // ---- A. statistics of x (every CTA, the whole vector): max |x|, sum x^2
-      float amax = 0.f, sum2 = 0.f;
-      int bad = 0;
-      for (int i4 = tid; i4 < g.d / 4; i4 += kNC) {
-        const float4 v = __ldcg(reinterpret_cast<const float4*>(x) + i4);
-        const float e[4] = {v.x, v.y, v.z, v.w};
+    // ---- B. pass 1: partial c over this CTA's basis rows
+    const unsigned n_p0 = n;
+    bool ok = true;
+#pragma unroll 1
+    for (int u = 0; u < q.vpl; ++u) {
+      const int cv = q.cl + u * LPR;
+      float a8[8];
 #pragma unroll
-        for (int q = 0; q < 4; ++q) {
-          amax = fmaxf(amax, fabsf(e[q]));
-          sum2 = fmaf(e[q], e[q], sum2);
-          bad |= !(fabsf(e[q]) <= 3.0e38f);
-          const int i = i4 * 4 + q;
-          if (i >= s.p0 && i < s.p1) s_x[i - s.p0] = e[q];
-        }
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-        sum2 += __shfl_xor_sync(0xffffffffu, sum2, o);
-        bad |= __shfl_xor_sync(0xffffffffu, bad, o);
-      }
-      if (lane == 0) {
-        s_red[warp * 4 + 0] = amax;
-        s_red[warp * 4 + 1] = sum2;
-        s_red[warp * 4 + 2] = (float)bad;
-      }
-      if (cta == gi % G) {  // clear the accumulators the NEXT step will use
-        for (int j = tid; j < k; j += kNC) g.acc_c[(size_t)(parity ^ 1u) * k + j] = 0ull;
-        if (tid == 0) g.bar[parity ^ 1u] = 0u;
-      }
-      csync();
-      if (tid == 0) {
-        float a = 0.f, q = 0.f, b = 0.f;
-        for (int w = 0; w < kNW; ++w) {
-          a = fmaxf(a, s_red[w * 4]);
-          q += s_red[w * 4 + 1];
-          b += s_red[w * 4 + 2];
-        }
-        misc->amax = a;
-        misc->sum2 = q;
-        misc->nonfinite = b != 0.f;
-      }
-      csync();
-      const int nonfinite = misc->nonfinite;
-      // fixed-point scale: |partial c_j| <= amax * rows * max|P| < 2^e
-      double scale = 0.0, inv_scale = 0.0;
-      {
-        const float bound = misc->amax * (float)g.p_rows * __ldg(g.pmax);
-        if (!nonfinite && bound > 0.f && bound < 3.0e38f) {
-          int e;
-          frexpf(bound, &e);
-          scale = ldexp(1.0, 43 - e);
-          inv_scale = ldexp(1.0, e - 43);
-        }
-      }
-
-      // ---- B. pass 1: partial c over this CTA's basis rows
-      const unsigned n_p0 = n;
-      const int pchunks = n_chunks(s.p1 - s.p0, rc);
-      float accv[VPL][8];
-#pragma unroll
-      for (int v = 0; v < VPL; ++v)
-#pragma unroll
-        for (int e = 0; e < 8; ++e) accv[v][e] = 0.f;
-      bool ok = true;
+      for (int e = 0; e < 8; ++e) a8[e] = 0.f;
+#pragma unroll 1
       for (int ci = 0; ci < pchunks; ++ci) {
         const unsigned sl = (n_p0 + ci) % kSlots, ph = ((n_p0 + ci) / kSlots) & 1u;
         ok = ok && mbar_wait(&full[sl], ph, abort);
         if (!ok) break;
+        tr.mark(2);
         const uint4* tile = reinterpret_cast<const uint4*>(ring + (size_t)sl * kChunk);
-        const int r_lo = ci * rc, rows = min(rc, s.p1 - s.p0 - r_lo);
-        for (int base = warp * RPP; base < rows; base += kNW * RPP) {
-          const int row = base + sub;
-          if (row < rows) {
-            const float xv = s_x[r_lo + row];
-#pragma unroll
-            for (int v = 0; v < VPL; ++v) {
-              float p8[8];
-              unpack_bf16x8(tile[(size_t)row * KV + cl + v * LPR], p8);
-#pragma unroll
-              for (int e = 0; e < 8; ++e) accv[v][e] = fmaf(p8[e], xv, accv[v][e]);
-            }
-          }
+        const int r_lo = ci << q.rc_log2, rows = min(rc, prow - r_lo);
+#pragma unroll 1
+        for (int row = (warp << rpp_log2) + q.sub; row < rows; row += kNW << rpp_log2) {
+          const float xv = s_x[r_lo + row];
+          const uint4 w = tile[(size_t)row * q.KV + cv];
+          a8[0] = fmaf(__uint_as_float(w.x << 16), xv, a8[0]);
+          a8[1] = fmaf(__uint_as_float(w.x & 0xFFFF0000u), xv, a8[1]);
+          a8[2] = fmaf(__uint_as_float(w.y << 16), xv, a8[2]);
+          a8[3] = fmaf(__uint_as_float(w.y & 0xFFFF0000u), xv, a8[3]);
+          a8[4] = fmaf(__uint_as_float(w.z << 16), xv, a8[4]);
+          a8[5] = fmaf(__uint_as_float(w.z & 0xFFFF0000u), xv, a8[5]);
+          a8[6] = fmaf(__uint_as_float(w.w << 16), xv, a8[6]);
+          a8[7] = fmaf(__uint_as_float(w.w & 0xFFFF0000u), xv, a8[7]);
         }
       }
-      if (!ok && !*abort) fail(p, misc);
+#pragma unroll 1
       for (int o = LPR; o < 32; o <<= 1) {
 #pragma unroll
-        for (int v = 0; v < VPL; ++v)
-#pragma unroll
-          for (int e = 0; e < 8; ++e) accv[v][e] += __shfl_xor_sync(0xffffffffu, accv[v][e], o);
+        for (int e = 0; e < 8; ++e) a8[e] += __shfl_xor_sync(0xffffffffu, a8[e], o);
       }
-      if (sub == 0) {
-#pragma unroll
-        for (int v = 0; v < VPL; ++v)
-#pragma unroll
-          for (int e = 0; e < 8; ++e) s_red[warp * 512 + (cl + v * LPR) * 8 + e] = accv[v][e];
+      if (q.sub == 0) {
+        float4* dst = reinterpret_cast<float4*>(s_red + warp * 512 + cv * 8);
+        dst[0] = make_float4(a8[0], a8[1], a8[2], a8[3]);
+        dst[1] = make_float4(a8[4], a8[5], a8[6], a8[7]);
       }
-      csync();
-      if (*abort) return false;
-      if (s.p1 > s.p0) {
-        for (int j = tid; j < k; j += kNC) {
-          float sum = 0.f;
-#pragma unroll
-          for (int w = 0; w < kNW; ++w) sum += s_red[w * 512 + j];
-          const long long q = scale != 0.0 ? __double2ll_rn((double)sum * scale) : 0ll;
-          red_add_u64(acc + j, (1ull << kCountShift) + (unsigned long long)q);
-        }
-      }
-
-      // ---- C. exchange 1: wait until every contributing CTA has been added
+    }
+    if (!ok && !*abort) fail(p, misc);
+    tr.mark(3);
+    csync();
+    if (*abort) return false;
+    if (prow > 0) {
+#pragma unroll 1
       for (int j = tid; j < k; j += kNC) {
-        unsigned long long w = 0;
-        unsigned it = 0;
-        for (;;) {
-          w = ld_relaxed_u64(acc + j);
-          const unsigned cnt = (unsigned)((w + (1ull << (kCountShift - 1))) >> kCountShift);
-          if (cnt == (unsigned)n_contrib) break;
-          if (++it > kSpinLimit || ((it & 1023u) == 0 && *abort)) {
-            if (!*abort) fail(p, misc);
-            break;
-          }
-        }
-        const long long val = (long long)(w - ((unsigned long long)n_contrib << kCountShift));
-        s_c[j] = (float)((double)val * inv_scale);
-      }
-      csync();
-      if (*abort) return false;
-
-      // ---- D. pass 2 (residual rows) and the image rows
-      float c8[VPL][8];
+        float sum = 0.f;
 #pragma unroll
-      for (int v = 0; v < VPL; ++v) {
-        const float4 a = *reinterpret_cast<const float4*>(s_c + (cl + v * LPR) * 8);
-        const float4 b = *reinterpret_cast<const float4*>(s_c + (cl + v * LPR) * 8 + 4);
-        c8[v][0] = a.x; c8[v][1] = a.y; c8[v][2] = a.z; c8[v][3] = a.w;
-        c8[v][4] = b.x; c8[v][5] = b.y; c8[v][6] = b.z; c8[v][7] = b.w;
+        for (int w = 0; w < kNW; ++w) sum += s_red[w * 512 + j];
+        const long long v = scale != 0.0 ? __double2ll_rn((double)sum * scale) : 0ll;
+        red_add_u64(acc + (size_t)j * kAccStride, (1ull << kCountShift) + (unsigned long long)v);
       }
-      float sr = 0.f;
-      for (int ci = 0; ci < pchunks; ++ci) {
+    }
+    tr.mark(4);
+
+    // ---- C. exchange 1: wait until every contributing CTA has been added.  One
+    //      thread watches one word (thousands of pollers on the accumulators
+    //      would delay the very atomics they wait for); then every thread
+    //      validates its own word, which is normally complete by then.
+    if (tid == 0) {
+      const unsigned long long* wp = acc + (size_t)(k - 1) * kAccStride;
+      unsigned it = 0;
+      for (;;) {
+        const unsigned long long w = ld_relaxed_u64(wp);
+        if ((unsigned)((w + (1ull << (kCountShift - 1))) >> kCountShift) == (unsigned)n_contrib) break;
+        if (++it > kSpinLimit || ((it & 1023u) == 0 && *abort)) {
+          if (!*abort) fail(p, misc);
+          break;
+        }
+      }
+    }
+    csync();
+    if (*abort) return false;
+#pragma unroll 1
+    for (int j = tid; j < k; j += kNC) {
+      unsigned long long w = 0;
+      unsigned it = 0;
+      for (;;) {
+        w = ld_relaxed_u64(acc + (size_t)j * kAccStride);
+        const unsigned cnt = (unsigned)((w + (1ull << (kCountShift - 1))) >> kCountShift);
+        if (cnt == (unsigned)n_contrib) break;
+        if (++it > kSpinLimit || ((it & 1023u) == 0 && *abort)) {
+          if (!*abort) fail(p, misc);
+          break;
+        }
+      }
+      const long long val = (long long)(w - ((unsigned long long)n_contrib << kCountShift));
+      s_c[j] = (float)((double)val * inv_scale);
+    }
+    csync();
+    if (*abort) return false;
+    tr.mark(5);
+
+    // ---- D. pass 2 (residual rows of the basis chunks, still in the ring) and
+    //      the image rows: the same eight-rows-per-lane-group loop over both
+    const int hold_log2 = q.lpr_log2 - 3;  // lanes per held row after reduce8
+    // all image chunks of this group must have landed (they were prefetched)
+#pragma unroll 1
+    for (int ci = 0; ci < ochunks; ++ci) {
+      const unsigned seq = n_p0 + pchunks + ci;
+      ok = ok && mbar_wait(&full[seq % kSlots], (seq / kSlots) & 1u, abort);
+    }
+    tr.mark(7);
+    float sr = 0.f;
+    if (ok) {
+      // work items: lane groups take eight rows at a time; item -> (chunk, rows)
+      const int ipc_log2 = q.rc_log2 - 3;              // items per chunk
+      const int n_items = (pchunks + ochunks) << ipc_log2;
+      const int lanegroups = kNW << rpp_log2;          // lane groups in the CTA
+      int released = 0;  // chunks this warp has already given back to the producer
+#pragma unroll 1
+      for (int item = (warp << rpp_log2) + q.sub; item < n_items; item += lanegroups) {
+        const int ci = item >> ipc_log2;
+        // items come in chunk order: every chunk before this warp's current one is done
+        // (n_items is a multiple of the lane groups per warp, so the warp stays converged)
+        const int ci_warp = __shfl_sync(0xffffffffu, ci, 0);
+        if (lane == 0)
+          for (; released < ci_warp; ++released) mbar_arrive(&empty[(n_p0 + released) % kSlots]);
+        released = ci_warp;
+        const bool image = ci >= pchunks;
+        const int cj = image ? ci - pchunks : ci;
         const unsigned sl = (n_p0 + ci) % kSlots;
         const uint4* tile = reinterpret_cast<const uint4*>(ring + (size_t)sl * kChunk);
-        const int r_lo = ci * rc, rows = min(rc, s.p1 - s.p0 - r_lo);
-        for (int base = warp * RPP; base < rows; base += kNW * RPP) {
-          const int row = base + sub;
-          float dot = 0.f;
-          if (row < rows) {
-#pragma unroll
-            for (int v = 0; v < VPL; ++v) {
-              float p8[8];
-              unpack_bf16x8(tile[(size_t)row * KV + cl + v * LPR], p8);
-#pragma unroll
-              for (int e = 0; e < 8; ++e) dot = fmaf(p8[e], c8[v][e], dot);
-            }
-          }
-          for (int o = LPR >> 1; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-          if (row < rows && cl == 0) {
+        const int r_lo = cj << q.rc_log2, rows = min(rc, (image ? orow : prow) - r_lo);
+        const int row0 = (item & ((1 << ipc_log2) - 1)) << 3;
+        float v[8];
+        dot8(tile, s_c, q, row0, rows, v);
+        const float dot = reduce8(v, q.cl, LPR);
+        const int row = row0 + (q.cl >> hold_log2);
+        if ((q.cl & ((1 << hold_log2) - 1)) == 0 && row < rows) {
+          if (image) {
+            g.y[s.o0 + r_lo + row] = nonfinite ? __int_as_float(0x7fc00000) : dot;
+          } else {
             const float rv = s_x[r_lo + row] - dot;
             g.r[s.p0 + r_lo + row] = rv;
             sr = fmaf(rv, rv, sr);
           }
         }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty[sl]);
-      }
-      n += pchunks;
-      const int ochunks = n_chunks(s.o1 - s.o0, rc);
-      for (int ci = 0; ci < ochunks; ++ci) {
-        const unsigned sl = (n + ci) % kSlots, ph = ((n + ci) / kSlots) & 1u;
-        ok = ok && mbar_wait(&full[sl], ph, abort);
-        if (!ok) break;
-        const uint4* tile = reinterpret_cast<const uint4*>(ring + (size_t)sl * kChunk);
-        const int r_lo = ci * rc, rows = min(rc, s.o1 - s.o0 - r_lo);
-        for (int base = warp * RPP; base < rows; base += kNW * RPP) {
-          const int row = base + sub;
-          float dot = 0.f;
-          if (row < rows) {
-#pragma unroll
-            for (int v = 0; v < VPL; ++v) {
-              float p8[8];
-              unpack_bf16x8(tile[(size_t)row * KV + cl + v * LPR], p8);
-#pragma unroll
-              for (int e = 0; e < 8; ++e) dot = fmaf(p8[e], c8[v][e], dot);
-            }
-          }
-          for (int o = LPR >> 1; o > 0; o >>= 1) dot += __shfl_xor_sync(0xffffffffu, dot, o);
-          if (row < rows && cl == 0)
-            g.y[s.o0 + r_lo + row] = nonfinite ? __int_as_float(0x7fc00000) : dot;
-        }
-        __syncwarp();
-        if (lane == 0) mbar_arrive(&empty[sl]);
-      }
-      if (!ok && !*abort) fail(p, misc);
-      n += ochunks;
-      sr = warp_sum(sr);
-      if (lane == 0) s_red[warp] = sr;
-      csync();
-      if (*abort) return false;
-
-      // ---- E. exchange 2: publish, collect, decide
-      if (tid == 0) {
-        float t = 0.f;
-        for (int w = 0; w < kNW; ++w) t += s_red[w];
-        // release: this CTA's y and r rows are visible to whoever reads the word
-        st_release_u64(g.slot_r + cta,
-                       ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(t));
-      }
-      for (int t = tid; t < G; t += kNC) {
-        unsigned long long w = 0;
-        unsigned it = 0;
-        for (;;) {
-          w = ld_relaxed_u64(g.slot_r + t);
-          if ((unsigned)(w >> 32) == tag) break;
-          if (++it > kSpinLimit || ((it & 1023u) == 0 && *abort)) {
-            if (!*abort) fail(p, misc);
-            break;
-          }
-        }
-        s_vals[t] = __uint_as_float((unsigned)w);
-      }
-      __threadfence();  // acquire side of the published words
-      csync();
-      if (*abort) return false;
-      if (tid == 0) {
-        double srt = 0.0;
-        for (int t = 0; t < G; ++t) srt += (double)s_vals[t];
-        const double nr = sqrt(srt), nx = sqrt((double)misc->sum2);
-        const bool fast = !nonfinite && (nr < (double)g.eps * nx);
-        misc->gate = fast ? 0 : 1;
-        if (cta == 0) {
-          const size_t at = (size_t)slot_io * p.log_step_stride + gi;
-          p.gate_log[at] = fast ? 0 : 1;
-          if (p.rho_log) p.rho_log[at] = nonfinite ? __int_as_float(0x7fc00000) : (float)(nr / nx);
-        }
-      }
-      csync();
-      gate = misc->gate && !(g.flags & GSI_FLAG_STATIC_PROJECTION) && !nonfinite;
-      rsrc = g.r;
-    } else {
-      if (cta == gi % G && tid == 0) g.bar[parity ^ 1u] = 0u;
-      if (cta == 0 && tid == 0) p.gate_log[(size_t)slot_io * p.log_step_stride + gi] = 1;
-    }
-
-    // ---- F. gated residual: y_rows (+)= W_rows . r   (dense baseline: r := x)
-    if (gate) {
-      const int rows = s.o1 - s.o0;
-      const int nsl = (g.d + kSlice - 1) / kSlice;
-      for (int sl = 0; sl < nsl; ++sl) {
-        const int c0 = sl * kSlice, cols = min(kSlice, g.d - c0), nv = cols / 16;
-        csync();
-        for (int v = tid; v < nv; v += kNC) {
-          const float4* src = reinterpret_cast<const float4*>(rsrc + c0 + v * 16);
-#pragma unroll
-          for (int q = 0; q < 4; ++q) s_rq[q * 256 + v] = __ldcg(src + q);
-        }
-        csync();
-        for (int rw = warp; rw < rows; rw += kNW) {
-          const int a = s.o0 + rw;
-          int j = 0;
-          while (j + 1 < g.n_maps && a >= g.off[j + 1]) ++j;
-          const uint16_t* wrow = g.W[j] + (size_t)(a - g.off[j]) * g.d + c0;
-          float acc = 0.f;
-          for (int v0 = lane; v0 < nv; v0 += 4 * 32) {
-            uint32_t w[4][8];
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              const int v = v0 + u * 32;
-              if (v < nv) ld256_stream(wrow + (size_t)v * 16, w[u]);
-            }
-#pragma unroll
-            for (int u = 0; u < 4; ++u) {
-              const int v = v0 + u * 32;
-              if (v < nv) {
-#pragma unroll
-                for (int q = 0; q < 4; ++q) {
-                  const float4 rr = s_rq[q * 256 + v];
-                  const uint32_t lo = w[u][2 * q], hi = w[u][2 * q + 1];
-                  acc = fmaf(__uint_as_float(lo << 16), rr.x, acc);
-                  acc = fmaf(__uint_as_float(lo & 0xFFFF0000u), rr.y, acc);
-                  acc = fmaf(__uint_as_float(hi << 16), rr.z, acc);
-                  acc = fmaf(__uint_as_float(hi & 0xFFFF0000u), rr.w, acc);
-                }
-              }
-            }
-          }
-          acc = warp_sum(acc);
-          if (lane == 0) s_yacc[rw] = (sl == 0 ? 0.f : s_yacc[rw]) + acc;
-        }
       }
       __syncwarp();
-      for (int rw = warp; rw < rows; rw += kNW) {
-        if (lane == 0) {
-          float* yp = g.y + s.o0 + rw;
-          *yp = dense ? s_yacc[rw] : (*yp + s_yacc[rw]);
-        }
+      if (lane == 0) {
+#pragma unroll 1
+        for (; released < pchunks + ochunks; ++released)
+          mbar_arrive(&empty[(n_p0 + released) % kSlots]);
       }
-      // grid barrier: the next group may read every row of y
-      csync();
-      if (tid == 0) {
-        red_release_u32(g.bar + parity, 1u);
-        unsigned it = 0;
-        while (ld_acquire_u32(g.bar + parity) < (unsigned)G) {
-          if (++it > kSpinLimit || *abort) {
-            if (!*abort) fail(p, misc);
-            break;
+    }
+    tr.mark(8);
+    if (!ok && !*abort) fail(p, misc);
+    n += pchunks + ochunks;
+    sr = warp_sum(sr);
+    if (lane == 0) s_red[warp] = sr;
+    csync();
+    if (*abort) return false;
+
+    // ---- E. exchange 2: publish, collect, decide.  The word carries its own
+    //      launch tag, so no fence is needed for the gate decision itself.
+    if (tid == 0) {
+      float t = 0.f;
+#pragma unroll
+      for (int w = 0; w < kNW; ++w) t += s_red[w];
+      st_relaxed_u64(g.slot_r + cta,
+                     ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(t));
+    }
+    tr.mark(9);
+    if (warp == 0) {
+      // one warp polls all words (lane l owns words l, l+32, ...); each word is
+      // validated by its launch tag
+      float vals[8];
+      unsigned it = 0;
+      bool done = false;
+      while (!done) {
+        bool all = true;
+#pragma unroll
+        for (int i = 0; i < 8; ++i) {
+          const int t = lane + 32 * i;
+          vals[i] = 0.f;
+          if (t < G) {
+            const unsigned long long w = ld_relaxed_u64(g.slot_r + t);
+            all = all && ((unsigned)(w >> 32) == tag);
+            vals[i] = __uint_as_float((unsigned)w);
           }
         }
+        done = __all_sync(0xffffffffu, all);
+        if (!done && (++it > kSpinLimit || ((it & 1023u) == 0 && *abort))) {
+          if (!*abort && lane == 0) fail(p, misc);
+          break;
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 8; ++i) s_vals[lane + 32 * i] = vals[i];
+    }
+    csync();
+    tr.mark(10);
+    if (*abort) return false;
+    {  // every warp folds the 256 slots in the same fixed order
+      float t = 0.f;
+#pragma unroll
+      for (int i = 0; i < 8; ++i) t += s_vals[lane + 32 * i];
+      t = warp_sum(t);
+      // ||r|| < eps ||x||  <=>  ||r||^2 < eps^2 ||x||^2  (both sides >= 0); NaN compares false
+      const double e2 = (double)g.eps * (double)g.eps;
+      const bool fast = !nonfinite && ((double)t < e2 * (double)sum2);
+      gate = fast ? 0 : 1;
+      if (cta == 0 && tid == 0) {
+        const size_t at = (size_t)slot_io * p.log_step_stride + gi;
+        p.gate_log[at] = (unsigned char)gate;
+        if (p.rho_log)
+          p.rho_log[at] = nonfinite ? __int_as_float(0x7fc00000) : sqrtf(__fdividef(t, sum2));
+      }
+    }
+    gate = gate && !(g.flags & GSI_FLAG_STATIC_PROJECTION) && !nonfinite;
+    rsrc = g.r;
+    tr.mark(11);
+  } else {
+    if (zeroer && tid < 3) g.bar[2 * tid + (parity ^ 1u)] = 0u;
+    if (cta == 0 && tid == 0) p.gate_log[(size_t)slot_io * p.log_step_stride + gi] = 1;
+    if (has_next && tid < kDescWords)
+      reinterpret_cast<uint32_t*>(smem + kOffDesc + ((gi + 1) % 3) * 512)[tid] = desc_word;
+    csync();
+    if (has_next) prefetch_next_x(g_next, slot_io);
+  }
+
+  if (gate) {
+    if (!dense) {
+      // r was written by every CTA: make it visible grid-wide before anyone reads it
+      // (release fence, arrival count, acquire fence).  Only gated groups pay for this.
+      if (tid == 0) {
+        __threadfence();
+        grid_arrive_wait(g.bar + 2 + parity, (unsigned)G, p, misc);
+        __threadfence();
       }
       csync();
       if (*abort) return false;
     }
+    gated_pass(g, s, rsrc, dense, smem);
+    // no CTA starts the next group before all have finished this one
+    csync();
+    tr.mark(12);
+    if (tid == 0) grid_arrive_wait(g.bar + parity, (unsigned)G, p, misc);
+    csync();
+    tr.mark(13);
+    if (*abort) return false;
   }
   return true;
 }
@@ -573,11 +779,14 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
   ctx.parity = (unsigned)epoch & 1u;
   ctx.tag = (unsigned)epoch + 1u;
   ctx.n = 0;
+  ctx.tr.start(p);
+  if (p.n_groups > 0 && threadIdx.x < kDescWords)
+    reinterpret_cast<uint32_t*>(smem + kOffDesc)[threadIdx.x] =
+        __ldg(reinterpret_cast<const uint32_t*>(p.groups) + threadIdx.x);
+  csync();
   bool ok = true;
-  for (int gi = 0; gi < p.n_groups && ok; ++gi) {
-    const int k = p.groups[gi].k;
-    ok = (k <= 256) ? group_phase<1>(p, smem, misc, ctx, gi) : group_phase<2>(p, smem, misc, ctx, gi);
-  }
+#pragma unroll 1
+  for (int gi = 0; gi < p.n_groups && ok; ++gi) ok = group_phase(p, smem, misc, ctx, gi);
   // Every CTA read the counters at its start and has since taken part in the
   // last group's exchange, so they may advance now.
   if (blockIdx.x == 0 && threadIdx.x == 0 && ok) {
@@ -621,7 +830,18 @@ __global__ void k_abs_max_bf16(const uint16_t* __restrict__ p, size_t n, float* 
   if ((threadIdx.x & 31) == 0) atomicMax(reinterpret_cast<int*>(out), __float_as_int(m));
 }
 
+__global__ void k_patch_pmax(PersistGroup* groups, const float* const* pmax_ptrs, int n) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i < n && pmax_ptrs[i]) groups[i].pmax = *pmax_ptrs[i];
+}
+
 }  // namespace
+
+cudaError_t launch_patch_pmax(PersistGroup* groups, const float* const* pmax_ptrs, int n,
+                              cudaStream_t st) {
+  k_patch_pmax<<<(n + 127) / 128, 128, 0, st>>>(groups, pmax_ptrs, n);
+  return cudaGetLastError();
+}
 
 int persist_smem_bytes() { return kSmemBytes; }
 int persist_threads() { return kThreadsP; }

@@ -9,6 +9,7 @@ constexpr int kPersistConsumerWarps = 12;
 constexpr int kPersistMaxPRows = 128;   // basis rows one CTA may own
 constexpr int kPersistMaxORows = 512;   // output rows one CTA may own
 constexpr int kPersistMaxGrid = 256;    // CTAs (exchange-2 slots per group)
+constexpr int kAccStride = 16;          // 64-bit words between c accumulators: one per 128-byte line
 
 struct PersistGroup {
   const uint16_t* P;                 // [d][k] bf16
@@ -19,13 +20,13 @@ struct PersistGroup {
   int d, k, O;
   float eps;
   unsigned flags;
-  const float* pmax;                 // device scalar: max |P|
+  float pmax;                        // max |P| (patched in on the device at bind time)
   const float* x;                    // [n_steps][d]
   float* y;                          // [O]
   float* r;                          // [d]
-  unsigned long long* acc_c;         // [2][k] fixed-point accumulators, one set per launch parity
+  unsigned long long* acc_c;         // [2][k][kAccStride] fixed-point accumulators, one set per launch parity
   unsigned long long* slot_r;        // [kPersistMaxGrid] (launch tag | partial ||r||^2)
-  unsigned* bar;                     // [2] end-of-residual barrier counters
+  unsigned* bar;                     // [6] arrival counters by launch parity: [0..1] after, [2..3] before the gated residual, [4..5] exchange 2
   int p_rows, o_rows;                // rows per CTA of P and of the outputs
   long long x_step_stride;
 };
@@ -41,11 +42,14 @@ struct PersistParams {
   float* rho_log;              // same shape or nullptr
   int log_step_stride;
   int* status;
+  unsigned long long* trace;   // device [16] cycle counters of CTA 0, or nullptr
 };
 
 int persist_smem_bytes();
 int persist_threads();
 cudaError_t launch_decode_step(const PersistParams& p, int grid, cudaStream_t st);
 cudaError_t launch_abs_max_bf16(const void* p, size_t n, float* out, cudaStream_t st);
+cudaError_t launch_patch_pmax(PersistGroup* groups, const float* const* pmax_ptrs, int n,
+                              cudaStream_t st);
 
 }  // namespace gsi

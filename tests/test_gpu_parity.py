@@ -397,7 +397,7 @@ def test_persistent_other_ranks_and_flags(k):
 
 def test_persistent_nonfinite_token():
     g = G()
-    x, P, Ws = make_small(256, 32, (64,), 3, seed=41)
+    x, P, Ws = make_small(256, 64, (64,), 3, seed=41)
     x[1, 7] = float("nan")
     lay = g.Layer([W.cuda() for W in Ws], P.cuda(), 0.5, max_tokens=1)
     stack = g.Stack([lay], mode=2)
