@@ -402,7 +402,8 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
       for (int j = 0; j <= gp.n_maps; ++j) pg.off[j] = gp.off[j];
       pg.n_maps = gp.n_maps;
       pg.d = gp.d;
-      pg.k = gp.k;
+      const bool dense_g = gp.flags & GSI_FLAG_DENSE;
+      pg.k = dense_g ? 256 : gp.k;
       pg.O = gp.O;
       pg.eps = gp.eps;
       pg.flags = gp.flags;

@@ -162,7 +162,7 @@ struct Trace {
 
 struct Slab {
   int p0, p1;  // basis rows owned by this CTA
-  int o0, o1;  // rows of the concatenated maps owned by this CTA
+  int o0, o1;  // rows of the concatenated maps owned by this CTA (image rows and W rows)
 };
 __device__ __forceinline__ Slab slab_of(const PersistGroup& g, int cta) {
   Slab s;
@@ -277,34 +277,54 @@ struct Geo {       // lane geometry of one group (k a power of two, 64..512)
   int sub, cl;     // this lane: row sub-group and column lane
 };
 
+// Two-wide fp32 FMA of sm_100: one instruction for a pair of bf16 weights.
+__device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+  return r;
+}
+__device__ __forceinline__ unsigned long long bf16x2_to_f32x2(uint32_t w) {
+  unsigned long long r;
+  asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(w << 16), "r"(w & 0xFFFF0000u));
+  return r;
+}
+__device__ __forceinline__ void fma2(unsigned long long& acc, unsigned long long a,
+                                     unsigned long long b) {
+  asm("fma.rn.f32x2 %0, %1, %2, %0;" : "+l"(acc) : "l"(a), "l"(b));
+}
+__device__ __forceinline__ float sum2(unsigned long long v) {
+  float lo, hi;
+  asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+  return lo + hi;
+}
+
 // out[i] = tile[row0 + i][:] . c   for eight rows, this lane's share of the columns
 __device__ __forceinline__ void dot8(const uint4* tile, const float* s_c, const Geo& q, int row0,
                                      int rows, float (&v)[8]) {
+  unsigned long long acc[8];
 #pragma unroll
-  for (int i = 0; i < 8; ++i) v[i] = 0.f;
+  for (int i = 0; i < 8; ++i) acc[i] = 0ull;
   const int LPR = 1 << q.lpr_log2;
 #pragma unroll 1
   for (int u = 0; u < q.vpl; ++u) {
     const int cv = q.cl + u * LPR;
     const float4 ca = *reinterpret_cast<const float4*>(s_c + cv * 8);
     const float4 cb = *reinterpret_cast<const float4*>(s_c + cv * 8 + 4);
+    const unsigned long long c0 = pack2(ca.x, ca.y), c1 = pack2(ca.z, ca.w);
+    const unsigned long long c2 = pack2(cb.x, cb.y), c3 = pack2(cb.z, cb.w);
 #pragma unroll
     for (int i = 0; i < 8; ++i) {
       if (row0 + i < rows) {
         const uint4 w = tile[(size_t)(row0 + i) * q.KV + cv];
-        float d = v[i];
-        d = fmaf(__uint_as_float(w.x << 16), ca.x, d);
-        d = fmaf(__uint_as_float(w.x & 0xFFFF0000u), ca.y, d);
-        d = fmaf(__uint_as_float(w.y << 16), ca.z, d);
-        d = fmaf(__uint_as_float(w.y & 0xFFFF0000u), ca.w, d);
-        d = fmaf(__uint_as_float(w.z << 16), cb.x, d);
-        d = fmaf(__uint_as_float(w.z & 0xFFFF0000u), cb.y, d);
-        d = fmaf(__uint_as_float(w.w << 16), cb.z, d);
-        d = fmaf(__uint_as_float(w.w & 0xFFFF0000u), cb.w, d);
-        v[i] = d;
+        fma2(acc[i], bf16x2_to_f32x2(w.x), c0);
+        fma2(acc[i], bf16x2_to_f32x2(w.y), c1);
+        fma2(acc[i], bf16x2_to_f32x2(w.z), c2);
+        fma2(acc[i], bf16x2_to_f32x2(w.w), c3);
       }
     }
   }
+#pragma unroll
+  for (int i = 0; i < 8; ++i) v[i] = sum2(acc[i]);
 }
 
 // 2^e as a double, e in the normal range
@@ -385,7 +405,7 @@ __device__ __noinline__ void gated_pass(const PersistGroup& g, const Slab& s, co
   for (int rw = warp; rw < rows; rw += kNW) {
     if (lane == 0) {
       float* yp = g.y + s.o0 + rw;
-      *yp = dense ? s_yacc[rw] : (*yp + s_yacc[rw]);
+      *yp = dense ? s_yacc[rw] : (__ldcg(yp) + s_yacc[rw]);
     }
   }
 }
@@ -448,7 +468,7 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
     q.cl = lane & (LPR - 1);
     const int rpp_log2 = 5 - q.lpr_log2;  // rows per warp pass
     const int rc = 1 << q.rc_log2;
-    const int n_contrib = (g.d + g.p_rows - 1) / g.p_rows;
+    const int n_contrib = (g.d + g.p_rows - 1) / g.p_rows;  // CTAs that own basis rows
     unsigned long long* acc = g.acc_c + (size_t)parity * k * kAccStride;
     const int prow = s.p1 - s.p0, orow = s.o1 - s.o0;
     const int pchunks = (prow + rc - 1) >> q.rc_log2, ochunks = (orow + rc - 1) >> q.rc_log2;

@@ -27,7 +27,7 @@ struct PersistGroup {
   unsigned long long* acc_c;         // [2][k][kAccStride] fixed-point accumulators, one set per launch parity
   unsigned long long* slot_r;        // [kPersistMaxGrid] (launch tag | partial ||r||^2)
   unsigned* bar;                     // [6] arrival counters by launch parity: [0..1] after, [2..3] before the gated residual, [4..5] exchange 2
-  int p_rows, o_rows;                // rows per CTA of P and of the outputs
+  int p_rows, o_rows;                // rows per CTA of P and of the outputs (ceil(rows / CTAs))
   long long x_step_stride;
 };
 
