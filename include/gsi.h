@@ -141,6 +141,41 @@ gsi_status_t gsi_forward_host(gsi_handle_t h, const float* x_host, int n_tokens,
                               float* y_host, unsigned char* gate_mask_host,
                               float* rho_host, gsi_stream_t stream);
 
+/*
+ * The same layer for callers that cannot allocate device memory.  (The paper has
+ * no counterpart: this is a packaging variant of gsi_forward_n, not a method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - a plugin inside
+ * a host application that owns all device memory, a library called while
+ * someone else's stream capture is open, a latency-critical path that may not
+ * enter the allocator.  Such a caller cannot provide the workspace gsi_create
+ * wants.  Here the scratch (coefficients, residual, partial sums, fired-token
+ * list) lives in a fixed array inside the library: about 2.5 MB that every GPU
+ * which loads the library holds until the process exits.
+ *
+ * The caller passes everything else: W_host_array (HOST array of n_maps DEVICE
+ * pointers, W_j [d_out_j][d] bf16), d_out (HOST array), P [d][k], and W_P, the
+ * images of all maps concatenated, [sum d_out][k] bf16, each built once with
+ * gsi_build_image (which does not allocate either).  x [n][d], y [n][sum d_out],
+ * gate_mask_out [n], rho_out [n] or NULL, as in gsi_forward_n.
+ *
+ * Limits: n_tokens <= 4, k <= 512, d <= 16384, n_maps <= GSI_MAX_MAPS; larger
+ * sizes return GSI_ERR_UNSUPPORTED and nothing is launched.
+ *
+ * The first call on each device resolves the array's device address (with that
+ * device current); make that first call before any stream capture begins.  The
+ * call allocates nothing and frees nothing.  All calls on a device share the one
+ * array, which keeps the previous call's contents: the counters that must start
+ * at zero are cleared on `stream` at the start of every call.  Two calls whose
+ * kernels overlap on the GPU (different streams, or one stream per thread) race
+ * on the array - serialise them.
+ */
+gsi_status_t gsi_forward_static(const void* const* W_host_array, const int* d_out, int n_maps,
+                                const void* P, gsi_dtype_t p_dtype, const void* W_P, int d,
+                                int k, float eps, const float* x, int n_tokens, float* y,
+                                unsigned char* gate_mask_out, float* rho_out,
+                                gsi_stream_t stream);
+
 /* Device pointer to the image of map j inside the workspace ([d_out_j][k] bf16),
  * so a caller can inspect or persist it. */
 gsi_status_t gsi_get_image(gsi_handle_t h, int map, const void** W_P_out);

@@ -19,7 +19,7 @@ GSI_MAX_MAPS, GSI_MAX_TOKENS = 8, 64
 
 EXPORTED = [
     "gsi_status_string", "gsi_build_image", "gsi_workspace_bytes", "gsi_create",
-    "gsi_forward", "gsi_forward_n", "gsi_forward_host", "gsi_get_image", "gsi_get_status",
+    "gsi_forward", "gsi_forward_n", "gsi_forward_host", "gsi_forward_static", "gsi_get_image", "gsi_get_status",
     "gsi_destroy", "gsi_stack_workspace_bytes", "gsi_stack_create", "gsi_stack_bind",
     "gsi_stack_set_mode", "gsi_stack_is_persistent", "gsi_stack_set_trace", "gsi_stack_seek", "gsi_stack_step", "gsi_stack_launches_per_step",
     "gsi_stack_step_host", "gsi_stack_get_status", "gsi_stack_destroy",
@@ -59,6 +59,8 @@ def _load():
     l.gsi_forward.argtypes = [vp, vp, vp, vp, vp]
     l.gsi_forward_n.argtypes = [vp, vp, i, vp, vp, vp, vp]
     l.gsi_forward_host.argtypes = [vp, vp, i, vp, vp, vp, vp]
+    l.gsi_forward_static.argtypes = [C.POINTER(vp), C.POINTER(i), i, vp, i, vp, i, i, C.c_float,
+                                     vp, i, vp, vp, vp, vp]
     l.gsi_get_image.argtypes = [vp, i, C.POINTER(vp)]
     l.gsi_get_status.argtypes = [vp, C.POINTER(i)]
     l.gsi_destroy.argtypes = [vp]
@@ -132,6 +134,31 @@ def gsi_build_image(W: torch.Tensor, P: torch.Tensor, out: torch.Tensor | None =
     _check(lib.gsi_build_image(W.data_ptr(), P.data_ptr(), o, d, k, _dtype_code(P),
                                out.data_ptr(), _stream_ptr(stream)), "gsi_build_image")
     return out
+
+
+def gsi_forward_static(Ws, P, W_P, eps, x, y=None, gate=None, rho=None, stream=None):
+    """Algorithm 1 through the entry point that allocates nothing inside the
+    library: scratch comes from an array built into ``libgsi_b200.so``.  For
+    callers that may not call cudaMalloc (see ``include/gsi.h``).  ``W_P`` is the
+    concatenation of ``gsi_build_image(W_j, P)`` over the maps.  The output
+    tensors are allocated HERE, by torch, only when the caller passes none."""
+    Ws = list(Ws)
+    n = int(x.shape[0])
+    d, k = int(P.shape[0]), int(P.shape[1])
+    d_out = [int(W.shape[0]) for W in Ws]
+    if y is None:
+        y = torch.empty((n, sum(d_out)), dtype=torch.float32, device=x.device)
+    if gate is None:
+        gate = torch.empty(n, dtype=torch.uint8, device=x.device)
+    if rho is None:
+        rho = torch.empty(n, dtype=torch.float32, device=x.device)
+    warr = (C.c_void_p * len(Ws))(*[W.data_ptr() for W in Ws])
+    darr = (C.c_int * len(Ws))(*d_out)
+    _check(lib.gsi_forward_static(warr, darr, len(Ws), P.data_ptr(), _dtype_code(P),
+                                  W_P.data_ptr(), d, k, float(eps), x.data_ptr(), n,
+                                  y.data_ptr(), gate.data_ptr(), rho.data_ptr(),
+                                  _stream_ptr(stream)), "gsi_forward_static")
+    return y, gate, rho
 
 
 class Layer:
