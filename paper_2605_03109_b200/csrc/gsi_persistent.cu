@@ -21,7 +21,8 @@
 //
 // Every wait is bounded; a wait that gives up records GSI_ERR_TIMEOUT in the
 // status word, the CTA drains its copies in flight and returns.
-#include <cooperative_groups.h>
+#include <cstdio>
+#include <cstdlib>
 
 #include "gsi_common.cuh"
 #include "gsi_persistent.cuh"
@@ -36,6 +37,7 @@ constexpr int kThreadsP = kNC + 32;         // + producer warp
 constexpr int kSlots = 10;
 constexpr int kChunk = 16384;
 constexpr int kSlice = 4096;                // columns of W per staged slice of r
+constexpr int kWLoads = 4;                  // 256-bit loads per lane in flight in the W stream
 constexpr unsigned kSpinLimit = 1u << 22;
 constexpr int kCountShift = 54;
 
@@ -365,23 +367,27 @@ __device__ __noinline__ void gated_pass(const PersistGroup& g, const Slab& s, co
       for (int q = 0; q < 4; ++q) s_rq[q * 256 + v] = __ldcg(sp + q);
     }
     csync();
-#pragma unroll 1
-    for (int rw = warp; rw < rows; rw += kNW) {
+    auto row_ptr = [&](int rw) -> const uint16_t* {
       const int a = s.o0 + rw;
       int j = 0;
       while (j + 1 < g.n_maps && a >= g.off[j + 1]) ++j;
-      const uint16_t* wrow = g.W[j] + (size_t)(a - g.off[j]) * g.d + c0;
+      return g.W[j] + (size_t)(a - g.off[j]) * g.d + c0;
+    };
+    // kWLoads x 256-bit loads per lane are in flight before the first FMA.
+#pragma unroll 1
+    for (int rw = warp; rw < rows; rw += kNW) {
+      const uint16_t* wrow = row_ptr(rw);
       float acc = 0.f;
 #pragma unroll 1
-      for (int v0 = lane; v0 < nv; v0 += 4 * 32) {
-        uint32_t w[4][8];
+      for (int v0 = lane; v0 < nv; v0 += kWLoads * 32) {
+        uint32_t w[kWLoads][8];
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < kWLoads; ++u) {
           const int v = v0 + u * 32;
           if (v < nv) ld256_stream(wrow + (size_t)v * 16, w[u]);
         }
 #pragma unroll
-        for (int u = 0; u < 4; ++u) {
+        for (int u = 0; u < kWLoads; ++u) {
           const int v = v0 + u * 32;
           if (v < nv) {
 #pragma unroll
@@ -885,8 +891,11 @@ cudaError_t launch_decode_step(const PersistParams& p, int grid, cudaStream_t st
   void* args[] = {&pp};
   // cooperative launch: all CTAs are guaranteed co-resident, which the
   // cross-CTA exchanges rely on
-  return cudaLaunchCooperativeKernel((void*)k_decode_step, dim3(grid), dim3(kThreadsP), args,
-                                     kSmemBytes, st);
+  cudaError_t e = cudaLaunchCooperativeKernel((void*)k_decode_step, dim3(grid), dim3(kThreadsP),
+                                              args, kSmemBytes, st);
+  if (e != cudaSuccess && getenv("GSI_VERBOSE"))
+    fprintf(stderr, "gsi: persistent launch failed: %s\n", cudaGetErrorString(e));
+  return e;
 }
 
 }  // namespace gsi

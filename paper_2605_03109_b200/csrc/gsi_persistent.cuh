@@ -5,7 +5,7 @@
 
 namespace gsi {
 
-constexpr int kPersistConsumerWarps = 12;
+constexpr int kPersistConsumerWarps = 15;  // + 1 producer warp = 16 warps: registers are allotted per 4 warps
 constexpr int kPersistMaxPRows = 128;   // basis rows one CTA may own
 constexpr int kPersistMaxORows = 512;   // output rows one CTA may own
 constexpr int kPersistMaxGrid = 256;    // CTAs (exchange-2 slots per group)
