@@ -28,6 +28,9 @@ if ROOT not in sys.path:
 
 METRIC = "decode tokens/s at GPT-J shapes, k=256, eps=0.05 (effective weight GB/s and % of HBM roofline alongside)"
 NOMINAL_HBM_GBS = 8000.0
+# dram bytes (read+write) per algorithmic byte of k_decode_step from the ncu capture summarised in
+# profiles/k_decode_step_gptj_L8_ncu_full.md (8-layer case; traffic grows in proportion to layers)
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.02
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -273,6 +276,9 @@ def main():
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--profile", action="store_true",
+                    help="profiling run: build the stack, launch warmup+steps plain decode steps "
+                         "(no graph, no dense arm, no host legs) and exit; for ncu captures")
     args = ap.parse_args()
     if args.impl == "gsi":
         args.steps = 256 if args.steps is None else args.steps
@@ -311,6 +317,15 @@ def main():
     layers, dense_layers, xs, keep = build_workload(spec, device, n_steps)
     stack = G.Stack(layers)
     stack.bind(xs, n_steps=n_steps)
+    if args.profile:
+        for _ in range(args.warmup + args.steps):
+            stack.step()
+        torch.cuda.synchronize()
+        print(json.dumps({"profile": True, "workload": spec.name, "launches": args.warmup + args.steps,
+                          "launches_per_step": stack.launches_per_step(),
+                          "status": stack.status(),
+                          "gate_rate": float(stack.gate_log.float().mean().item())}))
+        return
     dstack = G.Stack(dense_layers)
     dstack.bind(xs, n_steps=n_steps, want_rho=False)
     stream = torch.cuda.Stream(device)
@@ -374,8 +389,12 @@ def main():
             "bytes_per_step": {k: float(v) for k, v in ab.items()},
             "roofline": {
                 "bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                "frac": achieved / peak, "traffic": None,
-                "kernel": "whole decode step (all launches of one graph replay)",
+                "frac": achieved / peak,
+                "traffic": NCU_TRAFFIC_PER_ALGORITHMIC_BYTE * ab["total"],
+                "traffic_note": "ncu dram bytes of an 8-layer capture scaled by layers (profiles/)",
+                "algorithmic_bytes": ab["total"],
+                "kernel": "k_decode_step (one persistent launch = one decode step)"
+                          if launches == 1 else "whole decode step (all launches of one graph replay)",
                 "peak_source": f"{peak_kind} copy bandwidth",
                 "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS,
             },
