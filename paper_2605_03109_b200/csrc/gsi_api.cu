@@ -19,9 +19,18 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 struct Layout {
   size_t wp, c, cpart, r, normpart, ctrl, fired, rho, x_stage, y_stage, gate_stage, rho_stage,
-      pk_acc, pk_slot, total;
+      pk_acc, pk_slot, tc_rb, tc_ypart, total;
   int O, n_slabs, slab_rows;
+  bool tc;
 };
+
+constexpr int kTcMinFired = 5;  // fewer fired tokens: one pass of the CUDA-core GEMV
+
+bool tc_shapes_ok(const gsi_desc_t* d) {
+  for (int j = 0; j < d->n_maps; ++j)
+    if (d->d_out[j] % 128) return false;
+  return true;
+}
 
 gsi_status_t check_desc(const gsi_desc_t* d) {
   if (!d || !d->d_out) return GSI_ERR_INVALID_ARG;
@@ -68,6 +77,11 @@ Layout make_layout_ws(const gsi_desc_t* d) {
   L.rho_stage = take(B * 4);
   L.pk_acc = take(2 * k * 8 * kAccStride);          // persistent kernel: c accumulators
   L.pk_slot = take((size_t)kPersistMaxGrid * 8);    // persistent kernel: ||r||^2 words
+  // tensor-core gated residual: only for batches that can fire at least kTcMinFired tokens
+  const bool tc = !dense && d->max_tokens >= kTcMinFired && d->d % 64 == 0 && tc_shapes_ok(d);
+  L.tc_rb = take(tc ? (size_t)64 * d->d * 2 : 0);
+  L.tc_ypart = take(tc ? (size_t)tc_splits(O, d->d) * 64 * O * 4 : 0);
+  L.tc = tc;
   L.total = at;
   return L;
 }
@@ -195,6 +209,9 @@ gsi_status_t gsi_create(const gsi_desc_t* desc, const void* const* W, const void
   g.rho_scratch = reinterpret_cast<float*>(h->ws + L.rho);
   g.n_slabs = L.n_slabs;
   g.slab_rows = L.slab_rows;
+  g.tc_min_fired = L.tc ? kTcMinFired : 0;
+  g.rb = reinterpret_cast<uint16_t*>(h->ws + L.tc_rb);
+  g.ypart = reinterpret_cast<float*>(h->ws + L.tc_ypart);
 
   if (cudaMemsetAsync(ctrl, 0, 256, stream) != cudaSuccess ||
       cudaMemsetAsync(h->ws + L.pk_acc, 0, L.total - L.pk_acc, stream) != cudaSuccess) {
@@ -493,7 +510,7 @@ gsi_status_t gsi_stack_launches_per_step(gsi_stack_t s, int* n_out) {
   int n = 0;
   for (gsi_layer* h : s->groups) {
     if (h->desc.flags & GSI_FLAG_DENSE) n += 1;
-    else n += (h->desc.flags & GSI_FLAG_STATIC_PROJECTION) ? 4 : 5;
+    else n += (h->desc.flags & GSI_FLAG_STATIC_PROJECTION) ? 4 : (h->gp.tc_min_fired ? 8 : 5);
   }
   *n_out = n + 1;
   return GSI_OK;

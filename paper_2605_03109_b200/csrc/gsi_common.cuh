@@ -93,11 +93,19 @@ struct GroupParams {
   float* rho_scratch; // [B]
   int* status;      // [1]
   int n_slabs, slab_rows;
+  // tensor-core gated residual (batched): used when at least tc_min_fired tokens fired
+  int tc_min_fired;   // 0 = disabled
+  uint16_t* rb;       // [64][d] bf16: residuals of the fired tokens, compacted
+  float* ypart;       // [splits][64][O] split-K partial sums
 };
 
 cudaError_t launch_generic_forward(const GroupParams& g, const IoRef& io, int n_tokens,
                                    cudaStream_t stream, int* n_launches);
 cudaError_t launch_advance_step(int* step, cudaStream_t stream);
+cudaError_t launch_residual_gemm_tc(const GroupParams& g, const IoRef& io, int min_fired,
+                                    cudaStream_t stream, int* n_launches);
+int tc_splits(int O, int d);
+bool tc_eligible(const GroupParams& g);
 cudaError_t launch_build_image(const void* W, const void* P, int o, int d, int k, bool p_f32,
                                void* WP, cudaStream_t stream);
 

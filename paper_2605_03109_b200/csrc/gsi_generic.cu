@@ -296,6 +296,7 @@ __global__ void __launch_bounds__(kThreads)
 k_stream_gemv(GroupParams g, IoRef io, int n_tokens) {
   const int n = kDense ? n_tokens : *g.n_fired;
   if (n == 0) return;
+  if (!kDense && g.tc_min_fired > 0 && n >= g.tc_min_fired) return;  // tensor-core path takes it
   const int slot = io_slot(io);
   const float* src = kDense ? io.x + (long long)slot * io.x_step_stride : g.r;
   const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -418,6 +419,10 @@ cudaError_t launch_generic_forward(const GroupParams& g, const IoRef& io, int n_
   if (!(g.flags & GSI_FLAG_STATIC_PROJECTION)) {
     k_stream_gemv<false><<<grid, kThreads, 0, st>>>(g, io, n_tokens);
     *n_launches += 1;
+    if (g.tc_min_fired > 0) {
+      e = launch_residual_gemm_tc(g, io, g.tc_min_fired, st, n_launches);
+      if (e != cudaSuccess) return e;
+    }
   }
   return cudaGetLastError();
 }
