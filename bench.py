@@ -150,16 +150,37 @@ def time_graph(graph, stack, stream, steps, warmup, barrier=None):
     return e0.elapsed_time(e1) / steps  # ms per step
 
 
-def time_host_steps(stack, xs, steps, warmup, stream):
-    """End-to-end: host buffers in, host buffers out, copies inside the timed region."""
+def time_host_steps(layers, xs, steps, warmup, stream):
+    """End-to-end: host buffers in, host buffers out, copies inside the timed region.
+    The device and pinned host buffers of all groups are carved out of one arena each,
+    so a step is one H2D copy, one launch, two D2H copies (y and the gate bytes)."""
     import torch
-    n = len(stack.layers)
-    B = stack.B
-    xs_host = [x[:B].reshape(B, -1).cpu().contiguous().pin_memory() for x in xs]
-    ys_host = [torch.empty((B, l.O), dtype=torch.float32).pin_memory() for l in stack.layers]
+    import paper_2605_03109_b200 as G
+    n = len(layers)
+    B = layers[0].max_tokens
+    dev = layers[0].device
+    dx = [B * l.d for l in layers]
+    dy = [B * l.O for l in layers]
+    x_dev = torch.empty(sum(dx), dtype=torch.float32, device=dev)
+    y_dev = torch.empty(sum(dy), dtype=torch.float32, device=dev)
+    x_host = torch.empty(sum(dx), dtype=torch.float32).pin_memory()
+    y_host = torch.empty(sum(dy), dtype=torch.float32).pin_memory()
+
+    def carve(t, sizes):
+        out, at = [], 0
+        for sz in sizes:
+            out.append(t[at:at + sz])
+            at += sz
+        return out
+    xs_dev, ys_dev = carve(x_dev, dx), carve(y_dev, dy)
+    xs_host, ys_host = carve(x_host, dx), carve(y_host, dy)
+    for xh, x in zip(xs_host, xs):
+        xh.copy_(x[:B].reshape(-1).cpu())
+    stack = G.Stack(layers)
+    stack.bind(xs_dev, ys=[y.view(B, -1) for y in ys_dev], n_steps=1)
     gate_host = torch.empty((n, B), dtype=torch.uint8).pin_memory()
-    h2d = sum(x.numel() * 4 for x in xs_host)
-    d2h = sum(y.numel() * 4 for y in ys_host) + gate_host.numel()
+    h2d = x_host.numel() * 4
+    d2h = y_host.numel() * 4 + gate_host.numel()
     with torch.cuda.stream(stream):
         for _ in range(max(1, warmup)):
             stack.step_host(xs_host, ys_host, gate_host, stream)
@@ -173,6 +194,10 @@ def time_host_steps(stack, xs, steps, warmup, stream):
         stream.synchronize()
         wall = (time.perf_counter() - t0) * 1e3 / steps
     ms = max(e0.elapsed_time(e1) / steps, wall)
+    status = stack.status()
+    stack.close()
+    if status != 0:
+        raise SystemExit(f"device status word {status} in the host-buffer leg")
     return ms, h2d, d2h
 
 
@@ -364,7 +389,7 @@ def main():
 
     e2e = None
     if not args.no_e2e:
-        ms_e2e, h2d, d2h = time_host_steps(stack, xs, max(8, args.steps // 8), 3, stream)
+        ms_e2e, h2d, d2h = time_host_steps(layers, xs, max(8, args.steps // 8), 3, stream)
         e2e = {"value": world * spec.batch * 1e3 / ms_e2e, "unit": "tokens/s",
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 

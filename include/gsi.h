@@ -203,7 +203,9 @@ typedef struct {
 size_t gsi_stack_workspace_bytes(int n_groups);
 
 /* groups_host_array: HOST array of n_groups handles in execution order; all
- * must have the same max_tokens.  The handles must outlive the stack. */
+ * must have the same max_tokens.  The handles must outlive the stack.  A handle
+ * may belong to several stacks, but only the stack bound LAST may be stepped:
+ * gsi_stack_bind resets the handles' cross-CTA exchange state. */
 gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups_host_array,
                               void* workspace, size_t workspace_bytes,
                               gsi_stream_t stream, gsi_stack_t* out);
@@ -265,7 +267,9 @@ gsi_status_t gsi_stack_launches_per_step(gsi_stack_t s, int* n_out);
  * current step, run the step, copy every group's y and the step's gate bytes
  * back, synchronise.  x_host_array / y_host_array: HOST arrays [n_groups] of
  * HOST pointers ([max_tokens][d] and [max_tokens][sum d_out]); pinned memory
- * makes the copies asynchronous.  gate_host [n_groups][max_tokens].
+ * makes the copies asynchronous.  gate_host [n_groups][max_tokens].  Groups whose
+ * host buffers AND device buffers are adjacent in memory (carved out of one arena, in
+ * group order) are copied with a single transfer per direction.
  */
 gsi_status_t gsi_stack_step_host(gsi_stack_t s, const float* const* x_host_array,
                                  float* const* y_host_array, unsigned char* gate_host,

@@ -407,6 +407,17 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
     if (s->mode == 2 && !s->persistent) return GSI_ERR_UNSUPPORTED;
   }
   if (s->persistent) {
+    // The cross-CTA exchange state of every group (accumulators, tagged words, arrival
+    // counters) is tied to THIS stack's launch counter: start both from zero.  A handle
+    // can therefore serve only one bound stack at a time.
+    if (cudaMemsetAsync(s->epoch, 0, sizeof(int), stream) != cudaSuccess) return GSI_ERR_CUDA;
+    for (int i = 0; i < G; ++i) {
+      const gsi_layer* h = s->groups[i];
+      if (cudaMemsetAsync(h->ws + h->lay.pk_acc, 0, h->lay.tc_rb - h->lay.pk_acc, stream) !=
+              cudaSuccess ||
+          cudaMemsetAsync(h->bar, 0, 6 * sizeof(unsigned), stream) != cudaSuccess)
+        return GSI_ERR_CUDA;
+    }
     s->host_groups.assign(G, PersistGroup{});
     s->host_pmax_ptrs.assign(G, nullptr);
     for (int i = 0; i < G; ++i) {
@@ -520,22 +531,41 @@ gsi_status_t gsi_stack_step_host(gsi_stack_t s, const float* const* x_host, floa
                                  unsigned char* gate_host, gsi_stream_t stream) {
   if (!s || !s->bound || !x_host || !y_host || !gate_host) return GSI_ERR_INVALID_ARG;
   const int G = (int)s->groups.size();
-  for (int i = 0; i < G; ++i) {
+  for (int i = 0; i < G; ++i)
     if (!x_host[i] || !y_host[i]) return GSI_ERR_INVALID_ARG;
-    const size_t bytes = (size_t)s->B * s->groups[i]->desc.d * 4;
-    if (cudaMemcpyAsync(const_cast<float*>(s->io[i].x), x_host[i], bytes, cudaMemcpyHostToDevice,
-                        stream) != cudaSuccess)
-      return GSI_ERR_CUDA;
-  }
+  // Runs of groups whose buffers are adjacent both on the host and on the device
+  // (a caller that carves them out of one arena) travel as ONE copy.
+  auto copy_runs = [&](bool to_device) -> bool {
+    for (int i = 0; i < G;) {
+      const char* h0 = to_device ? reinterpret_cast<const char*>(x_host[i])
+                                 : reinterpret_cast<const char*>(y_host[i]);
+      const char* d0 = to_device ? reinterpret_cast<const char*>(s->io[i].x)
+                                 : reinterpret_cast<const char*>(s->io[i].y);
+      size_t bytes = 0;
+      int j = i;
+      for (; j < G; ++j) {
+        const size_t b = to_device ? (size_t)s->B * s->groups[j]->desc.d * 4
+                                   : (size_t)s->B * s->groups[j]->lay.O * 4;
+        const char* hj = to_device ? reinterpret_cast<const char*>(x_host[j])
+                                   : reinterpret_cast<const char*>(y_host[j]);
+        const char* dj = to_device ? reinterpret_cast<const char*>(s->io[j].x)
+                                   : reinterpret_cast<const char*>(s->io[j].y);
+        if (hj != h0 + bytes || dj != d0 + bytes) break;
+        bytes += b;
+      }
+      const cudaError_t e =
+          to_device ? cudaMemcpyAsync(const_cast<char*>(d0), h0, bytes, cudaMemcpyHostToDevice, stream)
+                    : cudaMemcpyAsync(const_cast<char*>(h0), d0, bytes, cudaMemcpyDeviceToHost, stream);
+      if (e != cudaSuccess) return false;
+      i = j;
+    }
+    return true;
+  };
+  if (!copy_runs(true)) return GSI_ERR_CUDA;
   s->last_stream = stream;
   gsi_status_t st = stack_enqueue(s, false, stream);
   if (st != GSI_OK) return st;
-  for (int i = 0; i < G; ++i) {
-    const size_t bytes = (size_t)s->B * s->groups[i]->lay.O * 4;
-    if (cudaMemcpyAsync(y_host[i], s->io[i].y, bytes, cudaMemcpyDeviceToHost, stream) !=
-        cudaSuccess)
-      return GSI_ERR_CUDA;
-  }
+  if (!copy_runs(false)) return GSI_ERR_CUDA;
   if (cudaMemcpyAsync(gate_host, s->gate_log, (size_t)G * s->B, cudaMemcpyDeviceToHost, stream) !=
       cudaSuccess)
     return GSI_ERR_CUDA;

@@ -476,3 +476,25 @@ def test_tensor_core_residual_gemm_gptj_shape_sampled_rows():
     Wsamp = [m["W"][0][torch.as_tensor(rows, device="cuda")].cpu()]
     compare_group(m["x"].cpu(), m["P"].cpu(), Wsamp, st.eps, y.cpu().numpy()[:, rows],
                   gate.cpu().numpy(), rho.cpu().numpy())
+
+
+def test_rebinding_a_second_stack_over_the_same_handles():
+    """gsi_stack_bind resets the exchange state of its handles, so a new stack over
+    handles that already ran in another stack works (the older stack must not be
+    stepped again)."""
+    st = S.config2()
+    stack, mats = build_stack(st, 1, 3, mode=2)
+    for _ in range(3):
+        stack.step()
+    torch.cuda.synchronize()
+    assert stack.status() == 0
+    ref = [y.cpu().clone() for y in stack.ys]
+    g = G()
+    again = g.Stack(stack.layers, mode=2)
+    again.bind(stack.xs, n_steps=3)
+    for _ in range(3):
+        again.step()
+    torch.cuda.synchronize()
+    assert again.status() == 0
+    for a, b in zip(ref, again.ys):
+        assert torch.equal(a, b.cpu())
