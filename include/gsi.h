@@ -34,9 +34,12 @@
  *     Argument errors are found on the host before anything is launched.
  *   - Ownership: the caller owns W, P, x, y, the logs and the workspace.  The
  *     library borrows W and P (they must outlive the handle) and owns what it
- *     places in the workspace.  Nothing below allocates device memory; the
- *     forward calls do not synchronise the host and may be stream-captured
- *     (the *_host variants copy and synchronise, and may not).
+ *     places in the workspace.  Nothing below allocates device memory.  The
+ *     set-up calls (gsi_create, gsi_stack_create, gsi_stack_bind) run their
+ *     device work on `stream` and synchronise it before returning, so what they
+ *     built may be used from any stream afterwards; they may not be captured.
+ *     The forward / step calls do not synchronise the host and may be
+ *     stream-captured (the *_host variants copy and synchronise, and may not).
  *   - One handle / stack may be used by one stream at a time.
  */
 #ifndef GSI_H_

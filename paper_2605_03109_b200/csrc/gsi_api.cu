@@ -235,6 +235,12 @@ gsi_status_t gsi_create(const gsi_desc_t* desc, const void* const* W, const void
       }
     }
   }
+  // A set-up call: return only when the images, max|P| and the cleared state are in
+  // place, so the handle may be used from any stream afterwards.
+  if (cudaStreamSynchronize(stream) != cudaSuccess) {
+    delete h;
+    return GSI_ERR_CUDA;
+  }
   *out = h;
   return GSI_OK;
 }
@@ -346,7 +352,8 @@ gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* wo
   s->grid = 0;
   s->bound = false;
   s->last_stream = stream;
-  if (cudaMemsetAsync(workspace, 0, 256, stream) != cudaSuccess) {
+  if (cudaMemsetAsync(workspace, 0, 256, stream) != cudaSuccess ||
+      cudaStreamSynchronize(stream) != cudaSuccess) {
     delete s;
     return GSI_ERR_CUDA;
   }
@@ -456,6 +463,9 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
         launch_patch_pmax(s->dev_groups, dev_ptrs, G, stream) != cudaSuccess)
       return GSI_ERR_CUDA;
   }
+  // A set-up call: the descriptor table and the cleared exchange state must be in
+  // device memory before a step may be enqueued on ANY stream.
+  if (cudaStreamSynchronize(stream) != cudaSuccess) return GSI_ERR_CUDA;
   s->bound = true;
   return GSI_OK;
 }

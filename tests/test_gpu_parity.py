@@ -498,3 +498,27 @@ def test_rebinding_a_second_stack_over_the_same_handles():
     assert again.status() == 0
     for a, b in zip(ref, again.ys):
         assert torch.equal(a, b.cpu())
+
+
+def test_step_on_another_stream_right_after_bind():
+    """Set-up calls finish their device work before returning, so a step may be
+    enqueued on a different (non-blocking) stream immediately afterwards."""
+    st = S.config1_fast()
+    m = S.materialize_group(st, 0, 0, 8)
+    g = G()
+    x = m["x"].cuda().contiguous()
+    Ws = [W.cuda() for W in m["W"]]
+    P = m["P"].cuda()
+    torch.cuda.synchronize()
+    for mode in (2, 1):
+        side = torch.cuda.Stream()
+        lay = g.Layer(Ws, P, st.eps, max_tokens=1)
+        stack = g.Stack([lay], mode=mode)
+        stack.bind([x], n_steps=8)
+        with torch.cuda.stream(side):
+            for _ in range(8):
+                stack.step(side)
+        side.synchronize()
+        assert stack.status() == 0
+        compare_group(m["x"][7:8], m["P"], m["W"], st.eps, stack.ys[0].cpu().numpy(),
+                      stack.gate_log[7, 0].cpu().numpy(), stack.rho_log[7, 0].cpu().numpy())
