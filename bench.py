@@ -470,7 +470,7 @@ def main():
             from oracle import gsi_oracle as O
             del stack, layers, dense_layers, keep
             torch.cuda.empty_cache()
-            sample = OracleSample(spec, n_layers=min(2, spec.n_layers), n_tokens=512)
+            sample = OracleSample(spec, n_layers=min(4, spec.n_layers), n_tokens=1280)
             v, dt, _ = sample.run()
             out["cpu_baseline"] = {"value": v, "unit": "tokens/s", "cores": O.num_threads(),
                                    "kind": "oracle", "sample": sample.describe(dt)}
