@@ -377,7 +377,7 @@ __device__ __noinline__ void gated_pass(const PersistGroup& g, const Slab& s, co
 #pragma unroll 1
     for (int rw = warp; rw < rows; rw += kNW) {
       const uint16_t* wrow = row_ptr(rw);
-      float acc = 0.f;
+      unsigned long long acc2 = 0ull;  // two fp32 partial sums (two-wide FMA)
 #pragma unroll 1
       for (int v0 = lane; v0 < nv; v0 += kWLoads * 32) {
         uint32_t w[kWLoads][8];
@@ -393,16 +393,13 @@ __device__ __noinline__ void gated_pass(const PersistGroup& g, const Slab& s, co
 #pragma unroll
             for (int q = 0; q < 4; ++q) {
               const float4 rr = s_rq[q * 256 + v];
-              const uint32_t lo = w[u][2 * q], hi = w[u][2 * q + 1];
-              acc = fmaf(__uint_as_float(lo << 16), rr.x, acc);
-              acc = fmaf(__uint_as_float(lo & 0xFFFF0000u), rr.y, acc);
-              acc = fmaf(__uint_as_float(hi << 16), rr.z, acc);
-              acc = fmaf(__uint_as_float(hi & 0xFFFF0000u), rr.w, acc);
+              fma2(acc2, bf16x2_to_f32x2(w[u][2 * q]), pack2(rr.x, rr.y));
+              fma2(acc2, bf16x2_to_f32x2(w[u][2 * q + 1]), pack2(rr.z, rr.w));
             }
           }
         }
       }
-      acc = warp_sum(acc);
+      const float acc = warp_sum(sum2(acc2));
       if (lane == 0) s_yacc[rw] = (sl == 0 ? 0.f : s_yacc[rw]) + acc;
     }
   }
