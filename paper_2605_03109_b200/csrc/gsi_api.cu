@@ -19,12 +19,13 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 struct Layout {
   size_t wp, c, cpart, r, normpart, ctrl, fired, rho, x_stage, y_stage, gate_stage, rho_stage,
-      pk_acc, pk_slot, tc_rb, tc_ypart, total;
+      pk_acc, pk_slot, tc_rb, tc_ypart, f_pt, f_xb, f_cb, f_cpart, f_normpart, total;
   int O, n_slabs, slab_rows;
-  bool tc;
+  bool tc, front;
 };
 
 constexpr int kTcMinFired = 5;  // fewer fired tokens: one pass of the CUDA-core GEMV
+constexpr int kFrontMinTokens = 8;  // fewer tokens in a call: the CUDA-core front end
 
 bool tc_shapes_ok(const gsi_desc_t* d) {
   for (int j = 0; j < d->n_maps; ++j)
@@ -82,6 +83,16 @@ Layout make_layout_ws(const gsi_desc_t* d) {
   L.tc_rb = take(tc ? (size_t)64 * d->d * 2 : 0);
   L.tc_ypart = take(tc ? (size_t)tc_splits(O, d->d) * 64 * O * 4 : 0);
   L.tc = tc;
+  // tensor-core projection / residual / image for batched calls
+  const bool front = !dense && d->max_tokens >= kFrontMinTokens && d->p_dtype == GSI_BF16 && d->k % 128 == 0 &&
+                     d->d % 128 == 0 && O % 128 == 0;
+  const size_t rows = front ? front_rows(d->max_tokens) : 0;
+  L.f_pt = take(front ? (size_t)d->k * d->d * 2 : 0);
+  L.f_xb = take(rows * d->d * 2);
+  L.f_cb = take(rows * k * 2);
+  L.f_cpart = take(front ? (size_t)front_proj_splits(d->d, d->k) * B * k * 4 : 0);
+  L.f_normpart = take(front ? (size_t)(d->d / 128) * B * 2 * 4 : 0);
+  L.front = front;
   L.total = at;
   return L;
 }
@@ -212,6 +223,13 @@ gsi_status_t gsi_create(const gsi_desc_t* desc, const void* const* W, const void
   g.tc_min_fired = L.tc ? kTcMinFired : 0;
   g.rb = reinterpret_cast<uint16_t*>(h->ws + L.tc_rb);
   g.ypart = reinterpret_cast<float*>(h->ws + L.tc_ypart);
+  g.front_min_tokens = L.front ? kFrontMinTokens : 0;
+  g.proj_splits = L.front ? front_proj_splits(desc->d, desc->k) : 0;
+  g.PT = reinterpret_cast<const uint16_t*>(h->ws + L.f_pt);
+  g.xb = reinterpret_cast<uint16_t*>(h->ws + L.f_xb);
+  g.cb = reinterpret_cast<uint16_t*>(h->ws + L.f_cb);
+  g.cpart3 = reinterpret_cast<float*>(h->ws + L.f_cpart);
+  g.normpart3 = reinterpret_cast<float*>(h->ws + L.f_normpart);
 
   if (cudaMemsetAsync(ctrl, 0, 256, stream) != cudaSuccess ||
       cudaMemsetAsync(h->ws + L.pk_acc, 0, L.total - L.pk_acc, stream) != cudaSuccess) {
@@ -222,6 +240,11 @@ gsi_status_t gsi_create(const gsi_desc_t* desc, const void* const* W, const void
   h->bar = reinterpret_cast<unsigned*>(ctrl + 16);
   if (!dense && !g.p_f32 &&
       launch_abs_max_bf16(P, (size_t)desc->d * desc->k, h->pmax, stream) != cudaSuccess) {
+    delete h;
+    return GSI_ERR_CUDA;
+  }
+  if (L.front &&
+      launch_transpose_bf16(P, desc->d, desc->k, h->ws + L.f_pt, stream) != cudaSuccess) {
     delete h;
     return GSI_ERR_CUDA;
   }
@@ -530,8 +553,7 @@ gsi_status_t gsi_stack_launches_per_step(gsi_stack_t s, int* n_out) {
   }
   int n = 0;
   for (gsi_layer* h : s->groups) {
-    if (h->desc.flags & GSI_FLAG_DENSE) n += 1;
-    else n += (h->desc.flags & GSI_FLAG_STATIC_PROJECTION) ? 4 : (h->gp.tc_min_fired ? 8 : 5);
+    n += generic_launch_count(h->gp, s->B);
   }
   *n_out = n + 1;
   return GSI_OK;

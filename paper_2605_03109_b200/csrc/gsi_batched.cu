@@ -1,0 +1,274 @@
+// Batched front end of the gated subspace layer on the 5th-gen tensor cores:
+// Algorithm 1 lines 1-5 for a batch of tokens as three skinny contractions,
+//
+//   c  = P^T x      A = P^T tile [128 of k][d],   B = terms of x [3n][d],  split over d
+//   Pc (-> r, gate) A = P tile   [128 of d][k],   B = terms of c [3n][k]
+//   y  = W_P c      A = W_P tile [128 of O][k],   B = terms of c [3n][k]
+//
+// The basis and the images are bf16 already; the fp32 activations and coefficients
+// enter as THREE bf16 terms each (v = hi + mid + lo, 24 significant bits), stored as
+// rows 3t, 3t+1, 3t+2 of the B operand, so every product is exact and the sums are
+// fp32 in tensor memory: the same arithmetic as the CUDA-core kernels up to the order
+// of the additions.  The epilogues add the three columns of a token and apply the rest
+// of the line: the split-K partial of c; r = x - Pc with the partial sums of ||r||^2
+// and ||x||^2 followed by the gate decision (Eq. (3.3)) in the last block; y.
+#include "gsi_umma.cuh"
+
+namespace gsi {
+
+namespace {
+
+using namespace umma;
+
+constexpr int kStages3 = 4;
+constexpr int kMaxN3 = 192;          // 3 terms x 64 tokens
+constexpr int kTmemCols3 = 256;      // power of two >= kMaxN3
+using Cfg3 = Cfg<kStages3, kMaxN3>;
+constexpr int kSmem3 = Cfg3::kSmem;  // 4 x (16 + 24) KB + slack
+
+__device__ __forceinline__ uint16_t bf16_bits(float v) {
+  const __nv_bfloat16 h = __float2bfloat16_rn(v);
+  return *reinterpret_cast<const uint16_t*>(&h);
+}
+__device__ __forceinline__ float bf16_val(uint16_t b) { return __uint_as_float((uint32_t)b << 16); }
+
+// v = hi + mid + lo exactly for every finite fp32 v whose low term is not subnormal.
+__device__ __forceinline__ void split3(float v, uint16_t& hi, uint16_t& mid, uint16_t& lo) {
+  hi = bf16_bits(v);
+  const float r1 = v - bf16_val(hi);
+  mid = bf16_bits(r1);
+  const float r2 = r1 - bf16_val(mid);
+  lo = bf16_bits(r2);
+}
+
+__device__ __forceinline__ int rows3(int n_tokens) { return (3 * n_tokens + 15) & ~15; }
+
+// src [n_tokens][len] fp32 -> dst [rows3][len] bf16 terms; rows past 3 n_tokens are zero.
+// One block row (blockIdx.y) per token slot, 8 elements per thread.
+__device__ __forceinline__ void store_terms(const float (&v)[8], bool live, uint16_t* dst, int slot,
+                                            int n_rows, size_t len, size_t at) {
+  uint32_t w[3][4];
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    uint16_t a[3], b[3];
+    if (live) {
+      split3(v[2 * e], a[0], a[1], a[2]);
+      split3(v[2 * e + 1], b[0], b[1], b[2]);
+    } else {
+      a[0] = a[1] = a[2] = b[0] = b[1] = b[2] = 0;
+    }
+#pragma unroll
+    for (int c = 0; c < 3; ++c) w[c][e] = (uint32_t)a[c] | ((uint32_t)b[c] << 16);
+  }
+#pragma unroll
+  for (int c = 0; c < 3; ++c) {
+    const int row = 3 * slot + c;
+    if (row < n_rows)
+      *reinterpret_cast<uint4*>(dst + (size_t)row * len + at) = make_uint4(w[c][0], w[c][1], w[c][2], w[c][3]);
+  }
+}
+
+__global__ void __launch_bounds__(256) k_split3_x(GroupParams g, IoRef io, int n_tokens) {
+  const int slot = blockIdx.y, n_rows = rows3(n_tokens);
+  const bool live = slot < n_tokens;
+  const float* x = io.x + (long long)io_slot(io) * io.x_step_stride + (size_t)slot * g.d;
+  for (int i8 = blockIdx.x * 256 + threadIdx.x; i8 < g.d / 8; i8 += gridDim.x * 256) {
+    float v[8] = {};
+    if (live) {
+      const float4 a = __ldg(reinterpret_cast<const float4*>(x) + 2 * i8);
+      const float4 b = __ldg(reinterpret_cast<const float4*>(x) + 2 * i8 + 1);
+      v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w;
+      v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    }
+    store_terms(v, live, g.xb, slot, n_rows, (size_t)g.d, (size_t)i8 * 8);
+  }
+}
+
+// Sum of the three term columns of 16 tokens: columns 48q .. 48q+47 of this lane.
+__device__ __forceinline__ void load_tokens16(uint32_t tmem_lane, int q, float (&s)[16]) {
+  uint32_t v[3][16];
+#pragma unroll
+  for (int i = 0; i < 3; ++i) tmem_ld16(tmem_lane + 48 * q + 16 * i, v[i]);
+  tmem_ld_wait();
+#pragma unroll
+  for (int tt = 0; tt < 16; ++tt) {
+    const int c = 3 * tt;
+    s[tt] = (__uint_as_float(v[c / 16][c % 16]) + __uint_as_float(v[(c + 1) / 16][(c + 1) % 16])) +
+            __uint_as_float(v[(c + 2) / 16][(c + 2) % 16]);
+  }
+}
+
+// c partials: cpart3[split][t][128*tile + lane row] over this split's share of d.
+__global__ void __launch_bounds__(kThreads, 1) k_proj_tc(GroupParams g, int n_tokens) {
+  extern __shared__ unsigned char smem_raw[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int splits = g.proj_splits;
+  const int tile = blockIdx.x / splits, split = blockIdx.x % splits;
+  const int nkb = g.d / kTK;
+  const int kb0 = (int)((long long)nkb * split / splits), kb1 = (int)((long long)nkb * (split + 1) / splits);
+  uint32_t tmem;
+  const bool ok = tile_mma<kStages3, kMaxN3, kTmemCols3>(
+      smem_raw, g.PT + (size_t)tile * kTM * g.d, (size_t)g.d, g.xb, (size_t)g.d, rows3(n_tokens), kb0,
+      kb1 - kb0, &tmem);
+  if (!ok) {
+    if (threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
+  } else {
+    const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);
+    float* out = g.cpart3 + (size_t)split * g.B * g.k + tile * kTM + warp * 32 + lane;
+    for (int q = 0; 16 * q < n_tokens; ++q) {
+      float s[16];
+      load_tokens16(tl, q, s);
+#pragma unroll
+      for (int tt = 0; tt < 16; ++tt)
+        if (16 * q + tt < n_tokens) out[(size_t)(16 * q + tt) * g.k] = s[tt];
+    }
+  }
+  tile_release<kTmemCols3>(tmem);
+}
+
+// c = sum of the split-K partials in split order; also its three bf16 terms.
+__global__ void __launch_bounds__(128) k_reduce_split3_c(GroupParams g, int n_tokens) {
+  const int slot = blockIdx.y, n_rows = rows3(n_tokens);
+  const bool live = slot < n_tokens;
+  const int j8 = blockIdx.x * 128 + threadIdx.x;
+  if (j8 >= g.k / 8) return;
+  float v[8] = {};
+  if (live) {
+    for (int s = 0; s < g.proj_splits; ++s) {
+      const float4* p = reinterpret_cast<const float4*>(g.cpart3 + ((size_t)s * g.B + slot) * g.k) + 2 * j8;
+      const float4 a = p[0], b = p[1];
+      v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w;
+      v[4] += b.x; v[5] += b.y; v[6] += b.z; v[7] += b.w;
+    }
+    float4* c = reinterpret_cast<float4*>(g.c + (size_t)slot * g.k) + 2 * j8;
+    c[0] = make_float4(v[0], v[1], v[2], v[3]);
+    c[1] = make_float4(v[4], v[5], v[6], v[7]);
+  }
+  store_terms(v, live, g.cb, slot, n_rows, (size_t)g.k, (size_t)j8 * 8);
+}
+
+// r = x - P c for 128 rows of d, the partial norms of the tile, then the gate.
+__global__ void __launch_bounds__(kThreads, 1) k_resid_tc(GroupParams g, IoRef io, int n_tokens) {
+  extern __shared__ unsigned char smem_raw[];
+  __shared__ float s_norm[kThreads / 32][GSI_MAX_TOKENS][2];
+  __shared__ int s_last;
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tile = blockIdx.x;
+  const int slot = io_slot(io);
+  uint32_t tmem;
+  const bool ok = tile_mma<kStages3, kMaxN3, kTmemCols3>(
+      smem_raw, reinterpret_cast<const uint16_t*>(g.P) + (size_t)tile * kTM * g.k, (size_t)g.k, g.cb,
+      (size_t)g.k, rows3(n_tokens), 0, g.k / kTK, &tmem);
+  if (!ok) {
+    if (threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
+    for (int i = threadIdx.x; i < (kThreads / 32) * GSI_MAX_TOKENS * 2; i += kThreads)
+      (&s_norm[0][0][0])[i] = 0.f;
+  } else {
+    const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);
+    const int row = tile * kTM + warp * 32 + lane;
+    const float* x = io.x + (long long)slot * io.x_step_stride + row;
+    for (int q = 0; 16 * q < n_tokens; ++q) {
+      float s[16];
+      load_tokens16(tl, q, s);
+#pragma unroll
+      for (int tt = 0; tt < 16; ++tt) {
+        const int t = 16 * q + tt;
+        if (t < n_tokens) {   // uniform over the warp
+          const float xv = __ldg(x + (size_t)t * g.d);
+          const float rv = xv - s[tt];
+          g.r[(size_t)t * g.d + row] = rv;
+          const float a = warp_sum(rv * rv), b = warp_sum(xv * xv);
+          if (lane == 0) {
+            s_norm[warp][t][0] = a;
+            s_norm[warp][t][1] = b;
+          }
+        }
+      }
+    }
+  }
+  __syncthreads();
+  for (int i = threadIdx.x; i < n_tokens * 2; i += kThreads) {
+    const int t = i >> 1, w = i & 1;
+    float s = 0.f;
+#pragma unroll
+    for (int wp = 0; wp < kThreads / 32; ++wp) s += s_norm[wp][t][w];
+    g.normpart3[((size_t)tile * g.B + t) * 2 + w] = s;
+  }
+  tile_release<kTmemCols3>(tmem);
+  decide_gate_last_block(g, io, slot, n_tokens, g.normpart3, (int)gridDim.x, &s_last);
+}
+
+// y = W_P c for 128 rows of the concatenated images.
+__global__ void __launch_bounds__(kThreads, 1) k_image_tc(GroupParams g, IoRef io, int n_tokens) {
+  extern __shared__ unsigned char smem_raw[];
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tile = blockIdx.x;
+  uint32_t tmem;
+  const bool ok = tile_mma<kStages3, kMaxN3, kTmemCols3>(smem_raw, g.WP + (size_t)tile * kTM * g.k,
+                                                         (size_t)g.k, g.cb, (size_t)g.k,
+                                                         rows3(n_tokens), 0, g.k / kTK, &tmem);
+  if (!ok) {
+    if (threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
+  } else {
+    const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);
+    float* y = io.y + tile * kTM + warp * 32 + lane;
+    for (int q = 0; 16 * q < n_tokens; ++q) {
+      float s[16];
+      load_tokens16(tl, q, s);
+#pragma unroll
+      for (int tt = 0; tt < 16; ++tt)
+        if (16 * q + tt < n_tokens) y[(size_t)(16 * q + tt) * g.O] = s[tt];
+    }
+  }
+  tile_release<kTmemCols3>(tmem);
+}
+
+// PT[j][i] = P[i][j], 32 x 32 tiles through shared memory.
+__global__ void __launch_bounds__(256) k_transpose_bf16(const uint16_t* __restrict__ P, int d, int k,
+                                                        uint16_t* __restrict__ PT) {
+  __shared__ uint16_t tile[32][33];
+  const int i0 = blockIdx.y * 32, j0 = blockIdx.x * 32;
+  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+  for (int r = ty; r < 32; r += 8)
+    if (i0 + r < d && j0 + tx < k) tile[r][tx] = P[(size_t)(i0 + r) * k + j0 + tx];
+  __syncthreads();
+  for (int r = ty; r < 32; r += 8)
+    if (j0 + r < k && i0 + tx < d) PT[(size_t)(j0 + r) * d + i0 + tx] = tile[tx][r];
+}
+
+}  // namespace
+
+int front_rows(int max_tokens) { return (3 * max_tokens + 15) & ~15; }
+
+int front_proj_splits(int d, int k) {
+  const int tiles = k / kTM, nkb = d / kTK;
+  int s = 148 / tiles;
+  if (s > nkb / 2) s = nkb / 2;
+  if (s < 1) s = 1;
+  return s;
+}
+
+cudaError_t launch_transpose_bf16(const void* P, int d, int k, void* PT, cudaStream_t st) {
+  k_transpose_bf16<<<dim3((k + 31) / 32, (d + 31) / 32), 256, 0, st>>>(
+      static_cast<const uint16_t*>(P), d, k, static_cast<uint16_t*>(PT));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_front_tc(const GroupParams& g, const IoRef& io, int n_tokens, cudaStream_t st,
+                            int* n_launches) {
+  cudaError_t e;
+  if ((e = cudaFuncSetAttribute(k_proj_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem3)) != cudaSuccess ||
+      (e = cudaFuncSetAttribute(k_resid_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem3)) != cudaSuccess ||
+      (e = cudaFuncSetAttribute(k_image_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem3)) != cudaSuccess)
+    return e;
+  const int slots = (front_rows(n_tokens) + 2) / 3;   // token slots covering every operand row
+  k_split3_x<<<dim3((g.d / 8 + 255) / 256, slots), 256, 0, st>>>(g, io, n_tokens);
+  k_proj_tc<<<(g.k / kTM) * g.proj_splits, kThreads, kSmem3, st>>>(g, n_tokens);
+  k_reduce_split3_c<<<dim3((g.k / 8 + 127) / 128, slots), 128, 0, st>>>(g, n_tokens);
+  k_resid_tc<<<g.d / kTM, kThreads, kSmem3, st>>>(g, io, n_tokens);
+  k_image_tc<<<g.O / kTM, kThreads, kSmem3, st>>>(g, io, n_tokens);
+  if (n_launches) *n_launches += 5;
+  return cudaGetLastError();
+}
+
+}  // namespace gsi

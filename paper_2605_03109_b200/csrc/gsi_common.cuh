@@ -97,7 +97,59 @@ struct GroupParams {
   int tc_min_fired;   // 0 = disabled
   uint16_t* rb;       // [64][d] bf16: residuals of the fired tokens, compacted
   float* ypart;       // [splits][64][O] split-K partial sums
+  // tensor-core projection / residual / image (batched): used for calls with at least
+  // front_min_tokens tokens.  fp32 operands enter as three bf16 terms (row 3t+c of the
+  // B operand is term c of token t), so products are exact and sums are fp32.
+  int front_min_tokens;   // 0 = disabled
+  int proj_splits;        // split-K CTAs per 128 columns of the projection
+  const uint16_t* PT;     // [k][d] bf16: the basis transposed (K-major for c = P^T x)
+  uint16_t* xb;           // [3B rounded up to 16][d] bf16 terms of x
+  uint16_t* cb;           // [3B rounded up to 16][k] bf16 terms of c
+  float* cpart3;          // [proj_splits][B][k] split-K partial sums of c
+  float* normpart3;       // [d/128][B][2] per-tile partial sums of ||r||^2, ||x||^2
 };
+
+// The block that arrives last (of gridDim.x) sums the per-part norm partials in part
+// order in double precision, writes gate / rho (Eq. (3.3)) and the ascending list of
+// fired tokens, and rearms the arrival counter.  Every thread of every block calls it
+// after its partials are written; s_last is a shared-memory word.
+__device__ __forceinline__ void decide_gate_last_block(const GroupParams& g, const IoRef& io,
+                                                       int slot, int n_tokens,
+                                                       const float* normpart, int n_parts,
+                                                       int* s_last) {
+  __threadfence();
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    const unsigned prev = atomicAdd(g.counter, 1u);
+    *s_last = (prev == gridDim.x - 1);
+  }
+  __syncthreads();
+  if (!*s_last) return;
+  __threadfence();
+  unsigned char* gate = io.gate + (long long)slot * io.log_step_stride;
+  float* rho = io.rho ? io.rho + (long long)slot * io.log_step_stride : g.rho_scratch;
+  for (int t = threadIdx.x; t < n_tokens; t += blockDim.x) {
+    double sr = 0.0, sx = 0.0;
+    for (int sl = 0; sl < n_parts; ++sl) {
+      sr += (double)__ldcg(normpart + ((size_t)sl * g.B + t) * 2);
+      sx += (double)__ldcg(normpart + ((size_t)sl * g.B + t) * 2 + 1);
+    }
+    const double nr = sqrt(sr), nx = sqrt(sx);
+    const bool fast = nr < (double)g.eps * nx;  // false for NaN and for x = 0
+    gate[t] = fast ? 0 : 1;
+    rho[t] = (float)(nr / nx);
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    int n = 0;
+    if (!(g.flags & GSI_FLAG_STATIC_PROJECTION)) {
+      for (int t = 0; t < n_tokens; ++t)
+        if (gate[t]) g.fired[n++] = t;
+    }
+    *g.n_fired = n;
+    *g.counter = 0u;
+  }
+}
 
 cudaError_t launch_generic_forward(const GroupParams& g, const IoRef& io, int n_tokens,
                                    cudaStream_t stream, int* n_launches);
@@ -106,6 +158,14 @@ cudaError_t launch_residual_gemm_tc(const GroupParams& g, const IoRef& io, int m
                                     cudaStream_t stream, int* n_launches);
 int tc_splits(int O, int d);
 bool tc_eligible(const GroupParams& g);
+// Batched front end on the tensor cores: c, r, gate and y = W_P c for n_tokens tokens.
+cudaError_t launch_front_tc(const GroupParams& g, const IoRef& io, int n_tokens,
+                            cudaStream_t stream, int* n_launches);
+cudaError_t launch_transpose_bf16(const void* P, int d, int k, void* PT, cudaStream_t stream);
+int front_proj_splits(int d, int k);
+int front_rows(int max_tokens);   // rows of the three-term operands
+// Kernel launches one generic forward of n_tokens tokens makes.
+int generic_launch_count(const GroupParams& g, int n_tokens);
 cudaError_t launch_build_image(const void* W, const void* P, int o, int d, int k, bool p_f32,
                                void* WP, cudaStream_t stream);
 

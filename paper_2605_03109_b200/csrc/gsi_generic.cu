@@ -229,38 +229,7 @@ k_residual_gate(GroupParams g, IoRef io, int n_tokens) {
   }
 
   // The last slab to arrive sums the norm partials in slab order and decides.
-  __threadfence();
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    const unsigned prev = atomicAdd(g.counter, 1u);
-    s_last = (prev == gridDim.x - 1);
-  }
-  __syncthreads();
-  if (!s_last) return;
-  __threadfence();
-  unsigned char* gate = io.gate + (long long)slot * io.log_step_stride;
-  float* rho = io.rho ? io.rho + (long long)slot * io.log_step_stride : g.rho_scratch;
-  for (int t = threadIdx.x; t < n_tokens; t += kThreads) {
-    double sr = 0.0, sx = 0.0;
-    for (int sl = 0; sl < g.n_slabs; ++sl) {
-      sr += (double)__ldcg(g.normpart + ((size_t)sl * g.B + t) * 2);
-      sx += (double)__ldcg(g.normpart + ((size_t)sl * g.B + t) * 2 + 1);
-    }
-    const double nr = sqrt(sr), nx = sqrt(sx);
-    const bool fast = nr < (double)g.eps * nx;  // false for NaN and for x = 0
-    gate[t] = fast ? 0 : 1;
-    rho[t] = (float)(nr / nx);
-  }
-  __syncthreads();
-  if (threadIdx.x == 0) {
-    int n = 0;
-    if (!(g.flags & GSI_FLAG_STATIC_PROJECTION)) {
-      for (int t = 0; t < n_tokens; ++t)
-        if (gate[t]) g.fired[n++] = t;
-    }
-    *g.n_fired = n;
-    *g.counter = 0u;
-  }
+  decide_gate_last_block(g, io, slot, n_tokens, g.normpart, g.n_slabs, &s_last);
 }
 
 template <int VPL>
@@ -408,12 +377,16 @@ cudaError_t launch_generic_forward(const GroupParams& g, const IoRef& io, int n_
   }
   const RowLayout L = make_layout(g.k);
   cudaError_t e;
-  switch (L.VPL) {
-    case 1: e = launch_vpl<1>(g, io, n_tokens, st, n_launches); break;
-    case 2: e = launch_vpl<2>(g, io, n_tokens, st, n_launches); break;
-    case 3: e = launch_vpl<3>(g, io, n_tokens, st, n_launches); break;
-    case 4: e = launch_vpl<4>(g, io, n_tokens, st, n_launches); break;
-    default: return cudaErrorInvalidValue;
+  if (g.front_min_tokens > 0 && n_tokens >= g.front_min_tokens) {
+    e = launch_front_tc(g, io, n_tokens, st, n_launches);
+  } else {
+    switch (L.VPL) {
+      case 1: e = launch_vpl<1>(g, io, n_tokens, st, n_launches); break;
+      case 2: e = launch_vpl<2>(g, io, n_tokens, st, n_launches); break;
+      case 3: e = launch_vpl<3>(g, io, n_tokens, st, n_launches); break;
+      case 4: e = launch_vpl<4>(g, io, n_tokens, st, n_launches); break;
+      default: return cudaErrorInvalidValue;
+    }
   }
   if (e != cudaSuccess) return e;
   if (!(g.flags & GSI_FLAG_STATIC_PROJECTION)) {
@@ -425,6 +398,13 @@ cudaError_t launch_generic_forward(const GroupParams& g, const IoRef& io, int n_
     }
   }
   return cudaGetLastError();
+}
+
+int generic_launch_count(const GroupParams& g, int n_tokens) {
+  if (g.flags & GSI_FLAG_DENSE) return 1;
+  int n = (g.front_min_tokens > 0 && n_tokens >= g.front_min_tokens) ? 5 : 4;
+  if (!(g.flags & GSI_FLAG_STATIC_PROJECTION)) n += 1 + (g.tc_min_fired > 0 ? 3 : 0);
+  return n;
 }
 
 cudaError_t launch_advance_step(int* step, cudaStream_t st) {
