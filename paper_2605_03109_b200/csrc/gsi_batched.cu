@@ -25,6 +25,7 @@ constexpr int kMaxN3 = 192;          // 3 terms x 64 tokens
 constexpr int kTmemCols3 = 256;      // power of two >= kMaxN3
 using Cfg3 = Cfg<kStages3, kMaxN3>;
 constexpr int kSmem3 = Cfg3::kSmem;  // 4 x (16 + 24) KB + slack
+constexpr int kSmemResid = Cfg<kStages3, 48>::kSmem;   // 16 tokens per block
 
 __device__ __forceinline__ uint16_t bf16_bits(float v) {
   const __nv_bfloat16 h = __float2bfloat16_rn(v);
@@ -127,75 +128,86 @@ __global__ void __launch_bounds__(kThreads, 1) k_proj_tc(GroupParams g, int n_to
 }
 
 // c = sum of the split-K partials in split order; also its three bf16 terms.
-__global__ void __launch_bounds__(128) k_reduce_split3_c(GroupParams g, int n_tokens) {
-  const int slot = blockIdx.y, n_rows = rows3(n_tokens);
+// One block per token slot, one coefficient per thread and pass.
+__global__ void __launch_bounds__(256) k_reduce_split3_c(GroupParams g, int n_tokens) {
+  const int slot = blockIdx.x, n_rows = rows3(n_tokens);
   const bool live = slot < n_tokens;
-  const int j8 = blockIdx.x * 128 + threadIdx.x;
-  if (j8 >= g.k / 8) return;
-  float v[8] = {};
-  if (live) {
-    for (int s = 0; s < g.proj_splits; ++s) {
-      const float4* p = reinterpret_cast<const float4*>(g.cpart3 + ((size_t)s * g.B + slot) * g.k) + 2 * j8;
-      const float4 a = p[0], b = p[1];
-      v[0] += a.x; v[1] += a.y; v[2] += a.z; v[3] += a.w;
-      v[4] += b.x; v[5] += b.y; v[6] += b.z; v[7] += b.w;
+  for (int j = threadIdx.x; j < g.k; j += 256) {
+    float v = 0.f;
+    if (live) {
+      const float* p = g.cpart3 + (size_t)slot * g.k + j;
+      const size_t stride = (size_t)g.B * g.k;
+      int s = 0;
+      for (; s + 8 <= g.proj_splits; s += 8) {
+        float u[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) u[i] = p[(size_t)(s + i) * stride];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) v += u[i];
+      }
+      for (; s < g.proj_splits; ++s) v += p[(size_t)s * stride];
+      g.c[(size_t)slot * g.k + j] = v;
     }
-    float4* c = reinterpret_cast<float4*>(g.c + (size_t)slot * g.k) + 2 * j8;
-    c[0] = make_float4(v[0], v[1], v[2], v[3]);
-    c[1] = make_float4(v[4], v[5], v[6], v[7]);
+    uint16_t term[3] = {0, 0, 0};
+    if (live) split3(v, term[0], term[1], term[2]);
+#pragma unroll
+    for (int c = 0; c < 3; ++c)
+      if (3 * slot + c < n_rows) g.cb[(size_t)(3 * slot + c) * g.k + j] = term[c];
   }
-  store_terms(v, live, g.cb, slot, n_rows, (size_t)g.k, (size_t)j8 * 8);
 }
 
-// r = x - P c for 128 rows of d, the partial norms of the tile, then the gate.
+// r = x - P c for 128 rows of d and 16 tokens, their partial norms, then the gate.
+// Block (tile, q) contracts against rows 48q.. of the c terms only, so that the narrow
+// inputs (d = 4096: 32 tiles) still spread over the machine.
 __global__ void __launch_bounds__(kThreads, 1) k_resid_tc(GroupParams g, IoRef io, int n_tokens) {
   extern __shared__ unsigned char smem_raw[];
-  __shared__ float s_norm[kThreads / 32][GSI_MAX_TOKENS][2];
+  __shared__ float s_norm[kThreads / 32][16][2];
   __shared__ int s_last;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile = blockIdx.x;
+  const int nq = (n_tokens + 15) / 16;
+  const int tile = blockIdx.x / nq, q = blockIdx.x % nq;
   const int slot = io_slot(io);
+  const int n_rows = min(48, rows3(n_tokens) - 48 * q);
+  const int row = tile * kTM + warp * 32 + lane;
+  const float* x = io.x + (long long)slot * io.x_step_stride + row;
+  float xv[16];
+#pragma unroll
+  for (int tt = 0; tt < 16; ++tt)
+    xv[tt] = (16 * q + tt < n_tokens) ? __ldg(x + (size_t)(16 * q + tt) * g.d) : 0.f;
   uint32_t tmem;
-  const bool ok = tile_mma<kStages3, kMaxN3, kTmemCols3>(
-      smem_raw, reinterpret_cast<const uint16_t*>(g.P) + (size_t)tile * kTM * g.k, (size_t)g.k, g.cb,
-      (size_t)g.k, rows3(n_tokens), 0, g.k / kTK, &tmem);
+  const bool ok = tile_mma<kStages3, 48, 64>(
+      smem_raw, reinterpret_cast<const uint16_t*>(g.P) + (size_t)tile * kTM * g.k, (size_t)g.k,
+      g.cb + (size_t)48 * q * g.k, (size_t)g.k, n_rows, 0, g.k / kTK, &tmem);
   if (!ok) {
     if (threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
-    for (int i = threadIdx.x; i < (kThreads / 32) * GSI_MAX_TOKENS * 2; i += kThreads)
-      (&s_norm[0][0][0])[i] = 0.f;
+    for (int i = threadIdx.x; i < (kThreads / 32) * 16 * 2; i += kThreads) (&s_norm[0][0][0])[i] = 0.f;
   } else {
-    const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);
-    const int row = tile * kTM + warp * 32 + lane;
-    const float* x = io.x + (long long)slot * io.x_step_stride + row;
-    for (int q = 0; 16 * q < n_tokens; ++q) {
-      float s[16];
-      load_tokens16(tl, q, s);
+    float s[16];
+    load_tokens16(tmem + ((uint32_t)(warp * 32) << 16), 0, s);
 #pragma unroll
-      for (int tt = 0; tt < 16; ++tt) {
-        const int t = 16 * q + tt;
-        if (t < n_tokens) {   // uniform over the warp
-          const float xv = __ldg(x + (size_t)t * g.d);
-          const float rv = xv - s[tt];
-          g.r[(size_t)t * g.d + row] = rv;
-          const float a = warp_sum(rv * rv), b = warp_sum(xv * xv);
-          if (lane == 0) {
-            s_norm[warp][t][0] = a;
-            s_norm[warp][t][1] = b;
-          }
-        }
+    for (int tt = 0; tt < 16; ++tt) {
+      const int t = 16 * q + tt;
+      const float rv = xv[tt] - s[tt];
+      if (t < n_tokens) g.r[(size_t)t * g.d + row] = rv;
+      const float a = warp_sum(rv * rv), b = warp_sum(xv[tt] * xv[tt]);
+      if (lane == 0) {
+        s_norm[warp][tt][0] = a;
+        s_norm[warp][tt][1] = b;
       }
     }
   }
   __syncthreads();
-  for (int i = threadIdx.x; i < n_tokens * 2; i += kThreads) {
-    const int t = i >> 1, w = i & 1;
-    float s = 0.f;
+  if (threadIdx.x < 32) {
+    const int tt = threadIdx.x >> 1, w = threadIdx.x & 1, t = 16 * q + tt;
+    if (t < n_tokens) {
+      float sum = 0.f;
 #pragma unroll
-    for (int wp = 0; wp < kThreads / 32; ++wp) s += s_norm[wp][t][w];
-    g.normpart3[((size_t)tile * g.B + t) * 2 + w] = s;
+      for (int wp = 0; wp < kThreads / 32; ++wp) sum += s_norm[wp][tt][w];
+      g.normpart3[((size_t)tile * g.B + t) * 2 + w] = sum;
+    }
   }
-  tile_release<kTmemCols3>(tmem);
-  decide_gate_last_block(g, io, slot, n_tokens, g.normpart3, (int)gridDim.x, &s_last);
+  tile_release<64>(tmem);
+  decide_gate_last_block(g, io, slot, n_tokens, g.normpart3, g.d / kTM, &s_last);
 }
 
 // y = W_P c for 128 rows of the concatenated images.
@@ -258,14 +270,14 @@ cudaError_t launch_front_tc(const GroupParams& g, const IoRef& io, int n_tokens,
                             int* n_launches) {
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(k_proj_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem3)) != cudaSuccess ||
-      (e = cudaFuncSetAttribute(k_resid_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem3)) != cudaSuccess ||
+      (e = cudaFuncSetAttribute(k_resid_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemResid)) != cudaSuccess ||
       (e = cudaFuncSetAttribute(k_image_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem3)) != cudaSuccess)
     return e;
   const int slots = (front_rows(n_tokens) + 2) / 3;   // token slots covering every operand row
   k_split3_x<<<dim3((g.d / 8 + 255) / 256, slots), 256, 0, st>>>(g, io, n_tokens);
   k_proj_tc<<<(g.k / kTM) * g.proj_splits, kThreads, kSmem3, st>>>(g, n_tokens);
-  k_reduce_split3_c<<<dim3((g.k / 8 + 127) / 128, slots), 128, 0, st>>>(g, n_tokens);
-  k_resid_tc<<<g.d / kTM, kThreads, kSmem3, st>>>(g, io, n_tokens);
+  k_reduce_split3_c<<<slots, 256, 0, st>>>(g, n_tokens);
+  k_resid_tc<<<(g.d / kTM) * ((n_tokens + 15) / 16), kThreads, kSmemResid, st>>>(g, io, n_tokens);
   k_image_tc<<<g.O / kTM, kThreads, kSmem3, st>>>(g, io, n_tokens);
   if (n_launches) *n_launches += 5;
   return cudaGetLastError();

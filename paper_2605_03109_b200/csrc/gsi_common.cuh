@@ -128,16 +128,41 @@ __device__ __forceinline__ void decide_gate_last_block(const GroupParams& g, con
   __threadfence();
   unsigned char* gate = io.gate + (long long)slot * io.log_step_stride;
   float* rho = io.rho ? io.rho + (long long)slot * io.log_step_stride : g.rho_scratch;
-  for (int t = threadIdx.x; t < n_tokens; t += blockDim.x) {
+  // L adjacent lanes share a token: each sums a contiguous range of parts in order (loads
+  // issued eight parts at a time), then the L sums are combined by a butterfly, so the
+  // result depends on n_tokens and the block size only through L and is reproducible.
+  int L = 1;
+  while (2 * L <= 32 && 2 * L * n_tokens <= (int)blockDim.x) L *= 2;
+  const int per_pass = blockDim.x / L;
+  for (int t0 = 0; t0 < n_tokens; t0 += per_pass) {   // block-uniform trip count
+    const int t = t0 + (int)threadIdx.x / L, l = (int)threadIdx.x % L;
+    const bool live = t < n_tokens;
+    const int p0 = (int)((long long)n_parts * l / L), p1 = (int)((long long)n_parts * (l + 1) / L);
     double sr = 0.0, sx = 0.0;
-    for (int sl = 0; sl < n_parts; ++sl) {
-      sr += (double)__ldcg(normpart + ((size_t)sl * g.B + t) * 2);
-      sx += (double)__ldcg(normpart + ((size_t)sl * g.B + t) * 2 + 1);
+    if (live) {
+      const float2* np = reinterpret_cast<const float2*>(normpart) + t;
+      for (int p = p0; p < p1; p += 8) {
+        float2 v[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u)
+          v[u] = (p + u < p1) ? __ldcg(np + (size_t)(p + u) * g.B) : make_float2(0.f, 0.f);
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+          sr += (double)v[u].x;
+          sx += (double)v[u].y;
+        }
+      }
     }
-    const double nr = sqrt(sr), nx = sqrt(sx);
-    const bool fast = nr < (double)g.eps * nx;  // false for NaN and for x = 0
-    gate[t] = fast ? 0 : 1;
-    rho[t] = (float)(nr / nx);
+    for (int o = 1; o < L; o <<= 1) {
+      sr += __shfl_xor_sync(0xffffffffu, sr, o);
+      sx += __shfl_xor_sync(0xffffffffu, sx, o);
+    }
+    if (live && l == 0) {
+      const double nr = sqrt(sr), nx = sqrt(sx);
+      const bool fast = nr < (double)g.eps * nx;  // false for NaN and for x = 0
+      gate[t] = fast ? 0 : 1;
+      rho[t] = (float)(nr / nx);
+    }
   }
   __syncthreads();
   if (threadIdx.x == 0) {
