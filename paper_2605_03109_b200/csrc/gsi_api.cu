@@ -80,11 +80,11 @@ Layout make_layout_ws(const gsi_desc_t* d) {
   L.pk_slot = take((size_t)kPersistMaxGrid * 8);    // persistent kernel: ||r||^2 words
   // tensor-core gated residual: only for batches that can fire at least kTcMinFired tokens
   const bool tc = !dense && d->max_tokens >= kTcMinFired && d->d % 64 == 0 && tc_shapes_ok(d);
-  L.tc_rb = take(tc ? (size_t)64 * d->d * 2 : 0);
+  L.tc_rb = take(tc ? (size_t)65 * d->d * 2 : 0);   // row 64 stays zero
   L.tc_ypart = take(tc ? (size_t)tc_splits(O, d->d) * 64 * O * 4 : 0);
   L.tc = tc;
   // tensor-core projection / residual / image for batched calls
-  const bool front = !dense && d->max_tokens >= kFrontMinTokens && d->p_dtype == GSI_BF16 && d->k % 128 == 0 &&
+  const bool front = tc && d->max_tokens >= kFrontMinTokens && d->p_dtype == GSI_BF16 && d->k % 128 == 0 &&
                      d->d % 128 == 0 && O % 128 == 0;
   const size_t rows = front ? front_rows(d->max_tokens) : 0;
   L.f_pt = take(front ? (size_t)d->k * d->d * 2 : 0);

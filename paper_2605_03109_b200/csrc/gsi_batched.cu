@@ -109,8 +109,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_proj_tc(GroupParams g, int n_to
   const int kb0 = (int)((long long)nkb * split / splits), kb1 = (int)((long long)nkb * (split + 1) / splits);
   uint32_t tmem;
   const bool ok = tile_mma<kStages3, kMaxN3, kTmemCols3>(
-      smem_raw, g.PT + (size_t)tile * kTM * g.d, (size_t)g.d, g.xb, (size_t)g.d, rows3(n_tokens), kb0,
-      kb1 - kb0, &tmem);
+      smem_raw, g.PT + (size_t)tile * kTM * g.d, (size_t)g.d, g.xb, (size_t)g.d, nullptr, rows3(n_tokens),
+      kb0, kb1 - kb0, &tmem);
   if (!ok) {
     if (threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
   } else {
@@ -156,44 +156,59 @@ __global__ void __launch_bounds__(256) k_reduce_split3_c(GroupParams g, int n_to
   }
 }
 
-// r = x - P c for 128 rows of d and 16 tokens, their partial norms, then the gate.
-// Block (tile, q) contracts against rows 48q.. of the c terms only, so that the narrow
-// inputs (d = 4096: 32 tiles) still spread over the machine.
-__global__ void __launch_bounds__(kThreads, 1) k_resid_tc(GroupParams g, IoRef io, int n_tokens) {
+// One launch for Algorithm 1 lines 2-5.  Every block contracts one 128-row tile against
+// the c terms of 16 tokens (operand rows 48q .. 48q+47), which spreads even the narrow
+// inputs (d = 4096: 32 tiles) over the machine:
+//   blocks [0, n_resid)   tile of P:   r = x - P c -> bf16 rows of rb, the partial norms of
+//                                      the tile, and in the block that finishes last the gate
+//   blocks [n_resid, ..)  tile of W_P: y = W_P c
+__global__ void __launch_bounds__(kThreads, 2)
+k_resid_image_tc(GroupParams g, IoRef io, int n_tokens) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ float s_norm[kThreads / 32][16][2];
   __shared__ int s_last;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nq = (n_tokens + 15) / 16;
-  const int tile = blockIdx.x / nq, q = blockIdx.x % nq;
-  const int slot = io_slot(io);
+  const int n_resid = (g.d / kTM) * nq;
+  const bool image = (int)blockIdx.x >= n_resid;
+  const int bid = image ? blockIdx.x - n_resid : blockIdx.x;
+  const int tile = bid / nq, q = bid % nq;
   const int n_rows = min(48, rows3(n_tokens) - 48 * q);
   const int row = tile * kTM + warp * 32 + lane;
-  const float* x = io.x + (long long)slot * io.x_step_stride + row;
+  const uint16_t* A = (image ? g.WP : reinterpret_cast<const uint16_t*>(g.P)) + (size_t)tile * kTM * g.k;
+  const int slot = io_slot(io);
+
   float xv[16];
+  if (!image) {
+    const float* x = io.x + (long long)slot * io.x_step_stride + row;
 #pragma unroll
-  for (int tt = 0; tt < 16; ++tt)
-    xv[tt] = (16 * q + tt < n_tokens) ? __ldg(x + (size_t)(16 * q + tt) * g.d) : 0.f;
+    for (int tt = 0; tt < 16; ++tt)
+      xv[tt] = (16 * q + tt < n_tokens) ? __ldg(x + (size_t)(16 * q + tt) * g.d) : 0.f;
+  }
   uint32_t tmem;
-  const bool ok = tile_mma<kStages3, 48, 64>(
-      smem_raw, reinterpret_cast<const uint16_t*>(g.P) + (size_t)tile * kTM * g.k, (size_t)g.k,
-      g.cb + (size_t)48 * q * g.k, (size_t)g.k, n_rows, 0, g.k / kTK, &tmem);
-  if (!ok) {
-    if (threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
-    for (int i = threadIdx.x; i < (kThreads / 32) * 16 * 2; i += kThreads) (&s_norm[0][0][0])[i] = 0.f;
-  } else {
-    float s[16];
-    load_tokens16(tmem + ((uint32_t)(warp * 32) << 16), 0, s);
+  const bool ok = tile_mma<kStages3, 48, 64>(smem_raw, A, (size_t)g.k, g.cb + (size_t)48 * q * g.k,
+                                             (size_t)g.k, nullptr, n_rows, 0, g.k / kTK, &tmem);
+  if (!ok && threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
+  float s[16];
+  if (ok) load_tokens16(tmem + ((uint32_t)(warp * 32) << 16), 0, s);
+  tile_release<64>(tmem);
+  if (image) {
+    if (ok) {
 #pragma unroll
-    for (int tt = 0; tt < 16; ++tt) {
-      const int t = 16 * q + tt;
-      const float rv = xv[tt] - s[tt];
-      if (t < n_tokens) g.r[(size_t)t * g.d + row] = rv;
-      const float a = warp_sum(rv * rv), b = warp_sum(xv[tt] * xv[tt]);
-      if (lane == 0) {
-        s_norm[warp][tt][0] = a;
-        s_norm[warp][tt][1] = b;
-      }
+      for (int tt = 0; tt < 16; ++tt)
+        if (16 * q + tt < n_tokens) io.y[(size_t)(16 * q + tt) * g.O + row] = s[tt];
+    }
+    return;
+  }
+#pragma unroll
+  for (int tt = 0; tt < 16; ++tt) {
+    const int t = 16 * q + tt;
+    const float rv = ok ? xv[tt] - s[tt] : 0.f;
+    if (ok && t < n_tokens) g.rb[(size_t)t * g.d + row] = bf16_bits(rv);
+    const float a = warp_sum(rv * rv), b = warp_sum(xv[tt] * xv[tt]);
+    if (lane == 0) {
+      s_norm[warp][tt][0] = a;
+      s_norm[warp][tt][1] = b;
     }
   }
   __syncthreads();
@@ -206,33 +221,7 @@ __global__ void __launch_bounds__(kThreads, 1) k_resid_tc(GroupParams g, IoRef i
       g.normpart3[((size_t)tile * g.B + t) * 2 + w] = sum;
     }
   }
-  tile_release<64>(tmem);
-  decide_gate_last_block(g, io, slot, n_tokens, g.normpart3, g.d / kTM, &s_last);
-}
-
-// y = W_P c for 128 rows of the concatenated images.
-__global__ void __launch_bounds__(kThreads, 1) k_image_tc(GroupParams g, IoRef io, int n_tokens) {
-  extern __shared__ unsigned char smem_raw[];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int tile = blockIdx.x;
-  uint32_t tmem;
-  const bool ok = tile_mma<kStages3, kMaxN3, kTmemCols3>(smem_raw, g.WP + (size_t)tile * kTM * g.k,
-                                                         (size_t)g.k, g.cb, (size_t)g.k,
-                                                         rows3(n_tokens), 0, g.k / kTK, &tmem);
-  if (!ok) {
-    if (threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
-  } else {
-    const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);
-    float* y = io.y + tile * kTM + warp * 32 + lane;
-    for (int q = 0; 16 * q < n_tokens; ++q) {
-      float s[16];
-      load_tokens16(tl, q, s);
-#pragma unroll
-      for (int tt = 0; tt < 16; ++tt)
-        if (16 * q + tt < n_tokens) y[(size_t)(16 * q + tt) * g.O] = s[tt];
-    }
-  }
-  tile_release<kTmemCols3>(tmem);
+  decide_gate_last_block(g, io, slot, n_tokens, g.normpart3, g.d / kTM, (unsigned)n_resid, &s_last);
 }
 
 // PT[j][i] = P[i][j], 32 x 32 tiles through shared memory.
@@ -270,16 +259,16 @@ cudaError_t launch_front_tc(const GroupParams& g, const IoRef& io, int n_tokens,
                             int* n_launches) {
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(k_proj_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem3)) != cudaSuccess ||
-      (e = cudaFuncSetAttribute(k_resid_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemResid)) != cudaSuccess ||
-      (e = cudaFuncSetAttribute(k_image_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem3)) != cudaSuccess)
+      (e = cudaFuncSetAttribute(k_resid_image_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemResid)) !=
+          cudaSuccess)
     return e;
   const int slots = (front_rows(n_tokens) + 2) / 3;   // token slots covering every operand row
+  const int nq = (n_tokens + 15) / 16;
   k_split3_x<<<dim3((g.d / 8 + 255) / 256, slots), 256, 0, st>>>(g, io, n_tokens);
   k_proj_tc<<<(g.k / kTM) * g.proj_splits, kThreads, kSmem3, st>>>(g, n_tokens);
   k_reduce_split3_c<<<slots, 256, 0, st>>>(g, n_tokens);
-  k_resid_tc<<<(g.d / kTM) * ((n_tokens + 15) / 16), kThreads, kSmemResid, st>>>(g, io, n_tokens);
-  k_image_tc<<<g.O / kTM, kThreads, kSmem3, st>>>(g, io, n_tokens);
-  if (n_launches) *n_launches += 5;
+  k_resid_image_tc<<<(g.d / kTM + g.O / kTM) * nq, kThreads, kSmemResid, st>>>(g, io, n_tokens);
+  if (n_launches) *n_launches += 4;
   return cudaGetLastError();
 }
 

@@ -95,7 +95,8 @@ struct GroupParams {
   int n_slabs, slab_rows;
   // tensor-core gated residual (batched): used when at least tc_min_fired tokens fired
   int tc_min_fired;   // 0 = disabled
-  uint16_t* rb;       // [64][d] bf16: residuals of the fired tokens, compacted
+  uint16_t* rb;       // [65][d] bf16 residuals: fired tokens compacted, or (batched front end)
+                      // row t = token t; row 64 stays zero
   float* ypart;       // [splits][64][O] split-K partial sums
   // tensor-core projection / residual / image (batched): used for calls with at least
   // front_min_tokens tokens.  fp32 operands enter as three bf16 terms (row 3t+c of the
@@ -109,19 +110,19 @@ struct GroupParams {
   float* normpart3;       // [d/128][B][2] per-tile partial sums of ||r||^2, ||x||^2
 };
 
-// The block that arrives last (of gridDim.x) sums the per-part norm partials in part
+// The block that arrives last (of n_blocks) sums the per-part norm partials in part
 // order in double precision, writes gate / rho (Eq. (3.3)) and the ascending list of
 // fired tokens, and rearms the arrival counter.  Every thread of every block calls it
 // after its partials are written; s_last is a shared-memory word.
 __device__ __forceinline__ void decide_gate_last_block(const GroupParams& g, const IoRef& io,
                                                        int slot, int n_tokens,
                                                        const float* normpart, int n_parts,
-                                                       int* s_last) {
+                                                       unsigned n_blocks, int* s_last) {
   __threadfence();
   __syncthreads();
   if (threadIdx.x == 0) {
     const unsigned prev = atomicAdd(g.counter, 1u);
-    *s_last = (prev == gridDim.x - 1);
+    *s_last = (prev == n_blocks - 1);
   }
   __syncthreads();
   if (!*s_last) return;
@@ -179,8 +180,10 @@ __device__ __forceinline__ void decide_gate_last_block(const GroupParams& g, con
 cudaError_t launch_generic_forward(const GroupParams& g, const IoRef& io, int n_tokens,
                                    cudaStream_t stream, int* n_launches);
 cudaError_t launch_advance_step(int* step, cudaStream_t stream);
+// mapped: rb holds every token's residual (row = token) and the fired list selects the
+// operand rows; otherwise a pack kernel first compacts the fired tokens of g.r into rb.
 cudaError_t launch_residual_gemm_tc(const GroupParams& g, const IoRef& io, int min_fired,
-                                    cudaStream_t stream, int* n_launches);
+                                    bool mapped, cudaStream_t stream, int* n_launches);
 int tc_splits(int O, int d);
 bool tc_eligible(const GroupParams& g);
 // Batched front end on the tensor cores: c, r, gate and y = W_P c for n_tokens tokens.

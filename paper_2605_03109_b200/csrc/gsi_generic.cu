@@ -229,7 +229,7 @@ k_residual_gate(GroupParams g, IoRef io, int n_tokens) {
   }
 
   // The last slab to arrive sums the norm partials in slab order and decides.
-  decide_gate_last_block(g, io, slot, n_tokens, g.normpart, g.n_slabs, &s_last);
+  decide_gate_last_block(g, io, slot, n_tokens, g.normpart, g.n_slabs, gridDim.x, &s_last);
 }
 
 template <int VPL>
@@ -377,7 +377,8 @@ cudaError_t launch_generic_forward(const GroupParams& g, const IoRef& io, int n_
   }
   const RowLayout L = make_layout(g.k);
   cudaError_t e;
-  if (g.front_min_tokens > 0 && n_tokens >= g.front_min_tokens) {
+  const bool front = g.front_min_tokens > 0 && n_tokens >= g.front_min_tokens;
+  if (front) {
     e = launch_front_tc(g, io, n_tokens, st, n_launches);
   } else {
     switch (L.VPL) {
@@ -390,11 +391,17 @@ cudaError_t launch_generic_forward(const GroupParams& g, const IoRef& io, int n_
   }
   if (e != cudaSuccess) return e;
   if (!(g.flags & GSI_FLAG_STATIC_PROJECTION)) {
-    k_stream_gemv<false><<<grid, kThreads, 0, st>>>(g, io, n_tokens);
-    *n_launches += 1;
-    if (g.tc_min_fired > 0) {
-      e = launch_residual_gemm_tc(g, io, g.tc_min_fired, st, n_launches);
+    if (front) {
+      // every gated token goes through the tensor-core contraction; r is in rb already
+      e = launch_residual_gemm_tc(g, io, 1, true, st, n_launches);
       if (e != cudaSuccess) return e;
+    } else {
+      k_stream_gemv<false><<<grid, kThreads, 0, st>>>(g, io, n_tokens);
+      *n_launches += 1;
+      if (g.tc_min_fired > 0) {
+        e = launch_residual_gemm_tc(g, io, g.tc_min_fired, false, st, n_launches);
+        if (e != cudaSuccess) return e;
+      }
     }
   }
   return cudaGetLastError();
@@ -402,9 +409,9 @@ cudaError_t launch_generic_forward(const GroupParams& g, const IoRef& io, int n_
 
 int generic_launch_count(const GroupParams& g, int n_tokens) {
   if (g.flags & GSI_FLAG_DENSE) return 1;
-  int n = (g.front_min_tokens > 0 && n_tokens >= g.front_min_tokens) ? 5 : 4;
-  if (!(g.flags & GSI_FLAG_STATIC_PROJECTION)) n += 1 + (g.tc_min_fired > 0 ? 3 : 0);
-  return n;
+  const bool stat = g.flags & GSI_FLAG_STATIC_PROJECTION;
+  if (g.front_min_tokens > 0 && n_tokens >= g.front_min_tokens) return stat ? 4 : 6;
+  return 4 + (stat ? 0 : 1 + (g.tc_min_fired > 0 ? 3 : 0));
 }
 
 cudaError_t launch_advance_step(int* step, cudaStream_t st) {

@@ -45,12 +45,15 @@ __global__ void __launch_bounds__(256) k_pack_fired_bf16(GroupParams g, int min_
 }
 
 __global__ void __launch_bounds__(kThreadsTc, 1)
-k_residual_gemm_tc(GroupParams g, int min_fired, int splits) {
+k_residual_gemm_tc(GroupParams g, int min_fired, int splits, int mapped) {
   const int n_fired = *g.n_fired;
   if (n_fired < min_fired) return;            // the CUDA-core GEMV handles the few-token case
   const int N = (n_fired + 15) & ~15;         // 16..64
 
   extern __shared__ unsigned char smem_raw[];
+  __shared__ int s_rows[kMaxN];   // operand row n <- row of rb (mapped mode)
+  if (mapped && threadIdx.x < kMaxN)
+    s_rows[threadIdx.x] = (int)threadIdx.x < n_fired ? g.fired[threadIdx.x] : kMaxN;   // row 64 is zero
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = blockIdx.x / splits, split = blockIdx.x % splits;
   const int row0 = tile * kTM;                 // first row of the concatenated maps
@@ -62,8 +65,8 @@ k_residual_gemm_tc(GroupParams g, int min_fired, int splits) {
   const int nloc = kb1 - kb0;
 
   uint32_t tmem;
-  const bool ok = tile_mma<kStages, kMaxN, kTmemCols>(smem_raw, Wt, (size_t)g.d, g.rb, (size_t)g.d, N,
-                                                      kb0, nloc, &tmem);
+  const bool ok = tile_mma<kStages, kMaxN, kTmemCols>(smem_raw, Wt, (size_t)g.d, g.rb, (size_t)g.d,
+                                                      mapped ? s_rows : nullptr, N, kb0, nloc, &tmem);
   if (!ok) {
     if (threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
   } else if (nloc > 0) {
@@ -114,15 +117,15 @@ bool tc_eligible(const GroupParams& g) {
 }
 
 cudaError_t launch_residual_gemm_tc(const GroupParams& g, const IoRef& io, int min_fired,
-                                    cudaStream_t st, int* n_launches) {
+                                    bool mapped, cudaStream_t st, int* n_launches) {
   cudaError_t e = cudaFuncSetAttribute(k_residual_gemm_tc,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);
   if (e != cudaSuccess) return e;
   const int splits = tc_splits(g.O, g.d);
-  k_pack_fired_bf16<<<dim3((g.d + 2047) / 2048, kMaxN), 256, 0, st>>>(g, min_fired);
-  k_residual_gemm_tc<<<(g.O / kTM) * splits, kThreadsTc, kTcSmem, st>>>(g, min_fired, splits);
+  if (!mapped) k_pack_fired_bf16<<<dim3((g.d + 2047) / 2048, kMaxN), 256, 0, st>>>(g, min_fired);
+  k_residual_gemm_tc<<<(g.O / kTM) * splits, kThreadsTc, kTcSmem, st>>>(g, min_fired, splits, mapped ? 1 : 0);
   k_add_partials<<<dim3((g.O + 1023) / 1024, g.B), 256, 0, st>>>(g, io, min_fired, splits);
-  if (n_launches) *n_launches += 3;
+  if (n_launches) *n_launches += mapped ? 2 : 3;
   return cudaGetLastError();
 }
 

@@ -101,16 +101,17 @@ __device__ __forceinline__ void tmem_ld_wait() {
 }
 
 // Runs the whole contraction of one tile: rows [0,128) of A (row stride lda
-// elements), rows [0,N) of B (row stride ldb), K blocks [kb0, kb0+nloc) of 64
-// elements.  N is a multiple of 16 in [16, kBRows].  All kThreads threads of the
+// elements), rows [0,N) of B (row stride ldb; operand row n is row b_rows[n] of B when
+// b_rows, a table the block wrote before the call, is not null), K blocks
+// [kb0, kb0+nloc) of 64 elements.  N is a multiple of 16 in [16, kBRows].  All kThreads threads of the
 // block call it.  On return *tmem_out holds the tensor-memory base of D (lane =
 // row, column = B row); the return value, the same for every thread, is false when a
 // wait ran out of time.  With nloc == 0 nothing is accumulated and D is undefined.
 // The caller must end with tile_release<kTmemCols>(*tmem_out).
 template <int kStages, int kBRows, int kTmemCols>
 __device__ __forceinline__ bool tile_mma(unsigned char* smem_raw, const uint16_t* A, size_t lda,
-                                         const uint16_t* B, size_t ldb, int N, int kb0, int nloc,
-                                         uint32_t* tmem_out) {
+                                         const uint16_t* B, size_t ldb, const int* b_rows, int N,
+                                         int kb0, int nloc, uint32_t* tmem_out) {
   using C = Cfg<kStages, kBRows>;
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -152,7 +153,8 @@ __device__ __forceinline__ bool tile_mma(unsigned char* smem_raw, const uint16_t
     }
     for (int idx = tid; idx < N * 8; idx += kThreads) {
       const int row = idx >> 3, ch = idx & 7;
-      cp_async16(s32(sb + row * 128 + ((ch ^ (row & 7)) << 4)), B + (size_t)row * ldb + koff + ch * 8);
+      const int src = b_rows ? b_rows[row] : row;
+      cp_async16(s32(sb + row * 128 + ((ch ^ (row & 7)) << 4)), B + (size_t)src * ldb + koff + ch * 8);
     }
   };
 
