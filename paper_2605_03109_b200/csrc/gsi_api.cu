@@ -5,6 +5,7 @@
 #include <cstring>
 
 #include "gsi_common.cuh"
+#include "gsi_umma.cuh"
 #include "gsi_persistent.cuh"
 
 using namespace gsi;
@@ -104,6 +105,8 @@ struct gsi_layer {
   int d_out[GSI_MAX_MAPS];
   Layout lay;
   GroupParams gp;
+  TmaMaps tm;          // tensor maps of the tensor-core kernels' operands
+  bool has_tm = false;
   char* ws;
   float* pmax;     // device: max |P| (bf16 basis only)
   unsigned* bar;   // device: [2] barrier counters of the persistent kernel
@@ -231,6 +234,14 @@ gsi_status_t gsi_create(const gsi_desc_t* desc, const void* const* W, const void
   g.cpart3 = reinterpret_cast<float*>(h->ws + L.f_cpart);
   g.normpart3 = reinterpret_cast<float*>(h->ws + L.f_normpart);
 
+  if (L.tc) {
+    if (!build_tma_maps(g, L.front, desc->max_tokens, &h->tm)) {
+      delete h;
+      return GSI_ERR_CUDA;
+    }
+    h->has_tm = true;
+  }
+
   if (cudaMemsetAsync(ctrl, 0, 256, stream) != cudaSuccess ||
       cudaMemsetAsync(h->ws + L.pk_acc, 0, L.total - L.pk_acc, stream) != cudaSuccess) {
     delete h;
@@ -282,7 +293,7 @@ gsi_status_t gsi_forward_n(gsi_handle_t h, const float* x, int n_tokens, float* 
   io.step = nullptr;
   io.n_steps = 1;
   h->last_stream = stream;
-  return launch_generic_forward(h->gp, io, n_tokens, stream, nullptr) == cudaSuccess ? GSI_OK
+  return launch_generic_forward(h->gp, h->has_tm ? &h->tm : nullptr, io, n_tokens, stream, nullptr) == cudaSuccess ? GSI_OK
                                                                                       : GSI_ERR_CUDA;
 }
 
@@ -532,7 +543,7 @@ static gsi_status_t stack_enqueue(gsi_stack_t s, bool use_counter, gsi_stream_t 
     io.x_step_stride = (long long)s->B * h->desc.d;
     io.log_step_stride = (long long)G * s->B;
     h->last_stream = stream;
-    if (launch_generic_forward(h->gp, io, s->B, stream, nullptr) != cudaSuccess)
+    if (launch_generic_forward(h->gp, h->has_tm ? &h->tm : nullptr, io, s->B, stream, nullptr) != cudaSuccess)
       return GSI_ERR_CUDA;
   }
   if (use_counter && launch_advance_step(s->step, stream) != cudaSuccess) return GSI_ERR_CUDA;

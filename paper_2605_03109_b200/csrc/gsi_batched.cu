@@ -100,7 +100,8 @@ __device__ __forceinline__ void load_tokens16(uint32_t tmem_lane, int q, float (
 }
 
 // c partials: cpart3[split][t][128*tile + lane row] over this split's share of d.
-__global__ void __launch_bounds__(kThreads, 1) k_proj_tc(GroupParams g, int n_tokens) {
+__global__ void __launch_bounds__(kThreads, 1)
+k_proj_tc(GroupParams g, const __grid_constant__ TmaMaps tm, int n_tokens) {
   extern __shared__ unsigned char smem_raw[];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int splits = g.proj_splits;
@@ -108,9 +109,8 @@ __global__ void __launch_bounds__(kThreads, 1) k_proj_tc(GroupParams g, int n_to
   const int nkb = g.d / kTK;
   const int kb0 = (int)((long long)nkb * split / splits), kb1 = (int)((long long)nkb * (split + 1) / splits);
   uint32_t tmem;
-  const bool ok = tile_mma<kStages3, kMaxN3, kTmemCols3>(
-      smem_raw, g.PT + (size_t)tile * kTM * g.d, (size_t)g.d, g.xb, (size_t)g.d, nullptr, rows3(n_tokens),
-      kb0, kb1 - kb0, &tmem);
+  const bool ok = tile_mma<kStages3, kMaxN3, kTmemCols3>(smem_raw, &tm.pt, tile * kTM, &tm.xb, 0,
+                                                         rows3(n_tokens), kb0, kb1 - kb0, &tmem);
   if (!ok) {
     if (threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
   } else {
@@ -163,7 +163,7 @@ __global__ void __launch_bounds__(256) k_reduce_split3_c(GroupParams g, int n_to
 //                                      the tile, and in the block that finishes last the gate
 //   blocks [n_resid, ..)  tile of W_P: y = W_P c
 __global__ void __launch_bounds__(kThreads, 2)
-k_resid_image_tc(GroupParams g, IoRef io, int n_tokens) {
+k_resid_image_tc(GroupParams g, const __grid_constant__ TmaMaps tm, IoRef io, int n_tokens) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ float s_norm[kThreads / 32][16][2];
   __shared__ int s_last;
@@ -175,7 +175,6 @@ k_resid_image_tc(GroupParams g, IoRef io, int n_tokens) {
   const int tile = bid / nq, q = bid % nq;
   const int n_rows = min(48, rows3(n_tokens) - 48 * q);
   const int row = tile * kTM + warp * 32 + lane;
-  const uint16_t* A = (image ? g.WP : reinterpret_cast<const uint16_t*>(g.P)) + (size_t)tile * kTM * g.k;
   const int slot = io_slot(io);
 
   float xv[16];
@@ -186,8 +185,8 @@ k_resid_image_tc(GroupParams g, IoRef io, int n_tokens) {
       xv[tt] = (16 * q + tt < n_tokens) ? __ldg(x + (size_t)(16 * q + tt) * g.d) : 0.f;
   }
   uint32_t tmem;
-  const bool ok = tile_mma<kStages3, 48, 64>(smem_raw, A, (size_t)g.k, g.cb + (size_t)48 * q * g.k,
-                                             (size_t)g.k, nullptr, n_rows, 0, g.k / kTK, &tmem);
+  const bool ok = tile_mma<kStages3, 48, 64>(smem_raw, image ? &tm.wp : &tm.p, tile * kTM, &tm.cb, 48 * q,
+                                             n_rows, 0, g.k / kTK, &tmem);
   if (!ok && threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
   float s[16];
   if (ok) load_tokens16(tmem + ((uint32_t)(warp * 32) << 16), 0, s);
@@ -255,8 +254,8 @@ cudaError_t launch_transpose_bf16(const void* P, int d, int k, void* PT, cudaStr
   return cudaGetLastError();
 }
 
-cudaError_t launch_front_tc(const GroupParams& g, const IoRef& io, int n_tokens, cudaStream_t st,
-                            int* n_launches) {
+cudaError_t launch_front_tc(const GroupParams& g, const TmaMaps& tm, const IoRef& io, int n_tokens,
+                            cudaStream_t st, int* n_launches) {
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(k_proj_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem3)) != cudaSuccess ||
       (e = cudaFuncSetAttribute(k_resid_image_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemResid)) !=
@@ -265,9 +264,9 @@ cudaError_t launch_front_tc(const GroupParams& g, const IoRef& io, int n_tokens,
   const int slots = (front_rows(n_tokens) + 2) / 3;   // token slots covering every operand row
   const int nq = (n_tokens + 15) / 16;
   k_split3_x<<<dim3((g.d / 8 + 255) / 256, slots), 256, 0, st>>>(g, io, n_tokens);
-  k_proj_tc<<<(g.k / kTM) * g.proj_splits, kThreads, kSmem3, st>>>(g, n_tokens);
+  k_proj_tc<<<(g.k / kTM) * g.proj_splits, kThreads, kSmem3, st>>>(g, tm, n_tokens);
   k_reduce_split3_c<<<slots, 256, 0, st>>>(g, n_tokens);
-  k_resid_image_tc<<<(g.d / kTM + g.O / kTM) * nq, kThreads, kSmemResid, st>>>(g, io, n_tokens);
+  k_resid_image_tc<<<(g.d / kTM + g.O / kTM) * nq, kThreads, kSmemResid, st>>>(g, tm, io, n_tokens);
   if (n_launches) *n_launches += 4;
   return cudaGetLastError();
 }

@@ -177,18 +177,24 @@ __device__ __forceinline__ void decide_gate_last_block(const GroupParams& g, con
   }
 }
 
-cudaError_t launch_generic_forward(const GroupParams& g, const IoRef& io, int n_tokens,
-                                   cudaStream_t stream, int* n_launches);
+struct TmaMaps;   // tensor maps of the layer's matrices (null when no tensor-core path is on)
+
+cudaError_t launch_generic_forward(const GroupParams& g, const TmaMaps* tm, const IoRef& io,
+                                   int n_tokens, cudaStream_t stream, int* n_launches);
 cudaError_t launch_advance_step(int* step, cudaStream_t stream);
 // mapped: rb holds every token's residual (row = token) and the fired list selects the
 // operand rows; otherwise a pack kernel first compacts the fired tokens of g.r into rb.
-cudaError_t launch_residual_gemm_tc(const GroupParams& g, const IoRef& io, int min_fired,
-                                    bool mapped, cudaStream_t stream, int* n_launches);
+cudaError_t launch_residual_gemm_tc(const GroupParams& g, const TmaMaps& tm, const IoRef& io,
+                                    int min_fired, bool mapped, int n_tokens,
+                                    cudaStream_t stream, int* n_launches);
 int tc_splits(int O, int d);
 bool tc_eligible(const GroupParams& g);
 // Batched front end on the tensor cores: c, r, gate and y = W_P c for n_tokens tokens.
-cudaError_t launch_front_tc(const GroupParams& g, const IoRef& io, int n_tokens,
-                            cudaStream_t stream, int* n_launches);
+cudaError_t launch_front_tc(const GroupParams& g, const TmaMaps& tm, const IoRef& io,
+                            int n_tokens, cudaStream_t stream, int* n_launches);
+// Encodes the layer's tensor maps (front: also those of the batched front end).
+// False when the driver's encoder is unavailable or rejects a shape.
+bool build_tma_maps(const GroupParams& g, bool front, int max_tokens, TmaMaps* out);
 cudaError_t launch_transpose_bf16(const void* P, int d, int k, void* PT, cudaStream_t stream);
 int front_proj_splits(int d, int k);
 int front_rows(int max_tokens);   // rows of the three-term operands

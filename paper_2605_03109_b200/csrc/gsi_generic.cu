@@ -364,8 +364,8 @@ cudaError_t launch_vpl(const GroupParams& g, const IoRef& io, int n_tokens, cuda
 
 }  // namespace
 
-cudaError_t launch_generic_forward(const GroupParams& g, const IoRef& io, int n_tokens,
-                                   cudaStream_t st, int* n_launches) {
+cudaError_t launch_generic_forward(const GroupParams& g, const TmaMaps* tm, const IoRef& io,
+                                   int n_tokens, cudaStream_t st, int* n_launches) {
   int dummy = 0;
   if (!n_launches) n_launches = &dummy;
   int grid = (g.O + kWarps - 1) / kWarps;
@@ -377,9 +377,9 @@ cudaError_t launch_generic_forward(const GroupParams& g, const IoRef& io, int n_
   }
   const RowLayout L = make_layout(g.k);
   cudaError_t e;
-  const bool front = g.front_min_tokens > 0 && n_tokens >= g.front_min_tokens;
+  const bool front = tm && g.front_min_tokens > 0 && n_tokens >= g.front_min_tokens;
   if (front) {
-    e = launch_front_tc(g, io, n_tokens, st, n_launches);
+    e = launch_front_tc(g, *tm, io, n_tokens, st, n_launches);
   } else {
     switch (L.VPL) {
       case 1: e = launch_vpl<1>(g, io, n_tokens, st, n_launches); break;
@@ -393,13 +393,13 @@ cudaError_t launch_generic_forward(const GroupParams& g, const IoRef& io, int n_
   if (!(g.flags & GSI_FLAG_STATIC_PROJECTION)) {
     if (front) {
       // every gated token goes through the tensor-core contraction; r is in rb already
-      e = launch_residual_gemm_tc(g, io, 1, true, st, n_launches);
+      e = launch_residual_gemm_tc(g, *tm, io, 1, true, n_tokens, st, n_launches);
       if (e != cudaSuccess) return e;
     } else {
       k_stream_gemv<false><<<grid, kThreads, 0, st>>>(g, io, n_tokens);
       *n_launches += 1;
-      if (g.tc_min_fired > 0) {
-        e = launch_residual_gemm_tc(g, io, g.tc_min_fired, false, st, n_launches);
+      if (tm && g.tc_min_fired > 0) {
+        e = launch_residual_gemm_tc(g, *tm, io, g.tc_min_fired, false, n_tokens, st, n_launches);
         if (e != cudaSuccess) return e;
       }
     }

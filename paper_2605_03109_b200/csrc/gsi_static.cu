@@ -127,6 +127,6 @@ extern "C" gsi_status_t gsi_forward_static(const void* const* W_host_array, cons
   io.rho = rho_out;
   io.step = nullptr;
   io.n_steps = 1;
-  return launch_generic_forward(g, io, n_tokens, stream, nullptr) == cudaSuccess ? GSI_OK
+  return launch_generic_forward(g, nullptr, io, n_tokens, stream, nullptr) == cudaSuccess ? GSI_OK
                                                                                   : GSI_ERR_CUDA;
 }

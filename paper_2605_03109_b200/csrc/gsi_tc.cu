@@ -7,8 +7,8 @@
 // tensor ridge), the tensor pipe is only the means to stay on the HBM roofline
 // once there are too many tokens for CUDA-core FMAs.
 //
-//   A (W tile, 128 x 64 bf16 per stage)   global -> shared by cp.async, written in the
-//   B (R tile,   N x 64 bf16 per stage)   128-byte-swizzled K-major layout tcgen05 reads
+//   A (W tile, 128 x 64 bf16 per stage)   global -> shared by TMA in the 128-byte-swizzled
+//   B (R tile,   N x 64 bf16 per stage)   K-major layout tcgen05 reads
 //   D (128 lanes x N columns fp32)        tensor memory; tcgen05.mma, one issuing thread
 //   epilogue                              tcgen05.ld -> registers -> partial-sum buffer
 //
@@ -24,7 +24,7 @@ namespace {
 
 using namespace umma;
 
-constexpr int kStages = 6;
+constexpr int kStages = 4;   // 4 x 24 KB: two blocks per SM
 constexpr int kMaxN = 64;
 constexpr int kTmemCols = 64;
 using TcCfg = Cfg<kStages, kMaxN>;
@@ -44,56 +44,72 @@ __global__ void __launch_bounds__(256) k_pack_fired_bf16(GroupParams g, int min_
   }
 }
 
-__global__ void __launch_bounds__(kThreadsTc, 1)
-k_residual_gemm_tc(GroupParams g, int min_fired, int splits, int mapped) {
+// mapped == 0: B rows are the fired tokens compacted (N = fired count rounded up to 16).
+// mapped == 1: B rows are all n_tokens tokens of the call (row = token); only the columns
+//              of fired tokens are written out.
+__global__ void __launch_bounds__(kThreadsTc, 2)
+k_residual_gemm_tc(GroupParams g, const __grid_constant__ TmaMaps tm, int min_fired, int splits,
+                   int mapped, int n_tokens) {
   const int n_fired = *g.n_fired;
-  if (n_fired < min_fired) return;            // the CUDA-core GEMV handles the few-token case
-  const int N = (n_fired + 15) & ~15;         // 16..64
+  if (n_fired < min_fired) return;            // nothing gated, or the CUDA-core GEMV takes the few
+  const int n_cols = mapped ? n_tokens : n_fired;
+  const int N = (n_cols + 15) & ~15;          // 16..64
 
   extern __shared__ unsigned char smem_raw[];
-  __shared__ int s_rows[kMaxN];   // operand row n <- row of rb (mapped mode)
-  if (mapped && threadIdx.x < kMaxN)
-    s_rows[threadIdx.x] = (int)threadIdx.x < n_fired ? g.fired[threadIdx.x] : kMaxN;   // row 64 is zero
+  __shared__ unsigned long long s_mask;       // columns to write out
+  if (threadIdx.x == 0) {
+    unsigned long long m = 0ull;
+    if (mapped) {
+      for (int n = 0; n < n_fired; ++n) m |= 1ull << g.fired[n];
+    } else {
+      m = n_fired >= 64 ? ~0ull : ((1ull << n_fired) - 1ull);
+    }
+    s_mask = m;
+  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = blockIdx.x / splits, split = blockIdx.x % splits;
   const int row0 = tile * kTM;                 // first row of the concatenated maps
   int j = 0;
-  while (j + 1 < g.n_maps && row0 >= g.off[j + 1]) ++j;
-  const uint16_t* Wt = g.W[j] + (size_t)(row0 - g.off[j]) * g.d;   // tile never straddles maps
+  while (j + 1 < g.n_maps && row0 >= g.off[j + 1]) ++j;   // a tile never straddles two maps
   const int nkb = g.d / kTK;
   const int kb0 = (int)((long long)nkb * split / splits), kb1 = (int)((long long)nkb * (split + 1) / splits);
   const int nloc = kb1 - kb0;
 
   uint32_t tmem;
-  const bool ok = tile_mma<kStages, kMaxN, kTmemCols>(smem_raw, Wt, (size_t)g.d, g.rb, (size_t)g.d,
-                                                      mapped ? s_rows : nullptr, N, kb0, nloc, &tmem);
+  const bool ok = tile_mma<kStages, kMaxN, kTmemCols>(smem_raw, &tm.w[j], row0 - g.off[j], &tm.rb, 0, N,
+                                                      kb0, nloc, &tmem);
   if (!ok) {
     if (threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
   } else if (nloc > 0) {
     // warp w owns tensor-memory lanes 32w..32w+31 = rows row0+32w+lane; 16 columns per load
+    const unsigned long long mask = s_mask;
     float* yp = g.ypart + ((size_t)split * kMaxN) * g.O + row0 + warp * 32 + lane;
     for (int c0 = 0; c0 < N; c0 += 16) {
+      if (((mask >> c0) & 0xFFFFull) == 0ull) continue;
       uint32_t v[16];
       tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + c0, v);
       tmem_ld_wait();
 #pragma unroll
       for (int c = 0; c < 16; ++c)
-        if (c0 + c < n_fired) yp[(size_t)(c0 + c) * g.O] = __uint_as_float(v[c]);
+        if ((mask >> (c0 + c)) & 1ull) yp[(size_t)(c0 + c) * g.O] = __uint_as_float(v[c]);
     }
   }
   tile_release<kTmemCols>(tmem);
 }
 
-// y[fired[n]][row] += sum over splits (fixed order)
-__global__ void __launch_bounds__(256) k_add_partials(GroupParams g, IoRef io, int min_fired, int splits) {
+// y[fired[n]][row] += sum over splits (fixed order); the partial sums of fired token n
+// are column n (compacted) or column fired[n] (mapped)
+__global__ void __launch_bounds__(256) k_add_partials(GroupParams g, IoRef io, int min_fired, int splits,
+                                                      int mapped) {
   const int n = *g.n_fired;
   if (n < min_fired) return;
   const int t = blockIdx.y;
   if (t >= n) return;
   const int tok = g.fired[t];
+  const int col = mapped ? tok : t;
   for (int row = blockIdx.x * 256 + threadIdx.x; row < g.O; row += gridDim.x * 256) {
     float s = 0.f;
-    for (int sp = 0; sp < splits; ++sp) s += g.ypart[((size_t)sp * kMaxN + t) * g.O + row];
+    for (int sp = 0; sp < splits; ++sp) s += g.ypart[((size_t)sp * kMaxN + col) * g.O + row];
     io.y[(size_t)tok * g.O + row] += s;
   }
 }
@@ -116,15 +132,17 @@ bool tc_eligible(const GroupParams& g) {
   return true;
 }
 
-cudaError_t launch_residual_gemm_tc(const GroupParams& g, const IoRef& io, int min_fired,
-                                    bool mapped, cudaStream_t st, int* n_launches) {
+cudaError_t launch_residual_gemm_tc(const GroupParams& g, const TmaMaps& tm, const IoRef& io,
+                                    int min_fired, bool mapped, int n_tokens, cudaStream_t st,
+                                    int* n_launches) {
   cudaError_t e = cudaFuncSetAttribute(k_residual_gemm_tc,
                                        cudaFuncAttributeMaxDynamicSharedMemorySize, kTcSmem);
   if (e != cudaSuccess) return e;
   const int splits = tc_splits(g.O, g.d);
   if (!mapped) k_pack_fired_bf16<<<dim3((g.d + 2047) / 2048, kMaxN), 256, 0, st>>>(g, min_fired);
-  k_residual_gemm_tc<<<(g.O / kTM) * splits, kThreadsTc, kTcSmem, st>>>(g, min_fired, splits, mapped ? 1 : 0);
-  k_add_partials<<<dim3((g.O + 1023) / 1024, g.B), 256, 0, st>>>(g, io, min_fired, splits);
+  k_residual_gemm_tc<<<(g.O / kTM) * splits, kThreadsTc, kTcSmem, st>>>(g, tm, min_fired, splits,
+                                                                        mapped ? 1 : 0, n_tokens);
+  k_add_partials<<<dim3((g.O + 1023) / 1024, g.B), 256, 0, st>>>(g, io, min_fired, splits, mapped ? 1 : 0);
   if (n_launches) *n_launches += mapped ? 2 : 3;
   return cudaGetLastError();
 }

@@ -2,14 +2,20 @@
 // kernels: D[128 x N] (fp32, tensor memory) = A[128 x K] * B[N x K]^T with bf16
 // operands that are both K-major in global memory.
 //
-//   A, B tiles (64 K-elements = 128 bytes per row and stage) go global -> shared by
-//   cp.async, written in the 128-byte-swizzled K-major layout the descriptors name;
-//   one thread issues tcgen05.mma; tcgen05.commit frees a stage through an mbarrier;
-//   the caller reads D with tcgen05.ld and then releases the tensor memory.
+//   producer thread   TMA (cp.async.bulk.tensor, 128-byte swizzle, no multicast) brings a
+//                     stage = A box 128 rows x 64 K-elements + N/16 B boxes of 16 rows into
+//                     shared memory and signals the stage's "full" mbarrier by byte count
+//   MMA thread        waits "full", issues tcgen05.mma (accumulator in tensor memory),
+//                     tcgen05.commit arrives on the stage's "empty" mbarrier
+//   all four warps    wait for the final commit, read D with tcgen05.ld (lane = row)
 //
-// Every wait is bounded: a timeout makes tile_mma return false (uniformly for the
-// block) and the caller reports it; the tensor memory is released in either case.
+// The two loops never meet at a block-wide barrier, so the stages in flight are limited
+// by shared memory only.  Every wait is bounded: a timeout makes tile_mma return false
+// (uniformly for the block) after a bounded wait for the copies still in flight; the
+// caller reports it and releases the tensor memory in either case.
 #pragma once
+
+#include <cuda.h>   // CUtensorMap (type only; the encoder is looked up at run time)
 
 #include "gsi_common.cuh"
 
@@ -18,6 +24,7 @@ namespace umma {
 
 constexpr int kTM = 128;          // rows of A per tile (tensor-memory lanes)
 constexpr int kTK = 64;           // K elements per stage: 128 bytes of bf16 = one swizzle row
+constexpr int kBBox = 16;         // rows per B box
 constexpr int kThreads = 128;
 constexpr int kABytes = kTM * kTK * 2;     // 16 KB
 constexpr unsigned kSpin = 1u << 22;
@@ -27,21 +34,18 @@ struct Cfg {
   static constexpr int kBBytes = kBRows * kTK * 2;
   static constexpr int kStageBytes = kABytes + kBBytes;
   static constexpr int kSmem = 1024 /*align slack*/ + kStages * kStageBytes + 256;
+  static_assert(kStageBytes % 1024 == 0, "stage bases must keep the 1024-byte swizzle alignment");
 };
 
 __device__ __forceinline__ uint32_t s32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
 }
-__device__ __forceinline__ void cp_async16(uint32_t dst, const void* src) {
-  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(src) : "memory");
-}
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
-template <int N>
-__device__ __forceinline__ void cp_async_wait() {
-  asm volatile("cp.async.wait_group %0;" ::"n"(N) : "memory");
-}
 __device__ __forceinline__ void mbar_init(uint64_t* b, int count) {
   asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s32(b)), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s32(b)), "r"(bytes)
+               : "memory");
 }
 __device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
   uint32_t ok;
@@ -53,10 +57,18 @@ __device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
       : "memory");
   return ok != 0;
 }
-__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity) {
-  for (unsigned it = 0; it < kSpin; ++it)
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, unsigned spin = kSpin) {
+  for (unsigned it = 0; it < spin; ++it)
     if (mbar_try(b, parity)) return true;
   return false;
+}
+// One box of a 2-D tensor map: x = first K element, y = first row.
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y,
+                                            uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(map), "r"(x), "r"(y), "r"(s32(bar))
+      : "memory");
 }
 
 // Shared-memory matrix descriptor, K-major operand in the 128-byte swizzle:
@@ -100,29 +112,32 @@ __device__ __forceinline__ void tmem_ld_wait() {
   asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
 
-// Runs the whole contraction of one tile: rows [0,128) of A (row stride lda
-// elements), rows [0,N) of B (row stride ldb; operand row n is row b_rows[n] of B when
-// b_rows, a table the block wrote before the call, is not null), K blocks
-// [kb0, kb0+nloc) of 64 elements.  N is a multiple of 16 in [16, kBRows].  All kThreads threads of the
-// block call it.  On return *tmem_out holds the tensor-memory base of D (lane =
-// row, column = B row); the return value, the same for every thread, is false when a
-// wait ran out of time.  With nloc == 0 nothing is accumulated and D is undefined.
-// The caller must end with tile_release<kTmemCols>(*tmem_out).
+// Runs the whole contraction of one tile: rows [a_row0, a_row0+128) of the matrix behind
+// map_a, rows [b_row0, b_row0+N) of the matrix behind map_b, K blocks [kb0, kb0+nloc)
+// of 64 elements.  N is a multiple of 16 in [16, kBRows].  All kThreads threads of the
+// block call it.  On return *tmem_out holds the tensor-memory base of D (lane = row,
+// column = B row); the return value, the same for every thread, is false when a wait ran
+// out of time.  With nloc == 0 nothing is accumulated and D is undefined.  The caller
+// must end with tile_release<kTmemCols>(*tmem_out).
 template <int kStages, int kBRows, int kTmemCols>
-__device__ __forceinline__ bool tile_mma(unsigned char* smem_raw, const uint16_t* A, size_t lda,
-                                         const uint16_t* B, size_t ldb, const int* b_rows, int N,
+__device__ __forceinline__ bool tile_mma(unsigned char* smem_raw, const CUtensorMap* map_a,
+                                         int a_row0, const CUtensorMap* map_b, int b_row0, int N,
                                          int kb0, int nloc, uint32_t* tmem_out) {
   using C = Cfg<kStages, kBRows>;
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
-  uint64_t* bar_free = reinterpret_cast<uint64_t*>(smem + kStages * C::kStageBytes);  // [kStages]
-  uint64_t* bar_done = bar_free + kStages;
+  uint64_t* bar_full = reinterpret_cast<uint64_t*>(smem + kStages * C::kStageBytes);  // [kStages]
+  uint64_t* bar_empty = bar_full + kStages;                                            // [kStages]
+  uint64_t* bar_done = bar_empty + kStages;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bar_done + 1);
   int* s_fail = reinterpret_cast<int*>(tmem_slot + 1);
-  const int tid = threadIdx.x, warp = tid >> 5;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
 
   if (tid == 0) {
-    for (int s = 0; s < kStages; ++s) mbar_init(&bar_free[s], 1);
+    for (int s = 0; s < kStages; ++s) {
+      mbar_init(&bar_full[s], 1);
+      mbar_init(&bar_empty[s], 1);
+    }
     mbar_init(bar_done, 1);
     *s_fail = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -139,64 +154,60 @@ __device__ __forceinline__ bool tile_mma(unsigned char* smem_raw, const uint16_t
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = *tmem_slot;
   *tmem_out = tmem;
+  const uint32_t stage_bytes = (uint32_t)(kABytes + N * kTK * 2);
 
-  // one stage: A tile 128 rows x 8 chunks of 16 B, B tile N rows x 8 chunks, both written
-  // at chunk ^ (row & 7): the 128-byte swizzle the descriptors announce
-  auto load_stage = [&](int kb, int stage) {
-    unsigned char* sa = smem + stage * C::kStageBytes;
-    unsigned char* sb = sa + kABytes;
-    const size_t koff = (size_t)kb * kTK;   // elements
-#pragma unroll
-    for (int it = 0; it < (kTM * 8) / kThreads; ++it) {
-      const int idx = it * kThreads + tid, row = idx >> 3, ch = idx & 7;
-      cp_async16(s32(sa + row * 128 + ((ch ^ (row & 7)) << 4)), A + (size_t)row * lda + koff + ch * 8);
-    }
-    for (int idx = tid; idx < N * 8; idx += kThreads) {
-      const int row = idx >> 3, ch = idx & 7;
-      const int src = b_rows ? b_rows[row] : row;
-      cp_async16(s32(sb + row * 128 + ((ch ^ (row & 7)) << 4)), B + (size_t)src * ldb + koff + ch * 8);
-    }
-  };
-
-  for (int s = 0; s < kStages - 1; ++s) {
-    if (s < nloc) load_stage(kb0 + s, s);
-    cp_async_commit();
-  }
-  const uint32_t idesc = instr_desc(kTM, N);
-  bool ok = true;
-  for (int i = 0; i < nloc && ok; ++i) {
-    const int stage = i % kStages;
-    cp_async_wait<kStages - 2>();                                    // block i of this thread landed
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");    // ...and is visible to the tensor core
-    __syncthreads();
-    if (tid == 0) {
-      asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
-      const uint32_t a0 = s32(smem + stage * C::kStageBytes), b0 = a0 + kABytes;
-#pragma unroll
-      for (int k = 0; k < kTK / 16; ++k)   // 32 bytes further along K per instruction
-        umma_bf16(tmem, smem_desc_sw128(a0 + k * 32), smem_desc_sw128(b0 + k * 32), idesc,
-                  (i > 0 || k > 0) ? 1u : 0u);
-      umma_commit(&bar_free[stage]);       // arrives when the tensor core has read this stage
-    }
-    // refill the stage block i-1 used with block i+kStages-1
-    const int nb = i + kStages - 1;
-    if (nb < nloc) {
-      if (i >= 1) {
-        const int ps = (i - 1) % kStages;
-        if (!mbar_wait(&bar_free[ps], ((i - 1) / kStages) & 1)) {
+  if (warp == 0) {
+    if (lane == 0) {   // producer
+      for (int i = 0; i < nloc; ++i) {
+        const int stage = i % kStages;
+        if (i >= kStages && !mbar_wait(&bar_empty[stage], ((i / kStages) - 1) & 1)) {
           *s_fail = 1;
-          ok = false;
+          break;
         }
+        mbar_expect_tx(&bar_full[stage], stage_bytes);
+        const uint32_t sa = s32(smem + stage * C::kStageBytes), sb = sa + kABytes;
+        const int x = (kb0 + i) * kTK;
+        tma_load_2d(sa, map_a, x, a_row0, &bar_full[stage]);
+        for (int j = 0; j < N / kBBox; ++j)
+          tma_load_2d(sb + j * (kBBox * kTK * 2), map_b, x, b_row0 + j * kBBox, &bar_full[stage]);
       }
-      if (ok) load_stage(kb0 + nb, nb % kStages);
     }
-    cp_async_commit();
+    __syncwarp();
+  } else if (warp == 1) {
+    if (lane == 0) {   // MMA issuer
+      const uint32_t idesc = instr_desc(kTM, N);
+      bool ok = true;
+      for (int i = 0; i < nloc; ++i) {
+        const int stage = i % kStages;
+        if (!mbar_wait(&bar_full[stage], (i / kStages) & 1)) {
+          ok = false;
+          break;
+        }
+        asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
+        const uint32_t a0 = s32(smem + stage * C::kStageBytes), b0 = a0 + kABytes;
+#pragma unroll
+        for (int k = 0; k < kTK / 16; ++k)   // 32 bytes further along K per instruction
+          umma_bf16(tmem, smem_desc_sw128(a0 + k * 32), smem_desc_sw128(b0 + k * 32), idesc,
+                    (i > 0 || k > 0) ? 1u : 0u);
+        umma_commit(&bar_empty[stage]);      // arrives when the tensor core has read this stage
+      }
+      if (ok) umma_commit(bar_done);
+      else *s_fail = 1;
+    }
+    __syncwarp();
   }
-  cp_async_wait<0>();
-  if (tid == 0) umma_commit(bar_done);
-  __syncthreads();
-  const bool mine = !*s_fail && mbar_wait(bar_done, 0);
+  // Everyone: the accumulator is complete when the last commit arrives.  Warps 2 and 3
+  // come straight here and poll while the pipeline runs.
+  bool mine = mbar_wait(bar_done, 0, kSpin * 8);
+  if (*reinterpret_cast<volatile int*>(s_fail)) mine = false;
   const bool done = __syncthreads_and(mine ? 1 : 0) != 0;   // the same answer for every thread
+  if (!done && tid == 0) {
+    // copies issued but not consumed: give them a bounded time to land before the block exits
+    for (int s = 0; s < kStages && s < nloc; ++s) {
+      const int last = ((nloc - 1 - s) / kStages) * kStages + s;   // last block that used stage s
+      (void)mbar_wait(&bar_full[s], (last / kStages) & 1, 1u << 16);
+    }
+  }
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   return done;
 }
@@ -211,4 +222,18 @@ __device__ __forceinline__ void tile_release(uint32_t tmem) {
 }
 
 }  // namespace umma
+
+// Tensor maps of one layer (host-encoded at set-up, passed to the kernels by value as a
+// __grid_constant__ parameter).  A operands use boxes of 128 rows, B operands of 16 rows;
+// every box is 64 K-elements wide with the 128-byte swizzle.
+struct alignas(64) TmaMaps {
+  CUtensorMap w[GSI_MAX_MAPS];   // W_j [d_out_j][d]
+  CUtensorMap p;                 // P   [d][k]
+  CUtensorMap pt;                // P^T [k][d]
+  CUtensorMap wp;                // W_P [O][k]
+  CUtensorMap xb;                // terms of x [rows][d]   (B operand)
+  CUtensorMap cb;                // terms of c [rows][k]   (B operand)
+  CUtensorMap rb;                // residuals  [65][d]     (B operand)
+};
+
 }  // namespace gsi
