@@ -70,6 +70,7 @@ __device__ __forceinline__ void store_terms(const float (&v)[8], bool live, uint
 }
 
 __global__ void __launch_bounds__(256) k_split3_x(GroupParams g, IoRef io, int n_tokens) {
+  pdl_launch_dependents();
   const int slot = blockIdx.y, n_rows = rows3(n_tokens);
   const bool live = slot < n_tokens;
   const float* x = io.x + (long long)io_slot(io) * io.x_step_stride + (size_t)slot * g.d;
@@ -103,6 +104,7 @@ __device__ __forceinline__ void load_tokens16(uint32_t tmem_lane, int q, float (
 __global__ void __launch_bounds__(kThreads, 1)
 k_proj_tc(GroupParams g, const __grid_constant__ TmaMaps tm, int n_tokens) {
   extern __shared__ unsigned char smem_raw[];
+  pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int splits = g.proj_splits;
   const int tile = blockIdx.x / splits, split = blockIdx.x % splits;
@@ -132,6 +134,8 @@ k_proj_tc(GroupParams g, const __grid_constant__ TmaMaps tm, int n_tokens) {
 __global__ void __launch_bounds__(256) k_reduce_split3_c(GroupParams g, int n_tokens) {
   const int slot = blockIdx.x, n_rows = rows3(n_tokens);
   const bool live = slot < n_tokens;
+  pdl_launch_dependents();
+  pdl_wait();
   for (int j = threadIdx.x; j < g.k; j += 256) {
     float v = 0.f;
     if (live) {
@@ -167,6 +171,7 @@ k_resid_image_tc(GroupParams g, const __grid_constant__ TmaMaps tm, IoRef io, in
   extern __shared__ unsigned char smem_raw[];
   __shared__ float s_norm[kThreads / 32][16][2];
   __shared__ int s_last;
+  pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nq = (n_tokens + 15) / 16;
   const int n_resid = (g.d / kTM) * nq;
@@ -264,9 +269,14 @@ cudaError_t launch_front_tc(const GroupParams& g, const TmaMaps& tm, const IoRef
   const int slots = (front_rows(n_tokens) + 2) / 3;   // token slots covering every operand row
   const int nq = (n_tokens + 15) / 16;
   k_split3_x<<<dim3((g.d / 8 + 255) / 256, slots), 256, 0, st>>>(g, io, n_tokens);
-  k_proj_tc<<<(g.k / kTM) * g.proj_splits, kThreads, kSmem3, st>>>(g, tm, n_tokens);
-  k_reduce_split3_c<<<slots, 256, 0, st>>>(g, n_tokens);
-  k_resid_image_tc<<<(g.d / kTM + g.O / kTM) * nq, kThreads, kSmemResid, st>>>(g, tm, io, n_tokens);
+  // the x the residual blocks read before their wait is an input of the call, complete before
+  // k_split3_x was launched
+  if ((e = launch_pdl(k_proj_tc, dim3((g.k / kTM) * g.proj_splits), dim3(kThreads), kSmem3, st, g, tm,
+                      n_tokens)) != cudaSuccess ||
+      (e = launch_pdl(k_reduce_split3_c, dim3(slots), dim3(256), 0, st, g, n_tokens)) != cudaSuccess ||
+      (e = launch_pdl(k_resid_image_tc, dim3((g.d / kTM + g.O / kTM) * nq), dim3(kThreads), kSmemResid, st,
+                      g, tm, io, n_tokens)) != cudaSuccess)
+    return e;
   if (n_launches) *n_launches += 4;
   return cudaGetLastError();
 }

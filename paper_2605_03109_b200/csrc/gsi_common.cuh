@@ -64,6 +64,16 @@ __device__ __forceinline__ uint4 ld_stream(const uint4* p) {
   return v;
 }
 
+// Programmatic dependent launch.  A kernel calls pdl_launch_dependents() first, so the next
+// kernel of the stream (if it was launched with launch_pdl) may be scheduled and run its
+// set-up while this one finishes, and pdl_wait() before it touches anything an earlier kernel
+// of the stream wrote or still reads; the wait returns once every earlier kernel has completed
+// and flushed.  Both are no-ops for a kernel launched the ordinary way.
+__device__ __forceinline__ void pdl_launch_dependents() {
+  asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -175,6 +185,24 @@ __device__ __forceinline__ void decide_gate_last_block(const GroupParams& g, con
     *g.n_fired = n;
     *g.counter = 0u;
   }
+}
+
+// Launch that lets the kernel start before its predecessor in the stream has finished
+// (the kernel must call pdl_wait()).
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                       cudaStream_t stream, Args... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kernel, KArgs(args)...);
 }
 
 struct TmaMaps;   // tensor maps of the layer's matrices (null when no tensor-core path is on)

@@ -50,6 +50,8 @@ __global__ void __launch_bounds__(256) k_pack_fired_bf16(GroupParams g, int min_
 __global__ void __launch_bounds__(kThreadsTc, 2)
 k_residual_gemm_tc(GroupParams g, const __grid_constant__ TmaMaps tm, int min_fired, int splits,
                    int mapped, int n_tokens) {
+  pdl_launch_dependents();
+  pdl_wait();   // the fired list comes from the kernel before
   const int n_fired = *g.n_fired;
   if (n_fired < min_fired) return;            // nothing gated, or the CUDA-core GEMV takes the few
   const int n_cols = mapped ? n_tokens : n_fired;
@@ -101,6 +103,8 @@ k_residual_gemm_tc(GroupParams g, const __grid_constant__ TmaMaps tm, int min_fi
 // are column n (compacted) or column fired[n] (mapped)
 __global__ void __launch_bounds__(256) k_add_partials(GroupParams g, IoRef io, int min_fired, int splits,
                                                       int mapped) {
+  pdl_launch_dependents();
+  pdl_wait();
   const int n = *g.n_fired;
   if (n < min_fired) return;
   const int t = blockIdx.y;
@@ -140,9 +144,18 @@ cudaError_t launch_residual_gemm_tc(const GroupParams& g, const TmaMaps& tm, con
   if (e != cudaSuccess) return e;
   const int splits = tc_splits(g.O, g.d);
   if (!mapped) k_pack_fired_bf16<<<dim3((g.d + 2047) / 2048, kMaxN), 256, 0, st>>>(g, min_fired);
-  k_residual_gemm_tc<<<(g.O / kTM) * splits, kThreadsTc, kTcSmem, st>>>(g, tm, min_fired, splits,
-                                                                        mapped ? 1 : 0, n_tokens);
-  k_add_partials<<<dim3((g.O + 1023) / 1024, g.B), 256, 0, st>>>(g, io, min_fired, splits, mapped ? 1 : 0);
+  if (mapped) {
+    // straight after the residual kernel: both may start while their predecessor drains
+    if ((e = launch_pdl(k_residual_gemm_tc, dim3((g.O / kTM) * splits), dim3(kThreadsTc), kTcSmem, st, g,
+                        tm, min_fired, splits, 1, n_tokens)) != cudaSuccess ||
+        (e = launch_pdl(k_add_partials, dim3((g.O + 1023) / 1024, g.B), dim3(256), 0, st, g, io,
+                        min_fired, splits, 1)) != cudaSuccess)
+      return e;
+  } else {
+    k_residual_gemm_tc<<<(g.O / kTM) * splits, kThreadsTc, kTcSmem, st>>>(g, tm, min_fired, splits, 0,
+                                                                          n_tokens);
+    k_add_partials<<<dim3((g.O + 1023) / 1024, g.B), 256, 0, st>>>(g, io, min_fired, splits, 0);
+  }
   if (n_launches) *n_launches += mapped ? 2 : 3;
   return cudaGetLastError();
 }

@@ -154,6 +154,7 @@ __device__ __forceinline__ bool tile_mma(unsigned char* smem_raw, const CUtensor
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = *tmem_slot;
   *tmem_out = tmem;
+  pdl_wait();   // the operands may come from the previous kernel of the stream
   const uint32_t stage_bytes = (uint32_t)(kABytes + N * kTK * 2);
 
   if (warp == 0) {
