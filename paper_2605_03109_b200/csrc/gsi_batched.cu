@@ -25,7 +25,6 @@ constexpr int kMaxN3 = 192;          // 3 terms x 64 tokens
 constexpr int kTmemCols3 = 256;      // power of two >= kMaxN3
 using Cfg3 = Cfg<kStages3, kMaxN3>;
 constexpr int kSmem3 = Cfg3::kSmem;  // 4 x (16 + 24) KB + slack
-constexpr int kSmemResid = Cfg<kStages3, 48>::kSmem;   // 16 tokens per block
 
 __device__ __forceinline__ uint16_t bf16_bits(float v) {
   const __nv_bfloat16 h = __float2bfloat16_rn(v);
@@ -161,67 +160,81 @@ __global__ void __launch_bounds__(256) k_reduce_split3_c(GroupParams g, int n_to
 }
 
 // One launch for Algorithm 1 lines 2-5.  Every block contracts one 128-row tile against
-// the c terms of 16 tokens (operand rows 48q .. 48q+47), which spreads even the narrow
-// inputs (d = 4096: 32 tiles) over the machine:
-//   blocks [0, n_resid)   tile of P:   r = x - P c -> bf16 rows of rb, the partial norms of
-//                                      the tile, and in the block that finishes last the gate
-//   blocks [n_resid, ..)  tile of W_P: y = W_P c
-__global__ void __launch_bounds__(kThreads, 2)
-k_resid_image_tc(GroupParams g, const __grid_constant__ TmaMaps tm, IoRef io, int n_tokens) {
+// the c terms of a range of 16-token groups (operand rows 48 q_lo .. 48 q_hi - 1):
+//   blocks [0, n_resid)   tile of P, one of rs token ranges (rs > 1 spreads the narrow
+//                         inputs, d = 4096: 32 tiles, over the machine):
+//                         r = x - P c -> bf16 rows of rb, the partial norms of the tile,
+//                         and in the block that finishes last the gate
+//   blocks [n_resid, ..)  tile of W_P, all tokens: y = W_P c
+__global__ void __launch_bounds__(kThreads, 1)
+k_resid_image_tc(GroupParams g, const __grid_constant__ TmaMaps tm, IoRef io, int n_tokens, int rs) {
   extern __shared__ unsigned char smem_raw[];
-  __shared__ float s_norm[kThreads / 32][16][2];
+  __shared__ float s_norm[kThreads / 32][GSI_MAX_TOKENS][2];
   __shared__ int s_last;
   pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int nq = (n_tokens + 15) / 16;
-  const int n_resid = (g.d / kTM) * nq;
+  const int n_resid = (g.d / kTM) * rs;
   const bool image = (int)blockIdx.x >= n_resid;
-  const int bid = image ? blockIdx.x - n_resid : blockIdx.x;
-  const int tile = bid / nq, q = bid % nq;
-  const int n_rows = min(48, rows3(n_tokens) - 48 * q);
+  const int tile = image ? (int)blockIdx.x - n_resid : (int)blockIdx.x / rs;
+  const int part = image ? 0 : (int)blockIdx.x % rs;
+  const int per = image ? nq : (nq + rs - 1) / rs;
+  const int q_lo = min(part * per, nq), q_hi = min(q_lo + per, nq);
   const int row = tile * kTM + warp * 32 + lane;
   const int slot = io_slot(io);
+  const float* x = io.x + (long long)slot * io.x_step_stride + row;
 
   float xv[16];
-  if (!image) {
-    const float* x = io.x + (long long)slot * io.x_step_stride + row;
+  if (!image && q_lo < q_hi) {
 #pragma unroll
     for (int tt = 0; tt < 16; ++tt)
-      xv[tt] = (16 * q + tt < n_tokens) ? __ldg(x + (size_t)(16 * q + tt) * g.d) : 0.f;
+      xv[tt] = (16 * q_lo + tt < n_tokens) ? __ldg(x + (size_t)(16 * q_lo + tt) * g.d) : 0.f;
   }
-  uint32_t tmem;
-  const bool ok = tile_mma<kStages3, 48, 64>(smem_raw, image ? &tm.wp : &tm.p, tile * kTM, &tm.cb, 48 * q,
-                                             n_rows, 0, g.k / kTK, &tmem);
-  if (!ok && threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
-  float s[16];
-  if (ok) load_tokens16(tmem + ((uint32_t)(warp * 32) << 16), 0, s);
-  tile_release<64>(tmem);
-  if (image) {
-    if (ok) {
+  uint32_t tmem = 0;
+  bool ok = true;
+  if (q_lo < q_hi) {   // block-uniform
+    const int n_rows = min(48 * (q_hi - q_lo), rows3(n_tokens) - 48 * q_lo);
+    ok = tile_mma<kStages3, kMaxN3, kTmemCols3>(smem_raw, image ? &tm.wp : &tm.p, tile * kTM, &tm.cb,
+                                                48 * q_lo, n_rows, 0, g.k / kTK, &tmem);
+    if (!ok && threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
+    const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);
+    for (int q = q_lo; q < q_hi && ok; ++q) {
+      float s[16];
+      load_tokens16(tl, q - q_lo, s);
+      if (image) {
+#pragma unroll
+        for (int tt = 0; tt < 16; ++tt)
+          if (16 * q + tt < n_tokens) io.y[(size_t)(16 * q + tt) * g.O + row] = s[tt];
+        continue;
+      }
+      float xn[16];   // the next group's x, in flight while this group is reduced
 #pragma unroll
       for (int tt = 0; tt < 16; ++tt)
-        if (16 * q + tt < n_tokens) io.y[(size_t)(16 * q + tt) * g.O + row] = s[tt];
-    }
-    return;
-  }
+        xn[tt] = (q + 1 < q_hi && 16 * (q + 1) + tt < n_tokens) ? __ldg(x + (size_t)(16 * (q + 1) + tt) * g.d)
+                                                                 : 0.f;
 #pragma unroll
-  for (int tt = 0; tt < 16; ++tt) {
-    const int t = 16 * q + tt;
-    const float rv = ok ? xv[tt] - s[tt] : 0.f;
-    if (ok && t < n_tokens) g.rb[(size_t)t * g.d + row] = bf16_bits(rv);
-    const float a = warp_sum(rv * rv), b = warp_sum(xv[tt] * xv[tt]);
-    if (lane == 0) {
-      s_norm[warp][tt][0] = a;
-      s_norm[warp][tt][1] = b;
+      for (int tt = 0; tt < 16; ++tt) {
+        const int t = 16 * q + tt;
+        const float rv = xv[tt] - s[tt];
+        if (t < n_tokens) g.rb[(size_t)t * g.d + row] = bf16_bits(rv);
+        const float a = warp_sum(rv * rv), b = warp_sum(xv[tt] * xv[tt]);
+        if (lane == 0 && t < n_tokens) {
+          s_norm[warp][t][0] = a;
+          s_norm[warp][t][1] = b;
+        }
+        xv[tt] = xn[tt];
+      }
     }
+    tile_release<kTmemCols3>(tmem);
   }
+  if (image) return;
   __syncthreads();
-  if (threadIdx.x < 32) {
-    const int tt = threadIdx.x >> 1, w = threadIdx.x & 1, t = 16 * q + tt;
+  for (int i = threadIdx.x; i < 32 * (q_hi - q_lo); i += kThreads) {
+    const int t = 16 * q_lo + (i >> 1), w = i & 1;
     if (t < n_tokens) {
       float sum = 0.f;
 #pragma unroll
-      for (int wp = 0; wp < kThreads / 32; ++wp) sum += s_norm[wp][tt][w];
+      for (int wp = 0; wp < kThreads / 32; ++wp) sum += ok ? s_norm[wp][t][w] : 0.f;
       g.normpart3[((size_t)tile * g.B + t) * 2 + w] = sum;
     }
   }
@@ -263,19 +276,21 @@ cudaError_t launch_front_tc(const GroupParams& g, const TmaMaps& tm, const IoRef
                             cudaStream_t st, int* n_launches) {
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(k_proj_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem3)) != cudaSuccess ||
-      (e = cudaFuncSetAttribute(k_resid_image_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemResid)) !=
+      (e = cudaFuncSetAttribute(k_resid_image_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem3)) !=
           cudaSuccess)
     return e;
   const int slots = (front_rows(n_tokens) + 2) / 3;   // token slots covering every operand row
-  const int nq = (n_tokens + 15) / 16;
+  const int nq = (n_tokens + 15) / 16, tiles = g.d / kTM;
+  int rs = tiles <= 37 ? 4 : tiles <= 74 ? 2 : 1;   // token ranges per residual tile
+  if (rs > nq) rs = nq;
   k_split3_x<<<dim3((g.d / 8 + 255) / 256, slots), 256, 0, st>>>(g, io, n_tokens);
   // the x the residual blocks read before their wait is an input of the call, complete before
   // k_split3_x was launched
   if ((e = launch_pdl(k_proj_tc, dim3((g.k / kTM) * g.proj_splits), dim3(kThreads), kSmem3, st, g, tm,
                       n_tokens)) != cudaSuccess ||
       (e = launch_pdl(k_reduce_split3_c, dim3(slots), dim3(256), 0, st, g, n_tokens)) != cudaSuccess ||
-      (e = launch_pdl(k_resid_image_tc, dim3((g.d / kTM + g.O / kTM) * nq), dim3(kThreads), kSmemResid, st,
-                      g, tm, io, n_tokens)) != cudaSuccess)
+      (e = launch_pdl(k_resid_image_tc, dim3((g.d / kTM) * rs + g.O / kTM), dim3(kThreads), kSmem3, st, g,
+                      tm, io, n_tokens, rs)) != cudaSuccess)
     return e;
   if (n_launches) *n_launches += 4;
   return cudaGetLastError();
