@@ -25,6 +25,8 @@ constexpr int kMaxN3 = 192;          // 3 terms x 64 tokens
 constexpr int kTmemCols3 = 256;      // power of two >= kMaxN3
 using Cfg3 = Cfg<kStages3, kMaxN3>;
 constexpr int kSmem3 = Cfg3::kSmem;  // 4 x (16 + 24) KB + slack
+constexpr int kStagesRI = 2;         // residual / image: K = k is short; two blocks per SM instead
+constexpr int kSmemRI = Cfg<kStagesRI, kMaxN3>::kSmem;
 
 __device__ __forceinline__ uint16_t bf16_bits(float v) {
   const __nv_bfloat16 h = __float2bfloat16_rn(v);
@@ -166,7 +168,7 @@ __global__ void __launch_bounds__(256) k_reduce_split3_c(GroupParams g, int n_to
 //                         r = x - P c -> bf16 rows of rb, the partial norms of the tile,
 //                         and in the block that finishes last the gate
 //   blocks [n_resid, ..)  tile of W_P, all tokens: y = W_P c
-__global__ void __launch_bounds__(kThreads, 1)
+__global__ void __launch_bounds__(kThreads, 2)
 k_resid_image_tc(GroupParams g, const __grid_constant__ TmaMaps tm, IoRef io, int n_tokens, int rs) {
   extern __shared__ unsigned char smem_raw[];
   __shared__ float s_norm[kThreads / 32][GSI_MAX_TOKENS][2];
@@ -194,7 +196,7 @@ k_resid_image_tc(GroupParams g, const __grid_constant__ TmaMaps tm, IoRef io, in
   bool ok = true;
   if (q_lo < q_hi) {   // block-uniform
     const int n_rows = min(48 * (q_hi - q_lo), rows3(n_tokens) - 48 * q_lo);
-    ok = tile_mma<kStages3, kMaxN3, kTmemCols3>(smem_raw, image ? &tm.wp : &tm.p, tile * kTM, &tm.cb,
+    ok = tile_mma<kStagesRI, kMaxN3, kTmemCols3>(smem_raw, image ? &tm.wp : &tm.p, tile * kTM, &tm.cb,
                                                 48 * q_lo, n_rows, 0, g.k / kTK, &tmem);
     if (!ok && threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
     const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);
@@ -276,7 +278,7 @@ cudaError_t launch_front_tc(const GroupParams& g, const TmaMaps& tm, const IoRef
                             cudaStream_t st, int* n_launches) {
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(k_proj_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem3)) != cudaSuccess ||
-      (e = cudaFuncSetAttribute(k_resid_image_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem3)) !=
+      (e = cudaFuncSetAttribute(k_resid_image_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemRI)) !=
           cudaSuccess)
     return e;
   const int slots = (front_rows(n_tokens) + 2) / 3;   // token slots covering every operand row
@@ -289,7 +291,7 @@ cudaError_t launch_front_tc(const GroupParams& g, const TmaMaps& tm, const IoRef
   if ((e = launch_pdl(k_proj_tc, dim3((g.k / kTM) * g.proj_splits), dim3(kThreads), kSmem3, st, g, tm,
                       n_tokens)) != cudaSuccess ||
       (e = launch_pdl(k_reduce_split3_c, dim3(slots), dim3(256), 0, st, g, n_tokens)) != cudaSuccess ||
-      (e = launch_pdl(k_resid_image_tc, dim3((g.d / kTM) * rs + g.O / kTM), dim3(kThreads), kSmem3, st, g,
+      (e = launch_pdl(k_resid_image_tc, dim3((g.d / kTM) * rs + g.O / kTM), dim3(kThreads), kSmemRI, st, g,
                       tm, io, n_tokens, rs)) != cudaSuccess)
     return e;
   if (n_launches) *n_launches += 4;

@@ -24,7 +24,7 @@ namespace {
 
 using namespace umma;
 
-constexpr int kStages = 4;   // 4 x 24 KB: two blocks per SM
+constexpr int kStages = 4;   // 4 x 24 KB, two blocks per SM (8 stages x 1 block and 3 x 3 measured slower)
 constexpr int kMaxN = 64;
 constexpr int kTmemCols = 64;
 using TcCfg = Cfg<kStages, kMaxN>;
