@@ -42,6 +42,7 @@ constexpr unsigned kSpinLimit = 1u << 22;
 constexpr int kCountShift = 54;
 
 // shared memory map (bytes)
+constexpr int kXBatch = 4;           // float4 loads of x in flight per thread
 constexpr int kOffBar = 0;          // full[kSlots], empty[kSlots]
 constexpr int kOffMisc = 256;       // abort flag, scalars
 constexpr int kOffX = 512;          // x of this CTA's basis rows      (kPersistMaxPRows floats)
@@ -481,15 +482,15 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
     float amax = 0.f, sum2 = 0.f;
     const int d4 = g.d >> 2;
 #pragma unroll 1
-    for (int i0 = tid; i0 < d4; i0 += 4 * kNC) {
-      float4 v[4];
+    for (int i0 = tid; i0 < d4; i0 += kXBatch * kNC) {   
+      float4 v[kXBatch];
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < kXBatch; ++u) {
         const int i4 = i0 + u * kNC;
         v[u] = i4 < d4 ? __ldcg(reinterpret_cast<const float4*>(x) + i4) : make_float4(0, 0, 0, 0);
       }
 #pragma unroll
-      for (int u = 0; u < 4; ++u) {
+      for (int u = 0; u < kXBatch; ++u) {
         amax = fmaxf(fmaxf(amax, fmaxf(fabsf(v[u].x), fabsf(v[u].y))),
                      fmaxf(fabsf(v[u].z), fabsf(v[u].w)));
         sum2 = fmaf(v[u].x, v[u].x, sum2);
@@ -509,9 +510,9 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
       amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
       sum2 += __shfl_xor_sync(0xffffffffu, sum2, o);
     }
-    if (lane == 0) {
-      s_red[warp * 2 + 0] = amax;
-      s_red[warp * 2 + 1] = sum2;
+    if (lane == 0) {   // s_vals is idle until this group's exchange 2
+      s_vals[warp * 2 + 0] = amax;
+      s_vals[warp * 2 + 1] = sum2;
     }
     if (zeroer) {  // clear what the NEXT launch will accumulate into
 #pragma unroll 1
@@ -525,8 +526,8 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
       float a = 0.f, t = 0.f;
 #pragma unroll
       for (int w = 0; w < kNW; ++w) {
-        a = fmaxf(a, s_red[w * 2]);
-        t += s_red[w * 2 + 1];
+        a = fmaxf(a, s_vals[w * 2]);
+        t += s_vals[w * 2 + 1];
       }
       amax = a;
       sum2 = t;
@@ -543,7 +544,6 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
         inv_scale = pow2d(e - 43);
       }
     }
-    csync();  // s_red is reused by pass 1
 
     // ---- B. pass 1: partial c over this CTA's basis rows
     const unsigned n_p0 = n;
@@ -877,12 +877,14 @@ cudaError_t launch_abs_max_bf16(const void* p, size_t n, float* out, cudaStream_
 }
 
 cudaError_t launch_decode_step(const PersistParams& p, int grid, cudaStream_t st) {
-  static bool configured = false;
-  if (!configured) {
+  static bool configured[64] = {};   // per device: the attribute belongs to the device's function
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
+  if (dev < 0 || dev >= 64 || !configured[dev]) {
     cudaError_t e = cudaFuncSetAttribute(k_decode_step, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                          kSmemBytes);
     if (e != cudaSuccess) return e;
-    configured = true;
+    if (dev >= 0 && dev < 64) configured[dev] = true;
   }
   PersistParams pp = p;
   void* args[] = {&pp};
