@@ -318,6 +318,7 @@ def main():
     ap.add_argument("--eps", type=float, default=0.05)
     ap.add_argument("--sigma-scale", type=float, default=1.0)
     ap.add_argument("--outlier", type=float, default=0.10)
+    ap.add_argument("--batch", type=int, default=64, help="tokens per step of the gptj_b64 workload")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -341,7 +342,7 @@ def main():
     elif args.workload == "opt":
         spec = S.config4(args.k, args.eps, args.sigma_scale)
     else:
-        spec = S.config5(args.outlier)
+        spec = S.config5(args.outlier, batch=args.batch)
     if args.layers:
         spec = replace(spec, n_layers=args.layers, name=f"{spec.name}_L{args.layers}")
 

@@ -107,7 +107,7 @@ gsi_status_t gsi_build_image(const void* W, const void* P, int o, int d, int k,
 
 /* Bytes of device workspace a handle for `desc` needs (0 if desc is invalid).
  * The workspace holds the images of all maps and the per-call scratch (c, r,
- * partial sums, fired-token list, status word; for max_tokens >= 8 also a
+ * partial sums, fired-token list, status word; for max_tokens >= 2 also a
  * transposed copy of the basis and the bf16 operands of the batched kernels). */
 size_t gsi_workspace_bytes(const gsi_desc_t* desc);
 
@@ -128,11 +128,11 @@ gsi_status_t gsi_create(const gsi_desc_t* desc, const void* const* W_host_array,
  * max_tokens tokens (gsi_forward_n).  x [n][d] fp32; y [n][sum d_out] fp32;
  * gate_mask_out [n] bytes (1 = slow path, W r added); rho_out [n] fp32 or NULL.
  * Each token is processed independently of the others in the call (Algorithm 1
- * is per token); its rounding can depend on the size of the call: calls of 8 or
- * more tokens (bf16 basis; k, d and sum d_out multiples of 128) run the
+ * is per token); its rounding can depend on the size of the call: calls of 2 or
+ * more tokens (bf16 basis; k, d and every d_out multiples of 128) run the
  * contractions on the tensor cores with exactly split operands and another
- * summation order, and calls with 5 or more gated tokens (any gated token in
- * calls of 8 or more) add W r from r rounded to bf16 (|dy| <= 3e-3 max|y|).
+ * summation order and add W r from r rounded to bf16 (|dy| <= 3e-3 max|y|);
+ * with other shapes that rounding applies from 5 gated tokens per call on.
  * Results of a given call are reproducible bit for bit.
  * Enqueues on `stream` and returns; n_tokens = 0 is a no-op.
  */

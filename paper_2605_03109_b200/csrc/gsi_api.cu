@@ -26,7 +26,7 @@ struct Layout {
 };
 
 constexpr int kTcMinFired = 5;  // fewer fired tokens: one pass of the CUDA-core GEMV
-constexpr int kFrontMinTokens = 8;  // fewer tokens in a call: the CUDA-core front end
+constexpr int kFrontMinTokens = 2;  // single-token calls: the CUDA-core front end
 
 bool tc_shapes_ok(const gsi_desc_t* d) {
   for (int j = 0; j < d->n_maps; ++j)
@@ -79,8 +79,8 @@ Layout make_layout_ws(const gsi_desc_t* d) {
   L.rho_stage = take(B * 4);
   L.pk_acc = take(2 * k * 8 * kAccStride);          // persistent kernel: c accumulators
   L.pk_slot = take((size_t)kPersistMaxGrid * 8);    // persistent kernel: ||r||^2 words
-  // tensor-core gated residual: only for batches that can fire at least kTcMinFired tokens
-  const bool tc = !dense && d->max_tokens >= kTcMinFired && d->d % 64 == 0 && tc_shapes_ok(d);
+  // tensor-core kernels: batched handles only
+  const bool tc = !dense && d->max_tokens >= kFrontMinTokens && d->d % 64 == 0 && tc_shapes_ok(d);
   L.tc_rb = take(tc ? (size_t)65 * d->d * 2 : 0);   // row 64 stays zero
   L.tc_ypart = take(tc ? (size_t)tc_splits(O, d->d) * 64 * O * 4 : 0);
   L.tc = tc;

@@ -95,18 +95,13 @@ def test_batches_and_batch_invariance(batch):
     compare_group(x, P, Ws, 0.05, y, gate, rho)
     _, y1, gate1, rho1 = run_layer(x, P, Ws, 0.05, 1)
     assert np.array_equal(gate, gate1)
-    if batch < 8:
-        # CUDA-core kernels, fixed-order fp32 reductions: a token's projection, residual
-        # and gate do not depend on its batch
-        assert np.array_equal(rho, rho1)
+    if batch == 1:
+        assert np.array_equal(rho, rho1) and np.array_equal(y, y1)
     else:
-        # calls of 8 or more tokens run those contractions on the tensor cores (exact
-        # three-term bf16 operands, fp32 sums in another order)
+        # calls of 2 or more tokens run the contractions on the tensor cores: exact
+        # three-term bf16 operands for x and c (fp32 sums in another order), r rounded to
+        # bf16 for the gated correction
         assert np.allclose(rho, rho1, rtol=2e-5, atol=0)
-    if batch < 5:
-        assert np.array_equal(y, y1)
-    else:
-        # >= 5 gated tokens per call go through the bf16 tensor-core contraction
         scale = np.max(np.abs(y1), axis=1, keepdims=True)
         assert np.all(np.abs(y - y1) <= 3e-3 * scale)
 
@@ -440,7 +435,7 @@ def test_persistent_falls_back_when_a_group_does_not_qualify():
 
 @pytest.mark.parametrize("n_out", [0, 4, 5, 16, 17, 33, 64])
 def test_tensor_core_residual_gemm_many_gated_tokens(n_out):
-    """Batch of 64 with n_out full-rank outliers: from 5 gated tokens on, the gated
+    """Batch of 64 with n_out full-rank outliers: the gated
     residual runs as the tcgen05 contraction (bf16 operands, fp32 accumulation in
     tensor memory, split-K partials added in a fixed order)."""
     d, k, d_out, B = 1024, 128, (1024, 256), 64
@@ -460,17 +455,40 @@ def test_tensor_core_residual_gemm_many_gated_tokens(n_out):
     _, y2, gate2, _ = run_layer(x, P, Ws, 0.05, B)
     assert np.array_equal(y, y2) and np.array_equal(gate, gate2)
     if n_out >= 5:
-        # the CUDA-core path (batches of 4) agrees within the bf16 rounding of r, not bitwise
-        _, y4, gate4, _ = run_layer(x, P, Ws, 0.05, 4)
+        # the CUDA-core path (single-token calls) agrees within the bf16 rounding of r, not bitwise
+        _, y4, gate4, _ = run_layer(x, P, Ws, 0.05, 1)
         assert np.array_equal(gate, gate4)
         scale = np.max(np.abs(y4), axis=1, keepdims=True)
         assert np.all(np.abs(y - y4) <= 3e-3 * scale)
         assert not np.array_equal(y[gate.astype(bool)], y4[gate.astype(bool)])
 
 
-@pytest.mark.parametrize("k,n_tokens", [(128, 8), (128, 21), (256, 22), (256, 37), (512, 64), (384, 11)])
+@pytest.mark.parametrize("n_out", [3, 7, 40])
+def test_tensor_core_residual_gemm_packed_rows_when_the_front_end_does_not_apply(n_out):
+    """k = 64 keeps the projection on CUDA cores (the tensor-core front end wants k % 128 == 0);
+    from 5 gated tokens on their residuals are compacted to bf16 rows and contracted on tcgen05."""
+    d, k, d_out, B = 1024, 64, (512, 256), 48
+    q = S.gen_basis(d, k, 930)
+    P = S.store_basis(q)
+    Ws = [S.gen_weight(o, d, 931 + j) for j, o in enumerate(d_out)]
+    pt = S.gen_true_basis(q, 32, 32, 933)
+    x, _ = S.gen_activations(pt, B, 0.004, 0.0, dict(z=934, noise=935, outlier_mask=0, outlier_values=0))
+    gen = torch.Generator().manual_seed(936 + n_out)
+    where = torch.randperm(B, generator=gen)[:n_out]
+    x[where] = torch.randn((n_out, d), generator=gen) * 0.25
+    x = x.contiguous()
+    lay, y, gate, rho = run_layer(x, P, Ws, 0.05, B)
+    assert int(gate.sum()) == n_out
+    compare_group(x, P, Ws, 0.05, y, gate, rho)
+    _, y1, gate1, rho1 = run_layer(x, P, Ws, 0.05, 1)
+    assert np.array_equal(gate, gate1) and np.array_equal(rho, rho1)   # same CUDA-core front end
+    if n_out < 5:
+        assert np.array_equal(y, y1)
+
+
+@pytest.mark.parametrize("k,n_tokens", [(128, 2), (128, 5), (128, 21), (256, 22), (256, 37), (512, 64), (384, 11)])
 def test_tensor_core_front_end_batched_projection_residual_image(k, n_tokens):
-    """Calls of 8 or more tokens run c = P^T x, r = x - P c and y = W_P c on the tensor
+    """Calls of 2 or more tokens run c = P^T x, r = x - P c and y = W_P c on the tensor
     cores with fp32 operands split into three bf16 terms: same gates, rho and y as the
     oracle, and rho as close to the oracle as the CUDA-core kernels get."""
     d, d_out, B = 1024, (768, 256, 128), 64
@@ -492,8 +510,8 @@ def test_tensor_core_front_end_batched_projection_residual_image(k, n_tokens):
     y, gate, rho = y.cpu().numpy(), gate.cpu().numpy(), rho.cpu().numpy()
     assert 0 < int(gate.sum()) < n_tokens
     compare_group(x, P, Ws, 0.05, y, gate, rho)
-    # the CUDA-core front end (a handle for batches of 4) agrees closely, not bitwise
-    _, y4, gate4, rho4 = run_layer(x, P, Ws, 0.05, 4)
+    # the CUDA-core front end (single-token calls) agrees closely, not bitwise
+    _, y4, gate4, rho4 = run_layer(x, P, Ws, 0.05, 1)
     assert np.array_equal(gate, gate4)
     assert np.allclose(rho, rho4, rtol=2e-5, atol=0)
     scale = np.max(np.abs(y4), axis=1, keepdims=True)
