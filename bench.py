@@ -150,7 +150,7 @@ def time_graph(graph, stack, stream, steps, warmup, barrier=None):
     return e0.elapsed_time(e1) / steps  # ms per step
 
 
-def time_host_steps(layers, xs, steps, warmup, stream):
+def time_host_steps(layers, xs, steps, warmup, stream, concurrent=()):
     """End-to-end: host buffers in, host buffers out, copies inside the timed region.
     The device and pinned host buffers of all groups are carved out of one arena each,
     so a step is one H2D copy, one launch, two D2H copies (y and the gate bytes)."""
@@ -176,7 +176,7 @@ def time_host_steps(layers, xs, steps, warmup, stream):
     xs_host, ys_host = carve(x_host, dx), carve(y_host, dy)
     for xh, x in zip(xs_host, xs):
         xh.copy_(x[:B].reshape(-1).cpu())
-    stack = G.Stack(layers)
+    stack = G.Stack(layers, concurrent=concurrent)
     stack.bind(xs_dev, ys=[y.view(B, -1) for y in ys_dev], n_steps=1)
     gate_host = torch.empty((n, B), dtype=torch.uint8).pin_memory()
     h2d = x_host.numel() * 4
@@ -320,6 +320,9 @@ def main():
     ap.add_argument("--outlier", type=float, default=0.10)
     ap.add_argument("--batch", type=int, default=64, help="tokens per step of the gptj_b64 workload")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
+    ap.add_argument("--no-concurrent", action="store_true",
+                    help="run the groups of a block strictly one after the other even where the "
+                         "workload marks two of them as parallel branches")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--profile", action="store_true",
@@ -368,7 +371,8 @@ def main():
 
     n_steps = min(spec.steps, max(args.steps, 1))
     layers, dense_layers, xs, keep = build_workload(spec, device, n_steps)
-    stack = G.Stack(layers)
+    concurrent = [] if args.no_concurrent else spec.concurrent_groups()
+    stack = G.Stack(layers, concurrent=concurrent)
     stack.bind(xs, n_steps=n_steps)
     if args.profile:
         for _ in range(args.warmup + args.steps):
@@ -405,7 +409,7 @@ def main():
 
     e2e = None
     if not args.no_e2e:
-        ms_e2e, h2d, d2h = time_host_steps(layers, xs, max(8, args.steps // 8), 3, stream)
+        ms_e2e, h2d, d2h = time_host_steps(layers, xs, max(8, args.steps // 8), 3, stream, concurrent)
         e2e = {"value": world * spec.batch * 1e3 / ms_e2e, "unit": "tokens/s",
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
@@ -431,6 +435,8 @@ def main():
                 "groups_per_layer": [f"{g.name}:{g.d}->{'+'.join(map(str, g.d_out))}" for g in spec.groups],
                 "k": spec.groups[0].k, "eps": spec.eps, "batch": spec.batch,
                 "persistent_launch": bool(stack.is_persistent()),
+                "parallel_branches": ("attn_out|proj of each block share a phase" if concurrent
+                                      else "none declared"),
                 "weights": "bf16", "basis": spec.groups[0].p_dtype, "activations": "f32",
                 "distinct_input_steps": n_steps,
                 "l2": "inputs_larger_than_l2 (0.88 GB of basis+image per step, distinct per layer)",

@@ -234,6 +234,18 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io_host_array,
                             gsi_stream_t stream);
 
 /*
+ * Declares that groups first_group and first_group + 1 do not read each other's
+ * outputs (two branches of one block: in GPT-J the attention output projection
+ * and the MLP down projection), so the persistent kernel may run their
+ * projections, gates and images at the same time on two parts of the grid
+ * (Algorithm 1 itself is unchanged; a gated residual still streams W with the
+ * whole grid).  Off by default; a group belongs to at most one pair; ignored
+ * outside persistent mode and when the rows of either group do not fit its
+ * share of the grid.  Takes effect at the next gsi_stack_bind.
+ */
+gsi_status_t gsi_stack_set_concurrent(gsi_stack_t s, int first_group, int enable);
+
+/*
  * Execution mode, taken at the next gsi_stack_bind:
  *   0 (default)  one persistent launch per step when every group qualifies
  *                (batch 1, bf16 basis with k in {64,128,256,512}, d a

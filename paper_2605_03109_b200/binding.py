@@ -21,7 +21,7 @@ EXPORTED = [
     "gsi_status_string", "gsi_build_image", "gsi_workspace_bytes", "gsi_create",
     "gsi_forward", "gsi_forward_n", "gsi_forward_host", "gsi_forward_static", "gsi_get_image", "gsi_get_status",
     "gsi_destroy", "gsi_stack_workspace_bytes", "gsi_stack_create", "gsi_stack_bind",
-    "gsi_stack_set_mode", "gsi_stack_is_persistent", "gsi_stack_set_trace", "gsi_stack_seek", "gsi_stack_step", "gsi_stack_launches_per_step",
+    "gsi_stack_set_mode", "gsi_stack_set_concurrent", "gsi_stack_is_persistent", "gsi_stack_set_trace", "gsi_stack_seek", "gsi_stack_step", "gsi_stack_launches_per_step",
     "gsi_stack_step_host", "gsi_stack_get_status", "gsi_stack_destroy",
 ]
 
@@ -69,6 +69,7 @@ def _load():
     l.gsi_stack_create.argtypes = [i, C.POINTER(vp), vp, sz, vp, C.POINTER(vp)]
     l.gsi_stack_bind.argtypes = [vp, C.POINTER(GsiStackIo), i, vp, vp, vp]
     l.gsi_stack_set_mode.argtypes = [vp, i]
+    l.gsi_stack_set_concurrent.argtypes = [vp, i, i]
     l.gsi_stack_is_persistent.argtypes = [vp, C.POINTER(i)]
     l.gsi_stack_set_trace.argtypes = [vp, vp]
     l.gsi_stack_seek.argtypes = [vp, i, vp]
@@ -248,7 +249,9 @@ class Layer:
 class Stack:
     """An ordered chain of groups stepped as one decode step."""
 
-    def __init__(self, layers, stream=None, mode: int = 0):
+    def __init__(self, layers, stream=None, mode: int = 0, concurrent=()):
+        """concurrent: indices i such that groups i and i+1 do not read each other's outputs
+        and may share a phase of the persistent kernel (gsi_stack_set_concurrent)."""
         self.layers = list(layers)
         self._mode = int(mode)
         n = len(self.layers)
@@ -264,6 +267,8 @@ class Stack:
         self.device = dev
         if self._mode:
             _check(lib.gsi_stack_set_mode(self.handle, self._mode), "gsi_stack_set_mode")
+        for first in concurrent:
+            _check(lib.gsi_stack_set_concurrent(self.handle, int(first), 1), "gsi_stack_set_concurrent")
 
     def is_persistent(self) -> bool:
         v = C.c_int()

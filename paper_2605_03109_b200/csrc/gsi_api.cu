@@ -1,5 +1,6 @@
 // C ABI of the gated subspace layer: argument checking, workspace layout,
 // handle and stack bookkeeping, kernel sequencing.  No arithmetic lives here.
+#include <algorithm>
 #include <new>
 #include <vector>
 #include <cstring>
@@ -124,6 +125,7 @@ struct gsi_stack {
   int* status;              // device
   unsigned long long* trace; // device, optional
   std::vector<gsi_layer*> groups;
+  std::vector<char> pair_first;   // group i and i+1 declared independent of each other
   std::vector<gsi_stack_io_t> io;
   int B;
   int n_steps;
@@ -371,6 +373,7 @@ gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* wo
   gsi_stack* s = new (std::nothrow) gsi_stack();
   if (!s) return GSI_ERR_ALLOC;
   s->groups.assign(groups, groups + n_groups);
+  s->pair_first.assign(n_groups, 0);
   s->io.resize(n_groups);
   s->B = groups[0]->desc.max_tokens;
   s->n_steps = 0;
@@ -398,14 +401,18 @@ gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* wo
 // Can this stack run as one persistent launch?  (batch 1, bf16 basis with a
 // power-of-two rank up to 512, rows that fit the per-CTA buffers, 32-byte
 // aligned weight rows for the 256-bit loads.)
+static bool rows_fit(const gsi_layer* h, int ctas) {
+  return ctas > 0 && (h->desc.d + ctas - 1) / ctas <= kPersistMaxPRows &&
+         (h->lay.O + ctas - 1) / ctas <= kPersistMaxORows;
+}
+
 static bool persistent_eligible(const gsi_stack* s, int grid) {
   if (s->B != 1 || grid <= 0 || grid > kPersistMaxGrid) return false;
   for (const gsi_layer* h : s->groups) {
     const gsi_desc_t& d = h->desc;
     const bool dense = d.flags & GSI_FLAG_DENSE;
     if (d.d % 16) return false;
-    if ((d.d + grid - 1) / grid > kPersistMaxPRows) return false;
-    if ((h->lay.O + grid - 1) / grid > kPersistMaxORows) return false;
+    if (!rows_fit(h, grid)) return false;
     for (int j = 0; j < d.n_maps; ++j)
       if (reinterpret_cast<uintptr_t>(h->gp.W[j]) & 31u) return false;
     if (!dense) {
@@ -414,6 +421,36 @@ static bool persistent_eligible(const gsi_stack* s, int grid) {
     }
   }
   return true;
+}
+
+// CTAs given to the first group of a pair: in proportion to the bytes its fast path
+// streams, between a quarter and three quarters of the grid; 0 if the rows of either
+// group do not fit its share (the pair then runs one group after the other).
+static int pair_split(const gsi_layer* a, const gsi_layer* b, int grid) {
+  if ((a->desc.flags | b->desc.flags) & GSI_FLAG_DENSE) return 0;
+  if (grid >= kPairSumSlot) return 0;
+  const double wa = (double)(a->desc.d + a->lay.O) * a->desc.k;
+  const double wb = (double)(b->desc.d + b->lay.O) * b->desc.k;
+  int na = (int)(grid * wa / (wa + wb) + 0.5);
+  na = std::max(grid / 4, std::min(grid - grid / 4, na));
+  // ring: all chunks of a group are resident at once
+  auto chunks = [](const gsi_layer* h, int ctas) {
+    const int rc = 16384 / (h->desc.k * 2);
+    return ((h->desc.d + ctas - 1) / ctas + rc - 1) / rc + ((h->lay.O + ctas - 1) / ctas + rc - 1) / rc;
+  };
+  if (!rows_fit(a, na) || !rows_fit(b, grid - na)) return 0;
+  if (chunks(a, na) > 10 || chunks(b, grid - na) > 10) return 0;
+  return na;
+}
+
+gsi_status_t gsi_stack_set_concurrent(gsi_stack_t s, int first_group, int enable) {
+  if (!s || first_group < 0 || first_group + 1 >= (int)s->groups.size()) return GSI_ERR_INVALID_ARG;
+  // a group belongs to at most one pair
+  if (enable && ((first_group > 0 && s->pair_first[first_group - 1]) || s->pair_first[first_group + 1]))
+    return GSI_ERR_INVALID_ARG;
+  s->pair_first[first_group] = enable ? 1 : 0;
+  s->bound = false;  // applied at bind time
+  return GSI_OK;
 }
 
 gsi_status_t gsi_stack_set_mode(gsi_stack_t s, int mode) {
@@ -484,9 +521,34 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
       pg.acc_c = reinterpret_cast<unsigned long long*>(h->ws + h->lay.pk_acc);
       pg.slot_r = reinterpret_cast<unsigned long long*>(h->ws + h->lay.pk_slot);
       pg.bar = h->bar;
-      pg.p_rows = (gp.d + s->grid - 1) / s->grid;
-      pg.o_rows = (gp.O + s->grid - 1) / s->grid;
+      pg.cta0 = 0;
+      pg.ncta = s->grid;
+      pg.phase_len = 1;
+      pg.o_rows_w = (gp.O + s->grid - 1) / s->grid;
       pg.x_step_stride = gp.d;
+    }
+    // pairs of independent groups split the grid
+    for (int i = 0; i + 1 < G; ++i) {
+      if (!s->pair_first[i]) continue;
+      const int na = pair_split(s->groups[i], s->groups[i + 1], s->grid);
+      if (na == 0) continue;
+      PersistGroup &a = s->host_groups[i], &b = s->host_groups[i + 1];
+      a.ncta = na;
+      b.cta0 = na;
+      b.ncta = s->grid - na;
+      a.phase_len = b.phase_len = 2;
+      b.slot_r = a.slot_r;   // one joint exchange
+    }
+    for (int i = 0; i < G; ++i) {
+      PersistGroup& pg = s->host_groups[i];
+      pg.p_rows = (pg.d + pg.ncta - 1) / pg.ncta;
+      pg.o_rows = (pg.O + pg.ncta - 1) / pg.ncta;
+    }
+    for (int i = 0; i < G;) {   // length of the phase after each group's
+      const int len = s->host_groups[i].phase_len;
+      const int nxt = i + len < G ? s->host_groups[i + len].phase_len : 0;
+      for (int j = 0; j < len; ++j) s->host_groups[i + j].next_len = nxt;
+      i += len;
     }
     const float** dev_ptrs = reinterpret_cast<const float**>(
         reinterpret_cast<char*>(s->dev_groups) + (size_t)G * 512);

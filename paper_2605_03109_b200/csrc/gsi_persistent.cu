@@ -46,16 +46,18 @@ constexpr int kXBatch = 4;           // float4 loads of x in flight per thread
 constexpr int kOffBar = 0;          // full[kSlots], empty[kSlots]
 constexpr int kOffMisc = 256;       // abort flag, scalars
 constexpr int kOffX = 512;          // x of this CTA's basis rows      (kPersistMaxPRows floats)
-constexpr int kOffC = 1024;         // c                                (512 floats)
-constexpr int kOffVals = 3072;      // exchange-2 values                (256 floats)
-constexpr int kOffDesc = 4096;      // 3 group descriptors, 512 B each (current, next, previous)
-constexpr int kOffRed = kOffDesc + 3 * 512;       // cross-warp scratch (kNW*512 floats)
+constexpr int kOffC = 1536;         // c                                (512 floats)
+constexpr int kOffVals = 3584;      // exchange-2 values                (256 floats)
+constexpr int kOffDesc = 4608;      // 4 group descriptors, 512 B each (this phase's and the next's)
+constexpr int kDescSlots = 4;
+constexpr int kOffRed = kOffDesc + kDescSlots * 512;   // cross-warp scratch (kNW*512 floats)
 constexpr int kOffRq = kOffRed + kNW * 512 * 4;   // staged r, 4 interleaved quarters (16 KB)
 constexpr int kOffYacc = kOffRq + 16384;          // per-row accumulators (kPersistMaxORows floats)
 constexpr int kOffRing = ((kOffYacc + kPersistMaxORows * 4 + 1023) / 1024) * 1024;
 constexpr int kSmemBytes = kOffRing + kSlots * kChunk;
 static_assert(kSmemBytes <= 232448, "shared memory budget of one sm_100 CTA");
 static_assert(sizeof(PersistGroup) <= 512 && sizeof(PersistGroup) % 4 == 0, "descriptor slot");
+static_assert(kOffC - kOffX >= kPersistMaxPRows * 4, "x slab");
 constexpr int kDescWords = (int)(sizeof(PersistGroup) / 4);
 
 struct Misc {
@@ -186,7 +188,9 @@ __device__ void producer(const PersistParams& p, unsigned char* smem, Misc* misc
   for (int gi = 0; gi < p.n_groups && !*abort; ++gi) {
     const PersistGroup& g = p.groups[gi];
     if (g.flags & GSI_FLAG_DENSE) continue;
-    const Slab s = slab_of(g, blockIdx.x);
+    const int lc = (int)blockIdx.x - g.cta0;
+    if (lc < 0 || lc >= g.ncta) continue;   // its partner's share of the grid
+    const Slab s = slab_of(g, lc);
     const int rc = kChunk / (g.k * 2);
     for (int part = 0; part < 2; ++part) {
       const int a = part ? s.o0 : s.p0, b = part ? s.o1 : s.p1;
@@ -223,6 +227,7 @@ drain:
 // per row, RPP = 32/LPR rows per warp pass, VPL = KV/LPR vectors per lane.
 struct Ctx {
   int step, slot_io;
+  int len;     // groups in the phase just run (1, or 2 for a pair)
   unsigned parity, tag;
   unsigned n;  // ring sequence number, advances exactly as in producer()
   Trace tr;
@@ -416,8 +421,8 @@ __device__ __noinline__ void gated_pass(const PersistGroup& g, const Slab& s, co
 
 // Make the next group's activations L2-resident while this group runs (a real
 // pipeline would find them there, written by the preceding operator).
-__device__ __forceinline__ void prefetch_next_x(const PersistGroup& gn, int slot_io) {
-  if (blockIdx.x == 0) {
+__device__ __forceinline__ void prefetch_next_x(const PersistGroup& gn, int slot_io, int who = 0) {
+  if ((int)blockIdx.x == who) {
     const char* xn = reinterpret_cast<const char*>(gn.x + (long long)slot_io * gn.x_step_stride);
     const int lines = (gn.d * 4 + 127) >> 7;
     for (int l = threadIdx.x; l < lines; l += kNC) prefetch_l2(xn + (size_t)l * 128);
@@ -443,21 +448,35 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
   unsigned& n = ctx.n;
   Trace& tr = ctx.tr;
 
-  // The descriptor of this group was staged in shared memory one group ago;
-  // stage the next one now (three slots: current, next, previous).
-  const PersistGroup& g = *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + (gi % 3) * 512);
-  const PersistGroup& g_next =
-      *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + ((gi + 1) % 3) * 512);
-  const bool has_next = gi + 1 < p.n_groups;
-  uint32_t desc_word = 0;  // one word of the next descriptor, in flight during section A
-  if (has_next && tid < kDescWords)
-    desc_word = __ldg(reinterpret_cast<const uint32_t*>(p.groups + gi + 1) + tid);
+  // The descriptors of this phase (one group, or a pair of independent groups that split
+  // the grid) were staged in shared memory one phase ago, descriptor i in slot i % 4;
+  // stage the next phase's now.
+  auto desc = [&](int i) -> const PersistGroup& {
+    return *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + (i & (kDescSlots - 1)) * 512);
+  };
+  const PersistGroup& gA = desc(gi);
+  const int len = gA.phase_len, next_len = gA.next_len;
+  const PersistGroup& gB = desc(gi + len - 1);   // gA itself when the group is alone
+  const bool second = len == 2 && cta >= gB.cta0;
+  const PersistGroup& g = second ? gB : gA;      // the group whose fast path this CTA runs
+  const int gi_mine = gi + (second ? 1 : 0);
+  const int lc = cta - g.cta0;                   // index within the group's share of the grid
+  const PersistGroup& g_next = desc(gi + len);
+  const bool has_next = next_len > 0;
+  ctx.len = len;
+  uint32_t desc_word = 0;  // one word of the next descriptors, in flight during section A
+  if (tid < next_len * kDescWords)
+    desc_word = __ldg(reinterpret_cast<const uint32_t*>(p.groups + gi + len) + tid);
+  uint32_t* const desc_dst =
+      reinterpret_cast<uint32_t*>(smem + kOffDesc +
+                                  ((gi + len + (tid >= kDescWords ? 1 : 0)) & (kDescSlots - 1)) * 512) +
+      (tid >= kDescWords ? tid - kDescWords : tid);
 
-  const Slab s = slab_of(g, cta);
+  const Slab s = slab_of(g, lc);
   const float* x = g.x + (long long)slot_io * g.x_step_stride;
   const bool dense = g.flags & GSI_FLAG_DENSE;
-  const bool zeroer = cta == gi % G;  // this CTA clears the group's counters for the next launch
-  int gate = 1;
+  const bool zeroer = lc == gi_mine % g.ncta;  // this CTA clears the group's counters for the next launch
+  int gate = 1, gate_other = 0;
   const float* rsrc = x;
 
   if (!dense) {
@@ -500,8 +519,7 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
       }
     }
     if (tid < prow) s_x[tid] = __ldcg(x + s.p0 + tid);
-    if (has_next && tid < kDescWords)
-      reinterpret_cast<uint32_t*>(smem + kOffDesc + ((gi + 1) % 3) * 512)[tid] = desc_word;
+    if (tid < next_len * kDescWords) *desc_dst = desc_word;
     tr.mark(0);
     // fmaxf drops NaN, the sum keeps it (and overflows to inf for huge inputs):
     // sum2 - sum2 is non-zero exactly when some x_i is NaN or inf (or x^2 overflowed)
@@ -522,6 +540,7 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
     }
     csync();
     if (has_next) prefetch_next_x(g_next, slot_io);
+    if (next_len == 2) prefetch_next_x(desc(gi + len + 1), slot_io, 1);
     {  // every thread folds the warp partials in the same order
       float a = 0.f, t = 0.f;
 #pragma unroll
@@ -704,12 +723,17 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
 
     // ---- E. exchange 2: publish, collect, decide.  The word carries its own
     //      launch tag, so no fence is needed for the gate decision itself.
+    // A pair shares the first group's slot array: word cta is this CTA's partial of its own
+    // group, words kPairSumSlot + u carry ||x||^2 of group u for the other half of the grid.
     if (tid == 0) {
       float t = 0.f;
 #pragma unroll
       for (int w = 0; w < kNW; ++w) t += s_red[w];
-      st_relaxed_u64(g.slot_r + cta,
+      st_relaxed_u64(gA.slot_r + cta,
                      ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(t));
+      if (len == 2 && lc == 0)
+        st_relaxed_u64(gA.slot_r + kPairSumSlot + (second ? 1 : 0),
+                       ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(sum2));
     }
     tr.mark(9);
     if (warp == 0) {
@@ -724,8 +748,8 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
         for (int i = 0; i < 8; ++i) {
           const int t = lane + 32 * i;
           vals[i] = 0.f;
-          if (t < G) {
-            const unsigned long long w = ld_relaxed_u64(g.slot_r + t);
+          if (t < G || (len == 2 && t >= kPairSumSlot)) {
+            const unsigned long long w = ld_relaxed_u64(gA.slot_r + t);
             all = all && ((unsigned)(w >> 32) == tag);
             vals[i] = __uint_as_float((unsigned)w);
           }
@@ -742,51 +766,76 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
     csync();
     tr.mark(10);
     if (*abort) return false;
-    {  // every warp folds the 256 slots in the same fixed order
-      float t = 0.f;
+    {  // every warp folds the slots of each group in the same fixed order
+      const int split = len == 2 ? gB.cta0 : G;
+      float tA = 0.f, tB = 0.f;
 #pragma unroll
-      for (int i = 0; i < 8; ++i) t += s_vals[lane + 32 * i];
-      t = warp_sum(t);
+      for (int i = 0; i < 8; ++i) {
+        const int t = lane + 32 * i;
+        const float v = s_vals[t];
+        if (t < split) tA += v;
+        else if (t < G) tB += v;
+      }
+      tA = warp_sum(tA);
+      tB = warp_sum(tB);
       // ||r|| < eps ||x||  <=>  ||r||^2 < eps^2 ||x||^2  (both sides >= 0); NaN compares false
+      const float t = second ? tB : tA;
       const double e2 = (double)g.eps * (double)g.eps;
       const bool fast = !nonfinite && ((double)t < e2 * (double)sum2);
       gate = fast ? 0 : 1;
-      if (cta == 0 && tid == 0) {
-        const size_t at = (size_t)slot_io * p.log_step_stride + gi;
+      if (lc == 0 && tid == 0) {
+        const size_t at = (size_t)slot_io * p.log_step_stride + gi_mine;
         p.gate_log[at] = (unsigned char)gate;
         if (p.rho_log)
           p.rho_log[at] = nonfinite ? __int_as_float(0x7fc00000) : sqrtf(__fdividef(t, sum2));
       }
+      if (len == 2) {  // the partner's decision, from its partial sums and its ||x||^2
+        const PersistGroup& go = second ? gA : gB;
+        const float to = second ? tA : tB, s2o = s_vals[kPairSumSlot + (second ? 0 : 1)];
+        const double e2o = (double)go.eps * (double)go.eps;
+        const bool finite_o = s2o - s2o == 0.f;
+        const bool fast_o = finite_o && ((double)to < e2o * (double)s2o);
+        gate_other = (!fast_o && finite_o && !(go.flags & GSI_FLAG_STATIC_PROJECTION)) ? 1 : 0;
+      }
     }
     gate = gate && !(g.flags & GSI_FLAG_STATIC_PROJECTION) && !nonfinite;
-    rsrc = g.r;
     tr.mark(11);
   } else {
     if (zeroer && tid < 3) g.bar[2 * tid + (parity ^ 1u)] = 0u;
     if (cta == 0 && tid == 0) p.gate_log[(size_t)slot_io * p.log_step_stride + gi] = 1;
-    if (has_next && tid < kDescWords)
-      reinterpret_cast<uint32_t*>(smem + kOffDesc + ((gi + 1) % 3) * 512)[tid] = desc_word;
+    if (tid < next_len * kDescWords) *desc_dst = desc_word;
     csync();
     if (has_next) prefetch_next_x(g_next, slot_io);
+    if (next_len == 2) prefetch_next_x(desc(gi + len + 1), slot_io, 1);
   }
 
-  if (gate) {
+  // ---- F. gated residual of every gated group of the phase, each with the whole grid
+#pragma unroll 1
+  for (int u = 0; u < len; ++u) {
+    const PersistGroup& gg = u ? gB : gA;
+    const int fire = ((u == 1) == second) ? gate : gate_other;
+    if (!fire) continue;
     if (!dense) {
-      // r was written by every CTA: make it visible grid-wide before anyone reads it
-      // (release fence, arrival count, acquire fence).  Only gated groups pay for this.
+      // r (and the image rows of y) were written by other CTAs: make them visible grid-wide
+      // before anyone reads them (release fence, arrival count, acquire fence).  Only gated
+      // groups pay for this.
       if (tid == 0) {
         __threadfence();
-        grid_arrive_wait(g.bar + 2 + parity, (unsigned)G, p, misc);
+        grid_arrive_wait(gg.bar + 2 + parity, (unsigned)G, p, misc);
         __threadfence();
       }
       csync();
       if (*abort) return false;
     }
-    gated_pass(g, s, rsrc, dense, smem);
+    Slab sw;
+    sw.p0 = sw.p1 = 0;
+    sw.o0 = min(gg.O, cta * gg.o_rows_w);
+    sw.o1 = min(gg.O, sw.o0 + gg.o_rows_w);
+    gated_pass(gg, sw, dense ? rsrc : gg.r, dense, smem);
     // no CTA starts the next group before all have finished this one
     csync();
     tr.mark(12);
-    if (tid == 0) grid_arrive_wait(g.bar + parity, (unsigned)G, p, misc);
+    if (tid == 0) grid_arrive_wait(gg.bar + parity, (unsigned)G, p, misc);
     csync();
     tr.mark(13);
     if (*abort) return false;
@@ -803,13 +852,17 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
   ctx.tag = (unsigned)epoch + 1u;
   ctx.n = 0;
   ctx.tr.start(p);
-  if (p.n_groups > 0 && threadIdx.x < kDescWords)
-    reinterpret_cast<uint32_t*>(smem + kOffDesc)[threadIdx.x] =
+  // the first phase's descriptors (the second slot is used only if the phase is a pair)
+  if ((int)threadIdx.x < min(p.n_groups, 2) * kDescWords) {
+    const int j = threadIdx.x >= kDescWords ? 1 : 0;
+    reinterpret_cast<uint32_t*>(smem + kOffDesc + j * 512)[threadIdx.x - j * kDescWords] =
         __ldg(reinterpret_cast<const uint32_t*>(p.groups) + threadIdx.x);
+  }
   csync();
   bool ok = true;
+  ctx.len = 1;
 #pragma unroll 1
-  for (int gi = 0; gi < p.n_groups && ok; ++gi) ok = group_phase(p, smem, misc, ctx, gi);
+  for (int gi = 0; gi < p.n_groups && ok; gi += ctx.len) ok = group_phase(p, smem, misc, ctx, gi);
   // Every CTA read the counters at its start and has since taken part in the
   // last group's exchange, so they may advance now.
   if (blockIdx.x == 0 && threadIdx.x == 0 && ok) {

@@ -6,7 +6,7 @@
 namespace gsi {
 
 constexpr int kPersistConsumerWarps = 15;  // + 1 producer warp = 16 warps: registers are allotted per 4 warps
-constexpr int kPersistMaxPRows = 128;   // basis rows one CTA may own
+constexpr int kPersistMaxPRows = 256;   // basis rows one CTA may own
 constexpr int kPersistMaxORows = 512;   // output rows one CTA may own
 constexpr int kPersistMaxGrid = 256;    // CTAs (exchange-2 slots per group)
 constexpr int kAccStride = 16;          // 64-bit words between c accumulators: one per 128-byte line
@@ -27,9 +27,19 @@ struct PersistGroup {
   unsigned long long* acc_c;         // [2][k][kAccStride] fixed-point accumulators, one set per launch parity
   unsigned long long* slot_r;        // [kPersistMaxGrid] (launch tag | partial ||r||^2)
   unsigned* bar;                     // [6] arrival counters by launch parity: [0..1] after, [2..3] before the gated residual, [4..5] exchange 2
-  int p_rows, o_rows;                // rows per CTA of P and of the outputs (ceil(rows / CTAs))
+  int p_rows, o_rows;                // rows per CTA of P and of the images (ceil(rows / ncta))
   long long x_step_stride;
+  // Two consecutive groups whose inputs do not depend on each other's outputs may form one
+  // phase: CTAs [cta0, cta0 + ncta) run this group's projection, gate and image while the
+  // rest of the grid runs its partner's; both gates come out of one joint exchange, and a
+  // gated residual always streams W with the whole grid.
+  int cta0, ncta;                    // this group's share of the grid (0, grid when alone)
+  int phase_len;                     // groups in this group's phase: 1, or 2 for both of a pair
+  int next_len;                      // groups in the phase after this group's (0 at the end)
+  int o_rows_w;                      // W rows per CTA of the gated residual: ceil(O / grid)
 };
+
+constexpr int kPairSumSlot = 254;    // slot_r[254 + u]: ||x||^2 of group u of a pair (slots < grid hold ||r||^2 partials)
 
 struct PersistParams {
   const PersistGroup* groups;  // device

@@ -38,6 +38,15 @@ class StackSpec:
     steps: int
     batch: int = 1
     note: str = ""
+    # indices i (within a layer) of groups whose successor i+1 sits on a parallel branch of the
+    # block: neither reads the other's output (GPT-J: attention output projection | MLP down
+    # projection; GPT-2 and OPT blocks are sequential, so none)
+    concurrent: tuple = ()
+
+    def concurrent_groups(self):
+        """Stack-wide indices of the first group of every independent pair."""
+        n = len(self.groups)
+        return [layer * n + i for layer in range(self.n_layers) for i in self.concurrent]
 
     @property
     def n_groups(self) -> int:
@@ -118,7 +127,7 @@ def config3(gate: str = "10") -> StackSpec:
     scale = {"10": 1.0, "0": 0.25, "23": 1.0303, "100": 4.0}[gate]
     s4, s16 = SIGMA_GPTJ_10[4096] * scale, SIGMA_GPTJ_10[16384] * scale
     return StackSpec(f"cfg3_gptj_gate{gate}", 3, 28, gptj_groups(256, 200, 200, s4, s16),
-                     0.05, 256, 1)
+                     0.05, 256, 1, concurrent=(1,))
 
 
 def config4(k: int, eps: float, sigma_scale: float, steps: int = 64) -> StackSpec:
@@ -138,7 +147,8 @@ def config5(p_outlier: float, batch: int = 64, steps: int = 128) -> StackSpec:
     the gate rate is forced by the outlier fraction."""
     s4, s16 = SIGMA_GPTJ_10[4096] * 0.2, SIGMA_GPTJ_10[16384] * 0.2
     return StackSpec(f"cfg5_gptj_b{batch}_p{p_outlier}", 5, 28,
-                     gptj_groups(256, 200, 200, s4, s16, p_outlier), 0.05, steps, batch)
+                     gptj_groups(256, 200, 200, s4, s16, p_outlier), 0.05, steps, batch,
+                     concurrent=(1,))
 
 
 def materialize_group(stack: StackSpec, layer: int, gi: int, n_tokens: int, device="cpu",

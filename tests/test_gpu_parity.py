@@ -303,7 +303,7 @@ def test_gptj_layer_full_size_sampled_rows():
         assert res["gate_rate"] < 0.6
 
 
-def _stack_against_oracle(st, n_layers, n_steps, mode, sample_rows=0, device="cuda"):
+def _stack_against_oracle(st, n_layers, n_steps, mode, sample_rows=0, device="cuda", concurrent=()):
     """Run n_steps decode steps and compare every group with the oracle (on a
     sample of output rows when the maps are large)."""
     g = G()
@@ -315,7 +315,7 @@ def _stack_against_oracle(st, n_layers, n_steps, mode, sample_rows=0, device="cu
             layers.append(g.Layer(m["W"], m["P"], st.eps, max_tokens=1))
             xs.append(m["x"].contiguous())
             mats.append(m)
-    stack = g.Stack(layers, mode=mode)
+    stack = g.Stack(layers, mode=mode, concurrent=concurrent)
     stack.bind(xs, n_steps=n_steps)
     ys = [[] for _ in mats]
     for s in range(n_steps):
@@ -353,6 +353,33 @@ def test_persistent_gptj_two_layers_full_size_sampled_rows():
     assert stack.is_persistent()
     rates = [s["gate_rate"] for s in stats]
     assert 0.0 < np.mean(rates) < 0.5   # both paths occur
+
+
+def test_persistent_gptj_parallel_branches_share_a_phase():
+    """attn_out and proj of a GPT-J block read outputs of the first group only: declared
+    concurrent, they run on two parts of the grid with one joint gate exchange.  Same
+    gates as the sequential schedule, every group within tolerance of the oracle, and a
+    gated residual of either (or both) still correct; bit-reproducible."""
+    st = S.config3("23")
+    n_layers, n_steps = 2, 16
+    pairs = [layer * 3 + 1 for layer in range(n_layers)]
+    a, stats, ys_a, gate_a = _stack_against_oracle(st, n_layers, n_steps, mode=2, sample_rows=40,
+                                                   concurrent=pairs)
+    assert a.is_persistent()
+    b, _, ys_b, gate_b = _stack_against_oracle(st, n_layers, n_steps, mode=2, sample_rows=40)
+    assert np.array_equal(gate_a, gate_b)
+    # both members of a pair gated in the same step, and only one of them, both occur
+    pair_gates = gate_a[:, [1, 2, 4, 5], 0].reshape(n_steps, 2, 2)
+    assert (pair_gates.sum(axis=2) == 2).any() and (pair_gates.sum(axis=2) == 1).any()
+    cat = lambda ts: torch.cat(ts).numpy()
+    for ya, yb in zip(ys_a, ys_b):
+        ya, yb = cat(ya), cat(yb)
+        assert np.max(np.abs(ya - yb)) <= 1e-4 * np.max(np.abs(yb))
+    c, _, ys_c, gate_c = _stack_against_oracle(st, n_layers, n_steps, mode=2, sample_rows=40,
+                                               concurrent=pairs)
+    assert np.array_equal(gate_a, gate_c)
+    for ya, yc in zip(ys_a, ys_c):
+        assert np.array_equal(cat(ya), cat(yc))
 
 
 def test_persistent_matches_generic_kernels_and_is_reproducible():
