@@ -567,6 +567,15 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
     // ---- B. pass 1: partial c over this CTA's basis rows
     const unsigned n_p0 = n;
     bool ok = true;
+    {  // the basis chunks of this group: one per lane, all waits in flight together
+      bool mine_ok = true;
+      if (lane < pchunks) {
+        const unsigned seq = n_p0 + lane;
+        mine_ok = mbar_wait(&full[seq % kSlots], (seq / kSlots) & 1u, abort);
+      }
+      ok = __all_sync(0xffffffffu, mine_ok);
+    }
+    tr.mark(2);
 #pragma unroll 1
     for (int u = 0; u < q.vpl; ++u) {
       const int cv = q.cl + u * LPR;
@@ -575,10 +584,8 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
       for (int e = 0; e < 8; ++e) a8[e] = 0.f;
 #pragma unroll 1
       for (int ci = 0; ci < pchunks; ++ci) {
-        const unsigned sl = (n_p0 + ci) % kSlots, ph = ((n_p0 + ci) / kSlots) & 1u;
-        ok = ok && mbar_wait(&full[sl], ph, abort);
         if (!ok) break;
-        tr.mark(2);
+        const unsigned sl = (n_p0 + ci) % kSlots;
         const uint4* tile = reinterpret_cast<const uint4*>(ring + (size_t)sl * kChunk);
         const int r_lo = ci << q.rc_log2, rows = min(rc, prow - r_lo);
 #pragma unroll 1
@@ -664,10 +671,14 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
     //      the image rows: the same eight-rows-per-lane-group loop over both
     const int hold_log2 = q.lpr_log2 - 3;  // lanes per held row after reduce8
     // all image chunks of this group must have landed (they were prefetched)
-#pragma unroll 1
-    for (int ci = 0; ci < ochunks; ++ci) {
-      const unsigned seq = n_p0 + pchunks + ci;
-      ok = ok && mbar_wait(&full[seq % kSlots], (seq / kSlots) & 1u, abort);
+    // (one chunk per lane, all waits in flight together; the warp then agrees)
+    {
+      bool mine_ok = true;
+      if (lane < ochunks) {
+        const unsigned seq = n_p0 + pchunks + lane;
+        mine_ok = mbar_wait(&full[seq % kSlots], (seq / kSlots) & 1u, abort);
+      }
+      ok = __all_sync(0xffffffffu, ok && mine_ok);
     }
     tr.mark(7);
     float sr = 0.f;
