@@ -683,26 +683,29 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
     tr.mark(7);
     float sr = 0.f;
     if (ok) {
-      // work items: lane groups take eight rows at a time; item -> (chunk, rows)
-      const int ipc_log2 = q.rc_log2 - 3;              // items per chunk
-      const int n_items = (pchunks + ochunks) << ipc_log2;
+      // work items: lane groups take eight rows at a time, first of the basis slab, then of
+      // the image slab (rows per chunk are a multiple of 8, so an item stays inside a chunk);
+      // only items with rows are enumerated, rounded up to a whole warp of lane groups
+      const int itemsP = (prow + 7) >> 3, n_live = itemsP + ((orow + 7) >> 3);
+      const int n_items = ((n_live + (1 << rpp_log2) - 1) >> rpp_log2) << rpp_log2;
       const int lanegroups = kNW << rpp_log2;          // lane groups in the CTA
       int released = 0;  // chunks this warp has already given back to the producer
 #pragma unroll 1
       for (int item = (warp << rpp_log2) + q.sub; item < n_items; item += lanegroups) {
-        const int ci = item >> ipc_log2;
+        const bool image = item >= itemsP;
+        const int row0g = (image ? item - itemsP : item) << 3;   // first row, within the slab
+        const int cj = row0g >> q.rc_log2;
+        const int ci = min((image ? pchunks : 0) + cj, pchunks + ochunks - 1);
         // items come in chunk order: every chunk before this warp's current one is done
         // (n_items is a multiple of the lane groups per warp, so the warp stays converged)
         const int ci_warp = __shfl_sync(0xffffffffu, ci, 0);
         if (lane == 0)
           for (; released < ci_warp; ++released) mbar_arrive(&empty[(n_p0 + released) % kSlots]);
         released = ci_warp;
-        const bool image = ci >= pchunks;
-        const int cj = image ? ci - pchunks : ci;
         const unsigned sl = (n_p0 + ci) % kSlots;
         const uint4* tile = reinterpret_cast<const uint4*>(ring + (size_t)sl * kChunk);
         const int r_lo = cj << q.rc_log2, rows = min(rc, (image ? orow : prow) - r_lo);
-        const int row0 = (item & ((1 << ipc_log2) - 1)) << 3;
+        const int row0 = row0g & (rc - 1);
         float v[8];
         dot8(tile, s_c, q, row0, rows, v);
         const float dot = reduce8(v, q.cl, LPR);
