@@ -401,9 +401,15 @@ gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* wo
 // Can this stack run as one persistent launch?  (batch 1, bf16 basis with a
 // power-of-two rank up to 512, rows that fit the per-CTA buffers, 32-byte
 // aligned weight rows for the 256-bit loads.)
+// Rows of one CTA fit its buffers, and all 16 KB chunks of the group fit the ring of ten
+// slots together (the row pass runs with every chunk of the group resident).
 static bool rows_fit(const gsi_layer* h, int ctas) {
-  return ctas > 0 && (h->desc.d + ctas - 1) / ctas <= kPersistMaxPRows &&
-         (h->lay.O + ctas - 1) / ctas <= kPersistMaxORows;
+  if (ctas <= 0) return false;
+  const int pr = (h->desc.d + ctas - 1) / ctas, orw = (h->lay.O + ctas - 1) / ctas;
+  if (pr > kPersistMaxPRows || orw > kPersistMaxORows) return false;
+  if ((h->desc.flags & GSI_FLAG_DENSE) || h->desc.k <= 0) return true;
+  const int rc = std::max(1, 16384 / (h->desc.k * 2));
+  return (pr + rc - 1) / rc + (orw + rc - 1) / rc <= 10;
 }
 
 static bool persistent_eligible(const gsi_stack* s, int grid) {
@@ -433,13 +439,7 @@ static int pair_split(const gsi_layer* a, const gsi_layer* b, int grid) {
   const double wb = (double)(b->desc.d + b->lay.O) * b->desc.k;
   int na = (int)(grid * wa / (wa + wb) + 0.5);
   na = std::max(grid / 4, std::min(grid - grid / 4, na));
-  // ring: all chunks of a group are resident at once
-  auto chunks = [](const gsi_layer* h, int ctas) {
-    const int rc = 16384 / (h->desc.k * 2);
-    return ((h->desc.d + ctas - 1) / ctas + rc - 1) / rc + ((h->lay.O + ctas - 1) / ctas + rc - 1) / rc;
-  };
   if (!rows_fit(a, na) || !rows_fit(b, grid - na)) return 0;
-  if (chunks(a, na) > 10 || chunks(b, grid - na) > 10) return 0;
   return na;
 }
 
