@@ -457,7 +457,7 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
   const PersistGroup& gA = desc(gi);
   const int len = gA.phase_len, next_len = gA.next_len;
   const PersistGroup& gB = desc(gi + len - 1);   // gA itself when the group is alone
-  const bool second = len == 2 && cta >= gB.cta0;
+  const bool second = cta >= gA.cta0 + gA.ncta;  // never when alone: its share is the whole grid
   const PersistGroup& g = second ? gB : gA;      // the group whose fast path this CTA runs
   const int gi_mine = gi + (second ? 1 : 0);
   const int lc = cta - g.cta0;                   // index within the group's share of the grid
@@ -781,17 +781,17 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
     tr.mark(10);
     if (*abort) return false;
     {  // every warp folds the slots of each group in the same fixed order
-      const int split = len == 2 ? gB.cta0 : G;
+      const int split = gA.ncta;   // the whole grid when the group is alone
       float tA = 0.f, tB = 0.f;
 #pragma unroll
       for (int i = 0; i < 8; ++i) {
         const int t = lane + 32 * i;
         const float v = s_vals[t];
-        if (t < split) tA += v;
-        else if (t < G) tB += v;
+        tA += t < split ? v : 0.f;
+        tB += (t >= split && t < G) ? v : 0.f;
       }
       tA = warp_sum(tA);
-      tB = warp_sum(tB);
+      if (len == 2) tB = warp_sum(tB);
       // ||r|| < eps ||x||  <=>  ||r||^2 < eps^2 ||x||^2  (both sides >= 0); NaN compares false
       const float t = second ? tB : tA;
       const double e2 = (double)g.eps * (double)g.eps;
