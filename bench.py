@@ -97,7 +97,7 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------
-def build_workload(spec, device, n_steps):
+def build_workload(spec, device, n_steps, static_projection=False):
     """Draw the whole stack on the device.  Returns (gsi layers, dense layers,
     x tensors per group, host-side copies needed later)."""
     import torch
@@ -107,7 +107,8 @@ def build_workload(spec, device, n_steps):
     for layer in range(spec.n_layers):
         for gi, g in enumerate(spec.groups):
             m = S.materialize_group(spec, layer, gi, n_steps * spec.batch, device=device)
-            lay = G.Layer(m["W"], m["P"], spec.eps, max_tokens=spec.batch)
+            lay = G.Layer(m["W"], m["P"], spec.eps, max_tokens=spec.batch,
+                          flags=G.GSI_FLAG_STATIC_PROJECTION if static_projection else 0)
             den = G.Layer(m["W"], None, 0.0, max_tokens=spec.batch, flags=G.GSI_FLAG_DENSE)
             layers.append(lay)
             dense.append(den)
@@ -320,6 +321,9 @@ def main():
     ap.add_argument("--outlier", type=float, default=0.10)
     ap.add_argument("--batch", type=int, default=64, help="tokens per step of the gptj_b64 workload")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
+    ap.add_argument("--static-projection", action="store_true",
+                    help="negative control (Section 4.1, static projection): the gate is computed and "
+                         "logged but W r is never added, so the step costs the fast path only")
     ap.add_argument("--no-concurrent", action="store_true",
                     help="run the groups of a block strictly one after the other even where the "
                          "workload marks two of them as parallel branches")
@@ -370,7 +374,7 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     n_steps = min(spec.steps, max(args.steps, 1))
-    layers, dense_layers, xs, keep = build_workload(spec, device, n_steps)
+    layers, dense_layers, xs, keep = build_workload(spec, device, n_steps, args.static_projection)
     concurrent = [] if args.no_concurrent else spec.concurrent_groups()
     stack = G.Stack(layers, concurrent=concurrent)
     stack.bind(xs, n_steps=n_steps)
@@ -403,6 +407,8 @@ def main():
     gate_log = stack.gate_log.cpu().numpy()          # [n_steps][groups][B]
     used_steps = min(args.steps, n_steps)
     fired = gate_log[:used_steps].any(axis=2)        # [steps][groups]
+    if args.static_projection:                       # the gate is logged but W is never read
+        fired = fired & False
     status = stack.status()
     if status != 0:
         raise SystemExit(f"device status word {status}: {G.gsi_status_string(status)}")
@@ -437,6 +443,7 @@ def main():
                 "persistent_launch": bool(stack.is_persistent()),
                 "parallel_branches": ("attn_out|proj of each block share a phase" if concurrent
                                       else "none declared"),
+                "static_projection": bool(args.static_projection),
                 "weights": "bf16", "basis": spec.groups[0].p_dtype, "activations": "f32",
                 "distinct_input_steps": n_steps,
                 "l2": "inputs_larger_than_l2 (0.88 GB of basis+image per step, distinct per layer)",
