@@ -21,7 +21,9 @@
  * Pinning: see tests/test_oracle_pins.py.  Every function below is pinned by
  * special cases that reduce to a library mat-vec, by the exact identity of
  * Eq. (3.2), by the bound of Theorem 3.1, by the monotonicity of
- * Proposition 2.3 and by brute force in rational arithmetic on tiny shapes.
+ * Proposition 2.3 and by brute force in rational arithmetic on tiny shapes;
+ * the online basis extension by a library QR, by the orthogonality its second
+ * pass restores, and by its special cases (empty, full, in-span).
  * What the paper measures on real model activations (gate rates, perplexity;
  * Tables 4-9) has no counterpart here: parity unpinned for those, they are out
  * of scope.
@@ -238,4 +240,68 @@ int gsi_oracle_map(const double* M, const uint16_t* W, const double* g,
     }
   }
   return 0;
+}
+
+/*
+ * Online extension of the basis by one vector (the paper's "time-dimension
+ * tracking" of Section 5.3 and "online basis adaptation" of Section 7.3):
+ * a token x is tested against the current basis, and if
+ *     rho = ||x - V V^T x|| / ||x||
+ * exceeds the threshold tau the basis is extended by one orthonormal vector.
+ * The vector is the residual orthogonalised against V TWICE and normalised
+ * (classical Gram-Schmidt with one re-orthogonalisation, the "DGKS" update):
+ *     r1 = x  - V (V^T x),   r2 = r1 - V (V^T r1),   v = r2 / ||r2||.
+ * The paper gives no further detail; readings taken here: the test uses the
+ * first-pass residual (the formula the paper prints, the same rho the layer's
+ * gate uses); nothing is appended when the basis is full or r2 vanishes.
+ *
+ * P: [d][k_cap] stored basis of which columns [0, k_act) are in use.
+ * x: [d] double.  Outputs: *rho_out; v_out [d] (unit vector, unrounded; written
+ * only when the function returns 1).  Returns 1 = extended, 0 = not, -1 = bad
+ * arguments.
+ */
+int gsi_oracle_extend(const void* P, int p_dtype, int d, int k_cap, int k_act,
+                      const double* x, double tau, double* rho_out, double* v_out) {
+  if (!P || !x || !rho_out || !v_out || d <= 0 || k_cap <= 0 || k_act < 0 || k_act > k_cap)
+    return -1;
+  double* r = (double*)malloc((size_t)d * sizeof(double));
+  double* g = (double*)malloc((size_t)(k_act > 0 ? k_act : 1) * sizeof(double));
+  if (!r || !g) {
+    free(r);
+    free(g);
+    return -1;
+  }
+  double sx = 0.0;
+  for (int i = 0; i < d; ++i) {
+    r[i] = x[i];
+    sx += x[i] * x[i];
+  }
+  double rho = 0.0;
+  for (int pass = 0; pass < 2; ++pass) {
+    for (int j = 0; j < k_act; ++j) {
+      double s = 0.0;
+      for (int i = 0; i < d; ++i) s += basis_at(P, p_dtype, (size_t)i * k_cap + j) * r[i];
+      g[j] = s;
+    }
+    double sr = 0.0;
+    for (int i = 0; i < d; ++i) {
+      double pg = 0.0;
+      for (int j = 0; j < k_act; ++j) pg += basis_at(P, p_dtype, (size_t)i * k_cap + j) * g[j];
+      r[i] -= pg;
+      sr += r[i] * r[i];
+    }
+    if (pass == 0) rho = sqrt(sr) / sqrt(sx);
+  }
+  *rho_out = rho;
+  double s2 = 0.0;
+  for (int i = 0; i < d; ++i) s2 += r[i] * r[i];
+  int extended = 0;
+  if (rho > tau && k_act < k_cap && s2 > 0.0) {
+    const double inv = 1.0 / sqrt(s2);
+    for (int i = 0; i < d; ++i) v_out[i] = r[i] * inv;
+    extended = 1;
+  }
+  free(r);
+  free(g);
+  return extended;
 }

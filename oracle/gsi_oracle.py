@@ -56,6 +56,8 @@ def _load():
         lib.gsi_oracle_project.restype = i
         lib.gsi_oracle_map.argtypes = [vp, vp, vp, vp, vp, vp, i, i, i, i, vp, vp]
         lib.gsi_oracle_map.restype = i
+        lib.gsi_oracle_extend.argtypes = [vp, i, i, i, i, vp, ctypes.c_double, vp, vp]
+        lib.gsi_oracle_extend.restype = i
         _lib = lib
     return _lib
 
@@ -138,6 +140,29 @@ def project(x, P, eps: float) -> dict:
     )
     if rc:
         raise RuntimeError("gsi_oracle_project failed")
+    return out
+
+
+def extend(P, k_act: int, x, tau: float) -> dict:
+    """Online basis extension by one vector (Sections 5.3 and 7.3): rho of the token
+    against columns [0, k_act) of the stored basis P [d][k_cap]; if rho > tau (and a
+    column is free) the unit vector v = twice-orthogonalised residual, in fp64.
+    ``v_bits`` is v rounded to bf16 (round to nearest even), the value a bf16 basis
+    stores in column k_act."""
+    P, pd = _basis(P)
+    d, k_cap = P.shape
+    x = _c(np.asarray(x, np.float64).reshape(-1), np.float64)
+    assert x.size == d
+    rho = ctypes.c_double()
+    v = np.zeros(d, np.float64)
+    rc = _load().gsi_oracle_extend(_ptr(P), pd, d, k_cap, int(k_act), _ptr(x), float(tau),
+                                   ctypes.byref(rho), _ptr(v))
+    if rc < 0:
+        raise RuntimeError("gsi_oracle_extend failed")
+    out = dict(rho=rho.value, extended=bool(rc))
+    if rc:
+        out["v"] = v
+        out["v_bits"] = f64_to_bf16_rne(v)
     return out
 
 

@@ -369,3 +369,88 @@ def test_P10_effective_parameters_and_storage_examples():
     assert abs(peff - 386e6) / 386e6 < 0.005
     assert abs(R.image_storage_bytes(28, 32768, 256) / 1e6 - 469) < 1
     assert abs(R.basis_storage_bytes(28, 4096, 256) / 1e6 - 59) < 0.5
+
+
+# ---- online basis extension (Sections 5.3 and 7.3) ----------------------------------
+def _partial_basis(d, k_act, k_cap, seed, dtype=np.float32):
+    rng = np.random.default_rng(seed)
+    q, _ = np.linalg.qr(rng.standard_normal((d, k_act)))
+    P = np.zeros((d, k_cap), dtype)
+    P[:, :k_act] = q.astype(dtype)
+    return P, rng
+
+
+def test_E1_extension_vector_is_the_last_column_of_a_library_qr():
+    """Appending the twice-orthogonalised residual is Gram-Schmidt on [V x]: the new vector
+    equals (up to sign) the last column of numpy's Householder QR of that matrix."""
+    d, k_act = 96, 12
+    P, rng = _partial_basis(d, k_act, 16, 41)
+    x = rng.standard_normal(d)
+    out = O.extend(P, k_act, x, 0.05)
+    assert out["extended"]
+    q, _ = np.linalg.qr(np.concatenate([P[:, :k_act].astype(np.float64), x[:, None]], axis=1))
+    last = q[:, -1]
+    assert min(np.linalg.norm(out["v"] - last), np.linalg.norm(out["v"] + last)) < 1e-6
+    assert abs(np.linalg.norm(out["v"]) - 1.0) < 1e-15
+    # rho is the first-pass residual ratio: the same number the layer's gate computes
+    pr = O.project(x.astype(np.float32)[None, :], np.ascontiguousarray(P[:, :k_act]), 0.05)
+    x32 = x.astype(np.float32).astype(np.float64)
+    out32 = O.extend(P, k_act, x32, 0.05)
+    assert abs(out32["rho"] - pr["rho"][0]) <= 1e-14 * pr["rho"][0]
+
+
+def test_E2_second_orthogonalisation_is_needed_and_enough():
+    """With a stored basis that is orthonormal only to ~1e-7 (fp32 storage) and a token that
+    is almost inside the span, one Gram-Schmidt pass leaves V^T v ~ 1e-7 / rho; the second
+    pass brings it to rounding level.  A dropped second pass fails this pin."""
+    d, k_act = 128, 24
+    P, rng = _partial_basis(d, k_act, 32, 42)
+    V = P[:, :k_act].astype(np.float64)
+    x = V @ rng.standard_normal(k_act) + 1e-3 * rng.standard_normal(d)
+    out = O.extend(P, k_act, x, 1e-6)
+    assert out["extended"] and 1e-4 < out["rho"] < 1e-2
+    assert np.abs(V.T @ out["v"]).max() < 1e-11
+    r1 = x - V @ (V.T @ x)                      # one pass only
+    one = r1 / np.linalg.norm(r1)
+    assert np.abs(V.T @ one).max() > 1e-6 * 0.1  # visibly worse: what the second pass removes
+
+
+def test_E3_special_cases():
+    d = 40
+    rng = np.random.default_rng(43)
+    x = rng.standard_normal(d)
+    # empty basis: the new vector is x / ||x||, rho = 1
+    out = O.extend(np.zeros((d, 8), np.float32), 0, x, 0.5)
+    assert out["extended"] and abs(out["rho"] - 1.0) < 1e-15
+    assert np.allclose(out["v"], x / np.linalg.norm(x), rtol=0, atol=1e-15)
+    # token inside the span: below any reasonable threshold, nothing appended
+    P, rng = _partial_basis(d, 6, 8, 44, np.float64)
+    P32 = P.astype(np.float32)
+    xin = P32[:, :6].astype(np.float64) @ rng.standard_normal(6)
+    out = O.extend(P32, 6, xin, 1e-3)
+    assert not out["extended"] and out["rho"] < 1e-6
+    # full basis: nothing appended even above the threshold
+    out = O.extend(P32[:, :6].copy(), 6, x, 0.05)
+    assert not out["extended"] and out["rho"] > 0.05
+    # threshold is strict: rho == tau does not extend
+    r = O.extend(P32, 6, x, 0.0)["rho"]
+    assert not O.extend(P32, 6, x, r)["extended"]
+    assert O.extend(P32, 6, x, np.nextafter(r, 0.0))["extended"]
+
+
+def test_E4_after_the_extension_the_token_lies_in_the_span():
+    """Storing v (here in fp32) as column k_act puts x inside the span of the stored basis:
+    its residual ratio drops from rho to storage rounding level, and the image column of the
+    extended basis is W v (Section 4.2 applied to the new column)."""
+    d, k_act, o = 80, 10, 24
+    P, rng = _partial_basis(d, k_act, 16, 45)
+    x = rng.standard_normal(d).astype(np.float32)
+    out = O.extend(P, k_act, x.astype(np.float64), 0.05)
+    assert out["extended"] and out["rho"] > 0.5
+    P2 = P.copy()
+    P2[:, k_act] = out["v"].astype(np.float32)
+    after = O.project(x[None, :], np.ascontiguousarray(P2[:, :k_act + 1]), 0.05)
+    assert after["rho"][0] < 1e-6 and after["gate"][0] == 0
+    W = O.f64_to_bf16_rne(rng.standard_normal((o, d)) * 0.1)
+    col = O.image(W, np.ascontiguousarray(P2[:, k_act:k_act + 1]))
+    assert np.allclose(col[:, 0], O.bf16_to_f64(W) @ P2[:, k_act].astype(np.float64), rtol=0, atol=1e-14)
