@@ -186,6 +186,32 @@ gsi_status_t gsi_forward_static(const void* const* W_host_array, const int* d_ou
                                 unsigned char* gate_mask_out, float* rho_out,
                                 gsi_stream_t stream);
 
+/*
+ * Online extension of the basis by one vector (the paper's "time-dimension
+ * tracking", Section 5.3, and "online basis adaptation", Section 7.3): the token
+ * x [d] (fp32, device) is tested against the basis in use; if
+ *     rho = ||x - P P^T x|| / ||x||  >  tau
+ * and a column is free, the residual orthogonalised against P twice
+ * (Gram-Schmidt with one re-orthogonalisation, "DGKS") and normalised is stored,
+ * rounded to the basis type, as column *k_active of P, and W times that stored
+ * column (Section 4.2), rounded to bf16, as column *k_active of every cached
+ * image; *k_active is then incremented.  Layout contract: columns
+ * [*k_active, k) of P are zero when the handle is created, so every forward
+ * call works on the full width k before and after.
+ *
+ * This call WRITES the caller's basis buffer P (the pointer given to
+ * gsi_create, which must therefore be writable) and the images in the
+ * workspace.  k_active: device int, in/out.  appended_out (device int, 0/1) and
+ * rho_out (device float) may be NULL.  tau >= 0.  A non-finite token never
+ * extends the basis.  Enqueues on `stream` (one pass over W when a column is
+ * appended) and returns; it must not overlap a forward call of the same handle,
+ * it overwrites the handle's per-call scratch, and a stack that has the handle
+ * bound must be bound again afterwards (it caches max|P|).  Not available for
+ * GSI_FLAG_DENSE handles.
+ */
+gsi_status_t gsi_extend_basis(gsi_handle_t h, const float* x, float tau, int* k_active,
+                              int* appended_out, float* rho_out, gsi_stream_t stream);
+
 /* Device pointer to the image of map j inside the workspace ([d_out_j][k] bf16),
  * so a caller can inspect or persist it. */
 gsi_status_t gsi_get_image(gsi_handle_t h, int map, const void** W_P_out);

@@ -19,7 +19,7 @@ GSI_MAX_MAPS, GSI_MAX_TOKENS = 8, 64
 
 EXPORTED = [
     "gsi_status_string", "gsi_build_image", "gsi_workspace_bytes", "gsi_create",
-    "gsi_forward", "gsi_forward_n", "gsi_forward_host", "gsi_forward_static", "gsi_get_image", "gsi_get_status",
+    "gsi_forward", "gsi_forward_n", "gsi_forward_host", "gsi_forward_static", "gsi_extend_basis", "gsi_get_image", "gsi_get_status",
     "gsi_destroy", "gsi_stack_workspace_bytes", "gsi_stack_create", "gsi_stack_bind",
     "gsi_stack_set_mode", "gsi_stack_set_concurrent", "gsi_stack_is_persistent", "gsi_stack_set_trace", "gsi_stack_seek", "gsi_stack_step", "gsi_stack_launches_per_step",
     "gsi_stack_step_host", "gsi_stack_get_status", "gsi_stack_destroy",
@@ -62,6 +62,7 @@ def _load():
     l.gsi_forward_static.argtypes = [C.POINTER(vp), C.POINTER(i), i, vp, i, vp, i, i, C.c_float,
                                      vp, i, vp, vp, vp, vp]
     l.gsi_get_image.argtypes = [vp, i, C.POINTER(vp)]
+    l.gsi_extend_basis.argtypes = [vp, vp, C.c_float, vp, vp, vp, vp]
     l.gsi_get_status.argtypes = [vp, C.POINTER(i)]
     l.gsi_destroy.argtypes = [vp]
     l.gsi_stack_workspace_bytes.restype = sz
@@ -219,6 +220,18 @@ class Layer:
         _check(lib.gsi_forward_host(self.handle, x.data_ptr(), n, y.data_ptr(), gate.data_ptr(),
                                     rho.data_ptr(), _stream_ptr(stream)), "gsi_forward_host")
         return y, gate, rho
+
+    def extend_basis(self, x: torch.Tensor, tau: float, k_active: torch.Tensor, stream=None):
+        """gsi_extend_basis for one token x [d]; k_active is a device int32 tensor (in/out).
+        Returns (appended, rho) as device tensors.  Writes the basis tensor given at creation."""
+        assert x.is_cuda and x.dtype == torch.float32 and x.is_contiguous() and x.numel() == self.d
+        assert k_active.is_cuda and k_active.dtype == torch.int32 and k_active.numel() == 1
+        appended = torch.zeros(1, dtype=torch.int32, device=x.device)
+        rho = torch.zeros(1, dtype=torch.float32, device=x.device)
+        _check(lib.gsi_extend_basis(self.handle, x.data_ptr(), float(tau), k_active.data_ptr(),
+                                    appended.data_ptr(), rho.data_ptr(), _stream_ptr(stream)),
+               "gsi_extend_basis")
+        return appended, rho
 
     def image(self, j: int) -> torch.Tensor:
         """Copy of the cached image of map j ([d_out_j][k] bf16)."""

@@ -331,6 +331,29 @@ gsi_status_t gsi_forward_host(gsi_handle_t h, const float* x_host, int n_tokens,
   return cudaStreamSynchronize(stream) == cudaSuccess ? GSI_OK : GSI_ERR_CUDA;
 }
 
+gsi_status_t gsi_extend_basis(gsi_handle_t h, const float* x, float tau, int* k_active,
+                              int* appended_out, float* rho_out, gsi_stream_t stream) {
+  if (!h || !x || !k_active || !aligned16(x) || !(tau >= 0.f)) return GSI_ERR_INVALID_ARG;
+  if (h->desc.flags & GSI_FLAG_DENSE) return GSI_ERR_UNSUPPORTED;
+  const Layout& L = h->lay;
+  int* ctrl = reinterpret_cast<int*>(h->ws + L.ctrl);
+  ExtendArgs a{};
+  a.x = x;
+  a.tau = tau;
+  a.k_active = k_active;
+  a.appended_out = appended_out;
+  a.rho_out = rho_out;
+  a.y_scratch = reinterpret_cast<float*>(h->ws + L.y_stage);
+  a.gate_scratch = reinterpret_cast<unsigned char*>(h->ws + L.gate_stage);
+  a.ctrl = ctrl + 24;                                       // words 24..27 of the control block
+  a.inv_norm = reinterpret_cast<float*>(ctrl + 28);         // words 28..29
+  a.x_scratch = reinterpret_cast<float*>(h->ws + L.x_stage);
+  a.pmax = h->gp.p_f32 ? nullptr : h->pmax;
+  a.PT = L.front ? const_cast<uint16_t*>(h->gp.PT) : nullptr;
+  h->last_stream = stream;
+  return launch_extend_basis(h->gp, a, stream) == cudaSuccess ? GSI_OK : GSI_ERR_CUDA;
+}
+
 gsi_status_t gsi_get_image(gsi_handle_t h, int map, const void** out) {
   if (!h || !out || map < 0 || map >= h->desc.n_maps) return GSI_ERR_INVALID_ARG;
   if (h->desc.flags & GSI_FLAG_DENSE) return GSI_ERR_UNSUPPORTED;

@@ -210,6 +210,27 @@ struct TmaMaps;   // tensor maps of the layer's matrices (null when no tensor-co
 cudaError_t launch_generic_forward(const GroupParams& g, const TmaMaps* tm, const IoRef& io,
                                    int n_tokens, cudaStream_t stream, int* n_launches);
 cudaError_t launch_advance_step(int* step, cudaStream_t stream);
+// One token on CUDA cores: c, r = x - P c into g.r (x may be g.r itself), rho into
+// g.rho_scratch[0] (or io.rho), gate byte, fired list.  No image product.
+cudaError_t launch_project_residual(const GroupParams& g, const IoRef& io, cudaStream_t stream);
+// io.y[0][:] += W g.r for the token in the fired list (nothing if the list is empty).
+cudaError_t launch_gated_gemv(const GroupParams& g, const IoRef& io, cudaStream_t stream);
+// Online basis extension by one vector (see gsi_extend_basis).
+struct ExtendArgs {
+  const float* x;        // [d] the token
+  float tau;
+  int* k_active;         // device, in/out
+  int* appended_out;     // device or null
+  float* rho_out;        // device or null
+  float* y_scratch;      // [O] device
+  unsigned char* gate_scratch;  // [1] device
+  int* ctrl;             // [4] device: appended, column, spare, spare
+  float* inv_norm;       // [2] device: 1/||r2||, rho of the token
+  float* x_scratch;      // [d] device: r1, the input of the second pass
+  float* pmax;           // [1] device: max |P| of the handle (bf16 basis) or null
+  uint16_t* PT;          // [k][d] transposed copy to keep in step, or null
+};
+cudaError_t launch_extend_basis(const GroupParams& g, const ExtendArgs& a, cudaStream_t stream);
 // mapped: rb holds every token's residual (row = token) and the fired list selects the
 // operand rows; otherwise a pack kernel first compacts the fired tokens of g.r into rb.
 cudaError_t launch_residual_gemm_tc(const GroupParams& g, const TmaMaps& tm, const IoRef& io,

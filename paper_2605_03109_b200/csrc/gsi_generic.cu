@@ -332,9 +332,10 @@ __global__ void k_advance_step(int* step) {
   if (threadIdx.x == 0 && blockIdx.x == 0) *step = *step + 1;
 }
 
+// Algorithm 1 lines 1-4 on CUDA cores: c, r, norms, gate (and, with_image, line 5).
 template <int VPL>
 cudaError_t launch_vpl(const GroupParams& g, const IoRef& io, int n_tokens, cudaStream_t st,
-                       int* n_launches) {
+                       int* n_launches, bool with_image = true) {
   const RowLayout L = make_layout(g.k);
   const size_t sm = (size_t)kWarps * TB * g.k * sizeof(float);
   cudaError_t e;
@@ -354,12 +355,26 @@ cudaError_t launch_vpl(const GroupParams& g, const IoRef& io, int n_tokens, cuda
     k_residual_gate<VPL, true><<<g.n_slabs, kThreads, 0, st>>>(g, io, n_tokens);
   else
     k_residual_gate<VPL, false><<<g.n_slabs, kThreads, 0, st>>>(g, io, n_tokens);
-  const int rows_per_pass = kWarps * L.RPP;
-  int grid = (g.O + rows_per_pass - 1) / rows_per_pass;
-  if (grid > 148 * 8) grid = 148 * 8;
-  k_image_gemv<VPL><<<grid, kThreads, 0, st>>>(g, io, n_tokens);
-  *n_launches += 4;
+  *n_launches += 3;
+  if (with_image) {
+    const int rows_per_pass = kWarps * L.RPP;
+    int grid = (g.O + rows_per_pass - 1) / rows_per_pass;
+    if (grid > 148 * 8) grid = 148 * 8;
+    k_image_gemv<VPL><<<grid, kThreads, 0, st>>>(g, io, n_tokens);
+    *n_launches += 1;
+  }
   return cudaGetLastError();
+}
+
+cudaError_t dispatch_vpl(const GroupParams& g, const IoRef& io, int n_tokens, cudaStream_t st,
+                         int* n_launches, bool with_image) {
+  switch (make_layout(g.k).VPL) {
+    case 1: return launch_vpl<1>(g, io, n_tokens, st, n_launches, with_image);
+    case 2: return launch_vpl<2>(g, io, n_tokens, st, n_launches, with_image);
+    case 3: return launch_vpl<3>(g, io, n_tokens, st, n_launches, with_image);
+    case 4: return launch_vpl<4>(g, io, n_tokens, st, n_launches, with_image);
+    default: return cudaErrorInvalidValue;
+  }
 }
 
 }  // namespace
@@ -375,19 +390,12 @@ cudaError_t launch_generic_forward(const GroupParams& g, const TmaMaps* tm, cons
     *n_launches += 1;
     return cudaGetLastError();
   }
-  const RowLayout L = make_layout(g.k);
   cudaError_t e;
   const bool front = tm && g.front_min_tokens > 0 && n_tokens >= g.front_min_tokens;
   if (front) {
     e = launch_front_tc(g, *tm, io, n_tokens, st, n_launches);
   } else {
-    switch (L.VPL) {
-      case 1: e = launch_vpl<1>(g, io, n_tokens, st, n_launches); break;
-      case 2: e = launch_vpl<2>(g, io, n_tokens, st, n_launches); break;
-      case 3: e = launch_vpl<3>(g, io, n_tokens, st, n_launches); break;
-      case 4: e = launch_vpl<4>(g, io, n_tokens, st, n_launches); break;
-      default: return cudaErrorInvalidValue;
-    }
+    e = dispatch_vpl(g, io, n_tokens, st, n_launches, true);
   }
   if (e != cudaSuccess) return e;
   if (!(g.flags & GSI_FLAG_STATIC_PROJECTION)) {
@@ -404,6 +412,18 @@ cudaError_t launch_generic_forward(const GroupParams& g, const TmaMaps* tm, cons
       }
     }
   }
+  return cudaGetLastError();
+}
+
+cudaError_t launch_project_residual(const GroupParams& g, const IoRef& io, cudaStream_t st) {
+  int n = 0;
+  return dispatch_vpl(g, io, 1, st, &n, false);
+}
+
+cudaError_t launch_gated_gemv(const GroupParams& g, const IoRef& io, cudaStream_t st) {
+  int grid = (g.O + kWarps - 1) / kWarps;
+  if (grid > 148 * 8) grid = 148 * 8;
+  k_stream_gemv<false><<<grid, kThreads, 0, st>>>(g, io, 1);
   return cudaGetLastError();
 }
 

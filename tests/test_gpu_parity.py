@@ -609,3 +609,126 @@ def test_step_on_another_stream_right_after_bind():
         assert stack.status() == 0
         compare_group(m["x"][7:8], m["P"], m["W"], st.eps, stack.ys[0].cpu().numpy(),
                       stack.gate_log[7, 0].cpu().numpy(), stack.rho_log[7, 0].cpu().numpy())
+
+
+# ---- online basis extension (Sections 5.3 and 7.3) ----------------------------------
+def _extend_case(d, k_act, k_cap, d_out, seed, p_dtype="bf16"):
+    q = S.gen_basis(d, k_act, seed)                       # fp64 orthonormal [d][k_act]
+    P = torch.zeros((d, k_cap), dtype=torch.float64)
+    P[:, :k_act] = q
+    P = S.store_basis(P, p_dtype).contiguous()            # zero columns stay zero
+    Ws = [S.gen_weight(o, d, seed + 10 + j) for j, o in enumerate(d_out)]
+    return q, P, Ws
+
+
+def _bits(t):
+    return S.bits_of(t)
+
+
+@pytest.mark.parametrize("p_dtype", ["bf16", "f32"])
+@pytest.mark.parametrize("kind", ["new_direction", "inside_span", "empty_basis", "full"])
+def test_extend_basis_single_token_matches_oracle(p_dtype, kind):
+    from oracle import gsi_oracle as O
+    d, k_cap, d_out = 1024, 128, (512, 256)
+    k_act = {"new_direction": 96, "inside_span": 96, "empty_basis": 0, "full": 128}[kind]
+    q, P, Ws = _extend_case(d, max(k_act, 1), k_cap, d_out, 700)
+    if k_act == 0:
+        P.zero_()
+    if p_dtype == "f32":
+        P = P.float()
+    gen = torch.Generator().manual_seed(701)
+    if kind == "inside_span":
+        x = (q[:, :k_act] @ torch.randn(k_act, generator=gen, dtype=torch.float64)).float()
+    else:
+        x = torch.randn(d, generator=gen)
+    tau = 0.05
+    ref = O.extend(_bits(P), k_act, x.double().numpy(), tau)
+    g = G()
+    Pd = P.cuda()
+    lay = g.Layer([W.cuda() for W in Ws], Pd, 0.05, max_tokens=4)
+    wp_before = [lay.image(j).cpu() for j in range(len(Ws))]
+    ka = torch.tensor([k_act], dtype=torch.int32, device="cuda")
+    appended, rho = lay.extend_basis(x.cuda(), tau, ka)
+    torch.cuda.synchronize()
+    assert lay.status() == 0
+    assert bool(appended.item()) == ref["extended"] == (kind in ("new_direction", "empty_basis"))
+    assert abs(rho.item() - ref["rho"]) <= 1e-4 * ref["rho"] + 1e-7
+    assert ka.item() == k_act + int(ref["extended"])
+    P_after = Pd.cpu()
+    if not ref["extended"]:
+        assert torch.equal(P_after, P)                     # nothing written
+        for j in range(len(Ws)):
+            assert torch.equal(lay.image(j).cpu(), wp_before[j])
+        return
+    # only column k_act changed; it holds v in the basis type
+    keep = [c for c in range(k_cap) if c != k_act]
+    assert torch.equal(P_after[:, keep], P[:, keep])
+    col = P_after[:, k_act].double().numpy()
+    if p_dtype == "bf16":
+        want = O.bf16_to_f64(ref["v_bits"])
+        assert np.all(np.abs(col - want) <= 2.0 ** -8 * np.abs(want) + 1e-9)   # at most one bf16 ulp
+        assert np.mean(col == want) > 0.97                                      # nearly all bit-equal
+        stored_ref = ref["v_bits"].reshape(d, 1)
+    else:
+        # fp32 sums over d terms: absolute error ~1e-7 of the largest entry
+        assert np.all(np.abs(col - ref["v"]) <= 2e-6 * np.abs(ref["v"]) + 1e-6 * np.max(np.abs(ref["v"])))
+        stored_ref = ref["v"].astype(np.float32).reshape(d, 1)
+    # image column = bf16(W v_stored) for every map, other columns untouched
+    for j, W in enumerate(Ws):
+        img = lay.image(j).cpu()
+        assert torch.equal(img[:, keep], wp_before[j][:, keep])
+        want_col = O.image(S.bits_of(W), stored_ref)[:, 0]
+        got = img[:, k_act].double().numpy()
+        assert np.all(np.abs(got - want_col) <= 2.0 ** -8 * np.abs(want_col) + 3e-3 * np.max(np.abs(want_col)))
+
+
+def test_extend_basis_sequence_then_forward_sees_the_new_columns():
+    """A stream of tokens, some in the span, some not: the GPU basis and the oracle's evolve
+    independently from the same start and stay together (same decisions, same columns to
+    bf16 rounding); afterwards the tokens that caused an extension take the fast path."""
+    from oracle import gsi_oracle as O
+    d, k_act0, k_cap, d_out = 1024, 120, 128, (512, 384)
+    q, P, Ws = _extend_case(d, k_act0, k_cap, d_out, 720)
+    gen = torch.Generator().manual_seed(721)
+    extra = torch.linalg.qr(torch.randn(d, 5, generator=gen, dtype=torch.float64))[0]
+    toks = []
+    for t in range(14):
+        base = q @ torch.randn(k_act0, generator=gen, dtype=torch.float64)
+        if t % 3 == 0:                                     # tokens 0,3,6,9,12: a direction outside
+            base = base + 6.0 * extra[:, (t // 3) % 5] * base.norm() / 10
+        toks.append(base.float())
+    x = torch.stack(toks).contiguous()
+    tau = 0.05
+    # oracle evolution
+    Pb = _bits(P).copy()
+    k_ref, decisions = k_act0, []
+    for t in range(x.shape[0]):
+        out = O.extend(Pb, k_ref, x[t].double().numpy(), tau)
+        decisions.append(out["extended"])
+        if out["extended"]:
+            Pb[:, k_ref] = out["v_bits"]
+            k_ref += 1
+    assert decisions == [t % 3 == 0 for t in range(14)]    # the five new directions, once each
+    # GPU evolution
+    g = G()
+    Pd = P.cuda()
+    lay = g.Layer([W.cuda() for W in Ws], Pd, tau, max_tokens=16)
+    ka = torch.tensor([k_act0], dtype=torch.int32, device="cuda")
+    got = []
+    for t in range(x.shape[0]):
+        appended, _ = lay.extend_basis(x[t].cuda().contiguous(), tau, ka)
+        got.append(bool(appended.item()))
+    assert got == decisions and ka.item() == k_ref == k_act0 + 5
+    Pg = O.bf16_to_f64(_bits(Pd))
+    Pr = O.bf16_to_f64(Pb)
+    assert np.max(np.abs(Pg - Pr)) <= 2.0 ** -7 * np.max(np.abs(Pr))
+    gram = Pg[:, :k_ref].T @ Pg[:, :k_ref]
+    assert np.max(np.abs(gram - np.eye(k_ref))) < 5e-3     # as orthonormal as a bf16-stored QR basis
+    # forward with the extended basis against the oracle with ITS extended basis and images
+    y, gate, rho = lay.forward(x[:14].cuda().contiguous())
+    torch.cuda.synchronize()
+    assert lay.status() == 0
+    assert gate.sum().item() == 0                          # every token is inside the span now
+    # (rho of these in-span tokens is storage rounding residue, ~1e-3, and not compared)
+    compare_group(x[:14], torch.from_numpy(Pb.view(np.int16)).view(torch.bfloat16), Ws, tau,
+                  y.cpu().numpy(), gate.cpu().numpy(), None)
