@@ -304,6 +304,52 @@ def run_reference(args, spec):
     print(json.dumps(out))
 
 
+def run_extend(args):
+    """Latency of one online basis extension (gsi_extend_basis) at the GPT-J q,k,v,fc group:
+    d = 4096, 28672 output rows, k = 256 with 200 columns in use.  Each timed call sees a token
+    with a new direction, so each appends a column (two projection passes, one pass over W)."""
+    import torch
+    import synthetic as S
+    import paper_2605_03109_b200 as G
+    dev = torch.device("cuda", int(os.environ.get("LOCAL_RANK", "0")))
+    torch.cuda.set_device(dev)
+    d, k_cap, k_act, d_out = 4096, 256, 200, (4096, 4096, 4096, 16384)
+    n = min(max(args.steps or 24, 1), k_cap - k_act - 4)
+    q = S.gen_basis(d, k_act + n + 4, 5100, device=dev)
+    P = torch.zeros((d, k_cap), dtype=torch.float64, device=dev)
+    P[:, :k_act] = q[:, :k_act]
+    P = S.store_basis(P).contiguous()
+    Ws = [S.gen_weight(o, d, 5101 + j, device=dev) for j, o in enumerate(d_out)]
+    lay = G.Layer(Ws, P, 0.05, max_tokens=1)
+    gen = torch.Generator(device=dev).manual_seed(5110)
+    toks = []
+    for t in range(n + 4):   # in-span part plus a component along an unused direction
+        base = q[:, :k_act] @ torch.randn(k_act, generator=gen, dtype=torch.float64, device=dev)
+        toks.append((base + 0.5 * base.norm() * q[:, k_act + t]).float())
+    x = torch.stack(toks).contiguous()
+    ka = torch.tensor([k_act], dtype=torch.int32, device=dev)
+    for t in range(4):       # warm-up extensions
+        lay.extend_basis(x[t], 0.05, ka)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(4, 4 + n):
+        lay.extend_basis(x[t], 0.05, ka)
+    e1.record()
+    torch.cuda.synchronize()
+    us = e0.elapsed_time(e1) * 1e3 / n
+    assert int(ka.item()) == k_act + 4 + n and lay.status() == 0
+    w_bytes = sum(d_out) * d * 2
+    print(json.dumps({
+        "metric": "online basis extension latency (gsi_extend_basis, one appended column)",
+        "value": us, "unit": "us", "higher_is_better": False, "n_gpus": 1, "steps": n, "warmup": 4,
+        "dtype": "f32", "data": "synthetic",
+        "config": {"workload": "extend_gptj_qkv_fc", "d": d, "k": k_cap, "k_active_start": k_act + 4,
+                   "rows": sum(d_out)},
+        "w_stream_gbs": w_bytes / (us * 1e-6) / 1e9,
+        "note": "two CUDA-core projection/residual passes over P and one W r pass; 11 launches"}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -312,7 +358,7 @@ def main():
     ap.add_argument("--impl", default="gsi", choices=["gsi", "reference"])
     ap.add_argument("--gate", default="10", choices=["0", "10", "23", "100"],
                     help="target gate rate of the GPT-J workload (percent)")
-    ap.add_argument("--workload", default="gptj", choices=["gptj", "gpt2", "opt", "gptj_b64"],
+    ap.add_argument("--workload", default="gptj", choices=["gptj", "gpt2", "opt", "gptj_b64", "extend"],
                     help="gptj: the headline (config 3); gpt2: config 2; opt: config 4 sweep point "
                          "(--k --eps --sigma-scale); gptj_b64: config 5 (--outlier)")
     ap.add_argument("--k", type=int, default=256)
@@ -340,6 +386,9 @@ def main():
         args.steps = 5 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup
 
+    if args.workload == "extend":
+        run_extend(args)
+        return
     import synthetic as S
     from dataclasses import replace
     if args.workload == "gptj":

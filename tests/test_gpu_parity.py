@@ -732,3 +732,46 @@ def test_extend_basis_sequence_then_forward_sees_the_new_columns():
     # (rho of these in-span tokens is storage rounding residue, ~1e-3, and not compared)
     compare_group(x[:14], torch.from_numpy(Pb.view(np.int16)).view(torch.bfloat16), Ws, tau,
                   y.cpu().numpy(), gate.cpu().numpy(), None)
+
+
+def test_extend_basis_then_persistent_stack_after_rebinding():
+    """The persistent kernel caches max|P| at bind time, so a stack is bound again after an
+    extension; its steps then use the wider basis (the token that caused the extension takes
+    the fast path) and still agree with the oracle run on the oracle's own extended basis."""
+    from oracle import gsi_oracle as O
+    d, k_act, k_cap, d_out = 1024, 56, 64, (1024, 512)
+    q, P, Ws = _extend_case(d, k_act, k_cap, d_out, 740)
+    gen = torch.Generator().manual_seed(741)
+    new_dir = torch.linalg.qr(torch.randn(d, 1, generator=gen, dtype=torch.float64))[0][:, 0]
+    toks = []
+    for t in range(6):
+        base = q @ torch.randn(k_act, generator=gen, dtype=torch.float64)
+        toks.append((base + (0.4 * base.norm() * new_dir if t % 2 else 0.0)).float())
+    x = torch.stack(toks).contiguous()                     # odd tokens leave the span along new_dir
+    g = G()
+    Pd = P.cuda()
+    lay = g.Layer([W.cuda() for W in Ws], Pd, 0.05, max_tokens=1)
+    stack = g.Stack([lay], mode=2)
+    stack.bind([x.cuda().contiguous()], n_steps=6)
+    for _ in range(6):
+        stack.step()
+    torch.cuda.synchronize()
+    assert stack.status() == 0
+    assert stack.gate_log.cpu().numpy()[:, 0, 0].tolist() == [0, 1, 0, 1, 0, 1]
+    ka = torch.tensor([k_act], dtype=torch.int32, device="cuda")
+    appended, _ = lay.extend_basis(x[1].cuda().contiguous(), 0.05, ka)
+    assert appended.item() == 1 and ka.item() == k_act + 1
+    stack.bind([x.cuda().contiguous()], n_steps=6)         # bind again: max|P| may have grown
+    ys = []
+    for _ in range(6):
+        stack.step()
+        torch.cuda.synchronize()
+        ys.append(stack.ys[0].cpu().clone())
+    assert stack.status() == 0
+    gate = stack.gate_log.cpu().numpy()[:, 0, 0]
+    assert gate.tolist() == [0] * 6                        # new_dir is inside the span now
+    ref = O.extend(_bits(P), k_act, x[1].double().numpy(), 0.05)
+    Pb = _bits(P).copy()
+    Pb[:, k_act] = ref["v_bits"]
+    compare_group(x, torch.from_numpy(Pb.view(np.int16)).view(torch.bfloat16), Ws, 0.05,
+                  torch.cat(ys).numpy(), gate, None)
