@@ -23,7 +23,7 @@ struct Layout {
   size_t wp, c, cpart, r, normpart, ctrl, fired, rho, x_stage, y_stage, gate_stage, rho_stage,
       pk_acc, pk_slot, tc_rb, tc_ypart, f_pt, f_xb, f_cb, f_cpart, f_normpart, total;
   int O, n_slabs, slab_rows;
-  bool tc, front;
+  bool tc, front, dense_tc;
 };
 
 constexpr int kTcMinFired = 5;  // fewer fired tokens: one pass of the CUDA-core GEMV
@@ -81,14 +81,17 @@ Layout make_layout_ws(const gsi_desc_t* d) {
   L.pk_acc = take(2 * k * 8 * kAccStride);          // persistent kernel: c accumulators
   L.pk_slot = take((size_t)kPersistMaxGrid * 8);    // persistent kernel: ||r||^2 words
   // tensor-core kernels: batched handles only
-  const bool tc = !dense && d->max_tokens >= kFrontMinTokens && d->d % 64 == 0 && tc_shapes_ok(d);
+  const bool tc_any = d->max_tokens >= kFrontMinTokens && d->d % 64 == 0 && tc_shapes_ok(d);
+  const bool tc = !dense && tc_any;
+  const bool dense_tc = dense && tc_any;   // the dense baseline of batched calls, same tile routine
   L.tc_rb = take(tc ? (size_t)65 * d->d * 2 : 0);   // row 64 stays zero
-  L.tc_ypart = take(tc ? (size_t)tc_splits(O, d->d) * 64 * O * 4 : 0);
+  L.tc_ypart = take(tc_any ? (size_t)tc_splits(O, d->d) * 64 * O * 4 : 0);
   L.tc = tc;
+  L.dense_tc = dense_tc;
   // tensor-core projection / residual / image for batched calls
   const bool front = tc && d->max_tokens >= kFrontMinTokens && d->p_dtype == GSI_BF16 && d->k % 128 == 0 &&
                      d->d % 128 == 0 && O % 128 == 0;
-  const size_t rows = front ? front_rows(d->max_tokens) : 0;
+  const size_t rows = (front || dense_tc) ? front_rows(d->max_tokens) : 0;
   L.f_pt = take(front ? (size_t)d->k * d->d * 2 : 0);
   L.f_xb = take(rows * d->d * 2);
   L.f_cb = take(rows * k * 2);
@@ -228,7 +231,7 @@ gsi_status_t gsi_create(const gsi_desc_t* desc, const void* const* W, const void
   g.tc_min_fired = L.tc ? kTcMinFired : 0;
   g.rb = reinterpret_cast<uint16_t*>(h->ws + L.tc_rb);
   g.ypart = reinterpret_cast<float*>(h->ws + L.tc_ypart);
-  g.front_min_tokens = L.front ? kFrontMinTokens : 0;
+  g.front_min_tokens = (L.front || L.dense_tc) ? kFrontMinTokens : 0;
   g.proj_splits = L.front ? front_proj_splits(desc->d, desc->k) : 0;
   g.PT = reinterpret_cast<const uint16_t*>(h->ws + L.f_pt);
   g.xb = reinterpret_cast<uint16_t*>(h->ws + L.f_xb);
@@ -236,7 +239,7 @@ gsi_status_t gsi_create(const gsi_desc_t* desc, const void* const* W, const void
   g.cpart3 = reinterpret_cast<float*>(h->ws + L.f_cpart);
   g.normpart3 = reinterpret_cast<float*>(h->ws + L.f_normpart);
 
-  if (L.tc) {
+  if (L.tc || L.dense_tc) {
     if (!build_tma_maps(g, L.front, desc->max_tokens, &h->tm)) {
       delete h;
       return GSI_ERR_CUDA;

@@ -43,7 +43,7 @@ __device__ __forceinline__ void split3(float v, uint16_t& hi, uint16_t& mid, uin
   lo = bf16_bits(r2);
 }
 
-__device__ __forceinline__ int rows3(int n_tokens) { return (3 * n_tokens + 15) & ~15; }
+__device__ __forceinline__ int rows3(int n_tokens) { return term_rows(n_tokens); }
 
 // src [n_tokens][len] fp32 -> dst [rows3][len] bf16 terms; rows past 3 n_tokens are zero.
 // One block row (blockIdx.y) per token slot, 8 elements per thread.
@@ -87,20 +87,6 @@ __global__ void __launch_bounds__(256) k_split3_x(GroupParams g, IoRef io, int n
   }
 }
 
-// Sum of the three term columns of 16 tokens: columns 48q .. 48q+47 of this lane.
-__device__ __forceinline__ void load_tokens16(uint32_t tmem_lane, int q, float (&s)[16]) {
-  uint32_t v[3][16];
-#pragma unroll
-  for (int i = 0; i < 3; ++i) tmem_ld16(tmem_lane + 48 * q + 16 * i, v[i]);
-  tmem_ld_wait();
-#pragma unroll
-  for (int tt = 0; tt < 16; ++tt) {
-    const int c = 3 * tt;
-    s[tt] = (__uint_as_float(v[c / 16][c % 16]) + __uint_as_float(v[(c + 1) / 16][(c + 1) % 16])) +
-            __uint_as_float(v[(c + 2) / 16][(c + 2) % 16]);
-  }
-}
-
 // c partials: cpart3[split][t][128*tile + lane row] over this split's share of d.
 __global__ void __launch_bounds__(kThreads, 1)
 k_proj_tc(GroupParams g, const __grid_constant__ TmaMaps tm, int n_tokens) {
@@ -121,7 +107,7 @@ k_proj_tc(GroupParams g, const __grid_constant__ TmaMaps tm, int n_tokens) {
     float* out = g.cpart3 + (size_t)split * g.B * g.k + tile * kTM + warp * 32 + lane;
     for (int q = 0; 16 * q < n_tokens; ++q) {
       float s[16];
-      load_tokens16(tl, q, s);
+      sum3_tokens16(tl, q, s);
 #pragma unroll
       for (int tt = 0; tt < 16; ++tt)
         if (16 * q + tt < n_tokens) out[(size_t)(16 * q + tt) * g.k] = s[tt];
@@ -202,7 +188,7 @@ k_resid_image_tc(GroupParams g, const __grid_constant__ TmaMaps tm, IoRef io, in
     const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);
     for (int q = q_lo; q < q_hi && ok; ++q) {
       float s[16];
-      load_tokens16(tl, q - q_lo, s);
+      sum3_tokens16(tl, q - q_lo, s);
       if (image) {
 #pragma unroll
         for (int tt = 0; tt < 16; ++tt)
@@ -271,6 +257,12 @@ int front_proj_splits(int d, int k) {
 cudaError_t launch_transpose_bf16(const void* P, int d, int k, void* PT, cudaStream_t st) {
   k_transpose_bf16<<<dim3((k + 31) / 32, (d + 31) / 32), 256, 0, st>>>(
       static_cast<const uint16_t*>(P), d, k, static_cast<uint16_t*>(PT));
+  return cudaGetLastError();
+}
+
+cudaError_t launch_split3_x(const GroupParams& g, const IoRef& io, int n_tokens, cudaStream_t st) {
+  const int slots = (front_rows(n_tokens) + 2) / 3;
+  k_split3_x<<<dim3((g.d / 8 + 255) / 256, slots), 256, 0, st>>>(g, io, n_tokens);
   return cudaGetLastError();
 }
 

@@ -244,6 +244,11 @@ cudaError_t launch_front_tc(const GroupParams& g, const TmaMaps& tm, const IoRef
 // Encodes the layer's tensor maps (front: also those of the batched front end).
 // False when the driver's encoder is unavailable or rejects a shape.
 bool build_tma_maps(const GroupParams& g, bool front, int max_tokens, TmaMaps* out);
+// xb = the three bf16 terms of every token of x (operand rows 3t, 3t+1, 3t+2).
+cudaError_t launch_split3_x(const GroupParams& g, const IoRef& io, int n_tokens, cudaStream_t stream);
+// Dense baseline for batched calls on the tensor cores: y = W x, x as exact bf16 terms.
+cudaError_t launch_dense_gemm_tc(const GroupParams& g, const TmaMaps& tm, const IoRef& io,
+                                 int n_tokens, cudaStream_t stream, int* n_launches);
 cudaError_t launch_transpose_bf16(const void* P, int d, int k, void* PT, cudaStream_t stream);
 int front_proj_splits(int d, int k);
 int front_rows(int max_tokens);   // rows of the three-term operands

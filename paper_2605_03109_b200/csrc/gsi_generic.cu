@@ -386,6 +386,8 @@ cudaError_t launch_generic_forward(const GroupParams& g, const TmaMaps* tm, cons
   int grid = (g.O + kWarps - 1) / kWarps;
   if (grid > 148 * 8) grid = 148 * 8;
   if (g.flags & GSI_FLAG_DENSE) {
+    if (tm && g.front_min_tokens > 0 && n_tokens >= g.front_min_tokens)
+      return launch_dense_gemm_tc(g, *tm, io, n_tokens, st, n_launches);
     k_stream_gemv<true><<<grid, kThreads, 0, st>>>(g, io, n_tokens);
     *n_launches += 1;
     return cudaGetLastError();
@@ -428,7 +430,8 @@ cudaError_t launch_gated_gemv(const GroupParams& g, const IoRef& io, cudaStream_
 }
 
 int generic_launch_count(const GroupParams& g, int n_tokens) {
-  if (g.flags & GSI_FLAG_DENSE) return 1;
+  if (g.flags & GSI_FLAG_DENSE)
+    return (g.front_min_tokens > 0 && n_tokens >= g.front_min_tokens) ? 3 : 1;
   const bool stat = g.flags & GSI_FLAG_STATIC_PROJECTION;
   if (g.front_min_tokens > 0 && n_tokens >= g.front_min_tokens) return stat ? 4 : 6;
   return 4 + (stat ? 0 : 1 + (g.tc_min_fired > 0 ? 3 : 0));

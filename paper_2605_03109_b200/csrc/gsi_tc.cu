@@ -118,7 +118,73 @@ __global__ void __launch_bounds__(256) k_add_partials(GroupParams g, IoRef io, i
   }
 }
 
+// ---- dense baseline for batched calls: y = W x on the same tile routine ----------------
+constexpr int kDenseStages = 4;
+constexpr int kDenseN = 192;         // 3 terms x 64 tokens
+constexpr int kDenseTmem = 256;
+constexpr int kDenseSmem = Cfg<kDenseStages, kDenseN>::kSmem;
+
+__global__ void __launch_bounds__(kThreadsTc, 1)
+k_dense_gemm_tc(GroupParams g, const __grid_constant__ TmaMaps tm, int splits, int n_tokens) {
+  extern __shared__ unsigned char smem_raw[];
+  pdl_launch_dependents();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int tile = blockIdx.x / splits, split = blockIdx.x % splits;
+  const int row0 = tile * kTM;
+  int j = 0;
+  while (j + 1 < g.n_maps && row0 >= g.off[j + 1]) ++j;
+  const int nkb = g.d / kTK;
+  const int kb0 = (int)((long long)nkb * split / splits), kb1 = (int)((long long)nkb * (split + 1) / splits);
+  uint32_t tmem;
+  const bool ok = tile_mma<kDenseStages, kDenseN, kDenseTmem>(smem_raw, &tm.w[j], row0 - g.off[j], &tm.xb, 0,
+                                                              term_rows(n_tokens), kb0, kb1 - kb0, &tmem);
+  if (!ok) {
+    if (threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
+  } else {
+    const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);
+    float* yp = g.ypart + ((size_t)split * kMaxN) * g.O + row0 + warp * 32 + lane;
+    for (int q = 0; 16 * q < n_tokens; ++q) {
+      float s[16];
+      sum3_tokens16(tl, q, s);
+#pragma unroll
+      for (int tt = 0; tt < 16; ++tt)
+        if (16 * q + tt < n_tokens) yp[(size_t)(16 * q + tt) * g.O] = s[tt];
+    }
+  }
+  tile_release<kDenseTmem>(tmem);
+}
+
+// y[t][row] = sum over splits (fixed order); the dense baseline reports every token as gated
+__global__ void __launch_bounds__(256) k_sum_partials(GroupParams g, IoRef io, int splits, int n_tokens) {
+  pdl_launch_dependents();
+  pdl_wait();
+  const int t = blockIdx.y;
+  if (blockIdx.x == 0 && threadIdx.x == 0)
+    io.gate[(long long)io_slot(io) * io.log_step_stride + t] = 1;
+  for (int row = blockIdx.x * 256 + threadIdx.x; row < g.O; row += gridDim.x * 256) {
+    float s = 0.f;
+    for (int sp = 0; sp < splits; ++sp) s += g.ypart[((size_t)sp * kMaxN + t) * g.O + row];
+    io.y[(size_t)t * g.O + row] = s;
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_dense_gemm_tc(const GroupParams& g, const TmaMaps& tm, const IoRef& io, int n_tokens,
+                                 cudaStream_t st, int* n_launches) {
+  cudaError_t e = cudaFuncSetAttribute(k_dense_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                       kDenseSmem);
+  if (e != cudaSuccess) return e;
+  const int splits = tc_splits(g.O, g.d);
+  if ((e = launch_split3_x(g, io, n_tokens, st)) != cudaSuccess) return e;
+  if ((e = launch_pdl(k_dense_gemm_tc, dim3((g.O / kTM) * splits), dim3(kThreadsTc), kDenseSmem, st, g, tm,
+                      splits, n_tokens)) != cudaSuccess ||
+      (e = launch_pdl(k_sum_partials, dim3((g.O + 1023) / 1024, n_tokens), dim3(256), 0, st, g, io, splits,
+                      n_tokens)) != cudaSuccess)
+    return e;
+  if (n_launches) *n_launches += 3;
+  return cudaGetLastError();
+}
 
 int tc_splits(int O, int d) {
   const int tiles = O / kTM, nkb = d / kTK;

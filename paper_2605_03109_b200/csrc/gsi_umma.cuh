@@ -213,6 +213,24 @@ __device__ __forceinline__ bool tile_mma(unsigned char* smem_raw, const CUtensor
   return done;
 }
 
+// fp32 operands enter the batched kernels as three bf16 terms in operand rows 3t, 3t+1,
+// 3t+2 (t = token): this adds the three columns of 16 tokens, columns 48q .. 48q+47 of
+// this thread's tensor-memory lane.
+__device__ __forceinline__ void sum3_tokens16(uint32_t tmem_lane, int q, float (&s)[16]) {
+  uint32_t v[3][16];
+#pragma unroll
+  for (int i = 0; i < 3; ++i) tmem_ld16(tmem_lane + 48 * q + 16 * i, v[i]);
+  tmem_ld_wait();
+#pragma unroll
+  for (int tt = 0; tt < 16; ++tt) {
+    const int c = 3 * tt;
+    s[tt] = (__uint_as_float(v[c / 16][c % 16]) + __uint_as_float(v[(c + 1) / 16][(c + 1) % 16])) +
+            __uint_as_float(v[(c + 2) / 16][(c + 2) % 16]);
+  }
+}
+// Operand rows of n tokens, rounded up to the 16-row boxes.
+__host__ __device__ __forceinline__ int term_rows(int n_tokens) { return (3 * n_tokens + 15) & ~15; }
+
 template <int kTmemCols>
 __device__ __forceinline__ void tile_release(uint32_t tmem) {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
