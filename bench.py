@@ -438,7 +438,7 @@ def main():
         return
     stream = torch.cuda.Stream(device)
     graph = capture_step(stack, stream)
-    dense_arm = True   # batch 1: the streaming GEMV; batched: the tensor-core GEMM with exact bf16 terms of x
+    dense_arm = True   # batch 1: the streaming GEMV; batched: the tensor-core GEMM on bf16(x)
     if dense_arm:
         dstack = G.Stack(dense_layers)
         dstack.bind(xs, n_steps=n_steps, want_rho=False)
@@ -519,7 +519,7 @@ def main():
                 "frac_of_peak": ab["dense"] / (ms_dense * 1e-3) / 1e9 / peak,
                 "speedup_of_gsi": ms_dense / ms_max,
                 "kernel": ("k_decode_step with GSI_FLAG_DENSE groups" if spec.batch == 1 else
-                           "k_split3_x + k_dense_gemm_tc + k_sum_partials per group (tcgen05)"),
+                           "k_pack_x_bf16 + k_dense_gemm_tc + k_sum_partials per group (tcgen05, x rounded to bf16)"),
             } if dense_arm else {
                 "ideal_ms_per_step_at_peak": ab["dense"] / (peak * 1e9) * 1e3,
                 "note": "no batched dense kernel here; figure is dense bytes / measured peak",

@@ -84,14 +84,14 @@ Layout make_layout_ws(const gsi_desc_t* d) {
   const bool tc_any = d->max_tokens >= kFrontMinTokens && d->d % 64 == 0 && tc_shapes_ok(d);
   const bool tc = !dense && tc_any;
   const bool dense_tc = dense && tc_any;   // the dense baseline of batched calls, same tile routine
-  L.tc_rb = take(tc ? (size_t)65 * d->d * 2 : 0);   // row 64 stays zero
+  L.tc_rb = take(tc_any ? (size_t)65 * d->d * 2 : 0);   // row 64 stays zero
   L.tc_ypart = take(tc_any ? (size_t)tc_splits(O, d->d) * 64 * O * 4 : 0);
   L.tc = tc;
   L.dense_tc = dense_tc;
   // tensor-core projection / residual / image for batched calls
   const bool front = tc && d->max_tokens >= kFrontMinTokens && d->p_dtype == GSI_BF16 && d->k % 128 == 0 &&
                      d->d % 128 == 0 && O % 128 == 0;
-  const size_t rows = (front || dense_tc) ? front_rows(d->max_tokens) : 0;
+  const size_t rows = front ? front_rows(d->max_tokens) : 0;
   L.f_pt = take(front ? (size_t)d->k * d->d * 2 : 0);
   L.f_xb = take(rows * d->d * 2);
   L.f_cb = take(rows * k * 2);

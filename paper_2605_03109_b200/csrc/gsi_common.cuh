@@ -246,7 +246,7 @@ cudaError_t launch_front_tc(const GroupParams& g, const TmaMaps& tm, const IoRef
 bool build_tma_maps(const GroupParams& g, bool front, int max_tokens, TmaMaps* out);
 // xb = the three bf16 terms of every token of x (operand rows 3t, 3t+1, 3t+2).
 cudaError_t launch_split3_x(const GroupParams& g, const IoRef& io, int n_tokens, cudaStream_t stream);
-// Dense baseline for batched calls on the tensor cores: y = W x, x as exact bf16 terms.
+// Dense baseline for batched calls on the tensor cores: y = W bf16(x).
 cudaError_t launch_dense_gemm_tc(const GroupParams& g, const TmaMaps& tm, const IoRef& io,
                                  int n_tokens, cudaStream_t stream, int* n_launches);
 cudaError_t launch_transpose_bf16(const void* P, int d, int k, void* PT, cudaStream_t stream);

@@ -118,13 +118,22 @@ __global__ void __launch_bounds__(256) k_add_partials(GroupParams g, IoRef io, i
   }
 }
 
-// ---- dense baseline for batched calls: y = W x on the same tile routine ----------------
-constexpr int kDenseStages = 4;
-constexpr int kDenseN = 192;         // 3 terms x 64 tokens
-constexpr int kDenseTmem = 256;
-constexpr int kDenseSmem = Cfg<kDenseStages, kDenseN>::kSmem;
+// ---- dense baseline for batched calls: y = W bf16(x) on the same tile routine -----------
+// The activations are rounded to bf16 as an ordinary bf16 GEMM would take them (one operand
+// row per token), which makes this the strongest dense comparator the tile routine offers:
+// the stage size and occupancy of the gated-residual GEMM, no pack by a fired list.
+__global__ void __launch_bounds__(256) k_pack_x_bf16(GroupParams g, IoRef io, int n_tokens) {
+  pdl_launch_dependents();
+  const int row = blockIdx.y;   // operand row = token; rows up to the next multiple of 16 are zero
+  const float* x = io.x + (long long)io_slot(io) * io.x_step_stride + (size_t)row * g.d;
+  for (int i = blockIdx.x * 256 + threadIdx.x; i < g.d; i += gridDim.x * 256) {
+    const float v = row < n_tokens ? __ldg(x + i) : 0.f;
+    const __nv_bfloat16 h = __float2bfloat16_rn(v);
+    g.rb[(size_t)row * g.d + i] = *reinterpret_cast<const uint16_t*>(&h);
+  }
+}
 
-__global__ void __launch_bounds__(kThreadsTc, 1)
+__global__ void __launch_bounds__(kThreadsTc, 2)
 k_dense_gemm_tc(GroupParams g, const __grid_constant__ TmaMaps tm, int splits, int n_tokens) {
   extern __shared__ unsigned char smem_raw[];
   pdl_launch_dependents();
@@ -135,23 +144,24 @@ k_dense_gemm_tc(GroupParams g, const __grid_constant__ TmaMaps tm, int splits, i
   while (j + 1 < g.n_maps && row0 >= g.off[j + 1]) ++j;
   const int nkb = g.d / kTK;
   const int kb0 = (int)((long long)nkb * split / splits), kb1 = (int)((long long)nkb * (split + 1) / splits);
+  const int N = (n_tokens + 15) & ~15;
   uint32_t tmem;
-  const bool ok = tile_mma<kDenseStages, kDenseN, kDenseTmem>(smem_raw, &tm.w[j], row0 - g.off[j], &tm.xb, 0,
-                                                              term_rows(n_tokens), kb0, kb1 - kb0, &tmem);
+  const bool ok = tile_mma<kStages, kMaxN, kTmemCols>(smem_raw, &tm.w[j], row0 - g.off[j], &tm.rb, 0, N,
+                                                      kb0, kb1 - kb0, &tmem);
   if (!ok) {
     if (threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
   } else {
-    const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);
     float* yp = g.ypart + ((size_t)split * kMaxN) * g.O + row0 + warp * 32 + lane;
-    for (int q = 0; 16 * q < n_tokens; ++q) {
-      float s[16];
-      sum3_tokens16(tl, q, s);
+    for (int c0 = 0; c0 < N; c0 += 16) {
+      uint32_t v[16];
+      tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + c0, v);
+      tmem_ld_wait();
 #pragma unroll
-      for (int tt = 0; tt < 16; ++tt)
-        if (16 * q + tt < n_tokens) yp[(size_t)(16 * q + tt) * g.O] = s[tt];
+      for (int c = 0; c < 16; ++c)
+        if (c0 + c < n_tokens) yp[(size_t)(c0 + c) * g.O] = __uint_as_float(v[c]);
     }
   }
-  tile_release<kDenseTmem>(tmem);
+  tile_release<kTmemCols>(tmem);
 }
 
 // y[t][row] = sum over splits (fixed order); the dense baseline reports every token as gated
@@ -173,11 +183,12 @@ __global__ void __launch_bounds__(256) k_sum_partials(GroupParams g, IoRef io, i
 cudaError_t launch_dense_gemm_tc(const GroupParams& g, const TmaMaps& tm, const IoRef& io, int n_tokens,
                                  cudaStream_t st, int* n_launches) {
   cudaError_t e = cudaFuncSetAttribute(k_dense_gemm_tc, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                       kDenseSmem);
+                                       kTcSmem);
   if (e != cudaSuccess) return e;
   const int splits = tc_splits(g.O, g.d);
-  if ((e = launch_split3_x(g, io, n_tokens, st)) != cudaSuccess) return e;
-  if ((e = launch_pdl(k_dense_gemm_tc, dim3((g.O / kTM) * splits), dim3(kThreadsTc), kDenseSmem, st, g, tm,
+  const int rows = (n_tokens + 15) & ~15;
+  k_pack_x_bf16<<<dim3((g.d + 2047) / 2048, rows), 256, 0, st>>>(g, io, n_tokens);
+  if ((e = launch_pdl(k_dense_gemm_tc, dim3((g.O / kTM) * splits), dim3(kThreadsTc), kTcSmem, st, g, tm,
                       splits, n_tokens)) != cudaSuccess ||
       (e = launch_pdl(k_sum_partials, dim3((g.O + 1023) / 1024, n_tokens), dim3(256), 0, st, g, io, splits,
                       n_tokens)) != cudaSuccess)

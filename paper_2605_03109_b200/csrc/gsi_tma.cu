@@ -46,9 +46,8 @@ bool build_tma_maps(const GroupParams& g, bool front, int max_tokens, TmaMaps* o
   for (int j = 0; j < g.n_maps; ++j)
     if (!encode(&out->w[j], g.W[j], (size_t)g.d_out[j], (size_t)g.d, umma::kTM)) return false;
   const size_t rows = (size_t)front_rows(max_tokens);
-  if (g.flags & GSI_FLAG_DENSE)   // dense baseline: W and the terms of x only
-    return encode(&out->xb, g.xb, rows, (size_t)g.d, umma::kBBox);
   if (!encode(&out->rb, g.rb, 65, (size_t)g.d, umma::kBBox)) return false;
+  if (g.flags & GSI_FLAG_DENSE) return true;   // dense baseline: W and bf16(x) in rb only
   if (!front) return true;
   return encode(&out->p, g.P, (size_t)g.d, (size_t)g.k, umma::kTM) &&
          encode(&out->pt, g.PT, (size_t)g.k, (size_t)g.d, umma::kTM) &&

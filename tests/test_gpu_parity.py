@@ -779,15 +779,17 @@ def test_extend_basis_then_persistent_stack_after_rebinding():
 
 @pytest.mark.parametrize("n_tokens", [2, 17, 64])
 def test_dense_baseline_batched_runs_on_the_tensor_cores(n_tokens):
-    """GSI_FLAG_DENSE handles take batched calls through the tcgen05 tile routine with x as
-    three exact bf16 terms: y = W x to fp32 accumulation accuracy, every token reported gated."""
+    """GSI_FLAG_DENSE handles take batched calls through the tcgen05 tile routine with x
+    rounded to bf16, as an ordinary bf16 GEMM takes its activations: y = W bf16(x) to fp32
+    accumulation accuracy (checked exactly against that product), every token reported gated."""
     g = G()
     d, d_out = 1024, (768, 256)
     Ws = [S.gen_weight(o, d, 810 + j) for j, o in enumerate(d_out)]
     x = torch.randn((n_tokens, d), generator=torch.Generator().manual_seed(812)) * 3.0
     lay, y, gate, rho = run_layer(x.contiguous(), None, Ws, 0.0, 64, flags=g.GSI_FLAG_DENSE)
     assert gate.all()
-    ref = torch.cat([x.to(torch.float64) @ W.to(torch.float64).T for W in Ws], dim=1).numpy()
+    xr = x.to(torch.bfloat16).to(torch.float64)
+    ref = torch.cat([xr @ W.to(torch.float64).T for W in Ws], dim=1).numpy()
     assert np.max(np.abs(y - ref)) <= 2e-5 * np.max(np.abs(ref))
-    _, y1, _, _ = run_layer(x.contiguous(), None, Ws, 0.0, 1, flags=g.GSI_FLAG_DENSE)   # streaming GEMV
-    assert np.max(np.abs(y - y1)) <= 2e-5 * np.max(np.abs(ref))
+    _, y1, _, _ = run_layer(x.contiguous(), None, Ws, 0.0, 1, flags=g.GSI_FLAG_DENSE)   # fp32 x, streaming GEMV
+    assert np.max(np.abs(y - y1)) <= 1e-2 * np.max(np.abs(ref))
