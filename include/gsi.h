@@ -75,8 +75,11 @@ enum {
   /* Static projection (Remark after Theorem 3.1, "Mode C"): never add W r.
      Gate bytes and rho are still reported. */
   GSI_FLAG_STATIC_PROJECTION = 1u,
-  /* Dense baseline: y = W x by the streaming GEMV, no projection, no image.
-     Gate bytes are written as 1.  Used to measure the speed-up honestly. */
+  /* Dense baseline: y = W x, no projection, no image; gate bytes are written as
+     1.  Used to measure the speed-up honestly.  Single-token calls: streaming
+     GEMV on the fp32 x.  Calls of 2 or more tokens (d a multiple of 64, every
+     d_out a multiple of 128): tensor-core GEMM with x rounded to bf16, as an
+     ordinary bf16 GEMM takes its activations. */
   GSI_FLAG_DENSE = 2u
 };
 
