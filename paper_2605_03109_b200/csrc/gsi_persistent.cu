@@ -42,7 +42,7 @@ constexpr unsigned kSpinLimit = 1u << 22;
 constexpr int kCountShift = 54;
 
 // shared memory map (bytes)
-constexpr int kXBatch = 4;           // float4 loads of x in flight per thread
+constexpr int kXBatch = 5;           // float4 loads of x in flight per thread
 constexpr int kOffBar = 0;          // full[kSlots], empty[kSlots]
 constexpr int kOffMisc = 256;       // abort flag, scalars
 constexpr int kOffX = 512;          // x of this CTA's basis rows      (kPersistMaxPRows floats)
