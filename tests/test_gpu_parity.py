@@ -793,3 +793,31 @@ def test_dense_baseline_batched_runs_on_the_tensor_cores(n_tokens):
     assert np.max(np.abs(y - ref)) <= 2e-5 * np.max(np.abs(ref))
     _, y1, _, _ = run_layer(x.contiguous(), None, Ws, 0.0, 1, flags=g.GSI_FLAG_DENSE)   # fp32 x, streaming GEMV
     assert np.max(np.abs(y - y1)) <= 1e-2 * np.max(np.abs(ref))
+
+
+def test_set_concurrent_validates_its_arguments_and_falls_back_when_rows_do_not_fit():
+    g = G()
+    x, P, Ws = make_small(256, 64, (256,), 4, seed=77)
+    lays = [g.Layer([W.cuda() for W in Ws], P.cuda(), 0.05, max_tokens=1) for _ in range(3)]
+    with pytest.raises(g.GsiError):
+        g.Stack(lays, concurrent=[2])            # no group after the last one
+    with pytest.raises(g.GsiError):
+        g.Stack(lays, concurrent=[-1])
+    with pytest.raises(g.GsiError):
+        g.Stack(lays, concurrent=[0, 1])         # group 1 would belong to two pairs
+    # a valid pair of small groups: same results as the sequential schedule
+    xs = [x.cuda().contiguous() for _ in range(3)]
+    outs = []
+    for conc in ([], [1]):
+        st = g.Stack(lays, mode=2, concurrent=conc)
+        st.bind(xs, n_steps=4)
+        ys = []
+        for _ in range(4):
+            st.step()
+            torch.cuda.synchronize()
+            ys.append(torch.cat([y.cpu() for y in st.ys], dim=1).clone())
+        assert st.status() == 0
+        outs.append((torch.cat(ys).numpy(), st.gate_log.cpu().numpy().copy()))
+    assert np.array_equal(outs[0][1], outs[1][1])
+    assert np.max(np.abs(outs[0][0] - outs[1][0])) <= 1e-4 * np.max(np.abs(outs[0][0]))
+    compare_group(x, P, Ws, 0.05, outs[1][0][:, 512:768], outs[1][1][:, 2, 0], None)
