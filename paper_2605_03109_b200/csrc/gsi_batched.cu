@@ -72,6 +72,7 @@ __device__ __forceinline__ void store_terms(const float (&v)[8], bool live, uint
 
 __global__ void __launch_bounds__(256) k_split3_x(GroupParams g, IoRef io, int n_tokens) {
   pdl_launch_dependents();
+  pdl_wait();   // xb may still be read by the previous call's projection
   const int slot = blockIdx.y, n_rows = rows3(n_tokens);
   const bool live = slot < n_tokens;
   const float* x = io.x + (long long)io_slot(io) * io.x_step_stride + (size_t)slot * g.d;
@@ -277,10 +278,11 @@ cudaError_t launch_front_tc(const GroupParams& g, const TmaMaps& tm, const IoRef
   const int nq = (n_tokens + 15) / 16, tiles = g.d / kTM;
   int rs = tiles <= 37 ? 4 : tiles <= 74 ? 2 : 1;   // token ranges per residual tile
   if (rs > nq) rs = nq;
-  k_split3_x<<<dim3((g.d / 8 + 255) / 256, slots), 256, 0, st>>>(g, io, n_tokens);
   // the x the residual blocks read before their wait is an input of the call, complete before
   // k_split3_x was launched
-  if ((e = launch_pdl(k_proj_tc, dim3((g.k / kTM) * g.proj_splits), dim3(kThreads), kSmem3, st, g, tm,
+  if ((e = launch_pdl(k_split3_x, dim3((g.d / 8 + 255) / 256, slots), dim3(256), 0, st, g, io, n_tokens)) !=
+          cudaSuccess ||
+      (e = launch_pdl(k_proj_tc, dim3((g.k / kTM) * g.proj_splits), dim3(kThreads), kSmem3, st, g, tm,
                       n_tokens)) != cudaSuccess ||
       (e = launch_pdl(k_reduce_split3_c, dim3(slots), dim3(256), 0, st, g, n_tokens)) != cudaSuccess ||
       (e = launch_pdl(k_resid_image_tc, dim3((g.d / kTM) * rs + g.O / kTM), dim3(kThreads), kSmemRI, st, g,
