@@ -199,6 +199,7 @@ cudaError_t launch_dense_gemm_tc(const GroupParams& g, const TmaMaps& tm, const 
 
 int tc_splits(int O, int d) {
   const int tiles = O / kTM, nkb = d / kTK;
+  if (tiles >= 148) return 1;   // a tile per CTA already fills the SMs: long pipelines, no partial sums to add
   int s = (2 * 148 + tiles - 1) / tiles;
   if (s > 8) s = 8;
   if (s > nkb / 4) s = nkb / 4;
