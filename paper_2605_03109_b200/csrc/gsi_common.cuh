@@ -140,7 +140,7 @@ __device__ __forceinline__ void decide_gate_last_block(const GroupParams& g, con
   unsigned char* gate = io.gate + (long long)slot * io.log_step_stride;
   float* rho = io.rho ? io.rho + (long long)slot * io.log_step_stride : g.rho_scratch;
   // L adjacent lanes share a token: each sums a contiguous range of parts in order (loads
-  // issued eight parts at a time), then the L sums are combined by a butterfly, so the
+  // issued sixteen parts at a time), then the L sums are combined by a butterfly, so the
   // result depends on n_tokens and the block size only through L and is reproducible.
   int L = 1;
   while (2 * L <= 32 && 2 * L * n_tokens <= (int)blockDim.x) L *= 2;
@@ -152,13 +152,13 @@ __device__ __forceinline__ void decide_gate_last_block(const GroupParams& g, con
     double sr = 0.0, sx = 0.0;
     if (live) {
       const float2* np = reinterpret_cast<const float2*>(normpart) + t;
-      for (int p = p0; p < p1; p += 8) {
-        float2 v[8];
+      for (int p = p0; p < p1; p += 16) {
+        float2 v[16];
 #pragma unroll
-        for (int u = 0; u < 8; ++u)
+        for (int u = 0; u < 16; ++u)
           v[u] = (p + u < p1) ? __ldcg(np + (size_t)(p + u) * g.B) : make_float2(0.f, 0.f);
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
+        for (int u = 0; u < 16; ++u) {
           sr += (double)v[u].x;
           sx += (double)v[u].y;
         }
