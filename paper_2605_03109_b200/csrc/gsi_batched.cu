@@ -276,7 +276,7 @@ cudaError_t launch_front_tc(const GroupParams& g, const TmaMaps& tm, const IoRef
     return e;
   const int slots = (front_rows(n_tokens) + 2) / 3;   // token slots covering every operand row
   const int nq = (n_tokens + 15) / 16, tiles = g.d / kTM;
-  int rs = tiles <= 37 ? 4 : tiles <= 74 ? 2 : 1;   // token ranges per residual tile
+  int rs = tiles <= 37 ? 4 : tiles <= 148 ? 2 : 1;   // token ranges per residual tile (measured: 4 for all is slower)
   if (rs > nq) rs = nq;
   // the x the residual blocks read before their wait is an input of the call, complete before
   // k_split3_x was launched
