@@ -821,3 +821,55 @@ def test_set_concurrent_validates_its_arguments_and_falls_back_when_rows_do_not_
     assert np.array_equal(outs[0][1], outs[1][1])
     assert np.max(np.abs(outs[0][0] - outs[1][0])) <= 1e-4 * np.max(np.abs(outs[0][0]))
     compare_group(x, P, Ws, 0.05, outs[1][0][:, 512:768], outs[1][1][:, 2, 0], None)
+
+
+def test_stack_of_batched_groups_on_the_tensor_cores_with_graph_replay():
+    """A chain of two groups stepped with 8 tokens per step: every contraction runs on tcgen05
+    (programmatic dependent launches inside a captured graph); steps and graph replays agree
+    with the oracle and with each other."""
+    g = G()
+    d, k, B, n_steps = 1024, 128, 8, 3
+    groups = []
+    for i, d_out in enumerate([(512, 256), (1024,)]):
+        q = S.gen_basis(d, k, 880 + i)
+        P = S.store_basis(q)
+        Ws = [S.gen_weight(o, d, 890 + 10 * i + j) for j, o in enumerate(d_out)]
+        pt = S.gen_true_basis(q, 64, 64, 885 + i)
+        x, _ = S.gen_activations(pt, n_steps * B, 0.004, 0.0,
+                                 dict(z=900 + i, noise=910 + i, outlier_mask=0, outlier_values=0))
+        gen = torch.Generator().manual_seed(920 + i)
+        x[::5] = torch.randn((len(range(0, n_steps * B, 5)), d), generator=gen)
+        groups.append((x.contiguous(), P, Ws))
+    layers = [g.Layer([W.cuda() for W in Ws], P.cuda(), 0.05, max_tokens=B) for _, P, Ws in groups]
+    stack = g.Stack(layers)
+    stack.bind([x.cuda() for x, _, _ in groups], n_steps=n_steps)
+    assert not stack.is_persistent() and stack.launches_per_step() == 2 * 6 + 1
+    ys = [[] for _ in groups]
+    for s in range(n_steps):
+        stack.step()
+        torch.cuda.synchronize()
+        for i, y in enumerate(stack.ys):
+            ys[i].append(y.cpu().clone())
+    assert stack.status() == 0
+    gate_log = stack.gate_log.cpu().numpy()               # [steps][groups][B]
+    rho_log = stack.rho_log.cpu().numpy()
+    for i, (x, P, Ws) in enumerate(groups):
+        compare_group(x, P, Ws, 0.05, torch.cat(ys[i]).numpy(), gate_log[:, i, :].reshape(-1),
+                      rho_log[:, i, :].reshape(-1))
+    assert 0 < gate_log.mean() < 0.5
+    stack.gate_log.zero_()
+    stack.seek(0)
+    stream = torch.cuda.Stream()
+    with torch.cuda.stream(stream):
+        stack.step(stream)
+        stack.seek(0, stream)
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            stack.step(stream)
+        for _ in range(n_steps):
+            graph.replay()
+    torch.cuda.synchronize()
+    assert stack.status() == 0
+    assert np.array_equal(stack.gate_log.cpu().numpy(), gate_log)
+    for i, y in enumerate(stack.ys):
+        assert torch.equal(y.cpu(), ys[i][-1])
