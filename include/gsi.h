@@ -276,9 +276,11 @@ gsi_status_t gsi_stack_set_concurrent(gsi_stack_t s, int first_group, int enable
 
 /*
  * Execution mode, taken at the next gsi_stack_bind:
- *   0 (default)  one persistent launch per step when every group qualifies
- *                (batch 1, bf16 basis with k in {64,128,256,512}, d a
- *                multiple of 16, 32-byte aligned W), else the per-stage kernels;
+ *   0 (default)  the persistent kernel, one launch per token of the step, when
+ *                every group qualifies (one or two tokens per step, no dense
+ *                group in a two-token stack, bf16 basis with k in
+ *                {64,128,256,512}, d a multiple of 16, 32-byte aligned W, rows
+ *                that fit the per-CTA buffers), else the per-stage / batched kernels;
  *   1            always the per-stage kernels;
  *   2            the persistent launch or GSI_ERR_UNSUPPORTED from bind.
  * Both modes compute the same layer; they differ in reduction order only.

@@ -424,9 +424,6 @@ gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* wo
   return GSI_OK;
 }
 
-// Can this stack run as one persistent launch?  (batch 1, bf16 basis with a
-// power-of-two rank up to 512, rows that fit the per-CTA buffers, 32-byte
-// aligned weight rows for the 256-bit loads.)
 // Rows of one CTA fit its buffers, and all 16 KB chunks of the group fit the ring of ten
 // slots together (the row pass runs with every chunk of the group resident).
 static bool rows_fit(const gsi_layer* h, int ctas) {
@@ -438,11 +435,15 @@ static bool rows_fit(const gsi_layer* h, int ctas) {
   return (pr + rc - 1) / rc + (orw + rc - 1) / rc <= 10;
 }
 
+// Can this stack run on the persistent kernel?  (one or two tokens per step, bf16 basis
+// with a power-of-two rank up to 512, rows that fit the per-CTA buffers and the ring,
+// 32-byte aligned weight rows for the 256-bit loads.)
 static bool persistent_eligible(const gsi_stack* s, int grid) {
-  if (s->B != 1 || grid <= 0 || grid > kPersistMaxGrid) return false;
+  if (s->B > kPersistMaxTokens || grid <= 0 || grid > kPersistMaxGrid) return false;
   for (const gsi_layer* h : s->groups) {
     const gsi_desc_t& d = h->desc;
     const bool dense = d.flags & GSI_FLAG_DENSE;
+    if (dense && s->B > 1) return false;   // a dense group streams W: once for all tokens (batched GEMM)
     if (d.d % 16) return false;
     if (!rows_fit(h, grid)) return false;
     for (int j = 0; j < d.n_maps; ++j)
@@ -551,7 +552,7 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
       pg.ncta = s->grid;
       pg.phase_len = 1;
       pg.o_rows_w = (gp.O + s->grid - 1) / s->grid;
-      pg.x_step_stride = gp.d;
+      pg.x_step_stride = (long long)s->B * gp.d;
     }
     // pairs of independent groups split the grid
     for (int i = 0; i + 1 < G; ++i) {
@@ -617,7 +618,15 @@ static gsi_status_t stack_enqueue(gsi_stack_t s, bool use_counter, gsi_stream_t 
     p.log_step_stride = G;
     p.status = s->status;
     p.trace = s->trace;
-    return launch_decode_step(p, s->grid, stream) == cudaSuccess ? GSI_OK : GSI_ERR_CUDA;
+    p.n_tokens = s->B;
+    // one launch per token of the step (up to kPersistMaxTokens; larger batches take the
+    // batched kernels): each is a complete decode step of that token, the last one advances
+    for (int t = 0; t < s->B; ++t) {
+      p.token = t;
+      p.advance = t == s->B - 1;
+      if (launch_decode_step(p, s->grid, stream) != cudaSuccess) return GSI_ERR_CUDA;
+    }
+    return GSI_OK;
   }
   for (int i = 0; i < G; ++i) {
     gsi_layer* h = s->groups[i];
@@ -647,7 +656,7 @@ gsi_status_t gsi_stack_step(gsi_stack_t s, gsi_stream_t stream) {
 gsi_status_t gsi_stack_launches_per_step(gsi_stack_t s, int* n_out) {
   if (!s || !n_out || !s->bound) return GSI_ERR_INVALID_ARG;
   if (s->persistent) {
-    *n_out = 1;
+    *n_out = s->B;
     return GSI_OK;
   }
   int n = 0;

@@ -356,7 +356,7 @@ __device__ __forceinline__ bool grid_arrive_wait(unsigned* ctr, unsigned target,
 // ---- F. gated residual: y_rows (+)= W_rows . src (src = r, or x for the dense
 // baseline).  Out of line: most groups skip it.
 __device__ __noinline__ void gated_pass(const PersistGroup& g, const Slab& s, const float* src,
-                                        bool dense, unsigned char* smem) {
+                                        float* y, bool dense, unsigned char* smem) {
   float4* s_rq = reinterpret_cast<float4*>(smem + kOffRq);
   float* s_yacc = reinterpret_cast<float*>(smem + kOffYacc);
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -413,7 +413,7 @@ __device__ __noinline__ void gated_pass(const PersistGroup& g, const Slab& s, co
 #pragma unroll 1
   for (int rw = warp; rw < rows; rw += kNW) {
     if (lane == 0) {
-      float* yp = g.y + s.o0 + rw;
+      float* yp = y + s.o0 + rw;
       *yp = dense ? s_yacc[rw] : (__ldcg(yp) + s_yacc[rw]);
     }
   }
@@ -421,10 +421,11 @@ __device__ __noinline__ void gated_pass(const PersistGroup& g, const Slab& s, co
 
 // Make the next group's activations L2-resident while this group runs (a real
 // pipeline would find them there, written by the preceding operator).
-__device__ __forceinline__ void prefetch_next_x(const PersistGroup& gn, int slot_io, int who = 0) {
+__device__ __forceinline__ void prefetch_next_x(const PersistGroup& gn, int slot_io, int n_tokens,
+                                                int who = 0) {
   if ((int)blockIdx.x == who) {
     const char* xn = reinterpret_cast<const char*>(gn.x + (long long)slot_io * gn.x_step_stride);
-    const int lines = (gn.d * 4 + 127) >> 7;
+    const int lines = (gn.d * 4 * n_tokens + 127) >> 7;
     for (int l = threadIdx.x; l < lines; l += kNC) prefetch_l2(xn + (size_t)l * 128);
   }
 }
@@ -473,7 +474,8 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
       (tid >= kDescWords ? tid - kDescWords : tid);
 
   const Slab s = slab_of(g, lc);
-  const float* x = g.x + (long long)slot_io * g.x_step_stride;
+  const float* x = g.x + (long long)slot_io * g.x_step_stride + (size_t)p.token * g.d;
+  float* const y_tok = g.y + (size_t)p.token * g.O;   // this launch's token
   const bool dense = g.flags & GSI_FLAG_DENSE;
   const bool zeroer = lc == gi_mine % g.ncta;  // this CTA clears the group's counters for the next launch
   int gate = 1, gate_other = 0;
@@ -539,8 +541,8 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
       if (tid < 3) g.bar[2 * tid + (parity ^ 1u)] = 0u;
     }
     csync();
-    if (has_next) prefetch_next_x(g_next, slot_io);
-    if (next_len == 2) prefetch_next_x(desc(gi + len + 1), slot_io, 1);
+    if (has_next) prefetch_next_x(g_next, slot_io, p.n_tokens);
+    if (next_len == 2) prefetch_next_x(desc(gi + len + 1), slot_io, p.n_tokens, 1);
     {  // every thread folds the warp partials in the same order
       float a = 0.f, t = 0.f;
 #pragma unroll
@@ -712,7 +714,7 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
         const int row = row0 + (q.cl >> hold_log2);
         if ((q.cl & ((1 << hold_log2) - 1)) == 0 && row < rows) {
           if (image) {
-            g.y[s.o0 + r_lo + row] = nonfinite ? __int_as_float(0x7fc00000) : dot;
+            y_tok[s.o0 + r_lo + row] = nonfinite ? __int_as_float(0x7fc00000) : dot;
           } else {
             const float rv = s_x[r_lo + row] - dot;
             g.r[s.p0 + r_lo + row] = rv;
@@ -798,7 +800,7 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
       const bool fast = !nonfinite && ((double)t < e2 * (double)sum2);
       gate = fast ? 0 : 1;
       if (lc == 0 && tid == 0) {
-        const size_t at = (size_t)slot_io * p.log_step_stride + gi_mine;
+        const size_t at = ((size_t)slot_io * p.log_step_stride + gi_mine) * p.n_tokens + p.token;
         p.gate_log[at] = (unsigned char)gate;
         if (p.rho_log)
           p.rho_log[at] = nonfinite ? __int_as_float(0x7fc00000) : sqrtf(__fdividef(t, sum2));
@@ -816,11 +818,12 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
     tr.mark(11);
   } else {
     if (zeroer && tid < 3) g.bar[2 * tid + (parity ^ 1u)] = 0u;
-    if (cta == 0 && tid == 0) p.gate_log[(size_t)slot_io * p.log_step_stride + gi] = 1;
+    if (cta == 0 && tid == 0)
+      p.gate_log[((size_t)slot_io * p.log_step_stride + gi) * p.n_tokens + p.token] = 1;
     if (tid < next_len * kDescWords) *desc_dst = desc_word;
     csync();
-    if (has_next) prefetch_next_x(g_next, slot_io);
-    if (next_len == 2) prefetch_next_x(desc(gi + len + 1), slot_io, 1);
+    if (has_next) prefetch_next_x(g_next, slot_io, p.n_tokens);
+    if (next_len == 2) prefetch_next_x(desc(gi + len + 1), slot_io, p.n_tokens, 1);
   }
 
   // ---- F. gated residual of every gated group of the phase, each with the whole grid
@@ -845,7 +848,7 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
     sw.p0 = sw.p1 = 0;
     sw.o0 = min(gg.O, cta * gg.o_rows_w);
     sw.o1 = min(gg.O, sw.o0 + gg.o_rows_w);
-    gated_pass(gg, sw, dense ? rsrc : gg.r, dense, smem);
+    gated_pass(gg, sw, dense ? rsrc : gg.r, gg.y + (size_t)p.token * gg.O, dense, smem);
     // no CTA starts the next group before all have finished this one
     csync();
     tr.mark(12);
@@ -881,7 +884,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
   // last group's exchange, so they may advance now.
   if (blockIdx.x == 0 && threadIdx.x == 0 && ok) {
     *p.epoch = epoch + 1;
-    if (p.use_counter) *p.step = ctx.step + 1;
+    if (p.use_counter && p.advance) *p.step = ctx.step + 1;
   }
 }
 

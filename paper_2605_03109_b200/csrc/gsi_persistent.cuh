@@ -9,6 +9,7 @@ constexpr int kPersistConsumerWarps = 15;  // + 1 producer warp = 16 warps: regi
 constexpr int kPersistMaxPRows = 256;   // basis rows one CTA may own
 constexpr int kPersistMaxORows = 512;   // output rows one CTA may own
 constexpr int kPersistMaxGrid = 256;    // CTAs (exchange-2 slots per group)
+constexpr int kPersistMaxTokens = 2;    // tokens per step served by one launch per token (more: batched kernels)
 constexpr int kAccStride = 16;          // 64-bit words between c accumulators: one per 128-byte line
 
 struct PersistGroup {
@@ -21,8 +22,8 @@ struct PersistGroup {
   float eps;
   unsigned flags;
   float pmax;                        // max |P| (patched in on the device at bind time)
-  const float* x;                    // [n_steps][d]
-  float* y;                          // [O]
+  const float* x;                    // [n_steps][tokens][d]
+  float* y;                          // [tokens][O]
   float* r;                          // [d]
   unsigned long long* acc_c;         // [2][k][kAccStride] fixed-point accumulators, one set per launch parity
   unsigned long long* slot_r;        // [kPersistMaxGrid] (launch tag | partial ||r||^2)
@@ -48,6 +49,8 @@ struct PersistParams {
   int* epoch;                  // device: launches so far (parity of the exchange buffers)
   int n_steps;
   int use_counter;             // 0: I/O slot 0, counter not advanced
+  int n_tokens, token;         // tokens per step, and the one this launch processes (one launch per token)
+  int advance;                 // this launch advances the step counter (the last token's launch)
   unsigned char* gate_log;     // [n_steps][n_groups]
   float* rho_log;              // same shape or nullptr
   int log_step_stride;

@@ -873,3 +873,53 @@ def test_stack_of_batched_groups_on_the_tensor_cores_with_graph_replay():
     assert np.array_equal(stack.gate_log.cpu().numpy(), gate_log)
     for i, y in enumerate(stack.ys):
         assert torch.equal(y.cpu(), ys[i][-1])
+
+
+def test_persistent_two_tokens_per_step_one_launch_per_token():
+    """Steps of two tokens run as two persistent launches (faster per token than the batched
+    kernels at this size): same logs layout as every other path, oracle parity, and the same
+    bits as the single-token stack fed the same tokens one by one."""
+    st = S.config3("23")
+    g = G()
+    n_steps, B = 5, 2
+    layers, xs, mats = [], [], []
+    for gi in range(len(st.groups)):
+        m = S.materialize_group(st, 0, gi, n_steps * B, device="cuda")
+        layers.append(g.Layer(m["W"], m["P"], st.eps, max_tokens=B))
+        xs.append(m["x"].contiguous())
+        mats.append(m)
+    stack = g.Stack(layers, concurrent=[1])
+    stack.bind(xs, n_steps=n_steps)
+    assert stack.is_persistent() and stack.launches_per_step() == 2
+    ys = [[] for _ in mats]
+    for s in range(n_steps):
+        stack.step()
+        torch.cuda.synchronize()
+        for i, y in enumerate(stack.ys):
+            ys[i].append(y.cpu().clone())
+    assert stack.status() == 0
+    gate_log = stack.gate_log.cpu().numpy()               # [steps][groups][2]
+    rho_log = stack.rho_log.cpu().numpy()
+    assert 0 < gate_log.mean() < 1
+    rng = np.random.default_rng(3)
+    for i, m in enumerate(mats):
+        y = torch.cat(ys[i]).numpy()                      # [steps * 2][O]
+        cols, Wsamp, off = [], [], 0
+        for W in m["W"]:
+            r = np.sort(rng.choice(W.shape[0], 40, replace=False))
+            Wsamp.append(W[torch.as_tensor(r, device="cuda")].cpu())
+            cols.append(off + r)
+            off += W.shape[0]
+        compare_group(m["x"].cpu(), m["P"].cpu(), Wsamp, st.eps, y[:, np.concatenate(cols)],
+                      gate_log[:, i, :].reshape(-1), rho_log[:, i, :].reshape(-1))
+    # the same tokens through single-token handles, one per step: bit-identical outputs
+    layers1 = [g.Layer(m["W"], m["P"], st.eps, max_tokens=1) for m in mats]
+    stack1 = g.Stack(layers1, concurrent=[1])
+    stack1.bind(xs, n_steps=n_steps * B)
+    for s in range(n_steps * B):
+        stack1.step()
+        torch.cuda.synchronize()
+        for i, y in enumerate(stack1.ys):
+            assert torch.equal(y.cpu()[0], ys[i][s // B][s % B])
+    assert np.array_equal(stack1.gate_log.cpu().numpy().reshape(n_steps, B, len(mats)).transpose(0, 2, 1),
+                          gate_log)
