@@ -923,3 +923,15 @@ def test_persistent_two_tokens_per_step_one_launch_per_token():
             assert torch.equal(y.cpu()[0], ys[i][s // B][s % B])
     assert np.array_equal(stack1.gate_log.cpu().numpy().reshape(n_steps, B, len(mats)).transpose(0, 2, 1),
                           gate_log)
+
+
+@pytest.mark.parametrize("k", [128, 512])
+def test_persistent_opt_layer_full_size_sampled_rows(k):
+    """One OPT-6.7B-shaped block (four sequential groups, d = 4096 / 16384) at the smallest and the
+    largest rank of the config-4 sweep, in the launch configuration the benchmark times; the
+    oracle evaluates a sample of the output rows of every map."""
+    st = S.config4(k, 0.05, 1.0, steps=8)
+    stack, stats, ys, gate_log = _stack_against_oracle(st, 1, 8, mode=2, sample_rows=32)
+    assert stack.is_persistent() and stack.launches_per_step() == 1
+    rates = [s["gate_rate"] for s in stats]
+    assert 0.0 < np.mean(rates) < 1.0   # sigma scale 1.0 puts the median rho on eps: both paths occur
