@@ -465,6 +465,7 @@ def main():
     e2e = None
     if not args.no_e2e:
         ms_e2e, h2d, d2h = time_host_steps(layers, xs, max(8, args.steps // 8), 3, stream, concurrent)
+        ms_e2e = max_over_ranks(ms_e2e, dist, device)   # every rank takes part: the slowest replica counts
         e2e = {"value": world * spec.batch * 1e3 / ms_e2e, "unit": "tokens/s",
                "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h}
 
