@@ -5,7 +5,8 @@
 // into a ring of shared-memory slots with bulk async copies, in program order
 // and independent of the data-dependent steps (weight addresses never depend
 // on x), so the next group's weights arrive while the current group waits on
-// its cross-CTA exchanges.  Twelve consumer warps run Algorithm 1 per group:
+// its cross-CTA exchanges.  Fifteen consumer warps run Algorithm 1 per group (two
+// consecutive groups declared independent share a phase on two parts of the grid):
 //
 //   pass 1     partial c = P_slab^T x_slab                     (line 1)
 //   exchange 1 c = sum over CTAs, by 64-bit fixed-point atomics whose words
@@ -13,9 +14,9 @@
 //              therefore bit-reproducible)
 //   pass 2     r_slab = x_slab - P_slab c, partial ||r||^2      (lines 2-3)
 //   image      y_rows = W_P,rows c                              (line 5)
-//   exchange 2 every CTA publishes (step tag | partial ||r||^2) in one 64-bit
-//              word with release semantics; every CTA sums the words in a fixed
-//              order and takes the same gate decision           (line 4)
+//   exchange 2 every CTA publishes (launch tag | partial ||r||^2) in one 64-bit
+//              word (relaxed: the tag validates it); every CTA sums the words in a
+//              fixed order and takes the same gate decision     (line 4)
 //   gated      y_rows += W_rows r, W streamed with 256-bit loads, then a grid
 //              barrier                                          (Eq. (3.2))
 //

@@ -114,7 +114,7 @@ def config2() -> StackSpec:
                      0.05, 512, 1, "L2-resident working set")
 
 
-# Noise scales found by bisection on the oracle's gate rate:
+# Noise scales found by bisection on the oracle's gate rate over 4096 tokens per input width:
 # rho ~ sigma*sqrt(d-k)/||z||, tuned so that ~10 % of tokens have rho >= 0.05.
 SIGMA_GPTJ_10 = {4096: 0.010667, 16384: 0.005206}
 
