@@ -358,7 +358,7 @@ def main():
     ap.add_argument("--impl", default="gsi", choices=["gsi", "reference"])
     ap.add_argument("--gate", default="10", choices=["0", "10", "23", "100"],
                     help="target gate rate of the GPT-J workload (percent)")
-    ap.add_argument("--workload", default="gptj", choices=["gptj", "gpt2", "opt", "gptj_b64", "extend"],
+    ap.add_argument("--workload", default="gptj", choices=["gptj", "gpt2", "opt", "gptj_b64", "cfg1", "cfg1_fast", "extend"],
                     help="gptj: the headline (config 3); gpt2: config 2; opt: config 4 sweep point "
                          "(--k --eps --sigma-scale); gptj_b64: config 5 (--outlier)")
     ap.add_argument("--k", type=int, default=256)
@@ -370,6 +370,9 @@ def main():
     ap.add_argument("--static-projection", action="store_true",
                     help="negative control (Section 4.1, static projection): the gate is computed and "
                          "logged but W r is never added, so the step costs the fast path only")
+    ap.add_argument("--per-stage", action="store_true",
+                    help="force the per-stage / batched kernels (stack mode 1) instead of the "
+                         "persistent launch")
     ap.add_argument("--no-concurrent", action="store_true",
                     help="run the groups of a block strictly one after the other even where the "
                          "workload marks two of them as parallel branches")
@@ -395,6 +398,10 @@ def main():
         spec = S.config3(args.gate)
     elif args.workload == "gpt2":
         spec = S.config2()
+    elif args.workload == "cfg1":
+        spec = S.config1()
+    elif args.workload == "cfg1_fast":
+        spec = S.config1_fast()
     elif args.workload == "opt":
         spec = S.config4(args.k, args.eps, args.sigma_scale)
     else:
@@ -425,7 +432,7 @@ def main():
     n_steps = min(spec.steps, max(args.steps, 1))
     layers, dense_layers, xs, keep = build_workload(spec, device, n_steps, args.static_projection)
     concurrent = [] if args.no_concurrent else spec.concurrent_groups()
-    stack = G.Stack(layers, concurrent=concurrent)
+    stack = G.Stack(layers, concurrent=concurrent, mode=1 if args.per_stage else 0)
     stack.bind(xs, n_steps=n_steps)
     if args.profile:
         for _ in range(args.warmup + args.steps):
