@@ -68,6 +68,7 @@ struct Misc {
   float sum2;
   int nonfinite;
   float sr;
+  int deposits;   // warps that have handed in their ||r||^2 partial in this phase
 };
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
@@ -535,6 +536,7 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
       s_vals[warp * 2 + 0] = amax;
       s_vals[warp * 2 + 1] = sum2;
     }
+    if (tid == 0) misc->deposits = 0;
     if (zeroer) {  // clear what the NEXT launch will accumulate into
 #pragma unroll 1
       for (int j = tid; j < k; j += kNC)
@@ -685,6 +687,31 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
     }
     tr.mark(7);
     float sr = 0.f;
+    // ---- E (first half). exchange 2 is published as soon as the residual rows are done, by
+    //      the warp that hands in the last partial, so that its latency runs under the image
+    //      rows.  The word carries its own launch tag: no fence is needed for the decision.
+    // A pair shares the first group's slot array: word cta is this CTA's partial of its own
+    // group, words kPairSumSlot + u carry ||x||^2 of group u for the other half of the grid.
+    auto deposit = [&]() {
+      sr = warp_sum(sr);
+      if (lane == 0) {
+        volatile float* part = s_red;
+        part[warp] = sr;
+        __threadfence_block();
+        if (atomicAdd(&misc->deposits, 1) == kNW - 1) {
+          __threadfence_block();
+          float t = 0.f;   // fixed order: the sum does not depend on who came last
+#pragma unroll
+          for (int w = 0; w < kNW; ++w) t += part[w];
+          st_relaxed_u64(gA.slot_r + cta,
+                         ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(t));
+          if (len == 2 && lc == 0)
+            st_relaxed_u64(gA.slot_r + kPairSumSlot + (second ? 1 : 0),
+                           ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(sum2));
+        }
+      }
+    };
+    bool deposited = false;
     if (ok) {
       // work items: lane groups take eight rows at a time, first of the basis slab, then of
       // the image slab (rows per chunk are a multiple of 8, so an item stays inside a chunk);
@@ -722,7 +749,13 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
             sr = fmaf(rv, rv, sr);
           }
         }
+        // basis items come first: once none is left for this warp, its partial is final
+        if (!deposited && item - q.sub + lanegroups >= itemsP) {
+          deposit();
+          deposited = true;
+        }
       }
+      if (!deposited) deposit();
       __syncwarp();
       if (lane == 0) {
 #pragma unroll 1
@@ -733,26 +766,8 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
     tr.mark(8);
     if (!ok && !*abort) fail(p, misc);
     n += pchunks + ochunks;
-    sr = warp_sum(sr);
-    if (lane == 0) s_red[warp] = sr;
-    csync();
-    if (*abort) return false;
 
-    // ---- E. exchange 2: publish, collect, decide.  The word carries its own
-    //      launch tag, so no fence is needed for the gate decision itself.
-    // A pair shares the first group's slot array: word cta is this CTA's partial of its own
-    // group, words kPairSumSlot + u carry ||x||^2 of group u for the other half of the grid.
-    if (tid == 0) {
-      float t = 0.f;
-#pragma unroll
-      for (int w = 0; w < kNW; ++w) t += s_red[w];
-      st_relaxed_u64(gA.slot_r + cta,
-                     ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(t));
-      if (len == 2 && lc == 0)
-        st_relaxed_u64(gA.slot_r + kPairSumSlot + (second ? 1 : 0),
-                       ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(sum2));
-    }
-    tr.mark(9);
+    // ---- E (second half). exchange 2: collect, decide.
     if (warp == 0) {
       // one warp polls all words (lane l owns words l, l+32, ...); each word is
       // validated by its launch tag
