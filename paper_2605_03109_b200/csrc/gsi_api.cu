@@ -121,6 +121,7 @@ struct gsi_stack {
   int mode;                 // 0 auto, 1 generic kernels, 2 persistent kernel required
   bool persistent;          // the persistent kernel is in use
   int grid;                 // CTAs of the persistent kernel (= SMs)
+  bool has_pairs;           // some phase of the persistent schedule holds two groups
   PersistGroup* dev_groups; // device table
   std::vector<PersistGroup> host_groups;
   std::vector<const float*> host_pmax_ptrs;
@@ -571,10 +572,12 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
       pg.p_rows = (pg.d + pg.ncta - 1) / pg.ncta;
       pg.o_rows = (pg.O + pg.ncta - 1) / pg.ncta;
     }
+    s->has_pairs = false;
     for (int i = 0; i < G;) {   // length of the phase after each group's
       const int len = s->host_groups[i].phase_len;
       const int nxt = i + len < G ? s->host_groups[i + len].phase_len : 0;
       for (int j = 0; j < len; ++j) s->host_groups[i + j].next_len = nxt;
+      if (len == 2) s->has_pairs = true;
       i += len;
     }
     const float** dev_ptrs = reinterpret_cast<const float**>(
@@ -624,7 +627,7 @@ static gsi_status_t stack_enqueue(gsi_stack_t s, bool use_counter, gsi_stream_t 
     for (int t = 0; t < s->B; ++t) {
       p.token = t;
       p.advance = t == s->B - 1;
-      if (launch_decode_step(p, s->grid, stream) != cudaSuccess) return GSI_ERR_CUDA;
+      if (launch_decode_step(p, s->grid, s->has_pairs, stream) != cudaSuccess) return GSI_ERR_CUDA;
     }
     return GSI_OK;
   }
