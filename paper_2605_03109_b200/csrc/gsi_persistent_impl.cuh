@@ -873,13 +873,17 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
     sw.o0 = min(gg.O, cta * gg.o_rows_w);
     sw.o1 = min(gg.O, sw.o0 + gg.o_rows_w);
     gated_pass(gg, sw, dense ? rsrc : gg.r, gg.y + (size_t)p.token * gg.O, dense, smem);
-    // no CTA starts the next group before all have finished this one
     csync();
     tr.mark(12);
-    if (tid == 0) grid_arrive_wait(gg.bar + parity, (unsigned)G, p, misc);
-    csync();
-    tr.mark(13);
-    if (*abort) return false;
+    // A dense group has no exchange: a grid barrier keeps the groups of a dense stack in
+    // model order.  After a gated residual none is needed: no CTA passes exchange 1 of the
+    // next phase before every CTA has posted its partial there, which it does after this.
+    if (dense) {
+      if (tid == 0) grid_arrive_wait(gg.bar + parity, (unsigned)G, p, misc);
+      csync();
+      tr.mark(13);
+      if (*abort) return false;
+    }
   }
   return true;
 }
