@@ -327,15 +327,21 @@ __device__ __forceinline__ void dot8(const uint4* tile, const float* s_c, const 
     const float4 cb = *reinterpret_cast<const float4*>(s_c + cv * 8 + 4);
     const unsigned long long c0 = pack2(ca.x, ca.y), c1 = pack2(ca.z, ca.w);
     const unsigned long long c2 = pack2(cb.x, cb.y), c3 = pack2(cb.z, cb.w);
+    // rows past the end of the slab read the last row again (no branch: the eight loads
+    // and FMA chains interleave); the caller drops their results
 #pragma unroll
-    for (int i = 0; i < 8; ++i) {
-      if (row0 + i < rows) {
-        const uint4 w = tile[(size_t)(row0 + i) * q.KV + cv];
-        fma2(acc[i], bf16x2_to_f32x2(w.x), c0);
-        fma2(acc[i], bf16x2_to_f32x2(w.y), c1);
-        fma2(acc[i], bf16x2_to_f32x2(w.z), c2);
-        fma2(acc[i], bf16x2_to_f32x2(w.w), c3);
+    for (int h = 0; h < 8; h += 4) {   // four rows at a time: eight would not fit the registers
+      uint4 w[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) w[i] = tile[max(min(row0 + h + i, rows - 1), 0) * q.KV + cv];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        fma2(acc[h + i], bf16x2_to_f32x2(w[i].x), c0);
+        fma2(acc[h + i], bf16x2_to_f32x2(w[i].y), c1);
+        fma2(acc[h + i], bf16x2_to_f32x2(w[i].z), c2);
+        fma2(acc[h + i], bf16x2_to_f32x2(w[i].w), c3);
       }
+      asm volatile("" ::: "memory");
     }
   }
 #pragma unroll
