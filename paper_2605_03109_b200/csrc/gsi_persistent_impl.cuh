@@ -725,14 +725,23 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
         }
       }
     };
-    bool deposited = false;
+    // work items: lane groups take eight rows at a time, first of the basis slab, then of
+    // the image slab (rows per chunk are a multiple of 8, so an item stays inside a chunk);
+    // only items with rows are enumerated, rounded up to a whole warp of lane groups
+    const int itemsP = (prow + 7) >> 3, n_live = itemsP + ((orow + 7) >> 3);
+    const int n_items = ((n_live + (1 << rpp_log2) - 1) >> rpp_log2) << rpp_log2;
+    const int lanegroups = kNW << rpp_log2;          // lane groups in the CTA
+    // The warps that hold basis items run them alone: the others hand in an empty partial
+    // and start their image items only when the last basis item is done (named barrier 2:
+    // they wait, the basis warps only arrive), so the partial is published as early as
+    // possible.  Every warp takes part exactly once per phase, whatever `ok` says.
+    const bool basis_warp = (warp << rpp_log2) < itemsP;
+    bool deposited = !basis_warp;
+    if (!basis_warp) {
+      deposit();
+      asm volatile("bar.sync 2, %0;" ::"n"(kNC) : "memory");
+    }
     if (ok) {
-      // work items: lane groups take eight rows at a time, first of the basis slab, then of
-      // the image slab (rows per chunk are a multiple of 8, so an item stays inside a chunk);
-      // only items with rows are enumerated, rounded up to a whole warp of lane groups
-      const int itemsP = (prow + 7) >> 3, n_live = itemsP + ((orow + 7) >> 3);
-      const int n_items = ((n_live + (1 << rpp_log2) - 1) >> rpp_log2) << rpp_log2;
-      const int lanegroups = kNW << rpp_log2;          // lane groups in the CTA
       int released = 0;  // chunks this warp has already given back to the producer
 #pragma unroll 1
       for (int item = (warp << rpp_log2) + q.sub; item < n_items; item += lanegroups) {
@@ -767,15 +776,19 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
         if (!deposited && item - q.sub + lanegroups >= itemsP) {
           deposit();
           deposited = true;
+          asm volatile("bar.arrive 2, %0;" ::"n"(kNC) : "memory");
         }
       }
-      if (!deposited) deposit();
       __syncwarp();
       if (lane == 0) {
 #pragma unroll 1
         for (; released < pchunks + ochunks; ++released)
           mbar_arrive(&empty[(n_p0 + released) % kSlots]);
       }
+    }
+    if (!deposited) {   // only after a failed wait: keep the barrier count whole
+      deposit();
+      asm volatile("bar.arrive 2, %0;" ::"n"(kNC) : "memory");
     }
     tr.mark(8);
     if (!ok && !*abort) fail(p, misc);
