@@ -268,9 +268,13 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io_host_array,
  * and the MLP down projection), so the persistent kernel may run their
  * projections, gates and images at the same time on two parts of the grid
  * (Algorithm 1 itself is unchanged; a gated residual still streams W with the
- * whole grid).  Off by default; a group belongs to at most one pair; ignored
- * outside persistent mode and when the rows of either group do not fit its
- * share of the grid.  Takes effect at the next gsi_stack_bind.
+ * whole grid).  Outside persistent mode (per-stage and batched kernels) the
+ * second group of a pair is enqueued on a stream of the stack's own, forked
+ * from and joined to the caller's stream by events, so the two chains of
+ * launches run side by side (and a stream capture records a fork and a join).
+ * Off by default; a group belongs to at most one pair; in persistent mode a
+ * pair whose rows do not fit its share of the grid runs one group after the
+ * other.  Takes effect at the next gsi_stack_bind.
  */
 gsi_status_t gsi_stack_set_concurrent(gsi_stack_t s, int first_group, int enable);
 

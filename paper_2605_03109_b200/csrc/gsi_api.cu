@@ -139,6 +139,15 @@ struct gsi_stack {
   bool bound;
   int seek_value;
   cudaStream_t last_stream;
+  // per-stage / batched path: the second group of a concurrent pair runs on a stream of
+  // the stack's own, forked from and joined to the caller's stream by events
+  cudaStream_t aux = nullptr;
+  cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  ~gsi_stack() {
+    if (ev_fork) cudaEventDestroy(ev_fork);
+    if (ev_join) cudaEventDestroy(ev_join);
+    if (aux) cudaStreamDestroy(aux);
+  }
 };
 
 extern "C" {
@@ -512,6 +521,14 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
     s->persistent = coop && persistent_eligible(s, sms);
     if (s->mode == 2 && !s->persistent) return GSI_ERR_UNSUPPORTED;
   }
+  if (!s->persistent && !s->aux) {
+    bool any = false;
+    for (char c : s->pair_first) any = any || c;
+    if (any && (cudaStreamCreateWithFlags(&s->aux, cudaStreamNonBlocking) != cudaSuccess ||
+                cudaEventCreateWithFlags(&s->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+                cudaEventCreateWithFlags(&s->ev_join, cudaEventDisableTiming) != cudaSuccess))
+      return GSI_ERR_CUDA;
+  }
   if (s->persistent) {
     // The cross-CTA exchange state of every group (accumulators, tagged words, arrival
     // counters) is tied to THIS stack's launch counter: start both from zero.  A handle
@@ -631,7 +648,7 @@ static gsi_status_t stack_enqueue(gsi_stack_t s, bool use_counter, gsi_stream_t 
     }
     return GSI_OK;
   }
-  for (int i = 0; i < G; ++i) {
+  auto enqueue_group = [&](int i, cudaStream_t st) -> bool {
     gsi_layer* h = s->groups[i];
     IoRef io{};
     io.x = s->io[i].x;
@@ -642,9 +659,25 @@ static gsi_status_t stack_enqueue(gsi_stack_t s, bool use_counter, gsi_stream_t 
     io.n_steps = s->n_steps;
     io.x_step_stride = (long long)s->B * h->desc.d;
     io.log_step_stride = (long long)G * s->B;
-    h->last_stream = stream;
-    if (launch_generic_forward(h->gp, h->has_tm ? &h->tm : nullptr, io, s->B, stream, nullptr) != cudaSuccess)
-      return GSI_ERR_CUDA;
+    h->last_stream = stream;   // the join below puts the pair's work in the caller's stream order
+    return launch_generic_forward(h->gp, h->has_tm ? &h->tm : nullptr, io, s->B, st, nullptr) ==
+           cudaSuccess;
+  };
+  for (int i = 0; i < G; ++i) {
+    if (s->aux && i + 1 < G && s->pair_first[i]) {
+      // groups i and i+1 do not read each other's outputs: two chains of dependent launches
+      // side by side (under stream capture this becomes a fork and a join in the graph)
+      if (cudaEventRecord(s->ev_fork, stream) != cudaSuccess ||
+          cudaStreamWaitEvent(s->aux, s->ev_fork, 0) != cudaSuccess)
+        return GSI_ERR_CUDA;
+      if (!enqueue_group(i, stream) || !enqueue_group(i + 1, s->aux)) return GSI_ERR_CUDA;
+      if (cudaEventRecord(s->ev_join, s->aux) != cudaSuccess ||
+          cudaStreamWaitEvent(stream, s->ev_join, 0) != cudaSuccess)
+        return GSI_ERR_CUDA;
+      ++i;
+      continue;
+    }
+    if (!enqueue_group(i, stream)) return GSI_ERR_CUDA;
   }
   if (use_counter && launch_advance_step(s->step, stream) != cudaSuccess) return GSI_ERR_CUDA;
   return GSI_OK;

@@ -823,10 +823,12 @@ def test_set_concurrent_validates_its_arguments_and_falls_back_when_rows_do_not_
     compare_group(x, P, Ws, 0.05, outs[1][0][:, 512:768], outs[1][1][:, 2, 0], None)
 
 
-def test_stack_of_batched_groups_on_the_tensor_cores_with_graph_replay():
-    """A chain of two groups stepped with 8 tokens per step: every contraction runs on tcgen05
+@pytest.mark.parametrize("concurrent", [(), (0,)])
+def test_stack_of_batched_groups_on_the_tensor_cores_with_graph_replay(concurrent):
+    """Two groups stepped with 8 tokens per step: every contraction runs on tcgen05
     (programmatic dependent launches inside a captured graph); steps and graph replays agree
-    with the oracle and with each other."""
+    with the oracle and with each other.  Declared concurrent, the second group runs on the
+    stack's own stream, forked and joined by events (a fork and a join in the captured graph)."""
     g = G()
     d, k, B, n_steps = 1024, 128, 8, 3
     groups = []
@@ -841,7 +843,7 @@ def test_stack_of_batched_groups_on_the_tensor_cores_with_graph_replay():
         x[::5] = torch.randn((len(range(0, n_steps * B, 5)), d), generator=gen)
         groups.append((x.contiguous(), P, Ws))
     layers = [g.Layer([W.cuda() for W in Ws], P.cuda(), 0.05, max_tokens=B) for _, P, Ws in groups]
-    stack = g.Stack(layers)
+    stack = g.Stack(layers, concurrent=concurrent)
     stack.bind([x.cuda() for x, _, _ in groups], n_steps=n_steps)
     assert not stack.is_persistent() and stack.launches_per_step() == 2 * 6 + 1
     ys = [[] for _ in groups]
