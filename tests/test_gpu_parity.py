@@ -382,6 +382,19 @@ def test_persistent_gptj_parallel_branches_share_a_phase():
         assert np.array_equal(cat(ya), cat(yc))
 
 
+def test_persistent_gptj_every_group_gated_back_to_back():
+    """Every group of every step gated (both members of each pair, and the groups before
+    and after them): gated residuals follow each other with no grid barrier in between,
+    only the next phase's exchange; paired and sequential schedules agree with the oracle
+    and with each other."""
+    st = S.config3("100")
+    for pairs in ([1, 4], []):
+        stack, stats, ys, gate_log = _stack_against_oracle(st, 2, 6, mode=2, sample_rows=40,
+                                                           concurrent=pairs)
+        assert stack.is_persistent()
+        assert gate_log.min() == 1
+
+
 def test_persistent_matches_generic_kernels_and_is_reproducible():
     st = S.config2()
     a, _, ys_a, gate_a = _stack_against_oracle(st, 1, 8, mode=2)
