@@ -122,6 +122,7 @@ struct gsi_stack {
   bool persistent;          // the persistent kernel is in use
   int grid;                 // CTAs of the persistent kernel (= SMs)
   bool has_pairs;           // some phase of the persistent schedule holds two groups
+  int common_k;             // rank shared by every gated group of the persistent schedule, or 0
   PersistGroup* dev_groups; // device table
   std::vector<PersistGroup> host_groups;
   std::vector<const float*> host_pmax_ptrs;
@@ -590,6 +591,13 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
       pg.o_rows = (pg.O + pg.ncta - 1) / pg.ncta;
     }
     s->has_pairs = false;
+    s->common_k = -1;
+    for (int i = 0; i < G; ++i) {
+      if (s->host_groups[i].flags & GSI_FLAG_DENSE) continue;
+      const int k = s->host_groups[i].k;
+      s->common_k = s->common_k < 0 || s->common_k == k ? k : 0;
+    }
+    if (s->common_k < 0) s->common_k = 0;
     for (int i = 0; i < G;) {   // length of the phase after each group's
       const int len = s->host_groups[i].phase_len;
       const int nxt = i + len < G ? s->host_groups[i + len].phase_len : 0;
@@ -644,7 +652,7 @@ static gsi_status_t stack_enqueue(gsi_stack_t s, bool use_counter, gsi_stream_t 
     for (int t = 0; t < s->B; ++t) {
       p.token = t;
       p.advance = t == s->B - 1;
-      if (launch_decode_step(p, s->grid, s->has_pairs, stream) != cudaSuccess) return GSI_ERR_CUDA;
+      if (launch_decode_step(p, s->grid, s->has_pairs, s->common_k, stream) != cudaSuccess) return GSI_ERR_CUDA;
     }
     return GSI_OK;
   }

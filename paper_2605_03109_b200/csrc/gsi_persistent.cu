@@ -43,11 +43,16 @@ cudaError_t launch_abs_max_bf16(const void* p, size_t n, float* out, cudaStream_
   return cudaGetLastError();
 }
 
-// the build that knows pairs of concurrent groups lives in its own translation unit
+// the other builds of the kernel live in translation units of their own
 cudaError_t launch_decode_step_pairs(const PersistParams& p, int grid, cudaStream_t st);
+cudaError_t launch_decode_step_k256(const PersistParams& p, int grid, cudaStream_t st);
+cudaError_t launch_decode_step_pairs_k256(const PersistParams& p, int grid, cudaStream_t st);
 
-cudaError_t launch_decode_step(const PersistParams& p, int grid, bool pairs, cudaStream_t st) {
-  return pairs ? launch_decode_step_pairs(p, grid, st) : launch_decode_step_t<false>(p, grid, st);
+cudaError_t launch_decode_step(const PersistParams& p, int grid, bool pairs, int common_k,
+                               cudaStream_t st) {
+  if (common_k == 256)
+    return pairs ? launch_decode_step_pairs_k256(p, grid, st) : launch_decode_step_k256(p, grid, st);
+  return pairs ? launch_decode_step_pairs(p, grid, st) : launch_decode_step_t<false, 0>(p, grid, st);
 }
 
 }  // namespace gsi

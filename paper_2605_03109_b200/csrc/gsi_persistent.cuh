@@ -60,8 +60,10 @@ struct PersistParams {
 
 int persist_smem_bytes();
 int persist_threads();
-// pairs: some phase of the table holds two groups (selects the build of the kernel that knows them)
-cudaError_t launch_decode_step(const PersistParams& p, int grid, bool pairs, cudaStream_t st);
+// pairs: some phase of the table holds two groups; common_k: the rank shared by every gated
+// group of the table, or 0 (both select a build of the kernel)
+cudaError_t launch_decode_step(const PersistParams& p, int grid, bool pairs, int common_k,
+                               cudaStream_t st);
 cudaError_t launch_abs_max_bf16(const void* p, size_t n, float* out, cudaStream_t st);
 cudaError_t launch_patch_pmax(PersistGroup* groups, const float* const* pmax_ptrs, int n,
                               cudaStream_t st);

@@ -23,8 +23,8 @@
 // Every wait is bounded; a wait that gives up records GSI_ERR_TIMEOUT in the
 // status word, the CTA drains its copies in flight and returns.
 //
-// This header holds the kernel; it is compiled twice, in two translation units (one per
-// value of kPairs): stacks without concurrent groups run a build without the pair logic.
+// This header holds the kernel; every build of it (with or without the pair logic, for any
+// rank or for rank 256 only) is compiled in a translation unit of its own.
 #pragma once
 
 #include <cstdio>
@@ -445,8 +445,10 @@ __device__ __forceinline__ void prefetch_next_x(const PersistGroup& gn, int slot
 
 // One group.  Returns false when the CTA must stop (a wait gave up).
 // kPairs = false compiles the pair logic out: stacks without concurrent groups run a smaller
-// loop (the per-phase code has to stay resident in the instruction cache).
-template <bool kPairs>
+// loop (the per-phase code has to stay resident in the instruction cache).  kK != 0 is a
+// build for stacks whose groups all have rank kK (shifts, strides and loop bounds become
+// constants); kK = 0 reads the rank from the descriptor.
+template <bool kPairs, int kK>
 __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* misc, Ctx& ctx,
                             int gi) {
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + kOffBar);
@@ -498,7 +500,7 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
   const float* rsrc = x;
 
   if (!dense) {
-    const int k = g.k;
+    const int k = kK ? kK : g.k;   // a build for one rank folds the whole lane geometry
     Geo q;
     q.KV = k >> 3;
     q.lpr_log2 = q.KV >= 32 ? 5 : 31 - __clz(q.KV);
@@ -907,7 +909,7 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
   return true;
 }
 
-template <bool kPairs>
+template <bool kPairs, int kK>
 __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc) {
   Ctx ctx;
   ctx.step = p.use_counter ? *p.step : 0;
@@ -927,7 +929,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
   bool ok = true;
   ctx.len = 1;
 #pragma unroll 1
-  for (int gi = 0; gi < p.n_groups && ok; gi += ctx.len) ok = group_phase<kPairs>(p, smem, misc, ctx, gi);
+  for (int gi = 0; gi < p.n_groups && ok; gi += ctx.len) ok = group_phase<kPairs, kK>(p, smem, misc, ctx, gi);
   // Every CTA read the counters at its start and has since taken part in the
   // last group's exchange, so they may advance now.
   if (blockIdx.x == 0 && threadIdx.x == 0 && ok) {
@@ -936,7 +938,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
   }
 }
 
-template <bool kPairs>
+template <bool kPairs, int kK>
 __global__ void __launch_bounds__(kThreadsP, 1) k_decode_step(PersistParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + kOffBar);
@@ -955,16 +957,16 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_decode_step(PersistParams p) {
     if (threadIdx.x == kNC) producer(p, smem, misc);
     return;
   }
-  consumer<kPairs>(p, smem, misc);
+  consumer<kPairs, kK>(p, smem, misc);
 }
 
-template <bool kPairs>
+template <bool kPairs, int kK>
 cudaError_t launch_decode_step_t(const PersistParams& p, int grid, cudaStream_t st) {
   static bool configured[64] = {};   // per device: the attribute belongs to the device's function
   int dev = 0;
   if (cudaGetDevice(&dev) != cudaSuccess) return cudaErrorInvalidDevice;
   if (dev < 0 || dev >= 64 || !configured[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(k_decode_step<kPairs>,
+    cudaError_t e = cudaFuncSetAttribute(k_decode_step<kPairs, kK>,
                                          cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemBytes);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) configured[dev] = true;
@@ -973,7 +975,7 @@ cudaError_t launch_decode_step_t(const PersistParams& p, int grid, cudaStream_t 
   void* args[] = {&pp};
   // cooperative launch: all CTAs are guaranteed co-resident, which the
   // cross-CTA exchanges rely on
-  cudaError_t e = cudaLaunchCooperativeKernel((void*)k_decode_step<kPairs>, dim3(grid),
+  cudaError_t e = cudaLaunchCooperativeKernel((void*)k_decode_step<kPairs, kK>, dim3(grid),
                                               dim3(kThreadsP), args, kSmemBytes, st);
   if (e != cudaSuccess && getenv("GSI_VERBOSE"))
     fprintf(stderr, "gsi: persistent launch failed: %s\n", cudaGetErrorString(e));
