@@ -45,14 +45,25 @@ cudaError_t launch_abs_max_bf16(const void* p, size_t n, float* out, cudaStream_
 
 // the other builds of the kernel live in translation units of their own
 cudaError_t launch_decode_step_pairs(const PersistParams& p, int grid, cudaStream_t st);
+cudaError_t launch_decode_step_k128(const PersistParams& p, int grid, cudaStream_t st);
+cudaError_t launch_decode_step_pairs_k128(const PersistParams& p, int grid, cudaStream_t st);
 cudaError_t launch_decode_step_k256(const PersistParams& p, int grid, cudaStream_t st);
 cudaError_t launch_decode_step_pairs_k256(const PersistParams& p, int grid, cudaStream_t st);
+cudaError_t launch_decode_step_k512(const PersistParams& p, int grid, cudaStream_t st);
+cudaError_t launch_decode_step_pairs_k512(const PersistParams& p, int grid, cudaStream_t st);
 
 cudaError_t launch_decode_step(const PersistParams& p, int grid, bool pairs, int common_k,
                                cudaStream_t st) {
-  if (common_k == 256)
-    return pairs ? launch_decode_step_pairs_k256(p, grid, st) : launch_decode_step_k256(p, grid, st);
-  return pairs ? launch_decode_step_pairs(p, grid, st) : launch_decode_step_t<false, 0>(p, grid, st);
+  switch (common_k) {
+    case 128:
+      return pairs ? launch_decode_step_pairs_k128(p, grid, st) : launch_decode_step_k128(p, grid, st);
+    case 256:
+      return pairs ? launch_decode_step_pairs_k256(p, grid, st) : launch_decode_step_k256(p, grid, st);
+    case 512:
+      return pairs ? launch_decode_step_pairs_k512(p, grid, st) : launch_decode_step_k512(p, grid, st);
+    default:
+      return pairs ? launch_decode_step_pairs(p, grid, st) : launch_decode_step_t<false, 0>(p, grid, st);
+  }
 }
 
 }  // namespace gsi

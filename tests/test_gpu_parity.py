@@ -442,6 +442,38 @@ def test_persistent_other_ranks_and_flags(k):
         assert np.max(np.abs(torch.cat(y1).numpy() - ref)) <= 1e-5 * np.max(np.abs(ref))
 
 
+def test_persistent_groups_of_different_rank_in_one_stack():
+    """Groups of rank 128 and 256 in one persistent stack (the build of the kernel that reads
+    the rank from the descriptor; stacks of one rank get a build with that rank compiled in)."""
+    g = G()
+    d, n_steps = 2048, 6
+    layers, xs, mats = [], [], []
+    for i, (k, d_out) in enumerate([(128, (1024,)), (256, (512, 512)), (128, (768,))]):
+        q = S.gen_basis(d, k, 700 + i)
+        P = S.store_basis(q)
+        Ws = [S.gen_weight(o, d, 710 + 10 * i + j) for j, o in enumerate(d_out)]
+        pt = S.gen_true_basis(q, k // 2, k // 2, 740 + i)
+        x, _ = S.gen_activations(pt, n_steps, 0.002, 0.0,
+                                 dict(z=750 + i, noise=760 + i, outlier_mask=0, outlier_values=0))
+        x[i::3] = torch.randn((len(range(i, n_steps, 3)), d), generator=torch.Generator().manual_seed(770 + i))
+        layers.append(g.Layer([W.cuda() for W in Ws], P.cuda(), 0.05, max_tokens=1))
+        xs.append(x.cuda().contiguous())
+        mats.append((x, P, Ws))
+    stack = g.Stack(layers, mode=2)
+    stack.bind(xs, n_steps=n_steps)
+    ys = [[] for _ in mats]
+    for s in range(n_steps):
+        stack.step()
+        torch.cuda.synchronize()
+        for i, y in enumerate(stack.ys):
+            ys[i].append(y.cpu().clone())
+    assert stack.status() == 0 and stack.is_persistent()
+    for i, (x, P, Ws) in enumerate(mats):
+        gate = stack.gate_log[:, i, 0].cpu().numpy()
+        compare_group(x, P, Ws, 0.05, torch.cat(ys[i]).numpy(), gate, stack.rho_log[:, i, 0].cpu().numpy())
+        assert 0 < gate.sum() < n_steps
+
+
 def test_persistent_nonfinite_token():
     g = G()
     x, P, Ws = make_small(256, 64, (64,), 3, seed=41)
