@@ -26,7 +26,7 @@ struct PersistGroup {
   float* y;                          // [tokens][O]
   float* r;                          // [d]
   unsigned long long* acc_c;         // [2][k][kAccStride] fixed-point accumulators, one set per launch parity
-  unsigned long long* slot_r;        // [kPersistMaxGrid] (launch tag | partial ||r||^2)
+  unsigned long long* slot_r;        // exchange 2: 32-bit words [grid + 2] (launch parity in the sign bit | partial ||r||^2)
   unsigned* bar;                     // [6] arrival counters by launch parity: [0..1] after, [2..3] before the gated residual, [4..5] exchange 2
   int p_rows, o_rows;                // rows per CTA of P and of the images (ceil(rows / ncta))
   long long x_step_stride;
@@ -40,7 +40,7 @@ struct PersistGroup {
   int o_rows_w;                      // W rows per CTA of the gated residual: ceil(O / grid)
 };
 
-constexpr int kPairSumSlot = 254;    // slot_r[254 + u]: ||x||^2 of group u of a pair (slots < grid hold ||r||^2 partials)
+constexpr int kPairSumSlot = 254;    // pairs need grid + 2 exchange-2 words in 256: word grid + u is ||x||^2 of group u of a pair
 
 struct PersistParams {
   const PersistGroup* groups;  // device

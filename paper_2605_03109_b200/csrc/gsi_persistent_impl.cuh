@@ -13,10 +13,14 @@
 //              also count arrivals (no separate flag, no fence, order-free and
 //              therefore bit-reproducible)
 //   pass 2     r_slab = x_slab - P_slab c, partial ||r||^2      (lines 2-3)
+//   exchange 2 every CTA publishes its partial ||r||^2 as one 32-bit word, the sign
+//              bit carrying the parity of the launch (relaxed store: the word
+//              validates itself, every launch rewrites every word), as soon as its
+//              residual rows are done ...
 //   image      y_rows = W_P,rows c                              (line 5)
-//   exchange 2 every CTA publishes (launch tag | partial ||r||^2) in one 64-bit
-//              word (relaxed: the tag validates it); every CTA sums the words in a
-//              fixed order and takes the same gate decision     (line 4)
+//              ... and collects the words after its image rows, so the exchange
+//              runs under them; every CTA sums the words in a fixed order and
+//              takes the same gate decision                     (line 4)
 //   gated      y_rows += W_rows r, W streamed with 256-bit loads, then a grid
 //              barrier                                          (Eq. (3.2))
 //
@@ -128,6 +132,9 @@ __device__ __forceinline__ void red_add_u64(unsigned long long* p, unsigned long
 }
 __device__ __forceinline__ void st_relaxed_u64(unsigned long long* p, unsigned long long v) {
   asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
+}
+__device__ __forceinline__ void st_relaxed_u32(unsigned* p, unsigned v) {
+  asm volatile("st.relaxed.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ unsigned ld_relaxed_u32(const unsigned* p) {
   unsigned v;
@@ -705,9 +712,13 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
     float sr = 0.f;
     // ---- E (first half). exchange 2 is published as soon as the residual rows are done, by
     //      the warp that hands in the last partial, so that its latency runs under the image
-    //      rows.  The word carries its own launch tag: no fence is needed for the decision.
+    //      rows.  A word is the partial (non-negative, or NaN) with the parity of the launch
+    //      in its sign bit: the arrays start as zeros, the first launch writes sign 1, and
+    //      every launch rewrites every word, so a word of this launch cannot be mistaken for
+    //      the previous one's and no fence is needed for the decision.  148 partials are
+    //      five 128-byte lines that every CTA reads.
     // A pair shares the first group's slot array: word cta is this CTA's partial of its own
-    // group, words kPairSumSlot + u carry ||x||^2 of group u for the other half of the grid.
+    // group, words G + u carry ||x||^2 of group u for the other half of the grid.
     auto deposit = [&]() {
       sr = warp_sum(sr);
       if (lane == 0) {
@@ -719,11 +730,11 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
           float t = 0.f;   // fixed order: the sum does not depend on who came last
 #pragma unroll
           for (int w = 0; w < kNW; ++w) t += part[w];
-          st_relaxed_u64(gA.slot_r + cta,
-                         ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(t));
+          unsigned* slots = reinterpret_cast<unsigned*>(gA.slot_r);
+          st_relaxed_u32(slots + cta, (__float_as_uint(t) & 0x7fffffffu) | (tag << 31));
           if (len == 2 && lc == 0)
-            st_relaxed_u64(gA.slot_r + kPairSumSlot + (second ? 1 : 0),
-                           ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(sum2));
+            st_relaxed_u32(slots + G + (second ? 1 : 0),
+                           (__float_as_uint(sum2) & 0x7fffffffu) | (tag << 31));
         }
       }
     };
@@ -799,7 +810,7 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
     // ---- E (second half). exchange 2: collect, decide.
     if (warp == 0) {
       // one warp polls all words (lane l owns words l, l+32, ...); each word is
-      // validated by its launch tag
+      // validated by the launch parity in its sign bit
       float vals[8];
       unsigned it = 0;
       bool done = false;
@@ -809,10 +820,10 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
         for (int i = 0; i < 8; ++i) {
           const int t = lane + 32 * i;
           vals[i] = 0.f;
-          if (t < G || (len == 2 && t >= kPairSumSlot)) {
-            const unsigned long long w = ld_relaxed_u64(gA.slot_r + t);
-            all = all && ((unsigned)(w >> 32) == tag);
-            vals[i] = __uint_as_float((unsigned)w);
+          if (t < G + (len == 2 ? 2 : 0)) {
+            const unsigned w = ld_relaxed_u32(reinterpret_cast<const unsigned*>(gA.slot_r) + t);
+            all = all && ((w >> 31) == (tag & 1u));
+            vals[i] = __uint_as_float(w & 0x7fffffffu);
           }
         }
         done = __all_sync(0xffffffffu, all);
@@ -852,7 +863,7 @@ __device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* m
       }
       if (len == 2) {  // the partner's decision, from its partial sums and its ||x||^2
         const PersistGroup& go = second ? gA : gB;
-        const float to = second ? tA : tB, s2o = s_vals[kPairSumSlot + (second ? 0 : 1)];
+        const float to = second ? tA : tB, s2o = s_vals[G + (second ? 0 : 1)];
         const double e2o = (double)go.eps * (double)go.eps;
         const bool finite_o = s2o - s2o == 0.f;
         const bool fast_o = finite_o && ((double)to < e2o * (double)s2o);
