@@ -137,10 +137,11 @@ __device__ __forceinline__ void decide_gate_last_block(const GroupParams& g, con
   __syncthreads();
   if (!*s_last) return;
   __threadfence();
+  __shared__ unsigned char s_gate[GSI_MAX_TOKENS];   // the decisions, for the list of gated tokens
   unsigned char* gate = io.gate + (long long)slot * io.log_step_stride;
   float* rho = io.rho ? io.rho + (long long)slot * io.log_step_stride : g.rho_scratch;
   // L adjacent lanes share a token: each sums a contiguous range of parts in order (loads
-  // issued sixteen parts at a time), then the L sums are combined by a butterfly, so the
+  // issued thirty-two parts at a time), then the L sums are combined by a butterfly, so the
   // result depends on n_tokens and the block size only through L and is reproducible.
   int L = 1;
   while (2 * L <= 32 && 2 * L * n_tokens <= (int)blockDim.x) L *= 2;
@@ -152,13 +153,13 @@ __device__ __forceinline__ void decide_gate_last_block(const GroupParams& g, con
     double sr = 0.0, sx = 0.0;
     if (live) {
       const float2* np = reinterpret_cast<const float2*>(normpart) + t;
-      for (int p = p0; p < p1; p += 16) {
-        float2 v[16];
+      for (int p = p0; p < p1; p += 32) {
+        float2 v[32];
 #pragma unroll
-        for (int u = 0; u < 16; ++u)
+        for (int u = 0; u < 32; ++u)
           v[u] = (p + u < p1) ? __ldcg(np + (size_t)(p + u) * g.B) : make_float2(0.f, 0.f);
 #pragma unroll
-        for (int u = 0; u < 16; ++u) {
+        for (int u = 0; u < 32; ++u) {
           sr += (double)v[u].x;
           sx += (double)v[u].y;
         }
@@ -172,6 +173,7 @@ __device__ __forceinline__ void decide_gate_last_block(const GroupParams& g, con
       const double nr = sqrt(sr), nx = sqrt(sx);
       const bool fast = nr < (double)g.eps * nx;  // false for NaN and for x = 0
       gate[t] = fast ? 0 : 1;
+      s_gate[t] = fast ? 0 : 1;
       rho[t] = (float)(nr / nx);
     }
   }
@@ -180,7 +182,7 @@ __device__ __forceinline__ void decide_gate_last_block(const GroupParams& g, con
     int n = 0;
     if (!(g.flags & GSI_FLAG_STATIC_PROJECTION)) {
       for (int t = 0; t < n_tokens; ++t)
-        if (gate[t]) g.fired[n++] = t;
+        if (s_gate[t]) g.fired[n++] = t;
     }
     *g.n_fired = n;
     *g.counter = 0u;
