@@ -301,9 +301,9 @@ gsi_status_t gsi_stack_is_persistent(gsi_stack_t s, int* out);
  * section of the per-group pipeline:
  *   0 loads of x           1 statistics of x     2 wait for basis slab
  *   3 pass 1               4 partial-c atomics   5 wait for c
- *   6 pass 2               7 wait for image slab 8 image rows
- *   9 publish ||r||^2      10 wait for all ||r||^2   11 gate decision
- *   12 gated residual      13 grid barrier after it
+ *   6 (unused)             7 wait for image slab 8 residual rows, publishing ||r||^2, image rows
+ *   9 (unused)             10 wait for all ||r||^2   11 gate decision
+ *   12 gated residual      13 grid barrier after it (dense groups only)
  * The caller clears and reads the counters.  Applies from the next step.
  */
 #define GSI_TRACE_SECTIONS 16
@@ -332,6 +332,13 @@ gsi_status_t gsi_stack_step_host(gsi_stack_t s, const float* const* x_host_array
                                  float* const* y_host_array, unsigned char* gate_host,
                                  gsi_stream_t stream);
 
+/*
+ * Synchronises the stack's last stream and returns the device status word (GSI_OK,
+ * or GSI_ERR_TIMEOUT if a bounded device-side wait gave up).  After a time-out the
+ * outputs of that step are undefined and the cross-CTA exchange state of the
+ * persistent kernel is stale: bind the stack again (gsi_stack_bind clears it)
+ * before stepping further.
+ */
 gsi_status_t gsi_stack_get_status(gsi_stack_t s, int* device_status);
 gsi_status_t gsi_stack_destroy(gsi_stack_t s);
 
