@@ -531,10 +531,12 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
       return GSI_ERR_CUDA;
   }
   if (s->persistent) {
-    // The cross-CTA exchange state of every group (accumulators, tagged words, arrival
+    // The cross-CTA exchange state of every group (accumulators, exchange words, arrival
     // counters) is tied to THIS stack's launch counter: start both from zero.  A handle
     // can therefore serve only one bound stack at a time.
-    if (cudaMemsetAsync(s->epoch, 0, sizeof(int), stream) != cudaSuccess) return GSI_ERR_CUDA;
+    if (cudaMemsetAsync(s->epoch, 0, sizeof(int), stream) != cudaSuccess ||
+        cudaMemsetAsync(s->status, 0, sizeof(int), stream) != cudaSuccess)   // a fresh start also after a time-out
+      return GSI_ERR_CUDA;
     for (int i = 0; i < G; ++i) {
       const gsi_layer* h = s->groups[i];
       if (cudaMemsetAsync(h->ws + h->lay.pk_acc, 0, h->lay.tc_rb - h->lay.pk_acc, stream) !=
