@@ -130,6 +130,13 @@ __global__ void __launch_bounds__(256) k_reduce_split3_c(GroupParams g, int n_to
       const float* p = g.cpart3 + (size_t)slot * g.k + j;
       const size_t stride = (size_t)g.B * g.k;
       int s = 0;
+      for (; s + 32 <= g.proj_splits; s += 32) {   // thirty-two partials in flight, summed in order
+        float u[32];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) u[i] = p[(size_t)(s + i) * stride];
+#pragma unroll
+        for (int i = 0; i < 32; ++i) v += u[i];
+      }
       for (; s + 8 <= g.proj_splits; s += 8) {
         float u[8];
 #pragma unroll
