@@ -71,8 +71,10 @@ __device__ __forceinline__ void store_terms(const float (&v)[8], bool live, uint
 }
 
 __global__ void __launch_bounds__(256) k_split3_x(GroupParams g, IoRef io, int n_tokens) {
-  pdl_launch_dependents();
+  // first kernel of the chain: wait first, so that nothing of the chain (its successors
+  // request weight tiles before their own waits) runs beside an earlier call's kernels
   pdl_wait();   // xb may still be read by the previous call's projection
+  pdl_launch_dependents();
   const int slot = blockIdx.y, n_rows = rows3(n_tokens);
   const bool live = slot < n_tokens;
   const float* x = io.x + (long long)io_slot(io) * io.x_step_stride + (size_t)slot * g.d;

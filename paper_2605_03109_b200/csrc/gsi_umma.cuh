@@ -154,21 +154,34 @@ __device__ __forceinline__ bool tile_mma(unsigned char* smem_raw, const CUtensor
   asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory");
   const uint32_t tmem = *tmem_slot;
   *tmem_out = tmem;
-  pdl_wait();   // the operands may come from the previous kernel of the stream
   const uint32_t stage_bytes = (uint32_t)(kABytes + N * kTK * 2);
+  // The A operand is a weight tile (set-up data, never written by the kernels of a call):
+  // its first kStages boxes are requested before the wait on the previous kernel, whose
+  // output only the B operand can be.  (The first kernel of every chain of dependent
+  // launches waits BEFORE it lets its successor start, so nothing launched ahead of the
+  // chain can still be writing weights.)
+  if (tid == 0) {
+    for (int i = 0; i < nloc && i < kStages; ++i) {
+      mbar_expect_tx(&bar_full[i], stage_bytes);
+      tma_load_2d(s32(smem + i * C::kStageBytes), map_a, (kb0 + i) * kTK, a_row0, &bar_full[i]);
+    }
+  }
+  pdl_wait();   // the B operand may come from the previous kernel of the stream
 
   if (warp == 0) {
     if (lane == 0) {   // producer
       for (int i = 0; i < nloc; ++i) {
         const int stage = i % kStages;
-        if (i >= kStages && !mbar_wait(&bar_empty[stage], ((i / kStages) - 1) & 1)) {
-          *s_fail = 1;
-          break;
-        }
-        mbar_expect_tx(&bar_full[stage], stage_bytes);
         const uint32_t sa = s32(smem + stage * C::kStageBytes), sb = sa + kABytes;
         const int x = (kb0 + i) * kTK;
-        tma_load_2d(sa, map_a, x, a_row0, &bar_full[stage]);
+        if (i >= kStages) {
+          if (!mbar_wait(&bar_empty[stage], ((i / kStages) - 1) & 1)) {
+            *s_fail = 1;
+            break;
+          }
+          mbar_expect_tx(&bar_full[stage], stage_bytes);
+          tma_load_2d(sa, map_a, x, a_row0, &bar_full[stage]);
+        }
         for (int j = 0; j < N / kBBox; ++j)
           tma_load_2d(sb + j * (kBBox * kTK * 2), map_b, x, b_row0 + j * kBBox, &bar_full[stage]);
       }
