@@ -25,8 +25,13 @@ constexpr int kMaxN3 = 192;          // 3 terms x 64 tokens
 constexpr int kTmemCols3 = 256;      // power of two >= kMaxN3
 using Cfg3 = Cfg<kStages3, kMaxN3>;
 constexpr int kSmem3 = Cfg3::kSmem;  // 4 x (16 + 24) KB + slack
-constexpr int kStagesRI = 2;         // residual / image: K = k is short; two blocks per SM instead
+// residual / image: K = k is short (four 64-wide blocks at k = 256).  Up to 32 tokens the B
+// operand is small enough for four stages with two blocks per SM, so every weight box of a
+// tile is requested before the wait on the previous kernel; beyond, two stages.
+constexpr int kStagesRI = 2, kStagesRIs = 4;
+constexpr int kMaxN3s = 96, kTmemCols3s = 128;   // 3 terms x 32 tokens
 constexpr int kSmemRI = Cfg<kStagesRI, kMaxN3>::kSmem;
+constexpr int kSmemRIs = Cfg<kStagesRIs, kMaxN3s>::kSmem;
 
 __device__ __forceinline__ uint16_t bf16_bits(float v) {
   const __nv_bfloat16 h = __float2bfloat16_rn(v);
@@ -164,6 +169,7 @@ __global__ void __launch_bounds__(256) k_reduce_split3_c(GroupParams g, int n_to
 //                         r = x - P c -> bf16 rows of rb, the partial norms of the tile,
 //                         and in the block that finishes last the gate
 //   blocks [n_resid, ..)  tile of W_P, all tokens: y = W_P c
+template <int kStagesT, int kMaxRows, int kTmemColsT>
 __global__ void __launch_bounds__(kThreads, 2)
 k_resid_image_tc(GroupParams g, const __grid_constant__ TmaMaps tm, IoRef io, int n_tokens, int rs) {
   extern __shared__ unsigned char smem_raw[];
@@ -192,7 +198,7 @@ k_resid_image_tc(GroupParams g, const __grid_constant__ TmaMaps tm, IoRef io, in
   bool ok = true;
   if (q_lo < q_hi) {   // block-uniform
     const int n_rows = min(48 * (q_hi - q_lo), rows3(n_tokens) - 48 * q_lo);
-    ok = tile_mma<kStagesRI, kMaxN3, kTmemCols3>(smem_raw, image ? &tm.wp : &tm.p, tile * kTM, &tm.cb,
+    ok = tile_mma<kStagesT, kMaxRows, kTmemColsT>(smem_raw, image ? &tm.wp : &tm.p, tile * kTM, &tm.cb,
                                                 48 * q_lo, n_rows, 0, g.k / kTK, &tmem);
     if (!ok && threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
     const uint32_t tl = tmem + ((uint32_t)(warp * 32) << 16);
@@ -223,7 +229,7 @@ k_resid_image_tc(GroupParams g, const __grid_constant__ TmaMaps tm, IoRef io, in
         xv[tt] = xn[tt];
       }
     }
-    tile_release<kTmemCols3>(tmem);
+    tile_release<kTmemColsT>(tmem);
   }
   if (image) return;
   __syncthreads();
@@ -280,9 +286,12 @@ cudaError_t launch_front_tc(const GroupParams& g, const TmaMaps& tm, const IoRef
                             cudaStream_t st, int* n_launches) {
   cudaError_t e;
   if ((e = cudaFuncSetAttribute(k_proj_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmem3)) != cudaSuccess ||
-      (e = cudaFuncSetAttribute(k_resid_image_tc, cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemRI)) !=
-          cudaSuccess)
+      (e = cudaFuncSetAttribute(k_resid_image_tc<kStagesRI, kMaxN3, kTmemCols3>,
+                                cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemRI)) != cudaSuccess ||
+      (e = cudaFuncSetAttribute(k_resid_image_tc<kStagesRIs, kMaxN3s, kTmemCols3s>,
+                                cudaFuncAttributeMaxDynamicSharedMemorySize, kSmemRIs)) != cudaSuccess)
     return e;
+  const bool small = term_rows(n_tokens) <= kMaxN3s;
   const int slots = (front_rows(n_tokens) + 2) / 3;   // token slots covering every operand row
   const int nq = (n_tokens + 15) / 16, tiles = g.d / kTM;
   int rs = tiles <= 37 ? 4 : tiles <= 148 ? 2 : 1;   // token ranges per residual tile (measured: 4 for all is slower)
@@ -294,8 +303,12 @@ cudaError_t launch_front_tc(const GroupParams& g, const TmaMaps& tm, const IoRef
       (e = launch_pdl(k_proj_tc, dim3((g.k / kTM) * g.proj_splits), dim3(kThreads), kSmem3, st, g, tm,
                       n_tokens)) != cudaSuccess ||
       (e = launch_pdl(k_reduce_split3_c, dim3(slots), dim3(256), 0, st, g, n_tokens)) != cudaSuccess ||
-      (e = launch_pdl(k_resid_image_tc, dim3((g.d / kTM) * rs + g.O / kTM), dim3(kThreads), kSmemRI, st, g,
-                      tm, io, n_tokens, rs)) != cudaSuccess)
+      (e = small ? launch_pdl(k_resid_image_tc<kStagesRIs, kMaxN3s, kTmemCols3s>,
+                              dim3((g.d / kTM) * rs + g.O / kTM), dim3(kThreads), kSmemRIs, st, g, tm, io,
+                              n_tokens, rs)
+                 : launch_pdl(k_resid_image_tc<kStagesRI, kMaxN3, kTmemCols3>,
+                              dim3((g.d / kTM) * rs + g.O / kTM), dim3(kThreads), kSmemRI, st, g, tm, io,
+                              n_tokens, rs)) != cudaSuccess)
     return e;
   if (n_launches) *n_launches += 4;
   return cudaGetLastError();
