@@ -27,6 +27,7 @@ using namespace umma;
 constexpr int kStages = 4;   // 4 x 24 KB, two blocks per SM (8 stages x 1 block and 3 x 3 measured slower)
 constexpr int kMaxN = 64;
 constexpr int kTmemCols = 64;
+constexpr int kSpeculateTokens = 16;   // tokens per call from which W tiles are requested before the gate is known
 using TcCfg = Cfg<kStages, kMaxN>;
 constexpr int kThreadsTc = kThreads;
 constexpr int kTcSmem = TcCfg::kSmem;
@@ -51,23 +52,21 @@ __global__ void __launch_bounds__(kThreadsTc, 2)
 k_residual_gemm_tc(GroupParams g, const __grid_constant__ TmaMaps tm, int min_fired, int splits,
                    int mapped, int n_tokens) {
   pdl_launch_dependents();
-  pdl_wait();   // the fired list comes from the kernel before
-  const int n_fired = *g.n_fired;
-  if (n_fired < min_fired) return;            // nothing gated, or the CUDA-core GEMV takes the few
+  // With many tokens per call some token is gated nearly always: the W tiles are then
+  // requested before the fired list of the kernel before is known (mapped operand rows only:
+  // their number does not depend on the list), and the block backs out if nobody fired.
+  const bool speculate = mapped && n_tokens >= kSpeculateTokens;
+  int n_fired = 0;
+  if (!speculate) {
+    pdl_wait();   // the fired list comes from the kernel before
+    n_fired = *g.n_fired;
+    if (n_fired < min_fired) return;          // nothing gated, or the CUDA-core GEMV takes the few
+  }
   const int n_cols = mapped ? n_tokens : n_fired;
   const int N = (n_cols + 15) & ~15;          // 16..64
 
   extern __shared__ unsigned char smem_raw[];
   __shared__ unsigned long long s_mask;       // columns to write out
-  if (threadIdx.x == 0) {
-    unsigned long long m = 0ull;
-    if (mapped) {
-      for (int n = 0; n < n_fired; ++n) m |= 1ull << g.fired[n];
-    } else {
-      m = n_fired >= 64 ? ~0ull : ((1ull << n_fired) - 1ull);
-    }
-    s_mask = m;
-  }
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int tile = blockIdx.x / splits, split = blockIdx.x % splits;
   const int row0 = tile * kTM;                 // first row of the concatenated maps
@@ -78,9 +77,26 @@ k_residual_gemm_tc(GroupParams g, const __grid_constant__ TmaMaps tm, int min_fi
   const int nloc = kb1 - kb0;
 
   uint32_t tmem;
+  bool skipped = false;
   const bool ok = tile_mma<kStages, kMaxN, kTmemCols>(smem_raw, &tm.w[j], row0 - g.off[j], &tm.rb, 0, N,
-                                                      kb0, nloc, &tmem);
-  if (!ok) {
+                                                      kb0, nloc, &tmem, speculate ? g.n_fired : nullptr,
+                                                      min_fired, &skipped);
+  if (!skipped) {   // past the wait on the kernel before: the fired list is there
+    if (threadIdx.x == 0) {
+      n_fired = *g.n_fired;
+      unsigned long long m = 0ull;
+      if (mapped) {
+        for (int n = 0; n < n_fired; ++n) m |= 1ull << g.fired[n];
+      } else {
+        m = n_fired >= 64 ? ~0ull : ((1ull << n_fired) - 1ull);
+      }
+      s_mask = m;
+    }
+    __syncthreads();
+  }
+  if (skipped) {
+    // nothing to write
+  } else if (!ok) {
     if (threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
   } else if (nloc > 0) {
     // warp w owns tensor-memory lanes 32w..32w+31 = rows row0+32w+lane; 16 columns per load

@@ -47,6 +47,13 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
   asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s32(b)), "r"(bytes)
                : "memory");
 }
+__device__ __forceinline__ void mbar_expect_tx_only(uint64_t* b, uint32_t bytes) {   // no arrival
+  asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(s32(b)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* b) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s32(b)) : "memory");
+}
 __device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -119,10 +126,15 @@ __device__ __forceinline__ void tmem_ld_wait() {
 // column = B row); the return value, the same for every thread, is false when a wait ran
 // out of time.  With nloc == 0 nothing is accumulated and D is undefined.  The caller
 // must end with tile_release<kTmemCols>(*tmem_out).
+// run_count / run_min: if run_count is given, it is read after the wait on the previous
+// kernel and the contraction runs only if *run_count >= run_min; otherwise the weight boxes
+// already requested are allowed to land, *skipped is set and the function returns true.
 template <int kStages, int kBRows, int kTmemCols>
 __device__ __forceinline__ bool tile_mma(unsigned char* smem_raw, const CUtensorMap* map_a,
                                          int a_row0, const CUtensorMap* map_b, int b_row0, int N,
-                                         int kb0, int nloc, uint32_t* tmem_out) {
+                                         int kb0, int nloc, uint32_t* tmem_out,
+                                         const int* run_count = nullptr, int run_min = 0,
+                                         bool* skipped = nullptr) {
   using C = Cfg<kStages, kBRows>;
   unsigned char* smem = reinterpret_cast<unsigned char*>(
       (reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~(uintptr_t)1023);
@@ -162,11 +174,22 @@ __device__ __forceinline__ bool tile_mma(unsigned char* smem_raw, const CUtensor
   // chain can still be writing weights.)
   if (tid == 0) {
     for (int i = 0; i < nloc && i < kStages; ++i) {
-      mbar_expect_tx(&bar_full[i], stage_bytes);
+      mbar_expect_tx_only(&bar_full[i], (uint32_t)kABytes);   // the arrival comes with the B boxes
       tma_load_2d(s32(smem + i * C::kStageBytes), map_a, (kb0 + i) * kTK, a_row0, &bar_full[i]);
     }
   }
   pdl_wait();   // the B operand may come from the previous kernel of the stream
+  if (run_count && *run_count < run_min) {   // the same answer for every thread
+    if (tid == 0) {
+      for (int i = 0; i < nloc && i < kStages; ++i) {
+        mbar_arrive(&bar_full[i]);
+        (void)mbar_wait(&bar_full[i], 0);   // the requested boxes land before the block exits
+      }
+    }
+    __syncthreads();
+    if (skipped) *skipped = true;
+    return true;
+  }
 
   if (warp == 0) {
     if (lane == 0) {   // producer
@@ -181,6 +204,8 @@ __device__ __forceinline__ bool tile_mma(unsigned char* smem_raw, const CUtensor
           }
           mbar_expect_tx(&bar_full[stage], stage_bytes);
           tma_load_2d(sa, map_a, x, a_row0, &bar_full[stage]);
+        } else {
+          mbar_expect_tx(&bar_full[stage], stage_bytes - (uint32_t)kABytes);   // A is on its way
         }
         for (int j = 0; j < N / kBBox; ++j)
           tma_load_2d(sb + j * (kBBox * kTK * 2), map_b, x, b_row0 + j * kBBox, &bar_full[stage]);
