@@ -266,6 +266,7 @@ int front_proj_splits(int d, int k) {
   const int tiles = k / kTM, nkb = d / kTK;
   int s = 148 / tiles;
   if (s > nkb / 2) s = nkb / 2;
+  if (s > 32) s = 32;   // more partials cost the reduction more than they save the projection (measured)
   if (s < 1) s = 1;
   return s;
 }
