@@ -1,4 +1,5 @@
-// A build of the persistent decode-step kernel (see gsi_persistent_impl.cuh): two independent groups may share a phase, every group of rank 256.
+// A build of the persistent decode-step kernel (see gsi_persistent_impl.cuh):
+// two independent groups may share a phase, every group of rank 256.
 // A translation unit of its own: each build of the kernel is compiled separately.
 #include "gsi_persistent_impl.cuh"
 
