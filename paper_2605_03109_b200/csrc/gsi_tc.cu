@@ -139,6 +139,9 @@ __global__ void __launch_bounds__(256) k_add_partials(GroupParams g, IoRef io, i
 // row per token), which makes this the strongest dense comparator the tile routine offers:
 // the stage size and occupancy of the gated-residual GEMM, no pack by a fired list.
 __global__ void __launch_bounds__(256) k_pack_x_bf16(GroupParams g, IoRef io, int n_tokens) {
+  // first kernel of the chain: wait first (rb may still be read by the previous call's GEMM,
+  // and the GEMM after this kernel requests weight tiles before its own wait)
+  pdl_wait();
   pdl_launch_dependents();
   const int row = blockIdx.y;   // operand row = token; rows up to the next multiple of 16 are zero
   const float* x = io.x + (long long)io_slot(io) * io.x_step_stride + (size_t)row * g.d;
