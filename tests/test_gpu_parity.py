@@ -610,6 +610,55 @@ def test_tensor_core_residual_gemm_gptj_shape_sampled_rows():
                   gate.cpu().numpy(), rho.cpu().numpy())
 
 
+def test_batched_gptj_block_full_size_sampled_rows_in_the_benchmarks_schedule():
+    """Config 5 as the benchmark runs it: one GPT-J block (the wide q,k,v,fc group, attn_out and
+    the d = 16384 proj group) at 64 tokens per step, attn_out and proj declared concurrent (two
+    streams), every contraction on the tensor cores; two steps, the second replayed from a
+    captured graph; the oracle evaluates a sample of the output rows of every map."""
+    g = G()
+    st = S.config5(0.10, batch=64, steps=2)
+    B, n_steps = 64, 2
+    rng = np.random.default_rng(11)
+    layers, xs, mats = [], [], []
+    for gi, spec in enumerate(st.groups):
+        m = S.materialize_group(st, 0, gi, n_steps * B, device="cuda")
+        layers.append(g.Layer(m["W"], m["P"], st.eps, max_tokens=B))
+        xs.append(m["x"].contiguous())
+        mats.append(m)
+    stack = g.Stack(layers, concurrent=st.concurrent_groups()[:1])
+    stack.bind(xs, n_steps=n_steps)
+    assert not stack.is_persistent()
+    stream = torch.cuda.Stream()
+    ys = [[] for _ in mats]
+    with torch.cuda.stream(stream):
+        stack.step(stream)
+        stream.synchronize()
+        for i, y in enumerate(stack.ys):
+            ys[i].append(y.cpu().clone())
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph, stream=stream):
+            stack.step(stream)
+        stack.seek(1, stream)
+        graph.replay()
+        stream.synchronize()
+        for i, y in enumerate(stack.ys):
+            ys[i].append(y.cpu().clone())
+    assert stack.status() == 0
+    gate_log = stack.gate_log.cpu().numpy()   # [steps][groups][B]
+    rho_log = stack.rho_log.cpu().numpy()
+    for i, m in enumerate(mats):
+        y = torch.cat(ys[i]).numpy()
+        cols, Wsamp, off = [], [], 0
+        for W in m["W"]:
+            r = np.sort(rng.choice(W.shape[0], 32, replace=False))
+            Wsamp.append(W[torch.as_tensor(r, device="cuda")].cpu())
+            cols.append(off + r)
+            off += W.shape[0]
+        compare_group(m["x"].cpu(), m["P"].cpu(), Wsamp, st.eps, y[:, np.concatenate(cols)],
+                      gate_log[:, i, :].reshape(-1), rho_log[:, i, :].reshape(-1))
+    assert 0.03 < gate_log.mean() < 0.2
+
+
 def test_rebinding_a_second_stack_over_the_same_handles():
     """gsi_stack_bind resets the exchange state of its handles, so a new stack over
     handles that already ran in another stack works (the older stack must not be
