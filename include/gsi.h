@@ -163,8 +163,9 @@ gsi_status_t gsi_forward_host(gsi_handle_t h, const float* x_host, int n_tokens,
  * someone else's stream capture is open, a latency-critical path that may not
  * enter the allocator.  Such a caller cannot provide the workspace gsi_create
  * wants.  Here the scratch (coefficients, residual, partial sums, fired-token
- * list) lives in a fixed array inside the library: about 2.5 MB that every GPU
- * which loads the library holds until the process exits.
+ * list) lives in a fixed array inside the library: about 1.5 MB that every GPU
+ * which loads the library holds until the process exits.  No device status word can
+ * be read back for this entry point (its kernels contain no bounded wait).
  *
  * The caller passes everything else: W_host_array (HOST array of n_maps DEVICE
  * pointers, W_j [d_out_j][d] bf16), d_out (HOST array), P [d][k], and W_P, the
@@ -243,8 +244,10 @@ size_t gsi_stack_workspace_bytes(int n_groups);
 
 /* groups_host_array: HOST array of n_groups handles in execution order; all
  * must have the same max_tokens.  The handles must outlive the stack.  A handle
- * may belong to several stacks, but only the stack bound LAST may be stepped:
- * gsi_stack_bind resets the handles' cross-CTA exchange state. */
+ * may appear only once in a stack (GSI_ERR_INVALID_ARG otherwise: its scratch and
+ * exchange state serve one use per step).  It may belong to several stacks, but
+ * only the stack bound LAST may be stepped: gsi_stack_bind resets the handles'
+ * cross-CTA exchange state. */
 gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups_host_array,
                               void* workspace, size_t workspace_bytes,
                               gsi_stream_t stream, gsi_stack_t* out);
@@ -283,13 +286,23 @@ gsi_status_t gsi_stack_set_concurrent(gsi_stack_t s, int first_group, int enable
  *   0 (default)  the persistent kernel, one launch per token of the step, when
  *                every group qualifies (one or two tokens per step, no dense
  *                group in a two-token stack, bf16 basis with k in
- *                {64,128,256,512}, d a multiple of 16, 32-byte aligned W, rows
- *                that fit the per-CTA buffers), else the per-stage / batched kernels;
+ *                {64,128,256,512}, d a multiple of 16, rows that fit the
+ *                per-CTA buffers), else the per-stage / batched kernels;
  *   1            always the per-stage kernels;
  *   2            the persistent launch or GSI_ERR_UNSUPPORTED from bind.
  * Both modes compute the same layer; they differ in reduction order only.
  */
 gsi_status_t gsi_stack_set_mode(gsi_stack_t s, int mode);
+
+/*
+ * Polls a cross-CTA wait of the persistent kernel (the exchange of a phase, the
+ * arrival counters) may take before it gives up, records GSI_ERR_TIMEOUT in the
+ * status word and lets every CTA drain its copies in flight and return; 0
+ * restores the default (2^22, about a second).  Waits inside a CTA (its own
+ * copies in flight) keep their own, larger limit.  Applies from the next step.
+ * A very small value makes the time-out path testable without hanging anything.
+ */
+gsi_status_t gsi_stack_set_spin_limit(gsi_stack_t s, unsigned polls);
 
 /* 1 if the bound stack runs as one persistent launch per step. */
 gsi_status_t gsi_stack_is_persistent(gsi_stack_t s, int* out);
@@ -298,12 +311,11 @@ gsi_status_t gsi_stack_is_persistent(gsi_stack_t s, int* out);
  * Tracing.  `cycles` is a DEVICE array [n_CTAs][GSI_TRACE_SECTIONS] of 64-bit
  * counters (n_CTAs = SM count; NULL switches tracing off).  While set, thread 0
  * of every CTA of the persistent launch adds the SM cycles it spends in each
- * section of the per-group pipeline:
- *   0 loads of x           1 statistics of x     2 wait for basis slab
- *   3 pass 1               4 partial-c atomics   5 wait for c
- *   6 (unused)             7 wait for image slab 8 residual rows, publishing ||r||^2, image rows
- *   9 (unused)             10 wait for all ||r||^2   11 gate decision
- *   12 gated residual      13 grid barrier after it (dense groups only)
+ * section of the per-phase pipeline:
+ *   0 statistics of x, descriptors      1 wait for basis slab     2 pass 1
+ *   3 collect max|x|                    4 fixed-point atomics     5 wait for the sums, gate of the previous phase
+ *   6 residual rows                     7 gated residuals (W stream)
+ *   8 wait for image slab               9 image rows              10 dense group (W stream, barrier)
  * The caller clears and reads the counters.  Applies from the next step.
  */
 #define GSI_TRACE_SECTIONS 16

@@ -21,7 +21,7 @@ EXPORTED = [
     "gsi_status_string", "gsi_build_image", "gsi_workspace_bytes", "gsi_create",
     "gsi_forward", "gsi_forward_n", "gsi_forward_host", "gsi_forward_static", "gsi_extend_basis", "gsi_get_image", "gsi_get_status",
     "gsi_destroy", "gsi_stack_workspace_bytes", "gsi_stack_create", "gsi_stack_bind",
-    "gsi_stack_set_mode", "gsi_stack_set_concurrent", "gsi_stack_is_persistent", "gsi_stack_set_trace", "gsi_stack_seek", "gsi_stack_step", "gsi_stack_launches_per_step",
+    "gsi_stack_set_mode", "gsi_stack_set_concurrent", "gsi_stack_is_persistent", "gsi_stack_set_trace", "gsi_stack_set_spin_limit", "gsi_stack_seek", "gsi_stack_step", "gsi_stack_launches_per_step",
     "gsi_stack_step_host", "gsi_stack_get_status", "gsi_stack_destroy",
 ]
 
@@ -73,6 +73,7 @@ def _load():
     l.gsi_stack_set_concurrent.argtypes = [vp, i, i]
     l.gsi_stack_is_persistent.argtypes = [vp, C.POINTER(i)]
     l.gsi_stack_set_trace.argtypes = [vp, vp]
+    l.gsi_stack_set_spin_limit.argtypes = [vp, C.c_uint]
     l.gsi_stack_seek.argtypes = [vp, i, vp]
     l.gsi_stack_step.argtypes = [vp, vp]
     l.gsi_stack_launches_per_step.argtypes = [vp, C.POINTER(i)]
@@ -313,6 +314,10 @@ class Stack:
         _check(lib.gsi_stack_set_trace(self.handle, self.trace.data_ptr() if on else None),
                "gsi_stack_set_trace")
         return self.trace
+
+    def set_spin_limit(self, polls: int):
+        """Polls a cross-CTA wait of the persistent kernel may take (0 = default)."""
+        _check(lib.gsi_stack_set_spin_limit(self.handle, int(polls)), "gsi_stack_set_spin_limit")
 
     def seek(self, step: int, stream=None):
         _check(lib.gsi_stack_seek(self.handle, int(step), _stream_ptr(stream)), "gsi_stack_seek")

@@ -78,8 +78,8 @@ Layout make_layout_ws(const gsi_desc_t* d) {
   L.y_stage = take(B * (size_t)O * 4);
   L.gate_stage = take(B);
   L.rho_stage = take(B * 4);
-  L.pk_acc = take(2 * k * 8 * kAccStride);          // persistent kernel: c accumulators
-  L.pk_slot = take((size_t)kPersistMaxGrid * 8);    // persistent kernel: ||r||^2 words
+  L.pk_acc = take(2 * (k + 2) * 8 * kAccStride);    // persistent kernel: accumulators of c, ||x||^2, ||r||^2
+  L.pk_slot = take((size_t)kPersistMaxGrid * 8);    // persistent kernel: tagged max|x| words, published ||x||^2
   // tensor-core kernels: batched handles only
   const bool tc_any = d->max_tokens >= kFrontMinTokens && d->d % 64 == 0 && tc_shapes_ok(d);
   const bool tc = !dense && tc_any;
@@ -124,7 +124,10 @@ struct gsi_stack {
   bool has_pairs;           // some phase of the persistent schedule holds two groups
   int common_k;             // rank shared by every gated group of the persistent schedule, or 0
   PersistGroup* dev_groups; // device table
+  char* dev_tmaps;          // device: GSI_MAX_MAPS tensor maps per group (the persistent kernel's W stream)
+  unsigned spin_limit;      // polls a cross-CTA wait of the persistent kernel may take
   std::vector<PersistGroup> host_groups;
+  std::vector<char> host_tmaps;
   std::vector<const float*> host_pmax_ptrs;
   int* epoch;               // device
   int* status;              // device
@@ -393,7 +396,8 @@ gsi_status_t gsi_destroy(gsi_handle_t h) {
 size_t gsi_stack_workspace_bytes(int n_groups) {
   if (n_groups <= 0) return 0;
   static_assert(sizeof(PersistGroup) <= 512, "group descriptor outgrew its slot");
-  return align_up(256) + align_up((size_t)n_groups * 512) + align_up((size_t)n_groups * 8);
+  return align_up(256) + align_up((size_t)n_groups * 512) + align_up((size_t)n_groups * 8) +
+         align_up((size_t)n_groups * GSI_MAX_MAPS * kPersistTmapBytes);
 }
 
 gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* workspace,
@@ -406,6 +410,9 @@ gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* wo
   for (int i = 0; i < n_groups; ++i) {
     if (!groups[i]) return GSI_ERR_INVALID_ARG;
     if (groups[i]->desc.max_tokens != groups[0]->desc.max_tokens) return GSI_ERR_INVALID_ARG;
+    // a handle's exchange state and scratch serve one use per step
+    for (int j = 0; j < i; ++j)
+      if (groups[j] == groups[i]) return GSI_ERR_INVALID_ARG;
   }
   gsi_stack* s = new (std::nothrow) gsi_stack();
   if (!s) return GSI_ERR_ALLOC;
@@ -420,6 +427,9 @@ gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* wo
   s->epoch = s->step + 1;
   s->status = s->step + 2;
   s->dev_groups = reinterpret_cast<PersistGroup*>(static_cast<char*>(workspace) + 256);
+  s->dev_tmaps = static_cast<char*>(workspace) + align_up(256) + align_up((size_t)n_groups * 512) +
+                 align_up((size_t)n_groups * 8);
+  s->spin_limit = kPersistSpinLimitDefault;
   s->mode = 0;
   s->trace = nullptr;
   s->persistent = false;
@@ -435,20 +445,39 @@ gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* wo
   return GSI_OK;
 }
 
-// Rows of one CTA fit its buffers, and all 16 KB chunks of the group fit the ring of ten
-// slots together (the row pass runs with every chunk of the group resident).
+// Rows of one CTA fit its buffers, and the 16 KB chunks of the group's basis slab, and of its
+// image slab, each fit the ring of ten slots together (pass 1 and the image rows run with
+// every chunk of their slab resident).
 static bool rows_fit(const gsi_layer* h, int ctas) {
   if (ctas <= 0) return false;
   const int pr = (h->desc.d + ctas - 1) / ctas, orw = (h->lay.O + ctas - 1) / ctas;
   if (pr > kPersistMaxPRows || orw > kPersistMaxORows) return false;
   if ((h->desc.flags & GSI_FLAG_DENSE) || h->desc.k <= 0) return true;
   const int rc = std::max(1, 16384 / (h->desc.k * 2));
-  return (pr + rc - 1) / rc + (orw + rc - 1) / rc <= 10;
+  return (pr + rc - 1) / rc <= 10 && (orw + rc - 1) / rc <= 10;
+}
+
+// W stream geometry of one map: rows per CTA, and rows per box (even, at most 30, chosen so
+// that the boxes of a CTA overshoot its rows as little as possible).
+static void w_geometry(int d_out, int grid, int* rows, int* rb) {
+  *rows = (d_out + grid - 1) / grid;
+  const int nblk = (*rows + kPersistBoxRowsMax - 1) / kPersistBoxRowsMax;
+  *rb = 2 * ((*rows + 2 * nblk - 1) / (2 * nblk));
+}
+
+// The per-row accumulators of the W stream hold every box row of every map of a group.
+static bool w_rows_fit(const gsi_layer* h, int grid) {
+  int total = 0;
+  for (int j = 0; j < h->desc.n_maps; ++j) {
+    int rows, rb;
+    w_geometry(h->d_out[j], grid, &rows, &rb);
+    total += (rows + rb - 1) / rb * rb;
+  }
+  return total <= kPersistMaxORows;
 }
 
 // Can this stack run on the persistent kernel?  (one or two tokens per step, bf16 basis
-// with a power-of-two rank up to 512, rows that fit the per-CTA buffers and the ring,
-// 32-byte aligned weight rows for the 256-bit loads.)
+// with a power-of-two rank up to 512, rows that fit the per-CTA buffers and the ring.)
 static bool persistent_eligible(const gsi_stack* s, int grid) {
   if (s->B > kPersistMaxTokens || grid <= 0 || grid > kPersistMaxGrid) return false;
   for (const gsi_layer* h : s->groups) {
@@ -456,9 +485,7 @@ static bool persistent_eligible(const gsi_stack* s, int grid) {
     const bool dense = d.flags & GSI_FLAG_DENSE;
     if (dense && s->B > 1) return false;   // a dense group streams W: once for all tokens (batched GEMM)
     if (d.d % 16) return false;
-    if (!rows_fit(h, grid)) return false;
-    for (int j = 0; j < d.n_maps; ++j)
-      if (reinterpret_cast<uintptr_t>(h->gp.W[j]) & 31u) return false;
+    if (!rows_fit(h, grid) || !w_rows_fit(h, grid)) return false;
     if (!dense) {
       if (d.p_dtype != GSI_BF16) return false;
       if (d.k < 64 || d.k > 512 || (d.k & (d.k - 1))) return false;
@@ -472,7 +499,6 @@ static bool persistent_eligible(const gsi_stack* s, int grid) {
 // group do not fit its share (the pair then runs one group after the other).
 static int pair_split(const gsi_layer* a, const gsi_layer* b, int grid) {
   if ((a->desc.flags | b->desc.flags) & GSI_FLAG_DENSE) return 0;
-  if (grid >= kPairSumSlot) return 0;
   const double wa = (double)(a->desc.d + a->lay.O) * a->desc.k;
   const double wb = (double)(b->desc.d + b->lay.O) * b->desc.k;
   int na = (int)(grid * wa / (wa + wb) + 0.5);
@@ -545,6 +571,7 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
         return GSI_ERR_CUDA;
     }
     s->host_groups.assign(G, PersistGroup{});
+    s->host_tmaps.assign((size_t)G * GSI_MAX_MAPS * kPersistTmapBytes, 0);
     s->host_pmax_ptrs.assign(G, nullptr);
     for (int i = 0; i < G; ++i) {
       const gsi_layer* h = s->groups[i];
@@ -552,7 +579,16 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
       const GroupParams& gp = h->gp;
       pg.P = static_cast<const uint16_t*>(gp.P);
       pg.WP = gp.WP;
-      for (int j = 0; j < gp.n_maps; ++j) pg.W[j] = gp.W[j];
+      pg.tmW = s->dev_tmaps + (size_t)i * GSI_MAX_MAPS * kPersistTmapBytes;
+      for (int j = 0; j < gp.n_maps; ++j) {
+        int rows, rb;
+        w_geometry(gp.d_out[j], s->grid, &rows, &rb);
+        pg.w_rows[j] = (short)rows;
+        pg.w_rb[j] = (short)rb;
+        if (!encode_w_stream_map(s->host_tmaps.data() + ((size_t)i * GSI_MAX_MAPS + j) * kPersistTmapBytes,
+                                 gp.W[j], (size_t)gp.d_out[j], (size_t)gp.d, (unsigned)rb))
+          return GSI_ERR_CUDA;
+      }
       for (int j = 0; j <= gp.n_maps; ++j) pg.off[j] = gp.off[j];
       pg.n_maps = gp.n_maps;
       pg.d = gp.d;
@@ -566,13 +602,13 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
       pg.x = io[i].x;
       pg.y = io[i].y;
       pg.r = gp.r;
-      pg.acc_c = reinterpret_cast<unsigned long long*>(h->ws + h->lay.pk_acc);
-      pg.slot_r = reinterpret_cast<unsigned long long*>(h->ws + h->lay.pk_slot);
+      pg.acc = reinterpret_cast<unsigned long long*>(h->ws + h->lay.pk_acc);
+      pg.xmax = reinterpret_cast<unsigned*>(h->ws + h->lay.pk_slot);
+      pg.pub = reinterpret_cast<unsigned long long*>(h->ws + h->lay.pk_slot + (size_t)kPersistMaxGrid * 4);
       pg.bar = h->bar;
       pg.cta0 = 0;
       pg.ncta = s->grid;
       pg.phase_len = 1;
-      pg.o_rows_w = (gp.O + s->grid - 1) / s->grid;
       pg.x_step_stride = (long long)s->B * gp.d;
     }
     // pairs of independent groups split the grid
@@ -585,7 +621,6 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
       b.cta0 = na;
       b.ncta = s->grid - na;
       a.phase_len = b.phase_len = 2;
-      b.slot_r = a.slot_r;   // one joint exchange
     }
     for (int i = 0; i < G; ++i) {
       PersistGroup& pg = s->host_groups[i];
@@ -612,6 +647,8 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
     if (cudaMemcpyAsync(s->dev_groups, s->host_groups.data(), sizeof(PersistGroup) * G,
                         cudaMemcpyHostToDevice, stream) != cudaSuccess ||
         cudaMemcpyAsync(dev_ptrs, s->host_pmax_ptrs.data(), sizeof(float*) * G,
+                        cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(s->dev_tmaps, s->host_tmaps.data(), s->host_tmaps.size(),
                         cudaMemcpyHostToDevice, stream) != cudaSuccess ||
         launch_patch_pmax(s->dev_groups, dev_ptrs, G, stream) != cudaSuccess)
       return GSI_ERR_CUDA;
@@ -648,6 +685,7 @@ static gsi_status_t stack_enqueue(gsi_stack_t s, bool use_counter, gsi_stream_t 
     p.log_step_stride = G;
     p.status = s->status;
     p.trace = s->trace;
+    p.spin_limit = s->spin_limit;
     p.n_tokens = s->B;
     // one launch per token of the step (up to kPersistMaxTokens; larger batches take the
     // batched kernels): each is a complete decode step of that token, the last one advances
@@ -761,6 +799,12 @@ gsi_status_t gsi_stack_step_host(gsi_stack_t s, const float* const* x_host, floa
 gsi_status_t gsi_stack_set_trace(gsi_stack_t s, unsigned long long* cycles) {
   if (!s) return GSI_ERR_INVALID_ARG;
   s->trace = cycles;
+  return GSI_OK;
+}
+
+gsi_status_t gsi_stack_set_spin_limit(gsi_stack_t s, unsigned polls) {
+  if (!s) return GSI_ERR_INVALID_ARG;
+  s->spin_limit = polls ? polls : kPersistSpinLimitDefault;
   return GSI_OK;
 }
 

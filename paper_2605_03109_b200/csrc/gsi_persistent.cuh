@@ -8,39 +8,47 @@ namespace gsi {
 constexpr int kPersistConsumerWarps = 15;  // + 1 producer warp = 16 warps: registers are allotted per 4 warps
 constexpr int kPersistMaxPRows = 256;   // basis rows one CTA may own
 constexpr int kPersistMaxORows = 512;   // output rows one CTA may own
-constexpr int kPersistMaxGrid = 256;    // CTAs (exchange-2 slots per group)
+constexpr int kPersistMaxGrid = 256;    // CTAs (tagged words per group)
 constexpr int kPersistMaxTokens = 2;    // tokens per step served by one launch per token (more: batched kernels)
-constexpr int kAccStride = 16;          // 64-bit words between c accumulators: one per 128-byte line
+constexpr int kAccStride = 16;          // 64-bit words between accumulators: one per 128-byte line
+constexpr int kPersistBoxCols = 256;    // columns of W in one streamed box
+constexpr int kPersistBoxRowsMax = 30;  // rows of W in one streamed box: two per consumer warp
+constexpr int kPersistTmapBytes = 128;  // one tensor map
 
 struct PersistGroup {
   const uint16_t* P;                 // [d][k] bf16
   const uint16_t* WP;                // [O][k] bf16, images of all maps concatenated
-  const uint16_t* W[GSI_MAX_MAPS];   // [d_out_j][d] bf16
+  const void* tmW;                   // n_maps tensor maps (device memory): W_j [d_out_j][d] bf16 in boxes of w_rb[j] rows x 256 columns
+  const float* x;                    // [n_steps][tokens][d]
+  float* y;                          // [tokens][O]
+  float* r;                          // [d]
+  // Cross-CTA state.  acc: per launch parity k + 2 fixed-point accumulators (one per 128-byte
+  // line) whose upper bits count arrivals: c_0..c_{k-1}, ||x||^2 and ||r||^2.  xmax: one
+  // 32-bit word per contributing CTA, max |x| over its rows with the launch parity in the
+  // sign bit.  pub: ||x||^2 as a double with the launch parity in the sign bit.
+  unsigned long long* acc;
+  unsigned* xmax;
+  unsigned long long* pub;
+  unsigned* bar;                     // arrival counters by launch parity: [0..1] after a dense group, [2..3] before a gated residual
+  long long x_step_stride;
   int off[GSI_MAX_MAPS + 1];
   int n_maps;
   int d, k, O;
   float eps;
   unsigned flags;
   float pmax;                        // max |P| (patched in on the device at bind time)
-  const float* x;                    // [n_steps][tokens][d]
-  float* y;                          // [tokens][O]
-  float* r;                          // [d]
-  unsigned long long* acc_c;         // [2][k][kAccStride] fixed-point accumulators, one set per launch parity
-  unsigned long long* slot_r;        // exchange 2: 32-bit words [grid + 2] (launch parity in the sign bit | partial ||r||^2)
-  unsigned* bar;                     // [6] arrival counters by launch parity: [0..1] after, [2..3] before the gated residual, [4..5] exchange 2
   int p_rows, o_rows;                // rows per CTA of P and of the images (ceil(rows / ncta))
-  long long x_step_stride;
   // Two consecutive groups whose inputs do not depend on each other's outputs may form one
-  // phase: CTAs [cta0, cta0 + ncta) run this group's projection, gate and image while the
-  // rest of the grid runs its partner's; both gates come out of one joint exchange, and a
-  // gated residual always streams W with the whole grid.
+  // phase: CTAs [cta0, cta0 + ncta) run this group's projection, residual and image while the
+  // rest of the grid runs its partner's.  A gated residual always streams W with the whole grid.
   int cta0, ncta;                    // this group's share of the grid (0, grid when alone)
   int phase_len;                     // groups in this group's phase: 1, or 2 for both of a pair
   int next_len;                      // groups in the phase after this group's (0 at the end)
-  int o_rows_w;                      // W rows per CTA of the gated residual: ceil(O / grid)
+  // W stream (gated residual, dense baseline): every CTA owns w_rows[j] consecutive rows of
+  // every map j, streamed as boxes of w_rb[j] rows (even, at most 30) x 256 columns.
+  short w_rows[GSI_MAX_MAPS];
+  short w_rb[GSI_MAX_MAPS];
 };
-
-constexpr int kPairSumSlot = 254;    // pairs need grid + 2 exchange-2 words in 256: word grid + u is ||x||^2 of group u of a pair
 
 struct PersistParams {
   const PersistGroup* groups;  // device
@@ -55,8 +63,11 @@ struct PersistParams {
   float* rho_log;              // same shape or nullptr
   int log_step_stride;
   int* status;
-  unsigned long long* trace;   // device [16] cycle counters of CTA 0, or nullptr
+  unsigned long long* trace;   // device [grid][16] cycle counters per CTA, or nullptr
+  unsigned spin_limit;         // polls a cross-CTA wait may take before it gives up
 };
+
+constexpr unsigned kPersistSpinLimitDefault = 1u << 22;
 
 int persist_smem_bytes();
 int persist_threads();
@@ -67,5 +78,8 @@ cudaError_t launch_decode_step(const PersistParams& p, int grid, bool pairs, int
 cudaError_t launch_abs_max_bf16(const void* p, size_t n, float* out, cudaStream_t st);
 cudaError_t launch_patch_pmax(PersistGroup* groups, const float* const* pmax_ptrs, int n,
                               cudaStream_t st);
+// Tensor map of one weight matrix for the persistent kernel's W stream: W [rows][cols] bf16
+// row-major, boxes of box_rows x 256 columns, no swizzle.  out: 128 bytes on the HOST.
+bool encode_w_stream_map(void* out, const void* W, size_t rows, size_t cols, unsigned box_rows);
 
 }  // namespace gsi

@@ -1,34 +1,41 @@
 // Persistent decode-step kernel: every group of the stack in ONE launch.
 //
-// One CTA per SM.  Each CTA owns a fixed slab of rows of every basis P and of
-// every (concatenated) image W_P.  A producer warp streams those slabs from HBM
-// into a ring of shared-memory slots with bulk async copies, in program order
-// and independent of the data-dependent steps (weight addresses never depend
-// on x), so the next group's weights arrive while the current group waits on
-// its cross-CTA exchanges.  Fifteen consumer warps run Algorithm 1 per group (two
-// consecutive groups declared independent share a phase on two parts of the grid):
+// One CTA per SM.  Each CTA owns a fixed slab of rows of every basis P and of every
+// (concatenated) image W_P, and a fixed set of rows of every weight matrix W.  A producer
+// warp streams ALL weights from HBM into a ring of shared-memory slots: the slabs of P and
+// W_P with bulk async copies, the rows of W (gated residual, dense baseline) as TMA boxes of
+// up to 30 rows x 256 columns.  Weight addresses never depend on x, so the next group's slabs
+// arrive while the current group waits on its exchange.  Fifteen consumer warps run
+// Algorithm 1 per group (two consecutive groups declared independent share a phase on two
+// parts of the grid).  A phase has ONE grid-wide exchange:
 //
-//   pass 1     partial c = P_slab^T x_slab                     (line 1)
-//   exchange 1 c = sum over CTAs, by 64-bit fixed-point atomics whose words
-//              also count arrivals (no separate flag, no fence, order-free and
-//              therefore bit-reproducible)
-//   pass 2     r_slab = x_slab - P_slab c, partial ||r||^2      (lines 2-3)
-//   exchange 2 every CTA publishes its partial ||r||^2 as one 32-bit word, the sign
-//              bit carrying the parity of the launch (relaxed store: the word
-//              validates itself, every launch rewrites every word), as soon as its
-//              residual rows are done ...
-//   image      y_rows = W_P,rows c                              (line 5)
-//              ... and collects the words after its image rows, so the exchange
-//              runs under them; every CTA sums the words in a fixed order and
-//              takes the same gate decision                     (line 4)
-//   gated      y_rows += W_rows r, W streamed with 256-bit loads, then a grid
-//              barrier                                          (Eq. (3.2))
+//   statistics  warp 0: max |x| and sum x^2 over this CTA's rows of x; the maximum is
+//               published as a tagged 32-bit word (no fence: the word validates itself)
+//   pass 1      partial c = P_slab^T x_slab                              (line 1)
+//   exchange    every CTA adds, as 64-bit fixed-point numbers whose upper bits count the
+//               arrivals (integer addition is order-free, so the sums are bit-reproducible):
+//               its partial c_j (scale from the global max |x|, collected from the tagged
+//               words meanwhile), its partial ||x||^2, and its partial ||r||^2 of the
+//               PREVIOUS phase; it then polls the words until all have arrived
+//   gate        of the previous phase, from the exact integer sums: the same decision on
+//               every CTA                                                (line 4, Eq. (3.3))
+//   pass 2      r_slab = x_slab - P_slab c, partial ||r||^2              (lines 2-3)
+//   gated       y_rows += W_rows r of the groups of the phase before the previous one
+//               whose gate fired (their boxes follow this phase's basis slab in the ring;
+//               r and the image rows were made visible by a fenced arrival counter that
+//               every CTA posted when the gate was decided)              (Eq. (3.2))
+//   image       y_rows = W_P,rows c                                      (line 5)
 //
-// Every wait is bounded; a wait that gives up records GSI_ERR_TIMEOUT in the
-// status word, the CTA drains its copies in flight and returns.
+// so the gate of a phase is known one exchange later and its residual runs one phase after
+// that: every group's inputs are pre-staged buffers (the contract of the stack driver), and
+// all of y is complete when the launch ends.  Two ticks after the last phase settle the
+// remaining gates and residuals.
+//
+// Every wait is bounded; a wait that gives up records GSI_ERR_TIMEOUT in the status word,
+// the CTA drains its copies in flight and returns.
 //
 // This header holds the kernel; every build of it (with or without the pair logic, for any
-// rank or for rank 256 only) is compiled in a translation unit of its own.
+// rank or for one rank) is compiled in a translation unit of its own.
 #pragma once
 
 #include <cstdio>
@@ -47,38 +54,39 @@ constexpr int kThreadsP = kNC + 32;         // + producer warp
 constexpr int kSlots = 10;
 constexpr int kChunk = 16384;
 constexpr int kSlice = 4096;                // columns of W per staged slice of r
-constexpr int kWLoads = 4;                  // 256-bit loads per lane in flight in the W stream
-constexpr unsigned kSpinLimit = 1u << 22;
+constexpr int kBoxCols = kPersistBoxCols;
+constexpr unsigned kLocalSpinLimit = 1u << 24;   // waits inside the CTA (ring, producer hand-off)
 constexpr int kCountShift = 54;
+constexpr unsigned long long kOne = 1ull << kCountShift;
 
 // shared memory map (bytes)
-constexpr int kXBatch = 5;           // float4 loads of x in flight per thread
 constexpr int kOffBar = 0;          // full[kSlots], empty[kSlots]
-constexpr int kOffMisc = 256;       // abort flag, scalars
-constexpr int kOffX = 512;          // x of this CTA's basis rows      (kPersistMaxPRows floats)
-constexpr int kOffC = 1536;         // c                                (512 floats)
-constexpr int kOffVals = 3584;      // exchange-2 values                (256 floats)
-constexpr int kOffDesc = 4608;      // 4 group descriptors, 512 B each (this phase's and the next's)
+constexpr int kOffMisc = 256;       // scalars
+constexpr int kOffX = 512;          // x of this CTA's basis rows, two buffers (kPersistMaxPRows floats each)
+constexpr int kOffC = kOffX + 2 * kPersistMaxPRows * 4;   // c (512 floats)
+constexpr int kOffDesc = kOffC + 2048;                    // 4 group descriptors, 512 B each
 constexpr int kDescSlots = 4;
-constexpr int kOffRed = kOffDesc + kDescSlots * 512;   // cross-warp scratch (kNW*512 floats)
-constexpr int kOffRq = kOffRed + kNW * 512 * 4;   // staged r, 4 interleaved quarters (16 KB)
-constexpr int kOffYacc = kOffRq + 16384;          // per-row accumulators (kPersistMaxORows floats)
+constexpr int kOffRed = kOffDesc + kDescSlots * 512;      // cross-warp scratch (kNW*512 floats)
+constexpr int kOffRs = kOffRed + kNW * 512 * 4;           // staged slice of r (16 KB)
+constexpr int kOffYacc = kOffRs + kSlice * 4;             // per-row accumulators (kPersistMaxORows floats)
 constexpr int kOffRing = ((kOffYacc + kPersistMaxORows * 4 + 1023) / 1024) * 1024;
 constexpr int kSmemBytes = kOffRing + kSlots * kChunk;
 static_assert(kSmemBytes <= 232448, "shared memory budget of one sm_100 CTA");
 static_assert(sizeof(PersistGroup) <= 512 && sizeof(PersistGroup) % 4 == 0, "descriptor slot");
-static_assert(kOffC - kOffX >= kPersistMaxPRows * 4, "x slab");
+static_assert(kPersistBoxRowsMax * kBoxCols * 2 <= kChunk, "a box fits a slot");
+static_assert(kPersistBoxRowsMax == 2 * kNW, "two rows of a box per consumer warp");
 constexpr int kDescWords = (int)(sizeof(PersistGroup) / 4);
 
 struct Misc {
   int abort;
-  int gate;
-  float amax;
-  float sum2;
-  int nonfinite;
-  float sr;
-  int deposits;   // warps that have handed in their ||r||^2 partial in this phase
+  unsigned amax_bits;       // max |x| of this phase's group (>= 0x7f800000: a non-finite token)
+  float x2_part;            // this CTA's sum of x^2 over its rows
+  double x2;                // ||x||^2 of this phase's group
+  int fire[4];              // decisions on the previous phase's groups, by tick parity: 1 = stream W
+  float sr[kNW];            // per-warp partial ||r||^2 of this phase
+  volatile unsigned decision[4];   // hand-off to the producer: (phase + 1) << 8 | fire mask
 };
+static_assert(sizeof(Misc) <= 256, "scalars");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -106,7 +114,7 @@ __device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
 }
 // Bounded wait; gives up when the limit is reached or another thread aborted.
 __device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, volatile int* abort) {
-  for (unsigned it = 0; it < kSpinLimit; ++it) {
+  for (unsigned it = 0; it < kLocalSpinLimit; ++it) {
     if (mbar_try(b, parity)) return true;
     if ((it & 1023u) == 1023u && *abort) return false;
   }
@@ -119,6 +127,19 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
       "l"(src), "r"(bytes), "r"(smem_u32(bar))
       : "memory");
 }
+// One box of a 2-D tensor map (no multicast): x = first column, y = first row.
+__device__ __forceinline__ void tma_box_g2s(void* dst, const void* tmap, int x, int y, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
+          smem_u32(dst)),
+      "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar))
+      : "memory");
+}
+__device__ __forceinline__ void cp_async4(void* dst, const void* src) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void csync() {  // consumer warps only
   asm volatile("bar.sync 1, %0;" ::"n"(kNC) : "memory");
 }
@@ -144,24 +165,14 @@ __device__ __forceinline__ unsigned ld_relaxed_u32(const unsigned* p) {
 __device__ __forceinline__ void red_relaxed_u32(unsigned* p, unsigned v) {
   asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-__device__ __forceinline__ void ld256_stream(const void* p, uint32_t (&v)[8]) {
-  asm volatile(
-      "ld.global.nc.L1::no_allocate.L2::evict_first.v8.b32 {%0,%1,%2,%3,%4,%5,%6,%7}, [%8];"
-      : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]),
-        "=r"(v[7])
-      : "l"(p));
-}
-__device__ __forceinline__ void prefetch_l2(const void* p) {
-  asm volatile("prefetch.global.L2 [%0];" ::"l"(p));
-}
 
 __device__ __forceinline__ void fail(const PersistParams& p, Misc* misc) {
   misc->abort = 1;
   atomicExch(p.status, (int)GSI_ERR_TIMEOUT);
 }
 
-// Optional cycle trace of CTA 0 (sections of the per-group pipeline, summed
-// over groups); p.trace == nullptr disables it.
+// Optional cycle trace (thread 0 of every CTA; sections of the per-phase pipeline, summed
+// over phases); p.trace == nullptr disables it.
 struct Trace {
   unsigned long long* out;
   long long t;
@@ -178,60 +189,141 @@ struct Trace {
   }
 };
 
-
 struct Slab {
   int p0, p1;  // basis rows owned by this CTA
-  int o0, o1;  // rows of the concatenated maps owned by this CTA (image rows and W rows)
+  int o0, o1;  // rows of the concatenated images owned by this CTA
 };
-__device__ __forceinline__ Slab slab_of(const PersistGroup& g, int cta) {
+__device__ __forceinline__ Slab slab_of(const PersistGroup& g, int lc) {
   Slab s;
-  s.p0 = min(g.d, cta * g.p_rows);
+  s.p0 = min(g.d, lc * g.p_rows);
   s.p1 = min(g.d, s.p0 + g.p_rows);
-  s.o0 = min(g.O, cta * g.o_rows);
+  s.o0 = min(g.O, lc * g.o_rows);
   s.o1 = min(g.O, s.o0 + g.o_rows);
   return s;
 }
 
 // ------------------------------------------------------------------ producer
-__device__ void producer(const PersistParams& p, unsigned char* smem, Misc* misc) {
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kOffBar);
-  uint64_t* empty = full + kSlots;
-  unsigned char* ring = smem + kOffRing;
-  volatile int* abort = &misc->abort;
-  unsigned n = 0;
-  for (int gi = 0; gi < p.n_groups && !*abort; ++gi) {
-    const PersistGroup& g = p.groups[gi];
-    if (g.flags & GSI_FLAG_DENSE) continue;
-    const int lc = (int)blockIdx.x - g.cta0;
-    if (lc < 0 || lc >= g.ncta) continue;   // its partner's share of the grid
-    const Slab s = slab_of(g, lc);
-    const int rc = kChunk / (g.k * 2);
-    for (int part = 0; part < 2; ++part) {
-      const int a = part ? s.o0 : s.p0, b = part ? s.o1 : s.p1;
-      const uint16_t* base = part ? g.WP : g.P;
-      for (int r = a; r < b; r += rc) {
-        const int rows = min(rc, b - r);
-        const unsigned slot = n % kSlots, ph = (n / kSlots) & 1u;
-        if (!mbar_wait(&empty[slot], ph ^ 1u, abort)) {
-          if (!*abort) fail(p, misc);
-          goto drain;
+struct Ring {
+  uint64_t* full;
+  uint64_t* empty;
+  unsigned char* slots;
+  unsigned n;   // sequence number of the next chunk
+};
+
+// Wait for the slot of chunk n to be free; false = give up.
+__device__ __forceinline__ bool ring_acquire(Ring& rg, volatile int* abort) {
+  const unsigned slot = rg.n % kSlots, ph = (rg.n / kSlots) & 1u;
+  return mbar_wait(&rg.empty[slot], ph ^ 1u, abort);
+}
+
+// The W boxes of one group for this CTA, in the order the consumers take them: column
+// slices of 4096 outermost (one staged slice of r serves them), then maps, then row blocks,
+// then the 256-column boxes of the slice.
+__device__ bool produce_w(const PersistGroup& g, Ring& rg, volatile int* abort) {
+  const int cta = blockIdx.x;
+  const int nsl = (g.d + kSlice - 1) / kSlice;
+  for (int sl = 0; sl < nsl; ++sl) {
+    const int c0 = sl * kSlice, ncb = (min(kSlice, g.d - c0) + kBoxCols - 1) / kBoxCols;
+    for (int j = 0; j < g.n_maps; ++j) {
+      const int dout = g.off[j + 1] - g.off[j], rows = g.w_rows[j], rb = g.w_rb[j];
+      const int row0 = cta * rows;
+      const int live = min(rows, dout - row0);
+      const char* tm = static_cast<const char*>(g.tmW) + (size_t)j * kPersistTmapBytes;
+      for (int b = 0; b * rb < live; ++b) {
+        for (int cb = 0; cb < ncb; ++cb) {
+          if (!ring_acquire(rg, abort)) return false;
+          const unsigned slot = rg.n % kSlots;
+          mbar_expect_tx(&rg.full[slot], (uint32_t)rb * kBoxCols * 2);
+          tma_box_g2s(rg.slots + (size_t)slot * kChunk, tm, c0 + cb * kBoxCols, row0 + b * rb,
+                      &rg.full[slot]);
+          ++rg.n;
         }
-        const uint32_t bytes = (uint32_t)rows * g.k * 2;
-        mbar_expect_tx(&full[slot], bytes);
-        bulk_g2s(ring + (size_t)slot * kChunk, base + (size_t)r * g.k, bytes, &full[slot]);
-        ++n;
       }
     }
   }
-drain:
+  return true;
+}
+
+// Rows [a, b) of a row-major [rows][k] bf16 matrix as chunks of whole rows.
+__device__ bool produce_rows(const uint16_t* base, int k, int a, int b, Ring& rg, volatile int* abort) {
+  const int rc = kChunk / (k * 2);
+  for (int r = a; r < b; r += rc) {
+    const int rows = min(rc, b - r);
+    if (!ring_acquire(rg, abort)) return false;
+    const unsigned slot = rg.n % kSlots;
+    const uint32_t bytes = (uint32_t)rows * k * 2;
+    mbar_expect_tx(&rg.full[slot], bytes);
+    bulk_g2s(rg.slots + (size_t)slot * kChunk, base + (size_t)r * k, bytes, &rg.full[slot]);
+    ++rg.n;
+  }
+  return true;
+}
+
+__device__ void producer(const PersistParams& p, unsigned char* smem, Misc* misc) {
+  Ring rg;
+  rg.full = reinterpret_cast<uint64_t*>(smem + kOffBar);
+  rg.empty = rg.full + kSlots;
+  rg.slots = smem + kOffRing;
+  rg.n = 0;
+  volatile int* abort = &misc->abort;
+  const int cta = blockIdx.x;
+  bool ok = true;
+  // ticks: tick t runs phase t (while there is one) and the gated residuals of phase t - 2
+  int gi = 0;        // first group of phase t
+  int g_pp = -1, len_pp = 0;   // phase t - 2
+  int g_p = -1, len_p = 0;     // phase t - 1
+  for (int t = 0; ok; ++t) {
+    const bool own = gi < p.n_groups;
+    if (!own && len_p == 0 && len_pp == 0) break;
+    int len = 0;
+    const PersistGroup* g = nullptr;
+    if (own) {
+      const PersistGroup& gA = p.groups[gi];
+      len = gA.phase_len;
+      g = (len == 2 && cta >= gA.cta0 + gA.ncta) ? &p.groups[gi + 1] : &gA;
+    }
+    const bool dense = own && (g->flags & GSI_FLAG_DENSE);
+    Slab s{};
+    if (own && !dense) {
+      s = slab_of(*g, cta - g->cta0);
+      ok = produce_rows(g->P, g->k, s.p0, s.p1, rg, abort);
+    }
+    if (ok && len_pp > 0) {
+      // the decision on phase t - 2 (taken by the consumers during tick t - 1)
+      const unsigned want = (unsigned)(t - 1);   // (phase + 1)
+      unsigned v = 0, it = 0;
+      for (;;) {
+        v = misc->decision[(t - 2) & 3];
+        if ((v >> 8) == want) break;
+        if (++it > kLocalSpinLimit || *abort) {
+          ok = false;
+          break;
+        }
+      }
+      for (int u = 0; ok && u < len_pp; ++u)
+        if (v & (1u << u)) ok = produce_w(p.groups[g_pp + u], rg, abort);
+    }
+    if (ok && own) {
+      if (dense)
+        ok = produce_w(*g, rg, abort);
+      else
+        ok = produce_rows(g->WP, g->k, s.o0, s.o1, rg, abort);
+    }
+    g_pp = g_p;
+    len_pp = len_p;
+    g_p = gi;
+    len_p = len;
+    gi += len;
+  }
+  if (!ok && !*abort) fail(p, misc);
   // Every copy issued must have landed before the CTA may give up its shared
   // memory: wait (bounded) for the last kSlots chunks.
   {
-    const unsigned first = n > (unsigned)kSlots ? n - kSlots : 0;
-    for (unsigned c = first; c < n; ++c) {
+    const unsigned first = rg.n > (unsigned)kSlots ? rg.n - kSlots : 0;
+    for (unsigned c = first; c < rg.n; ++c) {
       const unsigned slot = c % kSlots, ph = (c / kSlots) & 1u;
-      for (unsigned it = 0; it < kSpinLimit; ++it)
-        if (mbar_try(&full[slot], ph)) break;
+      for (unsigned it = 0; it < kLocalSpinLimit; ++it)
+        if (mbar_try(&rg.full[slot], ph)) break;
     }
   }
 }
@@ -239,19 +331,6 @@ drain:
 // ------------------------------------------------------------------ consumer
 // Lane layout over a row of k bf16: KV = k/8 vectors, LPR = min(32, KV) lanes
 // per row, RPP = 32/LPR rows per warp pass, VPL = KV/LPR vectors per lane.
-struct Ctx {
-  int step, slot_io;
-  int len;     // groups in the phase just run (1, or 2 for a pair)
-  unsigned parity, tag;
-  unsigned n;  // ring sequence number, advances exactly as in producer()
-  Trace tr;
-};
-
-// ---- consumer building blocks.  The per-group code below is executed once per
-// group and is deliberately compact (no templates, shifts instead of divisions,
-// the rarely-taken gated residual out of line): the per-group loop has to stay
-// resident in the SM's instruction cache, a loop that does not is bound by
-// instruction fetch, not by memory.
 
 // Sum eight per-lane row partials across the LPR = 1<<lpr_log2 lanes (8, 16 or
 // 32) that share the rows.  Halving exchange: each level sends half of the
@@ -357,15 +436,18 @@ __device__ __forceinline__ void dot8(const uint4* tile, const float* s_c, const 
 
 // 2^e as a double, e in the normal range
 __device__ __forceinline__ double pow2d(int e) { return __hiloint2double((1023 + e) << 20, 0); }
+// Smallest e with v < 2^e for a positive finite double v (binary exponent + 1).
+__device__ __forceinline__ int exp_above(double v) {
+  return ((__double2hiint(v) >> 20) & 0x7ff) - 1022;
+}
 
-// Grid-wide arrival counter: add one, wait (bounded) until `target` arrived.
-__device__ __forceinline__ bool grid_arrive_wait(unsigned* ctr, unsigned target,
-                                                 const PersistParams& p, Misc* misc) {
+// Grid-wide arrival counter: wait (bounded) until `target` arrivals have been added.
+__device__ __forceinline__ bool grid_wait(const unsigned* ctr, unsigned target, const PersistParams& p,
+                                          Misc* misc) {
   volatile int* abort = &misc->abort;
-  red_relaxed_u32(ctr, 1u);
   unsigned it = 0;
   while (ld_relaxed_u32(ctr) < target) {
-    if (++it > kSpinLimit || *abort) {
+    if (++it > p.spin_limit || *abort) {
       if (!*abort) fail(p, misc);
       return false;
     }
@@ -373,579 +455,627 @@ __device__ __forceinline__ bool grid_arrive_wait(unsigned* ctr, unsigned target,
   return true;
 }
 
-// ---- F. gated residual: y_rows (+)= W_rows . src (src = r, or x for the dense
-// baseline).  Out of line: most groups skip it.
-__device__ __noinline__ void gated_pass(const PersistGroup& g, const Slab& s, const float* src,
-                                        float* y, bool dense, unsigned char* smem) {
-  float4* s_rq = reinterpret_cast<float4*>(smem + kOffRq);
+// Poll one accumulator until `n` arrivals have been added; returns the signed sum.
+__device__ __forceinline__ long long poll_acc(const unsigned long long* wp, unsigned n,
+                                              const PersistParams& p, Misc* misc) {
+  volatile int* abort = &misc->abort;
+  unsigned long long w = 0;
+  unsigned it = 0;
+  for (;;) {
+    w = ld_relaxed_u64(wp);
+    if ((unsigned)((w + (kOne >> 1)) >> kCountShift) == n) break;
+    if (++it > p.spin_limit || ((it & 1023u) == 0 && *abort)) {
+      if (!*abort) fail(p, misc);
+      break;
+    }
+  }
+  return (long long)(w - ((unsigned long long)n << kCountShift));
+}
+
+struct Ctx {
+  int slot_io;
+  unsigned parity, tag;
+  Ring rg;        // consumer's view: n advances exactly as in producer()
+  Trace tr;
+};
+
+// ---- W stream: y_rows (+)= W_rows . src (src = r of a gated group, or x for the dense
+// baseline), boxes taken from the ring in the producer's order.  Out of line: most phases
+// skip it.  Returns false when a wait gave up.
+__device__ __noinline__ bool w_stream(const PersistParams& p, const PersistGroup& g, const float* src,
+                                      float* y, bool dense, unsigned char* smem, Ctx& ctx,
+                                      Misc* misc) {
+  float* s_rs = reinterpret_cast<float*>(smem + kOffRs);
   float* s_yacc = reinterpret_cast<float*>(smem + kOffYacc);
+  volatile int* abort = &misc->abort;
+  Ring& rg = ctx.rg;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int rows = s.o1 - s.o0;
+  const int cta = blockIdx.x;
   const int nsl = (g.d + kSlice - 1) / kSlice;
+  bool ok = true;
 #pragma unroll 1
   for (int sl = 0; sl < nsl; ++sl) {
-    const int c0 = sl * kSlice, cols = min(kSlice, g.d - c0), nv = cols >> 4;
+    const int c0 = sl * kSlice, cols = min(kSlice, g.d - c0);
+    const int ncb = (cols + kBoxCols - 1) / kBoxCols;
     csync();
+    // Stage the slice so that a lane's two 16-byte loads per box are conflict-free: within a
+    // 256-column block, the first halves of the 32 lanes' eight columns, then the second halves.
 #pragma unroll 1
-    for (int v = tid; v < nv; v += kNC) {
-      const float4* sp = reinterpret_cast<const float4*>(src + c0 + v * 16);
-#pragma unroll
-      for (int q = 0; q < 4; ++q) s_rq[q * 256 + v] = __ldcg(sp + q);
+    for (int i = tid; i < ncb * 64; i += kNC) {
+      const int col = i * 4;
+      const float4 v = col < cols ? __ldcg(reinterpret_cast<const float4*>(src + c0 + col))
+                                  : make_float4(0.f, 0.f, 0.f, 0.f);
+      const int blk = i >> 6, w4 = i & 63;
+      reinterpret_cast<float4*>(s_rs)[blk * 64 + (w4 & 1) * 32 + (w4 >> 1)] = v;
     }
     csync();
-    auto row_ptr = [&](int rw) -> const uint16_t* {
-      const int a = s.o0 + rw;
-      int j = 0;
-      while (j + 1 < g.n_maps && a >= g.off[j + 1]) ++j;
-      return g.W[j] + (size_t)(a - g.off[j]) * g.d + c0;
-    };
-    // kWLoads x 256-bit loads per lane are in flight before the first FMA.
+    int ybase = 0;
 #pragma unroll 1
-    for (int rw = warp; rw < rows; rw += kNW) {
-      const uint16_t* wrow = row_ptr(rw);
-      unsigned long long acc2 = 0ull;  // two fp32 partial sums (two-wide FMA)
+    for (int j = 0; j < g.n_maps; ++j) {
+      const int dout = g.off[j + 1] - g.off[j], rows = g.w_rows[j], rb = g.w_rb[j];
+      const int live = min(rows, dout - cta * rows);
+      const bool mine = 2 * warp < rb;
 #pragma unroll 1
-      for (int v0 = lane; v0 < nv; v0 += kWLoads * 32) {
-        uint32_t w[kWLoads][8];
-#pragma unroll
-        for (int u = 0; u < kWLoads; ++u) {
-          const int v = v0 + u * 32;
-          if (v < nv) ld256_stream(wrow + (size_t)v * 16, w[u]);
+      for (int b = 0; b * rb < live; ++b) {
+        unsigned long long a0 = 0ull, a1 = 0ull;
+#pragma unroll 1
+        for (int cb = 0; cb < ncb; ++cb) {
+          const unsigned slot = rg.n % kSlots, ph = (rg.n / kSlots) & 1u;
+          ++rg.n;
+          if (ok && !mbar_wait(&rg.full[slot], ph, abort)) ok = false;
+          if (ok && mine) {
+            const uint4* tile = reinterpret_cast<const uint4*>(rg.slots + (size_t)slot * kChunk);
+            const uint4 w0 = tile[(2 * warp) * (kBoxCols / 8) + lane];
+            const uint4 w1 = tile[(2 * warp + 1) * (kBoxCols / 8) + lane];
+            const float4 ra = reinterpret_cast<const float4*>(s_rs)[cb * 64 + lane];
+            const float4 rb4 = reinterpret_cast<const float4*>(s_rs)[cb * 64 + 32 + lane];
+            const unsigned long long r0 = pack2(ra.x, ra.y), r1 = pack2(ra.z, ra.w);
+            const unsigned long long r2 = pack2(rb4.x, rb4.y), r3 = pack2(rb4.z, rb4.w);
+            fma2(a0, bf16x2_to_f32x2(w0.x), r0);
+            fma2(a1, bf16x2_to_f32x2(w1.x), r0);
+            fma2(a0, bf16x2_to_f32x2(w0.y), r1);
+            fma2(a1, bf16x2_to_f32x2(w1.y), r1);
+            fma2(a0, bf16x2_to_f32x2(w0.z), r2);
+            fma2(a1, bf16x2_to_f32x2(w1.z), r2);
+            fma2(a0, bf16x2_to_f32x2(w0.w), r3);
+            fma2(a1, bf16x2_to_f32x2(w1.w), r3);
+          }
+          __syncwarp();
+          if (ok && lane == 0) mbar_arrive(&rg.empty[slot]);
         }
-#pragma unroll
-        for (int u = 0; u < kWLoads; ++u) {
-          const int v = v0 + u * 32;
-          if (v < nv) {
-#pragma unroll
-            for (int q = 0; q < 4; ++q) {
-              const float4 rr = s_rq[q * 256 + v];
-              fma2(acc2, bf16x2_to_f32x2(w[u][2 * q]), pack2(rr.x, rr.y));
-              fma2(acc2, bf16x2_to_f32x2(w[u][2 * q + 1]), pack2(rr.z, rr.w));
-            }
+        if (mine) {
+          const float t0 = warp_sum(sum2(a0)), t1 = warp_sum(sum2(a1));
+          if (lane == 0) {
+            const int i0 = ybase + b * rb + 2 * warp;
+            s_yacc[i0] = (sl == 0 ? 0.f : s_yacc[i0]) + t0;
+            s_yacc[i0 + 1] = (sl == 0 ? 0.f : s_yacc[i0 + 1]) + t1;
           }
         }
       }
-      const float acc = warp_sum(sum2(acc2));
-      if (lane == 0) s_yacc[rw] = (sl == 0 ? 0.f : s_yacc[rw]) + acc;
+      ybase += ((live > 0 ? (live + rb - 1) / rb : 0)) * rb;
     }
   }
-  __syncwarp();
+  if (!ok && !*abort) fail(p, misc);
+  csync();
+  // rows back to y: the same walk over the maps
+  {
+    int ybase = 0;
 #pragma unroll 1
-  for (int rw = warp; rw < rows; rw += kNW) {
-    if (lane == 0) {
-      float* yp = y + s.o0 + rw;
-      *yp = dense ? s_yacc[rw] : (__ldcg(yp) + s_yacc[rw]);
+    for (int j = 0; j < g.n_maps; ++j) {
+      const int dout = g.off[j + 1] - g.off[j], rows = g.w_rows[j], rb = g.w_rb[j];
+      const int live = min(rows, dout - cta * rows);
+      if (ok) {
+#pragma unroll 1
+        for (int i = tid; i < live; i += kNC) {
+          float* yp = y + g.off[j] + cta * rows + i;
+          *yp = dense ? s_yacc[ybase + i] : (__ldcg(yp) + s_yacc[ybase + i]);
+        }
+      }
+      ybase += ((live > 0 ? (live + rb - 1) / rb : 0)) * rb;
     }
   }
+  return ok;
 }
 
-// Make the next group's activations L2-resident while this group runs (a real
-// pipeline would find them there, written by the preceding operator).
-__device__ __forceinline__ void prefetch_next_x(const PersistGroup& gn, int slot_io, int n_tokens,
-                                                int who = 0) {
-  if ((int)blockIdx.x == who) {
-    const char* xn = reinterpret_cast<const char*>(gn.x + (long long)slot_io * gn.x_step_stride);
-    const int lines = (gn.d * 4 * n_tokens + 127) >> 7;
-    for (int l = threadIdx.x; l < lines; l += kNC) prefetch_l2(xn + (size_t)l * 128);
+
+// Items of eight rows (one lane group each) over the rows of `nchunks` ring chunks that start
+// at sequence number n0.  Item ids [id0, id0 + n_ids) of the phase's joint numbering belong to
+// this part; ids are dealt round-robin to the lane groups of the CTA, so the basis rows and the
+// image rows of a phase load the warps evenly.  kImage: out[row] = dot (NaN for a non-finite
+// token); otherwise out[row] = x[row] - dot and the return value is this lane's share of
+// ||r||^2.  Every warp gives every chunk back exactly once.
+template <bool kImage>
+__device__ __forceinline__ float row_items(const Geo& q, Ring& rg, unsigned n0, int nchunks, int nrows,
+                                           int id0, int n_ids, const float* s_c, const float* s_x,
+                                           float* out, bool nonfinite, bool ok) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  const int LPR = 1 << q.lpr_log2, rpp_log2 = 5 - q.lpr_log2, rc = 1 << q.rc_log2;
+  const int hold_log2 = q.lpr_log2 - 3;          // lanes per held row after reduce8
+  const int lanegroups = kNW << rpp_log2;
+  float sr = 0.f;
+  int released = 0;
+  if (ok) {
+    int id = (warp << rpp_log2) + q.sub;
+    if (id < id0) id += ((id0 - id + lanegroups - 1) / lanegroups) * lanegroups;
+#pragma unroll 1
+    for (; id < id0 + n_ids; id += lanegroups) {
+      const int row0g = (id - id0) << 3;                       // first row, within the slab
+      const int ci = min(row0g >> q.rc_log2, nchunks - 1);
+      const int ci_warp = __shfl_sync(0xffffffffu, ci, 0);     // ids ascend with the lane
+      if (lane == 0)
+        for (; released < ci_warp; ++released) mbar_arrive(&rg.empty[(n0 + released) % kSlots]);
+      released = ci_warp;
+      const uint4* tile =
+          reinterpret_cast<const uint4*>(rg.slots + (size_t)((n0 + ci) % kSlots) * kChunk);
+      const int r_lo = ci << q.rc_log2, rows = min(rc, nrows - r_lo);
+      const int row0 = row0g - r_lo;
+      float v[8];
+      dot8(tile, s_c, q, row0, rows, v);
+      const float dot = reduce8(v, q.cl, LPR);
+      const int row = row0 + (q.cl >> hold_log2);
+      if ((q.cl & ((1 << hold_log2) - 1)) == 0 && row < rows && row0g < nrows) {
+        if (kImage) {
+          out[r_lo + row] = nonfinite ? __int_as_float(0x7fc00000) : dot;
+        } else {
+          const float rv = s_x[r_lo + row] - dot;
+          out[r_lo + row] = rv;
+          sr = fmaf(rv, rv, sr);
+        }
+      }
+    }
+    __syncwarp();
+    if (lane == 0)
+      for (; released < nchunks; ++released) mbar_arrive(&rg.empty[(n0 + released) % kSlots]);
   }
+  return sr;
 }
 
-// One group.  Returns false when the CTA must stop (a wait gave up).
+// All chunks [n0, n0 + count) have landed (one chunk per lane, all waits in flight together).
+__device__ __forceinline__ bool chunks_landed(Ring& rg, unsigned n0, int count, volatile int* abort) {
+  const int lane = threadIdx.x & 31;
+  bool mine_ok = true;
+  for (int c = lane; c < count; c += 32) {
+    const unsigned seq = n0 + c;
+    mine_ok = mine_ok && mbar_wait(&rg.full[seq % kSlots], (seq / kSlots) & 1u, abort);
+  }
+  return __all_sync(0xffffffffu, mine_ok);
+}
+
 // kPairs = false compiles the pair logic out: stacks without concurrent groups run a smaller
 // loop (the per-phase code has to stay resident in the instruction cache).  kK != 0 is a
 // build for stacks whose groups all have rank kK (shifts, strides and loop bounds become
 // constants); kK = 0 reads the rank from the descriptor.
 template <bool kPairs, int kK>
-__device__ bool group_phase(const PersistParams& p, unsigned char* smem, Misc* misc, Ctx& ctx,
-                            int gi) {
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kOffBar);
-  uint64_t* empty = full + kSlots;
-  float* s_x = reinterpret_cast<float*>(smem + kOffX);
+__device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc) {
+  float* s_xb = reinterpret_cast<float*>(smem + kOffX);
   float* s_c = reinterpret_cast<float*>(smem + kOffC);
-  float* s_vals = reinterpret_cast<float*>(smem + kOffVals);
   float* s_red = reinterpret_cast<float*>(smem + kOffRed);
-  unsigned char* ring = smem + kOffRing;
   volatile int* abort = &misc->abort;
-
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = gridDim.x, cta = blockIdx.x;
-  const int slot_io = ctx.slot_io;
-  const unsigned parity = ctx.parity, tag = ctx.tag;
-  unsigned& n = ctx.n;
-  Trace& tr = ctx.tr;
 
-  // The descriptors of this phase (one group, or a pair of independent groups that split
-  // the grid) were staged in shared memory one phase ago, descriptor i in slot i % 4;
-  // stage the next phase's now.
+  Ctx ctx;
+  ctx.rg.full = reinterpret_cast<uint64_t*>(smem + kOffBar);
+  ctx.rg.empty = ctx.rg.full + kSlots;
+  ctx.rg.slots = smem + kOffRing;
+  ctx.rg.n = 0;
+  Ring& rg = ctx.rg;
+  const int step = p.use_counter ? *p.step : 0;
+  const int slot_io = step % p.n_steps;
+  ctx.slot_io = slot_io;
+  const int epoch = *p.epoch;
+  const unsigned parity = (unsigned)epoch & 1u, tag = ((unsigned)epoch + 1u) & 1u;
+  ctx.parity = parity;
+  ctx.tag = tag;
+  Trace& tr = ctx.tr;
+  tr.start(p);
+
   auto desc = [&](int i) -> const PersistGroup& {
     return *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + (i & (kDescSlots - 1)) * 512);
   };
-  const PersistGroup& gA = desc(gi);
-  const int len = kPairs ? gA.phase_len : 1, next_len = kPairs ? gA.next_len : min(gA.next_len, 1);
-  const PersistGroup& gB = desc(gi + len - 1);   // gA itself when the group is alone
-  const bool second = kPairs && cta >= gA.cta0 + gA.ncta;  // never when alone: its share is the whole grid
-  const PersistGroup& g = second ? gB : gA;      // the group whose fast path this CTA runs
-  const int gi_mine = gi + (second ? 1 : 0);
-  const int lc = cta - g.cta0;                   // index within the group's share of the grid
-  const PersistGroup& g_next = desc(gi + len);
-  const bool has_next = next_len > 0;
-  ctx.len = len;
-  uint32_t desc_word = 0;  // one word of the next descriptors, in flight during section A
-  if (tid < next_len * kDescWords)
-    desc_word = __ldg(reinterpret_cast<const uint32_t*>(p.groups + gi + len) + tid);
-  uint32_t* const desc_dst =
-      reinterpret_cast<uint32_t*>(smem + kOffDesc +
-                                  ((gi + len + (tid >= kDescWords ? 1 : 0)) & (kDescSlots - 1)) * 512) +
-      (tid >= kDescWords ? tid - kDescWords : tid);
+  // the group of phase [i, i + len) whose fast path this CTA runs
+  auto mine_of = [&](int i, int len) -> int {
+    if (!kPairs || len < 2) return i;
+    const PersistGroup& a = desc(i);
+    return cta >= a.cta0 + a.ncta ? i + 1 : i;
+  };
+  // warp 0: request this CTA's rows of x of group gn into buffer `buf`
+  auto request_x = [&](const PersistGroup& gn, int buf) {
+    if (gn.flags & GSI_FLAG_DENSE) return;
+    const Slab sn = slab_of(gn, cta - gn.cta0);
+    const float* src = gn.x + (long long)slot_io * gn.x_step_stride + (size_t)p.token * gn.d + sn.p0;
+    float* dst = s_xb + buf * kPersistMaxPRows;
+    for (int i = lane; i < sn.p1 - sn.p0; i += 32) cp_async4(dst + i, src + i);
+  };
 
-  const Slab s = slab_of(g, lc);
-  const float* x = g.x + (long long)slot_io * g.x_step_stride + (size_t)p.token * g.d;
-  float* const y_tok = g.y + (size_t)p.token * g.O;   // this launch's token
-  const bool dense = g.flags & GSI_FLAG_DENSE;
-  const bool zeroer = lc == gi_mine % g.ncta;  // this CTA clears the group's counters for the next launch
-  int gate = 1, gate_other = 0;
-  const float* rsrc = x;
+  // the first phase's descriptors (the second slot is used only if the phase is a pair)
+  if (tid < min(p.n_groups, 2) * kDescWords) {
+    const int j = tid >= kDescWords ? 1 : 0;
+    reinterpret_cast<uint32_t*>(smem + kOffDesc + j * 512)[tid - j * kDescWords] =
+        __ldg(reinterpret_cast<const uint32_t*>(p.groups) + tid);
+  }
+  if (tid == 0) {
+    misc->fire[0] = misc->fire[1] = misc->fire[2] = misc->fire[3] = 0;
+    misc->decision[0] = misc->decision[1] = misc->decision[2] = misc->decision[3] = 0u;
+  }
+  csync();
+  if (warp == 0) {
+    const int len0 = kPairs ? desc(0).phase_len : 1;
+    request_x(desc(mine_of(0, len0)), 0);
+    cp_async_commit();
+  }
 
-  if (!dense) {
-    const int k = kK ? kK : g.k;   // a build for one rank folds the whole lane geometry
-    Geo q;
-    q.KV = k >> 3;
-    q.lpr_log2 = q.KV >= 32 ? 5 : 31 - __clz(q.KV);
-    q.vpl = q.KV > 32 ? q.KV >> 5 : 1;
-    q.rc_log2 = 31 - __clz(kChunk / 2) - (31 - __clz(k));  // rows per chunk = 8192 / k
-    const int LPR = 1 << q.lpr_log2;
-    q.sub = lane >> q.lpr_log2;
-    q.cl = lane & (LPR - 1);
-    const int rpp_log2 = 5 - q.lpr_log2;  // rows per warp pass
-    const int rc = 1 << q.rc_log2;
-    const int n_contrib = (g.d + g.p_rows - 1) / g.p_rows;  // CTAs that own basis rows
-    unsigned long long* acc = g.acc_c + (size_t)parity * k * kAccStride;
+  int gi = 0;
+  int g_p = -1, len_p = 0;       // previous phase: its gates are settled in this tick
+  int g_pp = -1, len_pp = 0;     // the phase before: its gated residuals run in this tick
+  unsigned mask_pp = 0;
+  bool contrib_p = false;        // this CTA holds a partial ||r||^2 of the previous phase
+  int e_p = 0;                   // ... scaled by 2^(44 - e_p)
+  unsigned long long* r2word_p = nullptr;
+  bool ok = true;
+
+#pragma unroll 1
+  for (int t = 0; ok; ++t) {
+    const bool own = gi < p.n_groups;
+    if (!own && len_p == 0 && len_pp == 0) break;
+    int len = 0, next_len = 0, gi_mine = gi;
+    if (own) {
+      const PersistGroup& gA = desc(gi);
+      len = kPairs ? gA.phase_len : 1;
+      next_len = kPairs ? gA.next_len : min(gA.next_len, 1);
+      gi_mine = mine_of(gi, len);
+    }
+    const PersistGroup& g = desc(gi_mine);        // read only when `own`
+    const bool dense = own && (g.flags & GSI_FLAG_DENSE);
+    const bool gsi = own && !dense;
+    const int lc = own ? cta - g.cta0 : 0;
+    const int k = gsi ? (kK ? kK : g.k) : 0;
+    Slab s{};
+    if (gsi) s = slab_of(g, lc);
     const int prow = s.p1 - s.p0, orow = s.o1 - s.o0;
-    const int pchunks = (prow + rc - 1) >> q.rc_log2, ochunks = (orow + rc - 1) >> q.rc_log2;
+    float* s_x = s_xb + (t & 1) * kPersistMaxPRows;
+    unsigned long long* acc = gsi ? g.acc + (size_t)parity * (k + 2) * kAccStride : nullptr;
+    const int n_contrib = gsi ? (g.d + g.p_rows - 1) / g.p_rows : 0;
 
-    // ---- A. statistics of x (every CTA, the whole vector): max |x|, sum x^2,
-    //      non-finite flag; x of this CTA's basis rows goes to shared memory.
-    float amax = 0.f, sum2 = 0.f;
-    const int d4 = g.d >> 2;
+    Geo q{};
+    if (gsi) {
+      q.KV = k >> 3;
+      q.lpr_log2 = q.KV >= 32 ? 5 : 31 - __clz(q.KV);
+      q.vpl = q.KV > 32 ? q.KV >> 5 : 1;
+      q.rc_log2 = 31 - __clz(kChunk / 2) - (31 - __clz(k));  // rows per chunk = 8192 / k
+      q.sub = lane >> q.lpr_log2;
+      q.cl = lane & ((1 << q.lpr_log2) - 1);
+    }
+    const int LPR = 1 << q.lpr_log2, rpp_log2 = 5 - q.lpr_log2, rc = 1 << q.rc_log2;
+    const int pchunks = gsi ? (prow + rc - 1) >> q.rc_log2 : 0;
+    const int ochunks = gsi ? (orow + rc - 1) >> q.rc_log2 : 0;
+
+    // one word of the next phase's descriptors, in flight during the statistics
+    uint32_t desc_word = 0;
+    if (own && tid < next_len * kDescWords)
+      desc_word = __ldg(reinterpret_cast<const uint32_t*>(p.groups + gi + len) + tid);
+
+    // ---- A. statistics of this CTA's rows of x (warp 0), published at once
+    if (gsi && warp == 0) {
+      cp_async_wait_all();
+      __syncwarp();
+      float amax = 0.f, s2 = 0.f;
 #pragma unroll 1
-    for (int i0 = tid; i0 < d4; i0 += kXBatch * kNC) {   
-      float4 v[kXBatch];
-#pragma unroll
-      for (int u = 0; u < kXBatch; ++u) {
-        const int i4 = i0 + u * kNC;
-        v[u] = i4 < d4 ? __ldcg(reinterpret_cast<const float4*>(x) + i4) : make_float4(0, 0, 0, 0);
+      for (int i = lane; i < prow; i += 32) {
+        const float v = s_x[i];
+        amax = fmaxf(amax, fabsf(v));
+        s2 = fmaf(v, v, s2);
       }
 #pragma unroll
-      for (int u = 0; u < kXBatch; ++u) {
-        amax = fmaxf(fmaxf(amax, fmaxf(fabsf(v[u].x), fabsf(v[u].y))),
-                     fmaxf(fabsf(v[u].z), fabsf(v[u].w)));
-        sum2 = fmaf(v[u].x, v[u].x, sum2);
-        sum2 = fmaf(v[u].y, v[u].y, sum2);
-        sum2 = fmaf(v[u].z, v[u].z, sum2);
-        sum2 = fmaf(v[u].w, v[u].w, sum2);
+      for (int o = 16; o > 0; o >>= 1) {
+        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+        s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+      }
+      // fmaxf drops NaN, the sum keeps it (and overflows to inf for huge inputs):
+      // s2 - s2 is non-zero exactly when some x_i is NaN or inf (or x^2 overflowed)
+      if (lane == 0) {
+        const unsigned bits = (s2 - s2 == 0.f) ? __float_as_uint(amax) : 0x7fc00000u;
+        if (prow > 0) st_relaxed_u32(g.xmax + lc, bits | (tag << 31));
+        misc->x2_part = s2;
       }
     }
-    if (tid < prow) s_x[tid] = __ldcg(x + s.p0 + tid);
-    if (tid < next_len * kDescWords) *desc_dst = desc_word;
-    tr.mark(0);
-    // fmaxf drops NaN, the sum keeps it (and overflows to inf for huge inputs):
-    // sum2 - sum2 is non-zero exactly when some x_i is NaN or inf (or x^2 overflowed)
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-      sum2 += __shfl_xor_sync(0xffffffffu, sum2, o);
+    if (own && tid < next_len * kDescWords) {
+      uint32_t* dst = reinterpret_cast<uint32_t*>(
+                          smem + kOffDesc +
+                          ((gi + len + (tid >= kDescWords ? 1 : 0)) & (kDescSlots - 1)) * 512) +
+                      (tid >= kDescWords ? tid - kDescWords : tid);
+      *dst = desc_word;
     }
-    if (lane == 0) {   // s_vals is idle until this group's exchange 2
-      s_vals[warp * 2 + 0] = amax;
-      s_vals[warp * 2 + 1] = sum2;
-    }
-    if (tid == 0) misc->deposits = 0;
-    if (zeroer) {  // clear what the NEXT launch will accumulate into
+    if (tid == 0) misc->fire[(t & 1) * 2] = misc->fire[(t & 1) * 2 + 1] = 0;
+    if (own && lc == gi_mine % g.ncta) {  // this CTA clears the group's counters for the next launch
+      if (gsi) {
 #pragma unroll 1
-      for (int j = tid; j < k; j += kNC)
-        g.acc_c[((size_t)(parity ^ 1u) * k + j) * kAccStride] = 0ull;
-      if (tid < 3) g.bar[2 * tid + (parity ^ 1u)] = 0u;
+        for (int j = tid; j < k + 2; j += kNC)
+          g.acc[((size_t)(parity ^ 1u) * (k + 2) + j) * kAccStride] = 0ull;
+      }
+      if (tid < 2) g.bar[2 * tid + (parity ^ 1u)] = 0u;
     }
     csync();
-    if (has_next) prefetch_next_x(g_next, slot_io, p.n_tokens);
-    if (next_len == 2) prefetch_next_x(desc(gi + len + 1), slot_io, p.n_tokens, 1);
-    {  // every thread folds the warp partials in the same order
-      float a = 0.f, t = 0.f;
-#pragma unroll
-      for (int w = 0; w < kNW; ++w) {
-        a = fmaxf(a, s_vals[w * 2]);
-        t += s_vals[w * 2 + 1];
-      }
-      amax = a;
-      sum2 = t;
+    tr.mark(0);
+    if (warp == 0 && next_len > 0) {   // the next phase's rows of x travel while this phase runs
+      request_x(desc(mine_of(gi + len, next_len)), (t + 1) & 1);
+      cp_async_commit();
     }
-    const bool nonfinite = !(sum2 - sum2 == 0.f);
-    tr.mark(1);
-    // fixed-point scale: |partial c_j| <= amax * rows * max|P| < 2^e
-    double scale = 0.0, inv_scale = 0.0;
-    {
+
+    // ---- B. pass 1: partial c over this CTA's basis rows
+    const unsigned n_p0 = rg.n;
+    if (gsi) {
+      ok = chunks_landed(rg, n_p0, pchunks, abort);
+      tr.mark(1);
+#pragma unroll 1
+      for (int u = 0; u < q.vpl; ++u) {
+        const int cv = q.cl + u * LPR;
+        float a8[8];
+#pragma unroll
+        for (int e = 0; e < 8; ++e) a8[e] = 0.f;
+#pragma unroll 1
+        for (int ci = 0; ci < pchunks; ++ci) {
+          if (!ok) break;
+          const uint4* tile =
+              reinterpret_cast<const uint4*>(rg.slots + (size_t)((n_p0 + ci) % kSlots) * kChunk);
+          const int r_lo = ci << q.rc_log2, rows = min(rc, prow - r_lo);
+#pragma unroll 1
+          for (int row = (warp << rpp_log2) + q.sub; row < rows; row += kNW << rpp_log2) {
+            const float xv = s_x[r_lo + row];
+            const uint4 w = tile[(size_t)row * q.KV + cv];
+            a8[0] = fmaf(__uint_as_float(w.x << 16), xv, a8[0]);
+            a8[1] = fmaf(__uint_as_float(w.x & 0xFFFF0000u), xv, a8[1]);
+            a8[2] = fmaf(__uint_as_float(w.y << 16), xv, a8[2]);
+            a8[3] = fmaf(__uint_as_float(w.y & 0xFFFF0000u), xv, a8[3]);
+            a8[4] = fmaf(__uint_as_float(w.z << 16), xv, a8[4]);
+            a8[5] = fmaf(__uint_as_float(w.z & 0xFFFF0000u), xv, a8[5]);
+            a8[6] = fmaf(__uint_as_float(w.w << 16), xv, a8[6]);
+            a8[7] = fmaf(__uint_as_float(w.w & 0xFFFF0000u), xv, a8[7]);
+          }
+        }
+#pragma unroll 1
+        for (int o = LPR; o < 32; o <<= 1) {
+#pragma unroll
+          for (int e = 0; e < 8; ++e) a8[e] += __shfl_xor_sync(0xffffffffu, a8[e], o);
+        }
+        if (q.sub == 0) {
+          float4* dst = reinterpret_cast<float4*>(s_red + warp * 512 + cv * 8);
+          dst[0] = make_float4(a8[0], a8[1], a8[2], a8[3]);
+          dst[1] = make_float4(a8[4], a8[5], a8[6], a8[7]);
+        }
+      }
+      if (!ok && !*abort) fail(p, misc);
+      tr.mark(2);
+      // ---- C. the group's max |x|: warp 0 collects the tagged words (lane l owns words
+      //      l, l+32, ...), published about one pass earlier
+      if (warp == 0) {
+        unsigned m = 0, it = 0;
+        bool done = false;
+        while (!done) {
+          bool all = true;
+          m = 0;
+#pragma unroll
+          for (int i = 0; i < kPersistMaxGrid / 32; ++i) {
+            const int w_i = lane + 32 * i;
+            if (w_i < n_contrib) {
+              const unsigned w = ld_relaxed_u32(g.xmax + w_i);
+              all = all && ((w >> 31) == tag);
+              m = max(m, w & 0x7fffffffu);
+            }
+          }
+          done = __all_sync(0xffffffffu, all);
+          if (!done && (++it > p.spin_limit || ((it & 1023u) == 0 && *abort))) {
+            if (!*abort && lane == 0) fail(p, misc);
+            break;
+          }
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+        if (lane == 0) misc->amax_bits = m;
+      }
+    }
+    csync();
+    tr.mark(3);
+    if (*abort) return;
+
+    // ---- D. the exchange: this phase's partial c and ||x||^2, the previous phase's ||r||^2
+    bool nonfinite = false;
+    double inv_scale = 0.0;
+    if (gsi) {
+      const unsigned amax_bits = misc->amax_bits;
+      nonfinite = amax_bits >= 0x7f800000u;
+      const float amax = __uint_as_float(amax_bits);
+      // fixed-point scales: |partial c_j| <= amax * rows * max|P| < 2^e, partial ||x||^2 <= rows * amax^2 < 2^ex
+      double scale = 0.0, scale_x2 = 0.0;
       const float bound = amax * (float)g.p_rows * g.pmax;
       if (!nonfinite && bound > 0.f && bound < 3.0e38f) {
         const int e = max((int)((__float_as_uint(bound) >> 23) & 0xFFu), 1) - 126;
         scale = pow2d(43 - e);
         inv_scale = pow2d(e - 43);
+        scale_x2 = pow2d(43 - exp_above((double)amax * (double)amax * (double)g.p_rows));
       }
-    }
-
-    // ---- B. pass 1: partial c over this CTA's basis rows
-    const unsigned n_p0 = n;
-    bool ok = true;
-    {  // the basis chunks of this group: one per lane, all waits in flight together
-      bool mine_ok = true;
-      if (lane < pchunks) {
-        const unsigned seq = n_p0 + lane;
-        mine_ok = mbar_wait(&full[seq % kSlots], (seq / kSlots) & 1u, abort);
-      }
-      ok = __all_sync(0xffffffffu, mine_ok);
-    }
-    tr.mark(2);
+      if (prow > 0) {
 #pragma unroll 1
-    for (int u = 0; u < q.vpl; ++u) {
-      const int cv = q.cl + u * LPR;
-      float a8[8];
+        for (int j = tid; j < k; j += kNC) {
+          float sum = 0.f;
 #pragma unroll
-      for (int e = 0; e < 8; ++e) a8[e] = 0.f;
-#pragma unroll 1
-      for (int ci = 0; ci < pchunks; ++ci) {
-        if (!ok) break;
-        const unsigned sl = (n_p0 + ci) % kSlots;
-        const uint4* tile = reinterpret_cast<const uint4*>(ring + (size_t)sl * kChunk);
-        const int r_lo = ci << q.rc_log2, rows = min(rc, prow - r_lo);
-#pragma unroll 1
-        for (int row = (warp << rpp_log2) + q.sub; row < rows; row += kNW << rpp_log2) {
-          const float xv = s_x[r_lo + row];
-          const uint4 w = tile[(size_t)row * q.KV + cv];
-          a8[0] = fmaf(__uint_as_float(w.x << 16), xv, a8[0]);
-          a8[1] = fmaf(__uint_as_float(w.x & 0xFFFF0000u), xv, a8[1]);
-          a8[2] = fmaf(__uint_as_float(w.y << 16), xv, a8[2]);
-          a8[3] = fmaf(__uint_as_float(w.y & 0xFFFF0000u), xv, a8[3]);
-          a8[4] = fmaf(__uint_as_float(w.z << 16), xv, a8[4]);
-          a8[5] = fmaf(__uint_as_float(w.z & 0xFFFF0000u), xv, a8[5]);
-          a8[6] = fmaf(__uint_as_float(w.w << 16), xv, a8[6]);
-          a8[7] = fmaf(__uint_as_float(w.w & 0xFFFF0000u), xv, a8[7]);
+          for (int w = 0; w < kNW; ++w) sum += s_red[w * 512 + j];
+          const long long v = scale != 0.0 ? __double2ll_rn((double)sum * scale) : 0ll;
+          red_add_u64(acc + (size_t)j * kAccStride, kOne + (unsigned long long)v);
+        }
+        if (tid == kNC - 1) {
+          const long long v = scale_x2 != 0.0 ? __double2ll_rn((double)misc->x2_part * scale_x2) : 0ll;
+          red_add_u64(acc + (size_t)k * kAccStride, kOne + (unsigned long long)v);
         }
       }
-#pragma unroll 1
-      for (int o = LPR; o < 32; o <<= 1) {
-#pragma unroll
-        for (int e = 0; e < 8; ++e) a8[e] += __shfl_xor_sync(0xffffffffu, a8[e], o);
-      }
-      if (q.sub == 0) {
-        float4* dst = reinterpret_cast<float4*>(s_red + warp * 512 + cv * 8);
-        dst[0] = make_float4(a8[0], a8[1], a8[2], a8[3]);
-        dst[1] = make_float4(a8[4], a8[5], a8[6], a8[7]);
-      }
     }
-    if (!ok && !*abort) fail(p, misc);
-    tr.mark(3);
-    csync();
-    if (*abort) return false;
-    if (prow > 0) {
-#pragma unroll 1
-      for (int j = tid; j < k; j += kNC) {
-        float sum = 0.f;
+    if (contrib_p && tid == kNC - 2) {
+      float sr = 0.f;   // fixed order: the sum does not depend on which warp finished first
 #pragma unroll
-        for (int w = 0; w < kNW; ++w) sum += s_red[w * 512 + j];
-        const long long v = scale != 0.0 ? __double2ll_rn((double)sum * scale) : 0ll;
-        red_add_u64(acc + (size_t)j * kAccStride, (1ull << kCountShift) + (unsigned long long)v);
-      }
+      for (int w = 0; w < kNW; ++w) sr += misc->sr[w];
+      // at most 2^45 per CTA, so the sum of all CTAs stays below 2^53; a partial that large
+      // (||r||^2 > 2 ||x||^2) fires for every sensible eps
+      double vd = (double)sr * pow2d(44 - e_p);
+      if (!(vd < 35184372088832.0)) vd = 35184372088832.0;
+      if (!(vd >= 0.0)) vd = 0.0;
+      red_add_u64(r2word_p, kOne + (unsigned long long)__double2ll_rn(vd));
     }
     tr.mark(4);
 
-    // ---- C. exchange 1: wait until every contributing CTA has been added.  One
-    //      thread watches one word (thousands of pollers on the accumulators
-    //      would delay the very atomics they wait for); then every thread
-    //      validates its own word, which is normally complete by then.
-    if (tid == 0) {
-      const unsigned long long* wp = acc + (size_t)(k - 1) * kAccStride;
-      unsigned it = 0;
-      for (;;) {
-        const unsigned long long w = ld_relaxed_u64(wp);
-        if ((unsigned)((w + (1ull << (kCountShift - 1))) >> kCountShift) == (unsigned)n_contrib) break;
-        if (++it > kSpinLimit || ((it & 1023u) == 0 && *abort)) {
-          if (!*abort) fail(p, misc);
-          break;
-        }
-      }
-    }
-    csync();
-    if (*abort) return false;
+    // ---- E. wait until every contributing CTA has been added.  One thread watches one word
+    //      (thousands of pollers on the accumulators would delay the very atomics they wait
+    //      for); then every thread validates its own word, which is normally complete by then.
+    if (gsi) {
+      if (tid == 0) (void)poll_acc(acc + (size_t)(k - 1) * kAccStride, (unsigned)n_contrib, p, misc);
+      csync();
+      if (*abort) return;
 #pragma unroll 1
-    for (int j = tid; j < k; j += kNC) {
-      unsigned long long w = 0;
-      unsigned it = 0;
-      for (;;) {
-        w = ld_relaxed_u64(acc + (size_t)j * kAccStride);
-        const unsigned cnt = (unsigned)((w + (1ull << (kCountShift - 1))) >> kCountShift);
-        if (cnt == (unsigned)n_contrib) break;
-        if (++it > kSpinLimit || ((it & 1023u) == 0 && *abort)) {
-          if (!*abort) fail(p, misc);
-          break;
+      for (int j = tid; j < k; j += kNC) {
+        const long long val = poll_acc(acc + (size_t)j * kAccStride, (unsigned)n_contrib, p, misc);
+        s_c[j] = (float)((double)val * inv_scale);
+      }
+      if (tid == kNC - 1) {
+        const long long val = poll_acc(acc + (size_t)k * kAccStride, (unsigned)n_contrib, p, misc);
+        const double amax = (double)__uint_as_float(misc->amax_bits);
+        const double x2 = nonfinite ? __longlong_as_double(0x7ff8000000000000ll)
+                          : val > 0 ? (double)val * pow2d(exp_above(amax * amax * (double)g.p_rows) - 43)
+                                    : 0.0;
+        misc->x2 = x2;
+        // every CTA decides this group's gate in the next tick from the published value
+        if (lc == 0)
+          st_relaxed_u64(g.pub, ((unsigned long long)__double_as_longlong(x2) & ~(1ull << 63)) |
+                                    ((unsigned long long)tag << 63));
+      }
+    }
+    // the previous phase's gates: one thread per group collects ||r||^2 and ||x||^2 and decides
+    if (len_p > 0 && (tid == kNC - 3 || tid == kNC - 4) && kNC - 3 - tid < len_p) {
+      const int u = kNC - 3 - tid;
+      const PersistGroup* gp = p.groups + g_p + u;
+      const unsigned fl = __ldg(&gp->flags);
+      if (!(fl & GSI_FLAG_DENSE)) {
+        const int k_u = __ldg(&gp->k), d_u = __ldg(&gp->d), pr_u = __ldg(&gp->p_rows);
+        const unsigned n_u = (unsigned)((d_u + pr_u - 1) / pr_u);
+        const unsigned long long* acc_u =
+            reinterpret_cast<const unsigned long long*>(__ldg(reinterpret_cast<const unsigned long long*>(&gp->acc))) +
+            (size_t)parity * (k_u + 2) * kAccStride;
+        const unsigned long long* pub_u =
+            reinterpret_cast<const unsigned long long*>(__ldg(reinterpret_cast<const unsigned long long*>(&gp->pub)));
+        const long long val = poll_acc(acc_u + (size_t)(k_u + 1) * kAccStride, n_u, p, misc);
+        unsigned long long w = 0;
+        unsigned it = 0;
+        for (;;) {
+          w = ld_relaxed_u64(pub_u);
+          if ((unsigned)(w >> 63) == tag) break;
+          if (++it > p.spin_limit || ((it & 1023u) == 0 && *abort)) {
+            if (!*abort) fail(p, misc);
+            break;
+          }
+        }
+        const double x2 = __longlong_as_double((long long)(w & ~(1ull << 63)));
+        const bool finite = x2 == x2;
+        const double r2 = (double)val * pow2d((x2 > 0.0 ? exp_above(x2) : 0) - 44);
+        const double eps = (double)__ldg(&gp->eps);
+        // ||r|| < eps ||x||  <=>  ||r||^2 < eps^2 ||x||^2  (both sides >= 0); false for x = 0
+        const bool fast = finite && (r2 < eps * eps * x2);
+        misc->fire[(t & 1) * 2 + u] = (!fast && finite && !(fl & GSI_FLAG_STATIC_PROJECTION)) ? 1 : 0;
+        if (cta == 0) {
+          const size_t at = ((size_t)slot_io * p.log_step_stride + (g_p + u)) * p.n_tokens + p.token;
+          p.gate_log[at] = fast ? 0 : 1;
+          if (p.rho_log)
+            p.rho_log[at] = finite ? (float)sqrt(r2 / x2) : __int_as_float(0x7fc00000);
         }
       }
-      const long long val = (long long)(w - ((unsigned long long)n_contrib << kCountShift));
-      s_c[j] = (float)((double)val * inv_scale);
     }
     csync();
-    if (*abort) return false;
     tr.mark(5);
+    if (*abort) return;
 
-    // ---- D. pass 2 (residual rows of the basis chunks, still in the ring) and
-    //      the image rows: the same eight-rows-per-lane-group loop over both
-    const int hold_log2 = q.lpr_log2 - 3;  // lanes per held row after reduce8
-    // all image chunks of this group must have landed (they were prefetched)
-    // (one chunk per lane, all waits in flight together; the warp then agrees)
-    {
-      bool mine_ok = true;
-      if (lane < ochunks) {
-        const unsigned seq = n_p0 + pchunks + lane;
-        mine_ok = mbar_wait(&full[seq % kSlots], (seq / kSlots) & 1u, abort);
-      }
-      ok = __all_sync(0xffffffffu, ok && mine_ok);
+    // ---- F. hand the decision to the producer; a gated group's r and image rows must be
+    //      visible grid-wide before its W rows are streamed in the next tick: release fence
+    //      and arrival now, the wait comes then
+    const unsigned mask_p = (unsigned)misc->fire[(t & 1) * 2] | ((unsigned)misc->fire[(t & 1) * 2 + 1] << 1);
+    if (tid == 0 && t >= 1) {
+      misc->decision[(t - 1) & 3] = ((unsigned)t << 8) | mask_p;
+#pragma unroll 1
+      for (int u = 0; u < len_p; ++u)
+        if (mask_p & (1u << u)) {
+          __threadfence();
+          red_relaxed_u32(p.groups[g_p + u].bar + 2 + parity, 1u);
+        }
     }
-    tr.mark(7);
-    float sr = 0.f;
-    // ---- E (first half). exchange 2 is published as soon as the residual rows are done, by
-    //      the warp that hands in the last partial, so that its latency runs under the image
-    //      rows.  A word is the partial (non-negative, or NaN) with the parity of the launch
-    //      in its sign bit: the arrays start as zeros, the first launch writes sign 1, and
-    //      every launch rewrites every word, so a word of this launch cannot be mistaken for
-    //      the previous one's and no fence is needed for the decision.  148 partials are
-    //      five 128-byte lines that every CTA reads.
-    // A pair shares the first group's slot array: word cta is this CTA's partial of its own
-    // group, words G + u carry ||x||^2 of group u for the other half of the grid.
-    auto deposit = [&]() {
+    const double x2_own = gsi ? misc->x2 : 0.0;
+
+    // ---- G. pass 2: residual rows of the basis chunks (still in the ring)
+    const int itemsP = (prow + 7) >> 3, itemsO = (orow + 7) >> 3;
+    const int padP = ((itemsP + (1 << rpp_log2) - 1) >> rpp_log2) << rpp_log2;
+    const int padO = ((itemsO + (1 << rpp_log2) - 1) >> rpp_log2) << rpp_log2;
+    if (gsi) {
+      float sr = row_items<false>(q, rg, n_p0, pchunks, prow, 0, padP, s_c, s_x, g.r + s.p0, false, ok);
       sr = warp_sum(sr);
-      if (lane == 0) {
-        volatile float* part = s_red;
-        part[warp] = sr;
-        __threadfence_block();
-        if (atomicAdd(&misc->deposits, 1) == kNW - 1) {
-          __threadfence_block();
-          float t = 0.f;   // fixed order: the sum does not depend on who came last
-#pragma unroll
-          for (int w = 0; w < kNW; ++w) t += part[w];
-          unsigned* slots = reinterpret_cast<unsigned*>(gA.slot_r);
-          st_relaxed_u32(slots + cta, (__float_as_uint(t) & 0x7fffffffu) | (tag << 31));
-          if (len == 2 && lc == 0)
-            st_relaxed_u32(slots + G + (second ? 1 : 0),
-                           (__float_as_uint(sum2) & 0x7fffffffu) | (tag << 31));
-        }
-      }
-    };
-    // work items: lane groups take eight rows at a time, first of the basis slab, then of
-    // the image slab (rows per chunk are a multiple of 8, so an item stays inside a chunk);
-    // only items with rows are enumerated, rounded up to a whole warp of lane groups
-    const int itemsP = (prow + 7) >> 3, n_live = itemsP + ((orow + 7) >> 3);
-    const int n_items = ((n_live + (1 << rpp_log2) - 1) >> rpp_log2) << rpp_log2;
-    const int lanegroups = kNW << rpp_log2;          // lane groups in the CTA
-    // The warps that hold basis items run them alone: the others hand in an empty partial
-    // and start their image items only when the last basis item is done (named barrier 2:
-    // they wait, the basis warps only arrive), so the partial is published as early as
-    // possible.  Every warp takes part exactly once per phase, whatever `ok` says.
-    const bool basis_warp = (warp << rpp_log2) < itemsP;
-    bool deposited = !basis_warp;
-    if (!basis_warp) {
-      deposit();
-      asm volatile("bar.sync 2, %0;" ::"n"(kNC) : "memory");
+      if (lane == 0) misc->sr[warp] = sr;
+      rg.n += pchunks;
+      tr.mark(6);
     }
-    if (ok) {
-      int released = 0;  // chunks this warp has already given back to the producer
-#pragma unroll 1
-      for (int item = (warp << rpp_log2) + q.sub; item < n_items; item += lanegroups) {
-        const bool image = item >= itemsP;
-        const int row0g = (image ? item - itemsP : item) << 3;   // first row, within the slab
-        const int cj = row0g >> q.rc_log2;
-        const int ci = min((image ? pchunks : 0) + cj, pchunks + ochunks - 1);
-        // items come in chunk order: every chunk before this warp's current one is done
-        // (n_items is a multiple of the lane groups per warp, so the warp stays converged)
-        const int ci_warp = __shfl_sync(0xffffffffu, ci, 0);
-        if (lane == 0)
-          for (; released < ci_warp; ++released) mbar_arrive(&empty[(n_p0 + released) % kSlots]);
-        released = ci_warp;
-        const unsigned sl = (n_p0 + ci) % kSlots;
-        const uint4* tile = reinterpret_cast<const uint4*>(ring + (size_t)sl * kChunk);
-        const int r_lo = cj << q.rc_log2, rows = min(rc, (image ? orow : prow) - r_lo);
-        const int row0 = row0g & (rc - 1);
-        float v[8];
-        dot8(tile, s_c, q, row0, rows, v);
-        const float dot = reduce8(v, q.cl, LPR);
-        const int row = row0 + (q.cl >> hold_log2);
-        if ((q.cl & ((1 << hold_log2) - 1)) == 0 && row < rows) {
-          if (image) {
-            y_tok[s.o0 + r_lo + row] = nonfinite ? __int_as_float(0x7fc00000) : dot;
-          } else {
-            const float rv = s_x[r_lo + row] - dot;
-            g.r[s.p0 + r_lo + row] = rv;
-            sr = fmaf(rv, rv, sr);
-          }
-        }
-        // basis items come first: once none is left for this warp, its partial is final
-        if (!deposited && item - q.sub + lanegroups >= itemsP) {
-          deposit();
-          deposited = true;
-          asm volatile("bar.arrive 2, %0;" ::"n"(kNC) : "memory");
-        }
-      }
-      __syncwarp();
-      if (lane == 0) {
-#pragma unroll 1
-        for (; released < pchunks + ochunks; ++released)
-          mbar_arrive(&empty[(n_p0 + released) % kSlots]);
-      }
-    }
-    if (!deposited) {   // only after a failed wait: keep the barrier count whole
-      deposit();
-      asm volatile("bar.arrive 2, %0;" ::"n"(kNC) : "memory");
-    }
-    tr.mark(8);
-    if (!ok && !*abort) fail(p, misc);
-    n += pchunks + ochunks;
 
-    // ---- E (second half). exchange 2: collect, decide.
-    if (warp == 0) {
-      // one warp polls all words (lane l owns words l, l+32, ...); each word is
-      // validated by the launch parity in its sign bit
-      float vals[8];
-      unsigned it = 0;
-      bool done = false;
-      while (!done) {
-        bool all = true;
-#pragma unroll
-        for (int i = 0; i < 8; ++i) {
-          const int t = lane + 32 * i;
-          vals[i] = 0.f;
-          if (t < G + (len == 2 ? 2 : 0)) {
-            const unsigned w = ld_relaxed_u32(reinterpret_cast<const unsigned*>(gA.slot_r) + t);
-            all = all && ((w >> 31) == (tag & 1u));
-            vals[i] = __uint_as_float(w & 0x7fffffffu);
-          }
-        }
-        done = __all_sync(0xffffffffu, all);
-        if (!done && (++it > kSpinLimit || ((it & 1023u) == 0 && *abort))) {
-          if (!*abort && lane == 0) fail(p, misc);
-          break;
-        }
-      }
-#pragma unroll
-      for (int i = 0; i < 8; ++i) s_vals[lane + 32 * i] = vals[i];
-    }
-    csync();
-    tr.mark(10);
-    if (*abort) return false;
-    {  // every warp folds the slots of each group in the same fixed order
-      const int split = gA.ncta;   // the whole grid when the group is alone
-      float tA = 0.f, tB = 0.f;
-#pragma unroll
-      for (int i = 0; i < 8; ++i) {
-        const int t = lane + 32 * i;
-        const float v = s_vals[t];
-        tA += t < split ? v : 0.f;
-        tB += (t >= split && t < G) ? v : 0.f;
-      }
-      tA = warp_sum(tA);
-      if (len == 2) tB = warp_sum(tB);
-      // ||r|| < eps ||x||  <=>  ||r||^2 < eps^2 ||x||^2  (both sides >= 0); NaN compares false
-      const float t = second ? tB : tA;
-      const double e2 = (double)g.eps * (double)g.eps;
-      const bool fast = !nonfinite && ((double)t < e2 * (double)sum2);
-      gate = fast ? 0 : 1;
-      if (lc == 0 && tid == 0) {
-        const size_t at = ((size_t)slot_io * p.log_step_stride + gi_mine) * p.n_tokens + p.token;
-        p.gate_log[at] = (unsigned char)gate;
-        if (p.rho_log)
-          p.rho_log[at] = nonfinite ? __int_as_float(0x7fc00000) : sqrtf(__fdividef(t, sum2));
-      }
-      if (len == 2) {  // the partner's decision, from its partial sums and its ||x||^2
-        const PersistGroup& go = second ? gA : gB;
-        const float to = second ? tA : tB, s2o = s_vals[G + (second ? 0 : 1)];
-        const double e2o = (double)go.eps * (double)go.eps;
-        const bool finite_o = s2o - s2o == 0.f;
-        const bool fast_o = finite_o && ((double)to < e2o * (double)s2o);
-        gate_other = (!fast_o && finite_o && !(go.flags & GSI_FLAG_STATIC_PROJECTION)) ? 1 : 0;
-      }
-    }
-    gate = gate && !(g.flags & GSI_FLAG_STATIC_PROJECTION) && !nonfinite;
-    tr.mark(11);
-  } else {
-    if (zeroer && tid < 3) g.bar[2 * tid + (parity ^ 1u)] = 0u;
-    if (cta == 0 && tid == 0)
-      p.gate_log[((size_t)slot_io * p.log_step_stride + gi) * p.n_tokens + p.token] = 1;
-    if (tid < next_len * kDescWords) *desc_dst = desc_word;
-    csync();
-    if (has_next) prefetch_next_x(g_next, slot_io, p.n_tokens);
-    if (next_len == 2) prefetch_next_x(desc(gi + len + 1), slot_io, p.n_tokens, 1);
-  }
-
-  // ---- F. gated residual of every gated group of the phase, each with the whole grid
+    // ---- H. gated residuals of the phase before the previous one
+    if (mask_pp) {
 #pragma unroll 1
-  for (int u = 0; u < len; ++u) {
-    const PersistGroup& gg = u ? gB : gA;
-    const int fire = ((u == 1) == second) ? gate : gate_other;
-    if (!fire) continue;
-    if (!dense) {
-      // r (and the image rows of y) were written by other CTAs: make them visible grid-wide
-      // before anyone reads them (release fence, arrival count, acquire fence).  Only gated
-      // groups pay for this.
+      for (int u = 0; u < len_pp && ok; ++u) {
+        if (!(mask_pp & (1u << u))) continue;
+        const PersistGroup& gg = p.groups[g_pp + u];
+        if (tid == 0) {
+          grid_wait(gg.bar + 2 + parity, (unsigned)G, p, misc);
+          __threadfence();
+        }
+        csync();
+        if (*abort) return;
+        ok = w_stream(p, gg, gg.r, gg.y + (size_t)p.token * gg.O, false, smem, ctx, misc);
+      }
+      tr.mark(7);
+    }
+
+    // ---- I. image rows; or, for a dense group, its whole W stream and a grid barrier that
+    //      keeps the groups of a dense stack in model order
+    if (gsi) {
+      const unsigned n_o0 = rg.n;
+      ok = ok && chunks_landed(rg, n_o0, ochunks, abort);
+      tr.mark(8);
+      (void)row_items<true>(q, rg, n_o0, ochunks, orow, padP, padO, s_c, s_x,
+                            g.y + (size_t)p.token * g.O + s.o0, nonfinite, ok);
+      rg.n += ochunks;
+      if (!ok && !*abort) fail(p, misc);
+      tr.mark(9);
+    } else if (dense) {
+      const float* x = g.x + (long long)slot_io * g.x_step_stride + (size_t)p.token * g.d;
+      ok = ok && w_stream(p, g, x, g.y + (size_t)p.token * g.O, true, smem, ctx, misc);
       if (tid == 0) {
-        __threadfence();
-        grid_arrive_wait(gg.bar + 2 + parity, (unsigned)G, p, misc);
-        __threadfence();
+        red_relaxed_u32(g.bar + parity, 1u);
+        grid_wait(g.bar + parity, (unsigned)G, p, misc);
+        if (cta == 0)
+          p.gate_log[((size_t)slot_io * p.log_step_stride + gi) * p.n_tokens + p.token] = 1;
       }
       csync();
-      if (*abort) return false;
+      tr.mark(10);
     }
-    Slab sw;
-    sw.p0 = sw.p1 = 0;
-    sw.o0 = min(gg.O, cta * gg.o_rows_w);
-    sw.o1 = min(gg.O, sw.o0 + gg.o_rows_w);
-    gated_pass(gg, sw, dense ? rsrc : gg.r, gg.y + (size_t)p.token * gg.O, dense, smem);
-    csync();
-    tr.mark(12);
-    // A dense group has no exchange: a grid barrier keeps the groups of a dense stack in
-    // model order.  After a gated residual none is needed: no CTA passes exchange 1 of the
-    // next phase before every CTA has posted its partial there, which it does after this.
-    if (dense) {
-      if (tid == 0) grid_arrive_wait(gg.bar + parity, (unsigned)G, p, misc);
-      csync();
-      tr.mark(13);
-      if (*abort) return false;
-    }
-  }
-  return true;
-}
+    if (*abort) return;
 
-template <bool kPairs, int kK>
-__device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc) {
-  Ctx ctx;
-  ctx.step = p.use_counter ? *p.step : 0;
-  ctx.slot_io = ctx.step % p.n_steps;
-  const int epoch = *p.epoch;
-  ctx.parity = (unsigned)epoch & 1u;
-  ctx.tag = (unsigned)epoch + 1u;
-  ctx.n = 0;
-  ctx.tr.start(p);
-  // the first phase's descriptors (the second slot is used only if the phase is a pair)
-  if ((int)threadIdx.x < min(p.n_groups, 2) * kDescWords) {
-    const int j = threadIdx.x >= kDescWords ? 1 : 0;
-    reinterpret_cast<uint32_t*>(smem + kOffDesc + j * 512)[threadIdx.x - j * kDescWords] =
-        __ldg(reinterpret_cast<const uint32_t*>(p.groups) + threadIdx.x);
+    contrib_p = gsi && prow > 0;
+    if (gsi) {
+      e_p = x2_own > 0.0 ? exp_above(x2_own) : 0;
+      r2word_p = acc + (size_t)(k + 1) * kAccStride;
+    }
+    g_pp = g_p;
+    len_pp = len_p;
+    mask_pp = mask_p;
+    g_p = gi;
+    len_p = len;
+    gi += len;
   }
-  csync();
-  bool ok = true;
-  ctx.len = 1;
-#pragma unroll 1
-  for (int gi = 0; gi < p.n_groups && ok; gi += ctx.len) ok = group_phase<kPairs, kK>(p, smem, misc, ctx, gi);
   // Every CTA read the counters at its start and has since taken part in the
   // last group's exchange, so they may advance now.
-  if (blockIdx.x == 0 && threadIdx.x == 0 && ok) {
+  if (cta == 0 && tid == 0 && ok && !*abort) {
     *p.epoch = epoch + 1;
-    if (p.use_counter && p.advance) *p.step = ctx.step + 1;
+    if (p.use_counter && p.advance) *p.step = step + 1;
   }
 }
 
