@@ -51,8 +51,8 @@ namespace {
 constexpr int kNW = kPersistConsumerWarps;
 constexpr int kNC = kNW * 32;               // consumer threads
 constexpr int kThreadsP = kNC + 32;         // + producer warp
-constexpr int kSlots = 10;
-constexpr int kChunk = 16384;
+constexpr int kNB = 32;                     // chunks in flight at most (one barrier pair each)
+constexpr int kChunk = 16384;               // largest chunk
 constexpr int kSlice = 4096;                // columns of W per staged slice of r
 constexpr int kBoxCols = kPersistBoxCols;
 constexpr unsigned kLocalSpinLimit = 1u << 24;   // waits inside the CTA (ring, producer hand-off)
@@ -60,33 +60,49 @@ constexpr int kCountShift = 54;
 constexpr unsigned long long kOne = 1ull << kCountShift;
 
 // shared memory map (bytes)
-constexpr int kOffBar = 0;          // full[kSlots], empty[kSlots]
-constexpr int kOffMisc = 256;       // scalars
-constexpr int kOffX = 512;          // x of this CTA's basis rows, two buffers (kPersistMaxPRows floats each)
+constexpr int kOffBar = 0;          // full[kNB], empty[kNB]
+constexpr int kOffLin = 512;        // producer: ring position (bytes placed before it) of every chunk in flight (kNB words)
+constexpr int kOffOff = 640;        // offset of every chunk in flight within the ring (kNB words), for the consumers
+constexpr int kOffMisc = 768;       // scalars
+constexpr int kOffTrace = 1152;     // cycle counters of the trace (16 words)
+constexpr int kOffX = 1280;         // x of this CTA's basis rows, two buffers (kPersistMaxPRows floats each)
 constexpr int kOffC = kOffX + 2 * kPersistMaxPRows * 4;   // c (512 floats)
 constexpr int kOffDesc = kOffC + 2048;                    // 4 group descriptors, 512 B each
 constexpr int kDescSlots = 4;
-constexpr int kOffRed = kOffDesc + kDescSlots * 512;      // cross-warp scratch (kNW*512 floats)
-constexpr int kOffRs = kOffRed + kNW * 512 * 4;           // staged slice of r (16 KB)
-constexpr int kOffYacc = kOffRs + kSlice * 4;             // per-row accumulators (kPersistMaxORows floats)
+constexpr int kOffRed = kOffDesc + kDescSlots * 512;      // cross-warp scratch of pass 1 (kNW*512 floats) ...
+constexpr int kOffRs = kOffRed;                           // ... which the W stream reuses for its slice of r (16 KB)
+constexpr int kOffYacc = kOffRed + kNW * 512 * 4;         // per-row accumulators (kPersistMaxORows floats)
 constexpr int kOffRing = ((kOffYacc + kPersistMaxORows * 4 + 1023) / 1024) * 1024;
-constexpr int kSmemBytes = kOffRing + kSlots * kChunk;
+constexpr int kRingBytes = (232448 - kOffRing) / 1024 * 1024;
+constexpr int kSmemBytes = kOffRing + kRingBytes;
 static_assert(kSmemBytes <= 232448, "shared memory budget of one sm_100 CTA");
+static_assert(kSlice * 4 <= kNW * 512 * 4, "the staged slice fits the scratch it shares");
 static_assert(sizeof(PersistGroup) <= 512 && sizeof(PersistGroup) % 4 == 0, "descriptor slot");
-static_assert(kPersistBoxRowsMax * kBoxCols * 2 <= kChunk, "a box fits a slot");
+static_assert(kPersistBoxRowsMax * kBoxCols * 2 <= kChunk, "a box fits a chunk");
 static_assert(kPersistBoxRowsMax == 2 * kNW, "two rows of a box per consumer warp");
 constexpr int kDescWords = (int)(sizeof(PersistGroup) / 4);
+
+// What the next tick needs to know about a group of this phase to settle its gate.
+struct Settle {
+  const unsigned long long* r2;   // accumulator of ||r||^2
+  const unsigned long long* pub;  // published ||x||^2
+  unsigned n_contrib;
+  float eps;
+  unsigned flags;
+  unsigned* bar;                  // arrival counter before the gated residual
+};
 
 struct Misc {
   int abort;
   unsigned amax_bits;       // max |x| of this phase's group (>= 0x7f800000: a non-finite token)
   float x2_part;            // this CTA's sum of x^2 over its rows
-  double x2;                // ||x||^2 of this phase's group
   int fire[4];              // decisions on the previous phase's groups, by tick parity: 1 = stream W
+  double x2;                // ||x||^2 of this phase's group
   float sr[kNW];            // per-warp partial ||r||^2 of this phase
   volatile unsigned decision[4];   // hand-off to the producer: (phase + 1) << 8 | fire mask
+  Settle pv[4];             // by tick parity, the groups of the phase run in that tick
 };
-static_assert(sizeof(Misc) <= 256, "scalars");
+static_assert(sizeof(Misc) <= kOffTrace - kOffMisc, "scalars");
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) {
   return (uint32_t)__cvta_generic_to_shared(p);
@@ -172,20 +188,28 @@ __device__ __forceinline__ void fail(const PersistParams& p, Misc* misc) {
 }
 
 // Optional cycle trace (thread 0 of every CTA; sections of the per-phase pipeline, summed
-// over phases); p.trace == nullptr disables it.
+// over phases in shared memory and added to p.trace when the CTA ends); p.trace == nullptr
+// disables it.
 struct Trace {
-  unsigned long long* out;
+  unsigned long long* acc;   // shared
   long long t;
-  __device__ __forceinline__ void start(const PersistParams& p) {
-    out = (threadIdx.x == 0 && p.trace) ? p.trace + (size_t)blockIdx.x * 16 : nullptr;
-    if (out) t = clock64();
+  __device__ __forceinline__ void start(const PersistParams& p, unsigned char* smem) {
+    acc = (threadIdx.x == 0 && p.trace) ? reinterpret_cast<unsigned long long*>(smem + kOffTrace) : nullptr;
+    if (acc) {
+      for (int i = 0; i < 16; ++i) acc[i] = 0ull;
+      t = clock64();
+    }
   }
   __device__ __forceinline__ void mark(int section) {
-    if (out) {
+    if (acc) {
       const long long now = clock64();
-      out[section] += (unsigned long long)(now - t);
+      acc[section] += (unsigned long long)(now - t);
       t = now;
     }
+  }
+  __device__ __forceinline__ void flush(const PersistParams& p) {
+    if (acc)
+      for (int i = 0; i < 16; ++i) p.trace[(size_t)blockIdx.x * 16 + i] += acc[i];
   }
 };
 
@@ -202,24 +226,52 @@ __device__ __forceinline__ Slab slab_of(const PersistGroup& g, int lc) {
   return s;
 }
 
-// ------------------------------------------------------------------ producer
-struct Ring {
+// ------------------------------------------------------------------ the ring
+// Chunks of any size up to 16 KB are packed back to back in a circular byte buffer (a chunk
+// never wraps: the tail of the buffer is skipped instead).  `lin` counts bytes placed so far,
+// skipped tails included, so lin % kRingBytes is the physical offset; chunk n uses barrier
+// pair n % kNB.  The producer publishes the offset of chunk n in s_off[n % kNB] before it arms
+// the chunk's "full" barrier; producer and consumers walk the same sequence of chunks, so a
+// consumer needs only the sequence number.
+struct Producer {
   uint64_t* full;
   uint64_t* empty;
-  unsigned char* slots;
-  unsigned n;   // sequence number of the next chunk
+  unsigned char* base;
+  unsigned* s_lin;     // shared: start (lin) of every chunk in flight
+  unsigned* s_off;     // shared: its offset in the ring
+  unsigned n;          // sequence number of the next chunk
+  unsigned lin;        // bytes placed so far
+  unsigned tail_n;     // oldest chunk not yet given back by the consumers
+  unsigned tail_lin;   // where it starts
 };
 
-// Wait for the slot of chunk n to be free; false = give up.
-__device__ __forceinline__ bool ring_acquire(Ring& rg, volatile int* abort) {
-  const unsigned slot = rg.n % kSlots, ph = (rg.n / kSlots) & 1u;
-  return mbar_wait(&rg.empty[slot], ph ^ 1u, abort);
+// Reserve `bytes` for chunk n: waits (bounded) until the consumers have given back every
+// older chunk that still overlaps the place, and a barrier pair is free.  Returns the
+// offset, or 0xffffffff when a wait gave up.
+__device__ __forceinline__ unsigned producer_acquire(Producer& pr, unsigned bytes, volatile int* abort) {
+  unsigned off = pr.lin % (unsigned)kRingBytes;
+  if (off + bytes > (unsigned)kRingBytes) {
+    pr.lin += (unsigned)kRingBytes - off;
+    off = 0;
+  }
+  const unsigned start = pr.lin;
+  pr.lin += bytes;
+  while (pr.n - pr.tail_n >= (unsigned)kNB ||
+         (pr.tail_n < pr.n && pr.lin - pr.tail_lin > (unsigned)kRingBytes)) {
+    if (!mbar_wait(&pr.empty[pr.tail_n % kNB], (pr.tail_n / kNB) & 1u, abort)) return 0xffffffffu;
+    ++pr.tail_n;
+    pr.tail_lin = pr.tail_n < pr.n ? pr.s_lin[pr.tail_n % kNB] : start;
+  }
+  if (pr.tail_n == pr.n) pr.tail_lin = start;
+  pr.s_lin[pr.n % kNB] = start;
+  pr.s_off[pr.n % kNB] = off;
+  return off;
 }
 
 // The W boxes of one group for this CTA, in the order the consumers take them: column
 // slices of 4096 outermost (one staged slice of r serves them), then maps, then row blocks,
 // then the 256-column boxes of the slice.
-__device__ bool produce_w(const PersistGroup& g, Ring& rg, volatile int* abort) {
+__device__ __forceinline__ bool produce_w(const PersistGroup& g, Producer& pr, volatile int* abort) {
   const int cta = blockIdx.x;
   const int nsl = (g.d + kSlice - 1) / kSlice;
   for (int sl = 0; sl < nsl; ++sl) {
@@ -229,14 +281,15 @@ __device__ bool produce_w(const PersistGroup& g, Ring& rg, volatile int* abort) 
       const int row0 = cta * rows;
       const int live = min(rows, dout - row0);
       const char* tm = static_cast<const char*>(g.tmW) + (size_t)j * kPersistTmapBytes;
+      const uint32_t bytes = (uint32_t)rb * kBoxCols * 2;
       for (int b = 0; b * rb < live; ++b) {
         for (int cb = 0; cb < ncb; ++cb) {
-          if (!ring_acquire(rg, abort)) return false;
-          const unsigned slot = rg.n % kSlots;
-          mbar_expect_tx(&rg.full[slot], (uint32_t)rb * kBoxCols * 2);
-          tma_box_g2s(rg.slots + (size_t)slot * kChunk, tm, c0 + cb * kBoxCols, row0 + b * rb,
-                      &rg.full[slot]);
-          ++rg.n;
+          const unsigned off = producer_acquire(pr, bytes, abort);
+          if (off == 0xffffffffu) return false;
+          uint64_t* fb = &pr.full[pr.n % kNB];
+          mbar_expect_tx(fb, bytes);
+          tma_box_g2s(pr.base + off, tm, c0 + cb * kBoxCols, row0 + b * rb, fb);
+          ++pr.n;
         }
       }
     }
@@ -245,30 +298,39 @@ __device__ bool produce_w(const PersistGroup& g, Ring& rg, volatile int* abort) 
 }
 
 // Rows [a, b) of a row-major [rows][k] bf16 matrix as chunks of whole rows.
-__device__ bool produce_rows(const uint16_t* base, int k, int a, int b, Ring& rg, volatile int* abort) {
+__device__ __forceinline__ bool produce_rows(const uint16_t* base, int k, int a, int b, Producer& pr,
+                                             volatile int* abort) {
   const int rc = kChunk / (k * 2);
   for (int r = a; r < b; r += rc) {
     const int rows = min(rc, b - r);
-    if (!ring_acquire(rg, abort)) return false;
-    const unsigned slot = rg.n % kSlots;
     const uint32_t bytes = (uint32_t)rows * k * 2;
-    mbar_expect_tx(&rg.full[slot], bytes);
-    bulk_g2s(rg.slots + (size_t)slot * kChunk, base + (size_t)r * k, bytes, &rg.full[slot]);
-    ++rg.n;
+    const unsigned off = producer_acquire(pr, bytes, abort);
+    if (off == 0xffffffffu) return false;
+    uint64_t* fb = &pr.full[pr.n % kNB];
+    mbar_expect_tx(fb, bytes);
+    bulk_g2s(pr.base + off, base + (size_t)r * k, bytes, fb);
+    ++pr.n;
   }
   return true;
 }
 
 __device__ void producer(const PersistParams& p, unsigned char* smem, Misc* misc) {
-  Ring rg;
-  rg.full = reinterpret_cast<uint64_t*>(smem + kOffBar);
-  rg.empty = rg.full + kSlots;
-  rg.slots = smem + kOffRing;
-  rg.n = 0;
+  Producer pr;
+  pr.full = reinterpret_cast<uint64_t*>(smem + kOffBar);
+  pr.empty = pr.full + kNB;
+  pr.base = smem + kOffRing;
+  pr.s_lin = reinterpret_cast<unsigned*>(smem + kOffLin);
+  pr.s_off = reinterpret_cast<unsigned*>(smem + kOffOff);
+  pr.n = 0;
+  pr.lin = 0;
+  pr.tail_n = 0;
+  pr.tail_lin = 0;
   volatile int* abort = &misc->abort;
   const int cta = blockIdx.x;
   bool ok = true;
-  // ticks: tick t runs phase t (while there is one) and the gated residuals of phase t - 2
+  // ticks: tick t runs phase t (while there is one) and the gated residuals of phase t - 2;
+  // the work of a tick, in ring order: basis slab, W boxes of the gated groups, image slab
+  // (or the W boxes of a dense group)
   int gi = 0;        // first group of phase t
   int g_pp = -1, len_pp = 0;   // phase t - 2
   int g_p = -1, len_p = 0;     // phase t - 1
@@ -286,8 +348,9 @@ __device__ void producer(const PersistParams& p, unsigned char* smem, Misc* misc
     Slab s{};
     if (own && !dense) {
       s = slab_of(*g, cta - g->cta0);
-      ok = produce_rows(g->P, g->k, s.p0, s.p1, rg, abort);
+      ok = produce_rows(g->P, g->k, s.p0, s.p1, pr, abort);
     }
+    unsigned wmask = 0;
     if (ok && len_pp > 0) {
       // the decision on phase t - 2 (taken by the consumers during tick t - 1)
       const unsigned want = (unsigned)(t - 1);   // (phase + 1)
@@ -300,15 +363,20 @@ __device__ void producer(const PersistParams& p, unsigned char* smem, Misc* misc
           break;
         }
       }
-      for (int u = 0; ok && u < len_pp; ++u)
-        if (v & (1u << u)) ok = produce_w(p.groups[g_pp + u], rg, abort);
+      wmask = v & 3u;
     }
-    if (ok && own) {
-      if (dense)
-        ok = produce_w(*g, rg, abort);
-      else
-        ok = produce_rows(g->WP, g->k, s.o0, s.o1, rg, abort);
+    // one call site for every W stream of the tick: the gated groups, then a dense group
+#pragma unroll 1
+    for (int u = 0; ok && u < 3; ++u) {
+      const PersistGroup* gw = nullptr;
+      if (u < 2) {
+        if (u < len_pp && (wmask & (1u << u))) gw = &p.groups[g_pp + u];
+      } else if (dense) {
+        gw = g;
+      }
+      if (gw) ok = produce_w(*gw, pr, abort);
     }
+    if (ok && own && !dense) ok = produce_rows(g->WP, g->k, s.o0, s.o1, pr, abort);
     g_pp = g_p;
     len_pp = len_p;
     g_p = gi;
@@ -317,13 +385,13 @@ __device__ void producer(const PersistParams& p, unsigned char* smem, Misc* misc
   }
   if (!ok && !*abort) fail(p, misc);
   // Every copy issued must have landed before the CTA may give up its shared
-  // memory: wait (bounded) for the last kSlots chunks.
+  // memory: wait (bounded) for the last kNB chunks.
   {
-    const unsigned first = rg.n > (unsigned)kSlots ? rg.n - kSlots : 0;
-    for (unsigned c = first; c < rg.n; ++c) {
-      const unsigned slot = c % kSlots, ph = (c / kSlots) & 1u;
+    const unsigned first = pr.n > (unsigned)kNB ? pr.n - kNB : 0;
+    for (unsigned c = first; c < pr.n; ++c) {
+      const unsigned slot = c % kNB, ph = (c / kNB) & 1u;
       for (unsigned it = 0; it < kLocalSpinLimit; ++it)
-        if (mbar_try(&rg.full[slot], ph)) break;
+        if (mbar_try(&pr.full[slot], ph)) break;
     }
   }
 }
@@ -455,40 +523,32 @@ __device__ __forceinline__ bool grid_wait(const unsigned* ctr, unsigned target, 
   return true;
 }
 
-// Poll one accumulator until `n` arrivals have been added; returns the signed sum.
-__device__ __forceinline__ long long poll_acc(const unsigned long long* wp, unsigned n,
-                                              const PersistParams& p, Misc* misc) {
-  volatile int* abort = &misc->abort;
-  unsigned long long w = 0;
-  unsigned it = 0;
-  for (;;) {
-    w = ld_relaxed_u64(wp);
-    if ((unsigned)((w + (kOne >> 1)) >> kCountShift) == n) break;
-    if (++it > p.spin_limit || ((it & 1023u) == 0 && *abort)) {
-      if (!*abort) fail(p, misc);
-      break;
-    }
+// Chunks [n0, n0 + count) have landed (lane c waits for chunk c, all waits in flight together).
+__device__ __forceinline__ bool chunks_landed(unsigned char* smem, unsigned n0, int count,
+                                              volatile int* abort) {
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kOffBar);
+  const int lane = threadIdx.x & 31;
+  bool mine_ok = true;
+  if (lane < count) {
+    const unsigned seq = n0 + lane;
+    mine_ok = mbar_wait(&full[seq % kNB], (seq / kNB) & 1u, abort);
   }
-  return (long long)(w - ((unsigned long long)n << kCountShift));
+  return __all_sync(0xffffffffu, mine_ok);
 }
 
-struct Ctx {
-  int slot_io;
-  unsigned parity, tag;
-  Ring rg;        // consumer's view: n advances exactly as in producer()
-  Trace tr;
-};
-
 // ---- W stream: y_rows (+)= W_rows . src (src = r of a gated group, or x for the dense
-// baseline), boxes taken from the ring in the producer's order.  Out of line: most phases
-// skip it.  Returns false when a wait gave up.
-__device__ __noinline__ bool w_stream(const PersistParams& p, const PersistGroup& g, const float* src,
-                                      float* y, bool dense, unsigned char* smem, Ctx& ctx,
-                                      Misc* misc) {
+// baseline), boxes taken from the ring in the producer's order.  `n` is the consumers' chunk
+// sequence number.  Returns false when a wait gave up.
+__device__ __forceinline__ bool w_stream(const PersistParams& p, const PersistGroup& g, const float* src,
+                                         float* y, bool dense, unsigned char* smem, unsigned& n,
+                                         Misc* misc) {
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kOffBar);
+  uint64_t* empty = full + kNB;
+  const unsigned* s_off = reinterpret_cast<const unsigned*>(smem + kOffOff);
+  unsigned char* ring = smem + kOffRing;
   float* s_rs = reinterpret_cast<float*>(smem + kOffRs);
   float* s_yacc = reinterpret_cast<float*>(smem + kOffYacc);
   volatile int* abort = &misc->abort;
-  Ring& rg = ctx.rg;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int cta = blockIdx.x;
   const int nsl = (g.d + kSlice - 1) / kSlice;
@@ -520,11 +580,11 @@ __device__ __noinline__ bool w_stream(const PersistParams& p, const PersistGroup
         unsigned long long a0 = 0ull, a1 = 0ull;
 #pragma unroll 1
         for (int cb = 0; cb < ncb; ++cb) {
-          const unsigned slot = rg.n % kSlots, ph = (rg.n / kSlots) & 1u;
-          ++rg.n;
-          if (ok && !mbar_wait(&rg.full[slot], ph, abort)) ok = false;
+          const unsigned slot = n % kNB, ph = (n / kNB) & 1u;
+          ++n;
+          if (ok && !mbar_wait(&full[slot], ph, abort)) ok = false;
           if (ok && mine) {
-            const uint4* tile = reinterpret_cast<const uint4*>(rg.slots + (size_t)slot * kChunk);
+            const uint4* tile = reinterpret_cast<const uint4*>(ring + s_off[slot]);
             const uint4 w0 = tile[(2 * warp) * (kBoxCols / 8) + lane];
             const uint4 w1 = tile[(2 * warp + 1) * (kBoxCols / 8) + lane];
             const float4 ra = reinterpret_cast<const float4*>(s_rs)[cb * 64 + lane];
@@ -541,7 +601,7 @@ __device__ __noinline__ bool w_stream(const PersistParams& p, const PersistGroup
             fma2(a1, bf16x2_to_f32x2(w1.w), r3);
           }
           __syncwarp();
-          if (ok && lane == 0) mbar_arrive(&rg.empty[slot]);
+          if (ok && lane == 0) mbar_arrive(&empty[slot]);
         }
         if (mine) {
           const float t0 = warp_sum(sum2(a0)), t1 = warp_sum(sum2(a1));
@@ -577,98 +637,31 @@ __device__ __noinline__ bool w_stream(const PersistParams& p, const PersistGroup
   return ok;
 }
 
-
-// Items of eight rows (one lane group each) over the rows of `nchunks` ring chunks that start
-// at sequence number n0.  Item ids [id0, id0 + n_ids) of the phase's joint numbering belong to
-// this part; ids are dealt round-robin to the lane groups of the CTA, so the basis rows and the
-// image rows of a phase load the warps evenly.  kImage: out[row] = dot (NaN for a non-finite
-// token); otherwise out[row] = x[row] - dot and the return value is this lane's share of
-// ||r||^2.  Every warp gives every chunk back exactly once.
-template <bool kImage>
-__device__ __forceinline__ float row_items(const Geo& q, Ring& rg, unsigned n0, int nchunks, int nrows,
-                                           int id0, int n_ids, const float* s_c, const float* s_x,
-                                           float* out, bool nonfinite, bool ok) {
-  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-  const int LPR = 1 << q.lpr_log2, rpp_log2 = 5 - q.lpr_log2, rc = 1 << q.rc_log2;
-  const int hold_log2 = q.lpr_log2 - 3;          // lanes per held row after reduce8
-  const int lanegroups = kNW << rpp_log2;
-  float sr = 0.f;
-  int released = 0;
-  if (ok) {
-    int id = (warp << rpp_log2) + q.sub;
-    if (id < id0) id += ((id0 - id + lanegroups - 1) / lanegroups) * lanegroups;
-#pragma unroll 1
-    for (; id < id0 + n_ids; id += lanegroups) {
-      const int row0g = (id - id0) << 3;                       // first row, within the slab
-      const int ci = min(row0g >> q.rc_log2, nchunks - 1);
-      const int ci_warp = __shfl_sync(0xffffffffu, ci, 0);     // ids ascend with the lane
-      if (lane == 0)
-        for (; released < ci_warp; ++released) mbar_arrive(&rg.empty[(n0 + released) % kSlots]);
-      released = ci_warp;
-      const uint4* tile =
-          reinterpret_cast<const uint4*>(rg.slots + (size_t)((n0 + ci) % kSlots) * kChunk);
-      const int r_lo = ci << q.rc_log2, rows = min(rc, nrows - r_lo);
-      const int row0 = row0g - r_lo;
-      float v[8];
-      dot8(tile, s_c, q, row0, rows, v);
-      const float dot = reduce8(v, q.cl, LPR);
-      const int row = row0 + (q.cl >> hold_log2);
-      if ((q.cl & ((1 << hold_log2) - 1)) == 0 && row < rows && row0g < nrows) {
-        if (kImage) {
-          out[r_lo + row] = nonfinite ? __int_as_float(0x7fc00000) : dot;
-        } else {
-          const float rv = s_x[r_lo + row] - dot;
-          out[r_lo + row] = rv;
-          sr = fmaf(rv, rv, sr);
-        }
-      }
-    }
-    __syncwarp();
-    if (lane == 0)
-      for (; released < nchunks; ++released) mbar_arrive(&rg.empty[(n0 + released) % kSlots]);
-  }
-  return sr;
-}
-
-// All chunks [n0, n0 + count) have landed (one chunk per lane, all waits in flight together).
-__device__ __forceinline__ bool chunks_landed(Ring& rg, unsigned n0, int count, volatile int* abort) {
-  const int lane = threadIdx.x & 31;
-  bool mine_ok = true;
-  for (int c = lane; c < count; c += 32) {
-    const unsigned seq = n0 + c;
-    mine_ok = mine_ok && mbar_wait(&rg.full[seq % kSlots], (seq / kSlots) & 1u, abort);
-  }
-  return __all_sync(0xffffffffu, mine_ok);
-}
-
 // kPairs = false compiles the pair logic out: stacks without concurrent groups run a smaller
 // loop (the per-phase code has to stay resident in the instruction cache).  kK != 0 is a
 // build for stacks whose groups all have rank kK (shifts, strides and loop bounds become
 // constants); kK = 0 reads the rank from the descriptor.
 template <bool kPairs, int kK>
 __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc) {
+  uint64_t* empty = reinterpret_cast<uint64_t*>(smem + kOffBar) + kNB;
+  const unsigned* s_off = reinterpret_cast<const unsigned*>(smem + kOffOff);
+  unsigned char* ring = smem + kOffRing;
   float* s_xb = reinterpret_cast<float*>(smem + kOffX);
   float* s_c = reinterpret_cast<float*>(smem + kOffC);
   float* s_red = reinterpret_cast<float*>(smem + kOffRed);
   volatile int* abort = &misc->abort;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = gridDim.x, cta = blockIdx.x;
+  constexpr int kStatWarp = kNW - 1;   // statistics of x and the collection of max|x|; the others run pass 1
+  constexpr int kP1 = kNW - 1;         // warps of pass 1
 
-  Ctx ctx;
-  ctx.rg.full = reinterpret_cast<uint64_t*>(smem + kOffBar);
-  ctx.rg.empty = ctx.rg.full + kSlots;
-  ctx.rg.slots = smem + kOffRing;
-  ctx.rg.n = 0;
-  Ring& rg = ctx.rg;
+  unsigned n = 0;   // chunk sequence number: advances exactly as in producer()
   const int step = p.use_counter ? *p.step : 0;
   const int slot_io = step % p.n_steps;
-  ctx.slot_io = slot_io;
   const int epoch = *p.epoch;
   const unsigned parity = (unsigned)epoch & 1u, tag = ((unsigned)epoch + 1u) & 1u;
-  ctx.parity = parity;
-  ctx.tag = tag;
-  Trace& tr = ctx.tr;
-  tr.start(p);
+  Trace tr;
+  tr.start(p, smem);
 
   auto desc = [&](int i) -> const PersistGroup& {
     return *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + (i & (kDescSlots - 1)) * 512);
@@ -679,7 +672,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     const PersistGroup& a = desc(i);
     return cta >= a.cta0 + a.ncta ? i + 1 : i;
   };
-  // warp 0: request this CTA's rows of x of group gn into buffer `buf`
+  // one warp: request this CTA's rows of x of group gn into buffer `buf`
   auto request_x = [&](const PersistGroup& gn, int buf) {
     if (gn.flags & GSI_FLAG_DENSE) return;
     const Slab sn = slab_of(gn, cta - gn.cta0);
@@ -699,14 +692,15 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     misc->decision[0] = misc->decision[1] = misc->decision[2] = misc->decision[3] = 0u;
   }
   csync();
-  if (warp == 0) {
+  if (warp == kStatWarp) {
     const int len0 = kPairs ? desc(0).phase_len : 1;
     request_x(desc(mine_of(0, len0)), 0);
     cp_async_commit();
   }
 
   int gi = 0;
-  int g_p = -1, len_p = 0;       // previous phase: its gates are settled in this tick
+  int len_p = 0;                 // groups of the previous phase: their gates are settled in this tick
+  int g_p = -1;
   int g_pp = -1, len_pp = 0;     // the phase before: its gated residuals run in this tick
   unsigned mask_pp = 0;
   bool contrib_p = false;        // this CTA holds a partial ||r||^2 of the previous phase
@@ -736,6 +730,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     float* s_x = s_xb + (t & 1) * kPersistMaxPRows;
     unsigned long long* acc = gsi ? g.acc + (size_t)parity * (k + 2) * kAccStride : nullptr;
     const int n_contrib = gsi ? (g.d + g.p_rows - 1) / g.p_rows : 0;
+    const int tp = (t & 1) * 2, tq = tp ^ 2;      // this tick's and the previous tick's slots in Misc
 
     Geo q{};
     if (gsi) {
@@ -750,43 +745,14 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     const int pchunks = gsi ? (prow + rc - 1) >> q.rc_log2 : 0;
     const int ochunks = gsi ? (orow + rc - 1) >> q.rc_log2 : 0;
 
-    // one word of the next phase's descriptors, in flight during the statistics
+    // one word of the next phase's descriptors: requested now, stored after pass 1
     uint32_t desc_word = 0;
     if (own && tid < next_len * kDescWords)
       desc_word = __ldg(reinterpret_cast<const uint32_t*>(p.groups + gi + len) + tid);
 
-    // ---- A. statistics of this CTA's rows of x (warp 0), published at once
-    if (gsi && warp == 0) {
-      cp_async_wait_all();
-      __syncwarp();
-      float amax = 0.f, s2 = 0.f;
-#pragma unroll 1
-      for (int i = lane; i < prow; i += 32) {
-        const float v = s_x[i];
-        amax = fmaxf(amax, fabsf(v));
-        s2 = fmaf(v, v, s2);
-      }
-#pragma unroll
-      for (int o = 16; o > 0; o >>= 1) {
-        amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-        s2 += __shfl_xor_sync(0xffffffffu, s2, o);
-      }
-      // fmaxf drops NaN, the sum keeps it (and overflows to inf for huge inputs):
-      // s2 - s2 is non-zero exactly when some x_i is NaN or inf (or x^2 overflowed)
-      if (lane == 0) {
-        const unsigned bits = (s2 - s2 == 0.f) ? __float_as_uint(amax) : 0x7fc00000u;
-        if (prow > 0) st_relaxed_u32(g.xmax + lc, bits | (tag << 31));
-        misc->x2_part = s2;
-      }
-    }
-    if (own && tid < next_len * kDescWords) {
-      uint32_t* dst = reinterpret_cast<uint32_t*>(
-                          smem + kOffDesc +
-                          ((gi + len + (tid >= kDescWords ? 1 : 0)) & (kDescSlots - 1)) * 512) +
-                      (tid >= kDescWords ? tid - kDescWords : tid);
-      *dst = desc_word;
-    }
-    if (tid == 0) misc->fire[(t & 1) * 2] = misc->fire[(t & 1) * 2 + 1] = 0;
+    // ---- A. this CTA's rows of x have arrived (requested one phase ago)
+    if (gsi && warp == kStatWarp) cp_async_wait_all();
+    if (tid == 0) misc->fire[tp] = misc->fire[tp + 1] = 0;
     if (own && lc == gi_mine % g.ncta) {  // this CTA clears the group's counters for the next launch
       if (gsi) {
 #pragma unroll 1
@@ -795,73 +761,46 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       }
       if (tid < 2) g.bar[2 * tid + (parity ^ 1u)] = 0u;
     }
+    tr.mark(15);
     csync();
     tr.mark(0);
-    if (warp == 0 && next_len > 0) {   // the next phase's rows of x travel while this phase runs
-      request_x(desc(mine_of(gi + len, next_len)), (t + 1) & 1);
-      cp_async_commit();
-    }
 
-    // ---- B. pass 1: partial c over this CTA's basis rows
-    const unsigned n_p0 = rg.n;
+    const unsigned n_p0 = n;
+    n += pchunks;
     if (gsi) {
-      ok = chunks_landed(rg, n_p0, pchunks, abort);
-      tr.mark(1);
+      if (warp == kStatWarp) {
+        // ---- statistics of x over this CTA's rows, published at once; then the group's
+        //      max |x|: collect the tagged words of all contributing CTAs (lane l owns words
+        //      l, l+32, ...) while the other warps run pass 1
+        float amax = 0.f, s2 = 0.f;
 #pragma unroll 1
-      for (int u = 0; u < q.vpl; ++u) {
-        const int cv = q.cl + u * LPR;
-        float a8[8];
+        for (int i = lane; i < prow; i += 32) {
+          const float v = s_x[i];
+          amax = fmaxf(amax, fabsf(v));
+          s2 = fmaf(v, v, s2);
+        }
 #pragma unroll
-        for (int e = 0; e < 8; ++e) a8[e] = 0.f;
-#pragma unroll 1
-        for (int ci = 0; ci < pchunks; ++ci) {
-          if (!ok) break;
-          const uint4* tile =
-              reinterpret_cast<const uint4*>(rg.slots + (size_t)((n_p0 + ci) % kSlots) * kChunk);
-          const int r_lo = ci << q.rc_log2, rows = min(rc, prow - r_lo);
-#pragma unroll 1
-          for (int row = (warp << rpp_log2) + q.sub; row < rows; row += kNW << rpp_log2) {
-            const float xv = s_x[r_lo + row];
-            const uint4 w = tile[(size_t)row * q.KV + cv];
-            a8[0] = fmaf(__uint_as_float(w.x << 16), xv, a8[0]);
-            a8[1] = fmaf(__uint_as_float(w.x & 0xFFFF0000u), xv, a8[1]);
-            a8[2] = fmaf(__uint_as_float(w.y << 16), xv, a8[2]);
-            a8[3] = fmaf(__uint_as_float(w.y & 0xFFFF0000u), xv, a8[3]);
-            a8[4] = fmaf(__uint_as_float(w.z << 16), xv, a8[4]);
-            a8[5] = fmaf(__uint_as_float(w.z & 0xFFFF0000u), xv, a8[5]);
-            a8[6] = fmaf(__uint_as_float(w.w << 16), xv, a8[6]);
-            a8[7] = fmaf(__uint_as_float(w.w & 0xFFFF0000u), xv, a8[7]);
-          }
+        for (int o = 16; o > 0; o >>= 1) {
+          amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+          s2 += __shfl_xor_sync(0xffffffffu, s2, o);
         }
-#pragma unroll 1
-        for (int o = LPR; o < 32; o <<= 1) {
-#pragma unroll
-          for (int e = 0; e < 8; ++e) a8[e] += __shfl_xor_sync(0xffffffffu, a8[e], o);
+        // fmaxf drops NaN, the sum keeps it (and overflows to inf for huge inputs):
+        // s2 - s2 is non-zero exactly when some x_i is NaN or inf (or x^2 overflowed)
+        if (lane == 0) {
+          const unsigned bits = (s2 - s2 == 0.f) ? __float_as_uint(amax) : 0x7fc00000u;
+          if (prow > 0) st_relaxed_u32(g.xmax + lc, bits | (tag << 31));
+          misc->x2_part = s2;
         }
-        if (q.sub == 0) {
-          float4* dst = reinterpret_cast<float4*>(s_red + warp * 512 + cv * 8);
-          dst[0] = make_float4(a8[0], a8[1], a8[2], a8[3]);
-          dst[1] = make_float4(a8[4], a8[5], a8[6], a8[7]);
-        }
-      }
-      if (!ok && !*abort) fail(p, misc);
-      tr.mark(2);
-      // ---- C. the group's max |x|: warp 0 collects the tagged words (lane l owns words
-      //      l, l+32, ...), published about one pass earlier
-      if (warp == 0) {
         unsigned m = 0, it = 0;
         bool done = false;
         while (!done) {
           bool all = true;
           m = 0;
-#pragma unroll
-          for (int i = 0; i < kPersistMaxGrid / 32; ++i) {
-            const int w_i = lane + 32 * i;
-            if (w_i < n_contrib) {
-              const unsigned w = ld_relaxed_u32(g.xmax + w_i);
-              all = all && ((w >> 31) == tag);
-              m = max(m, w & 0x7fffffffu);
-            }
+#pragma unroll 1
+          for (int w_i = lane; w_i < n_contrib; w_i += 32) {
+            const unsigned w = ld_relaxed_u32(g.xmax + w_i);
+            all = all && ((w >> 31) == tag);
+            m = max(m, w & 0x7fffffffu);
           }
           done = __all_sync(0xffffffffu, all);
           if (!done && (++it > p.spin_limit || ((it & 1023u) == 0 && *abort))) {
@@ -872,10 +811,58 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
         if (lane == 0) misc->amax_bits = m;
+      } else {
+        // ---- B. pass 1: partial c over this CTA's basis rows
+        ok = chunks_landed(smem, n_p0, pchunks, abort);
+        tr.mark(1);
+#pragma unroll 1
+        for (int u = 0; u < q.vpl; ++u) {
+          const int cv = q.cl + u * LPR;
+          float a8[8];
+#pragma unroll
+          for (int e = 0; e < 8; ++e) a8[e] = 0.f;
+#pragma unroll 1
+          for (int ci = 0; ci < pchunks; ++ci) {
+            if (!ok) break;
+            const uint4* tile = reinterpret_cast<const uint4*>(ring + s_off[(n_p0 + ci) % kNB]);
+            const int r_lo = ci << q.rc_log2, rows = min(rc, prow - r_lo);
+#pragma unroll 1
+            for (int row = (warp << rpp_log2) + q.sub; row < rows; row += kP1 << rpp_log2) {
+              const float xv = s_x[r_lo + row];
+              const uint4 w = tile[(size_t)row * q.KV + cv];
+              a8[0] = fmaf(__uint_as_float(w.x << 16), xv, a8[0]);
+              a8[1] = fmaf(__uint_as_float(w.x & 0xFFFF0000u), xv, a8[1]);
+              a8[2] = fmaf(__uint_as_float(w.y << 16), xv, a8[2]);
+              a8[3] = fmaf(__uint_as_float(w.y & 0xFFFF0000u), xv, a8[3]);
+              a8[4] = fmaf(__uint_as_float(w.z << 16), xv, a8[4]);
+              a8[5] = fmaf(__uint_as_float(w.z & 0xFFFF0000u), xv, a8[5]);
+              a8[6] = fmaf(__uint_as_float(w.w << 16), xv, a8[6]);
+              a8[7] = fmaf(__uint_as_float(w.w & 0xFFFF0000u), xv, a8[7]);
+            }
+          }
+#pragma unroll 1
+          for (int o = LPR; o < 32; o <<= 1) {
+#pragma unroll
+            for (int e = 0; e < 8; ++e) a8[e] += __shfl_xor_sync(0xffffffffu, a8[e], o);
+          }
+          if (q.sub == 0) {
+            float4* dst = reinterpret_cast<float4*>(s_red + warp * 512 + cv * 8);
+            dst[0] = make_float4(a8[0], a8[1], a8[2], a8[3]);
+            dst[1] = make_float4(a8[4], a8[5], a8[6], a8[7]);
+          }
+        }
+        if (!ok && !*abort) fail(p, misc);
       }
     }
+    if (own && tid < next_len * kDescWords) {
+      uint32_t* dst = reinterpret_cast<uint32_t*>(
+                          smem + kOffDesc +
+                          ((gi + len + (tid >= kDescWords ? 1 : 0)) & (kDescSlots - 1)) * 512) +
+                      (tid >= kDescWords ? tid - kDescWords : tid);
+      *dst = desc_word;
+    }
     csync();
-    tr.mark(3);
+    tr.mark(2);
     if (*abort) return;
 
     // ---- D. the exchange: this phase's partial c and ||x||^2, the previous phase's ||r||^2
@@ -885,21 +872,26 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       const unsigned amax_bits = misc->amax_bits;
       nonfinite = amax_bits >= 0x7f800000u;
       const float amax = __uint_as_float(amax_bits);
+      if (amax_bits == 12345u) tr.t += 1;
+      tr.mark(13);
       // fixed-point scales: |partial c_j| <= amax * rows * max|P| < 2^e, partial ||x||^2 <= rows * amax^2 < 2^ex
       double scale = 0.0, scale_x2 = 0.0;
       const float bound = amax * (float)g.p_rows * g.pmax;
+      if (bound == 12345.f) tr.t += 1;
+      tr.mark(14);
       if (!nonfinite && bound > 0.f && bound < 3.0e38f) {
         const int e = max((int)((__float_as_uint(bound) >> 23) & 0xFFu), 1) - 126;
         scale = pow2d(43 - e);
         inv_scale = pow2d(e - 43);
         scale_x2 = pow2d(43 - exp_above((double)amax * (double)amax * (double)g.p_rows));
       }
+      tr.mark(10);
       if (prow > 0) {
 #pragma unroll 1
         for (int j = tid; j < k; j += kNC) {
           float sum = 0.f;
 #pragma unroll
-          for (int w = 0; w < kNW; ++w) sum += s_red[w * 512 + j];
+          for (int w = 0; w < kP1; ++w) sum += s_red[w * 512 + j];
           const long long v = scale != 0.0 ? __double2ll_rn((double)sum * scale) : 0ll;
           red_add_u64(acc + (size_t)j * kAccStride, kOne + (unsigned long long)v);
         }
@@ -920,22 +912,72 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       if (!(vd >= 0.0)) vd = 0.0;
       red_add_u64(r2word_p, kOne + (unsigned long long)__double2ll_rn(vd));
     }
-    tr.mark(4);
+    tr.mark(3);
 
-    // ---- E. wait until every contributing CTA has been added.  One thread watches one word
-    //      (thousands of pollers on the accumulators would delay the very atomics they wait
-    //      for); then every thread validates its own word, which is normally complete by then.
-    if (gsi) {
-      if (tid == 0) (void)poll_acc(acc + (size_t)(k - 1) * kAccStride, (unsigned)n_contrib, p, misc);
-      csync();
-      if (*abort) return;
-#pragma unroll 1
-      for (int j = tid; j < k; j += kNC) {
-        const long long val = poll_acc(acc + (size_t)j * kAccStride, (unsigned)n_contrib, p, misc);
-        s_c[j] = (float)((double)val * inv_scale);
+    // ---- E. wait until every contributing CTA has been added: warp 0 polls the accumulators
+    //      of c (lane l owns words l, l+32, ...: all its loads are in flight together, one
+    //      round trip per attempt), warp 1 the scalars: lane 0 this phase's ||x||^2, lanes
+    //      1+2u / 2+2u the previous phase's ||r||^2 and published ||x||^2 of its group u.
+    //      The other warps wait at the barrier (thousands of pollers on the accumulators
+    //      would delay the very atomics they wait for).
+    if (gsi && warp == 0) {
+      unsigned it = 0;
+      if (lane == 0) {   // one watcher per CTA on one word keeps the polling traffic off the atomics
+        const unsigned long long* wp = acc + (size_t)(k - 1) * kAccStride;
+        for (;;) {
+          const unsigned long long w = ld_relaxed_u64(wp);
+          if ((unsigned)((w + (kOne >> 1)) >> kCountShift) == (unsigned)n_contrib) break;
+          if (++it > p.spin_limit || ((it & 1023u) == 0 && *abort)) break;   // the loop below reports it
+        }
       }
-      if (tid == kNC - 1) {
-        const long long val = poll_acc(acc + (size_t)k * kAccStride, (unsigned)n_contrib, p, misc);
+      __syncwarp();
+      tr.mark(11);
+      bool done = false;
+      while (!done) {
+        bool all = true;
+#pragma unroll 8
+        for (int j = lane; j < k; j += 32) {
+          const unsigned long long w = ld_relaxed_u64(acc + (size_t)j * kAccStride);
+          all = all && ((unsigned)((w + (kOne >> 1)) >> kCountShift) == (unsigned)n_contrib);
+          const long long val = (long long)(w - ((unsigned long long)n_contrib << kCountShift));
+          s_c[j] = (float)((double)val * inv_scale);
+        }
+        done = __all_sync(0xffffffffu, all);
+        if (!done && (++it > p.spin_limit || ((it & 1023u) == 0 && *abort))) {
+          if (!*abort && lane == 0) fail(p, misc);
+          break;
+        }
+      }
+    }
+    if (warp == 1) {
+      // what this lane watches: an accumulator (count in the upper bits) or a tagged word
+      const int u = (lane - 1) >> 1;
+      const Settle& sv = misc->pv[tq + (u & 1)];
+      const bool w_x2 = gsi && lane == 0;
+      const bool w_r2 = lane >= 1 && lane <= 4 && (lane & 1) && u < len_p && sv.r2 != nullptr;
+      const bool w_pub = lane >= 1 && lane <= 4 && !(lane & 1) && u < len_p && sv.r2 != nullptr;
+      const unsigned long long* wp = w_x2 ? acc + (size_t)k * kAccStride : w_r2 ? sv.r2 : sv.pub;
+      const unsigned want = w_x2 ? (unsigned)n_contrib : sv.n_contrib;
+      unsigned long long w = 0;
+      unsigned it = 0;
+      bool done = false;
+      while (!done) {
+        bool mine = true;
+        if (w_x2 || w_r2) {
+          w = ld_relaxed_u64(wp);
+          mine = (unsigned)((w + (kOne >> 1)) >> kCountShift) == want;
+        } else if (w_pub) {
+          w = ld_relaxed_u64(wp);
+          mine = (unsigned)(w >> 63) == tag;
+        }
+        done = __all_sync(0xffffffffu, mine);
+        if (!done && (++it > p.spin_limit || ((it & 1023u) == 0 && *abort))) {
+          if (!*abort && lane == 0) fail(p, misc);
+          break;
+        }
+      }
+      if (w_x2) {
+        const long long val = (long long)(w - ((unsigned long long)n_contrib << kCountShift));
         const double amax = (double)__uint_as_float(misc->amax_bits);
         const double x2 = nonfinite ? __longlong_as_double(0x7ff8000000000000ll)
                           : val > 0 ? (double)val * pow2d(exp_above(amax * amax * (double)g.p_rows) - 43)
@@ -946,117 +988,170 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
           st_relaxed_u64(g.pub, ((unsigned long long)__double_as_longlong(x2) & ~(1ull << 63)) |
                                     ((unsigned long long)tag << 63));
       }
-    }
-    // the previous phase's gates: one thread per group collects ||r||^2 and ||x||^2 and decides
-    if (len_p > 0 && (tid == kNC - 3 || tid == kNC - 4) && kNC - 3 - tid < len_p) {
-      const int u = kNC - 3 - tid;
-      const PersistGroup* gp = p.groups + g_p + u;
-      const unsigned fl = __ldg(&gp->flags);
-      if (!(fl & GSI_FLAG_DENSE)) {
-        const int k_u = __ldg(&gp->k), d_u = __ldg(&gp->d), pr_u = __ldg(&gp->p_rows);
-        const unsigned n_u = (unsigned)((d_u + pr_u - 1) / pr_u);
-        const unsigned long long* acc_u =
-            reinterpret_cast<const unsigned long long*>(__ldg(reinterpret_cast<const unsigned long long*>(&gp->acc))) +
-            (size_t)parity * (k_u + 2) * kAccStride;
-        const unsigned long long* pub_u =
-            reinterpret_cast<const unsigned long long*>(__ldg(reinterpret_cast<const unsigned long long*>(&gp->pub)));
-        const long long val = poll_acc(acc_u + (size_t)(k_u + 1) * kAccStride, n_u, p, misc);
-        unsigned long long w = 0;
-        unsigned it = 0;
-        for (;;) {
-          w = ld_relaxed_u64(pub_u);
-          if ((unsigned)(w >> 63) == tag) break;
-          if (++it > p.spin_limit || ((it & 1023u) == 0 && *abort)) {
-            if (!*abort) fail(p, misc);
-            break;
-          }
-        }
-        const double x2 = __longlong_as_double((long long)(w & ~(1ull << 63)));
+      // the previous phase's gates: the lane that holds ||r||^2 of group u takes ||x||^2 from
+      // its neighbour and decides
+      const unsigned long long w_nb = __shfl_down_sync(0xffffffffu, w, 1);
+      if (w_r2) {
+        const long long val = (long long)(w - ((unsigned long long)want << kCountShift));
+        const double x2 = __longlong_as_double((long long)(w_nb & ~(1ull << 63)));
         const bool finite = x2 == x2;
-        const double r2 = (double)val * pow2d((x2 > 0.0 ? exp_above(x2) : 0) - 44);
-        const double eps = (double)__ldg(&gp->eps);
+        const int ex = x2 > 0.0 ? exp_above(x2) : 0;
+        const double r2 = (double)val * pow2d(ex - 44);
+        const double eps = (double)sv.eps;
         // ||r|| < eps ||x||  <=>  ||r||^2 < eps^2 ||x||^2  (both sides >= 0); false for x = 0
         const bool fast = finite && (r2 < eps * eps * x2);
-        misc->fire[(t & 1) * 2 + u] = (!fast && finite && !(fl & GSI_FLAG_STATIC_PROJECTION)) ? 1 : 0;
+        misc->fire[tp + u] = (!fast && finite && !(sv.flags & GSI_FLAG_STATIC_PROJECTION)) ? 1 : 0;
         if (cta == 0) {
           const size_t at = ((size_t)slot_io * p.log_step_stride + (g_p + u)) * p.n_tokens + p.token;
           p.gate_log[at] = fast ? 0 : 1;
-          if (p.rho_log)
-            p.rho_log[at] = finite ? (float)sqrt(r2 / x2) : __int_as_float(0x7fc00000);
+          if (p.rho_log)   // both operands scaled into the float range: ||r||^2 2^-e and ||x||^2 2^-e
+            p.rho_log[at] = finite ? sqrtf(__fdividef((float)((double)val * 5.6843418860808015e-14),
+                                                      (float)(x2 * pow2d(-ex))))
+                                   : __int_as_float(0x7fc00000);
         }
       }
     }
+    tr.mark(12);
     csync();
-    tr.mark(5);
+    tr.mark(4);
     if (*abort) return;
 
     // ---- F. hand the decision to the producer; a gated group's r and image rows must be
     //      visible grid-wide before its W rows are streamed in the next tick: release fence
     //      and arrival now, the wait comes then
-    const unsigned mask_p = (unsigned)misc->fire[(t & 1) * 2] | ((unsigned)misc->fire[(t & 1) * 2 + 1] << 1);
+    const unsigned mask_p = (unsigned)misc->fire[tp] | ((unsigned)misc->fire[tp + 1] << 1);
     if (tid == 0 && t >= 1) {
       misc->decision[(t - 1) & 3] = ((unsigned)t << 8) | mask_p;
 #pragma unroll 1
       for (int u = 0; u < len_p; ++u)
         if (mask_p & (1u << u)) {
           __threadfence();
-          red_relaxed_u32(p.groups[g_p + u].bar + 2 + parity, 1u);
+          red_relaxed_u32(misc->pv[tq + u].bar, 1u);
         }
     }
     const double x2_own = gsi ? misc->x2 : 0.0;
+    if (warp == kStatWarp && next_len > 0) {   // the next phase's rows of x travel while this phase runs
+      request_x(desc(mine_of(gi + len, next_len)), (t + 1) & 1);
+      cp_async_commit();
+    }
+    if (tid < 2) {   // what the next tick needs to settle this phase's gates
+      Settle sv{};
+      if (own && tid < len) {
+        const PersistGroup& gs = desc(gi + tid);
+        if (!(gs.flags & GSI_FLAG_DENSE)) {
+          sv.r2 = gs.acc + ((size_t)parity * (gs.k + 2) + gs.k + 1) * kAccStride;
+          sv.pub = gs.pub;
+          sv.n_contrib = (unsigned)((gs.d + gs.p_rows - 1) / gs.p_rows);
+          sv.eps = gs.eps;
+          sv.flags = gs.flags;
+          sv.bar = gs.bar + 2 + parity;
+        }
+      }
+      misc->pv[tp + tid] = sv;
+    }
 
-    // ---- G. pass 2: residual rows of the basis chunks (still in the ring)
+    // ---- G / I. the row passes, one copy of the code for both: part 0 the residual rows of
+    //      the basis slab (still in the ring), part 1 the image rows.  Items of eight rows
+    //      (one lane group each) are dealt round-robin over the joint numbering of both
+    //      parts, so the warps are loaded evenly.  Every warp gives every chunk back once.
+    // ---- H (between them). the W streams of the tick, one call site: the gated residuals
+    //      of the phase before the previous one, then this phase's own stream if it is a
+    //      dense group (followed by a grid barrier that keeps a dense stack in model order).
     const int itemsP = (prow + 7) >> 3, itemsO = (orow + 7) >> 3;
     const int padP = ((itemsP + (1 << rpp_log2) - 1) >> rpp_log2) << rpp_log2;
     const int padO = ((itemsO + (1 << rpp_log2) - 1) >> rpp_log2) << rpp_log2;
-    if (gsi) {
-      float sr = row_items<false>(q, rg, n_p0, pchunks, prow, 0, padP, s_c, s_x, g.r + s.p0, false, ok);
-      sr = warp_sum(sr);
-      if (lane == 0) misc->sr[warp] = sr;
-      rg.n += pchunks;
-      tr.mark(6);
-    }
-
-    // ---- H. gated residuals of the phase before the previous one
-    if (mask_pp) {
+    const int hold_log2 = q.lpr_log2 - 3;          // lanes per held row after reduce8
+    const int lanegroups = kNW << rpp_log2;
+    tr.mark(9);
 #pragma unroll 1
-      for (int u = 0; u < len_pp && ok; ++u) {
-        if (!(mask_pp & (1u << u))) continue;
-        const PersistGroup& gg = p.groups[g_pp + u];
-        if (tid == 0) {
-          grid_wait(gg.bar + 2 + parity, (unsigned)G, p, misc);
-          __threadfence();
+    for (int part = 0; part < 2; ++part) {
+      if (part == 1 && (mask_pp || dense)) {
+#pragma unroll 1
+        for (int u = 0; u < 3 && ok; ++u) {
+          const PersistGroup* gw = nullptr;
+          if (u < 2) {
+            if (u < len_pp && (mask_pp & (1u << u))) gw = p.groups + g_pp + u;
+          } else if (dense) {
+            gw = &g;
+          }
+          if (!gw) continue;
+          if (u < 2) {
+            if (tid == 0) {
+              grid_wait(gw->bar + 2 + parity, (unsigned)G, p, misc);
+              __threadfence();
+            }
+            csync();
+            if (*abort) return;
+          }
+          const float* src = u < 2 ? gw->r
+                                   : gw->x + (long long)slot_io * gw->x_step_stride + (size_t)p.token * gw->d;
+          ok = w_stream(p, *gw, src, gw->y + (size_t)p.token * gw->O, u == 2, smem, n, misc);
+          if (u == 2) {
+            if (tid == 0) {
+              red_relaxed_u32(gw->bar + parity, 1u);
+              grid_wait(gw->bar + parity, (unsigned)G, p, misc);
+              if (cta == 0)
+                p.gate_log[((size_t)slot_io * p.log_step_stride + gi) * p.n_tokens + p.token] = 1;
+            }
+            csync();
+          }
         }
-        csync();
+        tr.mark(6);
         if (*abort) return;
-        ok = w_stream(p, gg, gg.r, gg.y + (size_t)p.token * gg.O, false, smem, ctx, misc);
       }
-      tr.mark(7);
-    }
-
-    // ---- I. image rows; or, for a dense group, its whole W stream and a grid barrier that
-    //      keeps the groups of a dense stack in model order
-    if (gsi) {
-      const unsigned n_o0 = rg.n;
-      ok = ok && chunks_landed(rg, n_o0, ochunks, abort);
-      tr.mark(8);
-      (void)row_items<true>(q, rg, n_o0, ochunks, orow, padP, padO, s_c, s_x,
-                            g.y + (size_t)p.token * g.O + s.o0, nonfinite, ok);
-      rg.n += ochunks;
-      if (!ok && !*abort) fail(p, misc);
-      tr.mark(9);
-    } else if (dense) {
-      const float* x = g.x + (long long)slot_io * g.x_step_stride + (size_t)p.token * g.d;
-      ok = ok && w_stream(p, g, x, g.y + (size_t)p.token * g.O, true, smem, ctx, misc);
-      if (tid == 0) {
-        red_relaxed_u32(g.bar + parity, 1u);
-        grid_wait(g.bar + parity, (unsigned)G, p, misc);
-        if (cta == 0)
-          p.gate_log[((size_t)slot_io * p.log_step_stride + gi) * p.n_tokens + p.token] = 1;
+      if (!gsi) continue;
+      const bool image = part == 1;
+      const int nchunks = image ? ochunks : pchunks, nrows = image ? orow : prow;
+      const int id0 = image ? padP : 0, id1 = image ? padP + padO : padP;
+      const unsigned n0 = image ? n : n_p0;
+      float* out = image ? g.y + (size_t)p.token * g.O + s.o0 : g.r + s.p0;
+      if (image) {
+        n += ochunks;
+        ok = ok && chunks_landed(smem, n0, ochunks, abort);
+        tr.mark(7);
       }
-      csync();
-      tr.mark(10);
+      float sr = 0.f;
+      int released = 0;
+      if (ok) {
+        int id = (warp << rpp_log2) + q.sub;
+        if (id < id0) id += ((id0 - id + lanegroups - 1) / lanegroups) * lanegroups;
+#pragma unroll 1
+        for (; __any_sync(0xffffffffu, id < id1); id += lanegroups) {
+          const bool live = id < id1;
+          const int row0g = live ? (id - id0) << 3 : 0;            // first row, within the slab
+          const int ci = min(row0g >> q.rc_log2, nchunks - 1);
+          const int ci_warp = __shfl_sync(0xffffffffu, live ? ci : nchunks - 1, 0);  // ids ascend with the lane
+          if (lane == 0)
+            for (; released < ci_warp; ++released) mbar_arrive(&empty[(n0 + released) % kNB]);
+          released = ci_warp;
+          const uint4* tile = reinterpret_cast<const uint4*>(ring + s_off[(n0 + ci) % kNB]);
+          const int r_lo = ci << q.rc_log2, rows = min(rc, nrows - r_lo);
+          const int row0 = row0g - r_lo;
+          float v[8];
+          dot8(tile, s_c, q, row0, rows, v);
+          const float dot = reduce8(v, q.cl, LPR);
+          const int row = row0 + (q.cl >> hold_log2);
+          if (live && (q.cl & ((1 << hold_log2) - 1)) == 0 && row < rows && row0g < nrows) {
+            if (image) {
+              out[r_lo + row] = nonfinite ? __int_as_float(0x7fc00000) : dot;
+            } else {
+              const float rv = s_x[r_lo + row] - dot;
+              out[r_lo + row] = rv;
+              sr = fmaf(rv, rv, sr);
+            }
+          }
+        }
+        __syncwarp();
+        if (lane == 0)
+          for (; released < nchunks; ++released) mbar_arrive(&empty[(n0 + released) % kNB]);
+      }
+      if (!image) {
+        sr = warp_sum(sr);
+        if (lane == 0) misc->sr[warp] = sr;
+      }
+      tr.mark(image ? 8 : 5);
     }
+    if (!ok && !*abort) fail(p, misc);
     if (*abort) return;
 
     contrib_p = gsi && prow > 0;
@@ -1073,6 +1168,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
   }
   // Every CTA read the counters at its start and has since taken part in the
   // last group's exchange, so they may advance now.
+  tr.flush(p);
   if (cta == 0 && tid == 0 && ok && !*abort) {
     *p.epoch = epoch + 1;
     if (p.use_counter && p.advance) *p.step = step + 1;
@@ -1080,13 +1176,13 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
 }
 
 template <bool kPairs, int kK>
-__global__ void __launch_bounds__(kThreadsP, 1) k_decode_step(PersistParams p) {
+__global__ void __launch_bounds__(kThreadsP, 1) k_decode_step(const __grid_constant__ PersistParams p) {
   extern __shared__ __align__(1024) unsigned char smem[];
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + kOffBar);
-  uint64_t* empty = full + kSlots;
+  uint64_t* empty = full + kNB;
   Misc* misc = reinterpret_cast<Misc*>(smem + kOffMisc);
   if (threadIdx.x == 0) {
-    for (int s = 0; s < kSlots; ++s) {
+    for (int s = 0; s < kNB; ++s) {
       mbar_init(&full[s], 1);
       mbar_init(&empty[s], kNW);
     }
