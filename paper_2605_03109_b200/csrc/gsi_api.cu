@@ -78,7 +78,7 @@ Layout make_layout_ws(const gsi_desc_t* d) {
   L.y_stage = take(B * (size_t)O * 4);
   L.gate_stage = take(B);
   L.rho_stage = take(B * 4);
-  L.pk_acc = take(2 * (k + 2) * 8 * kAccStride);    // persistent kernel: accumulators of c, ||x||^2, ||r||^2
+  L.pk_acc = take(2 * (k + 4) * 8);                 // persistent kernel: accumulators of c, ||x||^2, ||r||^2
   L.pk_slot = take((size_t)kPersistMaxGrid * 8);    // persistent kernel: tagged max|x| words, published ||x||^2
   // tensor-core kernels: batched handles only
   const bool tc_any = d->max_tokens >= kFrontMinTokens && d->d % 64 == 0 && tc_shapes_ok(d);
@@ -124,6 +124,9 @@ struct gsi_stack {
   bool has_pairs;           // some phase of the persistent schedule holds two groups
   int common_k;             // rank shared by every gated group of the persistent schedule, or 0
   PersistGroup* dev_groups; // device table
+  int* dev_phase_first;     // device: first group of every phase of the persistent schedule
+  int n_phases;
+  std::vector<int> host_phase_first;
   char* dev_tmaps;          // device: GSI_MAX_MAPS tensor maps per group (the persistent kernel's W stream)
   unsigned spin_limit;      // polls a cross-CTA wait of the persistent kernel may take
   std::vector<PersistGroup> host_groups;
@@ -397,7 +400,7 @@ size_t gsi_stack_workspace_bytes(int n_groups) {
   if (n_groups <= 0) return 0;
   static_assert(sizeof(PersistGroup) <= 512, "group descriptor outgrew its slot");
   return align_up(256) + align_up((size_t)n_groups * 512) + align_up((size_t)n_groups * 8) +
-         align_up((size_t)n_groups * GSI_MAX_MAPS * kPersistTmapBytes);
+         align_up((size_t)n_groups * GSI_MAX_MAPS * kPersistTmapBytes) + align_up((size_t)n_groups * 4);
 }
 
 gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* workspace,
@@ -429,6 +432,7 @@ gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* wo
   s->dev_groups = reinterpret_cast<PersistGroup*>(static_cast<char*>(workspace) + 256);
   s->dev_tmaps = static_cast<char*>(workspace) + align_up(256) + align_up((size_t)n_groups * 512) +
                  align_up((size_t)n_groups * 8);
+  s->dev_phase_first = reinterpret_cast<int*>(s->dev_tmaps + align_up((size_t)n_groups * GSI_MAX_MAPS * kPersistTmapBytes));
   s->spin_limit = kPersistSpinLimitDefault;
   s->mode = 0;
   s->trace = nullptr;
@@ -480,6 +484,7 @@ static bool w_rows_fit(const gsi_layer* h, int grid) {
 // with a power-of-two rank up to 512, rows that fit the per-CTA buffers and the ring.)
 static bool persistent_eligible(const gsi_stack* s, int grid) {
   if (s->B > kPersistMaxTokens || grid <= 0 || grid > kPersistMaxGrid) return false;
+  if ((int)s->groups.size() + 2 > kPersistMaxTicks) return false;   // the launch's plan lives in shared memory
   for (const gsi_layer* h : s->groups) {
     const gsi_desc_t& d = h->desc;
     const bool dense = d.flags & GSI_FLAG_DENSE;
@@ -561,7 +566,7 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
     // counters) is tied to THIS stack's launch counter: start both from zero.  A handle
     // can therefore serve only one bound stack at a time.
     if (cudaMemsetAsync(s->epoch, 0, sizeof(int), stream) != cudaSuccess ||
-        cudaMemsetAsync(s->status, 0, sizeof(int), stream) != cudaSuccess)   // a fresh start also after a time-out
+        cudaMemsetAsync(s->status, 0, 2 * sizeof(int), stream) != cudaSuccess)   // a fresh start also after a time-out (status word, site of the wait that gave up)
       return GSI_ERR_CUDA;
     for (int i = 0; i < G; ++i) {
       const gsi_layer* h = s->groups[i];
@@ -626,6 +631,7 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
       PersistGroup& pg = s->host_groups[i];
       pg.p_rows = (pg.d + pg.ncta - 1) / pg.ncta;
       pg.o_rows = (pg.O + pg.ncta - 1) / pg.ncta;
+      pg.n_contrib = (pg.d + pg.p_rows - 1) / pg.p_rows;
     }
     s->has_pairs = false;
     s->common_k = -1;
@@ -635,13 +641,16 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
       s->common_k = s->common_k < 0 || s->common_k == k ? k : 0;
     }
     if (s->common_k < 0) s->common_k = 0;
+    s->host_phase_first.clear();
     for (int i = 0; i < G;) {   // length of the phase after each group's
       const int len = s->host_groups[i].phase_len;
+      s->host_phase_first.push_back(i);
       const int nxt = i + len < G ? s->host_groups[i + len].phase_len : 0;
       for (int j = 0; j < len; ++j) s->host_groups[i + j].next_len = nxt;
       if (len == 2) s->has_pairs = true;
       i += len;
     }
+    s->n_phases = (int)s->host_phase_first.size();
     const float** dev_ptrs = reinterpret_cast<const float**>(
         reinterpret_cast<char*>(s->dev_groups) + (size_t)G * 512);
     if (cudaMemcpyAsync(s->dev_groups, s->host_groups.data(), sizeof(PersistGroup) * G,
@@ -650,6 +659,8 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
                         cudaMemcpyHostToDevice, stream) != cudaSuccess ||
         cudaMemcpyAsync(s->dev_tmaps, s->host_tmaps.data(), s->host_tmaps.size(),
                         cudaMemcpyHostToDevice, stream) != cudaSuccess ||
+        cudaMemcpyAsync(s->dev_phase_first, s->host_phase_first.data(),
+                        s->host_phase_first.size() * sizeof(int), cudaMemcpyHostToDevice, stream) != cudaSuccess ||
         launch_patch_pmax(s->dev_groups, dev_ptrs, G, stream) != cudaSuccess)
       return GSI_ERR_CUDA;
   }
@@ -676,6 +687,8 @@ static gsi_status_t stack_enqueue(gsi_stack_t s, bool use_counter, gsi_stream_t 
     PersistParams p{};
     p.groups = s->dev_groups;
     p.n_groups = G;
+    p.phase_first = s->dev_phase_first;
+    p.n_phases = s->n_phases;
     p.step = s->step;
     p.epoch = s->epoch;
     p.n_steps = s->n_steps;

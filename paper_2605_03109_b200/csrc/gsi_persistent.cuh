@@ -10,7 +10,7 @@ constexpr int kPersistMaxPRows = 256;   // basis rows one CTA may own
 constexpr int kPersistMaxORows = 512;   // output rows one CTA may own
 constexpr int kPersistMaxGrid = 256;    // CTAs (tagged words per group)
 constexpr int kPersistMaxTokens = 2;    // tokens per step served by one launch per token (more: batched kernels)
-constexpr int kAccStride = 16;          // 64-bit words between accumulators: one per 128-byte line
+constexpr int kPersistMaxTicks = 160;   // phases of one launch + 2 (the per-CTA plan of a launch lives in shared memory)
 constexpr int kPersistBoxCols = 256;    // columns of W in one streamed box
 constexpr int kPersistBoxRowsMax = 30;  // rows of W in one streamed box: two per consumer warp
 constexpr int kPersistTmapBytes = 128;  // one tensor map
@@ -22,10 +22,11 @@ struct PersistGroup {
   const float* x;                    // [n_steps][tokens][d]
   float* y;                          // [tokens][O]
   float* r;                          // [d]
-  // Cross-CTA state.  acc: per launch parity k + 2 fixed-point accumulators (one per 128-byte
-  // line) whose upper bits count arrivals: c_0..c_{k-1}, ||x||^2 and ||r||^2.  xmax: one
-  // 32-bit word per contributing CTA, max |x| over its rows with the launch parity in the
-  // sign bit.  pub: ||x||^2 as a double with the launch parity in the sign bit.
+  // Cross-CTA state.  acc: per launch parity k + 4 contiguous 64-bit fixed-point accumulators
+  // whose upper bits count arrivals: c_0..c_{k-1}, ||x||^2, a spare, ||r||^2, a spare (every
+  // CTA adds its k + 2 leading words with ONE bulk reduction).  xmax: one 32-bit word per
+  // contributing CTA, max |x| over its rows with the launch parity in the sign bit.  pub:
+  // ||x||^2 as a double with the launch parity in the sign bit.
   unsigned long long* acc;
   unsigned* xmax;
   unsigned long long* pub;
@@ -38,6 +39,7 @@ struct PersistGroup {
   unsigned flags;
   float pmax;                        // max |P| (patched in on the device at bind time)
   int p_rows, o_rows;                // rows per CTA of P and of the images (ceil(rows / ncta))
+  int n_contrib;                     // CTAs that own basis rows: ceil(d / p_rows)
   // Two consecutive groups whose inputs do not depend on each other's outputs may form one
   // phase: CTAs [cta0, cta0 + ncta) run this group's projection, residual and image while the
   // rest of the grid runs its partner's.  A gated residual always streams W with the whole grid.
@@ -53,6 +55,8 @@ struct PersistGroup {
 struct PersistParams {
   const PersistGroup* groups;  // device
   int n_groups;
+  const int* phase_first;      // device [n_phases]: first group of every phase
+  int n_phases;
   int* step;                   // device: decode-step counter (selects the I/O slot)
   int* epoch;                  // device: launches so far (parity of the exchange buffers)
   int n_steps;

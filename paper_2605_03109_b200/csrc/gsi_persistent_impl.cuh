@@ -55,52 +55,59 @@ constexpr int kNB = 32;                     // chunks in flight at most (one bar
 constexpr int kChunk = 16384;               // largest chunk
 constexpr int kSlice = 4096;                // columns of W per staged slice of r
 constexpr int kBoxCols = kPersistBoxCols;
-constexpr unsigned kLocalSpinLimit = 1u << 24;   // waits inside the CTA (ring, producer hand-off)
+constexpr unsigned kLocalSpinLimit = 1u << 20;   // waits inside the CTA (ring, producer hand-off)
 constexpr int kCountShift = 54;
 constexpr unsigned long long kOne = 1ull << kCountShift;
+
+// What one CTA does in one tick of a launch, worked out once at the start of the launch.
+struct Plan {
+  short gi;        // the group whose fast path (or dense stream) this CTA runs in this tick
+  short gi0;       // first group of the tick's phase
+  unsigned char len, next_len;   // groups in this phase and in the next
+  unsigned char kind;            // 0 nothing (closing ticks), 1 gated subspace group, 2 dense group
+  unsigned char zeroer;          // this CTA clears the group's counters for the next launch
+  short prow, orow;              // rows of the basis slab and of the image slab
+  short pchunks, ochunks;        // ... and their ring chunks
+  int p0, o0;                    // first rows
+  short lc, n_contrib;           // index within the group's share of the grid; CTAs that own basis rows
+  int pad;
+};
+static_assert(sizeof(Plan) == 32, "one plan record");
 
 // shared memory map (bytes)
 constexpr int kOffBar = 0;          // full[kNB], empty[kNB]
 constexpr int kOffLin = 512;        // producer: ring position (bytes placed before it) of every chunk in flight (kNB words)
 constexpr int kOffOff = 640;        // offset of every chunk in flight within the ring (kNB words), for the consumers
 constexpr int kOffMisc = 768;       // scalars
-constexpr int kOffTrace = 1152;     // cycle counters of the trace (16 words)
+constexpr int kOffTrace = 1024;     // cycle counters of the trace (16 words)
 constexpr int kOffX = 1280;         // x of this CTA's basis rows, two buffers (kPersistMaxPRows floats each)
 constexpr int kOffC = kOffX + 2 * kPersistMaxPRows * 4;   // c (512 floats)
-constexpr int kOffDesc = kOffC + 2048;                    // 4 group descriptors, 512 B each
-constexpr int kDescSlots = 4;
-constexpr int kOffRed = kOffDesc + kDescSlots * 512;      // cross-warp scratch of pass 1 (kNW*512 floats) ...
+constexpr int kOffFx = kOffC + 2048;                      // fixed-point partial c and ||x||^2, source of the bulk reduction (514 words)
+constexpr int kOffPlan = kOffFx + 4224;                   // the launch's plan (kPersistMaxTicks records)
+constexpr int kOffDesc = kOffPlan + kPersistMaxTicks * 32;   // 8 group descriptors, 256 B each
+constexpr int kDescSlots = 8;
+constexpr int kOffRed = kOffDesc + kDescSlots * 256;      // cross-warp scratch of pass 1 ((kNW-1)*512 floats) ...
 constexpr int kOffRs = kOffRed;                           // ... which the W stream reuses for its slice of r (16 KB)
-constexpr int kOffYacc = kOffRed + kNW * 512 * 4;         // per-row accumulators (kPersistMaxORows floats)
+constexpr int kOffYacc = kOffRed + (kNW - 1) * 512 * 4;   // per-row accumulators (kPersistMaxORows floats)
 constexpr int kOffRing = ((kOffYacc + kPersistMaxORows * 4 + 1023) / 1024) * 1024;
 constexpr int kRingBytes = (232448 - kOffRing) / 1024 * 1024;
 constexpr int kSmemBytes = kOffRing + kRingBytes;
 static_assert(kSmemBytes <= 232448, "shared memory budget of one sm_100 CTA");
-static_assert(kSlice * 4 <= kNW * 512 * 4, "the staged slice fits the scratch it shares");
-static_assert(sizeof(PersistGroup) <= 512 && sizeof(PersistGroup) % 4 == 0, "descriptor slot");
+static_assert(kOffFx % 16 == 0 && kOffPlan % 16 == 0 && kOffDesc % 16 == 0, "alignment");
+static_assert(kSlice * 4 <= (kNW - 1) * 512 * 4, "the staged slice fits the scratch it shares");
+static_assert(sizeof(PersistGroup) <= 256 && sizeof(PersistGroup) % 4 == 0, "descriptor slot");
 static_assert(kPersistBoxRowsMax * kBoxCols * 2 <= kChunk, "a box fits a chunk");
 static_assert(kPersistBoxRowsMax == 2 * kNW, "two rows of a box per consumer warp");
 constexpr int kDescWords = (int)(sizeof(PersistGroup) / 4);
 
-// What the next tick needs to know about a group of this phase to settle its gate.
-struct Settle {
-  const unsigned long long* r2;   // accumulator of ||r||^2
-  const unsigned long long* pub;  // published ||x||^2
-  unsigned n_contrib;
-  float eps;
-  unsigned flags;
-  unsigned* bar;                  // arrival counter before the gated residual
-};
-
 struct Misc {
   int abort;
   unsigned amax_bits;       // max |x| of this phase's group (>= 0x7f800000: a non-finite token)
-  float x2_part;            // this CTA's sum of x^2 over its rows
+  float x2_part[2];         // this CTA's sum of x^2 over its rows, by tick parity
   int fire[4];              // decisions on the previous phase's groups, by tick parity: 1 = stream W
   double x2;                // ||x||^2 of this phase's group
   float sr[kNW];            // per-warp partial ||r||^2 of this phase
   volatile unsigned decision[4];   // hand-off to the producer: (phase + 1) << 8 | fire mask
-  Settle pv[4];             // by tick parity, the groups of the phase run in that tick
 };
 static_assert(sizeof(Misc) <= kOffTrace - kOffMisc, "scalars");
 
@@ -151,6 +158,18 @@ __device__ __forceinline__ void tma_box_g2s(void* dst, const void* tmap, int x, 
       "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar))
       : "memory");
 }
+// Element-wise atomic add of `bytes` / 8 64-bit words from shared to global memory by the bulk
+// copy engine (each element's addition is a relaxed atomic at the L2).
+__device__ __forceinline__ void bulk_reduce_add_u64(void* gdst, const void* ssrc, uint32_t bytes) {
+  asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+  asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.u64 [%0], [%1], %2;" ::"l"(gdst),
+               "r"(smem_u32(ssrc)), "r"(bytes)
+               : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+__device__ __forceinline__ void bulk_reduce_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
 __device__ __forceinline__ void cp_async4(void* dst, const void* src) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
 }
@@ -182,9 +201,12 @@ __device__ __forceinline__ void red_relaxed_u32(unsigned* p, unsigned v) {
   asm volatile("red.relaxed.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 
-__device__ __forceinline__ void fail(const PersistParams& p, Misc* misc) {
+// Records the time-out; `site` (which wait gave up, for diagnosis) goes to the word after
+// the status word, first failure only.
+__device__ __forceinline__ void fail(const PersistParams& p, Misc* misc, int site) {
   misc->abort = 1;
   atomicExch(p.status, (int)GSI_ERR_TIMEOUT);
+  atomicCAS(p.status + 1, 0, site);
 }
 
 // Optional cycle trace (thread 0 of every CTA; sections of the per-phase pipeline, summed
@@ -383,7 +405,7 @@ __device__ void producer(const PersistParams& p, unsigned char* smem, Misc* misc
     len_p = len;
     gi += len;
   }
-  if (!ok && !*abort) fail(p, misc);
+  if (!ok && !*abort) fail(p, misc, 1);
   // Every copy issued must have landed before the CTA may give up its shared
   // memory: wait (bounded) for the last kNB chunks.
   {
@@ -516,7 +538,7 @@ __device__ __forceinline__ bool grid_wait(const unsigned* ctr, unsigned target, 
   unsigned it = 0;
   while (ld_relaxed_u32(ctr) < target) {
     if (++it > p.spin_limit || *abort) {
-      if (!*abort) fail(p, misc);
+      if (!*abort) fail(p, misc, 2);
       return false;
     }
   }
@@ -615,7 +637,7 @@ __device__ __forceinline__ bool w_stream(const PersistParams& p, const PersistGr
       ybase += ((live > 0 ? (live + rb - 1) / rb : 0)) * rb;
     }
   }
-  if (!ok && !*abort) fail(p, misc);
+  if (!ok && !*abort) fail(p, misc, 3);
   csync();
   // rows back to y: the same walk over the maps
   {
@@ -638,9 +660,10 @@ __device__ __forceinline__ bool w_stream(const PersistParams& p, const PersistGr
 }
 
 // kPairs = false compiles the pair logic out: stacks without concurrent groups run a smaller
-// loop (the per-phase code has to stay resident in the instruction cache).  kK != 0 is a
-// build for stacks whose groups all have rank kK (shifts, strides and loop bounds become
-// constants); kK = 0 reads the rank from the descriptor.
+// loop (the per-phase code has to stay short: it is executed once per phase, straight through,
+// so its length is paid in instruction fetches).  kK != 0 is a build for stacks whose groups all
+// have rank kK (shifts, strides and loop bounds become constants); kK = 0 reads the rank from
+// the descriptor.
 template <bool kPairs, int kK>
 __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc) {
   uint64_t* empty = reinterpret_cast<uint64_t*>(smem + kOffBar) + kNB;
@@ -648,7 +671,9 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
   unsigned char* ring = smem + kOffRing;
   float* s_xb = reinterpret_cast<float*>(smem + kOffX);
   float* s_c = reinterpret_cast<float*>(smem + kOffC);
+  unsigned long long* s_fx = reinterpret_cast<unsigned long long*>(smem + kOffFx);
   float* s_red = reinterpret_cast<float*>(smem + kOffRed);
+  Plan* plan = reinterpret_cast<Plan*>(smem + kOffPlan);
   volatile int* abort = &misc->abort;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = gridDim.x, cta = blockIdx.x;
@@ -660,77 +685,128 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
   const int slot_io = step % p.n_steps;
   const int epoch = *p.epoch;
   const unsigned parity = (unsigned)epoch & 1u, tag = ((unsigned)epoch + 1u) & 1u;
+  const int n_ticks = p.n_phases + 2;
   Trace tr;
   tr.start(p, smem);
 
   auto desc = [&](int i) -> const PersistGroup& {
-    return *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + (i & (kDescSlots - 1)) * 512);
+    return *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + (i & (kDescSlots - 1)) * 256);
   };
-  // the group of phase [i, i + len) whose fast path this CTA runs
-  auto mine_of = [&](int i, int len) -> int {
-    if (!kPairs || len < 2) return i;
-    const PersistGroup& a = desc(i);
-    return cta >= a.cta0 + a.ncta ? i + 1 : i;
+  // groups [g0, g0 + cnt) from the device table into their slots (threads 0 .. cnt*kDescWords-1)
+  auto desc_load = [&](int g0, int cnt) -> uint32_t {
+    return tid < cnt * kDescWords ? __ldg(reinterpret_cast<const uint32_t*>(p.groups + g0) + tid) : 0u;
   };
-  // one warp: request this CTA's rows of x of group gn into buffer `buf`
-  auto request_x = [&](const PersistGroup& gn, int buf) {
-    if (gn.flags & GSI_FLAG_DENSE) return;
-    const Slab sn = slab_of(gn, cta - gn.cta0);
-    const float* src = gn.x + (long long)slot_io * gn.x_step_stride + (size_t)p.token * gn.d + sn.p0;
-    float* dst = s_xb + buf * kPersistMaxPRows;
-    for (int i = lane; i < sn.p1 - sn.p0; i += 32) cp_async4(dst + i, src + i);
+  auto desc_store = [&](int g0, int cnt, uint32_t w) {
+    if (tid < cnt * kDescWords) {
+      const int j = tid >= kDescWords ? 1 : 0;
+      reinterpret_cast<uint32_t*>(smem + kOffDesc + ((g0 + j) & (kDescSlots - 1)) * 256)[tid - j * kDescWords] = w;
+    }
+  };
+  // one warp: request this CTA's rows of x for tick `tt` into buffer tt & 1
+  auto request_x = [&](int tt) {
+    const Plan& pn = plan[tt];
+    if (pn.kind != 1) return;
+    const PersistGroup& gn = desc(pn.gi);
+    const float* src = gn.x + (long long)slot_io * gn.x_step_stride + (size_t)p.token * gn.d + pn.p0;
+    float* dst = s_xb + (tt & 1) * kPersistMaxPRows;
+    for (int i = lane; i < pn.prow; i += 32) cp_async4(dst + i, src + i);
   };
 
+  // the statistics warp: max |x| and sum x^2 over this CTA's rows of x for tick `tt` (the rows
+  // have been requested); the maximum is published at once as a tagged word, the sum is kept
+  // for the tick's exchange
+  auto publish_stats = [&](int tt) {
+    const Plan& pn = plan[tt];
+    if (pn.kind != 1) return;
+    cp_async_wait_all();
+    __syncwarp();
+    const float* sx = s_xb + (tt & 1) * kPersistMaxPRows;
+    float amax = 0.f, s2 = 0.f;
+#pragma unroll 1
+    for (int i = lane; i < pn.prow; i += 32) {
+      const float v = sx[i];
+      amax = fmaxf(amax, fabsf(v));
+      s2 = fmaf(v, v, s2);
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+      s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+    }
+    // fmaxf drops NaN, the sum keeps it (and overflows to inf for huge inputs):
+    // s2 - s2 is non-zero exactly when some x_i is NaN or inf (or x^2 overflowed)
+    if (lane == 0) {
+      const unsigned bits = (s2 - s2 == 0.f) ? __float_as_uint(amax) : 0x7fc00000u;
+      if (pn.prow > 0) st_relaxed_u32(desc(pn.gi).xmax + pn.lc, bits | (tag << 31));
+      misc->x2_part[tt & 1] = s2;
+    }
+  };
+
+  // ---- the plan of this launch for this CTA, one thread per tick
+#pragma unroll 1
+  for (int t = tid; t < n_ticks; t += kNC) {
+    Plan pl{};
+    pl.gi = pl.gi0 = -1;
+    if (t < p.n_phases) {
+      const int gi0 = __ldg(p.phase_first + t);
+      const PersistGroup* ga = p.groups + gi0;
+      const int len = kPairs ? __ldg(&ga->phase_len) : 1;
+      int gi = gi0;
+      if (kPairs && len == 2 && cta >= __ldg(&ga->cta0) + __ldg(&ga->ncta)) gi = gi0 + 1;
+      const PersistGroup* g = p.groups + gi;
+      const bool dense = __ldg(&g->flags) & GSI_FLAG_DENSE;
+      pl.gi = (short)gi;
+      pl.gi0 = (short)gi0;
+      pl.len = (unsigned char)len;
+      pl.next_len = (unsigned char)(kPairs ? __ldg(&ga->next_len) : min(__ldg(&ga->next_len), 1));
+      pl.kind = dense ? 2 : 1;
+      const int lc = cta - __ldg(&g->cta0), ncta = __ldg(&g->ncta);
+      pl.lc = (short)lc;
+      pl.zeroer = lc == gi % ncta;
+      if (!dense) {
+        const int d = __ldg(&g->d), O = __ldg(&g->O), pr = __ldg(&g->p_rows), orw = __ldg(&g->o_rows);
+        const int k = kK ? kK : __ldg(&g->k);
+        const int rc = kChunk / (k * 2);
+        const int p0 = min(d, lc * pr), p1 = min(d, p0 + pr);
+        const int o0 = min(O, lc * orw), o1 = min(O, o0 + orw);
+        pl.p0 = p0;
+        pl.o0 = o0;
+        pl.prow = (short)(p1 - p0);
+        pl.orow = (short)(o1 - o0);
+        pl.pchunks = (short)((p1 - p0 + rc - 1) / rc);
+        pl.ochunks = (short)((o1 - o0 + rc - 1) / rc);
+        pl.n_contrib = (short)__ldg(&g->n_contrib);
+      }
+    }
+    plan[t] = pl;
+  }
   // the first phase's descriptors (the second slot is used only if the phase is a pair)
-  if (tid < min(p.n_groups, 2) * kDescWords) {
-    const int j = tid >= kDescWords ? 1 : 0;
-    reinterpret_cast<uint32_t*>(smem + kOffDesc + j * 512)[tid - j * kDescWords] =
-        __ldg(reinterpret_cast<const uint32_t*>(p.groups) + tid);
-  }
-  if (tid == 0) {
-    misc->fire[0] = misc->fire[1] = misc->fire[2] = misc->fire[3] = 0;
-    misc->decision[0] = misc->decision[1] = misc->decision[2] = misc->decision[3] = 0u;
-  }
+  desc_store(0, min(p.n_groups, 2), desc_load(0, min(p.n_groups, 2)));
   csync();
   if (warp == kStatWarp) {
-    const int len0 = kPairs ? desc(0).phase_len : 1;
-    request_x(desc(mine_of(0, len0)), 0);
+    request_x(0);
     cp_async_commit();
+    publish_stats(0);
   }
 
-  int gi = 0;
-  int len_p = 0;                 // groups of the previous phase: their gates are settled in this tick
-  int g_p = -1;
-  int g_pp = -1, len_pp = 0;     // the phase before: its gated residuals run in this tick
-  unsigned mask_pp = 0;
+  unsigned mask_pp = 0;          // gates that fired in the phase before the previous one
   bool contrib_p = false;        // this CTA holds a partial ||r||^2 of the previous phase
   int e_p = 0;                   // ... scaled by 2^(44 - e_p)
   unsigned long long* r2word_p = nullptr;
   bool ok = true;
 
 #pragma unroll 1
-  for (int t = 0; ok; ++t) {
-    const bool own = gi < p.n_groups;
-    if (!own && len_p == 0 && len_pp == 0) break;
-    int len = 0, next_len = 0, gi_mine = gi;
-    if (own) {
-      const PersistGroup& gA = desc(gi);
-      len = kPairs ? gA.phase_len : 1;
-      next_len = kPairs ? gA.next_len : min(gA.next_len, 1);
-      gi_mine = mine_of(gi, len);
-    }
-    const PersistGroup& g = desc(gi_mine);        // read only when `own`
-    const bool dense = own && (g.flags & GSI_FLAG_DENSE);
-    const bool gsi = own && !dense;
-    const int lc = own ? cta - g.cta0 : 0;
+  for (int t = 0; t < n_ticks && ok; ++t) {
+    const Plan pl = plan[t];
+    const bool gsi = pl.kind == 1, dense = pl.kind == 2;
+    const PersistGroup& g = desc(pl.gi);        // read only when the tick has a group
     const int k = gsi ? (kK ? kK : g.k) : 0;
-    Slab s{};
-    if (gsi) s = slab_of(g, lc);
-    const int prow = s.p1 - s.p0, orow = s.o1 - s.o0;
+    const int prow = pl.prow, orow = pl.orow, pchunks = pl.pchunks, ochunks = pl.ochunks;
+    const int n_contrib = pl.n_contrib, lc = pl.lc;
+    const int len_p = t >= 1 ? plan[t - 1].len : 0, g_p = t >= 1 ? plan[t - 1].gi0 : 0;
     float* s_x = s_xb + (t & 1) * kPersistMaxPRows;
-    unsigned long long* acc = gsi ? g.acc + (size_t)parity * (k + 2) * kAccStride : nullptr;
-    const int n_contrib = gsi ? (g.d + g.p_rows - 1) / g.p_rows : 0;
-    const int tp = (t & 1) * 2, tq = tp ^ 2;      // this tick's and the previous tick's slots in Misc
+    unsigned long long* acc = gsi ? g.acc + (size_t)parity * (k + 4) : nullptr;
+    const int tp = (t & 1) * 2;
 
     Geo q{};
     if (gsi) {
@@ -742,26 +818,23 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       q.cl = lane & ((1 << q.lpr_log2) - 1);
     }
     const int LPR = 1 << q.lpr_log2, rpp_log2 = 5 - q.lpr_log2, rc = 1 << q.rc_log2;
-    const int pchunks = gsi ? (prow + rc - 1) >> q.rc_log2 : 0;
-    const int ochunks = gsi ? (orow + rc - 1) >> q.rc_log2 : 0;
 
-    // one word of the next phase's descriptors: requested now, stored after pass 1
-    uint32_t desc_word = 0;
-    if (own && tid < next_len * kDescWords)
-      desc_word = __ldg(reinterpret_cast<const uint32_t*>(p.groups + gi + len) + tid);
+    // the next phase's descriptors: requested now, stored after pass 1
+    const uint32_t desc_word = desc_load(pl.gi0 + pl.len, pl.next_len);
 
-    // ---- A. this CTA's rows of x have arrived (requested one phase ago)
-    if (gsi && warp == kStatWarp) cp_async_wait_all();
-    if (tid == 0) misc->fire[tp] = misc->fire[tp + 1] = 0;
-    if (own && lc == gi_mine % g.ncta) {  // this CTA clears the group's counters for the next launch
+    // ---- A. this CTA's rows of x have arrived (requested one phase ago); the bulk reduction
+    //      of the previous tick has read its source
+    if (tid == 0) {
+      bulk_reduce_wait_read();
+      misc->fire[tp] = misc->fire[tp + 1] = 0;
+    }
+    if (pl.zeroer) {  // this CTA clears the group's counters for the next launch
       if (gsi) {
 #pragma unroll 1
-        for (int j = tid; j < k + 2; j += kNC)
-          g.acc[((size_t)(parity ^ 1u) * (k + 2) + j) * kAccStride] = 0ull;
+        for (int j = tid; j < k + 4; j += kNC) g.acc[(size_t)(parity ^ 1u) * (k + 4) + j] = 0ull;
       }
       if (tid < 2) g.bar[2 * tid + (parity ^ 1u)] = 0u;
     }
-    tr.mark(15);
     csync();
     tr.mark(0);
 
@@ -769,42 +842,26 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     n += pchunks;
     if (gsi) {
       if (warp == kStatWarp) {
-        // ---- statistics of x over this CTA's rows, published at once; then the group's
-        //      max |x|: collect the tagged words of all contributing CTAs (lane l owns words
-        //      l, l+32, ...) while the other warps run pass 1
-        float amax = 0.f, s2 = 0.f;
-#pragma unroll 1
-        for (int i = lane; i < prow; i += 32) {
-          const float v = s_x[i];
-          amax = fmaxf(amax, fabsf(v));
-          s2 = fmaf(v, v, s2);
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) {
-          amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-          s2 += __shfl_xor_sync(0xffffffffu, s2, o);
-        }
-        // fmaxf drops NaN, the sum keeps it (and overflows to inf for huge inputs):
-        // s2 - s2 is non-zero exactly when some x_i is NaN or inf (or x^2 overflowed)
-        if (lane == 0) {
-          const unsigned bits = (s2 - s2 == 0.f) ? __float_as_uint(amax) : 0x7fc00000u;
-          if (prow > 0) st_relaxed_u32(g.xmax + lc, bits | (tag << 31));
-          misc->x2_part = s2;
-        }
+        // ---- the group's max |x|: collect the tagged words of all contributing CTAs (lane l
+        //      owns words l, l+32, ...; they were published during the previous tick) while
+        //      the other warps run pass 1
         unsigned m = 0, it = 0;
         bool done = false;
         while (!done) {
           bool all = true;
           m = 0;
-#pragma unroll 1
-          for (int w_i = lane; w_i < n_contrib; w_i += 32) {
-            const unsigned w = ld_relaxed_u32(g.xmax + w_i);
-            all = all && ((w >> 31) == tag);
-            m = max(m, w & 0x7fffffffu);
+#pragma unroll
+          for (int i = 0; i < kPersistMaxGrid / 32; ++i) {   // all loads in flight together
+            const int w_i = lane + 32 * i;
+            if (w_i < n_contrib) {
+              const unsigned w = ld_relaxed_u32(g.xmax + w_i);
+              all = all && ((w >> 31) == tag);
+              m = max(m, w & 0x7fffffffu);
+            }
           }
           done = __all_sync(0xffffffffu, all);
           if (!done && (++it > p.spin_limit || ((it & 1023u) == 0 && *abort))) {
-            if (!*abort && lane == 0) fail(p, misc);
+            if (!*abort && lane == 0) fail(p, misc, 4);
             break;
           }
         }
@@ -826,7 +883,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
             if (!ok) break;
             const uint4* tile = reinterpret_cast<const uint4*>(ring + s_off[(n_p0 + ci) % kNB]);
             const int r_lo = ci << q.rc_log2, rows = min(rc, prow - r_lo);
-#pragma unroll 1
+#pragma unroll 2
             for (int row = (warp << rpp_log2) + q.sub; row < rows; row += kP1 << rpp_log2) {
               const float xv = s_x[r_lo + row];
               const uint4 w = tile[(size_t)row * q.KV + cv];
@@ -851,41 +908,38 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
             dst[1] = make_float4(a8[4], a8[5], a8[6], a8[7]);
           }
         }
-        if (!ok && !*abort) fail(p, misc);
+        if (!ok && !*abort) fail(p, misc, 5);
       }
     }
-    if (own && tid < next_len * kDescWords) {
-      uint32_t* dst = reinterpret_cast<uint32_t*>(
-                          smem + kOffDesc +
-                          ((gi + len + (tid >= kDescWords ? 1 : 0)) & (kDescSlots - 1)) * 512) +
-                      (tid >= kDescWords ? tid - kDescWords : tid);
-      *dst = desc_word;
-    }
+    desc_store(pl.gi0 + pl.len, pl.next_len, desc_word);
     csync();
     tr.mark(2);
     if (*abort) return;
+    // the next phase's rows of x travel while this phase runs its exchange (its descriptors
+    // are in place now) ...
+    if (warp == kStatWarp && t + 1 < n_ticks) {
+      request_x(t + 1);
+      cp_async_commit();
+    }
 
-    // ---- D. the exchange: this phase's partial c and ||x||^2, the previous phase's ||r||^2
+    // ---- D. the exchange: this phase's partial c and ||x||^2 as ONE bulk reduction of k + 2
+    //      fixed-point words into the group's accumulators, the previous phase's ||r||^2 as
+    //      one atomic
     bool nonfinite = false;
     double inv_scale = 0.0;
     if (gsi) {
       const unsigned amax_bits = misc->amax_bits;
       nonfinite = amax_bits >= 0x7f800000u;
       const float amax = __uint_as_float(amax_bits);
-      if (amax_bits == 12345u) tr.t += 1;
-      tr.mark(13);
       // fixed-point scales: |partial c_j| <= amax * rows * max|P| < 2^e, partial ||x||^2 <= rows * amax^2 < 2^ex
       double scale = 0.0, scale_x2 = 0.0;
       const float bound = amax * (float)g.p_rows * g.pmax;
-      if (bound == 12345.f) tr.t += 1;
-      tr.mark(14);
       if (!nonfinite && bound > 0.f && bound < 3.0e38f) {
         const int e = max((int)((__float_as_uint(bound) >> 23) & 0xFFu), 1) - 126;
         scale = pow2d(43 - e);
         inv_scale = pow2d(e - 43);
         scale_x2 = pow2d(43 - exp_above((double)amax * (double)amax * (double)g.p_rows));
       }
-      tr.mark(10);
       if (prow > 0) {
 #pragma unroll 1
         for (int j = tid; j < k; j += kNC) {
@@ -893,15 +947,18 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
 #pragma unroll
           for (int w = 0; w < kP1; ++w) sum += s_red[w * 512 + j];
           const long long v = scale != 0.0 ? __double2ll_rn((double)sum * scale) : 0ll;
-          red_add_u64(acc + (size_t)j * kAccStride, kOne + (unsigned long long)v);
+          s_fx[j] = kOne + (unsigned long long)v;
         }
         if (tid == kNC - 1) {
-          const long long v = scale_x2 != 0.0 ? __double2ll_rn((double)misc->x2_part * scale_x2) : 0ll;
-          red_add_u64(acc + (size_t)k * kAccStride, kOne + (unsigned long long)v);
+          const long long v = scale_x2 != 0.0 ? __double2ll_rn((double)misc->x2_part[t & 1] * scale_x2) : 0ll;
+          s_fx[k] = kOne + (unsigned long long)v;
+          s_fx[k + 1] = 0ull;
         }
       }
     }
-    if (contrib_p && tid == kNC - 2) {
+    csync();
+    if (tid == 0 && gsi && prow > 0) bulk_reduce_add_u64(acc, s_fx, (uint32_t)(k + 2) * 8);
+    if (contrib_p && tid == 32) {
       float sr = 0.f;   // fixed order: the sum does not depend on which warp finished first
 #pragma unroll
       for (int w = 0; w < kNW; ++w) sr += misc->sr[w];
@@ -915,36 +972,24 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     tr.mark(3);
 
     // ---- E. wait until every contributing CTA has been added: warp 0 polls the accumulators
-    //      of c (lane l owns words l, l+32, ...: all its loads are in flight together, one
-    //      round trip per attempt), warp 1 the scalars: lane 0 this phase's ||x||^2, lanes
+    //      of c (contiguous: lane l owns words l, l+32, ..., all its loads in flight together,
+    //      one round trip per attempt), warp 1 the scalars: lane 0 this phase's ||x||^2, lanes
     //      1+2u / 2+2u the previous phase's ||r||^2 and published ||x||^2 of its group u.
-    //      The other warps wait at the barrier (thousands of pollers on the accumulators
-    //      would delay the very atomics they wait for).
     if (gsi && warp == 0) {
       unsigned it = 0;
-      if (lane == 0) {   // one watcher per CTA on one word keeps the polling traffic off the atomics
-        const unsigned long long* wp = acc + (size_t)(k - 1) * kAccStride;
-        for (;;) {
-          const unsigned long long w = ld_relaxed_u64(wp);
-          if ((unsigned)((w + (kOne >> 1)) >> kCountShift) == (unsigned)n_contrib) break;
-          if (++it > p.spin_limit || ((it & 1023u) == 0 && *abort)) break;   // the loop below reports it
-        }
-      }
-      __syncwarp();
-      tr.mark(11);
       bool done = false;
       while (!done) {
         bool all = true;
 #pragma unroll 8
         for (int j = lane; j < k; j += 32) {
-          const unsigned long long w = ld_relaxed_u64(acc + (size_t)j * kAccStride);
+          const unsigned long long w = ld_relaxed_u64(acc + j);
           all = all && ((unsigned)((w + (kOne >> 1)) >> kCountShift) == (unsigned)n_contrib);
           const long long val = (long long)(w - ((unsigned long long)n_contrib << kCountShift));
           s_c[j] = (float)((double)val * inv_scale);
         }
         done = __all_sync(0xffffffffu, all);
         if (!done && (++it > p.spin_limit || ((it & 1023u) == 0 && *abort))) {
-          if (!*abort && lane == 0) fail(p, misc);
+          if (!*abort && lane == 0) fail(p, misc, 6);
           break;
         }
       }
@@ -952,12 +997,14 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     if (warp == 1) {
       // what this lane watches: an accumulator (count in the upper bits) or a tagged word
       const int u = (lane - 1) >> 1;
-      const Settle& sv = misc->pv[tq + (u & 1)];
+      const bool settle = lane >= 1 && lane <= 4 && u < len_p && !(desc(g_p + u).flags & GSI_FLAG_DENSE);
+      const PersistGroup& gs = desc(g_p + (u & 1));   // read only when `settle`
       const bool w_x2 = gsi && lane == 0;
-      const bool w_r2 = lane >= 1 && lane <= 4 && (lane & 1) && u < len_p && sv.r2 != nullptr;
-      const bool w_pub = lane >= 1 && lane <= 4 && !(lane & 1) && u < len_p && sv.r2 != nullptr;
-      const unsigned long long* wp = w_x2 ? acc + (size_t)k * kAccStride : w_r2 ? sv.r2 : sv.pub;
-      const unsigned want = w_x2 ? (unsigned)n_contrib : sv.n_contrib;
+      const bool w_r2 = settle && (lane & 1), w_pub = settle && !(lane & 1);
+      const unsigned long long* wp = w_x2   ? acc + k
+                                     : w_r2 ? gs.acc + (size_t)parity * (gs.k + 4) + gs.k + 2
+                                            : gs.pub;
+      const unsigned want = w_x2 ? (unsigned)n_contrib : (unsigned)gs.n_contrib;
       unsigned long long w = 0;
       unsigned it = 0;
       bool done = false;
@@ -972,7 +1019,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
         }
         done = __all_sync(0xffffffffu, mine);
         if (!done && (++it > p.spin_limit || ((it & 1023u) == 0 && *abort))) {
-          if (!*abort && lane == 0) fail(p, misc);
+          if (!*abort && lane == 0) fail(p, misc, 7);
           break;
         }
       }
@@ -997,10 +1044,10 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
         const bool finite = x2 == x2;
         const int ex = x2 > 0.0 ? exp_above(x2) : 0;
         const double r2 = (double)val * pow2d(ex - 44);
-        const double eps = (double)sv.eps;
+        const double eps = (double)gs.eps;
         // ||r|| < eps ||x||  <=>  ||r||^2 < eps^2 ||x||^2  (both sides >= 0); false for x = 0
         const bool fast = finite && (r2 < eps * eps * x2);
-        misc->fire[tp + u] = (!fast && finite && !(sv.flags & GSI_FLAG_STATIC_PROJECTION)) ? 1 : 0;
+        misc->fire[tp + u] = (!fast && finite && !(gs.flags & GSI_FLAG_STATIC_PROJECTION)) ? 1 : 0;
         if (cta == 0) {
           const size_t at = ((size_t)slot_io * p.log_step_stride + (g_p + u)) * p.n_tokens + p.token;
           p.gate_log[at] = fast ? 0 : 1;
@@ -1011,7 +1058,6 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
         }
       }
     }
-    tr.mark(12);
     csync();
     tr.mark(4);
     if (*abort) return;
@@ -1026,29 +1072,12 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       for (int u = 0; u < len_p; ++u)
         if (mask_p & (1u << u)) {
           __threadfence();
-          red_relaxed_u32(misc->pv[tq + u].bar, 1u);
+          red_relaxed_u32(desc(g_p + u).bar + 2 + parity, 1u);
         }
     }
     const double x2_own = gsi ? misc->x2 : 0.0;
-    if (warp == kStatWarp && next_len > 0) {   // the next phase's rows of x travel while this phase runs
-      request_x(desc(mine_of(gi + len, next_len)), (t + 1) & 1);
-      cp_async_commit();
-    }
-    if (tid < 2) {   // what the next tick needs to settle this phase's gates
-      Settle sv{};
-      if (own && tid < len) {
-        const PersistGroup& gs = desc(gi + tid);
-        if (!(gs.flags & GSI_FLAG_DENSE)) {
-          sv.r2 = gs.acc + ((size_t)parity * (gs.k + 2) + gs.k + 1) * kAccStride;
-          sv.pub = gs.pub;
-          sv.n_contrib = (unsigned)((gs.d + gs.p_rows - 1) / gs.p_rows);
-          sv.eps = gs.eps;
-          sv.flags = gs.flags;
-          sv.bar = gs.bar + 2 + parity;
-        }
-      }
-      misc->pv[tp + tid] = sv;
-    }
+    // ... and their statistics are published a row pass ahead of the next phase's exchange
+    if (warp == kStatWarp && t + 1 < n_ticks) publish_stats(t + 1);
 
     // ---- G / I. the row passes, one copy of the code for both: part 0 the residual rows of
     //      the basis slab (still in the ring), part 1 the image rows.  Items of eight rows
@@ -1062,10 +1091,10 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     const int padO = ((itemsO + (1 << rpp_log2) - 1) >> rpp_log2) << rpp_log2;
     const int hold_log2 = q.lpr_log2 - 3;          // lanes per held row after reduce8
     const int lanegroups = kNW << rpp_log2;
-    tr.mark(9);
 #pragma unroll 1
     for (int part = 0; part < 2; ++part) {
       if (part == 1 && (mask_pp || dense)) {
+        const int len_pp = plan[t - 2 >= 0 ? t - 2 : 0].len, g_pp = plan[t - 2 >= 0 ? t - 2 : 0].gi0;
 #pragma unroll 1
         for (int u = 0; u < 3 && ok; ++u) {
           const PersistGroup* gw = nullptr;
@@ -1091,7 +1120,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
               red_relaxed_u32(gw->bar + parity, 1u);
               grid_wait(gw->bar + parity, (unsigned)G, p, misc);
               if (cta == 0)
-                p.gate_log[((size_t)slot_io * p.log_step_stride + gi) * p.n_tokens + p.token] = 1;
+                p.gate_log[((size_t)slot_io * p.log_step_stride + pl.gi) * p.n_tokens + p.token] = 1;
             }
             csync();
           }
@@ -1104,7 +1133,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       const int nchunks = image ? ochunks : pchunks, nrows = image ? orow : prow;
       const int id0 = image ? padP : 0, id1 = image ? padP + padO : padP;
       const unsigned n0 = image ? n : n_p0;
-      float* out = image ? g.y + (size_t)p.token * g.O + s.o0 : g.r + s.p0;
+      float* out = image ? g.y + (size_t)p.token * g.O + pl.o0 : g.r + pl.p0;
       if (image) {
         n += ochunks;
         ok = ok && chunks_landed(smem, n0, ochunks, abort);
@@ -1151,24 +1180,20 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       }
       tr.mark(image ? 8 : 5);
     }
-    if (!ok && !*abort) fail(p, misc);
+    if (!ok && !*abort) fail(p, misc, 8);
     if (*abort) return;
 
     contrib_p = gsi && prow > 0;
     if (gsi) {
       e_p = x2_own > 0.0 ? exp_above(x2_own) : 0;
-      r2word_p = acc + (size_t)(k + 1) * kAccStride;
+      r2word_p = acc + k + 2;
     }
-    g_pp = g_p;
-    len_pp = len_p;
     mask_pp = mask_p;
-    g_p = gi;
-    len_p = len;
-    gi += len;
   }
+  if (tid == 0) bulk_reduce_wait_read();
+  tr.flush(p);
   // Every CTA read the counters at its start and has since taken part in the
   // last group's exchange, so they may advance now.
-  tr.flush(p);
   if (cta == 0 && tid == 0 && ok && !*abort) {
     *p.epoch = epoch + 1;
     if (p.use_counter && p.advance) *p.step = step + 1;
@@ -1187,6 +1212,10 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_decode_step(const __grid_const
       mbar_init(&empty[s], kNW);
     }
     misc->abort = 0;
+    // shared memory keeps what the previous launch on this SM left: the producer must not
+    // mistake an old decision for this launch's
+    misc->fire[0] = misc->fire[1] = misc->fire[2] = misc->fire[3] = 0;
+    misc->decision[0] = misc->decision[1] = misc->decision[2] = misc->decision[3] = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   __syncthreads();
