@@ -21,9 +21,9 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 
 struct Layout {
   size_t wp, c, cpart, r, normpart, ctrl, fired, rho, x_stage, y_stage, gate_stage, rho_stage,
-      pk_acc, pk_slot, tc_rb, tc_ypart, f_pt, f_xb, f_cb, f_cpart, f_normpart, total;
+      pk_acc, pk_slot, tc_rb, tc_ypart, f_pt, f_xb, f_cb, f_cpart, f_normpart, pk_pp, pk_wpp, total;
   int O, n_slabs, slab_rows;
-  bool tc, front, dense_tc;
+  bool tc, front, dense_tc, packed;
 };
 
 constexpr int kTcMinFired = 5;  // fewer fired tokens: one pass of the CUDA-core GEMV
@@ -98,6 +98,13 @@ Layout make_layout_ws(const gsi_desc_t* d) {
   L.f_cpart = take(front ? (size_t)front_proj_splits(d->d, d->k) * B * k * 4 : 0);
   L.f_normpart = take(front ? (size_t)(d->d / 128) * B * 2 * 4 : 0);
   L.front = front;
+  // persistent kernel: the basis and the images once more, as 16 x 16 tiles in the operand
+  // order of the tensor-core instruction (rows padded to a multiple of 16)
+  const bool packed = !dense && d->p_dtype == GSI_BF16 && d->k >= 64 && d->k <= 512 &&
+                      (d->k & (d->k - 1)) == 0 && d->max_tokens <= kPersistMaxTokens;
+  L.pk_pp = take(packed ? (size_t)((d->d + 15) / 16 * 16) * k * 2 : 0);
+  L.pk_wpp = take(packed ? (size_t)((O + 15) / 16 * 16) * k * 2 : 0);
+  L.packed = packed;
   L.total = at;
   return L;
 }
@@ -156,6 +163,13 @@ struct gsi_stack {
     if (aux) cudaStreamDestroy(aux);
   }
 };
+
+// The tiled copies of the basis and of the images that the persistent kernel streams.
+static bool repack(gsi_layer* h, cudaStream_t stream) {
+  const Layout& L = h->lay;
+  return launch_pack_t16(h->gp.P, h->desc.d, h->desc.k, h->ws + L.pk_pp, stream) == cudaSuccess &&
+         launch_pack_t16(h->ws + L.wp, L.O, h->desc.k, h->ws + L.pk_wpp, stream) == cudaSuccess;
+}
 
 extern "C" {
 
@@ -291,6 +305,10 @@ gsi_status_t gsi_create(const gsi_desc_t* desc, const void* const* W, const void
       }
     }
   }
+  if (L.packed && !repack(h, stream)) {
+    delete h;
+    return GSI_ERR_CUDA;
+  }
   // A set-up call: return only when the images, max|P| and the cleared state are in
   // place, so the handle may be used from any stream afterwards.
   if (cudaStreamSynchronize(stream) != cudaSuccess) {
@@ -371,7 +389,9 @@ gsi_status_t gsi_extend_basis(gsi_handle_t h, const float* x, float tau, int* k_
   a.pmax = h->gp.p_f32 ? nullptr : h->pmax;
   a.PT = L.front ? const_cast<uint16_t*>(h->gp.PT) : nullptr;
   h->last_stream = stream;
-  return launch_extend_basis(h->gp, a, stream) == cudaSuccess ? GSI_OK : GSI_ERR_CUDA;
+  if (launch_extend_basis(h->gp, a, stream) != cudaSuccess) return GSI_ERR_CUDA;
+  if (L.packed && !repack(h, stream)) return GSI_ERR_CUDA;   // the tiled copies follow the new column
+  return GSI_OK;
 }
 
 gsi_status_t gsi_get_image(gsi_handle_t h, int map, const void** out) {
@@ -449,16 +469,17 @@ gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* wo
   return GSI_OK;
 }
 
-// Rows of one CTA fit its buffers, and the 16 KB chunks of the group's basis slab, and of its
-// image slab, each fit the ring of ten slots together (pass 1 and the image rows run with
-// every chunk of their slab resident).
+// The basis rows and the image rows are dealt to the CTAs of a group's share in units of 16
+// rows.  One CTA's share fits its buffers, and the 16 KB chunks of its basis slab, and of its
+// image slab, each fit the ring together (pass 1 and the image rows run with every chunk of
+// their slab resident; one chunk per lane is waited for).
 static bool rows_fit(const gsi_layer* h, int ctas) {
   if (ctas <= 0) return false;
-  const int pr = (h->desc.d + ctas - 1) / ctas, orw = (h->lay.O + ctas - 1) / ctas;
-  if (pr > kPersistMaxPRows || orw > kPersistMaxORows) return false;
   if ((h->desc.flags & GSI_FLAG_DENSE) || h->desc.k <= 0) return true;
-  const int rc = std::max(1, 16384 / (h->desc.k * 2));
-  return (pr + rc - 1) / rc <= 10 && (orw + rc - 1) / rc <= 10;
+  const int pg = ((h->desc.d + 15) / 16 + ctas - 1) / ctas, og = ((h->lay.O + 15) / 16 + ctas - 1) / ctas;
+  if (pg * 16 > kPersistMaxPRows || og * 16 > kPersistMaxORows) return false;
+  const int gc = std::max(1, 16384 / (h->desc.k * 32));   // groups per chunk
+  return (pg + gc - 1) / gc <= 10 && (og + gc - 1) / gc <= 10;
 }
 
 // W stream geometry of one map: rows per CTA, and rows per box (even, at most 30, chosen so
@@ -491,10 +512,7 @@ static bool persistent_eligible(const gsi_stack* s, int grid) {
     if (dense && s->B > 1) return false;   // a dense group streams W: once for all tokens (batched GEMM)
     if (d.d % 16) return false;
     if (!rows_fit(h, grid) || !w_rows_fit(h, grid)) return false;
-    if (!dense) {
-      if (d.p_dtype != GSI_BF16) return false;
-      if (d.k < 64 || d.k > 512 || (d.k & (d.k - 1))) return false;
-    }
+    if (!dense && !h->lay.packed) return false;
   }
   return true;
 }
@@ -582,8 +600,8 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
       const gsi_layer* h = s->groups[i];
       PersistGroup& pg = s->host_groups[i];
       const GroupParams& gp = h->gp;
-      pg.P = static_cast<const uint16_t*>(gp.P);
-      pg.WP = gp.WP;
+      pg.P = reinterpret_cast<const uint16_t*>(h->ws + h->lay.pk_pp);
+      pg.WP = reinterpret_cast<const uint16_t*>(h->ws + h->lay.pk_wpp);
       pg.tmW = s->dev_tmaps + (size_t)i * GSI_MAX_MAPS * kPersistTmapBytes;
       for (int j = 0; j < gp.n_maps; ++j) {
         int rows, rb;
@@ -629,9 +647,12 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
     }
     for (int i = 0; i < G; ++i) {
       PersistGroup& pg = s->host_groups[i];
-      pg.p_rows = (pg.d + pg.ncta - 1) / pg.ncta;
-      pg.o_rows = (pg.O + pg.ncta - 1) / pg.ncta;
-      pg.n_contrib = (pg.d + pg.p_rows - 1) / pg.p_rows;
+      // rows are dealt in groups of 16: CTA c of the share owns groups [c n / ncta, (c + 1) n / ncta)
+      // (the first n CTAs one group each when there are fewer groups than CTAs)
+      const int pgroups = (pg.d + 15) / 16, ogroups = (pg.O + 15) / 16;
+      pg.p_rows = 16 * ((pgroups + pg.ncta - 1) / pg.ncta);
+      pg.o_rows = 16 * ((ogroups + pg.ncta - 1) / pg.ncta);
+      pg.n_contrib = std::min(pg.ncta, pgroups);
     }
     s->has_pairs = false;
     s->common_k = -1;

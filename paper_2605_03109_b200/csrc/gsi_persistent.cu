@@ -25,7 +25,29 @@ __global__ void k_patch_pmax(PersistGroup* groups, const float* const* pmax_ptrs
   if (i < n && pmax_ptrs[i]) groups[i].pmax = *pmax_ptrs[i];
 }
 
+// One thread per 32-bit word of the tiled copy.
+__global__ void k_pack_t16(const uint16_t* __restrict__ src, int rows, int k, uint32_t* __restrict__ dst) {
+  const int kt = k >> 4;
+  const size_t n_words = (size_t)((rows + 15) / 16) * kt * 128;
+  for (size_t wi = (size_t)blockIdx.x * blockDim.x + threadIdx.x; wi < n_words;
+       wi += (size_t)gridDim.x * blockDim.x) {
+    const int reg = (int)(wi & 3), lane = (int)((wi >> 2) & 31);
+    const size_t tile = wi >> 7;
+    const int K = (int)(tile % kt);
+    const size_t R = tile / kt;
+    const int g = lane >> 2, t = lane & 3;
+    const size_t row = R * 16 + g + (reg & 1) * 8;
+    const int col = K * 16 + 2 * t + (reg >> 1) * 8;
+    dst[wi] = row < (size_t)rows ? *reinterpret_cast<const uint32_t*>(src + row * k + col) : 0u;
+  }
+}
+
 }  // namespace
+
+cudaError_t launch_pack_t16(const void* src, int rows, int k, void* dst, cudaStream_t st) {
+  k_pack_t16<<<592, 256, 0, st>>>(static_cast<const uint16_t*>(src), rows, k, static_cast<uint32_t*>(dst));
+  return cudaGetLastError();
+}
 
 cudaError_t launch_patch_pmax(PersistGroup* groups, const float* const* pmax_ptrs, int n,
                               cudaStream_t st) {

@@ -8,7 +8,7 @@ namespace gsi {
 constexpr int kPersistConsumerWarps = 15;  // + 1 producer warp = 16 warps: registers are allotted per 4 warps
 constexpr int kPersistMaxPRows = 256;   // basis rows one CTA may own
 constexpr int kPersistMaxORows = 512;   // output rows one CTA may own
-constexpr int kPersistMaxGrid = 256;    // CTAs (tagged words per group)
+constexpr int kPersistMaxGrid = 160;    // CTAs (tagged words per group)
 constexpr int kPersistMaxTokens = 2;    // tokens per step served by one launch per token (more: batched kernels)
 constexpr int kPersistMaxTicks = 160;   // phases of one launch + 2 (the per-CTA plan of a launch lives in shared memory)
 constexpr int kPersistBoxCols = 256;    // columns of W in one streamed box
@@ -16,8 +16,12 @@ constexpr int kPersistBoxRowsMax = 30;  // rows of W in one streamed box: two pe
 constexpr int kPersistTmapBytes = 128;  // one tensor map
 
 struct PersistGroup {
-  const uint16_t* P;                 // [d][k] bf16
-  const uint16_t* WP;                // [O][k] bf16, images of all maps concatenated
+  // Basis [d][k] and concatenated images [O][k], bf16, as 16 x 16 tiles: tile (R, K) at
+  // ((R * k/16 + K) * 512) bytes; its 16-byte word l = 4g + t holds elements (g, 2t..2t+1),
+  // (g+8, 2t..2t+1), (g, 2t+8..2t+9), (g+8, 2t+8..2t+9): the A operand of mma.m16n8k16.
+  // Rows past d (O) are zero.
+  const uint16_t* P;
+  const uint16_t* WP;
   const void* tmW;                   // n_maps tensor maps (device memory): W_j [d_out_j][d] bf16 in boxes of w_rb[j] rows x 256 columns
   const float* x;                    // [n_steps][tokens][d]
   float* y;                          // [tokens][O]
@@ -38,8 +42,8 @@ struct PersistGroup {
   float eps;
   unsigned flags;
   float pmax;                        // max |P| (patched in on the device at bind time)
-  int p_rows, o_rows;                // rows per CTA of P and of the images (ceil(rows / ncta))
-  int n_contrib;                     // CTAs that own basis rows: ceil(d / p_rows)
+  int p_rows, o_rows;                // most rows one CTA owns of P and of the images (multiples of 16)
+  int n_contrib;                     // CTAs that own basis rows: the first min(ncta, ceil(d / 16)) of the share
   // Two consecutive groups whose inputs do not depend on each other's outputs may form one
   // phase: CTAs [cta0, cta0 + ncta) run this group's projection, residual and image while the
   // rest of the grid runs its partner's.  A gated residual always streams W with the whole grid.
@@ -80,6 +84,8 @@ int persist_threads();
 cudaError_t launch_decode_step(const PersistParams& p, int grid, bool pairs, int common_k,
                                cudaStream_t st);
 cudaError_t launch_abs_max_bf16(const void* p, size_t n, float* out, cudaStream_t st);
+// Row-major [rows][k] bf16 -> the tiled layout described at PersistGroup::P.
+cudaError_t launch_pack_t16(const void* src, int rows, int k, void* dst, cudaStream_t st);
 cudaError_t launch_patch_pmax(PersistGroup* groups, const float* const* pmax_ptrs, int n,
                               cudaStream_t st);
 // Tensor map of one weight matrix for the persistent kernel's W stream: W [rows][cols] bf16

@@ -9,14 +9,20 @@
 // Algorithm 1 per group (two consecutive groups declared independent share a phase on two
 // parts of the grid).  A phase has ONE grid-wide exchange:
 //
-//   statistics  warp 0: max |x| and sum x^2 over this CTA's rows of x; the maximum is
-//               published as a tagged 32-bit word (no fence: the word validates itself)
+//   statistics  one warp: max |x| and sum x^2 over this CTA's rows of x (requested and
+//               published one row pass ahead: the inputs of a stack are pre-staged); the
+//               maximum goes out as a tagged 32-bit word (no fence: the word validates itself)
 //   pass 1      partial c = P_slab^T x_slab                              (line 1)
 //   exchange    every CTA adds, as 64-bit fixed-point numbers whose upper bits count the
-//               arrivals (integer addition is order-free, so the sums are bit-reproducible):
-//               its partial c_j (scale from the global max |x|, collected from the tagged
-//               words meanwhile), its partial ||x||^2, and its partial ||r||^2 of the
-//               PREVIOUS phase; it then polls the words until all have arrived
+//               arrivals (integer addition is order-free, so the sums are bit-reproducible),
+//               its partial c_j (scale from the group's max |x|, collected from the tagged
+//               words during pass 1) and its partial ||x||^2 with ONE bulk reduction
+//               (cp.reduce.async.bulk), and its partial ||r||^2 of the PREVIOUS phase; one
+//               warp then polls the accumulators until all have arrived
+// Basis and images are stored as 16 x 16 tiles in the operand order of mma.m16n8k16, so both
+// passes and the image rows run on the tensor cores with one 16-byte shared-memory load per
+// tile and lane: x and c enter as three bf16 terms each (hi + mid + lo = the fp32 value), so
+// every product is exact and the sums are fp32.
 //   gate        of the previous phase, from the exact integer sums: the same decision on
 //               every CTA                                                (line 4, Eq. (3.3))
 //   pass 2      r_slab = x_slab - P_slab c, partial ||r||^2              (lines 2-3)
@@ -60,41 +66,54 @@ constexpr int kCountShift = 54;
 constexpr unsigned long long kOne = 1ull << kCountShift;
 
 // What one CTA does in one tick of a launch, worked out once at the start of the launch.
+// Rows are dealt in groups of 16 (one tile row).
 struct Plan {
   short gi;        // the group whose fast path (or dense stream) this CTA runs in this tick
   short gi0;       // first group of the tick's phase
   unsigned char len, next_len;   // groups in this phase and in the next
   unsigned char kind;            // 0 nothing (closing ticks), 1 gated subspace group, 2 dense group
   unsigned char zeroer;          // this CTA clears the group's counters for the next launch
-  short prow, orow;              // rows of the basis slab and of the image slab
+  short pg, og;                  // 16-row groups of the basis slab and of the image slab
   short pchunks, ochunks;        // ... and their ring chunks
   int p0, o0;                    // first rows
   short lc, n_contrib;           // index within the group's share of the grid; CTAs that own basis rows
-  int pad;
+  short gc_log2, pad;            // log2 of the 16-row groups per 16 KB chunk
 };
 static_assert(sizeof(Plan) == 32, "one plan record");
+
+// Groups [a, b) of n that part i of `parts` owns: an even split, or one group each for the
+// first n parts when there are fewer groups than parts.
+__device__ __forceinline__ void deal(int n, int parts, int i, int& a, int& b) {
+  if (n >= parts) {   // i <= parts <= 256 and n < 2^20: the products fit 32 bits
+    a = (int)((unsigned)i * (unsigned)n / (unsigned)parts);
+    b = (int)((unsigned)(i + 1) * (unsigned)n / (unsigned)parts);
+  } else {
+    a = min(i, n);
+    b = min(i + 1, n);
+  }
+}
 
 // shared memory map (bytes)
 constexpr int kOffBar = 0;          // full[kNB], empty[kNB]
 constexpr int kOffLin = 512;        // producer: ring position (bytes placed before it) of every chunk in flight (kNB words)
 constexpr int kOffOff = 640;        // offset of every chunk in flight within the ring (kNB words), for the consumers
+constexpr int kOffProd = 1152;      // state of the producer thread (16 bytes)
 constexpr int kOffMisc = 768;       // scalars
 constexpr int kOffTrace = 1024;     // cycle counters of the trace (16 words)
 constexpr int kOffX = 1280;         // x of this CTA's basis rows, two buffers (kPersistMaxPRows floats each)
-constexpr int kOffC = kOffX + 2 * kPersistMaxPRows * 4;   // c (512 floats)
-constexpr int kOffFx = kOffC + 2048;                      // fixed-point partial c and ||x||^2, source of the bulk reduction (514 words)
+constexpr int kOffXt = kOffX + 2 * kPersistMaxPRows * 4;  // ... as three bf16 terms in A-operand order, two buffers (16 tile rows x 256 B each)
+constexpr int kOffCb = kOffXt + 2 * 4096;                 // c as three bf16 terms in B-operand order (32 tile columns x 256 B)
+constexpr int kOffFx = kOffCb + 8192;                     // fixed-point partial c and ||x||^2, source of the bulk reduction (514 words)
 constexpr int kOffPlan = kOffFx + 4224;                   // the launch's plan (kPersistMaxTicks records)
 constexpr int kOffDesc = kOffPlan + kPersistMaxTicks * 32;   // 8 group descriptors, 256 B each
 constexpr int kDescSlots = 8;
-constexpr int kOffRed = kOffDesc + kDescSlots * 256;      // cross-warp scratch of pass 1 ((kNW-1)*512 floats) ...
-constexpr int kOffRs = kOffRed;                           // ... which the W stream reuses for its slice of r (16 KB)
-constexpr int kOffYacc = kOffRed + (kNW - 1) * 512 * 4;   // per-row accumulators (kPersistMaxORows floats)
+constexpr int kOffRs = kOffDesc + kDescSlots * 256;       // W stream: staged slice of r (16 KB)
+constexpr int kOffYacc = kOffRs + kSlice * 4;             // per-row accumulators (kPersistMaxORows floats)
 constexpr int kOffRing = ((kOffYacc + kPersistMaxORows * 4 + 1023) / 1024) * 1024;
 constexpr int kRingBytes = (232448 - kOffRing) / 1024 * 1024;
 constexpr int kSmemBytes = kOffRing + kRingBytes;
 static_assert(kSmemBytes <= 232448, "shared memory budget of one sm_100 CTA");
-static_assert(kOffFx % 16 == 0 && kOffPlan % 16 == 0 && kOffDesc % 16 == 0, "alignment");
-static_assert(kSlice * 4 <= (kNW - 1) * 512 * 4, "the staged slice fits the scratch it shares");
+static_assert(kOffXt % 16 == 0 && kOffCb % 16 == 0 && kOffFx % 16 == 0 && kOffPlan % 16 == 0 && kOffDesc % 16 == 0 && kOffRs % 16 == 0, "alignment");
 static_assert(sizeof(PersistGroup) <= 256 && sizeof(PersistGroup) % 4 == 0, "descriptor slot");
 static_assert(kPersistBoxRowsMax * kBoxCols * 2 <= kChunk, "a box fits a chunk");
 static_assert(kPersistBoxRowsMax == 2 * kNW, "two rows of a box per consumer warp");
@@ -102,7 +121,7 @@ constexpr int kDescWords = (int)(sizeof(PersistGroup) / 4);
 
 struct Misc {
   int abort;
-  unsigned amax_bits;       // max |x| of this phase's group (>= 0x7f800000: a non-finite token)
+  unsigned amax_bits[2];    // by tick parity: max |x| of the phase's group (>= 0x7f800000: a non-finite token)
   float x2_part[2];         // this CTA's sum of x^2 over its rows, by tick parity
   int fire[4];              // decisions on the previous phase's groups, by tick parity: 1 = stream W
   double x2;                // ||x||^2 of this phase's group
@@ -203,11 +222,12 @@ __device__ __forceinline__ void red_relaxed_u32(unsigned* p, unsigned v) {
 
 // Records the time-out; `site` (which wait gave up, for diagnosis) goes to the word after
 // the status word, first failure only.
-__device__ __forceinline__ void fail(const PersistParams& p, Misc* misc, int site) {
+__device__ __noinline__ void fail_at(int* status, Misc* misc, int site) {
   misc->abort = 1;
-  atomicExch(p.status, (int)GSI_ERR_TIMEOUT);
-  atomicCAS(p.status + 1, 0, site);
+  atomicExch(status, (int)GSI_ERR_TIMEOUT);
+  atomicCAS(status + 1, 0, site);
 }
+__device__ __forceinline__ void fail(const PersistParams& p, Misc* misc, int site) { fail_at(p.status, misc, site); }
 
 // Optional cycle trace (thread 0 of every CTA; sections of the per-phase pipeline, summed
 // over phases in shared memory and added to p.trace when the CTA ends); p.trace == nullptr
@@ -235,19 +255,6 @@ struct Trace {
   }
 };
 
-struct Slab {
-  int p0, p1;  // basis rows owned by this CTA
-  int o0, o1;  // rows of the concatenated images owned by this CTA
-};
-__device__ __forceinline__ Slab slab_of(const PersistGroup& g, int lc) {
-  Slab s;
-  s.p0 = min(g.d, lc * g.p_rows);
-  s.p1 = min(g.d, s.p0 + g.p_rows);
-  s.o0 = min(g.O, lc * g.o_rows);
-  s.o1 = min(g.O, s.o0 + g.o_rows);
-  return s;
-}
-
 // ------------------------------------------------------------------ the ring
 // Chunks of any size up to 16 KB are packed back to back in a circular byte buffer (a chunk
 // never wraps: the tail of the buffer is skipped instead).  `lin` counts bytes placed so far,
@@ -255,12 +262,7 @@ __device__ __forceinline__ Slab slab_of(const PersistGroup& g, int lc) {
 // pair n % kNB.  The producer publishes the offset of chunk n in s_off[n % kNB] before it arms
 // the chunk's "full" barrier; producer and consumers walk the same sequence of chunks, so a
 // consumer needs only the sequence number.
-struct Producer {
-  uint64_t* full;
-  uint64_t* empty;
-  unsigned char* base;
-  unsigned* s_lin;     // shared: start (lin) of every chunk in flight
-  unsigned* s_off;     // shared: its offset in the ring
+struct Producer {      // state of the producer thread, kept in shared memory
   unsigned n;          // sequence number of the next chunk
   unsigned lin;        // bytes placed so far
   unsigned tail_n;     // oldest chunk not yet given back by the consumers
@@ -269,110 +271,136 @@ struct Producer {
 
 // Reserve `bytes` for chunk n: waits (bounded) until the consumers have given back every
 // older chunk that still overlaps the place, and a barrier pair is free.  Returns the
-// offset, or 0xffffffff when a wait gave up.
-__device__ __forceinline__ unsigned producer_acquire(Producer& pr, unsigned bytes, volatile int* abort) {
-  unsigned off = pr.lin % (unsigned)kRingBytes;
+// offset, or 0xffffffff when a wait gave up.  Out of line: one copy for every kind of chunk.
+__device__ __noinline__ unsigned producer_acquire(unsigned char* smem, unsigned bytes) {
+  Producer& pr = *reinterpret_cast<Producer*>(smem + kOffProd);
+  uint64_t* empty = reinterpret_cast<uint64_t*>(smem + kOffBar) + kNB;
+  unsigned* s_lin = reinterpret_cast<unsigned*>(smem + kOffLin);
+  unsigned* s_off = reinterpret_cast<unsigned*>(smem + kOffOff);
+  volatile int* abort = &reinterpret_cast<Misc*>(smem + kOffMisc)->abort;
+  unsigned n = pr.n, lin = pr.lin, tail_n = pr.tail_n, tail_lin = pr.tail_lin;
+  unsigned off = lin % (unsigned)kRingBytes;
   if (off + bytes > (unsigned)kRingBytes) {
-    pr.lin += (unsigned)kRingBytes - off;
+    lin += (unsigned)kRingBytes - off;
     off = 0;
   }
-  const unsigned start = pr.lin;
-  pr.lin += bytes;
-  while (pr.n - pr.tail_n >= (unsigned)kNB ||
-         (pr.tail_n < pr.n && pr.lin - pr.tail_lin > (unsigned)kRingBytes)) {
-    if (!mbar_wait(&pr.empty[pr.tail_n % kNB], (pr.tail_n / kNB) & 1u, abort)) return 0xffffffffu;
-    ++pr.tail_n;
-    pr.tail_lin = pr.tail_n < pr.n ? pr.s_lin[pr.tail_n % kNB] : start;
+  const unsigned start = lin;
+  lin += bytes;
+  while (n - tail_n >= (unsigned)kNB || (tail_n < n && lin - tail_lin > (unsigned)kRingBytes)) {
+    if (!mbar_wait(&empty[tail_n % kNB], (tail_n / kNB) & 1u, abort)) return 0xffffffffu;
+    ++tail_n;
+    tail_lin = tail_n < n ? s_lin[tail_n % kNB] : start;
   }
-  if (pr.tail_n == pr.n) pr.tail_lin = start;
-  pr.s_lin[pr.n % kNB] = start;
-  pr.s_off[pr.n % kNB] = off;
+  if (tail_n == n) tail_lin = start;
+  s_lin[n % kNB] = start;
+  s_off[n % kNB] = off;
+  pr.lin = lin;
+  pr.tail_n = tail_n;
+  pr.tail_lin = tail_lin;
   return off;
 }
 
 // The W boxes of one group for this CTA, in the order the consumers take them: column
 // slices of 4096 outermost (one staged slice of r serves them), then maps, then row blocks,
 // then the 256-column boxes of the slice.
-__device__ __forceinline__ bool produce_w(const PersistGroup& g, Producer& pr, volatile int* abort) {
+__device__ __forceinline__ bool produce_w(const PersistGroup& g, unsigned char* smem) {
+  Producer& prs = *reinterpret_cast<Producer*>(smem + kOffProd);
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kOffBar);
+  uint64_t* empty = full + kNB;
+  unsigned* s_lin = reinterpret_cast<unsigned*>(smem + kOffLin);
+  unsigned* s_off = reinterpret_cast<unsigned*>(smem + kOffOff);
+  unsigned char* base = smem + kOffRing;
+  volatile int* abort = &reinterpret_cast<Misc*>(smem + kOffMisc)->abort;
+  // the ring state in registers for the length of the stream (thousands of boxes, one every
+  // few hundred cycles: the out-of-line acquire with its state in shared memory is too slow)
+  unsigned n = prs.n, lin = prs.lin, tail_n = prs.tail_n, tail_lin = prs.tail_lin;
+  bool ok = true;
   const int cta = blockIdx.x;
   const int nsl = (g.d + kSlice - 1) / kSlice;
-  for (int sl = 0; sl < nsl; ++sl) {
+  for (int sl = 0; sl < nsl && ok; ++sl) {
     const int c0 = sl * kSlice, ncb = (min(kSlice, g.d - c0) + kBoxCols - 1) / kBoxCols;
-    for (int j = 0; j < g.n_maps; ++j) {
+    for (int j = 0; j < g.n_maps && ok; ++j) {
       const int dout = g.off[j + 1] - g.off[j], rows = g.w_rows[j], rb = g.w_rb[j];
       const int row0 = cta * rows;
       const int live = min(rows, dout - row0);
       const char* tm = static_cast<const char*>(g.tmW) + (size_t)j * kPersistTmapBytes;
       const uint32_t bytes = (uint32_t)rb * kBoxCols * 2;
-      for (int b = 0; b * rb < live; ++b) {
+      for (int b = 0; b * rb < live && ok; ++b) {
         for (int cb = 0; cb < ncb; ++cb) {
-          const unsigned off = producer_acquire(pr, bytes, abort);
-          if (off == 0xffffffffu) return false;
-          uint64_t* fb = &pr.full[pr.n % kNB];
+          unsigned off = lin % (unsigned)kRingBytes;
+          if (off + bytes > (unsigned)kRingBytes) {
+            lin += (unsigned)kRingBytes - off;
+            off = 0;
+          }
+          const unsigned start = lin;
+          lin += bytes;
+          while (n - tail_n >= (unsigned)kNB || (tail_n < n && lin - tail_lin > (unsigned)kRingBytes)) {
+            if (!mbar_wait(&empty[tail_n % kNB], (tail_n / kNB) & 1u, abort)) {
+              ok = false;
+              break;
+            }
+            ++tail_n;
+            tail_lin = tail_n < n ? s_lin[tail_n % kNB] : start;
+          }
+          if (!ok) break;
+          if (tail_n == n) tail_lin = start;
+          s_lin[n % kNB] = start;
+          s_off[n % kNB] = off;
+          uint64_t* fb = &full[n % kNB];
           mbar_expect_tx(fb, bytes);
-          tma_box_g2s(pr.base + off, tm, c0 + cb * kBoxCols, row0 + b * rb, fb);
-          ++pr.n;
+          tma_box_g2s(base + off, tm, c0 + cb * kBoxCols, row0 + b * rb, fb);
+          ++n;
         }
       }
     }
   }
-  return true;
+  prs.n = n;
+  prs.lin = lin;
+  prs.tail_n = tail_n;
+  prs.tail_lin = tail_lin;
+  return ok;
 }
 
-// Rows [a, b) of a row-major [rows][k] bf16 matrix as chunks of whole rows.
-__device__ __forceinline__ bool produce_rows(const uint16_t* base, int k, int a, int b, Producer& pr,
-                                             volatile int* abort) {
-  const int rc = kChunk / (k * 2);
-  for (int r = a; r < b; r += rc) {
-    const int rows = min(rc, b - r);
-    const uint32_t bytes = (uint32_t)rows * k * 2;
-    const unsigned off = producer_acquire(pr, bytes, abort);
+// Tile rows [a, b) (16 matrix rows each) of a tiled [rows][k] bf16 matrix as chunks of whole
+// tile rows.
+__device__ __forceinline__ bool produce_rows(const uint16_t* base, int k, int a, int b, unsigned char* smem) {
+  Producer& pr = *reinterpret_cast<Producer*>(smem + kOffProd);
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kOffBar);
+  const int gc = kChunk / (k * 32);
+  for (int r = a; r < b; r += gc) {
+    const int groups = min(gc, b - r);
+    const uint32_t bytes = (uint32_t)groups * k * 32;
+    const unsigned off = producer_acquire(smem, bytes);
     if (off == 0xffffffffu) return false;
-    uint64_t* fb = &pr.full[pr.n % kNB];
+    uint64_t* fb = &full[pr.n % kNB];
     mbar_expect_tx(fb, bytes);
-    bulk_g2s(pr.base + off, base + (size_t)r * k, bytes, fb);
+    bulk_g2s(smem + kOffRing + off, base + (size_t)r * k * 16, bytes, fb);
     ++pr.n;
   }
   return true;
 }
 
 __device__ void producer(const PersistParams& p, unsigned char* smem, Misc* misc) {
-  Producer pr;
-  pr.full = reinterpret_cast<uint64_t*>(smem + kOffBar);
-  pr.empty = pr.full + kNB;
-  pr.base = smem + kOffRing;
-  pr.s_lin = reinterpret_cast<unsigned*>(smem + kOffLin);
-  pr.s_off = reinterpret_cast<unsigned*>(smem + kOffOff);
+  Producer& pr = *reinterpret_cast<Producer*>(smem + kOffProd);
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kOffBar);
   pr.n = 0;
   pr.lin = 0;
   pr.tail_n = 0;
   pr.tail_lin = 0;
   volatile int* abort = &misc->abort;
-  const int cta = blockIdx.x;
   bool ok = true;
   // ticks: tick t runs phase t (while there is one) and the gated residuals of phase t - 2;
   // the work of a tick, in ring order: basis slab, W boxes of the gated groups, image slab
   // (or the W boxes of a dense group)
-  int gi = 0;        // first group of phase t
-  int g_pp = -1, len_pp = 0;   // phase t - 2
-  int g_p = -1, len_p = 0;     // phase t - 1
-  for (int t = 0; ok; ++t) {
-    const bool own = gi < p.n_groups;
-    if (!own && len_p == 0 && len_pp == 0) break;
-    int len = 0;
-    const PersistGroup* g = nullptr;
-    if (own) {
-      const PersistGroup& gA = p.groups[gi];
-      len = gA.phase_len;
-      g = (len == 2 && cta >= gA.cta0 + gA.ncta) ? &p.groups[gi + 1] : &gA;
-    }
-    const bool dense = own && (g->flags & GSI_FLAG_DENSE);
-    Slab s{};
-    if (own && !dense) {
-      s = slab_of(*g, cta - g->cta0);
-      ok = produce_rows(g->P, g->k, s.p0, s.p1, pr, abort);
-    }
+  const Plan* plan = reinterpret_cast<const Plan*>(smem + kOffPlan);
+  const int n_ticks = p.n_phases + 2;
+#pragma unroll 1
+  for (int t = 0; t < n_ticks && ok; ++t) {
+    const Plan& pl = plan[t];
+    const PersistGroup* g = p.groups + pl.gi;   // read only when the tick has a group
+    if (pl.kind == 1) ok = produce_rows(g->P, g->k, pl.p0 >> 4, (pl.p0 >> 4) + pl.pg, smem);
     unsigned wmask = 0;
+    const int len_pp = t >= 2 ? plan[t - 2].len : 0, g_pp = t >= 2 ? plan[t - 2].gi0 : 0;
     if (ok && len_pp > 0) {
       // the decision on phase t - 2 (taken by the consumers during tick t - 1)
       const unsigned want = (unsigned)(t - 1);   // (phase + 1)
@@ -388,22 +416,19 @@ __device__ void producer(const PersistParams& p, unsigned char* smem, Misc* misc
       wmask = v & 3u;
     }
     // one call site for every W stream of the tick: the gated groups, then a dense group
+    if (wmask || pl.kind == 2) {
 #pragma unroll 1
-    for (int u = 0; ok && u < 3; ++u) {
-      const PersistGroup* gw = nullptr;
-      if (u < 2) {
-        if (u < len_pp && (wmask & (1u << u))) gw = &p.groups[g_pp + u];
-      } else if (dense) {
-        gw = g;
+      for (int u = 0; ok && u < 3; ++u) {
+        const PersistGroup* gw = nullptr;
+        if (u < 2) {
+          if (u < len_pp && (wmask & (1u << u))) gw = &p.groups[g_pp + u];
+        } else if (pl.kind == 2) {
+          gw = g;
+        }
+        if (gw) ok = produce_w(*gw, smem);
       }
-      if (gw) ok = produce_w(*gw, pr, abort);
     }
-    if (ok && own && !dense) ok = produce_rows(g->WP, g->k, s.o0, s.o1, pr, abort);
-    g_pp = g_p;
-    len_pp = len_p;
-    g_p = gi;
-    len_p = len;
-    gi += len;
+    if (ok && pl.kind == 1) ok = produce_rows(g->WP, g->k, pl.o0 >> 4, (pl.o0 >> 4) + pl.og, smem);
   }
   if (!ok && !*abort) fail(p, misc, 1);
   // Every copy issued must have landed before the CTA may give up its shared
@@ -413,61 +438,12 @@ __device__ void producer(const PersistParams& p, unsigned char* smem, Misc* misc
     for (unsigned c = first; c < pr.n; ++c) {
       const unsigned slot = c % kNB, ph = (c / kNB) & 1u;
       for (unsigned it = 0; it < kLocalSpinLimit; ++it)
-        if (mbar_try(&pr.full[slot], ph)) break;
+        if (mbar_try(&full[slot], ph)) break;
     }
   }
 }
 
 // ------------------------------------------------------------------ consumer
-// Lane layout over a row of k bf16: KV = k/8 vectors, LPR = min(32, KV) lanes
-// per row, RPP = 32/LPR rows per warp pass, VPL = KV/LPR vectors per lane.
-
-// Sum eight per-lane row partials across the LPR = 1<<lpr_log2 lanes (8, 16 or
-// 32) that share the rows.  Halving exchange: each level sends half of the
-// values to the partner lane, so eight rows cost 4+2+1 shuffles plus
-// log2(LPR/8) for the tail instead of 8*log2(LPR).  On return the lanes with
-// cl % (LPR/8) == 0 hold the total of row cl / (LPR/8).
-__device__ __forceinline__ float reduce8(float (&v)[8], int cl, int LPR) {
-  int m = LPR >> 1;
-  {
-    const bool up = cl & m;
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      const float send = up ? v[i] : v[i + 4];
-      const float recv = __shfl_xor_sync(0xffffffffu, send, m);
-      v[i] = (up ? v[i + 4] : v[i]) + recv;
-    }
-  }
-  m >>= 1;
-  {
-    const bool up = cl & m;
-#pragma unroll
-    for (int i = 0; i < 2; ++i) {
-      const float send = up ? v[i] : v[i + 2];
-      const float recv = __shfl_xor_sync(0xffffffffu, send, m);
-      v[i] = (up ? v[i + 2] : v[i]) + recv;
-    }
-  }
-  m >>= 1;
-  {
-    const bool up = cl & m;
-    const float send = up ? v[0] : v[1];
-    const float recv = __shfl_xor_sync(0xffffffffu, send, m);
-    v[0] = (up ? v[1] : v[0]) + recv;
-  }
-#pragma unroll 1
-  for (m >>= 1; m > 0; m >>= 1) v[0] += __shfl_xor_sync(0xffffffffu, v[0], m);
-  return v[0];
-}
-
-struct Geo {       // lane geometry of one group (k a power of two, 64..512)
-  int KV;          // 16-byte vectors per row
-  int lpr_log2;    // log2(lanes per row), lanes per row = min(32, KV)
-  int vpl;         // vectors per lane (1, or 2 for k = 512)
-  int rc_log2;     // log2(rows per 16 KB chunk)
-  int sub, cl;     // this lane: row sub-group and column lane
-};
-
 // Two-wide fp32 FMA of sm_100: one instruction for a pair of bf16 weights.
 __device__ __forceinline__ unsigned long long pack2(float lo, float hi) {
   unsigned long long r;
@@ -489,39 +465,37 @@ __device__ __forceinline__ float sum2(unsigned long long v) {
   return lo + hi;
 }
 
-// out[i] = tile[row0 + i][:] . c   for eight rows, this lane's share of the columns
-__device__ __forceinline__ void dot8(const uint4* tile, const float* s_c, const Geo& q, int row0,
-                                     int rows, float (&v)[8]) {
-  unsigned long long acc[8];
-#pragma unroll
-  for (int i = 0; i < 8; ++i) acc[i] = 0ull;
-  const int LPR = 1 << q.lpr_log2;
-#pragma unroll 1
-  for (int u = 0; u < q.vpl; ++u) {
-    const int cv = q.cl + u * LPR;
-    const float4 ca = *reinterpret_cast<const float4*>(s_c + cv * 8);
-    const float4 cb = *reinterpret_cast<const float4*>(s_c + cv * 8 + 4);
-    const unsigned long long c0 = pack2(ca.x, ca.y), c1 = pack2(ca.z, ca.w);
-    const unsigned long long c2 = pack2(cb.x, cb.y), c3 = pack2(cb.z, cb.w);
-    // rows past the end of the slab read the last row again (no branch: the eight loads
-    // and FMA chains interleave); the caller drops their results
-#pragma unroll
-    for (int h = 0; h < 8; h += 4) {   // four rows at a time: eight would not fit the registers
-      uint4 w[4];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) w[i] = tile[max(min(row0 + h + i, rows - 1), 0) * q.KV + cv];
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        fma2(acc[h + i], bf16x2_to_f32x2(w[i].x), c0);
-        fma2(acc[h + i], bf16x2_to_f32x2(w[i].y), c1);
-        fma2(acc[h + i], bf16x2_to_f32x2(w[i].z), c2);
-        fma2(acc[h + i], bf16x2_to_f32x2(w[i].w), c3);
-      }
-      asm volatile("" ::: "memory");
-    }
-  }
-#pragma unroll
-  for (int i = 0; i < 8; ++i) v[i] = sum2(acc[i]);
+// D (16 x 8, fp32) += A (16 x 16, bf16) B (16 x 8, bf16) on the tensor cores.
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint4& a, uint32_t b0, uint32_t b1) {
+  asm volatile(
+      "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, "
+      "{%0,%1,%2,%3};"
+      : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+      : "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b0), "r"(b1));
+}
+// Transposes an 8 x 8 block of 16-bit elements held one row pair per lane.
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
+  uint32_t d;
+  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+  return d;
+}
+// v = hi + mid + lo, each a bf16 (round to nearest; the remainders are exact in fp32).
+__device__ __forceinline__ void split3(float v, unsigned short (&t)[3]) {
+  const __nv_bfloat16 h = __float2bfloat16_rn(v);
+  const float r1 = v - __bfloat162float(h);
+  const __nv_bfloat16 m = __float2bfloat16_rn(r1);
+  const float r2 = r1 - __bfloat162float(m);
+  const __nv_bfloat16 l = __float2bfloat16_rn(r2);
+  t[0] = __bfloat16_as_ushort(h);
+  t[1] = __bfloat16_as_ushort(m);
+  t[2] = __bfloat16_as_ushort(l);
+}
+// Element e (0..15) of vector chunk `blk` as term g of a three-term operand: index of its
+// 16-bit slot in an array of 256-byte blocks laid out one 8-byte word per lane (the A operand
+// rows 0..2 of mma.m16n8k16, or its B operand columns 0..2: lane = 4 g + (e % 8) / 2, word half
+// e / 8, element e % 2).
+__device__ __forceinline__ int term_slot(int blk, int e, int g) {
+  return (((blk * 32 + g * 4 + ((e & 7) >> 1)) * 2 + (e >> 3)) * 2) + (e & 1);
 }
 
 // 2^e as a double, e in the normal range
@@ -659,6 +633,156 @@ __device__ __forceinline__ bool w_stream(const PersistParams& p, const PersistGr
   return ok;
 }
 
+// The statistics warp: the group's max |x| for tick `tt` from the tagged words of all
+// contributing CTAs (lane l owns words l, l+32, ...).  `first` holds a first round of loads
+// issued earlier (split phase: they flew while the warp did other work); further rounds are
+// polled here.  Out of line.
+constexpr int kXmaxWords = (kPersistMaxGrid + 31) / 32;
+__device__ __forceinline__ void xmax_issue(const unsigned* xmax, int n_contrib, unsigned (&w)[kXmaxWords]) {
+  const int lane = threadIdx.x & 31;
+#pragma unroll
+  for (int i = 0; i < kXmaxWords; ++i) {
+    const int w_i = lane + 32 * i;
+    w[i] = w_i < n_contrib ? ld_relaxed_u32(xmax + w_i) : 0xffffffffu;   // all loads in flight together
+  }
+}
+__device__ __noinline__ void xmax_collect(unsigned char* smem, int tt, unsigned tag, unsigned spin_limit,
+                                          int* status, unsigned w0, unsigned w1, unsigned w2,
+                                          unsigned w3, unsigned w4) {
+  static_assert(kXmaxWords == 5, "argument list");
+  const Plan& pn = reinterpret_cast<const Plan*>(smem + kOffPlan)[tt];
+  Misc* misc = reinterpret_cast<Misc*>(smem + kOffMisc);
+  const PersistGroup& gn =
+      *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + (pn.gi & (kDescSlots - 1)) * 256);
+  const int lane = threadIdx.x & 31;
+  unsigned w[kXmaxWords] = {w0, w1, w2, w3, w4};
+  unsigned m = 0, it = 0;
+  for (;;) {
+    bool all = true;
+    m = 0;
+#pragma unroll
+    for (int i = 0; i < kXmaxWords; ++i) {
+      if (lane + 32 * i < pn.n_contrib) {
+        all = all && ((w[i] >> 31) == tag);
+        m = max(m, w[i] & 0x7fffffffu);
+      }
+    }
+    if (__all_sync(0xffffffffu, all)) break;
+    if (++it > spin_limit || ((it & 1023u) == 0 && misc->abort)) {
+      if (!misc->abort && lane == 0) fail_at(status, misc, 4);
+      break;
+    }
+    xmax_issue(gn.xmax, pn.n_contrib, w);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
+  if (lane == 0) misc->amax_bits[tt & 1] = m;
+}
+
+// The statistics warp, for tick `tt`: (request = true) ask for this CTA's rows of x into buffer
+// tt & 1; (request = false) wait for them, take max |x| and sum x^2 over them, publish the
+// maximum at once as a tagged word, keep the sum for the tick's exchange, and leave x as three
+// bf16 terms in the operand order of pass 1.  Out of line: two call sites, one copy.
+__device__ __noinline__ void stat_warp_step(unsigned char* smem, int tt, bool request, int slot_io, int token,
+                                            unsigned tag) {
+  const Plan& pn = reinterpret_cast<const Plan*>(smem + kOffPlan)[tt];
+  if (pn.kind != 1) return;
+  const int lane = threadIdx.x & 31;
+  const PersistGroup& gn =
+      *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + (pn.gi & (kDescSlots - 1)) * 256);
+  float* sx = reinterpret_cast<float*>(smem + kOffX) + (tt & 1) * kPersistMaxPRows;
+  const int rows = pn.pg * 16;
+  if (request) {
+    const float* src = gn.x + (long long)slot_io * gn.x_step_stride + (size_t)token * gn.d + pn.p0;
+    const int live = min(rows, gn.d - pn.p0);   // rows past d belong to the zero padding of P
+#pragma unroll 1
+    for (int i = lane; i < rows; i += 32) {
+      if (i < live)
+        cp_async4(sx + i, src + i);
+      else
+        sx[i] = 0.f;
+    }
+    cp_async_commit();
+    return;
+  }
+  cp_async_wait_all();
+  __syncwarp();
+  unsigned short* xt = reinterpret_cast<unsigned short*>(smem + kOffXt) + (tt & 1) * 2048;
+  Misc* misc = reinterpret_cast<Misc*>(smem + kOffMisc);
+  float amax = 0.f, s2 = 0.f;
+#pragma unroll 1
+  for (int i = lane; i < rows; i += 32) {
+    const float v = sx[i];
+    amax = fmaxf(amax, fabsf(v));
+    s2 = fmaf(v, v, s2);
+    unsigned short tm[3];
+    split3(v, tm);
+    const int slot = term_slot(i >> 4, i & 15, 0);
+    xt[slot] = tm[0];
+    xt[slot + 16] = tm[1];   // the next term is the next row of the operand: four lanes on
+    xt[slot + 32] = tm[2];
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    s2 += __shfl_xor_sync(0xffffffffu, s2, o);
+  }
+  // fmaxf drops NaN, the sum keeps it (and overflows to inf for huge inputs):
+  // s2 - s2 is non-zero exactly when some x_i is NaN or inf (or x^2 overflowed)
+  if (lane == 0) {
+    const unsigned bits = (s2 - s2 == 0.f) ? __float_as_uint(amax) : 0x7fc00000u;
+    if (pn.pg > 0) st_relaxed_u32(gn.xmax + pn.lc, bits | (tag << 31));
+    misc->x2_part[tt & 1] = s2;
+  }
+}
+
+// The plan of this launch for this CTA, one thread per tick (all threads of the CTA, before
+// the producer and the consumers part).
+template <bool kPairs, int kK>
+__device__ __forceinline__ void make_plan(const PersistParams& p, unsigned char* smem) {
+  Plan* plan = reinterpret_cast<Plan*>(smem + kOffPlan);
+  const int cta = blockIdx.x, n_ticks = p.n_phases + 2;
+#pragma unroll 1
+  for (int t = threadIdx.x; t < n_ticks; t += kThreadsP) {
+    Plan pl{};
+    pl.gi = pl.gi0 = -1;
+    if (t < p.n_phases) {
+      const int gi0 = __ldg(p.phase_first + t);
+      const PersistGroup* ga = p.groups + gi0;
+      const int len = kPairs ? __ldg(&ga->phase_len) : 1;
+      int gi = gi0;
+      if (kPairs && len == 2 && cta >= __ldg(&ga->cta0) + __ldg(&ga->ncta)) gi = gi0 + 1;
+      const PersistGroup* g = p.groups + gi;
+      const bool dense = __ldg(&g->flags) & GSI_FLAG_DENSE;
+      pl.gi = (short)gi;
+      pl.gi0 = (short)gi0;
+      pl.len = (unsigned char)len;
+      pl.next_len = (unsigned char)(kPairs ? __ldg(&ga->next_len) : min(__ldg(&ga->next_len), 1));
+      pl.kind = dense ? 2 : 1;
+      const int lc = cta - __ldg(&g->cta0), ncta = __ldg(&g->ncta);
+      pl.lc = (short)lc;
+      pl.zeroer = lc == gi % ncta;
+      if (!dense) {
+        const int k = kK ? kK : __ldg(&g->k);
+        const int gcl = 31 - __clz(kChunk / (k * 32));
+        const int gc = 1 << gcl;
+        int a, b;
+        deal((__ldg(&g->d) + 15) >> 4, ncta, lc, a, b);
+        pl.p0 = a * 16;
+        pl.pg = (short)(b - a);
+        pl.pchunks = (short)((b - a + gc - 1) >> gcl);
+        deal((__ldg(&g->O) + 15) >> 4, ncta, lc, a, b);
+        pl.o0 = a * 16;
+        pl.og = (short)(b - a);
+        pl.ochunks = (short)((b - a + gc - 1) >> gcl);
+        pl.n_contrib = (short)__ldg(&g->n_contrib);
+        pl.gc_log2 = (short)gcl;
+      }
+    }
+    plan[t] = pl;
+  }
+}
+
 // kPairs = false compiles the pair logic out: stacks without concurrent groups run a smaller
 // loop (the per-phase code has to stay short: it is executed once per phase, straight through,
 // so its length is paid in instruction fetches).  kK != 0 is a build for stacks whose groups all
@@ -670,13 +794,14 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
   const unsigned* s_off = reinterpret_cast<const unsigned*>(smem + kOffOff);
   unsigned char* ring = smem + kOffRing;
   float* s_xb = reinterpret_cast<float*>(smem + kOffX);
-  float* s_c = reinterpret_cast<float*>(smem + kOffC);
+  unsigned short* s_xt = reinterpret_cast<unsigned short*>(smem + kOffXt);
+  unsigned short* s_cb = reinterpret_cast<unsigned short*>(smem + kOffCb);
   unsigned long long* s_fx = reinterpret_cast<unsigned long long*>(smem + kOffFx);
-  float* s_red = reinterpret_cast<float*>(smem + kOffRed);
   Plan* plan = reinterpret_cast<Plan*>(smem + kOffPlan);
   volatile int* abort = &misc->abort;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = gridDim.x, cta = blockIdx.x;
+  const int lg = lane >> 2, lt = lane & 3;   // row and column pair of this lane in a tensor-core operand
   constexpr int kStatWarp = kNW - 1;   // statistics of x and the collection of max|x|; the others run pass 1
   constexpr int kP1 = kNW - 1;         // warps of pass 1
 
@@ -698,95 +823,26 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
   };
   auto desc_store = [&](int g0, int cnt, uint32_t w) {
     if (tid < cnt * kDescWords) {
-      const int j = tid >= kDescWords ? 1 : 0;
+      const int j = tid / kDescWords;
       reinterpret_cast<uint32_t*>(smem + kOffDesc + ((g0 + j) & (kDescSlots - 1)) * 256)[tid - j * kDescWords] = w;
     }
   };
-  // one warp: request this CTA's rows of x for tick `tt` into buffer tt & 1
-  auto request_x = [&](int tt) {
-    const Plan& pn = plan[tt];
-    if (pn.kind != 1) return;
-    const PersistGroup& gn = desc(pn.gi);
-    const float* src = gn.x + (long long)slot_io * gn.x_step_stride + (size_t)p.token * gn.d + pn.p0;
-    float* dst = s_xb + (tt & 1) * kPersistMaxPRows;
-    for (int i = lane; i < pn.prow; i += 32) cp_async4(dst + i, src + i);
-  };
-
-  // the statistics warp: max |x| and sum x^2 over this CTA's rows of x for tick `tt` (the rows
-  // have been requested); the maximum is published at once as a tagged word, the sum is kept
-  // for the tick's exchange
-  auto publish_stats = [&](int tt) {
-    const Plan& pn = plan[tt];
-    if (pn.kind != 1) return;
-    cp_async_wait_all();
-    __syncwarp();
-    const float* sx = s_xb + (tt & 1) * kPersistMaxPRows;
-    float amax = 0.f, s2 = 0.f;
-#pragma unroll 1
-    for (int i = lane; i < pn.prow; i += 32) {
-      const float v = sx[i];
-      amax = fmaxf(amax, fabsf(v));
-      s2 = fmaf(v, v, s2);
-    }
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-      amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
-      s2 += __shfl_xor_sync(0xffffffffu, s2, o);
-    }
-    // fmaxf drops NaN, the sum keeps it (and overflows to inf for huge inputs):
-    // s2 - s2 is non-zero exactly when some x_i is NaN or inf (or x^2 overflowed)
-    if (lane == 0) {
-      const unsigned bits = (s2 - s2 == 0.f) ? __float_as_uint(amax) : 0x7fc00000u;
-      if (pn.prow > 0) st_relaxed_u32(desc(pn.gi).xmax + pn.lc, bits | (tag << 31));
-      misc->x2_part[tt & 1] = s2;
-    }
-  };
-
-  // ---- the plan of this launch for this CTA, one thread per tick
-#pragma unroll 1
-  for (int t = tid; t < n_ticks; t += kNC) {
-    Plan pl{};
-    pl.gi = pl.gi0 = -1;
-    if (t < p.n_phases) {
-      const int gi0 = __ldg(p.phase_first + t);
-      const PersistGroup* ga = p.groups + gi0;
-      const int len = kPairs ? __ldg(&ga->phase_len) : 1;
-      int gi = gi0;
-      if (kPairs && len == 2 && cta >= __ldg(&ga->cta0) + __ldg(&ga->ncta)) gi = gi0 + 1;
-      const PersistGroup* g = p.groups + gi;
-      const bool dense = __ldg(&g->flags) & GSI_FLAG_DENSE;
-      pl.gi = (short)gi;
-      pl.gi0 = (short)gi0;
-      pl.len = (unsigned char)len;
-      pl.next_len = (unsigned char)(kPairs ? __ldg(&ga->next_len) : min(__ldg(&ga->next_len), 1));
-      pl.kind = dense ? 2 : 1;
-      const int lc = cta - __ldg(&g->cta0), ncta = __ldg(&g->ncta);
-      pl.lc = (short)lc;
-      pl.zeroer = lc == gi % ncta;
-      if (!dense) {
-        const int d = __ldg(&g->d), O = __ldg(&g->O), pr = __ldg(&g->p_rows), orw = __ldg(&g->o_rows);
-        const int k = kK ? kK : __ldg(&g->k);
-        const int rc = kChunk / (k * 2);
-        const int p0 = min(d, lc * pr), p1 = min(d, p0 + pr);
-        const int o0 = min(O, lc * orw), o1 = min(O, o0 + orw);
-        pl.p0 = p0;
-        pl.o0 = o0;
-        pl.prow = (short)(p1 - p0);
-        pl.orow = (short)(o1 - o0);
-        pl.pchunks = (short)((p1 - p0 + rc - 1) / rc);
-        pl.ochunks = (short)((o1 - o0 + rc - 1) / rc);
-        pl.n_contrib = (short)__ldg(&g->n_contrib);
-      }
-    }
-    plan[t] = pl;
+  // the operand rows / columns beyond the three terms stay zero for the whole launch
+  for (int i = tid; i < (2 * 4096 + 8192) / 4; i += kNC) reinterpret_cast<uint32_t*>(smem + kOffXt)[i] = 0u;
+  // the descriptors of the first two phases (descriptors are staged two phases ahead)
+  {
+    const int cnt = plan[0].len + (p.n_phases > 1 ? plan[1].len : 0);
+    desc_store(0, cnt, desc_load(0, cnt));
   }
-  // the first phase's descriptors (the second slot is used only if the phase is a pair)
-  desc_store(0, min(p.n_groups, 2), desc_load(0, min(p.n_groups, 2)));
   csync();
-  if (warp == kStatWarp) {
-    request_x(0);
-    cp_async_commit();
-    publish_stats(0);
+  if (warp == kStatWarp) {   // the first tick's rows of x: nothing ran ahead of it
+    stat_warp_step(smem, 0, true, slot_io, p.token, tag);
+    stat_warp_step(smem, 0, false, slot_io, p.token, tag);
+    if (plan[0].kind == 1) {
+      unsigned xw[kXmaxWords];
+      xmax_issue(desc(plan[0].gi).xmax, plan[0].n_contrib, xw);
+      xmax_collect(smem, 0, tag, p.spin_limit, p.status, xw[0], xw[1], xw[2], xw[3], xw[4]);
+    }
   }
 
   unsigned mask_pp = 0;          // gates that fired in the phase before the previous one
@@ -801,33 +857,23 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     const bool gsi = pl.kind == 1, dense = pl.kind == 2;
     const PersistGroup& g = desc(pl.gi);        // read only when the tick has a group
     const int k = gsi ? (kK ? kK : g.k) : 0;
-    const int prow = pl.prow, orow = pl.orow, pchunks = pl.pchunks, ochunks = pl.ochunks;
+    const int KT = k >> 4;                      // tile columns
+    const int pg = pl.pg, og = pl.og, pchunks = pl.pchunks, ochunks = pl.ochunks, gcl = pl.gc_log2;
     const int n_contrib = pl.n_contrib, lc = pl.lc;
     const int len_p = t >= 1 ? plan[t - 1].len : 0, g_p = t >= 1 ? plan[t - 1].gi0 : 0;
-    float* s_x = s_xb + (t & 1) * kPersistMaxPRows;
+    const float* s_x = s_xb + (t & 1) * kPersistMaxPRows;
     unsigned long long* acc = gsi ? g.acc + (size_t)parity * (k + 4) : nullptr;
     const int tp = (t & 1) * 2;
 
-    Geo q{};
-    if (gsi) {
-      q.KV = k >> 3;
-      q.lpr_log2 = q.KV >= 32 ? 5 : 31 - __clz(q.KV);
-      q.vpl = q.KV > 32 ? q.KV >> 5 : 1;
-      q.rc_log2 = 31 - __clz(kChunk / 2) - (31 - __clz(k));  // rows per chunk = 8192 / k
-      q.sub = lane >> q.lpr_log2;
-      q.cl = lane & ((1 << q.lpr_log2) - 1);
-    }
-    const int LPR = 1 << q.lpr_log2, rpp_log2 = 5 - q.lpr_log2, rc = 1 << q.rc_log2;
+    // the descriptors of the phase after the next: requested now, stored after pass 1
+    const int g_stage = t + 2 < p.n_phases ? plan[t + 2].gi0 : 0, n_stage = t + 2 < p.n_phases ? plan[t + 2].len : 0;
+    const uint32_t desc_word = desc_load(g_stage, n_stage);
 
-    // the next phase's descriptors: requested now, stored after pass 1
-    const uint32_t desc_word = desc_load(pl.gi0 + pl.len, pl.next_len);
-
-    // ---- A. this CTA's rows of x have arrived (requested one phase ago); the bulk reduction
-    //      of the previous tick has read its source
-    if (tid == 0) {
-      bulk_reduce_wait_read();
-      misc->fire[tp] = misc->fire[tp + 1] = 0;
-    }
+    // ---- A. this CTA's rows of x have arrived and are in operand form (the statistics warp
+    //      saw to it during the previous tick); the bulk reduction of the previous tick has
+    //      read its source
+    if (lane == 0 || tid == kNC - 1) bulk_reduce_wait_read();   // the lanes that issue bulk reductions
+    if (tid == 0) misc->fire[tp] = misc->fire[tp + 1] = 0;
     if (pl.zeroer) {  // this CTA clears the group's counters for the next launch
       if (gsi) {
 #pragma unroll 1
@@ -837,98 +883,81 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     }
     csync();
     tr.mark(0);
+    // the statistics warp works one tick ahead: the next phase's rows of x are requested now,
+    // their statistics are published while this phase's exchange is in flight, and the other
+    // CTAs' words are collected during the row passes (the inputs of a stack are pre-staged)
+    if (warp == kStatWarp && t + 1 < n_ticks) stat_warp_step(smem, t + 1, true, slot_io, p.token, tag);
 
     const unsigned n_p0 = n;
     n += pchunks;
+    // partial c of this warp's tile columns kt = warp * tpw + s: lanes 0..3 hold, after the
+    // folds below, columns 16 kt + 8 m + 2 lane + v in cacc[s][m][v]
+    constexpr int kTpwMax = kK ? (kK / 16 + kP1 - 1) / kP1 : 3;
+    const int tpw = kK ? kTpwMax : (KT + kP1 - 1) / kP1;
+    float cacc[kTpwMax][2][4];
     if (gsi) {
       if (warp == kStatWarp) {
-        // ---- the group's max |x|: collect the tagged words of all contributing CTAs (lane l
-        //      owns words l, l+32, ...; they were published during the previous tick) while
-        //      the other warps run pass 1
-        unsigned m = 0, it = 0;
-        bool done = false;
-        while (!done) {
-          bool all = true;
-          m = 0;
-#pragma unroll
-          for (int i = 0; i < kPersistMaxGrid / 32; ++i) {   // all loads in flight together
-            const int w_i = lane + 32 * i;
-            if (w_i < n_contrib) {
-              const unsigned w = ld_relaxed_u32(g.xmax + w_i);
-              all = all && ((w >> 31) == tag);
-              m = max(m, w & 0x7fffffffu);
-            }
-          }
-          done = __all_sync(0xffffffffu, all);
-          if (!done && (++it > p.spin_limit || ((it & 1023u) == 0 && *abort))) {
-            if (!*abort && lane == 0) fail(p, misc, 4);
-            break;
-          }
-        }
-#pragma unroll
-        for (int o = 16; o > 0; o >>= 1) m = max(m, __shfl_xor_sync(0xffffffffu, m, o));
-        if (lane == 0) misc->amax_bits = m;
+        // (the group's max |x| was collected by this warp during the previous tick)
       } else {
-        // ---- B. pass 1: partial c over this CTA's basis rows
+        // ---- B. pass 1 on the tensor cores: D[term of x][column j] += X[term][row i] P[i][j];
+        //      the rows of x are the A operand (three terms in rows 0..2), a tile of P, each of
+        //      its four 8 x 8 blocks transposed in registers, is the B operand of two
+        //      instructions (columns 0..7 and 8..15 of the tile)
         ok = chunks_landed(smem, n_p0, pchunks, abort);
         tr.mark(1);
-#pragma unroll 1
-        for (int u = 0; u < q.vpl; ++u) {
-          const int cv = q.cl + u * LPR;
-          float a8[8];
 #pragma unroll
-          for (int e = 0; e < 8; ++e) a8[e] = 0.f;
+        for (int s3 = 0; s3 < kTpwMax; ++s3)
+#pragma unroll
+          for (int m = 0; m < 2; ++m)
+#pragma unroll
+            for (int v = 0; v < 4; ++v) cacc[s3][m][v] = 0.f;
+        const unsigned short* xt = s_xt + (t & 1) * 2048;
+        if (ok) {
 #pragma unroll 1
-          for (int ci = 0; ci < pchunks; ++ci) {
-            if (!ok) break;
-            const uint4* tile = reinterpret_cast<const uint4*>(ring + s_off[(n_p0 + ci) % kNB]);
-            const int r_lo = ci << q.rc_log2, rows = min(rc, prow - r_lo);
-#pragma unroll 2
-            for (int row = (warp << rpp_log2) + q.sub; row < rows; row += kP1 << rpp_log2) {
-              const float xv = s_x[r_lo + row];
-              const uint4 w = tile[(size_t)row * q.KV + cv];
-              a8[0] = fmaf(__uint_as_float(w.x << 16), xv, a8[0]);
-              a8[1] = fmaf(__uint_as_float(w.x & 0xFFFF0000u), xv, a8[1]);
-              a8[2] = fmaf(__uint_as_float(w.y << 16), xv, a8[2]);
-              a8[3] = fmaf(__uint_as_float(w.y & 0xFFFF0000u), xv, a8[3]);
-              a8[4] = fmaf(__uint_as_float(w.z << 16), xv, a8[4]);
-              a8[5] = fmaf(__uint_as_float(w.z & 0xFFFF0000u), xv, a8[5]);
-              a8[6] = fmaf(__uint_as_float(w.w << 16), xv, a8[6]);
-              a8[7] = fmaf(__uint_as_float(w.w & 0xFFFF0000u), xv, a8[7]);
+          for (int R = 0; R < pg; ++R) {
+            const uint2 ax = *reinterpret_cast<const uint2*>(xt + (R * 32 + lane) * 4);
+            const uint4 a = make_uint4(ax.x, 0u, ax.y, 0u);
+            const int ci = R >> gcl, rr = R - (ci << gcl);
+            const unsigned char* trow = ring + s_off[(n_p0 + ci) % kNB] + (size_t)rr * KT * 512 + lane * 16;
+#pragma unroll
+            for (int s3 = 0; s3 < kTpwMax; ++s3) {
+              const int kt = warp * tpw + s3;
+              if (s3 < tpw && kt < KT) {
+                const uint4 w = *reinterpret_cast<const uint4*>(trow + kt * 512);
+                mma_bf16(cacc[s3][0], a, movmatrix_trans(w.x), movmatrix_trans(w.y));
+                mma_bf16(cacc[s3][1], a, movmatrix_trans(w.z), movmatrix_trans(w.w));
+              }
             }
           }
-#pragma unroll 1
-          for (int o = LPR; o < 32; o <<= 1) {
-#pragma unroll
-            for (int e = 0; e < 8; ++e) a8[e] += __shfl_xor_sync(0xffffffffu, a8[e], o);
-          }
-          if (q.sub == 0) {
-            float4* dst = reinterpret_cast<float4*>(s_red + warp * 512 + cv * 8);
-            dst[0] = make_float4(a8[0], a8[1], a8[2], a8[3]);
-            dst[1] = make_float4(a8[4], a8[5], a8[6], a8[7]);
-          }
         }
+        // the three terms of x sit in rows 0..2 = lanes 0-3, 4-7, 8-11: fold them onto lanes 0-3
+#pragma unroll
+        for (int s3 = 0; s3 < kTpwMax; ++s3)
+#pragma unroll
+          for (int m = 0; m < 2; ++m)
+#pragma unroll
+            for (int v = 0; v < 2; ++v) {
+              float z = cacc[s3][m][v];
+              z += __shfl_down_sync(0xffffffffu, z, 4) + __shfl_down_sync(0xffffffffu, z, 8);
+              cacc[s3][m][v] = z;
+            }
         if (!ok && !*abort) fail(p, misc, 5);
       }
     }
-    desc_store(pl.gi0 + pl.len, pl.next_len, desc_word);
+    desc_store(g_stage, n_stage, desc_word);
     csync();
     tr.mark(2);
     if (*abort) return;
     // the next phase's rows of x travel while this phase runs its exchange (its descriptors
     // are in place now) ...
-    if (warp == kStatWarp && t + 1 < n_ticks) {
-      request_x(t + 1);
-      cp_async_commit();
-    }
 
-    // ---- D. the exchange: this phase's partial c and ||x||^2 as ONE bulk reduction of k + 2
-    //      fixed-point words into the group's accumulators, the previous phase's ||r||^2 as
-    //      one atomic
+    // ---- D. the exchange: this phase's partial c and ||x||^2 as bulk reductions of
+    //      fixed-point words into the group's accumulators (one per pass-1 warp), the previous
+    //      phase's ||r||^2 as one atomic
     bool nonfinite = false;
     double inv_scale = 0.0;
     if (gsi) {
-      const unsigned amax_bits = misc->amax_bits;
+      const unsigned amax_bits = misc->amax_bits[t & 1];
       nonfinite = amax_bits >= 0x7f800000u;
       const float amax = __uint_as_float(amax_bits);
       // fixed-point scales: |partial c_j| <= amax * rows * max|P| < 2^e, partial ||x||^2 <= rows * amax^2 < 2^ex
@@ -940,24 +969,40 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
         inv_scale = pow2d(e - 43);
         scale_x2 = pow2d(43 - exp_above((double)amax * (double)amax * (double)g.p_rows));
       }
-      if (prow > 0) {
-#pragma unroll 1
-        for (int j = tid; j < k; j += kNC) {
-          float sum = 0.f;
+      if (pg > 0) {
+        // every pass-1 warp converts its own columns and sends them off with a bulk reduction
+        // of its own: no barrier of the CTA stands between pass 1 and the exchange
+        if (warp * tpw < KT && warp < kP1) {
+          if (lane < 4) {
 #pragma unroll
-          for (int w = 0; w < kP1; ++w) sum += s_red[w * 512 + j];
-          const long long v = scale != 0.0 ? __double2ll_rn((double)sum * scale) : 0ll;
-          s_fx[j] = kOne + (unsigned long long)v;
+            for (int s3 = 0; s3 < kTpwMax; ++s3) {
+              const int kt = warp * tpw + s3;
+              if (s3 < tpw && kt < KT) {
+#pragma unroll
+                for (int m = 0; m < 2; ++m)
+#pragma unroll
+                  for (int v = 0; v < 2; ++v) {
+                    const long long fx =
+                        scale != 0.0 ? __double2ll_rn((double)cacc[s3][m][v] * scale) : 0ll;
+                    s_fx[16 * kt + 8 * m + 2 * lane + v] = kOne + (unsigned long long)fx;
+                  }
+              }
+            }
+          }
+          __syncwarp();
+          if (lane == 0) {
+            const int c0 = 16 * warp * tpw, c1 = min(k, c0 + 16 * tpw);
+            bulk_reduce_add_u64(acc + c0, s_fx + c0, (uint32_t)(c1 - c0) * 8);
+          }
         }
         if (tid == kNC - 1) {
           const long long v = scale_x2 != 0.0 ? __double2ll_rn((double)misc->x2_part[t & 1] * scale_x2) : 0ll;
           s_fx[k] = kOne + (unsigned long long)v;
           s_fx[k + 1] = 0ull;
+          bulk_reduce_add_u64(acc + k, s_fx + k, 16u);
         }
       }
     }
-    csync();
-    if (tid == 0 && gsi && prow > 0) bulk_reduce_add_u64(acc, s_fx, (uint32_t)(k + 2) * 8);
     if (contrib_p && tid == 32) {
       float sr = 0.f;   // fixed order: the sum does not depend on which warp finished first
 #pragma unroll
@@ -969,53 +1014,74 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       if (!(vd >= 0.0)) vd = 0.0;
       red_add_u64(r2word_p, kOne + (unsigned long long)__double2ll_rn(vd));
     }
+    if (warp == kStatWarp && t + 1 < n_ticks) stat_warp_step(smem, t + 1, false, slot_io, p.token, tag);
     tr.mark(3);
 
-    // ---- E. wait until every contributing CTA has been added: warp 0 polls the accumulators
-    //      of c (contiguous: lane l owns words l, l+32, ..., all its loads in flight together,
-    //      one round trip per attempt), warp 1 the scalars: lane 0 this phase's ||x||^2, lanes
-    //      1+2u / 2+2u the previous phase's ||r||^2 and published ||x||^2 of its group u.
-    if (gsi && warp == 0) {
+    // ---- E. wait until every contributing CTA has been added: four warps poll a quarter of
+    //      the accumulators of c each (contiguous words, all loads of a lane in flight together,
+    //      one round trip per attempt) and leave c as three bf16 terms in operand order;
+    //      warp 1 polls the scalars: lane 0 this phase's ||x||^2, lanes 1+2u / 2+2u the
+    //      previous phase's ||r||^2 and published ||x||^2 of its group u.
+    if (gsi && (warp == 0 || (warp >= 2 && warp <= 4))) {
+      constexpr int kWpl = kK ? (kK + 127) / 128 : 4;   // words per lane
+      const int q4 = warp == 0 ? 0 : warp - 1;          // this warp's quarter of the words
+      unsigned long long w[kWpl];
       unsigned it = 0;
       bool done = false;
       while (!done) {
         bool all = true;
-#pragma unroll 8
-        for (int j = lane; j < k; j += 32) {
-          const unsigned long long w = ld_relaxed_u64(acc + j);
-          all = all && ((unsigned)((w + (kOne >> 1)) >> kCountShift) == (unsigned)n_contrib);
-          const long long val = (long long)(w - ((unsigned long long)n_contrib << kCountShift));
-          s_c[j] = (float)((double)val * inv_scale);
+#pragma unroll
+        for (int i = 0; i < kWpl; ++i) {
+          const int j = (q4 + 4 * i) * 32 + lane;
+          w[i] = j < k ? ld_relaxed_u64(acc + j) : ((unsigned long long)n_contrib << kCountShift);
         }
+#pragma unroll
+        for (int i = 0; i < kWpl; ++i)
+          all = all && ((unsigned)((w[i] + (kOne >> 1)) >> kCountShift) == (unsigned)n_contrib);
         done = __all_sync(0xffffffffu, all);
         if (!done && (++it > p.spin_limit || ((it & 1023u) == 0 && *abort))) {
           if (!*abort && lane == 0) fail(p, misc, 6);
           break;
         }
       }
+#pragma unroll
+      for (int i = 0; i < kWpl; ++i) {
+        const int j = (q4 + 4 * i) * 32 + lane;
+        if (j < k) {
+          const long long val = (long long)(w[i] - ((unsigned long long)n_contrib << kCountShift));
+          unsigned short tm[3];
+          split3((float)((double)val * inv_scale), tm);
+          const int slot = term_slot(j >> 4, j & 15, 0);
+          s_cb[slot] = tm[0];
+          s_cb[slot + 16] = tm[1];   // the next term is the next column of the operand: four lanes on
+          s_cb[slot + 32] = tm[2];
+        }
+      }
     }
     if (warp == 1) {
-      // what this lane watches: an accumulator (count in the upper bits) or a tagged word
-      const int u = (lane - 1) >> 1;
-      const bool settle = lane >= 1 && lane <= 4 && u < len_p && !(desc(g_p + u).flags & GSI_FLAG_DENSE);
-      const PersistGroup& gs = desc(g_p + (u & 1));   // read only when `settle`
-      const bool w_x2 = gsi && lane == 0;
-      const bool w_r2 = settle && (lane & 1), w_pub = settle && !(lane & 1);
+      // lane 0: this phase's ||x||^2 (an accumulator: arrivals in the upper bits); lanes
+      // 1 + 2u / 2 + 2u: the previous phase's ||r||^2 (accumulator) and its gate threshold
+      // (tagged word) of group u
+      // (on CTA 0, which writes the logs, lanes 5 + u also fetch the group's published ||x||^2)
+      const int u = lane <= 4 ? (lane - 1) >> 1 : lane - 5;
+      const bool live_u = u >= 0 && u < len_p && !(desc(g_p + u).flags & GSI_FLAG_DENSE);
+      const bool settle = lane >= 1 && lane <= 4 && live_u;
+      const PersistGroup& gs = desc(g_p + (u & 1));   // read only when `live_u`
+      const bool w_x2 = gsi && lane == 0, w_r2 = settle && (lane & 1);
+      const bool w_thr = (settle && !(lane & 1)) || (cta == 0 && lane >= 5 && lane <= 6 && live_u);
       const unsigned long long* wp = w_x2   ? acc + k
                                      : w_r2 ? gs.acc + (size_t)parity * (gs.k + 4) + gs.k + 2
-                                            : gs.pub;
+                                            : gs.pub + (lane <= 4 ? 1 : 0);
       const unsigned want = w_x2 ? (unsigned)n_contrib : (unsigned)gs.n_contrib;
       unsigned long long w = 0;
       unsigned it = 0;
       bool done = false;
       while (!done) {
         bool mine = true;
-        if (w_x2 || w_r2) {
+        if (w_x2 || w_r2 || w_thr) {
           w = ld_relaxed_u64(wp);
-          mine = (unsigned)((w + (kOne >> 1)) >> kCountShift) == want;
-        } else if (w_pub) {
-          w = ld_relaxed_u64(wp);
-          mine = (unsigned)(w >> 63) == tag;
+          mine = w_thr ? (unsigned)(w >> 63) == tag
+                       : (unsigned)((w + (kOne >> 1)) >> kCountShift) == want;
         }
         done = __all_sync(0xffffffffu, mine);
         if (!done && (++it > p.spin_limit || ((it & 1023u) == 0 && *abort))) {
@@ -1025,33 +1091,38 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       }
       if (w_x2) {
         const long long val = (long long)(w - ((unsigned long long)n_contrib << kCountShift));
-        const double amax = (double)__uint_as_float(misc->amax_bits);
+        const double amax = (double)__uint_as_float(misc->amax_bits[t & 1]);
         const double x2 = nonfinite ? __longlong_as_double(0x7ff8000000000000ll)
                           : val > 0 ? (double)val * pow2d(exp_above(amax * amax * (double)g.p_rows) - 43)
                                     : 0.0;
         misc->x2 = x2;
-        // every CTA decides this group's gate in the next tick from the published value
-        if (lc == 0)
+        if (lc == 0) {
+          // Every CTA settles this group's gate in the next tick by comparing integers:
+          // ||r||^2 < eps^2 ||x||^2 (both sides >= 0; false for x = 0) in the fixed-point
+          // units 2^(e - 44) of ||r||^2 is sum < ceil(eps^2 ||x||^2 2^(44 - e)).  Bit 62 marks a
+          // non-finite token (never fast, never streamed).  ||x||^2 itself goes out for rho.
+          const double eps = (double)g.eps;
+          const double thr = fmin(ceil(eps * eps * x2 * pow2d(44 - (x2 > 0.0 ? exp_above(x2) : 0))), 2305843009213693952.0);
+          const unsigned long long tw = nonfinite ? (1ull << 62) : (unsigned long long)thr;
+          st_relaxed_u64(g.pub + 1, tw | ((unsigned long long)tag << 63));
           st_relaxed_u64(g.pub, ((unsigned long long)__double_as_longlong(x2) & ~(1ull << 63)) |
                                     ((unsigned long long)tag << 63));
+        }
       }
-      // the previous phase's gates: the lane that holds ||r||^2 of group u takes ||x||^2 from
-      // its neighbour and decides
+      // the lane that holds ||r||^2 of group u takes the threshold from its neighbour
       const unsigned long long w_nb = __shfl_down_sync(0xffffffffu, w, 1);
+      const unsigned long long wx = __shfl_sync(0xffffffffu, w, 5 + (u & 1));
       if (w_r2) {
-        const long long val = (long long)(w - ((unsigned long long)want << kCountShift));
-        const double x2 = __longlong_as_double((long long)(w_nb & ~(1ull << 63)));
-        const bool finite = x2 == x2;
-        const int ex = x2 > 0.0 ? exp_above(x2) : 0;
-        const double r2 = (double)val * pow2d(ex - 44);
-        const double eps = (double)gs.eps;
-        // ||r|| < eps ||x||  <=>  ||r||^2 < eps^2 ||x||^2  (both sides >= 0); false for x = 0
-        const bool fast = finite && (r2 < eps * eps * x2);
+        const unsigned long long val = w - ((unsigned long long)want << kCountShift);
+        const bool finite = !(w_nb & (1ull << 62));
+        const bool fast = finite && val < (w_nb & ((1ull << 62) - 1));
         misc->fire[tp + u] = (!fast && finite && !(gs.flags & GSI_FLAG_STATIC_PROJECTION)) ? 1 : 0;
-        if (cta == 0) {
+        if (cta == 0) {   // the logs: rho from ||r||^2 2^-e and ||x||^2 2^-e, both in the float range
+          const double x2 = __longlong_as_double((long long)(wx & ~(1ull << 63)));
+          const int ex = x2 > 0.0 ? exp_above(x2) : 0;
           const size_t at = ((size_t)slot_io * p.log_step_stride + (g_p + u)) * p.n_tokens + p.token;
           p.gate_log[at] = fast ? 0 : 1;
-          if (p.rho_log)   // both operands scaled into the float range: ||r||^2 2^-e and ||x||^2 2^-e
+          if (p.rho_log)
             p.rho_log[at] = finite ? sqrtf(__fdividef((float)((double)val * 5.6843418860808015e-14),
                                                       (float)(x2 * pow2d(-ex))))
                                    : __int_as_float(0x7fc00000);
@@ -1077,20 +1148,21 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     }
     const double x2_own = gsi ? misc->x2 : 0.0;
     // ... and their statistics are published a row pass ahead of the next phase's exchange
-    if (warp == kStatWarp && t + 1 < n_ticks) publish_stats(t + 1);
+    // (this warp then fetches the words of the other CTAs for the next phase: the loads fly
+    // during its row units, the check comes after them)
+    unsigned xw[kXmaxWords];
+    const bool xmax_next = warp == kStatWarp && t + 1 < n_ticks && plan[t + 1].kind == 1;
+    if (xmax_next) xmax_issue(desc(plan[t + 1].gi).xmax, plan[t + 1].n_contrib, xw);
 
-    // ---- G / I. the row passes, one copy of the code for both: part 0 the residual rows of
-    //      the basis slab (still in the ring), part 1 the image rows.  Items of eight rows
-    //      (one lane group each) are dealt round-robin over the joint numbering of both
+    // ---- G / I. the row passes on the tensor cores, one copy of the code for both: part 0 the
+    //      residual rows of the basis slab (still in the ring), part 1 the image rows.  A unit
+    //      is a tile row (16 matrix rows): D[row][term of c] += T[row][column] C[column][term],
+    //      the tiles as they lie in the ring are the A operand, c (three terms in columns
+    //      0..2) the B operand.  Units are dealt round-robin over the joint numbering of both
     //      parts, so the warps are loaded evenly.  Every warp gives every chunk back once.
     // ---- H (between them). the W streams of the tick, one call site: the gated residuals
     //      of the phase before the previous one, then this phase's own stream if it is a
     //      dense group (followed by a grid barrier that keeps a dense stack in model order).
-    const int itemsP = (prow + 7) >> 3, itemsO = (orow + 7) >> 3;
-    const int padP = ((itemsP + (1 << rpp_log2) - 1) >> rpp_log2) << rpp_log2;
-    const int padO = ((itemsO + (1 << rpp_log2) - 1) >> rpp_log2) << rpp_log2;
-    const int hold_log2 = q.lpr_log2 - 3;          // lanes per held row after reduce8
-    const int lanegroups = kNW << rpp_log2;
 #pragma unroll 1
     for (int part = 0; part < 2; ++part) {
       if (part == 1 && (mask_pp || dense)) {
@@ -1130,10 +1202,11 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       }
       if (!gsi) continue;
       const bool image = part == 1;
-      const int nchunks = image ? ochunks : pchunks, nrows = image ? orow : prow;
-      const int id0 = image ? padP : 0, id1 = image ? padP + padO : padP;
+      const int nchunks = image ? ochunks : pchunks, ngroups = image ? og : pg;
+      const int id0 = image ? pg : 0;
       const unsigned n0 = image ? n : n_p0;
-      float* out = image ? g.y + (size_t)p.token * g.O + pl.o0 : g.r + pl.p0;
+      const int row_base = image ? pl.o0 : pl.p0, row_end = image ? g.O : g.d;
+      float* out = image ? g.y + (size_t)p.token * g.O : g.r;
       if (image) {
         n += ochunks;
         ok = ok && chunks_landed(smem, n0, ochunks, abort);
@@ -1142,31 +1215,44 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       float sr = 0.f;
       int released = 0;
       if (ok) {
-        int id = (warp << rpp_log2) + q.sub;
-        if (id < id0) id += ((id0 - id + lanegroups - 1) / lanegroups) * lanegroups;
+        int id = warp;
+        if (id < id0) id += ((id0 - id + kNW - 1) / kNW) * kNW;
 #pragma unroll 1
-        for (; __any_sync(0xffffffffu, id < id1); id += lanegroups) {
-          const bool live = id < id1;
-          const int row0g = live ? (id - id0) << 3 : 0;            // first row, within the slab
-          const int ci = min(row0g >> q.rc_log2, nchunks - 1);
-          const int ci_warp = __shfl_sync(0xffffffffu, live ? ci : nchunks - 1, 0);  // ids ascend with the lane
+        for (; id < id0 + ngroups; id += kNW) {
+          const int R = id - id0;
+          const int ci = R >> gcl, rr = R - (ci << gcl);
           if (lane == 0)
-            for (; released < ci_warp; ++released) mbar_arrive(&empty[(n0 + released) % kNB]);
-          released = ci_warp;
-          const uint4* tile = reinterpret_cast<const uint4*>(ring + s_off[(n0 + ci) % kNB]);
-          const int r_lo = ci << q.rc_log2, rows = min(rc, nrows - r_lo);
-          const int row0 = row0g - r_lo;
-          float v[8];
-          dot8(tile, s_c, q, row0, rows, v);
-          const float dot = reduce8(v, q.cl, LPR);
-          const int row = row0 + (q.cl >> hold_log2);
-          if (live && (q.cl & ((1 << hold_log2) - 1)) == 0 && row < rows && row0g < nrows) {
-            if (image) {
-              out[r_lo + row] = nonfinite ? __int_as_float(0x7fc00000) : dot;
-            } else {
-              const float rv = s_x[r_lo + row] - dot;
-              out[r_lo + row] = rv;
-              sr = fmaf(rv, rv, sr);
+            for (; released < ci; ++released) mbar_arrive(&empty[(n0 + released) % kNB]);
+          released = ci;
+          const unsigned char* trow = ring + s_off[(n0 + ci) % kNB] + (size_t)rr * KT * 512 + lane * 16;
+          const unsigned char* cb = reinterpret_cast<const unsigned char*>(s_cb) + lane * 8;
+          float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll 2
+          for (int K = 0; K < KT; K += 2) {   // two chains of dependent instructions
+            const uint4 a0 = *reinterpret_cast<const uint4*>(trow + K * 512);
+            const uint2 b0 = *reinterpret_cast<const uint2*>(cb + K * 256);
+            const uint4 a1 = *reinterpret_cast<const uint4*>(trow + K * 512 + 512);
+            const uint2 b1 = *reinterpret_cast<const uint2*>(cb + K * 256 + 256);
+            mma_bf16(d0, a0, b0.x, b0.y);
+            mma_bf16(d1, a1, b1.x, b1.y);
+          }
+          // columns 0, 1 (lane pair 0) and 2 (lane pair 1) of D are the three terms of c
+          const float lo = d0[0] + d1[0], lo1 = d0[1] + d1[1], hi = d0[2] + d1[2], hi1 = d0[3] + d1[3];
+          const float lo2 = __shfl_down_sync(0xffffffffu, lo, 1), hi2 = __shfl_down_sync(0xffffffffu, hi, 1);
+          if (lt == 0) {
+#pragma unroll
+            for (int h = 0; h < 2; ++h) {
+              const float dot = h ? (hi + hi1) + hi2 : (lo + lo1) + lo2;
+              const int row = R * 16 + lg + 8 * h;
+              if (row_base + row < row_end) {
+                if (image) {
+                  out[row_base + row] = nonfinite ? __int_as_float(0x7fc00000) : dot;
+                } else {
+                  const float rv = s_x[row] - dot;
+                  out[row_base + row] = rv;
+                  sr = fmaf(rv, rv, sr);
+                }
+              }
             }
           }
         }
@@ -1182,15 +1268,16 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     }
     if (!ok && !*abort) fail(p, misc, 8);
     if (*abort) return;
+    if (xmax_next) xmax_collect(smem, t + 1, tag, p.spin_limit, p.status, xw[0], xw[1], xw[2], xw[3], xw[4]);
 
-    contrib_p = gsi && prow > 0;
+    contrib_p = gsi && pg > 0;
     if (gsi) {
       e_p = x2_own > 0.0 ? exp_above(x2_own) : 0;
       r2word_p = acc + k + 2;
     }
     mask_pp = mask_p;
   }
-  if (tid == 0) bulk_reduce_wait_read();
+  if (lane == 0 || tid == kNC - 1) bulk_reduce_wait_read();
   tr.flush(p);
   // Every CTA read the counters at its start and has since taken part in the
   // last group's exchange, so they may advance now.
@@ -1218,6 +1305,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_decode_step(const __grid_const
     misc->decision[0] = misc->decision[1] = misc->decision[2] = misc->decision[3] = 0u;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  make_plan<kPairs, kK>(p, smem);
   __syncthreads();
   if (threadIdx.x >= kNC) {
     if (threadIdx.x == kNC) producer(p, smem, misc);
