@@ -865,7 +865,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     unsigned long long* acc = gsi ? g.acc + (size_t)parity * (k + 4) : nullptr;
     const int tp = (t & 1) * 2;
 
-    // the descriptors of the phase after the next: requested now, stored after pass 1
+    // the descriptors of the phase after the next: requested now, stored before the barrier that ends the exchange
     const int g_stage = t + 2 < p.n_phases ? plan[t + 2].gi0 : 0, n_stage = t + 2 < p.n_phases ? plan[t + 2].len : 0;
     const uint32_t desc_word = desc_load(g_stage, n_stage);
 
@@ -944,10 +944,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
         if (!ok && !*abort) fail(p, misc, 5);
       }
     }
-    desc_store(g_stage, n_stage, desc_word);
-    csync();
     tr.mark(2);
-    if (*abort) return;
     // the next phase's rows of x travel while this phase runs its exchange (its descriptors
     // are in place now) ...
 
@@ -1129,6 +1126,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
         }
       }
     }
+    desc_store(g_stage, n_stage, desc_word);
     csync();
     tr.mark(4);
     if (*abort) return;
