@@ -28,9 +28,11 @@ if ROOT not in sys.path:
 
 METRIC = "decode tokens/s at GPT-J shapes, k=256, eps=0.05 (effective weight GB/s and % of HBM roofline alongside)"
 NOMINAL_HBM_GBS = 8000.0
-# dram bytes (read+write) per algorithmic byte of k_decode_step from the ncu capture summarised in
-# profiles/k_decode_step_gptj_L8_ncu_full.md (8-layer case; traffic grows in proportion to layers)
+# dram bytes (read+write) per algorithmic byte of k_decode_step, from an ncu capture of an
+# 8-layer case (traffic grows in proportion to the layers: every layer has its own weights)
 NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.02
+MIN_TIMED_SECONDS = 0.3     # the timed repeats together last at least this long
+MIN_REPEATS = 3
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -59,7 +61,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.index}", f"--query-gpu={self.Q}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "25"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -166,25 +168,36 @@ def capture_step(stack, stream):
     return graph
 
 
-def time_graph(graph, stack, stream, steps, warmup, barrier=None):
+def time_graph(graph, stack, stream, steps, warmup, barrier=None, repeats=MIN_REPEATS,
+               min_seconds=MIN_TIMED_SECONDS):
+    """Times `repeats` (at least three, and enough of them to last min_seconds) regions of
+    exactly `steps` replays each with CUDA events on the launch stream; every region walks
+    the pre-staged inputs from step 0.  Returns (median ms per step, [ms per step of every
+    region])."""
     import torch
+    per_region = []
     with torch.cuda.stream(stream):
         stack.seek(0, stream)
         for _ in range(warmup):
             graph.replay()
         stream.synchronize()
-        stack.seek(0, stream)
         if barrier:
             barrier()
         torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        e0.record(stream)
-        for _ in range(steps):
-            graph.replay()
-        e1.record(stream)
-        stream.synchronize()
+        elapsed = 0.0
+        while len(per_region) < repeats or (elapsed < min_seconds and len(per_region) < 64):
+            stack.seek(0, stream)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(steps):
+                graph.replay()
+            e1.record(stream)
+            stream.synchronize()
+            ms = e0.elapsed_time(e1)
+            per_region.append(ms / steps)
+            elapsed += ms * 1e-3
         torch.cuda.synchronize()
-    return e0.elapsed_time(e1) / steps  # ms per step
+    return statistics.median(per_region), per_region
 
 
 def time_host_steps(layers, xs, steps, warmup, stream, concurrent=()):
@@ -493,9 +506,9 @@ def main():
 
     sampler = ClockSampler(local_rank)
     sampler.start()
-    ms = time_graph(graph, stack, stream, args.steps, args.warmup, barrier)
+    ms, ms_regions = time_graph(graph, stack, stream, args.steps, args.warmup, barrier)
     clocks = sampler.stop()
-    ms_dense = time_graph(dgraph, dstack, stream, max(8, args.steps // 8), 3) if dense_arm else None
+    ms_dense = time_graph(dgraph, dstack, stream, max(8, args.steps // 8), 3, min_seconds=0.05)[0] if dense_arm else None
     ms_lib = time_library_dense(keep, xs, spec.batch, stream, max(8, args.steps // 8))
     gate_log = stack.gate_log.cpu().numpy()          # [n_steps][groups][B]
     used_steps = min(args.steps, n_steps)
@@ -528,6 +541,11 @@ def main():
             "unit": "tokens/s",
             "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_max, "higher_is_better": True,
+            "timing": {"repeats": len(ms_regions), "ms_per_step_median": statistics.median(ms_regions),
+                       "ms_per_step_min": min(ms_regions), "ms_per_step_max": max(ms_regions),
+                       "timed_seconds": sum(ms_regions) * args.steps * 1e-3,
+                       "protocol": "CUDA graph of one step; warm-up replays; >= 3 regions of exactly "
+                                   "`steps` replays each, CUDA events on the launch stream, median"},
             "scaling": "weak", "vs_baseline": None, "dtype": "f32",
             "data": "synthetic",
             "config": {
@@ -579,8 +597,31 @@ def main():
         }
         if e2e:
             out["e2e"] = e2e
+        if spec.batch > 1:   # fired tokens per (step, group): how often the gated GEMM runs, and how wide
+            nf = gate_log[:used_steps].sum(axis=2).reshape(-1)
+            edges = [0, 1, 2, 5, 9, 17, 33, spec.batch + 1]
+            out["n_fired_histogram"] = {
+                (f"{a}" if b == a + 1 else f"{a}-{b - 1}"): int(((nf >= a) & (nf < b)).sum())
+                for a, b in zip(edges[:-1], edges[1:]) if a <= spec.batch}
         if not args.no_cpu_baseline and world == 1:
             from oracle import gsi_oracle as O
+            # parity of the timed steps: the gate bytes the kernels logged against the oracle's
+            # decision on the same tokens (Algorithm 1 lines 1-4), every group of every layer
+            xs_cpu = [x.reshape(-1, x.shape[-1])[:used_steps * spec.batch].cpu().numpy() for x in xs]
+            flips = in_band = outside = 0
+            for gi, ((_, P), x) in enumerate(zip(keep, xs_cpu)):
+                pr = O.project(x, S.bits_of(P.cpu()), spec.eps)
+                got = gate_log[:used_steps, gi, :].reshape(-1)
+                with np.errstate(divide="ignore", invalid="ignore"):
+                    near = np.abs(pr["rho"] / np.float32(spec.eps) - 1.0) < 1e-3 if spec.eps > 0 else np.zeros(len(got), bool)
+                mism = pr["gate"] != got
+                flips += int(mism.sum())
+                in_band += int(near.sum())
+                outside += int((mism & ~near).sum())
+            out["parity"] = {"tokens_checked": int(sum(len(x) for x in xs_cpu)),
+                             "gate_mismatches_outside_band": outside, "gate_mismatches": flips,
+                             "tokens_within_1e-3_of_eps": in_band,
+                             "against": "oracle.project on the timed steps' inputs, all groups"}
             del stack, layers, dense_layers, keep
             torch.cuda.empty_cache()
             sample = OracleSample(spec, n_layers=min(4, spec.n_layers), n_tokens=1280)
