@@ -719,7 +719,7 @@ static gsi_status_t stack_enqueue(gsi_stack_t s, bool use_counter, gsi_stream_t 
     p.log_step_stride = G;
     p.status = s->status;
     p.trace = s->trace;
-    p.spin_limit = s->spin_limit;
+    p.spin_limit = s->spin_limit - 1;   // the kernels give up when a wait has polled more than this many times without success
     p.n_tokens = s->B;
     // one launch per token of the step (up to kPersistMaxTokens; larger batches take the
     // batched kernels): each is a complete decode step of that token, the last one advances

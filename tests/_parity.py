@@ -59,6 +59,26 @@ def compare_group(x, P, Ws, eps, y_gpu, gate_gpu, rho_gpu=None, rows=None, stati
                 max_rel_err=max_rel, oracle=pr)
 
 
+def boundary_rows(n_rows, n_random, rng, grid=148):
+    """Output rows a sampled-row test always looks at, besides `n_random` random ones: the first
+    and last rows of the map, the edges of the 16-row tiles, the first and last rows of the
+    slabs the CTAs own (image rows dealt in tiles of 16 over 148, 42 and 106 CTAs, the shares
+    the benchmark's schedule uses; W rows dealt ceil(n / grid) per CTA), i.e. the ragged tails
+    the kernels clamp."""
+    rows = {0, 1, 15, 16, 17, n_rows - 17, n_rows - 16, n_rows - 2, n_rows - 1}
+    tiles = (n_rows + 15) // 16
+    for share in (grid, 42, 106):
+        for c in (0, 1, share // 2, share - 2, share - 1):
+            a = c * tiles // share if tiles >= share else min(c, tiles)
+            rows.update({16 * a - 1, 16 * a, 16 * a + 15})
+    per = (n_rows + grid - 1) // grid
+    for c in (1, grid // 2, grid - 1):
+        rows.update({c * per - 1, c * per, c * per + per - 1})
+    rows = {r for r in rows if 0 <= r < n_rows}
+    extra = rng.choice(n_rows, min(n_random, n_rows), replace=False)
+    return np.array(sorted(rows | set(int(e) for e in extra)))
+
+
 def image_ulp_check(W, P, wp_gpu):
     """The stored image is bf16_rne(W P) with fp32 accumulation: it must lie
     within one bf16 ulp of the fp64 product (half an ulp of rounding plus ties),

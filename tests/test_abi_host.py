@@ -79,5 +79,6 @@ def test_null_and_misaligned_arguments_are_rejected_on_the_host():
     assert lib.gsi_stack_workspace_bytes(84) > 0
     assert lib.gsi_stack_set_concurrent(None, 0, 1) == INVALID
     assert lib.gsi_stack_set_mode(None, 0) == INVALID
+    assert lib.gsi_stack_set_spin_limit(None, 1) == INVALID
     assert lib.gsi_extend_basis(None, 4096, 0.05, 4096, None, None, None) == INVALID
     assert lib.gsi_get_status(None, None) == INVALID

@@ -6,7 +6,7 @@ component's stream capture is open, a hot path that must never enter the CUDA
 allocator.  ``gsi_forward_static`` serves them from a scratch array compiled
 into the library.  This test drives it through the C ABI, twice in a row (the
 array keeps the first call's contents, so the second call proves the clearing),
-and compares with ``gsi_forward_n``.  It is collected last on purpose.
+and compares with ``gsi_forward_n`` and with the fp64 oracle.  It is collected last on purpose.
 """
 import ctypes as C
 
@@ -15,7 +15,7 @@ import pytest
 import torch
 
 import synthetic as S
-from _parity import Y_TOL
+from _parity import Y_TOL, compare_group
 
 pytestmark = pytest.mark.gpu
 
@@ -56,6 +56,8 @@ def test_static_entry_point_matches_workspace_entry_point_twice():
             scale = y_ref.abs().amax(dim=1, keepdim=True)
             assert ((y - y_ref).abs() <= Y_TOL * scale).all(), f"call {call}"
             assert torch.allclose(rho, rho_ref, rtol=1e-5, atol=0), f"call {call}"
+            # ... and against the oracle itself, at the acceptance bar of every other entry point
+            compare_group(x, P, Ws, eps, y.cpu().numpy(), gate.cpu().numpy(), rho.cpu().numpy())
 
 
 def test_static_entry_point_rejects_what_its_scratch_cannot_hold():
