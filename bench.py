@@ -417,7 +417,7 @@ def main():
     ap.add_argument("--batch", type=int, default=64, help="tokens per step of the gptj_b64 workload")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
     ap.add_argument("--static-projection", action="store_true",
-                    help="negative control (Section 4.1, static projection): the gate is computed and "
+                    help="negative control (remark after Theorem 3.1, Section 3.3, and Section 6.7 \"Negative control\"): the gate is computed and "
                          "logged but W r is never added, so the step costs the fast path only")
     ap.add_argument("--per-stage", action="store_true",
                     help="force the per-stage / batched kernels (stack mode 1) instead of the "

@@ -100,7 +100,7 @@ typedef struct {
 const char* gsi_status_string(gsi_status_t s);
 
 /*
- * Cached image of Eq. (3.2) / Section 4.2 ("computed once per weight matrix"):
+ * Cached image of Eq. (3.2) / Section 4.2 (built once per weight matrix, off the per-token path):
  *   W_P[a][j] = bf16_rne( sum_i W[a][i] * P[i][j] ),  fp32 accumulation.
  * W [o][d] bf16, P [d][k] of p_dtype, W_P_out [o][k] bf16; all device.
  * Enqueued on `stream`; no host synchronisation.
@@ -192,7 +192,7 @@ gsi_status_t gsi_forward_static(const void* const* W_host_array, const int* d_ou
 
 /*
  * Online extension of the basis by one vector (the paper's "time-dimension
- * tracking", Section 5.3, and "online basis adaptation", Section 7.3): the token
+ * tracking", Section 5.4, and "online basis adaptation", Section 7.2): the token
  * x [d] (fp32, device) is tested against the basis in use; if
  *     rho = ||x - P P^T x|| / ||x||  >  tau
  * and a column is free, the residual orthogonalised against P twice

@@ -244,7 +244,7 @@ int gsi_oracle_map(const double* M, const uint16_t* W, const double* g,
 
 /*
  * Online extension of the basis by one vector (the paper's "time-dimension
- * tracking" of Section 5.3 and "online basis adaptation" of Section 7.3):
+ * tracking" of Section 5.4 and "online basis adaptation" of Section 7.2):
  * a token x is tested against the current basis, and if
  *     rho = ||x - V V^T x|| / ||x||
  * exceeds the threshold tau the basis is extended by one orthonormal vector.

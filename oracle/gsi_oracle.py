@@ -144,7 +144,7 @@ def project(x, P, eps: float) -> dict:
 
 
 def extend(P, k_act: int, x, tau: float) -> dict:
-    """Online basis extension by one vector (Sections 5.3 and 7.3): rho of the token
+    """Online basis extension by one vector (Sections 5.4 and 7.2): rho of the token
     against columns [0, k_act) of the stored basis P [d][k_cap]; if rho > tau (and a
     column is free) the unit vector v = twice-orthogonalised residual, in fp64.
     ``v_bits`` is v rounded to bf16 (round to nearest even), the value a bf16 basis

@@ -1,5 +1,5 @@
 // Online extension of the basis by one vector (the paper's "time-dimension tracking",
-// Section 5.3, and "online basis adaptation", Section 7.3): a token is tested against
+// Section 5.4, and "online basis adaptation", Section 7.2): a token is tested against
 // the basis in use; if rho = ||x - P P^T x|| / ||x|| exceeds a threshold, the residual,
 // orthogonalised against P twice (Gram-Schmidt with one re-orthogonalisation, "DGKS") and
 // normalised, becomes column k_active of P, and W times that column (Section 4.2) becomes

@@ -765,7 +765,7 @@ def test_step_on_another_stream_right_after_bind():
                       stack.gate_log[7, 0].cpu().numpy(), stack.rho_log[7, 0].cpu().numpy())
 
 
-# ---- online basis extension (Sections 5.3 and 7.3) ----------------------------------
+# ---- online basis extension (Sections 5.4 and 7.2) ----------------------------------
 def _extend_case(d, k_act, k_cap, d_out, seed, p_dtype="bf16"):
     q = S.gen_basis(d, k_act, seed)                       # fp64 orthonormal [d][k_act]
     P = torch.zeros((d, k_cap), dtype=torch.float64)

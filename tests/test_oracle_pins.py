@@ -371,7 +371,7 @@ def test_P10_effective_parameters_and_storage_examples():
     assert abs(R.basis_storage_bytes(28, 4096, 256) / 1e6 - 59) < 0.5
 
 
-# ---- online basis extension (Sections 5.3 and 7.3) ----------------------------------
+# ---- online basis extension (Sections 5.4 and 7.2) ----------------------------------
 def _partial_basis(d, k_act, k_cap, seed, dtype=np.float32):
     rng = np.random.default_rng(seed)
     q, _ = np.linalg.qr(rng.standard_normal((d, k_act)))
