@@ -134,10 +134,8 @@ struct gsi_stack {
   int* dev_phase_first;     // device: first group of every phase of the persistent schedule
   int n_phases;
   std::vector<int> host_phase_first;
-  char* dev_tmaps;          // device: GSI_MAX_MAPS tensor maps per group (the persistent kernel's W stream)
   unsigned spin_limit;      // polls a cross-CTA wait of the persistent kernel may take
   std::vector<PersistGroup> host_groups;
-  std::vector<char> host_tmaps;
   std::vector<const float*> host_pmax_ptrs;
   int* epoch;               // device
   int* status;              // device
@@ -420,7 +418,7 @@ size_t gsi_stack_workspace_bytes(int n_groups) {
   if (n_groups <= 0) return 0;
   static_assert(sizeof(PersistGroup) <= 512, "group descriptor outgrew its slot");
   return align_up(256) + align_up((size_t)n_groups * 512) + align_up((size_t)n_groups * 8) +
-         align_up((size_t)n_groups * GSI_MAX_MAPS * kPersistTmapBytes) + align_up((size_t)n_groups * 4);
+         align_up((size_t)n_groups * 4);
 }
 
 gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* workspace,
@@ -450,9 +448,8 @@ gsi_status_t gsi_stack_create(int n_groups, const gsi_handle_t* groups, void* wo
   s->epoch = s->step + 1;
   s->status = s->step + 2;
   s->dev_groups = reinterpret_cast<PersistGroup*>(static_cast<char*>(workspace) + 256);
-  s->dev_tmaps = static_cast<char*>(workspace) + align_up(256) + align_up((size_t)n_groups * 512) +
-                 align_up((size_t)n_groups * 8);
-  s->dev_phase_first = reinterpret_cast<int*>(s->dev_tmaps + align_up((size_t)n_groups * GSI_MAX_MAPS * kPersistTmapBytes));
+  s->dev_phase_first = reinterpret_cast<int*>(static_cast<char*>(workspace) + align_up(256) +
+                                              align_up((size_t)n_groups * 512) + align_up((size_t)n_groups * 8));
   s->spin_limit = kPersistSpinLimitDefault;
   s->mode = 0;
   s->trace = nullptr;
@@ -482,23 +479,16 @@ static bool rows_fit(const gsi_layer* h, int ctas) {
   return (pg + gc - 1) / gc <= 10 && (og + gc - 1) / gc <= 10;
 }
 
-// W stream geometry of one map: rows per CTA, and rows per box (even, at most 30, chosen so
-// that the boxes of a CTA overshoot its rows as little as possible).
-static void w_geometry(int d_out, int grid, int* rows, int* rb) {
-  *rows = (d_out + grid - 1) / grid;
-  const int nblk = (*rows + kPersistBoxRowsMax - 1) / kPersistBoxRowsMax;
-  *rb = 2 * ((*rows + 2 * nblk - 1) / (2 * nblk));
-}
+// W stream geometry of a group: whole rows per contiguous piece of at most 32 KB.
+static int w_piece_rows(int d) { return std::max(1, kPersistPieceBytes / (d * 2)); }
 
-// The per-row accumulators of the W stream hold every box row of every map of a group.
+// A row of W fits a piece, and the per-warp partial results of the W stream hold every row a
+// CTA owns of every map of a group.
 static bool w_rows_fit(const gsi_layer* h, int grid) {
+  if (h->desc.d > kPersistMaxD) return false;
   int total = 0;
-  for (int j = 0; j < h->desc.n_maps; ++j) {
-    int rows, rb;
-    w_geometry(h->d_out[j], grid, &rows, &rb);
-    total += (rows + rb - 1) / rb * rb;
-  }
-  return total <= kPersistMaxORows;
+  for (int j = 0; j < h->desc.n_maps; ++j) total += (h->d_out[j] + grid - 1) / grid;
+  return total <= kPersistMaxWRows;
 }
 
 // Can this stack run on the persistent kernel?  (one or two tokens per step, bf16 basis
@@ -594,7 +584,6 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
         return GSI_ERR_CUDA;
     }
     s->host_groups.assign(G, PersistGroup{});
-    s->host_tmaps.assign((size_t)G * GSI_MAX_MAPS * kPersistTmapBytes, 0);
     s->host_pmax_ptrs.assign(G, nullptr);
     for (int i = 0; i < G; ++i) {
       const gsi_layer* h = s->groups[i];
@@ -602,16 +591,11 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
       const GroupParams& gp = h->gp;
       pg.P = reinterpret_cast<const uint16_t*>(h->ws + h->lay.pk_pp);
       pg.WP = reinterpret_cast<const uint16_t*>(h->ws + h->lay.pk_wpp);
-      pg.tmW = s->dev_tmaps + (size_t)i * GSI_MAX_MAPS * kPersistTmapBytes;
       for (int j = 0; j < gp.n_maps; ++j) {
-        int rows, rb;
-        w_geometry(gp.d_out[j], s->grid, &rows, &rb);
-        pg.w_rows[j] = (short)rows;
-        pg.w_rb[j] = (short)rb;
-        if (!encode_w_stream_map(s->host_tmaps.data() + ((size_t)i * GSI_MAX_MAPS + j) * kPersistTmapBytes,
-                                 gp.W[j], (size_t)gp.d_out[j], (size_t)gp.d, (unsigned)rb))
-          return GSI_ERR_CUDA;
+        pg.W[j] = gp.W[j];
+        pg.w_rows[j] = (short)((gp.d_out[j] + s->grid - 1) / s->grid);
       }
+      pg.w_pr = w_piece_rows(gp.d);
       for (int j = 0; j <= gp.n_maps; ++j) pg.off[j] = gp.off[j];
       pg.n_maps = gp.n_maps;
       pg.d = gp.d;
@@ -677,8 +661,6 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
     if (cudaMemcpyAsync(s->dev_groups, s->host_groups.data(), sizeof(PersistGroup) * G,
                         cudaMemcpyHostToDevice, stream) != cudaSuccess ||
         cudaMemcpyAsync(dev_ptrs, s->host_pmax_ptrs.data(), sizeof(float*) * G,
-                        cudaMemcpyHostToDevice, stream) != cudaSuccess ||
-        cudaMemcpyAsync(s->dev_tmaps, s->host_tmaps.data(), s->host_tmaps.size(),
                         cudaMemcpyHostToDevice, stream) != cudaSuccess ||
         cudaMemcpyAsync(s->dev_phase_first, s->host_phase_first.data(),
                         s->host_phase_first.size() * sizeof(int), cudaMemcpyHostToDevice, stream) != cudaSuccess ||

@@ -11,9 +11,9 @@ constexpr int kPersistMaxORows = 512;   // output rows one CTA may own
 constexpr int kPersistMaxGrid = 160;    // CTAs (tagged words per group)
 constexpr int kPersistMaxTokens = 2;    // tokens per step served by one launch per token (more: batched kernels)
 constexpr int kPersistMaxTicks = 160;   // phases of one launch + 2 (the per-CTA plan of a launch lives in shared memory)
-constexpr int kPersistBoxCols = 256;    // columns of W in one streamed box
-constexpr int kPersistBoxRowsMax = 30;  // rows of W in one streamed box: two per consumer warp
-constexpr int kPersistTmapBytes = 128;  // one tensor map
+constexpr int kPersistPieceBytes = 32768;   // largest contiguous piece of the W stream
+constexpr int kPersistMaxD = 16384;     // widest input: a row of W fits one piece, a lane's share of r fits its registers
+constexpr int kPersistMaxWRows = 256;   // rows of W (all maps of a group) one CTA may own
 
 struct PersistGroup {
   // Basis [d][k] and concatenated images [O][k], bf16, as 16 x 16 tiles: tile (R, K) at
@@ -22,7 +22,7 @@ struct PersistGroup {
   // Rows past d (O) are zero.
   const uint16_t* P;
   const uint16_t* WP;
-  const void* tmW;                   // n_maps tensor maps (device memory): W_j [d_out_j][d] bf16 in boxes of w_rb[j] rows x 256 columns
+  const uint16_t* W[GSI_MAX_MAPS];   // [d_out_j][d] bf16
   const float* x;                    // [n_steps][tokens][d]
   float* y;                          // [tokens][O]
   float* r;                          // [d]
@@ -51,9 +51,10 @@ struct PersistGroup {
   int phase_len;                     // groups in this group's phase: 1, or 2 for both of a pair
   int next_len;                      // groups in the phase after this group's (0 at the end)
   // W stream (gated residual, dense baseline): every CTA owns w_rows[j] consecutive rows of
-  // every map j, streamed as boxes of w_rb[j] rows (even, at most 30) x 256 columns.
+  // every map j (one contiguous run of memory), copied as contiguous pieces of w_pr whole rows
+  // (at most 32 KB).
   short w_rows[GSI_MAX_MAPS];
-  short w_rb[GSI_MAX_MAPS];
+  int w_pr;
 };
 
 struct PersistParams {
@@ -88,8 +89,5 @@ cudaError_t launch_abs_max_bf16(const void* p, size_t n, float* out, cudaStream_
 cudaError_t launch_pack_t16(const void* src, int rows, int k, void* dst, cudaStream_t st);
 cudaError_t launch_patch_pmax(PersistGroup* groups, const float* const* pmax_ptrs, int n,
                               cudaStream_t st);
-// Tensor map of one weight matrix for the persistent kernel's W stream: W [rows][cols] bf16
-// row-major, boxes of box_rows x 256 columns, no swizzle.  out: 128 bytes on the HOST.
-bool encode_w_stream_map(void* out, const void* W, size_t rows, size_t cols, unsigned box_rows);
 
 }  // namespace gsi

@@ -57,10 +57,9 @@ namespace {
 constexpr int kNW = kPersistConsumerWarps;
 constexpr int kNC = kNW * 32;               // consumer threads
 constexpr int kThreadsP = kNC + 32;         // + producer warp
-constexpr int kNB = 32;                     // chunks in flight at most (one barrier pair each)
+constexpr int kNB = 64;                     // chunks in flight at most (one barrier pair each)
 constexpr int kChunk = 16384;               // largest chunk
-constexpr int kSlice = 4096;                // columns of W per staged slice of r
-constexpr int kBoxCols = kPersistBoxCols;
+constexpr int kWVecMax = 5;                 // 16-byte vectors of a row one lane may own in the W stream (d <= 16384)
 constexpr unsigned kLocalSpinLimit = 1u << 20;   // waits inside the CTA (ring, producer hand-off)
 constexpr int kCountShift = 54;
 constexpr unsigned long long kOne = 1ull << kCountShift;
@@ -95,28 +94,25 @@ __device__ __forceinline__ void deal(int n, int parts, int i, int& a, int& b) {
 
 // shared memory map (bytes)
 constexpr int kOffBar = 0;          // full[kNB], empty[kNB]
-constexpr int kOffLin = 512;        // producer: ring position (bytes placed before it) of every chunk in flight (kNB words)
-constexpr int kOffOff = 640;        // offset of every chunk in flight within the ring (kNB words), for the consumers
-constexpr int kOffProd = 1152;      // state of the producer thread (16 bytes)
-constexpr int kOffMisc = 768;       // scalars
-constexpr int kOffTrace = 1024;     // cycle counters of the trace (16 words)
-constexpr int kOffX = 1280;         // x of this CTA's basis rows, two buffers (kPersistMaxPRows floats each)
+constexpr int kOffLin = 1024;       // producer: ring position (bytes placed before it) of every chunk in flight (kNB words)
+constexpr int kOffOff = 1280;       // offset of every chunk in flight within the ring (kNB words), for the consumers
+constexpr int kOffMisc = 1536;      // scalars
+constexpr int kOffTrace = 1792;     // cycle counters of the trace (16 words)
+constexpr int kOffProd = 1920;      // state of the producer thread (16 bytes)
+constexpr int kOffX = 2048;         // x of this CTA's basis rows, two buffers (kPersistMaxPRows floats each)
 constexpr int kOffXt = kOffX + 2 * kPersistMaxPRows * 4;  // ... as three bf16 terms in A-operand order, two buffers (16 tile rows x 256 B each)
 constexpr int kOffCb = kOffXt + 2 * 4096;                 // c as three bf16 terms in B-operand order (32 tile columns x 256 B)
 constexpr int kOffFx = kOffCb + 8192;                     // fixed-point partial c and ||x||^2, source of the bulk reduction (514 words)
 constexpr int kOffPlan = kOffFx + 4224;                   // the launch's plan (kPersistMaxTicks records)
 constexpr int kOffDesc = kOffPlan + kPersistMaxTicks * 32;   // 8 group descriptors, 256 B each
 constexpr int kDescSlots = 8;
-constexpr int kOffRs = kOffDesc + kDescSlots * 256;       // W stream: staged slice of r (16 KB)
-constexpr int kOffYacc = kOffRs + kSlice * 4;             // per-row accumulators (kPersistMaxORows floats)
-constexpr int kOffRing = ((kOffYacc + kPersistMaxORows * 4 + 1023) / 1024) * 1024;
+constexpr int kOffYacc = kOffDesc + kDescSlots * 512;     // W stream: per-warp partial results (kNW x kPersistMaxWRows floats)
+constexpr int kOffRing = ((kOffYacc + kNW * kPersistMaxWRows * 4 + 1023) / 1024) * 1024;
 constexpr int kRingBytes = (232448 - kOffRing) / 1024 * 1024;
 constexpr int kSmemBytes = kOffRing + kRingBytes;
 static_assert(kSmemBytes <= 232448, "shared memory budget of one sm_100 CTA");
-static_assert(kOffXt % 16 == 0 && kOffCb % 16 == 0 && kOffFx % 16 == 0 && kOffPlan % 16 == 0 && kOffDesc % 16 == 0 && kOffRs % 16 == 0, "alignment");
-static_assert(sizeof(PersistGroup) <= 256 && sizeof(PersistGroup) % 4 == 0, "descriptor slot");
-static_assert(kPersistBoxRowsMax * kBoxCols * 2 <= kChunk, "a box fits a chunk");
-static_assert(kPersistBoxRowsMax == 2 * kNW, "two rows of a box per consumer warp");
+static_assert(kOffXt % 16 == 0 && kOffCb % 16 == 0 && kOffFx % 16 == 0 && kOffPlan % 16 == 0 && kOffDesc % 16 == 0, "alignment");
+static_assert(sizeof(PersistGroup) <= 512 && sizeof(PersistGroup) % 4 == 0, "descriptor slot");
 constexpr int kDescWords = (int)(sizeof(PersistGroup) / 4);
 
 struct Misc {
@@ -144,6 +140,9 @@ __device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
 __device__ __forceinline__ void mbar_arrive(uint64_t* b) {
   asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(b)) : "memory");
 }
+__device__ __forceinline__ void mbar_arrive_n(uint64_t* b, uint32_t count) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(b)), "r"(count) : "memory");
+}
 __device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
   uint32_t ok;
   asm volatile(
@@ -167,14 +166,6 @@ __device__ __forceinline__ void bulk_g2s(void* dst, const void* src, uint32_t by
       "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(
           smem_u32(dst)),
       "l"(src), "r"(bytes), "r"(smem_u32(bar))
-      : "memory");
-}
-// One box of a 2-D tensor map (no multicast): x = first column, y = first row.
-__device__ __forceinline__ void tma_box_g2s(void* dst, const void* tmap, int x, int y, uint64_t* bar) {
-  asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];" ::"r"(
-          smem_u32(dst)),
-      "l"(tmap), "r"(x), "r"(y), "r"(smem_u32(bar))
       : "memory");
 }
 // Element-wise atomic add of `bytes` / 8 64-bit words from shared to global memory by the bulk
@@ -300,9 +291,9 @@ __device__ __noinline__ unsigned producer_acquire(unsigned char* smem, unsigned 
   return off;
 }
 
-// The W boxes of one group for this CTA, in the order the consumers take them: column
-// slices of 4096 outermost (one staged slice of r serves them), then maps, then row blocks,
-// then the 256-column boxes of the slice.
+// The W stream of one group for this CTA: its w_rows[j] consecutive rows of every map j are
+// one contiguous run of memory, copied as contiguous pieces of w_pr whole rows (at most 32 KB:
+// large contiguous copies are what reaches the memory system's bandwidth).
 __device__ __forceinline__ bool produce_w(const PersistGroup& g, unsigned char* smem) {
   Producer& prs = *reinterpret_cast<Producer*>(smem + kOffProd);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + kOffBar);
@@ -311,47 +302,41 @@ __device__ __forceinline__ bool produce_w(const PersistGroup& g, unsigned char* 
   unsigned* s_off = reinterpret_cast<unsigned*>(smem + kOffOff);
   unsigned char* base = smem + kOffRing;
   volatile int* abort = &reinterpret_cast<Misc*>(smem + kOffMisc)->abort;
-  // the ring state in registers for the length of the stream (thousands of boxes, one every
+  // the ring state in registers for the length of the stream (thousands of pieces, one every
   // few hundred cycles: the out-of-line acquire with its state in shared memory is too slow)
   unsigned n = prs.n, lin = prs.lin, tail_n = prs.tail_n, tail_lin = prs.tail_lin;
   bool ok = true;
   const int cta = blockIdx.x;
-  const int nsl = (g.d + kSlice - 1) / kSlice;
-  for (int sl = 0; sl < nsl && ok; ++sl) {
-    const int c0 = sl * kSlice, ncb = (min(kSlice, g.d - c0) + kBoxCols - 1) / kBoxCols;
-    for (int j = 0; j < g.n_maps && ok; ++j) {
-      const int dout = g.off[j + 1] - g.off[j], rows = g.w_rows[j], rb = g.w_rb[j];
-      const int row0 = cta * rows;
-      const int live = min(rows, dout - row0);
-      const char* tm = static_cast<const char*>(g.tmW) + (size_t)j * kPersistTmapBytes;
-      const uint32_t bytes = (uint32_t)rb * kBoxCols * 2;
-      for (int b = 0; b * rb < live && ok; ++b) {
-        for (int cb = 0; cb < ncb; ++cb) {
-          unsigned off = lin % (unsigned)kRingBytes;
-          if (off + bytes > (unsigned)kRingBytes) {
-            lin += (unsigned)kRingBytes - off;
-            off = 0;
-          }
-          const unsigned start = lin;
-          lin += bytes;
-          while (n - tail_n >= (unsigned)kNB || (tail_n < n && lin - tail_lin > (unsigned)kRingBytes)) {
-            if (!mbar_wait(&empty[tail_n % kNB], (tail_n / kNB) & 1u, abort)) {
-              ok = false;
-              break;
-            }
-            ++tail_n;
-            tail_lin = tail_n < n ? s_lin[tail_n % kNB] : start;
-          }
-          if (!ok) break;
-          if (tail_n == n) tail_lin = start;
-          s_lin[n % kNB] = start;
-          s_off[n % kNB] = off;
-          uint64_t* fb = &full[n % kNB];
-          mbar_expect_tx(fb, bytes);
-          tma_box_g2s(base + off, tm, c0 + cb * kBoxCols, row0 + b * rb, fb);
-          ++n;
-        }
+  const int d = g.d, pr = g.w_pr;
+  for (int j = 0; j < g.n_maps && ok; ++j) {
+    const int dout = g.off[j + 1] - g.off[j], rows = g.w_rows[j];
+    const int row0 = cta * rows;
+    const int live = min(rows, dout - row0);
+    for (int r0 = 0; r0 < live; r0 += pr) {
+      const uint32_t bytes = (uint32_t)min(pr, live - r0) * d * 2;
+      unsigned off = lin % (unsigned)kRingBytes;
+      if (off + bytes > (unsigned)kRingBytes) {
+        lin += (unsigned)kRingBytes - off;
+        off = 0;
       }
+      const unsigned start = lin;
+      lin += bytes;
+      while (n - tail_n >= (unsigned)kNB || (tail_n < n && lin - tail_lin > (unsigned)kRingBytes)) {
+        if (!mbar_wait(&empty[tail_n % kNB], (tail_n / kNB) & 1u, abort)) {
+          ok = false;
+          break;
+        }
+        ++tail_n;
+        tail_lin = tail_n < n ? s_lin[tail_n % kNB] : start;
+      }
+      if (!ok) break;
+      if (tail_n == n) tail_lin = start;
+      s_lin[n % kNB] = start;
+      s_off[n % kNB] = off;
+      uint64_t* fb = &full[n % kNB];
+      mbar_expect_tx(fb, bytes);
+      bulk_g2s(base + off, g.W[j] + (size_t)(row0 + r0) * d, bytes, fb);
+      ++n;
     }
   }
   prs.n = n;
@@ -390,15 +375,18 @@ __device__ void producer(const PersistParams& p, unsigned char* smem, Misc* misc
   volatile int* abort = &misc->abort;
   bool ok = true;
   // ticks: tick t runs phase t (while there is one) and the gated residuals of phase t - 2;
-  // the work of a tick, in ring order: basis slab, W boxes of the gated groups, image slab
-  // (or the W boxes of a dense group)
+  // the work of a tick, in ring order: basis slab, image slab, W pieces of the gated groups
+  // (or the W pieces of a dense group)
   const Plan* plan = reinterpret_cast<const Plan*>(smem + kOffPlan);
   const int n_ticks = p.n_phases + 2;
 #pragma unroll 1
   for (int t = 0; t < n_ticks && ok; ++t) {
     const Plan& pl = plan[t];
     const PersistGroup* g = p.groups + pl.gi;   // read only when the tick has a group
-    if (pl.kind == 1) ok = produce_rows(g->P, g->k, pl.p0 >> 4, (pl.p0 >> 4) + pl.pg, smem);
+    if (pl.kind == 1) {
+      ok = produce_rows(g->P, g->k, pl.p0 >> 4, (pl.p0 >> 4) + pl.pg, smem);
+      if (ok) ok = produce_rows(g->WP, g->k, pl.o0 >> 4, (pl.o0 >> 4) + pl.og, smem);
+    }
     unsigned wmask = 0;
     const int len_pp = t >= 2 ? plan[t - 2].len : 0, g_pp = t >= 2 ? plan[t - 2].gi0 : 0;
     if (ok && len_pp > 0) {
@@ -428,7 +416,6 @@ __device__ void producer(const PersistParams& p, unsigned char* smem, Misc* misc
         if (gw) ok = produce_w(*gw, smem);
       }
     }
-    if (ok && pl.kind == 1) ok = produce_rows(g->WP, g->k, pl.o0 >> 4, (pl.o0 >> 4) + pl.og, smem);
   }
   if (!ok && !*abort) fail(p, misc, 1);
   // Every copy issued must have landed before the CTA may give up its shared
@@ -532,105 +519,176 @@ __device__ __forceinline__ bool chunks_landed(unsigned char* smem, unsigned n0, 
   return __all_sync(0xffffffffu, mine_ok);
 }
 
+// One piece of the W stream for one warp: rows_p rows of rvec vectors; this lane owns vectors
+// lane + 32 i (i < VPL) of the warp's range (first = pointer to its first vector of row 0,
+// nvalid = how many of its VPL vectors exist); `in` holds its share of the input.  RPI rows at
+// a time (2 or 1: more rows in flight cost registers that the tick loop around the stream
+// needs); two rows share five shuffles (the first level sends half of the values to the
+// partner).  Results to part[row].
+// The piece goes back to the producer (release_n arrivals on `eb`) as soon as its last rows
+// are in registers, before the sums over the lanes: the arrival is predicated on a value that
+// every load of the warp feeds (a comparison that never fails), so it cannot be issued before
+// those loads have returned.
+template <int VPL, int RPI>
+__device__ __forceinline__ void w_piece(const uint4* first, int rvec, int rows_p, int nvalid,
+                                        const unsigned long long (&in)[kWVecMax][4], float* part,
+                                        uint64_t* eb, uint32_t release_n) {
+  const int lane = threadIdx.x & 31;
+  constexpr unsigned kNever = 0x7fc5a5a5u;   // a NaN pattern no arithmetic instruction produces
+#pragma unroll 1
+  for (int ra = 0; ra < rows_p; ra += RPI) {
+    unsigned long long a[RPI], b[RPI];   // two chains of dependent additions per row
+#pragma unroll
+    for (int q = 0; q < RPI; ++q) a[q] = b[q] = 0ull;
+    uint4 w[VPL][RPI];
+#pragma unroll
+    for (int i = 0; i < VPL; ++i)
+#pragma unroll
+      for (int q = 0; q < RPI; ++q) {
+        // rows past the piece read the last row again (dropped below); vectors past the row's
+        // end are not read at all
+        w[i][q] = make_uint4(0u, 0u, 0u, 0u);
+        if (i < nvalid) w[i][q] = first[(size_t)min(ra + q, rows_p - 1) * rvec + 32 * i];
+      }
+#pragma unroll
+    for (int i = 0; i < VPL; ++i)
+#pragma unroll
+      for (int q = 0; q < RPI; ++q) {
+        fma2(a[q], bf16x2_to_f32x2(w[i][q].x), in[i][0]);
+        fma2(b[q], bf16x2_to_f32x2(w[i][q].y), in[i][1]);
+        fma2(a[q], bf16x2_to_f32x2(w[i][q].z), in[i][2]);
+        fma2(b[q], bf16x2_to_f32x2(w[i][q].w), in[i][3]);
+      }
+    float v[RPI];
+#pragma unroll
+    for (int q = 0; q < RPI; ++q) v[q] = sum2(a[q]) + sum2(b[q]);
+    const bool last = ra + RPI >= rows_p;
+    float v0 = v[0];
+    int q_mine = 0, keep = 31;   // the row this lane ends up with, and which lanes write (lane & keep == 0)
+    if constexpr (RPI == 2) {
+      const bool up = lane & 16;
+      const float s0 = up ? v[0] : v[1];
+      const float r0v = __shfl_xor_sync(0xffffffffu, s0, 16);
+      v0 = (up ? v[1] : v[0]) + r0v;
+      q_mine = lane >> 4;
+      keep = 15;
+    }
+    // v0 now depends on every row loaded above
+    if (last) {
+      __syncwarp();
+      if (lane == 0 && __float_as_uint(v0) != kNever) mbar_arrive_n(eb, release_n);
+    }
+    if constexpr (RPI == 1) v0 += __shfl_xor_sync(0xffffffffu, v0, 16);
+    v0 += __shfl_xor_sync(0xffffffffu, v0, 8);
+    v0 += __shfl_xor_sync(0xffffffffu, v0, 4);
+    v0 += __shfl_xor_sync(0xffffffffu, v0, 2);
+    v0 += __shfl_xor_sync(0xffffffffu, v0, 1);
+    if ((lane & keep) == 0 && ra + q_mine < rows_p) part[ra + q_mine] = v0;
+  }
+}
+
 // ---- W stream: y_rows (+)= W_rows . src (src = r of a gated group, or x for the dense
-// baseline), boxes taken from the ring in the producer's order.  `n` is the consumers' chunk
-// sequence number.  Returns false when a wait gave up.
-__device__ __forceinline__ bool w_stream(const PersistParams& p, const PersistGroup& g, const float* src,
-                                         float* y, bool dense, unsigned char* smem, unsigned& n,
-                                         Misc* misc) {
+// baseline), pieces of whole rows taken from the ring in the producer's order.  The consumer
+// warps form teams of nw warps; a team takes every T-th piece, so T pieces are worked on at
+// once and the latency of one piece (wait, loads, sums over the lanes) is hidden by the
+// others.  Within a team every warp owns a range of columns and keeps its share of src in
+// registers for the whole stream (four or five 16-byte vectors of W per lane and row; no
+// staging in shared memory).  The partial sums of a row meet in shared memory and are added
+// in warp order at the end (reproducible).  `n` is the consumers' chunk sequence number on
+// entry, the return value the one after the stream; a wait that gave up sets the abort flag.
+// Inlined at its two call sites (an out-of-line call makes the tick loop keep its state in
+// local memory); both sit where little of the tick's state is alive.
+__device__ __forceinline__ unsigned w_stream(const PersistGroup* gp, const float* src, float* y, bool dense,
+                                          unsigned char* smem, unsigned n, int* status, bool traced) {
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + kOffBar);
   uint64_t* empty = full + kNB;
   const unsigned* s_off = reinterpret_cast<const unsigned*>(smem + kOffOff);
   unsigned char* ring = smem + kOffRing;
-  float* s_rs = reinterpret_cast<float*>(smem + kOffRs);
-  float* s_yacc = reinterpret_cast<float*>(smem + kOffYacc);
+  float* s_part = reinterpret_cast<float*>(smem + kOffYacc);
+  Misc* misc = reinterpret_cast<Misc*>(smem + kOffMisc);
   volatile int* abort = &misc->abort;
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int cta = blockIdx.x;
-  const int nsl = (g.d + kSlice - 1) / kSlice;
+  Trace tr;
+  tr.acc = (traced && tid == 0) ? reinterpret_cast<unsigned long long*>(smem + kOffTrace) : nullptr;
+  tr.t = clock64();
+  const int d = gp->d, pr = gp->w_pr, n_maps = gp->n_maps;
+  const int rvec = d >> 3;                                   // 16-byte vectors per row
+  const int vpl = rvec > 4 * kNC ? 5 : 4;
+  const int nw = (rvec + 32 * vpl - 1) / (32 * vpl);         // warps of a team
+  const int T = kNW / nw;                                    // teams
+  const int team = warp / nw, wi = warp - team * nw;
+  const bool active = team < T;
+  const int v_lo = min(rvec, wi * 32 * vpl), v_hi = min(rvec, v_lo + 32 * vpl);   // this warp's vectors of every row
+  const int nvalid = (v_hi - v_lo - lane + 31) >> 5;         // how many of this lane's vectors exist
+  const uint32_t release_n = wi == 0 ? (uint32_t)(kNW - nw + 1) : 1u;   // a team's first warp also arrives for all other warps
   bool ok = true;
-#pragma unroll 1
-  for (int sl = 0; sl < nsl; ++sl) {
-    const int c0 = sl * kSlice, cols = min(kSlice, g.d - c0);
-    const int ncb = (cols + kBoxCols - 1) / kBoxCols;
-    csync();
-    // Stage the slice so that a lane's two 16-byte loads per box are conflict-free: within a
-    // 256-column block, the first halves of the 32 lanes' eight columns, then the second halves.
-#pragma unroll 1
-    for (int i = tid; i < ncb * 64; i += kNC) {
-      const int col = i * 4;
-      const float4 v = col < cols ? __ldcg(reinterpret_cast<const float4*>(src + c0 + col))
-                                  : make_float4(0.f, 0.f, 0.f, 0.f);
-      const int blk = i >> 6, w4 = i & 63;
-      reinterpret_cast<float4*>(s_rs)[blk * 64 + (w4 & 1) * 32 + (w4 >> 1)] = v;
+  // this lane's share of the input: vectors v_lo + lane + 32 i
+  unsigned long long in[kWVecMax][4];
+#pragma unroll
+  for (int i = 0; i < kWVecMax; ++i) {
+    const int v = v_lo + lane + 32 * i;
+    float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
+    if (active && v < v_hi) {
+      a = __ldcg(reinterpret_cast<const float4*>(src) + 2 * v);
+      b = __ldcg(reinterpret_cast<const float4*>(src) + 2 * v + 1);
     }
-    csync();
-    int ybase = 0;
-#pragma unroll 1
-    for (int j = 0; j < g.n_maps; ++j) {
-      const int dout = g.off[j + 1] - g.off[j], rows = g.w_rows[j], rb = g.w_rb[j];
-      const int live = min(rows, dout - cta * rows);
-      const bool mine = 2 * warp < rb;
-#pragma unroll 1
-      for (int b = 0; b * rb < live; ++b) {
-        unsigned long long a0 = 0ull, a1 = 0ull;
-#pragma unroll 1
-        for (int cb = 0; cb < ncb; ++cb) {
-          const unsigned slot = n % kNB, ph = (n / kNB) & 1u;
-          ++n;
-          if (ok && !mbar_wait(&full[slot], ph, abort)) ok = false;
-          if (ok && mine) {
-            const uint4* tile = reinterpret_cast<const uint4*>(ring + s_off[slot]);
-            const uint4 w0 = tile[(2 * warp) * (kBoxCols / 8) + lane];
-            const uint4 w1 = tile[(2 * warp + 1) * (kBoxCols / 8) + lane];
-            const float4 ra = reinterpret_cast<const float4*>(s_rs)[cb * 64 + lane];
-            const float4 rb4 = reinterpret_cast<const float4*>(s_rs)[cb * 64 + 32 + lane];
-            const unsigned long long r0 = pack2(ra.x, ra.y), r1 = pack2(ra.z, ra.w);
-            const unsigned long long r2 = pack2(rb4.x, rb4.y), r3 = pack2(rb4.z, rb4.w);
-            fma2(a0, bf16x2_to_f32x2(w0.x), r0);
-            fma2(a1, bf16x2_to_f32x2(w1.x), r0);
-            fma2(a0, bf16x2_to_f32x2(w0.y), r1);
-            fma2(a1, bf16x2_to_f32x2(w1.y), r1);
-            fma2(a0, bf16x2_to_f32x2(w0.z), r2);
-            fma2(a1, bf16x2_to_f32x2(w1.z), r2);
-            fma2(a0, bf16x2_to_f32x2(w0.w), r3);
-            fma2(a1, bf16x2_to_f32x2(w1.w), r3);
-          }
-          __syncwarp();
-          if (ok && lane == 0) mbar_arrive(&empty[slot]);
-        }
-        if (mine) {
-          const float t0 = warp_sum(sum2(a0)), t1 = warp_sum(sum2(a1));
-          if (lane == 0) {
-            const int i0 = ybase + b * rb + 2 * warp;
-            s_yacc[i0] = (sl == 0 ? 0.f : s_yacc[i0]) + t0;
-            s_yacc[i0 + 1] = (sl == 0 ? 0.f : s_yacc[i0 + 1]) + t1;
-          }
-        }
-      }
-      ybase += ((live > 0 ? (live + rb - 1) / rb : 0)) * rb;
-    }
+    in[i][0] = pack2(a.x, a.y);
+    in[i][1] = pack2(a.z, a.w);
+    in[i][2] = pack2(b.x, b.y);
+    in[i][3] = pack2(b.z, b.w);
   }
-  if (!ok && !*abort) fail(p, misc, 3);
-  csync();
-  // rows back to y: the same walk over the maps
-  {
-    int ybase = 0;
+  int ybase = 0, pi = 0;   // rows of the maps before this one; pieces of this stream so far
+  tr.mark(10);
 #pragma unroll 1
-    for (int j = 0; j < g.n_maps; ++j) {
-      const int dout = g.off[j + 1] - g.off[j], rows = g.w_rows[j], rb = g.w_rb[j];
+  for (int j = 0; j < n_maps; ++j) {
+    const int dout = gp->off[j + 1] - gp->off[j], rows = gp->w_rows[j];
+    const int live = min(rows, dout - cta * rows);
+#pragma unroll 1
+    for (int r0 = 0; r0 < live; r0 += pr, ++pi) {
+      const int rows_p = min(pr, live - r0);
+      const unsigned slot = n % kNB, ph = (n / kNB) & 1u;
+      ++n;
+      if (!active || pi % T != team) continue;
+      if (ok && !mbar_wait(&full[slot], ph, abort)) ok = false;
+      tr.mark(11);
+      if (ok) {
+        const uint4* piece = reinterpret_cast<const uint4*>(ring + s_off[slot]) + v_lo + lane;
+        float* part = s_part + wi * kPersistMaxWRows + ybase + r0;
+        uint64_t* eb = &empty[slot];
+        if (vpl == 5) w_piece<5, 1>(piece, rvec, rows_p, nvalid, in, part, eb, release_n);
+        else if (pr >= 2) w_piece<4, 2>(piece, rvec, rows_p, nvalid, in, part, eb, release_n);
+        else w_piece<4, 1>(piece, rvec, rows_p, nvalid, in, part, eb, release_n);
+      }
+      tr.mark(12);
+    }
+    ybase += max(live, 0);
+  }
+  if (!ok && !*abort) fail_at(status, misc, 3);
+  csync();
+  // rows back to y: the same walk over the maps; the warps' partial sums in warp order
+  {
+    int yb = 0;
+#pragma unroll 1
+    for (int j = 0; j < n_maps; ++j) {
+      const int dout = gp->off[j + 1] - gp->off[j], rows = gp->w_rows[j];
       const int live = min(rows, dout - cta * rows);
       if (ok) {
 #pragma unroll 1
         for (int i = tid; i < live; i += kNC) {
-          float* yp = y + g.off[j] + cta * rows + i;
-          *yp = dense ? s_yacc[ybase + i] : (__ldcg(yp) + s_yacc[ybase + i]);
+          float acc = 0.f;
+#pragma unroll 1
+          for (int q = 0; q < nw; ++q) acc += s_part[q * kPersistMaxWRows + yb + i];
+          float* yp = y + gp->off[j] + cta * rows + i;
+          *yp = dense ? acc : (__ldcg(yp) + acc);
         }
       }
-      ybase += ((live > 0 ? (live + rb - 1) / rb : 0)) * rb;
+      yb += max(live, 0);
     }
   }
-  return ok;
+  csync();   // the partial sums may be overwritten by the next stream
+  tr.mark(13);
+  return n;
 }
 
 // The statistics warp: the group's max |x| for tick `tt` from the tagged words of all
@@ -653,7 +711,7 @@ __device__ __noinline__ void xmax_collect(unsigned char* smem, int tt, unsigned 
   const Plan& pn = reinterpret_cast<const Plan*>(smem + kOffPlan)[tt];
   Misc* misc = reinterpret_cast<Misc*>(smem + kOffMisc);
   const PersistGroup& gn =
-      *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + (pn.gi & (kDescSlots - 1)) * 256);
+      *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + (pn.gi & (kDescSlots - 1)) * 512);
   const int lane = threadIdx.x & 31;
   unsigned w[kXmaxWords] = {w0, w1, w2, w3, w4};
   unsigned m = 0, it = 0;
@@ -689,7 +747,7 @@ __device__ __noinline__ void stat_warp_step(unsigned char* smem, int tt, bool re
   if (pn.kind != 1) return;
   const int lane = threadIdx.x & 31;
   const PersistGroup& gn =
-      *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + (pn.gi & (kDescSlots - 1)) * 256);
+      *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + (pn.gi & (kDescSlots - 1)) * 512);
   float* sx = reinterpret_cast<float*>(smem + kOffX) + (tt & 1) * kPersistMaxPRows;
   const int rows = pn.pg * 16;
   if (request) {
@@ -815,7 +873,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
   tr.start(p, smem);
 
   auto desc = [&](int i) -> const PersistGroup& {
-    return *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + (i & (kDescSlots - 1)) * 256);
+    return *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + (i & (kDescSlots - 1)) * 512);
   };
   // groups [g0, g0 + cnt) from the device table into their slots (threads 0 .. cnt*kDescWords-1)
   auto desc_load = [&](int g0, int cnt) -> uint32_t {
@@ -824,7 +882,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
   auto desc_store = [&](int g0, int cnt, uint32_t w) {
     if (tid < cnt * kDescWords) {
       const int j = tid / kDescWords;
-      reinterpret_cast<uint32_t*>(smem + kOffDesc + ((g0 + j) & (kDescSlots - 1)) * 256)[tid - j * kDescWords] = w;
+      reinterpret_cast<uint32_t*>(smem + kOffDesc + ((g0 + j) & (kDescSlots - 1)) * 512)[tid - j * kDescWords] = w;
     }
   };
   // the operand rows / columns beyond the three terms stay zero for the whole launch
@@ -869,6 +927,49 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     const int g_stage = t + 2 < p.n_phases ? plan[t + 2].gi0 : 0, n_stage = t + 2 < p.n_phases ? plan[t + 2].len : 0;
     const uint32_t desc_word = desc_load(g_stage, n_stage);
 
+    // ---- a dense group among dense groups (the dense baseline): nothing of the exchange
+    //      machinery has work in this tick.  Post the (empty) decision on the previous phase
+    //      for the producer and go straight to the stream at the end of the tick.  The next
+    //      dense group's input is asked into the L2 meanwhile (the inputs of a stack are
+    //      staged before the step).
+    const bool plain = dense && !contrib_p && !mask_pp && (t == 0 || plan[t - 1].kind == 2);
+    const unsigned mask_stream = mask_pp;   // the gated residuals this tick streams: phase t - 2
+    if (plain) {
+      if (pl.zeroer && tid < 2) g.bar[2 * tid + (parity ^ 1u)] = 0u;
+      if (tid == 0 && t >= 1) misc->decision[(t - 1) & 3] = (unsigned)t << 8;
+      desc_store(g_stage, n_stage, desc_word);
+      if (warp == kStatWarp && t + 1 < n_ticks) {
+        const Plan& pn = plan[t + 1];
+        if (pn.kind == 2) {
+          const PersistGroup& gn = desc(pn.gi);
+          const char* xn = reinterpret_cast<const char*>(gn.x + (long long)slot_io * gn.x_step_stride +
+                                                         (size_t)p.token * gn.d);
+          for (int i = lane * 128; i < gn.d * 4; i += 32 * 128)
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(xn + i));
+        } else if (pn.kind == 1) {   // a projected group follows: its statistics, as in every other tick
+          stat_warp_step(smem, t + 1, true, slot_io, p.token, tag);
+          stat_warp_step(smem, t + 1, false, slot_io, p.token, tag);
+          unsigned xw[kXmaxWords];
+          xmax_issue(desc(pn.gi).xmax, pn.n_contrib, xw);
+          xmax_collect(smem, t + 1, tag, p.spin_limit, p.status, xw[0], xw[1], xw[2], xw[3], xw[4]);
+        }
+      }
+      mask_pp = 0;
+      tr.mark(0);
+      n = w_stream(&g, g.x + (long long)slot_io * g.x_step_stride + (size_t)p.token * g.d,
+                   g.y + (size_t)p.token * g.O, true, smem, n, p.status, p.trace != nullptr);
+      if (tr.acc) tr.t = clock64();
+      if (*abort) return;
+      if (tid == 0) {
+        red_relaxed_u32(g.bar + parity, 1u);
+        grid_wait(g.bar + parity, (unsigned)G, p, misc);
+        if (cta == 0) p.gate_log[((size_t)slot_io * p.log_step_stride + pl.gi) * p.n_tokens + p.token] = 1;
+      }
+      csync();
+      tr.mark(6);
+      if (*abort) return;
+      continue;
+    } else {
     // ---- A. this CTA's rows of x have arrived and are in operand form (the statistics warp
     //      saw to it during the previous tick); the bulk reduction of the previous tick has
     //      read its source
@@ -1158,46 +1259,8 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     //      the tiles as they lie in the ring are the A operand, c (three terms in columns
     //      0..2) the B operand.  Units are dealt round-robin over the joint numbering of both
     //      parts, so the warps are loaded evenly.  Every warp gives every chunk back once.
-    // ---- H (between them). the W streams of the tick, one call site: the gated residuals
-    //      of the phase before the previous one, then this phase's own stream if it is a
-    //      dense group (followed by a grid barrier that keeps a dense stack in model order).
 #pragma unroll 1
     for (int part = 0; part < 2; ++part) {
-      if (part == 1 && (mask_pp || dense)) {
-        const int len_pp = plan[t - 2 >= 0 ? t - 2 : 0].len, g_pp = plan[t - 2 >= 0 ? t - 2 : 0].gi0;
-#pragma unroll 1
-        for (int u = 0; u < 3 && ok; ++u) {
-          const PersistGroup* gw = nullptr;
-          if (u < 2) {
-            if (u < len_pp && (mask_pp & (1u << u))) gw = p.groups + g_pp + u;
-          } else if (dense) {
-            gw = &g;
-          }
-          if (!gw) continue;
-          if (u < 2) {
-            if (tid == 0) {
-              grid_wait(gw->bar + 2 + parity, (unsigned)G, p, misc);
-              __threadfence();
-            }
-            csync();
-            if (*abort) return;
-          }
-          const float* src = u < 2 ? gw->r
-                                   : gw->x + (long long)slot_io * gw->x_step_stride + (size_t)p.token * gw->d;
-          ok = w_stream(p, *gw, src, gw->y + (size_t)p.token * gw->O, u == 2, smem, n, misc);
-          if (u == 2) {
-            if (tid == 0) {
-              red_relaxed_u32(gw->bar + parity, 1u);
-              grid_wait(gw->bar + parity, (unsigned)G, p, misc);
-              if (cta == 0)
-                p.gate_log[((size_t)slot_io * p.log_step_stride + pl.gi) * p.n_tokens + p.token] = 1;
-            }
-            csync();
-          }
-        }
-        tr.mark(6);
-        if (*abort) return;
-      }
       if (!gsi) continue;
       const bool image = part == 1;
       const int nchunks = image ? ochunks : pchunks, ngroups = image ? og : pg;
@@ -1274,6 +1337,50 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       r2word_p = acc + k + 2;
     }
     mask_pp = mask_p;
+    }
+
+    // ---- H. the W streams of the tick, one call site, after the row passes (little of the
+    //      tick's state is alive here): the gated residuals of the phase before the previous
+    //      one, then this phase's own stream if it is a dense group (followed by a grid barrier
+    //      that keeps a dense stack in model order).
+    if (mask_stream || dense) {
+      const int len_pp = plan[t - 2 >= 0 ? t - 2 : 0].len, g_pp = plan[t - 2 >= 0 ? t - 2 : 0].gi0;
+#pragma unroll 1
+      for (int u = 0; u < 3; ++u) {
+        const PersistGroup* gw = nullptr;
+        if (u < 2) {
+          if (u < len_pp && (mask_stream & (1u << u))) gw = p.groups + g_pp + u;
+        } else if (dense) {
+          gw = &desc(plan[t].gi);
+        }
+        if (!gw) continue;
+        if (u < 2) {
+          if (tid == 0) {
+            grid_wait(gw->bar + 2 + parity, (unsigned)G, p, misc);
+            __threadfence();
+          }
+          csync();
+          if (*abort) return;
+        }
+        const float* src = u < 2 ? gw->r
+                                 : gw->x + (long long)slot_io * gw->x_step_stride + (size_t)p.token * gw->d;
+        tr.mark(9);
+        n = w_stream(gw, src, gw->y + (size_t)p.token * gw->O, u == 2, smem, n, p.status, p.trace != nullptr);
+        if (tr.acc) tr.t = clock64();
+        if (*abort) return;
+        if (u == 2) {
+          if (tid == 0) {
+            red_relaxed_u32(gw->bar + parity, 1u);
+            grid_wait(gw->bar + parity, (unsigned)G, p, misc);
+            if (cta == 0)
+              p.gate_log[((size_t)slot_io * p.log_step_stride + plan[t].gi) * p.n_tokens + p.token] = 1;
+          }
+          csync();
+        }
+      }
+      tr.mark(6);
+      if (*abort) return;
+    }
   }
   if (lane == 0 || tid == kNC - 1) bulk_reduce_wait_read();
   tr.flush(p);

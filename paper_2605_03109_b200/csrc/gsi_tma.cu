@@ -4,7 +4,6 @@
 #include <cstring>
 
 #include "gsi_umma.cuh"
-#include "gsi_persistent.cuh"
 
 namespace gsi {
 
@@ -41,23 +40,6 @@ bool encode(CUtensorMap* m, const void* base, size_t rows, size_t cols, unsigned
 }
 
 }  // namespace
-
-bool encode_w_stream_map(void* out, const void* W, size_t rows, size_t cols, unsigned box_rows) {
-  static_assert(sizeof(CUtensorMap) == kPersistTmapBytes, "tensor map size");
-  EncodeTiledFn fn = encoder();
-  if (!fn || !W || !out) return false;
-  alignas(64) CUtensorMap m;
-  const cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
-  const cuuint64_t strides[1] = {(cuuint64_t)cols * 2};
-  const cuuint32_t box[2] = {(cuuint32_t)kPersistBoxCols, box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  if (fn(&m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(W), dims, strides, box, estr,
-         CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
-         CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
-    return false;
-  std::memcpy(out, &m, sizeof m);
-  return true;
-}
 
 bool build_tma_maps(const GroupParams& g, bool front, int max_tokens, TmaMaps* out) {
   std::memset(out, 0, sizeof *out);
