@@ -312,10 +312,12 @@ gsi_status_t gsi_stack_is_persistent(gsi_stack_t s, int* out);
  * counters (n_CTAs = SM count; NULL switches tracing off).  While set, thread 0
  * of every CTA of the persistent launch adds the SM cycles it spends in each
  * section of the per-phase pipeline:
- *   0 statistics of x, descriptors      1 wait for basis slab     2 pass 1
- *   3 collect max|x|                    4 fixed-point atomics     5 wait for the sums, gate of the previous phase
- *   6 residual rows                     7 gated residuals (W stream)
- *   8 wait for image slab               9 image rows              10 dense group (W stream, barrier)
+ *   0 barrier that opens the tick        1 wait for basis slab     2 pass 1
+ *   3 fixed-point conversion, reductions 4 wait for the sums, gate of the previous phase
+ *   5 residual rows                      7 wait for image slab     8 image rows
+ *   9 before a W stream (visibility of r) 10 the stream's share of its input into registers
+ *  11 wait for W pieces   12 arithmetic on W pieces   13 partial sums into y
+ *   6 after the streams of a tick (the grid barrier that follows a dense group)
  * The caller clears and reads the counters.  Applies from the next step.
  */
 #define GSI_TRACE_SECTIONS 16
