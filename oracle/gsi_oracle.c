@@ -305,3 +305,100 @@ int gsi_oracle_extend(const void* P, int p_dtype, int d, int k_cap, int k_act,
   free(g);
   return extended;
 }
+
+/* ------------------------------------------------------------------------ *
+ * FP8 storage of the cached image (Section 7.4: the image M = W V_k kept in
+ * FP8 halves the fast-path read volume).  The paper names no format, scaling
+ * or rounding; this reading is the common one: E4M3 codes (1 sign, 4 exponent
+ * bits with bias 7, 3 fraction bits; no infinities, S.1111.111 is NaN, largest
+ * finite value 448; exponent field 0 holds the subnormals m/8 * 2^-6), one
+ * fp32 scale per output row chosen so that the row's largest magnitude maps to
+ * 448, round to nearest with ties to the even code, saturating.
+ * ------------------------------------------------------------------------ */
+
+/* Value of an E4M3 code, from the definition of the format. */
+double gsi_oracle_e4m3_decode(uint8_t code) {
+  int s = code >> 7, e = (code >> 3) & 0xF, m = code & 7;
+  if (e == 15 && m == 7) return NAN;
+  double v = e == 0 ? ldexp((double)m / 8.0, -6) : ldexp(1.0 + (double)m / 8.0, e - 7);
+  return s ? -v : v;
+}
+
+/*
+ * Nearest E4M3 code of a float (ties to the even code), saturating at +-448;
+ * NaN gives the NaN code.  By exact arithmetic: within the binade 2^E the
+ * codes are spaced 2^(E-3) apart (E >= -6; below, the subnormal spacing 2^-9).
+ */
+uint8_t gsi_oracle_f32_to_e4m3_rne_sat(float vf) {
+  double v = (double)vf;
+  if (v != v) return 0x7F;
+  uint8_t sign = signbit(v) ? 0x80 : 0;
+  double a = fabs(v);
+  if (a >= 448.0) return (uint8_t)(sign | 0x7E); /* also +-inf: saturating */
+  if (a == 0.0) return sign;
+  int e;
+  (void)frexp(a, &e);
+  int E = e - 1;
+  if (E < -6) E = -6;
+  double scaled = ldexp(a, 3 - E); /* in units of the spacing: [8, 16) for normals, [0, 8) below */
+  double fl = floor(scaled);
+  double rem = scaled - fl;
+  unsigned q = (unsigned)fl;
+  if (rem > 0.5 || (rem == 0.5 && (q & 1))) q += 1;
+  if (q >= 16) { /* carried into the next binade */
+    q = 8;
+    E += 1;
+  }
+  unsigned bits;
+  if (q >= 8) {
+    bits = ((unsigned)(E + 7) << 3) | (q - 8);
+    if (bits > 0x7E) bits = 0x7E; /* 464 and above round past the largest code */
+  } else {
+    bits = q;
+  }
+  return (uint8_t)(sign | bits);
+}
+
+void gsi_oracle_e4m3_decode_array(const uint8_t* src, size_t n, double* dst) {
+  for (size_t i = 0; i < n; ++i) dst[i] = gsi_oracle_e4m3_decode(src[i]);
+}
+void gsi_oracle_f32_to_e4m3_array(const float* src, size_t n, uint8_t* dst) {
+  for (size_t i = 0; i < n; ++i) dst[i] = gsi_oracle_f32_to_e4m3_rne_sat(src[i]);
+}
+
+/*
+ * The image as stored in FP8.  Input: the image M [o][k] in double (Eq. (3.2)).
+ * Per row a:  m_j     = bf16_rne(M[a][j])            (the BF16 image of Section 4.2 is what gets quantised)
+ *             amax    = max_j |m_j|
+ *             scale_a = amax / 448 in fp32           (1 when the row is zero)
+ *             code_j  = e4m3_rne_sat( m_j / scale_a in fp32 )
+ *             Mq[a][j] = decode(code_j) * scale_a    (double)
+ * The two divisions are single fp32 operations, so that an implementation in
+ * fp32 arrives at the same codes from the same m_j.
+ * Outputs (any may be NULL): codes [o][k], scales [o], Mq [o][k].
+ */
+int gsi_oracle_quantise_image_e4m3(const double* M, int o, int k, uint8_t* codes,
+                                   float* scales, double* Mq) {
+  if (!M || o < 0 || k <= 0) return 1;
+#pragma omp parallel for schedule(static)
+  for (int a = 0; a < o; ++a) {
+    const double* Ma = M + (size_t)a * k;
+    float amax = 0.0f;
+    for (int j = 0; j < k; ++j) {
+      float m = (float)bf16_bits_to_f64(gsi_oracle_f64_to_bf16_rne(Ma[j]));
+      float am = fabsf(m);
+      if (am > amax) amax = am;
+    }
+    volatile float scale_v = amax > 0.0f ? amax / 448.0f : 1.0f;
+    const float scale = scale_v;
+    if (scales) scales[a] = scale;
+    for (int j = 0; j < k; ++j) {
+      float m = (float)bf16_bits_to_f64(gsi_oracle_f64_to_bf16_rne(Ma[j]));
+      volatile float t = m / scale;
+      uint8_t c = gsi_oracle_f32_to_e4m3_rne_sat(t);
+      if (codes) codes[(size_t)a * k + j] = c;
+      if (Mq) Mq[(size_t)a * k + j] = gsi_oracle_e4m3_decode(c) * (double)scale;
+    }
+  }
+  return 0;
+}

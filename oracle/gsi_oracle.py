@@ -58,6 +58,10 @@ def _load():
         lib.gsi_oracle_map.restype = i
         lib.gsi_oracle_extend.argtypes = [vp, i, i, i, i, vp, ctypes.c_double, vp, vp]
         lib.gsi_oracle_extend.restype = i
+        lib.gsi_oracle_e4m3_decode_array.argtypes = [vp, sz, vp]
+        lib.gsi_oracle_f32_to_e4m3_array.argtypes = [vp, sz, vp]
+        lib.gsi_oracle_quantise_image_e4m3.argtypes = [vp, i, i, vp, vp, vp]
+        lib.gsi_oracle_quantise_image_e4m3.restype = i
         _lib = lib
     return _lib
 
@@ -116,6 +120,36 @@ def image(W, P) -> np.ndarray:
     if rc:
         raise RuntimeError("gsi_oracle_image failed")
     return M
+
+
+def e4m3_decode(codes) -> np.ndarray:
+    """Values of E4M3 codes (Section 7.4 reading: the FP8 format of the image)."""
+    codes = _c(codes, np.uint8)
+    out = np.empty(codes.shape, np.float64)
+    _load().gsi_oracle_e4m3_decode_array(_ptr(codes), codes.size, _ptr(out))
+    return out
+
+
+def e4m3_encode(v) -> np.ndarray:
+    """Nearest E4M3 code of each float32 (ties to even, saturating)."""
+    v = _c(v, np.float32)
+    out = np.empty(v.shape, np.uint8)
+    _load().gsi_oracle_f32_to_e4m3_array(_ptr(v), v.size, _ptr(out))
+    return out
+
+
+def quantise_image_e4m3(M) -> dict:
+    """The image as stored in FP8 (Section 7.4): per-row scale, E4M3 codes of
+    the BF16 image, and the image those codes stand for (``Mq``, fp64)."""
+    M = _c(M, np.float64)
+    o, k = M.shape
+    codes = np.empty((o, k), np.uint8)
+    scales = np.empty(o, np.float32)
+    Mq = np.empty((o, k), np.float64)
+    rc = _load().gsi_oracle_quantise_image_e4m3(_ptr(M), o, k, _ptr(codes), _ptr(scales), _ptr(Mq))
+    if rc:
+        raise RuntimeError("gsi_oracle_quantise_image_e4m3 failed")
+    return {"codes": codes, "scales": scales, "Mq": Mq}
 
 
 def project(x, P, eps: float) -> dict:
@@ -191,7 +225,7 @@ def apply_map(M, W, g, r, gate, x=None, want_alt: bool = False):
     return (y, y_alt) if want_alt else y
 
 
-def forward(x, P, eps: float, Ws, gate_override=None, rows=None) -> dict:
+def forward(x, P, eps: float, Ws, gate_override=None, rows=None, fp8_image: bool = False) -> dict:
     """The whole layer for one input group: the maps in ``Ws`` share x, P, g, r
     and one gate decision per token.
 
@@ -199,7 +233,7 @@ def forward(x, P, eps: float, Ws, gate_override=None, rows=None) -> dict:
     of its output rows; the projection and the gate always use the full basis.
     ``gate_override`` substitutes given gate bytes when forming y (used for
     tokens whose rho sits on the threshold); the oracle's own decision is still
-    returned as ``gate``.
+    returned as ``gate``.  ``fp8_image`` stores the image in FP8 first.
     """
     pr = project(x, P, eps)
     gate_used = pr["gate"] if gate_override is None else _c(gate_override, np.uint8)
@@ -209,6 +243,8 @@ def forward(x, P, eps: float, Ws, gate_override=None, rows=None) -> dict:
         if rows is not None and rows[j] is not None:
             W = np.ascontiguousarray(W[np.asarray(rows[j])])
         M = image(W, P)
+        if fp8_image:   # the image as stored in FP8 (Section 7.4)
+            M = quantise_image_e4m3(M)["Mq"]
         ys.append(apply_map(M, W, pr["g"], pr["r"], gate_used))
     pr["y"] = ys
     pr["gate_used"] = gate_used

@@ -454,3 +454,108 @@ def test_E4_after_the_extension_the_token_lies_in_the_span():
     W = O.f64_to_bf16_rne(rng.standard_normal((o, d)) * 0.1)
     col = O.image(W, np.ascontiguousarray(P2[:, k_act:k_act + 1]))
     assert np.allclose(col[:, 0], O.bf16_to_f64(W) @ P2[:, k_act].astype(np.float64), rtol=0, atol=1e-14)
+
+
+# ---------------------------------------------------------------- FP8 image (Section 7.4)
+def _e4m3_table():
+    """Every non-negative finite E4M3 value from the format's definition, by
+    exact rational arithmetic (independent of the oracle's decoder)."""
+    vals = []
+    for e in range(16):
+        for m in range(8):
+            if e == 15 and m == 7:
+                continue
+            vals.append(Fraction(m, 8) * Fraction(1, 64) if e == 0
+                        else (1 + Fraction(m, 8)) * Fraction(2) ** (e - 7))
+    return vals
+
+
+def test_F1_e4m3_decode_is_the_format_definition():
+    codes = np.arange(256, dtype=np.uint8)
+    v = O.e4m3_decode(codes)
+    table = _e4m3_table()
+    assert len(table) == 127
+    assert [Fraction(float(x)) for x in v[:127]] == table          # exact, all finite codes
+    assert np.isnan(v[0x7F]) and np.isnan(v[0xFF])
+    np.testing.assert_array_equal(v[128:255], -v[0:127])
+    # landmarks: smallest subnormal, smallest normal, one, largest finite
+    assert v[0x01] == 2.0 ** -9 and v[0x08] == 2.0 ** -6 and v[0x38] == 1.0 and v[0x7E] == 448.0
+    assert np.all(np.diff(v[:127]) > 0)
+
+
+def test_F2_e4m3_encode_is_nearest_with_ties_to_even_by_brute_force():
+    table = _e4m3_table()
+    tf = np.array([float(t) for t in table])
+    rng = np.random.default_rng(7)
+    samples = np.concatenate([
+        tf,                                               # the values themselves
+        (tf[:-1] + tf[1:]) / 2,                           # every midpoint (exact in fp32: 5 significant bits)
+        np.nextafter(((tf[:-1] + tf[1:]) / 2).astype(np.float32), np.float32(np.inf)).astype(np.float64),
+        np.nextafter(((tf[:-1] + tf[1:]) / 2).astype(np.float32), np.float32(0)).astype(np.float64),
+        np.abs(rng.normal(0, 100, 4000)), np.abs(rng.normal(0, 1, 4000)), np.abs(rng.normal(0, 0.01, 4000)),
+    ]).astype(np.float32)
+    samples = samples[samples <= 448]
+    got = O.e4m3_encode(samples)
+    for s, c in zip(samples.tolist(), got.tolist()):
+        fs = Fraction(s)
+        dist = [abs(fs - t) for t in table]
+        best = min(dist)
+        cands = [i for i, dd in enumerate(dist) if dd == best]
+        want = cands[0] if len(cands) == 1 else [i for i in cands if i % 2 == 0][0]
+        assert c == want, (s, c, want)
+    # sign, saturation, NaN
+    neg = O.e4m3_encode(-samples)
+    np.testing.assert_array_equal(neg & 0x7F, got)
+    assert np.all((neg >> 7) == 1)
+    big = np.array([448.0, 449.0, 463.9, 464.0, 1e6, np.inf, -np.inf, -500.0], np.float32)
+    np.testing.assert_array_equal(O.e4m3_encode(big), [0x7E] * 6 + [0xFE] * 2)
+    assert O.e4m3_encode(np.array([np.nan], np.float32))[0] & 0x7F == 0x7F
+
+
+def test_F3_e4m3_encode_agrees_with_the_library_conversion():
+    torch = pytest.importorskip("torch")
+    if not hasattr(torch, "float8_e4m3fn"):
+        pytest.skip("no float8 in this torch")
+    rng = np.random.default_rng(11)
+    v = np.concatenate([rng.normal(0, 120, 20000), rng.normal(0, 1, 20000), rng.normal(0, 0.004, 20000)])
+    v = np.clip(v, -448, 448).astype(np.float32)
+    lib = torch.from_numpy(v).to(torch.float8_e4m3fn).view(torch.uint8).numpy()
+    got = O.e4m3_encode(v)
+    # -0 and +0 are the same number
+    same = (lib == got) | (((lib | got) & 0x7F) == 0)
+    assert same.all()
+
+
+def test_F4_fp8_image_scales_codes_and_error_bound():
+    rng = np.random.default_rng(3)
+    Wb, W, P_store, P, q, x = rand_problem(rng, 40, 96, 16, 4)
+    M = O.image(Wb, P_store)
+    M[7] = 0.0                                             # a zero row
+    M[9, 3] = 50.0 * np.abs(M[9]).max()                    # a row with a wide spread (subnormal codes)
+    qz = O.quantise_image_e4m3(M)
+    codes, scales, Mq = qz["codes"], qz["scales"], qz["Mq"]
+    _, mb = f32_to_bf16_bits_trunc_safe(M)                 # the BF16 image, by numpy
+    amax = np.abs(mb).max(axis=1)
+    # scale: amax / 448 as one fp32 division (numpy float32 arithmetic), 1 for the zero row
+    want_scale = np.where(amax > 0, amax.astype(np.float32) / np.float32(448), np.float32(1))
+    np.testing.assert_array_equal(scales, want_scale)
+    assert np.all(codes[7] == 0) and np.all(Mq[7] == 0)
+    # the largest element of every other row takes the largest code
+    for a in range(40):
+        if a != 7:
+            assert codes[a, np.abs(mb[a]).argmax()] & 0x7F == 0x7E
+    # the stored image is decode(code) * scale, and lies within half a code spacing of the BF16 image
+    np.testing.assert_array_equal(Mq, O.e4m3_decode(codes) * scales.astype(np.float64)[:, None])
+    t = np.abs(mb) / scales.astype(np.float64)[:, None]
+    spacing = np.where(t < 2.0 ** -6, 2.0 ** -9, 2.0 ** (np.floor(np.log2(np.maximum(t, 2.0 ** -6))) - 3))
+    err = np.abs(Mq - mb) / scales.astype(np.float64)[:, None]
+    assert np.all(err <= spacing / 2 * (1 + 1e-6) + 1e-6 * t)
+    assert np.any(t[9] < 2.0 ** -6)                        # the subnormal range is exercised
+    # forward(fp8_image=True) is forward() with the image replaced by Mq
+    Ws = [Wb]
+    a = O.forward(x, P_store, 0.05, Ws, fp8_image=True)
+    g = a["g"]
+    M0 = O.quantise_image_e4m3(O.image(Wb, P_store))["Mq"]
+    fast = a["gate"] == 0
+    if fast.any():
+        np.testing.assert_allclose(a["y"][0][fast], (g @ M0.T)[fast], rtol=1e-12, atol=1e-14)
