@@ -99,7 +99,7 @@ class ClockSampler:
 
 
 # ----------------------------------------------------------------------------
-def build_workload(spec, device, n_steps, static_projection=False):
+def build_workload(spec, device, n_steps, static_projection=False, fp8_image=False):
     """Draw the whole stack on the device.  Returns (gsi layers, dense layers,
     x tensors per group, host-side copies needed later)."""
     import torch
@@ -110,7 +110,8 @@ def build_workload(spec, device, n_steps, static_projection=False):
         for gi, g in enumerate(spec.groups):
             m = S.materialize_group(spec, layer, gi, n_steps * spec.batch, device=device)
             lay = G.Layer(m["W"], m["P"], spec.eps, max_tokens=spec.batch,
-                          flags=G.GSI_FLAG_STATIC_PROJECTION if static_projection else 0)
+                          flags=(G.GSI_FLAG_STATIC_PROJECTION if static_projection else 0) |
+                          (G.GSI_FLAG_FP8_IMAGE if fp8_image else 0))
             den = G.Layer(m["W"], None, 0.0, max_tokens=spec.batch, flags=G.GSI_FLAG_DENSE)
             layers.append(lay)
             dense.append(den)
@@ -265,12 +266,14 @@ def whole_job_tokens_per_s(world: int, batch: int, ms_max: float) -> float:
     return world * batch / (ms_max * 1e-3)
 
 
-def algorithmic_bytes(spec, fired_per_group_step):
+def algorithmic_bytes(spec, fired_per_group_step, fp8_image=False):
     """bytes(P) + bytes(W_P) + fired*bytes(W) + activations, per step, from the
     REALISED fired indicator (any token of the batch gated -> W streamed once)."""
     ng = len(spec.groups)
     wbytes = spec.bytes_w_per_group()
     fast = spec.bytes_fast_per_step()
+    if fp8_image:   # one byte per image entry and one fp32 scale per output row instead of two bytes
+        fast -= sum(sum(g.d_out) * (g.k - 4) for g in spec.groups) * spec.n_layers
     act = spec.bytes_act_per_token() * spec.batch
     w = 0.0
     for gi in range(ng):
@@ -416,6 +419,9 @@ def main():
     ap.add_argument("--outlier", type=float, default=0.10)
     ap.add_argument("--batch", type=int, default=64, help="tokens per step of the gptj_b64 workload")
     ap.add_argument("--layers", type=int, default=0, help="override the layer count (profiling)")
+    ap.add_argument("--fp8-image", action="store_true",
+                    help="keep the cached images in FP8 (E4M3 codes, one fp32 scale per output row; Section 7.4): "
+                         "halves the image bytes of the fast path; batch-1 persistent stacks only")
     ap.add_argument("--static-projection", action="store_true",
                     help="negative control (remark after Theorem 3.1, Section 3.3, and Section 6.7 \"Negative control\"): the gate is computed and "
                          "logged but W r is never added, so the step costs the fast path only")
@@ -479,7 +485,7 @@ def main():
         dist.init_process_group("nccl", device_id=device)
 
     n_steps = min(spec.steps, max(args.steps, 1))
-    layers, dense_layers, xs, keep = build_workload(spec, device, n_steps, args.static_projection)
+    layers, dense_layers, xs, keep = build_workload(spec, device, n_steps, args.static_projection, args.fp8_image)
     concurrent = [] if args.no_concurrent else spec.concurrent_groups()
     stack = G.Stack(layers, concurrent=concurrent, mode=1 if args.per_stage else 0)
     stack.bind(xs, n_steps=n_steps)
@@ -530,7 +536,7 @@ def main():
 
     if rank == 0:
         peaks, peak_kind = measured_peaks()
-        ab = algorithmic_bytes(spec, fired)
+        ab = algorithmic_bytes(spec, fired, args.fp8_image)
         sec = ms_max * 1e-3
         achieved = ab["total"] / sec / 1e9
         peak = float(peaks["hbm_gbs"])
@@ -556,6 +562,7 @@ def main():
                 "parallel_branches": ("attn_out|proj of each block share a phase" if concurrent
                                       else "none declared"),
                 "static_projection": bool(args.static_projection),
+                "image": "fp8 e4m3, fp32 scale per output row" if args.fp8_image else "bf16",
                 "weights": "bf16", "basis": spec.groups[0].p_dtype, "activations": "f32",
                 "distinct_input_steps": n_steps,
                 "l2": "inputs_larger_than_l2 (0.88 GB of basis+image per step, distinct per layer)",

@@ -80,7 +80,17 @@ enum {
      GEMV on the fp32 x.  Calls of 2 or more tokens (d a multiple of 64, every
      d_out a multiple of 128): tensor-core GEMM with x rounded to bf16, as an
      ordinary bf16 GEMM takes its activations. */
-  GSI_FLAG_DENSE = 2u
+  GSI_FLAG_DENSE = 2u,
+  /* The image is kept in FP8 (Section 7.4: halves the bytes the fast path
+     reads; the paper leaves format and quality open).  Here: E4M3 codes of the
+     BF16 image with one fp32 scale per output row, scale = max|row| / 448 (1 for
+     a zero row), code = nearest E4M3 (ties to even, saturating) of
+     element / scale, both divisions single fp32 operations; y = scale * (codes . c).
+     Served by the persistent stack kernel only (bf16 basis, k a power of two in
+     64..512, max_tokens <= 2): gsi_create returns GSI_ERR_UNSUPPORTED otherwise,
+     and so do the single-group forward calls and binding a stack that cannot run
+     persistently.  Not combinable with GSI_FLAG_DENSE. */
+  GSI_FLAG_FP8_IMAGE = 4u
 };
 
 typedef struct {
@@ -219,6 +229,16 @@ gsi_status_t gsi_extend_basis(gsi_handle_t h, const float* x, float tau, int* k_
 /* Device pointer to the image of map j inside the workspace ([d_out_j][k] bf16),
  * so a caller can inspect or persist it. */
 gsi_status_t gsi_get_image(gsi_handle_t h, int map, const void** W_P_out);
+
+/* GSI_FLAG_FP8_IMAGE handles: device pointer to the FP8 image of ALL maps
+ * (rows in map order, O = sum d_out, padded with zero rows to a multiple of 16)
+ * as the persistent kernel streams it, and its size in bytes.  Per 16 rows R:
+ * k/16 tiles of 256 bytes, then the 16 row scales (fp32).  In tile K, the 8
+ * bytes at 8*l (l = 4g + t, g < 8, t < 4) are the codes of elements (row, column
+ * within the tile) (g,2t) (g,2t+1) (g+8,2t) (g+8,2t+1) (g,2t+8) (g,2t+9)
+ * (g+8,2t+8) (g+8,2t+9).  gsi_get_image still returns the BF16 image the codes
+ * were taken from. */
+gsi_status_t gsi_get_image_fp8(gsi_handle_t h, const void** tiled_out, size_t* bytes_out);
 
 /* Synchronises the handle's last stream and returns the device status word:
  * 0, or a GSI_ERR_* code recorded by a kernel (e.g. a bounded wait that gave

@@ -14,12 +14,12 @@ import torch
 from . import build as _build
 
 GSI_BF16, GSI_F32 = 0, 1
-GSI_FLAG_NONE, GSI_FLAG_STATIC_PROJECTION, GSI_FLAG_DENSE = 0, 1, 2
+GSI_FLAG_NONE, GSI_FLAG_STATIC_PROJECTION, GSI_FLAG_DENSE, GSI_FLAG_FP8_IMAGE = 0, 1, 2, 4
 GSI_MAX_MAPS, GSI_MAX_TOKENS = 8, 64
 
 EXPORTED = [
     "gsi_status_string", "gsi_build_image", "gsi_workspace_bytes", "gsi_create",
-    "gsi_forward", "gsi_forward_n", "gsi_forward_host", "gsi_forward_static", "gsi_extend_basis", "gsi_get_image", "gsi_get_status",
+    "gsi_forward", "gsi_forward_n", "gsi_forward_host", "gsi_forward_static", "gsi_extend_basis", "gsi_get_image", "gsi_get_image_fp8", "gsi_get_status",
     "gsi_destroy", "gsi_stack_workspace_bytes", "gsi_stack_create", "gsi_stack_bind",
     "gsi_stack_set_mode", "gsi_stack_set_concurrent", "gsi_stack_is_persistent", "gsi_stack_set_trace", "gsi_stack_set_spin_limit", "gsi_stack_seek", "gsi_stack_step", "gsi_stack_launches_per_step",
     "gsi_stack_step_host", "gsi_stack_get_status", "gsi_stack_destroy",
@@ -62,6 +62,7 @@ def _load():
     l.gsi_forward_static.argtypes = [C.POINTER(vp), C.POINTER(i), i, vp, i, vp, i, i, C.c_float,
                                      vp, i, vp, vp, vp, vp]
     l.gsi_get_image.argtypes = [vp, i, C.POINTER(vp)]
+    l.gsi_get_image_fp8.argtypes = [vp, C.POINTER(vp), C.POINTER(C.c_size_t)]
     l.gsi_extend_basis.argtypes = [vp, vp, C.c_float, vp, vp, vp, vp]
     l.gsi_get_status.argtypes = [vp, C.POINTER(i)]
     l.gsi_destroy.argtypes = [vp]
@@ -242,6 +243,23 @@ class Layer:
         off = p.value - base
         nbytes = self.d_out[j] * self.k * 2
         return self.workspace[off:off + nbytes].view(torch.bfloat16).view(self.d_out[j], self.k).clone()
+
+    def image_fp8(self):
+        """The FP8 image of all maps as stored (GSI_FLAG_FP8_IMAGE handles): codes
+        ``[sum d_out][k]`` uint8 and row scales ``[sum d_out]`` fp32, copied out of
+        the tiled layout the header documents (a rearrangement of bytes only)."""
+        p, n = C.c_void_p(), C.c_size_t()
+        _check(lib.gsi_get_image_fp8(self.handle, C.byref(p), C.byref(n)), "gsi_get_image_fp8")
+        off = p.value - self.workspace.data_ptr()
+        raw = self.workspace[off:off + n.value]
+        O, k = sum(self.d_out), self.k
+        R, KT = (O + 15) // 16, k // 16
+        raw = raw.view(R, KT * 256 + 64)
+        # tile bytes [R][K][g][t][c8][r8][e]: element (row g + 8 r8, column 2 t + 8 c8 + e)
+        tiles = raw[:, :KT * 256].reshape(R, KT, 8, 4, 2, 2, 2)
+        codes = tiles.permute(0, 5, 2, 1, 4, 3, 6).reshape(R * 16, k)[:O].clone()
+        scales = raw[:, KT * 256:].contiguous().view(torch.float32).reshape(R * 16)[:O].clone()
+        return codes, scales
 
     def status(self) -> int:
         v = C.c_int()

@@ -45,6 +45,7 @@ gsi_status_t check_desc(const gsi_desc_t* d) {
     if (d->d_out[j] <= 0) return GSI_ERR_INVALID_ARG;
     if (d->d_out[j] % 8) return GSI_ERR_UNSUPPORTED;
   }
+  if ((d->flags & GSI_FLAG_FP8_IMAGE) && (d->flags & GSI_FLAG_DENSE)) return GSI_ERR_INVALID_ARG;
   if (!(d->flags & GSI_FLAG_DENSE)) {
     if (d->k <= 0) return GSI_ERR_INVALID_ARG;
     if (d->k % 8 || d->k > 1024 || d->k > d->d) return GSI_ERR_UNSUPPORTED;
@@ -103,7 +104,7 @@ Layout make_layout_ws(const gsi_desc_t* d) {
   const bool packed = !dense && d->p_dtype == GSI_BF16 && d->k >= 64 && d->k <= 512 &&
                       (d->k & (d->k - 1)) == 0 && d->max_tokens <= kPersistMaxTokens;
   L.pk_pp = take(packed ? (size_t)((d->d + 15) / 16 * 16) * k * 2 : 0);
-  L.pk_wpp = take(packed ? (size_t)((O + 15) / 16 * 16) * k * 2 : 0);
+  L.pk_wpp = take(packed ? (size_t)((O + 15) / 16) * persist_image_row_bytes(d->k, d->flags & GSI_FLAG_FP8_IMAGE) : 0);
   L.packed = packed;
   L.total = at;
   return L;
@@ -165,8 +166,10 @@ struct gsi_stack {
 // The tiled copies of the basis and of the images that the persistent kernel streams.
 static bool repack(gsi_layer* h, cudaStream_t stream) {
   const Layout& L = h->lay;
-  return launch_pack_t16(h->gp.P, h->desc.d, h->desc.k, h->ws + L.pk_pp, stream) == cudaSuccess &&
-         launch_pack_t16(h->ws + L.wp, L.O, h->desc.k, h->ws + L.pk_wpp, stream) == cudaSuccess;
+  if (launch_pack_t16(h->gp.P, h->desc.d, h->desc.k, h->ws + L.pk_pp, stream) != cudaSuccess) return false;
+  return ((h->desc.flags & GSI_FLAG_FP8_IMAGE)
+              ? launch_pack_t16_fp8(h->ws + L.wp, L.O, h->desc.k, h->ws + L.pk_wpp, stream)
+              : launch_pack_t16(h->ws + L.wp, L.O, h->desc.k, h->ws + L.pk_wpp, stream)) == cudaSuccess;
 }
 
 extern "C" {
@@ -214,6 +217,7 @@ gsi_status_t gsi_create(const gsi_desc_t* desc, const void* const* W, const void
   for (int j = 0; j < desc->n_maps; ++j)
     if (!W[j] || !aligned16(W[j])) return GSI_ERR_INVALID_ARG;
   Layout L = make_layout_ws(desc);
+  if ((desc->flags & GSI_FLAG_FP8_IMAGE) && !L.packed) return GSI_ERR_UNSUPPORTED;   // the persistent kernel alone reads FP8 images
   if (workspace_bytes < L.total) return GSI_ERR_WORKSPACE;
 
   gsi_layer* h = new (std::nothrow) gsi_layer();
@@ -320,6 +324,7 @@ gsi_status_t gsi_create(const gsi_desc_t* desc, const void* const* W, const void
 gsi_status_t gsi_forward_n(gsi_handle_t h, const float* x, int n_tokens, float* y,
                            unsigned char* gate_mask_out, float* rho_out, gsi_stream_t stream) {
   if (!h || n_tokens < 0 || n_tokens > h->desc.max_tokens) return GSI_ERR_INVALID_ARG;
+  if (h->desc.flags & GSI_FLAG_FP8_IMAGE) return GSI_ERR_UNSUPPORTED;   // stacks on the persistent kernel only
   if (n_tokens == 0) return GSI_OK;
   if (!x || !y || !gate_mask_out) return GSI_ERR_INVALID_ARG;
   if (!aligned16(x) || !aligned16(y)) return GSI_ERR_INVALID_ARG;
@@ -396,6 +401,14 @@ gsi_status_t gsi_get_image(gsi_handle_t h, int map, const void** out) {
   if (!h || !out || map < 0 || map >= h->desc.n_maps) return GSI_ERR_INVALID_ARG;
   if (h->desc.flags & GSI_FLAG_DENSE) return GSI_ERR_UNSUPPORTED;
   *out = h->ws + h->lay.wp + (size_t)h->gp.off[map] * h->desc.k * 2;
+  return GSI_OK;
+}
+
+gsi_status_t gsi_get_image_fp8(gsi_handle_t h, const void** out, size_t* bytes_out) {
+  if (!h || !out || !bytes_out) return GSI_ERR_INVALID_ARG;
+  if (!(h->desc.flags & GSI_FLAG_FP8_IMAGE)) return GSI_ERR_UNSUPPORTED;
+  *out = h->ws + h->lay.pk_wpp;
+  *bytes_out = (size_t)((h->lay.O + 15) / 16) * persist_image_row_bytes(h->desc.k, true);
   return GSI_OK;
 }
 
@@ -561,6 +574,9 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
     s->persistent = coop && persistent_eligible(s, sms);
     if (s->mode == 2 && !s->persistent) return GSI_ERR_UNSUPPORTED;
   }
+  if (!s->persistent)
+    for (const gsi_layer* h : s->groups)
+      if (h->desc.flags & GSI_FLAG_FP8_IMAGE) return GSI_ERR_UNSUPPORTED;
   if (!s->persistent && !s->aux) {
     bool any = false;
     for (char c : s->pair_first) any = any || c;

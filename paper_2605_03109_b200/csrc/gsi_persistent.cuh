@@ -15,11 +15,16 @@ constexpr int kPersistPieceBytes = 32768;   // largest contiguous piece of the W
 constexpr int kPersistMaxD = 16384;     // widest input: a row of W fits one piece, a lane's share of r fits its registers
 constexpr int kPersistMaxWRows = 256;   // rows of W (all maps of a group) one CTA may own
 
+// Bytes of 16 rows of a tiled matrix of rank k.
+__host__ __device__ inline int persist_image_row_bytes(int k, bool fp8) { return fp8 ? k * 16 + 64 : k * 32; }
+
 struct PersistGroup {
   // Basis [d][k] and concatenated images [O][k], bf16, as 16 x 16 tiles: tile (R, K) at
   // ((R * k/16 + K) * 512) bytes; its 16-byte word l = 4g + t holds elements (g, 2t..2t+1),
   // (g+8, 2t..2t+1), (g, 2t+8..2t+9), (g+8, 2t+8..2t+9): the A operand of mma.m16n8k16.
-  // Rows past d (O) are zero.
+  // Rows past d (O) are zero.  With GSI_FLAG_FP8_IMAGE the image holds one byte (an E4M3
+  // code) per element in the same order (tiles of 256 bytes), and every 16 rows end with
+  // their 16 fp32 row scales: persist_image_row_bytes(k, true) bytes per 16 rows.
   const uint16_t* P;
   const uint16_t* WP;
   const uint16_t* W[GSI_MAX_MAPS];   // [d_out_j][d] bf16
@@ -87,6 +92,8 @@ cudaError_t launch_decode_step(const PersistParams& p, int grid, bool pairs, int
 cudaError_t launch_abs_max_bf16(const void* p, size_t n, float* out, cudaStream_t st);
 // Row-major [rows][k] bf16 -> the tiled layout described at PersistGroup::P.
 cudaError_t launch_pack_t16(const void* src, int rows, int k, void* dst, cudaStream_t st);
+// Row-major [rows][k] bf16 -> E4M3 codes with per-row scales, tiled (see PersistGroup::P).
+cudaError_t launch_pack_t16_fp8(const void* src, int rows, int k, void* dst, cudaStream_t st);
 cudaError_t launch_patch_pmax(PersistGroup* groups, const float* const* pmax_ptrs, int n,
                               cudaStream_t st);
 

@@ -346,20 +346,21 @@ __device__ __forceinline__ bool produce_w(const PersistGroup& g, unsigned char* 
   return ok;
 }
 
-// Tile rows [a, b) (16 matrix rows each) of a tiled [rows][k] bf16 matrix as chunks of whole
-// tile rows.
-__device__ __forceinline__ bool produce_rows(const uint16_t* base, int k, int a, int b, unsigned char* smem) {
+// Tile rows [a, b) (16 matrix rows each, row_bytes bytes) of a tiled matrix of rank k as chunks
+// of whole tile rows (as many per chunk as 16 KB hold of the bf16 form).
+__device__ __forceinline__ bool produce_rows(const void* base, int k, int row_bytes, int a, int b,
+                                             unsigned char* smem) {
   Producer& pr = *reinterpret_cast<Producer*>(smem + kOffProd);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + kOffBar);
   const int gc = kChunk / (k * 32);
   for (int r = a; r < b; r += gc) {
     const int groups = min(gc, b - r);
-    const uint32_t bytes = (uint32_t)groups * k * 32;
+    const uint32_t bytes = (uint32_t)(groups * row_bytes);
     const unsigned off = producer_acquire(smem, bytes);
     if (off == 0xffffffffu) return false;
     uint64_t* fb = &full[pr.n % kNB];
     mbar_expect_tx(fb, bytes);
-    bulk_g2s(smem + kOffRing + off, base + (size_t)r * k * 16, bytes, fb);
+    bulk_g2s(smem + kOffRing + off, static_cast<const char*>(base) + (size_t)r * row_bytes, bytes, fb);
     ++pr.n;
   }
   return true;
@@ -384,8 +385,10 @@ __device__ void producer(const PersistParams& p, unsigned char* smem, Misc* misc
     const Plan& pl = plan[t];
     const PersistGroup* g = p.groups + pl.gi;   // read only when the tick has a group
     if (pl.kind == 1) {
-      ok = produce_rows(g->P, g->k, pl.p0 >> 4, (pl.p0 >> 4) + pl.pg, smem);
-      if (ok) ok = produce_rows(g->WP, g->k, pl.o0 >> 4, (pl.o0 >> 4) + pl.og, smem);
+      ok = produce_rows(g->P, g->k, g->k * 32, pl.p0 >> 4, (pl.p0 >> 4) + pl.pg, smem);
+      if (ok)
+        ok = produce_rows(g->WP, g->k, persist_image_row_bytes(g->k, g->flags & GSI_FLAG_FP8_IMAGE), pl.o0 >> 4,
+                          (pl.o0 >> 4) + pl.og, smem);
     }
     unsigned wmask = 0;
     const int len_pp = t >= 2 ? plan[t - 2].len : 0, g_pp = t >= 2 ? plan[t - 2].gi0 : 0;
@@ -450,6 +453,19 @@ __device__ __forceinline__ float sum2(unsigned long long v) {
   float lo, hi;
   asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
   return lo + hi;
+}
+
+// Two E4M3 codes -> two bf16 (exact: every E4M3 value is a bf16 value), low byte to low half.
+__device__ __forceinline__ uint32_t e4m3x2_to_bf16x2(uint32_t two) {
+  uint32_t h, out;
+  unsigned short lo16, hi16;
+  float lo, hi;
+  asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h) : "h"((unsigned short)two));
+  asm("mov.b32 {%0, %1}, %2;" : "=h"(lo16), "=h"(hi16) : "r"(h));
+  asm("cvt.f32.f16 %0, %1;" : "=f"(lo) : "h"(lo16));
+  asm("cvt.f32.f16 %0, %1;" : "=f"(hi) : "h"(hi16));
+  asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(out) : "f"(hi), "f"(lo));
+  return out;
 }
 
 // D (16 x 8, fp32) += A (16 x 16, bf16) B (16 x 8, bf16) on the tensor cores.
@@ -1268,6 +1284,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       const unsigned n0 = image ? n : n_p0;
       const int row_base = image ? pl.o0 : pl.p0, row_end = image ? g.O : g.d;
       float* out = image ? g.y + (size_t)p.token * g.O : g.r;
+      const bool f8 = image && (g.flags & GSI_FLAG_FP8_IMAGE);
       if (image) {
         n += ochunks;
         ok = ok && chunks_landed(smem, n0, ochunks, abort);
@@ -1285,17 +1302,39 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
           if (lane == 0)
             for (; released < ci; ++released) mbar_arrive(&empty[(n0 + released) % kNB]);
           released = ci;
-          const unsigned char* trow = ring + s_off[(n0 + ci) % kNB] + (size_t)rr * KT * 512 + lane * 16;
           const unsigned char* cb = reinterpret_cast<const unsigned char*>(s_cb) + lane * 8;
           float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
+          float sc_lo = 1.f, sc_hi = 1.f;   // FP8 image: the scales of rows lg and lg + 8
+          if (f8) {
+            // tiles of one byte per element, expanded to bf16 in registers; the row scales follow the tiles
+            const unsigned char* trow8 = ring + s_off[(n0 + ci) % kNB] + (size_t)rr * (KT * 256 + 64);
+            sc_lo = *reinterpret_cast<const float*>(trow8 + KT * 256 + lg * 4);
+            sc_hi = *reinterpret_cast<const float*>(trow8 + KT * 256 + lg * 4 + 32);
+            trow8 += lane * 8;
 #pragma unroll 2
-          for (int K = 0; K < KT; K += 2) {   // two chains of dependent instructions
-            const uint4 a0 = *reinterpret_cast<const uint4*>(trow + K * 512);
-            const uint2 b0 = *reinterpret_cast<const uint2*>(cb + K * 256);
-            const uint4 a1 = *reinterpret_cast<const uint4*>(trow + K * 512 + 512);
-            const uint2 b1 = *reinterpret_cast<const uint2*>(cb + K * 256 + 256);
-            mma_bf16(d0, a0, b0.x, b0.y);
-            mma_bf16(d1, a1, b1.x, b1.y);
+            for (int K = 0; K < KT; K += 2) {
+              const uint2 q0 = *reinterpret_cast<const uint2*>(trow8 + K * 256);
+              const uint2 b0 = *reinterpret_cast<const uint2*>(cb + K * 256);
+              const uint2 q1 = *reinterpret_cast<const uint2*>(trow8 + K * 256 + 256);
+              const uint2 b1 = *reinterpret_cast<const uint2*>(cb + K * 256 + 256);
+              const uint4 a0 = make_uint4(e4m3x2_to_bf16x2(q0.x), e4m3x2_to_bf16x2(q0.x >> 16),
+                                          e4m3x2_to_bf16x2(q0.y), e4m3x2_to_bf16x2(q0.y >> 16));
+              const uint4 a1 = make_uint4(e4m3x2_to_bf16x2(q1.x), e4m3x2_to_bf16x2(q1.x >> 16),
+                                          e4m3x2_to_bf16x2(q1.y), e4m3x2_to_bf16x2(q1.y >> 16));
+              mma_bf16(d0, a0, b0.x, b0.y);
+              mma_bf16(d1, a1, b1.x, b1.y);
+            }
+          } else {
+            const unsigned char* trow = ring + s_off[(n0 + ci) % kNB] + (size_t)rr * KT * 512 + lane * 16;
+#pragma unroll 2
+            for (int K = 0; K < KT; K += 2) {   // two chains of dependent instructions
+              const uint4 a0 = *reinterpret_cast<const uint4*>(trow + K * 512);
+              const uint2 b0 = *reinterpret_cast<const uint2*>(cb + K * 256);
+              const uint4 a1 = *reinterpret_cast<const uint4*>(trow + K * 512 + 512);
+              const uint2 b1 = *reinterpret_cast<const uint2*>(cb + K * 256 + 256);
+              mma_bf16(d0, a0, b0.x, b0.y);
+              mma_bf16(d1, a1, b1.x, b1.y);
+            }
           }
           // columns 0, 1 (lane pair 0) and 2 (lane pair 1) of D are the three terms of c
           const float lo = d0[0] + d1[0], lo1 = d0[1] + d1[1], hi = d0[2] + d1[2], hi1 = d0[3] + d1[3];
@@ -1303,7 +1342,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
           if (lt == 0) {
 #pragma unroll
             for (int h = 0; h < 2; ++h) {
-              const float dot = h ? (hi + hi1) + hi2 : (lo + lo1) + lo2;
+              const float dot = h ? ((hi + hi1) + hi2) * sc_hi : ((lo + lo1) + lo2) * sc_lo;
               const int row = R * 16 + lg + 8 * h;
               if (row_base + row < row_end) {
                 if (image) {

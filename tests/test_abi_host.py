@@ -13,7 +13,7 @@ ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
 def declared_symbols():
     text = open(os.path.join(ROOT, "include", "gsi.h")).read()
     text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
-    names = set(re.findall(r"\b(gsi_[a-z_]+)\s*\(", text))
+    names = set(re.findall(r"\b(gsi_[a-z0-9_]+)\s*\(", text))
     return sorted(names)
 
 
