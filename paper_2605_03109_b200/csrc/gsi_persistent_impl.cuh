@@ -59,6 +59,7 @@ constexpr int kNC = kNW * 32;               // consumer threads
 constexpr int kThreadsP = kNC + 32;         // + producer warp
 constexpr int kNB = 64;                     // chunks in flight at most (one barrier pair each)
 constexpr int kChunk = 16384;               // largest chunk
+static_assert(kPersistMaxWRows <= kPersistConsumerWarps * 32, "one thread per row of a W stream");
 constexpr int kWVecMax = 5;                 // 16-byte vectors of a row one lane may own in the W stream (d <= 16384)
 constexpr unsigned kLocalSpinLimit = 1u << 20;   // waits inside the CTA (ring, producer hand-off)
 constexpr int kCountShift = 54;
@@ -654,6 +655,21 @@ __device__ __forceinline__ unsigned w_stream(const PersistGroup* gp, const float
     in[i][2] = pack2(b.x, b.y);
     in[i][3] = pack2(b.z, b.w);
   }
+  // thread i owns row i of this CTA's rows (all maps, in order): its y so far (the image row,
+  // written by another CTA and visible by now) is fetched while the stream runs
+  float* yp = nullptr;
+  float yold = 0.f;
+  {
+    int yb = 0;
+#pragma unroll 1
+    for (int j = 0; j < n_maps; ++j) {
+      const int dout = gp->off[j + 1] - gp->off[j], rows = gp->w_rows[j];
+      const int live = max(min(rows, dout - cta * rows), 0);
+      if (tid >= yb && tid < yb + live) yp = y + gp->off[j] + cta * rows + (tid - yb);
+      yb += live;
+    }
+    if (yp && !dense) yold = __ldcg(yp);
+  }
   int ybase = 0, pi = 0;   // rows of the maps before this one; pieces of this stream so far
   tr.mark(10);
 #pragma unroll 1
@@ -682,25 +698,12 @@ __device__ __forceinline__ unsigned w_stream(const PersistGroup* gp, const float
   }
   if (!ok && !*abort) fail_at(status, misc, 3);
   csync();
-  // rows back to y: the same walk over the maps; the warps' partial sums in warp order
-  {
-    int yb = 0;
+  // rows back to y: the warps' partial sums in warp order, onto the value fetched at the start
+  if (ok && yp) {
+    float acc = 0.f;
 #pragma unroll 1
-    for (int j = 0; j < n_maps; ++j) {
-      const int dout = gp->off[j + 1] - gp->off[j], rows = gp->w_rows[j];
-      const int live = min(rows, dout - cta * rows);
-      if (ok) {
-#pragma unroll 1
-        for (int i = tid; i < live; i += kNC) {
-          float acc = 0.f;
-#pragma unroll 1
-          for (int q = 0; q < nw; ++q) acc += s_part[q * kPersistMaxWRows + yb + i];
-          float* yp = y + gp->off[j] + cta * rows + i;
-          *yp = dense ? acc : (__ldcg(yp) + acc);
-        }
-      }
-      yb += max(live, 0);
-    }
+    for (int q = 0; q < nw; ++q) acc += s_part[q * kPersistMaxWRows + tid];
+    *yp = yold + acc;
   }
   csync();   // the partial sums may be overwritten by the next stream
   tr.mark(13);
@@ -942,6 +945,11 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     // the descriptors of the phase after the next: requested now, stored before the barrier that ends the exchange
     const int g_stage = t + 2 < p.n_phases ? plan[t + 2].gi0 : 0, n_stage = t + 2 < p.n_phases ? plan[t + 2].len : 0;
     const uint32_t desc_word = desc_load(g_stage, n_stage);
+    // (warp 1, lanes 7 and 8) the arrival counter that guards this tick's gated residual of
+    // group lane - 7 of phase t - 2: the address now, the wait with the exchange
+    const unsigned* bar_pp = nullptr;
+    if (warp == 1 && (lane == 7 || lane == 8) && t >= 2 && (mask_pp & (1u << (lane - 7))))
+      bar_pp = p.groups[plan[t - 2].gi0 + (lane - 7)].bar + 2 + parity;
 
     // ---- a dense group among dense groups (the dense baseline): nothing of the exchange
     //      machinery has work in this tick.  Post the (empty) decision on the previous phase
@@ -1183,6 +1191,9 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       const PersistGroup& gs = desc(g_p + (u & 1));   // read only when `live_u`
       const bool w_x2 = gsi && lane == 0, w_r2 = settle && (lane & 1);
       const bool w_thr = (settle && !(lane & 1)) || (cta == 0 && lane >= 5 && lane <= 6 && live_u);
+      // lanes 7, 8: the arrivals before the gated residual this tick streams (phase t - 2, group
+      // lane - 7): every CTA has made its r and image rows visible (they arrived a tick ago)
+      const bool w_bar = bar_pp != nullptr;
       const unsigned long long* wp = w_x2   ? acc + k
                                      : w_r2 ? gs.acc + (size_t)parity * (gs.k + 4) + gs.k + 2
                                             : gs.pub + (lane <= 4 ? 1 : 0);
@@ -1196,6 +1207,8 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
           w = ld_relaxed_u64(wp);
           mine = w_thr ? (unsigned)(w >> 63) == tag
                        : (unsigned)((w + (kOne >> 1)) >> kCountShift) == want;
+        } else if (w_bar) {
+          mine = ld_relaxed_u32(bar_pp) >= (unsigned)G;
         }
         done = __all_sync(0xffffffffu, mine);
         if (!done && (++it > p.spin_limit || ((it & 1023u) == 0 && *abort))) {
@@ -1203,6 +1216,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
           break;
         }
       }
+      if (w_bar) __threadfence();   // acquire: the barrier below hands the visibility on to the CTA
       if (w_x2) {
         const long long val = (long long)(w - ((unsigned long long)n_contrib << kCountShift));
         const double amax = (double)__uint_as_float(misc->amax_bits[t & 1]);
@@ -1393,14 +1407,8 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
           gw = &desc(plan[t].gi);
         }
         if (!gw) continue;
-        if (u < 2) {
-          if (tid == 0) {
-            grid_wait(gw->bar + 2 + parity, (unsigned)G, p, misc);
-            __threadfence();
-          }
-          csync();
-          if (*abort) return;
-        }
+        // (a gated group's r and image rows are visible: warp 1 waited for every CTA's arrival
+        // during this tick's exchange)
         const float* src = u < 2 ? gw->r
                                  : gw->x + (long long)slot_io * gw->x_step_stride + (size_t)p.token * gw->d;
         tr.mark(9);
