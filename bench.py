@@ -30,7 +30,7 @@ METRIC = "decode tokens/s at GPT-J shapes, k=256, eps=0.05 (effective weight GB/
 NOMINAL_HBM_GBS = 8000.0
 # dram bytes (read+write) per algorithmic byte of k_decode_step, from an ncu capture of an
 # 8-layer case (traffic grows in proportion to the layers: every layer has its own weights)
-NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.02
+NCU_TRAFFIC_PER_ALGORITHMIC_BYTE = 1.014
 MIN_TIMED_SECONDS = 0.3     # the timed repeats together last at least this long
 MIN_REPEATS = 3
 FALLBACK_HBM_GBS = 6650.0
