@@ -615,6 +615,73 @@ def test_persistent_groups_of_different_rank_in_one_stack():
         assert 0 < gate.sum() < n_steps
 
 
+W_STREAM_SHAPES = [                 # (d, d_out): every geometry of the W stream
+    (768, (1000, 72)),              # one warp per piece, ragged last CTAs, a map with fewer rows than CTAs
+    (4096, (608, 296)),             # teams of four warps, two rows of W per pass
+    (8192, (304,)),                 # pieces of two rows, one team of eight warps
+    (10240, (152,)),                # pieces of one row, four vectors per lane
+    (16384, (296, 8)),              # pieces of one row, five vectors per lane, a map of eight rows
+]
+
+
+def test_persistent_dense_stack_every_w_stream_geometry():
+    """A stack of dense-baseline groups only (the ticks that skip the exchange machinery and ask
+    the next group's input into the L2), one group per geometry of the W stream, against the
+    fp64 product."""
+    g = G()
+    n_steps = 3
+    layers, xs, mats = [], [], []
+    for i, (d, d_out) in enumerate(W_STREAM_SHAPES):
+        Ws = [S.gen_weight(o, d, 5100 + 10 * i + j) for j, o in enumerate(d_out)]
+        x = torch.randn((n_steps, d), generator=torch.Generator().manual_seed(5200 + i))
+        layers.append(g.Layer([W.cuda() for W in Ws], None, 0.0, max_tokens=1, flags=g.GSI_FLAG_DENSE))
+        xs.append(x.cuda().contiguous())
+        mats.append((x, Ws))
+    stack = g.Stack(layers, mode=2)
+    stack.bind(xs, n_steps=n_steps)
+    assert stack.is_persistent()
+    ys = [[] for _ in mats]
+    for s in range(n_steps):
+        stack.step()
+        torch.cuda.synchronize()
+        for i, y in enumerate(stack.ys):
+            ys[i].append(y.cpu().clone())
+    assert stack.status() == 0
+    assert stack.gate_log.cpu().numpy().all()
+    for i, (x, Ws) in enumerate(mats):
+        ref = torch.cat([x.to(torch.float64) @ W.to(torch.float64).T for W in Ws], dim=1).numpy()
+        got = torch.cat(ys[i]).numpy()
+        assert got.shape == ref.shape
+        assert np.max(np.abs(got - ref)) <= 2e-5 * np.max(np.abs(ref)), W_STREAM_SHAPES[i]
+
+
+def test_persistent_gated_residual_every_w_stream_geometry():
+    """The same geometries through the gated residual (eps = 0 gates every token, so every
+    group streams its W two ticks after its projection), against the oracle."""
+    g = G()
+    n_steps = 3
+    layers, xs, mats = [], [], []
+    for i, (d, d_out) in enumerate(W_STREAM_SHAPES):
+        x, P, Ws = make_small(d, 64, d_out, n_steps, seed=5300 + 20 * i)
+        layers.append(g.Layer([W.cuda() for W in Ws], P.cuda(), 0.0, max_tokens=1))
+        xs.append(x.cuda().contiguous())
+        mats.append((x, P, Ws))
+    stack = g.Stack(layers, mode=2)
+    stack.bind(xs, n_steps=n_steps)
+    assert stack.is_persistent()
+    ys = [[] for _ in mats]
+    for s in range(n_steps):
+        stack.step()
+        torch.cuda.synchronize()
+        for i, y in enumerate(stack.ys):
+            ys[i].append(y.cpu().clone())
+    assert stack.status() == 0
+    for i, (x, P, Ws) in enumerate(mats):
+        gate = stack.gate_log[:, i, 0].cpu().numpy()
+        assert gate.all()
+        compare_group(x, P, Ws, 0.0, torch.cat(ys[i]).numpy(), gate, stack.rho_log[:, i, 0].cpu().numpy())
+
+
 def test_persistent_nonfinite_token():
     g = G()
     x, P, Ws = make_small(256, 64, (64,), 3, seed=41)
