@@ -559,3 +559,25 @@ def test_F4_fp8_image_scales_codes_and_error_bound():
     fast = a["gate"] == 0
     if fast.any():
         np.testing.assert_allclose(a["y"][0][fast], (g @ M0.T)[fast], rtol=1e-12, atol=1e-14)
+
+
+def test_F5_fp8_image_output_error_is_bounded_against_the_unquantised_layer():
+    """y with the FP8 image differs from y with the exact image by at most
+    sum_j |Mq_ij - M_ij| |g_j|, and every |Mq_ij - M_ij| is at most 2^-4 |bf16(M_ij)| (normal
+    codes) or scale * 2^-10 (subnormal codes) plus the BF16 rounding 2^-9 |M_ij|."""
+    rng = np.random.default_rng(21)
+    Wb, W, P_store, P, q, x = rand_problem(rng, 64, 128, 32, 6)
+    a = O.forward(x, P_store, 0.05, [Wb])
+    b = O.forward(x, P_store, 0.05, [Wb], fp8_image=True)
+    np.testing.assert_array_equal(a["gate"], b["gate"])          # the gate does not see the image
+    M = O.image(Wb, P_store)
+    qz = O.quantise_image_e4m3(M)
+    per_entry = np.maximum(2.0 ** -4 * np.abs(M) * (1 + 2.0 ** -8), qz["scales"].astype(np.float64)[:, None] * 2.0 ** -10) \
+        + 2.0 ** -9 * np.abs(M)
+    assert np.all(np.abs(qz["Mq"] - M) <= per_entry)
+    bound = np.abs(a["g"]) @ per_entry.T                          # [T][o]
+    diff = np.abs(b["y"][0] - a["y"][0])
+    assert np.all(diff <= bound * (1 + 1e-12) + 1e-300)
+    assert diff.max() > 0                                          # the quantisation is visible
+    # and in the aggregate it is a few percent of ||y||_inf, not more (3 mantissa bits)
+    assert diff.max() <= 0.05 * np.abs(a["y"][0]).max()
