@@ -327,7 +327,8 @@ class Stack:
                                   _stream_ptr(stream)), "gsi_stack_bind")
 
     def set_trace(self, on: bool = True):
-        """Per-section SM-cycle counters of CTA 0 (persistent launch only)."""
+        """Per-section SM-cycle counters, one row per CTA (persistent launch only); the
+        sections are listed at gsi_stack_set_trace in the header."""
         self.trace = torch.zeros((256, 16), dtype=torch.int64, device=self.device) if on else None
         _check(lib.gsi_stack_set_trace(self.handle, self.trace.data_ptr() if on else None),
                "gsi_stack_set_trace")

@@ -682,6 +682,44 @@ def test_persistent_gated_residual_every_w_stream_geometry():
         compare_group(x, P, Ws, 0.0, torch.cat(ys[i]).numpy(), gate, stack.rho_log[:, i, 0].cpu().numpy())
 
 
+def test_persistent_trace_counters_do_not_change_results():
+    """Tracing (per-CTA cycle counters per section of a tick) is an observer: the outputs of a
+    traced step are bit-identical to an untraced one, the counters of the sections that ran are
+    non-zero (the W-stream sections only once a group has fired), and switching it off stops them."""
+    g = G()
+    n_steps = 4
+    x, P, Ws = make_small(2048, 128, (1024, 512), n_steps, seed=6100, noise=0.002, outlier_every=2)
+    lay = g.Layer([W.cuda() for W in Ws], P.cuda(), 0.05, max_tokens=1)
+    stack = g.Stack([lay], mode=2)
+    stack.bind([x.cuda().contiguous()], n_steps=n_steps)
+    plain = []
+    for s in range(n_steps):
+        stack.step()
+        torch.cuda.synchronize()
+        plain.append(stack.ys[0].cpu().clone())
+    gate = stack.gate_log[:, 0, 0].cpu().numpy().copy()
+    assert 0 < gate.sum() < n_steps
+    tr = stack.set_trace(True)
+    stack.seek(0)
+    traced = []
+    for s in range(n_steps):
+        stack.step()
+        torch.cuda.synchronize()
+        traced.append(stack.ys[0].cpu().clone())
+    assert stack.status() == 0
+    for a, b in zip(plain, traced):
+        assert torch.equal(a, b)
+    assert np.array_equal(gate, stack.gate_log[:, 0, 0].cpu().numpy())
+    T = tr.cpu().numpy()[:torch.cuda.get_device_properties(0).multi_processor_count]   # one row per CTA = per SM
+    assert T.shape[1] == 16 and (T[:, [0, 2, 3, 4, 5, 8]] > 0).all()   # barrier, pass 1, conversion, exchange, residual, image rows
+    assert (T[:, [10, 13]] > 0).all() and (T[0, 10:14] > 0).all()      # a group fired: input share, wait, arithmetic, sums (the last CTAs own no rows of W)
+    stack.set_trace(False)
+    before = tr.clone()
+    stack.step()
+    torch.cuda.synchronize()
+    assert torch.equal(before, tr)
+
+
 def test_persistent_nonfinite_token():
     g = G()
     x, P, Ws = make_small(256, 64, (64,), 3, seed=41)
