@@ -156,10 +156,20 @@ struct gsi_stack {
   // the stack's own, forked from and joined to the caller's stream by events
   cudaStream_t aux = nullptr;
   cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+  // batched steps: the chains of small kernels (projection, residual, gate, image) run on a
+  // stream of the stack's own with the highest priority, the gated-residual contractions stay
+  // on the caller's stream: a contraction is ordered behind its group's gate by an event and
+  // runs beside the chains of the groups that follow (inputs are staged before the step)
+  cudaStream_t front_stream = nullptr;
+  cudaEvent_t ev_resid = nullptr, ev_front_fork = nullptr, ev_front_join = nullptr;
   ~gsi_stack() {
     if (ev_fork) cudaEventDestroy(ev_fork);
     if (ev_join) cudaEventDestroy(ev_join);
     if (aux) cudaStreamDestroy(aux);
+    if (ev_resid) cudaEventDestroy(ev_resid);
+    if (ev_front_fork) cudaEventDestroy(ev_front_fork);
+    if (ev_front_join) cudaEventDestroy(ev_front_join);
+    if (front_stream) cudaStreamDestroy(front_stream);
   }
 };
 
@@ -580,9 +590,24 @@ gsi_status_t gsi_stack_bind(gsi_stack_t s, const gsi_stack_io_t* io, int n_steps
   if (!s->persistent && !s->aux) {
     bool any = false;
     for (char c : s->pair_first) any = any || c;
-    if (any && (cudaStreamCreateWithFlags(&s->aux, cudaStreamNonBlocking) != cudaSuccess ||
+    int least = 0, greatest = 0;
+    if (any && (cudaDeviceGetStreamPriorityRange(&least, &greatest) != cudaSuccess ||
+                cudaStreamCreateWithPriority(&s->aux, cudaStreamNonBlocking, greatest) != cudaSuccess ||
                 cudaEventCreateWithFlags(&s->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
                 cudaEventCreateWithFlags(&s->ev_join, cudaEventDisableTiming) != cudaSuccess))
+      return GSI_ERR_CUDA;
+  }
+  if (!s->persistent && !s->front_stream) {
+    bool any = false;   // some group takes the tensor-core front end at this batch
+    for (const gsi_layer* h : s->groups)
+      any = any || (h->has_tm && h->gp.front_min_tokens > 0 && s->B >= h->gp.front_min_tokens &&
+                    !(h->desc.flags & (GSI_FLAG_DENSE | GSI_FLAG_STATIC_PROJECTION)));
+    int least = 0, greatest = 0;
+    if (any && (cudaDeviceGetStreamPriorityRange(&least, &greatest) != cudaSuccess ||
+                cudaStreamCreateWithPriority(&s->front_stream, cudaStreamNonBlocking, greatest) != cudaSuccess ||
+                cudaEventCreateWithFlags(&s->ev_resid, cudaEventDisableTiming) != cudaSuccess ||
+                cudaEventCreateWithFlags(&s->ev_front_fork, cudaEventDisableTiming) != cudaSuccess ||
+                cudaEventCreateWithFlags(&s->ev_front_join, cudaEventDisableTiming) != cudaSuccess))
       return GSI_ERR_CUDA;
   }
   if (s->persistent) {
@@ -728,6 +753,15 @@ static gsi_status_t stack_enqueue(gsi_stack_t s, bool use_counter, gsi_stream_t 
     }
     return GSI_OK;
   }
+  // fs: the stream the chains of small kernels run on
+  cudaStream_t fs = stream;
+  ResidualLane lane{stream, s->ev_resid, false};
+  if (s->front_stream) {
+    if (cudaEventRecord(s->ev_front_fork, stream) != cudaSuccess ||
+        cudaStreamWaitEvent(s->front_stream, s->ev_front_fork, 0) != cudaSuccess)
+      return GSI_ERR_CUDA;
+    fs = s->front_stream;
+  }
   auto enqueue_group = [&](int i, cudaStream_t st) -> bool {
     gsi_layer* h = s->groups[i];
     IoRef io{};
@@ -739,26 +773,30 @@ static gsi_status_t stack_enqueue(gsi_stack_t s, bool use_counter, gsi_stream_t 
     io.n_steps = s->n_steps;
     io.x_step_stride = (long long)s->B * h->desc.d;
     io.log_step_stride = (long long)G * s->B;
-    h->last_stream = stream;   // the join below puts the pair's work in the caller's stream order
-    return launch_generic_forward(h->gp, h->has_tm ? &h->tm : nullptr, io, s->B, st, nullptr) ==
-           cudaSuccess;
+    h->last_stream = stream;   // the joins below put all of the step's work in the caller's stream order
+    return launch_generic_forward(h->gp, h->has_tm ? &h->tm : nullptr, io, s->B, st, nullptr,
+                                  s->front_stream ? &lane : nullptr) == cudaSuccess;
   };
   for (int i = 0; i < G; ++i) {
     if (s->aux && i + 1 < G && s->pair_first[i]) {
       // groups i and i+1 do not read each other's outputs: two chains of dependent launches
       // side by side (under stream capture this becomes a fork and a join in the graph)
-      if (cudaEventRecord(s->ev_fork, stream) != cudaSuccess ||
+      if (cudaEventRecord(s->ev_fork, fs) != cudaSuccess ||
           cudaStreamWaitEvent(s->aux, s->ev_fork, 0) != cudaSuccess)
         return GSI_ERR_CUDA;
-      if (!enqueue_group(i, stream) || !enqueue_group(i + 1, s->aux)) return GSI_ERR_CUDA;
+      if (!enqueue_group(i, fs) || !enqueue_group(i + 1, s->aux)) return GSI_ERR_CUDA;
       if (cudaEventRecord(s->ev_join, s->aux) != cudaSuccess ||
-          cudaStreamWaitEvent(stream, s->ev_join, 0) != cudaSuccess)
+          cudaStreamWaitEvent(fs, s->ev_join, 0) != cudaSuccess)
         return GSI_ERR_CUDA;
       ++i;
       continue;
     }
-    if (!enqueue_group(i, stream)) return GSI_ERR_CUDA;
+    if (!enqueue_group(i, fs)) return GSI_ERR_CUDA;
   }
+  if (s->front_stream &&   // the chains join the caller's stream, which holds the contractions
+      (cudaEventRecord(s->ev_front_join, fs) != cudaSuccess ||
+       cudaStreamWaitEvent(stream, s->ev_front_join, 0) != cudaSuccess))
+    return GSI_ERR_CUDA;
   if (use_counter && launch_advance_step(s->step, stream) != cudaSuccess) return GSI_ERR_CUDA;
   return GSI_OK;
 }

@@ -209,8 +209,19 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t s
 
 struct TmaMaps;   // tensor maps of the layer's matrices (null when no tensor-core path is on)
 
+// A second stream for the gated-residual contraction of batched calls: the contraction of a
+// group is ordered behind that group's residual/gate kernel by the event and may run beside the
+// projection of the groups that follow (their inputs are staged before the step); the caller
+// joins the stream back at the end of the step.
+struct ResidualLane {
+  cudaStream_t stream;
+  cudaEvent_t ev;
+  bool used;
+};
+
 cudaError_t launch_generic_forward(const GroupParams& g, const TmaMaps* tm, const IoRef& io,
-                                   int n_tokens, cudaStream_t stream, int* n_launches);
+                                   int n_tokens, cudaStream_t stream, int* n_launches,
+                                   ResidualLane* lane = nullptr);
 cudaError_t launch_advance_step(int* step, cudaStream_t stream);
 // One token on CUDA cores: c, r = x - P c into g.r (x may be g.r itself), rho into
 // g.rho_scratch[0] (or io.rho), gate byte, fired list.  No image product.

@@ -380,7 +380,7 @@ cudaError_t dispatch_vpl(const GroupParams& g, const IoRef& io, int n_tokens, cu
 }  // namespace
 
 cudaError_t launch_generic_forward(const GroupParams& g, const TmaMaps* tm, const IoRef& io,
-                                   int n_tokens, cudaStream_t st, int* n_launches) {
+                                   int n_tokens, cudaStream_t st, int* n_launches, ResidualLane* lane) {
   int dummy = 0;
   if (!n_launches) n_launches = &dummy;
   int grid = (g.O + kWarps - 1) / kWarps;
@@ -403,7 +403,15 @@ cudaError_t launch_generic_forward(const GroupParams& g, const TmaMaps* tm, cons
   if (!(g.flags & GSI_FLAG_STATIC_PROJECTION)) {
     if (front) {
       // every gated token goes through the tensor-core contraction; r is in rb already
-      e = launch_residual_gemm_tc(g, *tm, io, 1, true, n_tokens, st, n_launches);
+      cudaStream_t sr = st;
+      if (lane) {   // behind this group's gate, beside the next groups' projections
+        if ((e = cudaEventRecord(lane->ev, st)) != cudaSuccess ||
+            (e = cudaStreamWaitEvent(lane->stream, lane->ev, 0)) != cudaSuccess)
+          return e;
+        sr = lane->stream;
+        lane->used = true;
+      }
+      e = launch_residual_gemm_tc(g, *tm, io, 1, true, n_tokens, sr, n_launches);
       if (e != cudaSuccess) return e;
     } else {
       k_stream_gemv<false><<<grid, kThreads, 0, st>>>(g, io, n_tokens);
