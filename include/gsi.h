@@ -251,6 +251,17 @@ gsi_status_t gsi_destroy(gsi_handle_t h);
  * Stack driver: one decode step = every group of every layer, in order, on
  * one stream (Section 1: the method is applied to all linear maps of all
  * layers).  Groups keep their own handles; the stack only chains them.
+ *
+ * Contract on inputs and order: the inputs x of ALL groups for a step are in
+ * device memory before the step is enqueued (gsi_stack_bind).  Groups start in
+ * the given order and each group's own chain (projection, residual, gate,
+ * image, gated residual) is Algorithm 1, but consecutive groups overlap: a
+ * group's gate may be settled, and its W r added, while later groups already
+ * project their inputs (the persistent kernel reads a group's x one phase
+ * ahead and settles a gate one phase later; batched stacks run the gated
+ * residual contraction of a group beside the kernels of the groups after it).
+ * Every y, gate byte and rho of a step is final when the step's work has
+ * completed in the order of `stream`, not earlier.
  * ------------------------------------------------------------------------ */
 
 typedef struct {
