@@ -615,38 +615,39 @@ __device__ __forceinline__ void w_piece(const uint4* first, int rvec, int rows_p
 // entry, the return value the one after the stream; a wait that gave up sets the abort flag.
 // Inlined at its two call sites (an out-of-line call makes the tick loop keep its state in
 // local memory); both sit where little of the tick's state is alive.
-__device__ __forceinline__ unsigned w_stream(const PersistGroup* gp, const float* src, float* y, bool dense,
-                                          unsigned char* smem, unsigned n, int* status, bool traced) {
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kOffBar);
-  uint64_t* empty = full + kNB;
-  const unsigned* s_off = reinterpret_cast<const unsigned*>(smem + kOffOff);
-  unsigned char* ring = smem + kOffRing;
-  float* s_part = reinterpret_cast<float*>(smem + kOffYacc);
-  Misc* misc = reinterpret_cast<Misc*>(smem + kOffMisc);
-  volatile int* abort = &misc->abort;
-  const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-  const int cta = blockIdx.x;
-  Trace tr;
-  tr.acc = (traced && tid == 0) ? reinterpret_cast<unsigned long long*>(smem + kOffTrace) : nullptr;
-  tr.t = clock64();
-  const int d = gp->d, pr = gp->w_pr, n_maps = gp->n_maps;
-  const int rvec = d >> 3;                                   // 16-byte vectors per row
-  const int vpl = rvec > 4 * kNC ? 5 : 4;
-  const int nw = (rvec + 32 * vpl - 1) / (32 * vpl);         // warps of a team
-  const int T = kNW / nw;                                    // teams
-  const int team = warp / nw, wi = warp - team * nw;
-  const bool active = team < T;
-  const int v_lo = min(rvec, wi * 32 * vpl), v_hi = min(rvec, v_lo + 32 * vpl);   // this warp's vectors of every row
-  const int nvalid = (v_hi - v_lo - lane + 31) >> 5;         // how many of this lane's vectors exist
-  const uint32_t release_n = wi == 0 ? (uint32_t)(kNW - nw + 1) : 1u;   // a team's first warp also arrives for all other warps
-  bool ok = true;
-  // this lane's share of the input: vectors v_lo + lane + 32 i
-  unsigned long long in[kWVecMax][4];
+// How the consumer warps share a W stream of input width d.
+struct WGeo {
+  int d, pr, n_maps, rvec, vpl, nw, T, team, wi, v_lo, v_hi, nvalid;
+  bool active;
+  uint32_t release_n;
+};
+__device__ __forceinline__ WGeo w_geometry(const PersistGroup* gp) {
+  const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+  WGeo q;
+  q.d = gp->d;
+  q.pr = gp->w_pr;
+  q.n_maps = gp->n_maps;
+  q.rvec = q.d >> 3;                                         // 16-byte vectors per row
+  q.vpl = q.rvec > 4 * kNC ? 5 : 4;
+  q.nw = (q.rvec + 32 * q.vpl - 1) / (32 * q.vpl);           // warps of a team
+  q.T = kNW / q.nw;                                          // teams
+  q.team = warp / q.nw;
+  q.wi = warp - q.team * q.nw;
+  q.active = q.team < q.T;
+  q.v_lo = min(q.rvec, q.wi * 32 * q.vpl);                   // this warp's vectors of every row
+  q.v_hi = min(q.rvec, q.v_lo + 32 * q.vpl);
+  q.nvalid = (q.v_hi - q.v_lo - lane + 31) >> 5;             // how many of this lane's vectors exist
+  q.release_n = q.wi == 0 ? (uint32_t)(kNW - q.nw + 1) : 1u; // a team's first warp also arrives for all other warps
+  return q;
+}
+// This lane's share of the input: vectors v_lo + lane + 32 i.
+__device__ __forceinline__ void w_load_in(const WGeo& q, const float* src, unsigned long long (&in)[kWVecMax][4]) {
+  const int lane = threadIdx.x & 31;
 #pragma unroll
   for (int i = 0; i < kWVecMax; ++i) {
-    const int v = v_lo + lane + 32 * i;
+    const int v = q.v_lo + lane + 32 * i;
     float4 a = make_float4(0.f, 0.f, 0.f, 0.f), b = a;
-    if (active && v < v_hi) {
+    if (q.active && v < q.v_hi) {
       a = __ldcg(reinterpret_cast<const float4*>(src) + 2 * v);
       b = __ldcg(reinterpret_cast<const float4*>(src) + 2 * v + 1);
     }
@@ -655,6 +656,26 @@ __device__ __forceinline__ unsigned w_stream(const PersistGroup* gp, const float
     in[i][2] = pack2(b.x, b.y);
     in[i][3] = pack2(b.z, b.w);
   }
+}
+
+__device__ __forceinline__ unsigned w_run(const PersistGroup* gp, const WGeo& q,
+                                          const unsigned long long (&in)[kWVecMax][4], float* y, bool dense,
+                                          unsigned char* smem, unsigned n, int* status, bool traced) {
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + kOffBar);
+  uint64_t* empty = full + kNB;
+  const unsigned* s_off = reinterpret_cast<const unsigned*>(smem + kOffOff);
+  unsigned char* ring = smem + kOffRing;
+  float* s_part = reinterpret_cast<float*>(smem + kOffYacc);
+  Misc* misc = reinterpret_cast<Misc*>(smem + kOffMisc);
+  volatile int* abort = &misc->abort;
+  const int tid = threadIdx.x, lane = tid & 31;
+  const int cta = blockIdx.x;
+  Trace tr;
+  tr.acc = (traced && tid == 0) ? reinterpret_cast<unsigned long long*>(smem + kOffTrace) : nullptr;
+  tr.t = clock64();
+  const int pr = q.pr, n_maps = q.n_maps, rvec = q.rvec, nw = q.nw, T = q.T, team = q.team, wi = q.wi;
+  const bool active = q.active;
+  bool ok = true;
   // thread i owns row i of this CTA's rows (all maps, in order): its y so far (the image row,
   // written by another CTA and visible by now) is fetched while the stream runs
   float* yp = nullptr;
@@ -685,12 +706,12 @@ __device__ __forceinline__ unsigned w_stream(const PersistGroup* gp, const float
       if (ok && !mbar_wait(&full[slot], ph, abort)) ok = false;
       tr.mark(11);
       if (ok) {
-        const uint4* piece = reinterpret_cast<const uint4*>(ring + s_off[slot]) + v_lo + lane;
+        const uint4* piece = reinterpret_cast<const uint4*>(ring + s_off[slot]) + q.v_lo + lane;
         float* part = s_part + wi * kPersistMaxWRows + ybase + r0;
         uint64_t* eb = &empty[slot];
-        if (vpl == 5) w_piece<5, 1>(piece, rvec, rows_p, nvalid, in, part, eb, release_n);
-        else if (pr >= 2) w_piece<4, 2>(piece, rvec, rows_p, nvalid, in, part, eb, release_n);
-        else w_piece<4, 1>(piece, rvec, rows_p, nvalid, in, part, eb, release_n);
+        if (q.vpl == 5) w_piece<5, 1>(piece, rvec, rows_p, q.nvalid, in, part, eb, q.release_n);
+        else if (pr >= 2) w_piece<4, 2>(piece, rvec, rows_p, q.nvalid, in, part, eb, q.release_n);
+        else w_piece<4, 1>(piece, rvec, rows_p, q.nvalid, in, part, eb, q.release_n);
       }
       tr.mark(12);
     }
@@ -708,6 +729,16 @@ __device__ __forceinline__ unsigned w_stream(const PersistGroup* gp, const float
   csync();   // the partial sums may be overwritten by the next stream
   tr.mark(13);
   return n;
+}
+
+
+// Geometry, input share and stream in one go.
+__device__ __forceinline__ unsigned w_stream(const PersistGroup* gp, const float* src, float* y, bool dense,
+                                             unsigned char* smem, unsigned n, int* status, bool traced) {
+  const WGeo q = w_geometry(gp);
+  unsigned long long in[kWVecMax][4];
+  w_load_in(q, src, in);
+  return w_run(gp, q, in, y, dense, smem, n, status, traced);
 }
 
 // The statistics warp: the group's max |x| for tick `tt` from the tagged words of all
@@ -951,47 +982,68 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     if (warp == 1 && (lane == 7 || lane == 8) && t >= 2 && (mask_pp & (1u << (lane - 7))))
       bar_pp = p.groups[plan[t - 2].gi0 + (lane - 7)].bar + 2 + parity;
 
-    // ---- a dense group among dense groups (the dense baseline): nothing of the exchange
-    //      machinery has work in this tick.  Post the (empty) decision on the previous phase
-    //      for the producer and go straight to the stream at the end of the tick.  The next
-    //      dense group's input is asked into the L2 meanwhile (the inputs of a stack are
-    //      staged before the step).
+    // ---- a run of dense groups (the dense baseline): nothing of the exchange machinery has
+    //      work in these ticks.  Per tick: post the (empty) decision on the previous phase for
+    //      the producer, stream, close with the grid barrier that keeps a dense stack in model
+    //      order.  The inputs of a stack are staged before the step, so the next group's input
+    //      is asked into the L2 while this group streams, and this CTA's share of it into
+    //      registers while the barrier is waited for.
     const bool plain = dense && !contrib_p && !mask_pp && (t == 0 || plan[t - 1].kind == 2);
     const unsigned mask_stream = mask_pp;   // the gated residuals this tick streams: phase t - 2
     if (plain) {
-      if (pl.zeroer && tid < 2) g.bar[2 * tid + (parity ^ 1u)] = 0u;
-      if (tid == 0 && t >= 1) misc->decision[(t - 1) & 3] = (unsigned)t << 8;
-      desc_store(g_stage, n_stage, desc_word);
-      if (warp == kStatWarp && t + 1 < n_ticks) {
-        const Plan& pn = plan[t + 1];
-        if (pn.kind == 2) {
-          const PersistGroup& gn = desc(pn.gi);
-          const char* xn = reinterpret_cast<const char*>(gn.x + (long long)slot_io * gn.x_step_stride +
-                                                         (size_t)p.token * gn.d);
-          for (int i = lane * 128; i < gn.d * 4; i += 32 * 128)
-            asm volatile("prefetch.global.L2 [%0];" ::"l"(xn + i));
-        } else if (pn.kind == 1) {   // a projected group follows: its statistics, as in every other tick
-          stat_warp_step(smem, t + 1, true, slot_io, p.token, tag);
-          stat_warp_step(smem, t + 1, false, slot_io, p.token, tag);
-          unsigned xw[kXmaxWords];
-          xmax_issue(desc(pn.gi).xmax, pn.n_contrib, xw);
-          xmax_collect(smem, t + 1, tag, p.spin_limit, p.status, xw[0], xw[1], xw[2], xw[3], xw[4]);
+      auto x_of = [&](const PersistGroup& gg) {
+        return gg.x + (long long)slot_io * gg.x_step_stride + (size_t)p.token * gg.d;
+      };
+      unsigned long long in[kWVecMax][4];
+      WGeo q = w_geometry(&g);
+      w_load_in(q, x_of(g), in);
+      uint32_t dword = desc_word;   // descriptors of the phase after the next, requested at the top of the tick
+      int tt = t;
+      for (;;) {
+        const Plan plc = plan[tt];
+        const PersistGroup& gc = desc(plc.gi);
+        const int gs = tt + 2 < p.n_phases ? plan[tt + 2].gi0 : 0, ns = tt + 2 < p.n_phases ? plan[tt + 2].len : 0;
+        if (tt != t) dword = desc_load(gs, ns);
+        if (plc.zeroer && tid < 2) gc.bar[2 * tid + (parity ^ 1u)] = 0u;
+        if (tid == 0 && tt >= 1) misc->decision[(tt - 1) & 3] = (unsigned)tt << 8;
+        const bool more = tt + 1 < n_ticks && plan[tt + 1].kind == 2;
+        if (warp == kStatWarp && tt + 1 < n_ticks) {
+          const Plan& pn = plan[tt + 1];
+          if (pn.kind == 2) {
+            const char* xn = reinterpret_cast<const char*>(x_of(desc(pn.gi)));
+            for (int i = lane * 128; i < desc(pn.gi).d * 4; i += 32 * 128)
+              asm volatile("prefetch.global.L2 [%0];" ::"l"(xn + i));
+          } else if (pn.kind == 1) {   // a projected group follows: its statistics, as in every other tick
+            stat_warp_step(smem, tt + 1, true, slot_io, p.token, tag);
+            stat_warp_step(smem, tt + 1, false, slot_io, p.token, tag);
+            unsigned xw[kXmaxWords];
+            xmax_issue(desc(pn.gi).xmax, pn.n_contrib, xw);
+            xmax_collect(smem, tt + 1, tag, p.spin_limit, p.status, xw[0], xw[1], xw[2], xw[3], xw[4]);
+          }
         }
+        tr.mark(0);
+        n = w_run(&gc, q, in, gc.y + (size_t)p.token * gc.O, true, smem, n, p.status, p.trace != nullptr);
+        if (tr.acc) tr.t = clock64();
+        if (*abort) return;
+        desc_store(gs, ns, dword);   // (their latency ran under the stream)
+        if (tid == 0) red_relaxed_u32(gc.bar + parity, 1u);
+        if (more) {   // in flight while the barrier is waited for
+          const PersistGroup& gn = desc(plan[tt + 1].gi);
+          q = w_geometry(&gn);
+          w_load_in(q, x_of(gn), in);
+        }
+        if (tid == 0) {
+          grid_wait(gc.bar + parity, (unsigned)G, p, misc);
+          if (cta == 0) p.gate_log[((size_t)slot_io * p.log_step_stride + plc.gi) * p.n_tokens + p.token] = 1;
+        }
+        csync();
+        tr.mark(6);
+        if (*abort) return;
+        if (!more) break;
+        ++tt;
       }
+      t = tt;   // the loop's increment moves on to the tick after the run
       mask_pp = 0;
-      tr.mark(0);
-      n = w_stream(&g, g.x + (long long)slot_io * g.x_step_stride + (size_t)p.token * g.d,
-                   g.y + (size_t)p.token * g.O, true, smem, n, p.status, p.trace != nullptr);
-      if (tr.acc) tr.t = clock64();
-      if (*abort) return;
-      if (tid == 0) {
-        red_relaxed_u32(g.bar + parity, 1u);
-        grid_wait(g.bar + parity, (unsigned)G, p, misc);
-        if (cta == 0) p.gate_log[((size_t)slot_io * p.log_step_stride + pl.gi) * p.n_tokens + p.token] = 1;
-      }
-      csync();
-      tr.mark(6);
-      if (*abort) return;
       continue;
     } else {
     // ---- A. this CTA's rows of x have arrived and are in operand form (the statistics warp
