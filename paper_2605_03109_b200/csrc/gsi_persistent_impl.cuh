@@ -101,12 +101,12 @@ constexpr int kOffMisc = 1536;      // scalars
 constexpr int kOffTrace = 1792;     // cycle counters of the trace (16 words)
 constexpr int kOffProd = 1920;      // state of the producer thread (16 bytes)
 constexpr int kOffX = 2048;         // x of this CTA's basis rows, two buffers (kPersistMaxPRows floats each)
-constexpr int kOffXt = kOffX + 2 * kPersistMaxPRows * 4;  // ... as three bf16 terms in A-operand order, two buffers (16 tile rows x 256 B each)
+constexpr int kOffXt = kOffX + 3 * kPersistMaxPRows * 4;  // ... as three bf16 terms in A-operand order, two buffers (16 tile rows x 256 B each)
 constexpr int kOffCb = kOffXt + 2 * 4096;                 // c as three bf16 terms in B-operand order (32 tile columns x 256 B)
 constexpr int kOffFx = kOffCb + 8192;                     // fixed-point partial c and ||x||^2, source of the bulk reduction (514 words)
 constexpr int kOffPlan = kOffFx + 4224;                   // the launch's plan (kPersistMaxTicks records)
 constexpr int kOffDesc = kOffPlan + kPersistMaxTicks * 32;   // 8 group descriptors, 256 B each
-constexpr int kDescSlots = 8;
+constexpr int kDescSlots = 16;
 constexpr int kOffYacc = kOffDesc + kDescSlots * 512;     // W stream: per-warp partial results (kNW x kPersistMaxWRows floats)
 constexpr int kOffRing = ((kOffYacc + kNW * kPersistMaxWRows * 4 + 1023) / 1024) * 1024;
 constexpr int kRingBytes = (232448 - kOffRing) / 1024 * 1024;
@@ -124,6 +124,9 @@ struct Misc {
   double x2;                // ||x||^2 of this phase's group
   float sr[kNW];            // per-warp partial ||r||^2 of this phase
   volatile unsigned decision[4];   // hand-off to the producer: (phase + 1) << 8 | fire mask
+  int r2_cnt;               // warps that have handed in their partial ||r||^2 of the tick's phase
+  volatile int stop[2];     // the abort flag as thread 0 saw it before a barrier (one word per barrier of the tick, so that
+                            // a warp still reading one cannot see the next write): every warp leaves at the same barrier
 };
 static_assert(sizeof(Misc) <= kOffTrace - kOffMisc, "scalars");
 
@@ -180,6 +183,12 @@ __device__ __forceinline__ void bulk_reduce_add_u64(void* gdst, const void* ssrc
 }
 __device__ __forceinline__ void bulk_reduce_wait_read() {
   asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+}
+// Before a thread that issued bulk reductions or asynchronous copies leaves the kernel: all of
+// them complete (a CTA must not retire with such operations in flight).
+__device__ __forceinline__ void async_drain() {
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+  asm volatile("cp.async.wait_all;" ::: "memory");
 }
 __device__ __forceinline__ void cp_async4(void* dst, const void* src) {
   asm volatile("cp.async.ca.shared.global [%0], [%1], 4;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
@@ -376,17 +385,28 @@ __device__ void producer(const PersistParams& p, unsigned char* smem, Misc* misc
   pr.tail_lin = 0;
   volatile int* abort = &misc->abort;
   bool ok = true;
-  // ticks: tick t runs phase t (while there is one) and the gated residuals of phase t - 2;
-  // the work of a tick, in ring order: basis slab, image slab, W pieces of the gated groups
-  // (or the W pieces of a dense group)
+  // ticks: tick t runs the rows of phase t, pass 1 of phase t + 1 and the gated residuals of
+  // phase t - 2; the work of a tick, in ring order (the order in which the consumers give the
+  // chunks back): the basis slab of phase t + 1 for pass 1 (that of the first phase comes before
+  // the first tick), the basis slab of phase t again for its residual rows, the image slab of
+  // phase t, the W pieces of the gated groups (or of a dense group)
   const Plan* plan = reinterpret_cast<const Plan*>(smem + kOffPlan);
   const int n_ticks = p.n_phases + 2;
+  if (plan[0].kind == 1) {
+    const PersistGroup* g0 = p.groups + plan[0].gi;
+    ok = produce_rows(g0->P, g0->k, g0->k * 32, plan[0].p0 >> 4, (plan[0].p0 >> 4) + plan[0].pg, smem);
+  }
 #pragma unroll 1
   for (int t = 0; t < n_ticks && ok; ++t) {
     const Plan& pl = plan[t];
     const PersistGroup* g = p.groups + pl.gi;   // read only when the tick has a group
-    if (pl.kind == 1) {
-      ok = produce_rows(g->P, g->k, g->k * 32, pl.p0 >> 4, (pl.p0 >> 4) + pl.pg, smem);
+    if (t + 1 < p.n_phases && plan[t + 1].kind == 1) {
+      const Plan& pn = plan[t + 1];
+      const PersistGroup* gn = p.groups + pn.gi;
+      ok = produce_rows(gn->P, gn->k, gn->k * 32, pn.p0 >> 4, (pn.p0 >> 4) + pn.pg, smem);
+    }
+    if (ok && pl.kind == 1) {
+      ok = produce_rows(g->P, g->k, g->k * 32, pl.p0 >> 4, (pl.p0 >> 4) + pl.pg, smem);   // once more, for the residual rows
       if (ok)
         ok = produce_rows(g->WP, g->k, persist_image_row_bytes(g->k, g->flags & GSI_FLAG_FP8_IMAGE), pl.o0 >> 4,
                           (pl.o0 >> 4) + pl.og, smem);
@@ -703,7 +723,7 @@ __device__ __forceinline__ unsigned w_run(const PersistGroup* gp, const WGeo& q,
       const unsigned slot = n % kNB, ph = (n / kNB) & 1u;
       ++n;
       if (!active || pi % T != team) continue;
-      if (ok && !mbar_wait(&full[slot], ph, abort)) ok = false;
+      if (ok && !__all_sync(0xffffffffu, mbar_wait(&full[slot], ph, abort))) ok = false;   // (for the warp as a whole)
       tr.mark(11);
       if (ok) {
         const uint4* piece = reinterpret_cast<const uint4*>(ring + s_off[slot]) + q.v_lo + lane;
@@ -798,7 +818,7 @@ __device__ __noinline__ void stat_warp_step(unsigned char* smem, int tt, bool re
   const int lane = threadIdx.x & 31;
   const PersistGroup& gn =
       *reinterpret_cast<const PersistGroup*>(smem + kOffDesc + (pn.gi & (kDescSlots - 1)) * 512);
-  float* sx = reinterpret_cast<float*>(smem + kOffX) + (tt & 1) * kPersistMaxPRows;
+  float* sx = reinterpret_cast<float*>(smem + kOffX) + (tt % 3) * kPersistMaxPRows;
   const int rows = pn.pg * 16;
   if (request) {
     const float* src = gn.x + (long long)slot_io * gn.x_step_stride + (size_t)token * gn.d + pn.p0;
@@ -898,7 +918,8 @@ __device__ __forceinline__ void make_plan(const PersistParams& p, unsigned char*
 // the descriptor.
 template <bool kPairs, int kK>
 __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc) {
-  uint64_t* empty = reinterpret_cast<uint64_t*>(smem + kOffBar) + kNB;
+  uint64_t* full_b = reinterpret_cast<uint64_t*>(smem + kOffBar);
+  uint64_t* empty = full_b + kNB;
   const unsigned* s_off = reinterpret_cast<const unsigned*>(smem + kOffOff);
   unsigned char* ring = smem + kOffRing;
   float* s_xb = reinterpret_cast<float*>(smem + kOffX);
@@ -910,8 +931,9 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
   const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   const int G = gridDim.x, cta = blockIdx.x;
   const int lg = lane >> 2, lt = lane & 3;   // row and column pair of this lane in a tensor-core operand
-  constexpr int kStatWarp = kNW - 1;   // statistics of x and the collection of max|x|; the others run pass 1
-  constexpr int kP1 = kNW - 1;         // warps of pass 1
+  constexpr int kStatWarp = kNW - 1;   // statistics of x and the collection of max|x|
+  constexpr int kP1First = 5;          // warps 0..4 wait for the exchange of the tick's phase ...
+  constexpr int kP1 = kStatWarp - kP1First;   // ... while warps 5..13 run pass 1 of the phase after it
 
   unsigned n = 0;   // chunk sequence number: advances exactly as in producer()
   const int step = p.use_counter ? *p.step : 0;
@@ -937,13 +959,14 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
   };
   // the operand rows / columns beyond the three terms stay zero for the whole launch
   for (int i = tid; i < (2 * 4096 + 8192) / 4; i += kNC) reinterpret_cast<uint32_t*>(smem + kOffXt)[i] = 0u;
-  // the descriptors of the first two phases (descriptors are staged two phases ahead)
+  // the descriptors of the first two phases (descriptors are staged three phases ahead; the
+  // tick before the first phase stages the third)
   {
     const int cnt = plan[0].len + (p.n_phases > 1 ? plan[1].len : 0);
     desc_store(0, cnt, desc_load(0, cnt));
   }
   csync();
-  if (warp == kStatWarp) {   // the first tick's rows of x: nothing ran ahead of it
+  if (warp == kStatWarp) {   // the first phase's rows of x: nothing ran ahead of them
     stat_warp_step(smem, 0, true, slot_io, p.token, tag);
     stat_warp_step(smem, 0, false, slot_io, p.token, tag);
     if (plan[0].kind == 1) {
@@ -954,27 +977,27 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
   }
 
   unsigned mask_pp = 0;          // gates that fired in the phase before the previous one
-  bool contrib_p = false;        // this CTA holds a partial ||r||^2 of the previous phase
-  int e_p = 0;                   // ... scaled by 2^(44 - e_p)
-  unsigned long long* r2word_p = nullptr;
   bool ok = true;
 
 #pragma unroll 1
-  for (int t = 0; t < n_ticks && ok; ++t) {
-    const Plan pl = plan[t];
-    const bool gsi = pl.kind == 1, dense = pl.kind == 2;
+  // Tick t runs the rows of phase t (whose exchange was sent during tick t - 1) and, beside
+  // the wait for that exchange, pass 1 and the send of phase t + 1; tick -1 has only the latter.
+  for (int t = -1; t < n_ticks; ++t) {   // (a warp whose wait gave up stays in step: the CTA leaves together)
+    const Plan pl = t >= 0 ? plan[t] : Plan{};
+    const Plan pf = t + 1 < p.n_phases ? plan[t + 1] : Plan{};   // the phase whose pass 1 runs in this tick
+    const bool gsi = pl.kind == 1, dense = pl.kind == 2, gsi_f = pf.kind == 1;
     const PersistGroup& g = desc(pl.gi);        // read only when the tick has a group
     const int k = gsi ? (kK ? kK : g.k) : 0;
     const int KT = k >> 4;                      // tile columns
     const int pg = pl.pg, og = pl.og, pchunks = pl.pchunks, ochunks = pl.ochunks, gcl = pl.gc_log2;
     const int n_contrib = pl.n_contrib, lc = pl.lc;
     const int len_p = t >= 1 ? plan[t - 1].len : 0, g_p = t >= 1 ? plan[t - 1].gi0 : 0;
-    const float* s_x = s_xb + (t & 1) * kPersistMaxPRows;
+    const float* s_x = s_xb + ((t + 3) % 3) * kPersistMaxPRows;
     unsigned long long* acc = gsi ? g.acc + (size_t)parity * (k + 4) : nullptr;
     const int tp = (t & 1) * 2;
 
-    // the descriptors of the phase after the next: requested now, stored before the barrier that ends the exchange
-    const int g_stage = t + 2 < p.n_phases ? plan[t + 2].gi0 : 0, n_stage = t + 2 < p.n_phases ? plan[t + 2].len : 0;
+    // the descriptors of the phase three ahead: requested now, stored before the barrier that ends the exchange
+    const int g_stage = t + 3 < p.n_phases ? plan[t + 3].gi0 : 0, n_stage = t + 3 < p.n_phases ? plan[t + 3].len : 0;
     const uint32_t desc_word = desc_load(g_stage, n_stage);
     // (warp 1, lanes 7 and 8) the arrival counter that guards this tick's gated residual of
     // group lane - 7 of phase t - 2: the address now, the wait with the exchange
@@ -988,7 +1011,8 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     //      order.  The inputs of a stack are staged before the step, so the next group's input
     //      is asked into the L2 while this group streams, and this CTA's share of it into
     //      registers while the barrier is waited for.
-    const bool plain = dense && !contrib_p && !mask_pp && (t == 0 || plan[t - 1].kind == 2);
+    auto not_gated = [&](int ph) { return ph >= p.n_phases || plan[ph].kind != 1; };
+    const bool plain = dense && !mask_pp && (t == 0 || plan[t - 1].kind == 2) && not_gated(t + 1) && not_gated(t + 2);
     const unsigned mask_stream = mask_pp;   // the gated residuals this tick streams: phase t - 2
     if (plain) {
       auto x_of = [&](const PersistGroup& gg) {
@@ -1002,29 +1026,22 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       for (;;) {
         const Plan plc = plan[tt];
         const PersistGroup& gc = desc(plc.gi);
-        const int gs = tt + 2 < p.n_phases ? plan[tt + 2].gi0 : 0, ns = tt + 2 < p.n_phases ? plan[tt + 2].len : 0;
+        const int gs = tt + 3 < p.n_phases ? plan[tt + 3].gi0 : 0, ns = tt + 3 < p.n_phases ? plan[tt + 3].len : 0;
         if (tt != t) dword = desc_load(gs, ns);
         if (plc.zeroer && tid < 2) gc.bar[2 * tid + (parity ^ 1u)] = 0u;
         if (tid == 0 && tt >= 1) misc->decision[(tt - 1) & 3] = (unsigned)tt << 8;
-        const bool more = tt + 1 < n_ticks && plan[tt + 1].kind == 2;
+        const bool more = tt + 1 < n_ticks && plan[tt + 1].kind == 2 && not_gated(tt + 2) && not_gated(tt + 3);
         if (warp == kStatWarp && tt + 1 < n_ticks) {
           const Plan& pn = plan[tt + 1];
           if (pn.kind == 2) {
             const char* xn = reinterpret_cast<const char*>(x_of(desc(pn.gi)));
             for (int i = lane * 128; i < desc(pn.gi).d * 4; i += 32 * 128)
               asm volatile("prefetch.global.L2 [%0];" ::"l"(xn + i));
-          } else if (pn.kind == 1) {   // a projected group follows: its statistics, as in every other tick
-            stat_warp_step(smem, tt + 1, true, slot_io, p.token, tag);
-            stat_warp_step(smem, tt + 1, false, slot_io, p.token, tag);
-            unsigned xw[kXmaxWords];
-            xmax_issue(desc(pn.gi).xmax, pn.n_contrib, xw);
-            xmax_collect(smem, tt + 1, tag, p.spin_limit, p.status, xw[0], xw[1], xw[2], xw[3], xw[4]);
           }
         }
         tr.mark(0);
         n = w_run(&gc, q, in, gc.y + (size_t)p.token * gc.O, true, smem, n, p.status, p.trace != nullptr);
         if (tr.acc) tr.t = clock64();
-        if (*abort) return;
         desc_store(gs, ns, dword);   // (their latency ran under the stream)
         if (tid == 0) red_relaxed_u32(gc.bar + parity, 1u);
         if (more) {   // in flight while the barrier is waited for
@@ -1035,10 +1052,14 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
         if (tid == 0) {
           grid_wait(gc.bar + parity, (unsigned)G, p, misc);
           if (cta == 0) p.gate_log[((size_t)slot_io * p.log_step_stride + plc.gi) * p.n_tokens + p.token] = 1;
+          misc->stop[1] = *abort;
         }
         csync();
         tr.mark(6);
-        if (*abort) return;
+        if (misc->stop[1]) {   // decided before the barrier: the same for every warp
+      async_drain();
+      return;
+    }
         if (!more) break;
         ++tt;
       }
@@ -1046,150 +1067,144 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       mask_pp = 0;
       continue;
     } else {
-    // ---- A. this CTA's rows of x have arrived and are in operand form (the statistics warp
-    //      saw to it during the previous tick); the bulk reduction of the previous tick has
-    //      read its source
+    // ---- A. the bulk reduction of the previous tick has read its source
     if (lane == 0 || tid == kNC - 1) bulk_reduce_wait_read();   // the lanes that issue bulk reductions
     if (tid == 0) misc->fire[tp] = misc->fire[tp + 1] = 0;
-    if (pl.zeroer) {  // this CTA clears the group's counters for the next launch
+    if (t >= 0 && pl.zeroer) {  // this CTA clears the group's counters for the next launch
       if (gsi) {
 #pragma unroll 1
         for (int j = tid; j < k + 4; j += kNC) g.acc[(size_t)(parity ^ 1u) * (k + 4) + j] = 0ull;
       }
       if (tid < 2) g.bar[2 * tid + (parity ^ 1u)] = 0u;
     }
+    if (tid == 0) misc->stop[0] = *abort;
     csync();
+    if (misc->stop[0]) {   // decided before the barrier: the same for every warp
+      async_drain();
+      return;
+    }
     tr.mark(0);
-    // the statistics warp works one tick ahead: the next phase's rows of x are requested now,
-    // their statistics are published while this phase's exchange is in flight, and the other
-    // CTAs' words are collected during the row passes (the inputs of a stack are pre-staged)
-    if (warp == kStatWarp && t + 1 < n_ticks) stat_warp_step(smem, t + 1, true, slot_io, p.token, tag);
+    // the statistics warp works two ticks ahead: the rows of x of phase t + 2 are requested now,
+    // their statistics are published during this tick, and the other CTAs' words are collected
+    // during the row passes (the inputs of a stack are staged before the step)
+    if (warp == kStatWarp && t + 2 < n_ticks) stat_warp_step(smem, t + 2, true, slot_io, p.token, tag);
 
-    const unsigned n_p0 = n;
-    n += pchunks;
-    // partial c of this warp's tile columns kt = warp * tpw + s: lanes 0..3 hold, after the
-    // folds below, columns 16 kt + 8 m + 2 lane + v in cacc[s][m][v]
-    constexpr int kTpwMax = kK ? (kK / 16 + kP1 - 1) / kP1 : 3;
-    const int tpw = kK ? kTpwMax : (KT + kP1 - 1) / kP1;
-    float cacc[kTpwMax][2][4];
-    if (gsi) {
-      if (warp == kStatWarp) {
-        // (the group's max |x| was collected by this warp during the previous tick)
-      } else {
-        // ---- B. pass 1 on the tensor cores: D[term of x][column j] += X[term][row i] P[i][j];
-        //      the rows of x are the A operand (three terms in rows 0..2), a tile of P, each of
-        //      its four 8 x 8 blocks transposed in registers, is the B operand of two
-        //      instructions (columns 0..7 and 8..15 of the tile)
-        ok = chunks_landed(smem, n_p0, pchunks, abort);
-        tr.mark(1);
+    // ---- B / D. (warps 5..13) pass 1 and the send of phase t + 1, beside the wait for the
+    //      exchange of phase t.  Pass 1 on the tensor cores: D[term of x][column j] +=
+    //      X[term][row i] P[i][j]; the rows of x are the A operand (three terms in rows 0..2), a
+    //      tile of P, each of its four 8 x 8 blocks transposed in registers, is the B operand of
+    //      two instructions.  Then every warp converts its own columns to fixed point and sends
+    //      them off with a bulk reduction of its own into the group's accumulators.
+    // chunk sequence of the tick: the basis slab of phase t + 1 for its pass 1 (given back
+    // before the barrier that ends the exchange), the basis slab of phase t once more for its
+    // residual rows (the second read comes from the L2: the ring is a FIFO, and a slab kept
+    // across the tick boundary would pin everything placed after it), the image slab of phase t
+    const unsigned n_pf = n;
+    if (gsi_f) n += pf.pchunks;
+    const unsigned n_pr = n;
+    if (gsi) n += pchunks;
+    if (gsi_f && warp >= kP1First && warp < kStatWarp) {
+      const PersistGroup& gf = desc(pf.gi);
+      const int kf = kK ? kK : gf.k, KTf = kf >> 4, gclf = pf.gc_log2, wp1 = warp - kP1First;
+      // partial c of this warp's tile columns kt = wp1 * tpw + s: lanes 0..3 hold, after the
+      // folds below, columns 16 kt + 8 m + 2 lane + v in cacc[s][m][v]
+      constexpr int kTpwMax = kK ? (kK / 16 + kP1 - 1) / kP1 : 4;
+      const int tpw = kK ? kTpwMax : (KTf + kP1 - 1) / kP1;
+      float cacc[kTpwMax][2][4];
+      bool okf = chunks_landed(smem, n_pf, pf.pchunks, abort);
 #pragma unroll
-        for (int s3 = 0; s3 < kTpwMax; ++s3)
+      for (int s3 = 0; s3 < kTpwMax; ++s3)
 #pragma unroll
-          for (int m = 0; m < 2; ++m)
+        for (int m = 0; m < 2; ++m)
 #pragma unroll
-            for (int v = 0; v < 4; ++v) cacc[s3][m][v] = 0.f;
-        const unsigned short* xt = s_xt + (t & 1) * 2048;
-        if (ok) {
+          for (int v = 0; v < 4; ++v) cacc[s3][m][v] = 0.f;
+      const unsigned short* xt = s_xt + ((t + 1) & 1) * 2048;
+      if (okf) {
 #pragma unroll 1
-          for (int R = 0; R < pg; ++R) {
-            const uint2 ax = *reinterpret_cast<const uint2*>(xt + (R * 32 + lane) * 4);
-            const uint4 a = make_uint4(ax.x, 0u, ax.y, 0u);
-            const int ci = R >> gcl, rr = R - (ci << gcl);
-            const unsigned char* trow = ring + s_off[(n_p0 + ci) % kNB] + (size_t)rr * KT * 512 + lane * 16;
+        for (int R = 0; R < pf.pg; ++R) {
+          const uint2 ax = *reinterpret_cast<const uint2*>(xt + (R * 32 + lane) * 4);
+          const uint4 a = make_uint4(ax.x, 0u, ax.y, 0u);
+          const int ci = R >> gclf, rr = R - (ci << gclf);
+          const unsigned char* trow = ring + s_off[(n_pf + ci) % kNB] + (size_t)rr * KTf * 512 + lane * 16;
 #pragma unroll
-            for (int s3 = 0; s3 < kTpwMax; ++s3) {
-              const int kt = warp * tpw + s3;
-              if (s3 < tpw && kt < KT) {
-                const uint4 w = *reinterpret_cast<const uint4*>(trow + kt * 512);
-                mma_bf16(cacc[s3][0], a, movmatrix_trans(w.x), movmatrix_trans(w.y));
-                mma_bf16(cacc[s3][1], a, movmatrix_trans(w.z), movmatrix_trans(w.w));
-              }
+          for (int s3 = 0; s3 < kTpwMax; ++s3) {
+            const int kt = wp1 * tpw + s3;
+            if (s3 < tpw && kt < KTf) {
+              const uint4 w = *reinterpret_cast<const uint4*>(trow + kt * 512);
+              mma_bf16(cacc[s3][0], a, movmatrix_trans(w.x), movmatrix_trans(w.y));
+              mma_bf16(cacc[s3][1], a, movmatrix_trans(w.z), movmatrix_trans(w.w));
             }
           }
         }
-        // the three terms of x sit in rows 0..2 = lanes 0-3, 4-7, 8-11: fold them onto lanes 0-3
+      }
+      // the three terms of x sit in rows 0..2 = lanes 0-3, 4-7, 8-11: fold them onto lanes 0-3
 #pragma unroll
-        for (int s3 = 0; s3 < kTpwMax; ++s3)
+      for (int s3 = 0; s3 < kTpwMax; ++s3)
 #pragma unroll
-          for (int m = 0; m < 2; ++m)
+        for (int m = 0; m < 2; ++m)
 #pragma unroll
-            for (int v = 0; v < 2; ++v) {
-              float z = cacc[s3][m][v];
-              z += __shfl_down_sync(0xffffffffu, z, 4) + __shfl_down_sync(0xffffffffu, z, 8);
-              cacc[s3][m][v] = z;
+          for (int v = 0; v < 2; ++v) {
+            float z = cacc[s3][m][v];
+            z += __shfl_down_sync(0xffffffffu, z, 4) + __shfl_down_sync(0xffffffffu, z, 8);
+            cacc[s3][m][v] = z;
+          }
+      if (!okf && !*abort) fail(p, misc, 5);
+      // fixed-point scale: |partial c_j| <= amax * rows * max|P| < 2^e
+      const unsigned amax_f = misc->amax_bits[(t + 1) & 1];
+      const float bound = __uint_as_float(amax_f) * (float)gf.p_rows * gf.pmax;
+      double scale = 0.0;
+      if (amax_f < 0x7f800000u && bound > 0.f && bound < 3.0e38f)
+        scale = pow2d(43 - (max((int)((__float_as_uint(bound) >> 23) & 0xFFu), 1) - 126));
+      if (pf.pg > 0 && wp1 * tpw < KTf) {
+        unsigned long long* acc_f = gf.acc + (size_t)parity * (kf + 4);
+        if (lane < 4) {
+#pragma unroll
+          for (int s3 = 0; s3 < kTpwMax; ++s3) {
+            const int kt = wp1 * tpw + s3;
+            if (s3 < tpw && kt < KTf) {
+#pragma unroll
+              for (int m = 0; m < 2; ++m)
+#pragma unroll
+                for (int v = 0; v < 2; ++v) {
+                  const long long fx = scale != 0.0 ? __double2ll_rn((double)cacc[s3][m][v] * scale) : 0ll;
+                  s_fx[16 * kt + 8 * m + 2 * lane + v] = kOne + (unsigned long long)fx;
+                }
             }
-        if (!ok && !*abort) fail(p, misc, 5);
+          }
+        }
+        __syncwarp();
+        if (lane == 0) {
+          const int c0 = 16 * wp1 * tpw, c1 = min(kf, c0 + 16 * tpw);
+          bulk_reduce_add_u64(acc_f + c0, s_fx + c0, (uint32_t)(c1 - c0) * 8);
+        }
       }
     }
-    tr.mark(2);
-    // the next phase's rows of x travel while this phase runs its exchange (its descriptors
-    // are in place now) ...
+    if (gsi_f && tid == kNC - 1 && pf.pg > 0) {   // ||x||^2 of phase t + 1 over this CTA's rows
+      const PersistGroup& gf = desc(pf.gi);
+      const int kf = kK ? kK : gf.k;
+      const unsigned amax_f = misc->amax_bits[(t + 1) & 1];
+      const double amax = (double)__uint_as_float(amax_f);
+      const float bound = __uint_as_float(amax_f) * (float)gf.p_rows * gf.pmax;
+      const bool fin = amax_f < 0x7f800000u && bound > 0.f && bound < 3.0e38f;
+      const double scale_x2 = fin ? pow2d(43 - exp_above(amax * amax * (double)gf.p_rows)) : 0.0;
+      const long long v = scale_x2 != 0.0 ? __double2ll_rn((double)misc->x2_part[(t + 1) & 1] * scale_x2) : 0ll;
+      s_fx[kf] = kOne + (unsigned long long)v;
+      s_fx[kf + 1] = 0ull;
+      bulk_reduce_add_u64(gf.acc + (size_t)parity * (kf + 4) + kf, s_fx + kf, 16u);
+    }
+    if (warp == kStatWarp && t + 2 < n_ticks) stat_warp_step(smem, t + 2, false, slot_io, p.token, tag);
+    tr.mark(3);
 
-    // ---- D. the exchange: this phase's partial c and ||x||^2 as bulk reductions of
-    //      fixed-point words into the group's accumulators (one per pass-1 warp), the previous
-    //      phase's ||r||^2 as one atomic
+    // the scale of the sums of phase t (sent a tick ago), and whether its token is finite
     bool nonfinite = false;
     double inv_scale = 0.0;
     if (gsi) {
       const unsigned amax_bits = misc->amax_bits[t & 1];
       nonfinite = amax_bits >= 0x7f800000u;
-      const float amax = __uint_as_float(amax_bits);
-      // fixed-point scales: |partial c_j| <= amax * rows * max|P| < 2^e, partial ||x||^2 <= rows * amax^2 < 2^ex
-      double scale = 0.0, scale_x2 = 0.0;
-      const float bound = amax * (float)g.p_rows * g.pmax;
-      if (!nonfinite && bound > 0.f && bound < 3.0e38f) {
-        const int e = max((int)((__float_as_uint(bound) >> 23) & 0xFFu), 1) - 126;
-        scale = pow2d(43 - e);
-        inv_scale = pow2d(e - 43);
-        scale_x2 = pow2d(43 - exp_above((double)amax * (double)amax * (double)g.p_rows));
-      }
-      if (pg > 0) {
-        // every pass-1 warp converts its own columns and sends them off with a bulk reduction
-        // of its own: no barrier of the CTA stands between pass 1 and the exchange
-        if (warp * tpw < KT && warp < kP1) {
-          if (lane < 4) {
-#pragma unroll
-            for (int s3 = 0; s3 < kTpwMax; ++s3) {
-              const int kt = warp * tpw + s3;
-              if (s3 < tpw && kt < KT) {
-#pragma unroll
-                for (int m = 0; m < 2; ++m)
-#pragma unroll
-                  for (int v = 0; v < 2; ++v) {
-                    const long long fx =
-                        scale != 0.0 ? __double2ll_rn((double)cacc[s3][m][v] * scale) : 0ll;
-                    s_fx[16 * kt + 8 * m + 2 * lane + v] = kOne + (unsigned long long)fx;
-                  }
-              }
-            }
-          }
-          __syncwarp();
-          if (lane == 0) {
-            const int c0 = 16 * warp * tpw, c1 = min(k, c0 + 16 * tpw);
-            bulk_reduce_add_u64(acc + c0, s_fx + c0, (uint32_t)(c1 - c0) * 8);
-          }
-        }
-        if (tid == kNC - 1) {
-          const long long v = scale_x2 != 0.0 ? __double2ll_rn((double)misc->x2_part[t & 1] * scale_x2) : 0ll;
-          s_fx[k] = kOne + (unsigned long long)v;
-          s_fx[k + 1] = 0ull;
-          bulk_reduce_add_u64(acc + k, s_fx + k, 16u);
-        }
-      }
+      const float bound = __uint_as_float(amax_bits) * (float)g.p_rows * g.pmax;
+      if (!nonfinite && bound > 0.f && bound < 3.0e38f)
+        inv_scale = pow2d(max((int)((__float_as_uint(bound) >> 23) & 0xFFu), 1) - 126 - 43);
     }
-    if (contrib_p && tid == 32) {
-      float sr = 0.f;   // fixed order: the sum does not depend on which warp finished first
-#pragma unroll
-      for (int w = 0; w < kNW; ++w) sr += misc->sr[w];
-      // at most 2^45 per CTA, so the sum of all CTAs stays below 2^53; a partial that large
-      // (||r||^2 > 2 ||x||^2) fires for every sensible eps
-      double vd = (double)sr * pow2d(44 - e_p);
-      if (!(vd < 35184372088832.0)) vd = 35184372088832.0;
-      if (!(vd >= 0.0)) vd = 0.0;
-      red_add_u64(r2word_p, kOne + (unsigned long long)__double2ll_rn(vd));
-    }
-    if (warp == kStatWarp && t + 1 < n_ticks) stat_warp_step(smem, t + 1, false, slot_io, p.token, tag);
-    tr.mark(3);
 
     // ---- E. wait until every contributing CTA has been added: four warps poll a quarter of
     //      the accumulators of c each (contiguous words, all loads of a lane in flight together,
@@ -1309,10 +1324,22 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
         }
       }
     }
+    if (gsi_f) {   // every warp gives the chunks of pass 1 back (they landed before pass 1 ran)
+#pragma unroll 1
+      for (int c = 0; c < pf.pchunks; ++c) {
+        const unsigned seq = n_pf + c;
+        if (!__all_sync(0xffffffffu, mbar_wait(&full_b[seq % kNB], (seq / kNB) & 1u, abort))) ok = false;
+        if (ok && lane == 0) mbar_arrive(&empty[seq % kNB]);
+      }
+    }
     desc_store(g_stage, n_stage, desc_word);
+    if (tid == 0) misc->stop[1] = *abort;
     csync();
     tr.mark(4);
-    if (*abort) return;
+    if (misc->stop[1]) {   // decided before the barrier: the same for every warp
+      async_drain();
+      return;
+    }
 
     // ---- F. hand the decision to the producer; a gated group's r and image rows must be
     //      visible grid-wide before its W rows are streamed in the next tick: release fence
@@ -1332,8 +1359,8 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     // (this warp then fetches the words of the other CTAs for the next phase: the loads fly
     // during its row units, the check comes after them)
     unsigned xw[kXmaxWords];
-    const bool xmax_next = warp == kStatWarp && t + 1 < n_ticks && plan[t + 1].kind == 1;
-    if (xmax_next) xmax_issue(desc(plan[t + 1].gi).xmax, plan[t + 1].n_contrib, xw);
+    const bool xmax_next = warp == kStatWarp && t + 2 < n_ticks && plan[t + 2].kind == 1;
+    if (xmax_next) xmax_issue(desc(plan[t + 2].gi).xmax, plan[t + 2].n_contrib, xw);
 
     // ---- G / I. the row passes on the tensor cores, one copy of the code for both: part 0 the
     //      residual rows of the basis slab (still in the ring), part 1 the image rows.  A unit
@@ -1347,27 +1374,39 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       const bool image = part == 1;
       const int nchunks = image ? ochunks : pchunks, ngroups = image ? og : pg;
       const int id0 = image ? pg : 0;
-      const unsigned n0 = image ? n : n_p0;
+      const unsigned n0 = image ? n : n_pr;
       const int row_base = image ? pl.o0 : pl.p0, row_end = image ? g.O : g.d;
       float* out = image ? g.y + (size_t)p.token * g.O : g.r;
       const bool f8 = image && (g.flags & GSI_FLAG_FP8_IMAGE);
-      if (image) {
-        n += ochunks;
-        ok = ok && chunks_landed(smem, n0, ochunks, abort);
-        tr.mark(7);
-      }
+      if (image) n += ochunks;
       float sr = 0.f;
       int released = 0;
+      // The chunks of a slab are taken in order: a warp waits for a chunk, runs its units that
+      // lie in it, and gives it back (every warp gives every chunk back once, also those it has
+      // no unit in).  The image slab need not be resident as a whole: its chunks stream through
+      // the space that the basis slab of the next phase leaves.
+      auto pass_chunks = [&](int upto) {   // chunks [released, upto): wait, give back
+#pragma unroll 1
+        for (; released < upto && ok; ++released) {
+          const unsigned seq = n0 + released;
+          // (the outcome is taken for the warp as a whole: lanes must not part ways here)
+          if (!__all_sync(0xffffffffu, mbar_wait(&full_b[seq % kNB], (seq / kNB) & 1u, abort))) ok = false;
+          if (ok && lane == 0) mbar_arrive(&empty[seq % kNB]);
+        }
+      };
       if (ok) {
         int id = warp;
         if (id < id0) id += ((id0 - id + kNW - 1) / kNW) * kNW;
 #pragma unroll 1
-        for (; id < id0 + ngroups; id += kNW) {
+        for (; id < id0 + ngroups && ok; id += kNW) {
           const int R = id - id0;
           const int ci = R >> gcl, rr = R - (ci << gcl);
-          if (lane == 0)
-            for (; released < ci; ++released) mbar_arrive(&empty[(n0 + released) % kNB]);
-          released = ci;
+          pass_chunks(ci);
+          {
+            const unsigned seq = n0 + ci;
+            if (!__all_sync(0xffffffffu, mbar_wait(&full_b[seq % kNB], (seq / kNB) & 1u, abort))) ok = false;
+          }
+          if (!ok) break;
           const unsigned char* cb = reinterpret_cast<const unsigned char*>(s_cb) + lane * 8;
           float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
           float sc_lo = 1.f, sc_hi = 1.f;   // FP8 image: the scales of rows lg and lg + 8
@@ -1422,25 +1461,40 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
             }
           }
         }
-        __syncwarp();
-        if (lane == 0)
-          for (; released < nchunks; ++released) mbar_arrive(&empty[(n0 + released) % kNB]);
+        pass_chunks(nchunks);
+        if (image) tr.mark(7);
       }
       if (!image) {
+        // ||r||^2: the warp that finishes its residual rows last adds the warps' partial sums in
+        // warp order (the sum does not depend on who finished first) and sends the CTA's share
+        // as one atomic; the next tick's exchange settles the gate
         sr = warp_sum(sr);
-        if (lane == 0) misc->sr[warp] = sr;
+        if (lane == 0) {
+          misc->sr[warp] = sr;
+          __threadfence_block();
+          if (atomicAdd(&misc->r2_cnt, 1) == kNW - 1) {
+            misc->r2_cnt = 0;
+    misc->stop[0] = misc->stop[1] = 0;
+            __threadfence_block();
+            if (pg > 0) {
+              float s = 0.f;
+#pragma unroll
+              for (int w = 0; w < kNW; ++w) s += reinterpret_cast<volatile float*>(misc->sr)[w];
+              // at most 2^45 per CTA, so the sum of all CTAs stays below 2^53; a partial that large
+              // (||r||^2 > 2 ||x||^2) fires for every sensible eps
+              double vd = (double)s * pow2d(44 - (x2_own > 0.0 ? exp_above(x2_own) : 0));
+              if (!(vd < 35184372088832.0)) vd = 35184372088832.0;
+              if (!(vd >= 0.0)) vd = 0.0;
+              red_add_u64(acc + k + 2, kOne + (unsigned long long)__double2ll_rn(vd));
+            }
+          }
+        }
       }
       tr.mark(image ? 8 : 5);
     }
-    if (!ok && !*abort) fail(p, misc, 8);
-    if (*abort) return;
-    if (xmax_next) xmax_collect(smem, t + 1, tag, p.spin_limit, p.status, xw[0], xw[1], xw[2], xw[3], xw[4]);
+    if (!ok && !*abort) fail(p, misc, 8);   // (the CTA leaves together, behind the next barrier)
+    if (xmax_next) xmax_collect(smem, t + 2, tag, p.spin_limit, p.status, xw[0], xw[1], xw[2], xw[3], xw[4]);
 
-    contrib_p = gsi && pg > 0;
-    if (gsi) {
-      e_p = x2_own > 0.0 ? exp_above(x2_own) : 0;
-      r2word_p = acc + k + 2;
-    }
     mask_pp = mask_p;
     }
 
@@ -1466,7 +1520,6 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
         tr.mark(9);
         n = w_stream(gw, src, gw->y + (size_t)p.token * gw->O, u == 2, smem, n, p.status, p.trace != nullptr);
         if (tr.acc) tr.t = clock64();
-        if (*abort) return;
         if (u == 2) {
           if (tid == 0) {
             red_relaxed_u32(gw->bar + parity, 1u);
@@ -1478,10 +1531,9 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
         }
       }
       tr.mark(6);
-      if (*abort) return;
     }
   }
-  if (lane == 0 || tid == kNC - 1) bulk_reduce_wait_read();
+  async_drain();
   tr.flush(p);
   // Every CTA read the counters at its start and has since taken part in the
   // last group's exchange, so they may advance now.
@@ -1503,6 +1555,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_decode_step(const __grid_const
       mbar_init(&empty[s], kNW);
     }
     misc->abort = 0;
+    misc->r2_cnt = 0;
     // shared memory keeps what the previous launch on this SM left: the producer must not
     // mistake an old decision for this launch's
     misc->fire[0] = misc->fire[1] = misc->fire[2] = misc->fire[3] = 0;

@@ -711,7 +711,7 @@ def test_persistent_trace_counters_do_not_change_results():
         assert torch.equal(a, b)
     assert np.array_equal(gate, stack.gate_log[:, 0, 0].cpu().numpy())
     T = tr.cpu().numpy()[:torch.cuda.get_device_properties(0).multi_processor_count]   # one row per CTA = per SM
-    assert T.shape[1] == 16 and (T[:, [0, 2, 3, 4, 5, 8]] > 0).all()   # barrier, pass 1, conversion, exchange, residual, image rows
+    assert T.shape[1] == 16 and (T[:, [0, 3, 4, 5, 8]] > 0).all()   # opening barrier, pass 1 of the next phase, exchange, residual, image rows
     assert (T[:, [10, 13]] > 0).all() and (T[0, 10:14] > 0).all()      # a group fired: input share, wait, arithmetic, sums (the last CTAs own no rows of W)
     stack.set_trace(False)
     before = tr.clone()
