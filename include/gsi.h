@@ -257,9 +257,10 @@ gsi_status_t gsi_destroy(gsi_handle_t h);
  * the given order and each group's own chain (projection, residual, gate,
  * image, gated residual) is Algorithm 1, but consecutive groups overlap: a
  * group's gate may be settled, and its W r added, while later groups already
- * project their inputs (the persistent kernel reads a group's x one phase
- * ahead and settles a gate one phase later; batched stacks run the gated
- * residual contraction of a group beside the kernels of the groups after it).
+ * project their inputs (the persistent kernel reads a group's x two phases
+ * ahead, projects it one phase ahead and settles a gate one phase later;
+ * batched stacks run the gated residual contraction of a group beside the
+ * kernels of the groups after it).
  * Every y, gate byte and rho of a step is final when the step's work has
  * completed in the order of `stream`, not earlier.
  * ------------------------------------------------------------------------ */
@@ -343,10 +344,13 @@ gsi_status_t gsi_stack_is_persistent(gsi_stack_t s, int* out);
  * counters (n_CTAs = SM count; NULL switches tracing off).  While set, thread 0
  * of every CTA of the persistent launch adds the SM cycles it spends in each
  * section of the per-phase pipeline:
- *   0 barrier that opens the tick        1 wait for basis slab     2 pass 1
- *   3 fixed-point conversion, reductions 4 wait for the sums, gate of the previous phase
- *   5 residual rows                      7 wait for image slab     8 image rows
- *   9 before a W stream (visibility of r) 10 the stream's share of its input into registers
+ *   0 barrier that opens the tick
+ *   3 (thread 0 belongs to the warps that wait for the sums; pass 1 and the send of the next
+ *     phase run on other warps meanwhile) the statistics hand-over of the phase after the next
+ *   4 wait for the sums of the tick's phase, gate of the previous phase, barrier
+ *   5 residual rows (with the wait for the basis slab's second copy)
+ *   7 image rows (with the waits for the chunks of the image slab)      8 end of the row passes
+ *   9 before a W stream                  10 the stream's share of its input into registers
  *  11 wait for W pieces   12 arithmetic on W pieces   13 partial sums into y
  *   6 after the streams of a tick (the grid barrier that follows a dense group)
  * The caller clears and reads the counters.  Applies from the next step.
