@@ -33,13 +33,13 @@ __global__ void k_pack_t16(const uint16_t* __restrict__ src, int rows, int k, ui
   const size_t n_words = (size_t)((rows + 15) / 16) * kt * 128;
   for (size_t wi = (size_t)blockIdx.x * blockDim.x + threadIdx.x; wi < n_words;
        wi += (size_t)gridDim.x * blockDim.x) {
-    const int reg = (int)(wi & 3), lane = (int)((wi >> 2) & 31);
+    // within a tile: four 8 x 8 blocks of 128 bytes, each row-major with 16-byte rows
+    const int blk = (int)((wi >> 5) & 3), g = (int)((wi >> 2) & 7), t = (int)(wi & 3);
     const size_t tile = wi >> 7;
     const int K = (int)(tile % kt);
     const size_t R = tile / kt;
-    const int g = lane >> 2, t = lane & 3;
-    const size_t row = R * 16 + g + (reg & 1) * 8;
-    const int col = K * 16 + 2 * t + (reg >> 1) * 8;
+    const size_t row = R * 16 + g + (blk & 1) * 8;
+    const int col = K * 16 + 2 * t + (blk >> 1) * 8;
     dst[wi] = row < (size_t)rows ? *reinterpret_cast<const uint32_t*>(src + row * k + col) : 0u;
   }
 }

@@ -497,11 +497,30 @@ __device__ __forceinline__ void mma_bf16(float (&d)[4], const uint4& a, uint32_t
       : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
       : "r"(a.x), "r"(a.y), "r"(a.z), "r"(a.w), "r"(b0), "r"(b1));
 }
-// Transposes an 8 x 8 block of 16-bit elements held one row pair per lane.
-__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a) {
-  uint32_t d;
-  asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
-  return d;
+// One 16 x 16 bf16 tile (512 bytes: its four 8 x 8 blocks one after the other, each row-major
+// with 16-byte rows; block order (rows 0-7, columns 0-7), (8-15, 0-7), (0-7, 8-15), (8-15, 8-15))
+// from shared memory; `lane_row` = the tile's base + 16 * lane.  Plain: the A operand of
+// mma.m16n8k16 over the tile.  Transposed: every block transposed, i.e. the tile as the B
+// operands of two instructions that contract over the tile's ROWS (x, y for columns 0-7;
+// z, w for columns 8-15).
+__device__ __forceinline__ uint4 ldsm_tile(const void* lane_row) {
+  uint4 r;
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "r"(smem_u32(lane_row)));
+  return r;
+}
+__device__ __forceinline__ uint4 ldsm_tile_trans(const void* lane_row) {
+  uint4 r;
+  asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+               : "=r"(r.x), "=r"(r.y), "=r"(r.z), "=r"(r.w)
+               : "r"(smem_u32(lane_row)));
+  return r;
+}
+// Arrivals that the unit `j` of `u` units sharing a chunk owes the chunk's "empty" barrier
+// (which expects kNW): the shares of a chunk's units add up to kNW.
+__device__ __forceinline__ uint32_t unit_share(int j, int u) {
+  return (uint32_t)(kNW / u + (j < kNW % u ? 1 : 0));
 }
 // v = hi + mid + lo, each a bf16 (round to nearest; the remainders are exact in fp32).
 __device__ __forceinline__ void split3(float v, unsigned short (&t)[3]) {
@@ -1111,7 +1130,10 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       constexpr int kTpwMax = kK ? (kK / 16 + kP1 - 1) / kP1 : 4;
       const int tpw = kK ? kTpwMax : (KTf + kP1 - 1) / kP1;
       float cacc[kTpwMax][2][4];
-      bool okf = chunks_landed(smem, n_pf, pf.pchunks, abort);
+      // the warps that own tile columns wait for the slab and, between them, give it back
+      const int nf = min(kP1, (KTf + tpw - 1) / tpw);
+      const bool p1_active = wp1 < nf && pf.pg > 0;
+      bool okf = !p1_active || chunks_landed(smem, n_pf, pf.pchunks, abort);
 #pragma unroll
       for (int s3 = 0; s3 < kTpwMax; ++s3)
 #pragma unroll
@@ -1130,12 +1152,17 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
           for (int s3 = 0; s3 < kTpwMax; ++s3) {
             const int kt = wp1 * tpw + s3;
             if (s3 < tpw && kt < KTf) {
-              const uint4 w = *reinterpret_cast<const uint4*>(trow + kt * 512);
-              mma_bf16(cacc[s3][0], a, movmatrix_trans(w.x), movmatrix_trans(w.y));
-              mma_bf16(cacc[s3][1], a, movmatrix_trans(w.z), movmatrix_trans(w.w));
+              const uint4 w = ldsm_tile_trans(trow + kt * 512);
+              mma_bf16(cacc[s3][0], a, w.x, w.y);
+              mma_bf16(cacc[s3][1], a, w.z, w.w);
             }
           }
         }
+      }
+      if (okf && p1_active && lane == 0) {   // (every tile of the slab is in registers: the last mma has issued)
+        const uint32_t share = unit_share(wp1, nf);
+#pragma unroll 1
+        for (int c = 0; c < pf.pchunks; ++c) mbar_arrive_n(&empty[(n_pf + c) % kNB], share);
       }
       // the three terms of x sit in rows 0..2 = lanes 0-3, 4-7, 8-11: fold them onto lanes 0-3
 #pragma unroll
@@ -1324,14 +1351,6 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
         }
       }
     }
-    if (gsi_f) {   // every warp gives the chunks of pass 1 back (they landed before pass 1 ran)
-#pragma unroll 1
-      for (int c = 0; c < pf.pchunks; ++c) {
-        const unsigned seq = n_pf + c;
-        if (!__all_sync(0xffffffffu, mbar_wait(&full_b[seq % kNB], (seq / kNB) & 1u, abort))) ok = false;
-        if (ok && lane == 0) mbar_arrive(&empty[seq % kNB]);
-      }
-    }
     desc_store(g_stage, n_stage, desc_word);
     if (tid == 0) misc->stop[1] = *abort;
     csync();
@@ -1372,7 +1391,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     for (int part = 0; part < 2; ++part) {
       if (!gsi) continue;
       const bool image = part == 1;
-      const int nchunks = image ? ochunks : pchunks, ngroups = image ? og : pg;
+      const int ngroups = image ? og : pg;
       const int id0 = image ? pg : 0;
       const unsigned n0 = image ? n : n_pr;
       const int row_base = image ? pl.o0 : pl.p0, row_end = image ? g.O : g.d;
@@ -1380,20 +1399,10 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
       const bool f8 = image && (g.flags & GSI_FLAG_FP8_IMAGE);
       if (image) n += ochunks;
       float sr = 0.f;
-      int released = 0;
-      // The chunks of a slab are taken in order: a warp waits for a chunk, runs its units that
-      // lie in it, and gives it back (every warp gives every chunk back once, also those it has
-      // no unit in).  The image slab need not be resident as a whole: its chunks stream through
-      // the space that the basis slab of the next phase leaves.
-      auto pass_chunks = [&](int upto) {   // chunks [released, upto): wait, give back
-#pragma unroll 1
-        for (; released < upto && ok; ++released) {
-          const unsigned seq = n0 + released;
-          // (the outcome is taken for the warp as a whole: lanes must not part ways here)
-          if (!__all_sync(0xffffffffu, mbar_wait(&full_b[seq % kNB], (seq / kNB) & 1u, abort))) ok = false;
-          if (ok && lane == 0) mbar_arrive(&empty[seq % kNB]);
-        }
-      };
+      // A warp touches only the chunks its units lie in: it waits for the chunk, runs the unit
+      // and hands in the unit's share of the chunk's arrivals (the chunk goes back to the
+      // producer when all its units are done).  The image slab need not be resident as a whole:
+      // its chunks stream through the space that the basis slab of the next phase leaves.
       if (ok) {
         int id = warp;
         if (id < id0) id += ((id0 - id + kNW - 1) / kNW) * kNW;
@@ -1401,11 +1410,9 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
         for (; id < id0 + ngroups && ok; id += kNW) {
           const int R = id - id0;
           const int ci = R >> gcl, rr = R - (ci << gcl);
-          pass_chunks(ci);
-          {
-            const unsigned seq = n0 + ci;
-            if (!__all_sync(0xffffffffu, mbar_wait(&full_b[seq % kNB], (seq / kNB) & 1u, abort))) ok = false;
-          }
+          const unsigned seq = n0 + ci;
+          // (the outcome is taken for the warp as a whole: lanes must not part ways here)
+          if (!__all_sync(0xffffffffu, mbar_wait(&full_b[seq % kNB], (seq / kNB) & 1u, abort))) ok = false;
           if (!ok) break;
           const unsigned char* cb = reinterpret_cast<const unsigned char*>(s_cb) + lane * 8;
           float d0[4] = {0.f, 0.f, 0.f, 0.f}, d1[4] = {0.f, 0.f, 0.f, 0.f};
@@ -1433,14 +1440,16 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
             const unsigned char* trow = ring + s_off[(n0 + ci) % kNB] + (size_t)rr * KT * 512 + lane * 16;
 #pragma unroll 2
             for (int K = 0; K < KT; K += 2) {   // two chains of dependent instructions
-              const uint4 a0 = *reinterpret_cast<const uint4*>(trow + K * 512);
+              const uint4 a0 = ldsm_tile(trow + K * 512);
               const uint2 b0 = *reinterpret_cast<const uint2*>(cb + K * 256);
-              const uint4 a1 = *reinterpret_cast<const uint4*>(trow + K * 512 + 512);
+              const uint4 a1 = ldsm_tile(trow + K * 512 + 512);
               const uint2 b1 = *reinterpret_cast<const uint2*>(cb + K * 256 + 256);
               mma_bf16(d0, a0, b0.x, b0.y);
               mma_bf16(d1, a1, b1.x, b1.y);
             }
           }
+          // the unit's tiles are in registers (the last mma has issued): its share of the chunk goes back
+          if (lane == 0) mbar_arrive_n(&empty[seq % kNB], unit_share(rr, min(1 << gcl, ngroups - (ci << gcl))));
           // columns 0, 1 (lane pair 0) and 2 (lane pair 1) of D are the three terms of c
           const float lo = d0[0] + d1[0], lo1 = d0[1] + d1[1], hi = d0[2] + d1[2], hi1 = d0[3] + d1[3];
           const float lo2 = __shfl_down_sync(0xffffffffu, lo, 1), hi2 = __shfl_down_sync(0xffffffffu, hi, 1);
@@ -1461,7 +1470,6 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
             }
           }
         }
-        pass_chunks(nchunks);
         if (image) tr.mark(7);
       }
       if (!image) {
