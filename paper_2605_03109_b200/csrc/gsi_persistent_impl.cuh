@@ -122,9 +122,8 @@ struct Misc {
   float x2_part[2];         // this CTA's sum of x^2 over its rows, by tick parity
   int fire[4];              // decisions on the previous phase's groups, by tick parity: 1 = stream W
   double x2;                // ||x||^2 of this phase's group
-  float sr[kNW];            // per-warp partial ||r||^2 of this phase
+  unsigned long long r2_acc;   // this CTA's ||r||^2 of the tick's phase in fixed point; the upper bits count the warps
   volatile unsigned decision[4];   // hand-off to the producer: (phase + 1) << 8 | fire mask
-  int r2_cnt;               // warps that have handed in their partial ||r||^2 of the tick's phase
   volatile int stop[2];     // the abort flag as thread 0 saw it before a barrier (one word per barrier of the tick, so that
                             // a warp still reading one cannot see the next write): every warp leaves at the same barrier
 };
@@ -1473,27 +1472,24 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
         if (image) tr.mark(7);
       }
       if (!image) {
-        // ||r||^2: the warp that finishes its residual rows last adds the warps' partial sums in
-        // warp order (the sum does not depend on who finished first) and sends the CTA's share
-        // as one atomic; the next tick's exchange settles the gate
+        // ||r||^2: every warp adds its rows' share, in the fixed-point units 2^(e - 44) of the
+        // exchange, to one word of shared memory whose upper bits count the warps (integers: the
+        // sum does not depend on who finished first; no fence: the one atomic carries value and
+        // count); the warp that arrives last sends the CTA's share as one atomic; the next
+        // tick's exchange settles the gate.  A share is at most 2^45, so the sum of all CTAs
+        // stays below 2^53; a partial that large (||r||^2 > 2 ||x||^2) fires for every sensible eps
         sr = warp_sum(sr);
         if (lane == 0) {
-          misc->sr[warp] = sr;
-          __threadfence_block();
-          if (atomicAdd(&misc->r2_cnt, 1) == kNW - 1) {
-            misc->r2_cnt = 0;
-    misc->stop[0] = misc->stop[1] = 0;
-            __threadfence_block();
+          double vd = (double)sr * pow2d(44 - (x2_own > 0.0 ? exp_above(x2_own) : 0));
+          if (!(vd < 35184372088832.0)) vd = 35184372088832.0;
+          if (!(vd >= 0.0)) vd = 0.0;
+          const unsigned long long mine = kOne + (unsigned long long)__double2ll_rn(vd);
+          const unsigned long long before = atomicAdd(&misc->r2_acc, mine);
+          if ((unsigned)((before + mine) >> kCountShift) == (unsigned)kNW) {
+            misc->r2_acc = 0ull;   // (next used behind two barriers)
             if (pg > 0) {
-              float s = 0.f;
-#pragma unroll
-              for (int w = 0; w < kNW; ++w) s += reinterpret_cast<volatile float*>(misc->sr)[w];
-              // at most 2^45 per CTA, so the sum of all CTAs stays below 2^53; a partial that large
-              // (||r||^2 > 2 ||x||^2) fires for every sensible eps
-              double vd = (double)s * pow2d(44 - (x2_own > 0.0 ? exp_above(x2_own) : 0));
-              if (!(vd < 35184372088832.0)) vd = 35184372088832.0;
-              if (!(vd >= 0.0)) vd = 0.0;
-              red_add_u64(acc + k + 2, kOne + (unsigned long long)__double2ll_rn(vd));
+              const unsigned long long sum = before + mine - ((unsigned long long)kNW << kCountShift);
+              red_add_u64(acc + k + 2, kOne + (sum < 35184372088832ull ? sum : 35184372088832ull));
             }
           }
         }
@@ -1563,7 +1559,7 @@ __global__ void __launch_bounds__(kThreadsP, 1) k_decode_step(const __grid_const
       mbar_init(&empty[s], kNW);
     }
     misc->abort = 0;
-    misc->r2_cnt = 0;
+    misc->r2_acc = 0ull;
     // shared memory keeps what the previous launch on this SM left: the producer must not
     // mistake an old decision for this launch's
     misc->fire[0] = misc->fire[1] = misc->fire[2] = misc->fire[3] = 0;
