@@ -19,10 +19,11 @@
 //               words during pass 1) and its partial ||x||^2 with ONE bulk reduction
 //               (cp.reduce.async.bulk), and its partial ||r||^2 of the PREVIOUS phase; one
 //               warp then polls the accumulators until all have arrived
-// Basis and images are stored as 16 x 16 tiles in the operand order of mma.m16n8k16, so both
-// passes and the image rows run on the tensor cores with one 16-byte shared-memory load per
-// tile and lane: x and c enter as three bf16 terms each (hi + mid + lo = the fp32 value), so
-// every product is exact and the sums are fp32.
+// Basis and images are stored as 16 x 16 tiles of four row-major 8 x 8 blocks, so both passes
+// and the image rows run on the tensor cores with one ldmatrix per tile (plain: the A operand
+// of the row passes; transposed: the B operands of pass 1, which contracts over the tile's
+// rows): x and c enter as three bf16 terms each (hi + mid + lo = the fp32 value), so every
+// product is exact and the sums are fp32.
 //   gate        of the previous phase, from the exact integer sums: the same decision on
 //               every CTA                                                (line 4, Eq. (3.3))
 //   pass 2      r_slab = x_slab - P_slab c, partial ||r||^2              (lines 2-3)
@@ -1110,11 +1111,11 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     // ---- B / D. (warps 5..13) pass 1 and the send of phase t + 1, beside the wait for the
     //      exchange of phase t.  Pass 1 on the tensor cores: D[term of x][column j] +=
     //      X[term][row i] P[i][j]; the rows of x are the A operand (three terms in rows 0..2), a
-    //      tile of P, each of its four 8 x 8 blocks transposed in registers, is the B operand of
+    //      tile of P, each of its four 8 x 8 blocks transposed by the load, is the B operand of
     //      two instructions.  Then every warp converts its own columns to fixed point and sends
     //      them off with a bulk reduction of its own into the group's accumulators.
     // chunk sequence of the tick: the basis slab of phase t + 1 for its pass 1 (given back
-    // before the barrier that ends the exchange), the basis slab of phase t once more for its
+    // by the pass-1 warps as soon as its tiles are in registers), the basis slab of phase t once more for its
     // residual rows (the second read comes from the L2: the ring is a FIFO, and a slab kept
     // across the tick boundary would pin everything placed after it), the image slab of phase t
     const unsigned n_pf = n;
@@ -1385,7 +1386,7 @@ __device__ void consumer(const PersistParams& p, unsigned char* smem, Misc* misc
     //      is a tile row (16 matrix rows): D[row][term of c] += T[row][column] C[column][term],
     //      the tiles as they lie in the ring are the A operand, c (three terms in columns
     //      0..2) the B operand.  Units are dealt round-robin over the joint numbering of both
-    //      parts, so the warps are loaded evenly.  Every warp gives every chunk back once.
+    //      parts, so the warps are loaded evenly.
 #pragma unroll 1
     for (int part = 0; part < 2; ++part) {
       if (!gsi) continue;
