@@ -549,6 +549,37 @@ def test_persistent_matches_generic_kernels_and_is_reproducible():
             assert (ys_a[i][s] - ref).abs().max() <= 1e-4 * ref.abs().max()
 
 
+def test_persistent_chunks_shared_by_many_units():
+    """Rank 64: a ring chunk holds up to eight 16-row units, each run by another warp, and the
+    chunk goes back to the producer when all of them have handed in their share of its arrivals.
+    Sizes chosen so that a CTA owns several units per slab (basis: 3-4 tile rows, image: 8-9), with
+    full and ragged chunks; the second group repeats the first, so every chunk's barrier pair is
+    used more than once."""
+    g = G()
+    k, d, d_out, n_steps = 64, 8192, (20480,), 6
+    q = S.gen_basis(d, k, 1700)
+    P = S.store_basis(q)
+    Ws = [S.gen_weight(o, d, 1710 + j) for j, o in enumerate(d_out)]
+    pt = S.gen_true_basis(q, k // 2, k // 2, 1720)
+    x, _ = S.gen_activations(pt, n_steps, 0.002, 0.0, dict(z=1730, noise=1731, outlier_mask=0, outlier_values=0))
+    x[::2] = torch.randn((len(range(0, n_steps, 2)), d), generator=torch.Generator().manual_seed(1732))
+    lays = [g.Layer([W.cuda() for W in Ws], P.cuda(), 0.05, max_tokens=1) for _ in range(3)]
+    stack = g.Stack(lays, mode=2)
+    stack.bind([x.cuda().contiguous() for _ in lays], n_steps=n_steps)
+    ys = [[] for _ in lays]
+    for s in range(n_steps):
+        stack.step()
+        torch.cuda.synchronize()
+        for i in range(len(lays)):
+            ys[i].append(stack.ys[i].cpu().clone())
+    assert stack.status() == 0 and stack.is_persistent()
+    for i in range(len(lays)):
+        gate = stack.gate_log[:, i, 0].cpu().numpy()
+        rho = stack.rho_log[:, i, 0].cpu().numpy()
+        compare_group(x, P, Ws, 0.05, torch.cat(ys[i]).numpy(), gate, rho)
+        assert 0 < gate.sum() < n_steps   # both paths occur
+
+
 @pytest.mark.parametrize("k", [64, 128, 512])
 def test_persistent_other_ranks_and_flags(k):
     g = G()
