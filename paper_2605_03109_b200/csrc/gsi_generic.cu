@@ -438,11 +438,13 @@ cudaError_t launch_gated_gemv(const GroupParams& g, const IoRef& io, cudaStream_
 }
 
 int generic_launch_count(const GroupParams& g, int n_tokens) {
+  // (a tensor-core contraction with one split over the depth writes y itself: no kernel that adds partial sums)
+  const int add = tc_splits(g.O, g.d) > 1 ? 1 : 0;
   if (g.flags & GSI_FLAG_DENSE)
-    return (g.front_min_tokens > 0 && n_tokens >= g.front_min_tokens) ? 3 : 1;
+    return (g.front_min_tokens > 0 && n_tokens >= g.front_min_tokens) ? 2 + add : 1;
   const bool stat = g.flags & GSI_FLAG_STATIC_PROJECTION;
-  if (g.front_min_tokens > 0 && n_tokens >= g.front_min_tokens) return stat ? 4 : 6;
-  return 4 + (stat ? 0 : 1 + (g.tc_min_fired > 0 ? 3 : 0));
+  if (g.front_min_tokens > 0 && n_tokens >= g.front_min_tokens) return stat ? 4 : 5 + add;
+  return 4 + (stat ? 0 : 1 + (g.tc_min_fired > 0 ? 2 + add : 0));
 }
 
 cudaError_t launch_advance_step(int* step, cudaStream_t st) {

@@ -49,7 +49,7 @@ __global__ void __launch_bounds__(256) k_pack_fired_bf16(GroupParams g, int min_
 // mapped == 1: B rows are all n_tokens tokens of the call (row = token); only the columns
 //              of fired tokens are written out.
 __global__ void __launch_bounds__(kThreadsTc, 2)
-k_residual_gemm_tc(GroupParams g, const __grid_constant__ TmaMaps tm, int min_fired, int splits,
+k_residual_gemm_tc(GroupParams g, const __grid_constant__ TmaMaps tm, IoRef io, int min_fired, int splits,
                    int mapped, int n_tokens) {
   pdl_launch_dependents();
   // With many tokens per call some token is gated nearly always: the W tiles are then
@@ -100,16 +100,32 @@ k_residual_gemm_tc(GroupParams g, const __grid_constant__ TmaMaps tm, int min_fi
     if (threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
   } else if (nloc > 0) {
     // warp w owns tensor-memory lanes 32w..32w+31 = rows row0+32w+lane; 16 columns per load
+    // One split: the tile's rows belong to this block alone, and y holds the image product of
+    // the kernels before: the sums are added to y here (no partial sums, no second kernel).
     const unsigned long long mask = s_mask;
-    float* yp = g.ypart + ((size_t)split * kMaxN) * g.O + row0 + warp * 32 + lane;
+    const int row = row0 + warp * 32 + lane;
+    float* yp = g.ypart + ((size_t)split * kMaxN) * g.O + row;
     for (int c0 = 0; c0 < N; c0 += 16) {
       if (((mask >> c0) & 0xFFFFull) == 0ull) continue;
       uint32_t v[16];
       tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + c0, v);
       tmem_ld_wait();
+      if (splits == 1) {
+        // (an addition at the L2 without a round trip; one writer per element, so the result
+        // does not depend on any order)
 #pragma unroll
-      for (int c = 0; c < 16; ++c)
-        if ((mask >> (c0 + c)) & 1ull) yp[(size_t)(c0 + c) * g.O] = __uint_as_float(v[c]);
+        for (int c = 0; c < 16; ++c)
+          if ((mask >> (c0 + c)) & 1ull) {
+            const int tok = mapped ? c0 + c : g.fired[c0 + c];
+            asm volatile("red.relaxed.gpu.global.add.f32 [%0], %1;" ::"l"(io.y + (size_t)tok * g.O + row),
+                         "f"(__uint_as_float(v[c]))
+                         : "memory");
+          }
+      } else {
+#pragma unroll
+        for (int c = 0; c < 16; ++c)
+          if ((mask >> (c0 + c)) & 1ull) yp[(size_t)(c0 + c) * g.O] = __uint_as_float(v[c]);
+      }
     }
   }
   tile_release<kTmemCols>(tmem);
@@ -153,7 +169,7 @@ __global__ void __launch_bounds__(256) k_pack_x_bf16(GroupParams g, IoRef io, in
 }
 
 __global__ void __launch_bounds__(kThreadsTc, 2)
-k_dense_gemm_tc(GroupParams g, const __grid_constant__ TmaMaps tm, int splits, int n_tokens) {
+k_dense_gemm_tc(GroupParams g, const __grid_constant__ TmaMaps tm, IoRef io, int splits, int n_tokens) {
   extern __shared__ unsigned char smem_raw[];
   pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -170,14 +186,23 @@ k_dense_gemm_tc(GroupParams g, const __grid_constant__ TmaMaps tm, int splits, i
   if (!ok) {
     if (threadIdx.x == 0) atomicExch(g.status, (int)GSI_ERR_TIMEOUT);
   } else {
-    float* yp = g.ypart + ((size_t)split * kMaxN) * g.O + row0 + warp * 32 + lane;
+    // (one split: straight to y, and this kernel reports every token as gated)
+    const int row = row0 + warp * 32 + lane;
+    float* yp = g.ypart + ((size_t)split * kMaxN) * g.O + row;
+    if (splits == 1 && blockIdx.x == 0 && threadIdx.x < n_tokens)
+      io.gate[(long long)io_slot(io) * io.log_step_stride + threadIdx.x] = 1;
     for (int c0 = 0; c0 < N; c0 += 16) {
       uint32_t v[16];
       tmem_ld16(tmem + ((uint32_t)(warp * 32) << 16) + c0, v);
       tmem_ld_wait();
 #pragma unroll
       for (int c = 0; c < 16; ++c)
-        if (c0 + c < n_tokens) yp[(size_t)(c0 + c) * g.O] = __uint_as_float(v[c]);
+        if (c0 + c < n_tokens) {
+          if (splits == 1)
+            io.y[(size_t)(c0 + c) * g.O + row] = __uint_as_float(v[c]);
+          else
+            yp[(size_t)(c0 + c) * g.O] = __uint_as_float(v[c]);
+        }
     }
   }
   tile_release<kTmemCols>(tmem);
@@ -207,12 +232,14 @@ cudaError_t launch_dense_gemm_tc(const GroupParams& g, const TmaMaps& tm, const 
   const int splits = tc_splits(g.O, g.d);
   const int rows = (n_tokens + 15) & ~15;
   k_pack_x_bf16<<<dim3((g.d + 2047) / 2048, rows), 256, 0, st>>>(g, io, n_tokens);
-  if ((e = launch_pdl(k_dense_gemm_tc, dim3((g.O / kTM) * splits), dim3(kThreadsTc), kTcSmem, st, g, tm,
-                      splits, n_tokens)) != cudaSuccess ||
+  if ((e = launch_pdl(k_dense_gemm_tc, dim3((g.O / kTM) * splits), dim3(kThreadsTc), kTcSmem, st, g, tm, io,
+                      splits, n_tokens)) != cudaSuccess)
+    return e;
+  if (splits > 1 &&
       (e = launch_pdl(k_sum_partials, dim3((g.O + 1023) / 1024, n_tokens), dim3(256), 0, st, g, io, splits,
                       n_tokens)) != cudaSuccess)
     return e;
-  if (n_launches) *n_launches += 3;
+  if (n_launches) *n_launches += splits > 1 ? 3 : 2;
   return cudaGetLastError();
 }
 
@@ -244,16 +271,18 @@ cudaError_t launch_residual_gemm_tc(const GroupParams& g, const TmaMaps& tm, con
   if (mapped) {
     // straight after the residual kernel: both may start while their predecessor drains
     if ((e = launch_pdl(k_residual_gemm_tc, dim3((g.O / kTM) * splits), dim3(kThreadsTc), kTcSmem, st, g,
-                        tm, min_fired, splits, 1, n_tokens)) != cudaSuccess ||
+                        tm, io, min_fired, splits, 1, n_tokens)) != cudaSuccess)
+      return e;
+    if (splits > 1 &&
         (e = launch_pdl(k_add_partials, dim3((g.O + 1023) / 1024, g.B), dim3(256), 0, st, g, io,
                         min_fired, splits, 1)) != cudaSuccess)
       return e;
   } else {
-    k_residual_gemm_tc<<<(g.O / kTM) * splits, kThreadsTc, kTcSmem, st>>>(g, tm, min_fired, splits, 0,
+    k_residual_gemm_tc<<<(g.O / kTM) * splits, kThreadsTc, kTcSmem, st>>>(g, tm, io, min_fired, splits, 0,
                                                                           n_tokens);
-    k_add_partials<<<dim3((g.O + 1023) / 1024, g.B), 256, 0, st>>>(g, io, min_fired, splits, 0);
+    if (splits > 1) k_add_partials<<<dim3((g.O + 1023) / 1024, g.B), 256, 0, st>>>(g, io, min_fired, splits, 0);
   }
-  if (n_launches) *n_launches += mapped ? 2 : 3;
+  if (n_launches) *n_launches += (mapped ? 1 : 2) + (splits > 1 ? 1 : 0);
   return cudaGetLastError();
 }
 
